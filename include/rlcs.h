@@ -1,0 +1,196 @@
+/*
+ * rlcs -- fused credit-assignment scans for reinforcement learning on NVIDIA B200 (sm_100a).
+ *
+ * Seven entry points, one fused kernel launch each.  Every call reads raw rollout tensors of
+ * shape [N, T] (N = num_envs rows, T = timesteps per row), builds the per-step affine
+ * coefficients (alpha_t, beta_t) of Table 1 on chip, and solves the first-order linear recurrence
+ * of Eq. 1,  A_t = alpha_t + beta_t * A_{t+1}  (or the forward mirror with A_{t-1}),  as a
+ * segmented associative scan under the combine operator of Eq. 2.  Episode boundaries reset the
+ * scan; bootstrap values enter at truncations and at the rollout-window edge (Section 3.2).
+ *
+ * CONVENTIONS COMMON TO ALL ENTRY POINTS
+ *
+ * Pointers.  Every pointer except `cuda_stream` is a DEVICE pointer.  The caller owns every
+ *   buffer, including `workspace`; the library allocates nothing and keeps no state between
+ *   calls.  Outputs must not overlap inputs or each other.
+ * Layout.  Every [N, T] tensor is contiguous row-major: element (n, t) at index n*T + t.
+ *   Floating-point tensors are fp32 (Section 4.4: the method is fp32-only).  Masks are uint8,
+ *   zero = false, any non-zero value = true.
+ * Flags.  For the five backward algorithms `dones` is the termination flag d^term and `truncs`
+ *   the truncation flag d^trunc; d_t = d^term_t OR d^trunc_t severs the recurrence (Table 1
+ *   caption).  `truncs` and `trunc_bootstrap` are both NULL (no per-step truncation handling,
+ *   the HAS_TRUNCATIONS=False case of Section 4.2) or both non-NULL.  The two forward scans take
+ *   ONE already-combined flag (term OR trunc) in `dones`.
+ * Successor value of step t (Section 3.2), written X_next(t) below, for X = values or expected_q:
+ *     0                       if dones[n,t]            (termination wins when both flags are set)
+ *     trunc_bootstrap[n,t]    else if truncs[n,t]      (supplied continuation value)
+ *     bootstrap[n]            else if t == T-1         (rollout-window edge; NULL pointer = 0,
+ *                                                       the HAS_BOOTSTRAP=False case)
+ *     X[n,t+1]                otherwise.
+ *   The recurrence continues from t into t+1 ("cont_t") only when no flag is set at t and
+ *   t < T-1.  trunc_bootstrap is read only where truncs is set and dones is not.
+ * Sizes.  N >= 0, 0 <= T < 2^31, N*T < 2^40.  N == 0 or T == 0 returns RLCS_OK without a launch.
+ * Parameters.  gamma and lambda must lie in [0, 1] (1 is valid); clip thresholds must be >= 0
+ *   (+inf = no clipping).  NaN is rejected.
+ * Alignment.  fp32 pointers must be 4-byte aligned.  When every fp32 pointer is 16-byte aligned
+ *   and every mask pointer 8-byte aligned the vectorised kernels run; otherwise a slower
+ *   element-wise variant of the same kernel is used (same results).
+ * Workspace.  Rows that straddle the kernels' tiles need a carry between thread blocks, passed
+ *   through `workspace`: at least rlcs_workspace_bytes(N, T) bytes, 16-byte aligned, initialised
+ *   once with rlcs_workspace_init and then reusable by any number of calls, of any of the entry
+ *   points, that are ordered on one stream.  Two calls that may run concurrently need two
+ *   workspaces.  When rlcs_workspace_bytes(N, T) is 0 the workspace may be NULL.
+ * Execution.  Work is enqueued on `cuda_stream` (a cudaStream_t passed as void*; NULL = the
+ *   default stream) and the call returns without synchronising.  Argument errors are returned
+ *   before anything is launched.  The only device-side wait is the bounded carry wait between
+ *   thread blocks; if it ever gives up, the kernel still terminates normally, the outputs of that
+ *   call are unspecified, and rlcs_last_device_status reports RLCS_ERR_TIMEOUT.
+ * Inputs are assumed finite.  Resets are applied by selection, not by multiplying with zero, so
+ *   a non-finite value inside one episode cannot leak into a neighbouring episode.
+ * Results are deterministic: the same inputs give bit-identical outputs on every call.
+ */
+#ifndef RLCS_H_
+#define RLCS_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    RLCS_OK = 0,
+    RLCS_ERR_NULL = 1,       /* a required pointer is NULL, or exactly one of truncs/trunc_bootstrap */
+    RLCS_ERR_SIZE = 2,       /* negative or too large N / T */
+    RLCS_ERR_ARG = 3,        /* gamma / lambda / clip out of range or NaN */
+    RLCS_ERR_ALIGN = 4,      /* fp32 pointer not 4-byte aligned, workspace not 16-byte aligned */
+    RLCS_ERR_WORKSPACE = 5,  /* workspace NULL or too small for this (N, T) */
+    RLCS_ERR_CUDA = 6,       /* the launch itself failed (cudaGetLastError) */
+    RLCS_ERR_TIMEOUT = 7     /* device status: a bounded carry wait gave up */
+} rlcs_status_t;
+
+/* Human-readable name of a status code (static storage, never NULL). */
+const char* rlcs_status_string(int status);
+
+/* Bytes of workspace sufficient for any entry point at this (N, T); 0 when no row can straddle a
+ * tile (then `workspace` may be NULL).  Returns 0 for invalid sizes as well. */
+size_t rlcs_workspace_bytes(int64_t N, int64_t T);
+
+/* Prepare a workspace (zero the tile records, set the call counter): enqueued on `cuda_stream`.
+ * Needed once per workspace buffer, not once per call. */
+int rlcs_workspace_init(void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* Synchronises `cuda_stream`, reads the workspace's device status word and clears it.  Returns
+ * RLCS_OK, RLCS_ERR_TIMEOUT, or RLCS_ERR_CUDA if the copy failed.  NULL workspace returns RLCS_OK. */
+int rlcs_last_device_status(void* workspace, void* cuda_stream);
+
+/*
+ * Generalized Advantage Estimation -- Section 3.3.1, Table 1 row "GAE", boundaries of Section 3.2.
+ *   delta_t = rewards_t + gamma * values_next(t) - values_t
+ *   A_t     = delta_t + (cont_t ? gamma*lambda * A_{t+1} : 0)           (boundary carry A_T = 0)
+ *   advantages[n,t] = A_t;   returns[n,t] = A_t + values_t   (returns may be NULL)
+ * rewards, values, dones: [N,T]; truncs, trunc_bootstrap: [N,T] or NULL; bootstrap: [N] or NULL.
+ */
+int rlcs_gae(const float* rewards, const float* values, const uint8_t* dones, const uint8_t* truncs,
+             const float* trunc_bootstrap, const float* bootstrap, float* advantages, float* returns,
+             int64_t N, int64_t T, float gamma, float lambda,
+             void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * V-Trace -- Section 3.3.2, Table 1 row "V-Trace".  log_rhos[n,t] = log pi(a_t|s_t) - log mu(a_t|s_t).
+ *   rho_t = min(rho_bar, exp(log_rhos_t));   c_t = min(c_bar, exp(log_rhos_t))
+ *   Delta_t = rho_t*(rewards_t + gamma*values_next(t) - values_t) + (cont_t ? gamma*c_t*Delta_{t+1} : 0)
+ *   vs[n,t] = values_t + Delta_t                                        (boundary carry Delta_T = 0)
+ *   pg_advantages[n,t] = rho_t*(rewards_t + gamma*v_next - values_t),  v_next = cont_t ? vs_{t+1}
+ *                        : values_next(t)                               (pg_advantages may be NULL)
+ */
+int rlcs_vtrace(const float* rewards, const float* values, const float* log_rhos, const uint8_t* dones,
+                const uint8_t* truncs, const float* trunc_bootstrap, const float* bootstrap,
+                float* vs, float* pg_advantages, int64_t N, int64_t T, float gamma, float rho_bar,
+                float c_bar, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Retrace(lambda) -- Section 3.3.3, Table 1 row "Retrace".  q_sa[n,t] = Q(s_t,a_t);
+ * expected_q[n,t] = E_pi Q(s_t,.) (column 0 is never read); bootstrap[n] = E_pi Q(s_T,.).
+ *   c_t = lambda * min(c_bar, exp(log_rhos_t))
+ *   Delta_t = rewards_t + gamma*expected_q_next(t) - q_sa_t + (cont_t ? gamma*c_{t+1}*Delta_{t+1} : 0)
+ *   q_targets[n,t] = q_sa_t + Delta_t          (index shift: the decay uses the NEXT step's c;
+ *                                               Delta_T = 0 and log_rhos[n,T] is never needed)
+ */
+int rlcs_retrace(const float* rewards, const float* q_sa, const float* expected_q, const float* log_rhos,
+                 const uint8_t* dones, const uint8_t* truncs, const float* trunc_bootstrap,
+                 const float* bootstrap, float* q_targets, int64_t N, int64_t T, float gamma,
+                 float lambda, float c_bar, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * TD(lambda) returns -- Section 3.3.4, Table 1 row "TD(lambda)".
+ *   G_t = rewards_t + gamma*[(1-lambda)*values_next(t) + lambda*G_{t+1}]     where cont_t,
+ *   G_t = rewards_t + gamma*values_next(t)                                    elsewhere
+ * (the window-edge bootstrap is priced once: gamma*(1-lambda) in alpha_{T-1} plus gamma*lambda
+ * through the carry G_T = bootstrap).
+ */
+int rlcs_td_lambda(const float* rewards, const float* values, const uint8_t* dones, const uint8_t* truncs,
+                   const float* trunc_bootstrap, const float* bootstrap, float* returns,
+                   int64_t N, int64_t T, float gamma, float lambda,
+                   void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Discounted returns -- Section 3.3.4 (lambda = 1, no value function), Table 1 row "Disc. Returns".
+ *   G_t = rewards_t + gamma * (cont_t ? G_{t+1} : 0 | trunc_bootstrap_t | bootstrap per Section 3.2)
+ */
+int rlcs_discounted_return(const float* rewards, const uint8_t* dones, const uint8_t* truncs,
+                           const float* trunc_bootstrap, const float* bootstrap, float* returns,
+                           int64_t N, int64_t T, float gamma,
+                           void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Eligibility trace, scalar per step, forward in time -- Section 3.3.5.
+ *   z_t = x_t + ((t > 0 and not dones_{t-1}) ? gamma*lambda * z_{t-1} : 0)
+ */
+int rlcs_elig_trace(const float* x, const uint8_t* dones, float* traces, int64_t N, int64_t T,
+                    float gamma, float lambda,
+                    void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Episodic prefix sum, forward in time -- Section 3.3.6.
+ *   starts_at == 0 ("ends_at", the flag closes a segment):  C_t = x_t + ((t>0 and not dones_{t-1}) ? C_{t-1} : 0)
+ *   starts_at != 0 (the flag opens a segment):              C_t = x_t + ((t>0 and not dones_t)     ? C_{t-1} : 0)
+ */
+int rlcs_episodic_prefix_sum(const float* x, const uint8_t* dones, float* sums, int64_t N, int64_t T,
+                             int starts_at, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Test hook: the bare scan of Eq. 1 / Eq. 2 on caller-supplied coefficients, every row with
+ * boundary carry 0 (the paper's generic kernel of Section 4.1).
+ *   forward == 0:  out_t = alpha_t + (t < T-1 ? beta_t * out_{t+1} : 0)
+ *   forward != 0:  out_t = alpha_t + (t > 0   ? beta_t * out_{t-1} : 0)
+ */
+int rlcs_affine_scan(const float* alpha, const float* beta, float* out, int64_t N, int64_t T, int forward,
+                     void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Test hook: choose the kernels' tile shape for subsequent calls in this process (not thread-safe).
+ * variant 0 = default.  Other variants change threads per block / steps per thread, hence where
+ * tiles and warps cut the rows; results must agree across variants to rounding and exactly at
+ * severed steps.  Returns RLCS_ERR_ARG for an unknown variant.  rlcs_workspace_bytes is an upper
+ * bound over all variants.
+ */
+int rlcs_debug_set_tile_variant(int variant);
+
+/* Elements per tile of a variant (0 for an unknown variant). */
+int rlcs_debug_tile_elems(int variant);
+
+/*
+ * Test hook for the bounded carry wait: for subsequent calls in this process, the thread block
+ * whose scan-order index is `mute_tile` does not publish its tile record (negative = publish
+ * normally), and the wait gives up after `spin_cap` polls (<= 0 = default).  A dependent block
+ * then runs out of polls within microseconds, records RLCS_ERR_TIMEOUT in the workspace status
+ * word and finishes normally -- nothing hangs or faults.
+ */
+int rlcs_debug_set_carry_fault(int64_t mute_tile, int64_t spin_cap);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RLCS_H_ */

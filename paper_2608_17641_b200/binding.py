@@ -1,0 +1,235 @@
+"""ctypes binding of ``librlcs.so``: same names as the C ABI, argument marshalling only.
+
+Every function takes CUDA ``torch.Tensor`` arguments (fp32 / uint8 / bool, contiguous), passes their
+device pointers and the current CUDA stream to the C entry point and returns the output tensors.
+Nothing is computed here; there is no CPU path.  A missing library raises at first use.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import threading
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "librlcs.so")
+
+RLCS_OK = 0
+RLCS_ERR_NULL, RLCS_ERR_SIZE, RLCS_ERR_ARG, RLCS_ERR_ALIGN = 1, 2, 3, 4
+RLCS_ERR_WORKSPACE, RLCS_ERR_CUDA, RLCS_ERR_TIMEOUT = 5, 6, 7
+
+_vp, _i64, _f, _sz, _int = ctypes.c_void_p, ctypes.c_int64, ctypes.c_float, ctypes.c_size_t, ctypes.c_int
+_TAIL = [_vp, _sz, _vp]          # workspace, workspace_bytes, cuda_stream
+
+# name -> argtypes, exactly the declarations of include/rlcs.h
+SIGNATURES = {
+    "rlcs_status_string": ([_int], ctypes.c_char_p),
+    "rlcs_workspace_bytes": ([_i64, _i64], _sz),
+    "rlcs_workspace_init": ([_vp, _sz, _vp], _int),
+    "rlcs_last_device_status": ([_vp, _vp], _int),
+    "rlcs_gae": ([_vp] * 8 + [_i64, _i64, _f, _f] + _TAIL, _int),
+    "rlcs_vtrace": ([_vp] * 9 + [_i64, _i64, _f, _f, _f] + _TAIL, _int),
+    "rlcs_retrace": ([_vp] * 9 + [_i64, _i64, _f, _f, _f] + _TAIL, _int),
+    "rlcs_td_lambda": ([_vp] * 7 + [_i64, _i64, _f, _f] + _TAIL, _int),
+    "rlcs_discounted_return": ([_vp] * 6 + [_i64, _i64, _f] + _TAIL, _int),
+    "rlcs_elig_trace": ([_vp] * 3 + [_i64, _i64, _f, _f] + _TAIL, _int),
+    "rlcs_episodic_prefix_sum": ([_vp] * 3 + [_i64, _i64, _int] + _TAIL, _int),
+    "rlcs_affine_scan": ([_vp] * 3 + [_i64, _i64, _int] + _TAIL, _int),
+    "rlcs_debug_set_tile_variant": ([_int], _int),
+    "rlcs_debug_tile_elems": ([_int], _int),
+    "rlcs_debug_set_carry_fault": ([_i64, _i64], _int),
+}
+
+_lib = None
+_lock = threading.Lock()
+
+
+class RlcsError(RuntimeError):
+    def __init__(self, status: int):
+        self.status = status
+        super().__init__(lib().rlcs_status_string(status).decode())
+
+
+def lib() -> ctypes.CDLL:
+    """The loaded C library (loaded once).  Raises if it has not been built."""
+    global _lib
+    with _lock:
+        if _lib is None:
+            if not os.path.exists(LIB_PATH):
+                raise RuntimeError(
+                    f"{LIB_PATH} is missing: build it with `python -m paper_2608_17641_b200.build` "
+                    "(there is no fallback path)")
+            L = ctypes.CDLL(LIB_PATH)
+            for name, (argtypes, restype) in SIGNATURES.items():
+                fn = getattr(L, name)
+                fn.argtypes = argtypes
+                fn.restype = restype
+            _lib = L
+    return _lib
+
+
+def _check(status: int):
+    if status != RLCS_OK:
+        raise RlcsError(status)
+
+
+def _torch():
+    import torch
+    return torch
+
+
+def _ptr(t, dtype_kind: str, shape=None):
+    """Device pointer of a tensor (None -> NULL) after dtype / device / layout checks."""
+    if t is None:
+        return None
+    torch = _torch()
+    if not t.is_cuda:
+        raise TypeError("rlcs takes CUDA tensors (device pointers); there is no CPU path")
+    if dtype_kind == "f32":
+        if t.dtype != torch.float32:
+            raise TypeError(f"expected float32, got {t.dtype}")     # the method is fp32-only
+    elif t.dtype not in (torch.uint8, torch.bool):
+        raise TypeError(f"expected a uint8/bool mask, got {t.dtype}")
+    if not t.is_contiguous():
+        raise ValueError("rlcs takes contiguous row-major tensors")
+    if shape is not None and tuple(t.shape) != tuple(shape):
+        raise ValueError(f"expected shape {tuple(shape)}, got {tuple(t.shape)}")
+    return t.data_ptr()
+
+
+def _stream(stream=None):
+    torch = _torch()
+    s = torch.cuda.current_stream() if stream is None else stream
+    return s.cuda_stream
+
+
+class Workspace:
+    """Caller-owned carry workspace (device memory held by a torch tensor), initialised once."""
+
+    def __init__(self, N: int, T: int, device="cuda", stream=None, nbytes: int | None = None):
+        torch = _torch()
+        self.nbytes = int(lib().rlcs_workspace_bytes(N, T)) if nbytes is None else int(nbytes)
+        self.buf = torch.empty(max(self.nbytes, 16), dtype=torch.uint8, device=device) if self.nbytes else None
+        if self.buf is not None:
+            _check(lib().rlcs_workspace_init(self.buf.data_ptr(), self.nbytes, _stream(stream)))
+
+    @property
+    def ptr(self):
+        return None if self.buf is None else self.buf.data_ptr()
+
+    def device_status(self, stream=None) -> int:
+        return lib().rlcs_last_device_status(self.ptr, _stream(stream))
+
+
+def workspace_bytes(N: int, T: int) -> int:
+    return int(lib().rlcs_workspace_bytes(N, T))
+
+
+def _ws(ws: Workspace | None):
+    return (None, 0) if ws is None else (ws.ptr, ws.nbytes)
+
+
+def _out(like, out):
+    torch = _torch()
+    return torch.empty_like(like, dtype=torch.float32) if out is None else out
+
+
+def rlcs_gae(rewards, values, dones, truncs=None, trunc_bootstrap=None, bootstrap=None, *, gamma, lam,
+             advantages=None, returns=None, want_returns=True, workspace=None, stream=None):
+    N, T = rewards.shape
+    adv = _out(rewards, advantages)
+    ret = (_out(rewards, returns) if want_returns else None)
+    wp, wb = _ws(workspace)
+    _check(lib().rlcs_gae(_ptr(rewards, "f32"), _ptr(values, "f32", (N, T)), _ptr(dones, "u8", (N, T)),
+                          _ptr(truncs, "u8", (N, T)), _ptr(trunc_bootstrap, "f32", (N, T)),
+                          _ptr(bootstrap, "f32", (N,)), _ptr(adv, "f32", (N, T)), _ptr(ret, "f32", (N, T)),
+                          N, T, gamma, lam, wp, wb, _stream(stream)))
+    return (adv, ret) if want_returns else adv
+
+
+def rlcs_vtrace(rewards, values, log_rhos, dones, truncs=None, trunc_bootstrap=None, bootstrap=None, *,
+                gamma, rho_bar=1.0, c_bar=1.0, vs=None, pg_advantages=None, want_advantages=True,
+                workspace=None, stream=None):
+    N, T = rewards.shape
+    vs = _out(rewards, vs)
+    adv = (_out(rewards, pg_advantages) if want_advantages else None)
+    wp, wb = _ws(workspace)
+    _check(lib().rlcs_vtrace(_ptr(rewards, "f32"), _ptr(values, "f32", (N, T)), _ptr(log_rhos, "f32", (N, T)),
+                             _ptr(dones, "u8", (N, T)), _ptr(truncs, "u8", (N, T)),
+                             _ptr(trunc_bootstrap, "f32", (N, T)), _ptr(bootstrap, "f32", (N,)),
+                             _ptr(vs, "f32", (N, T)), _ptr(adv, "f32", (N, T)), N, T, gamma, rho_bar, c_bar,
+                             wp, wb, _stream(stream)))
+    return (vs, adv) if want_advantages else vs
+
+
+def rlcs_retrace(rewards, q_sa, expected_q, log_rhos, dones, truncs=None, trunc_bootstrap=None,
+                 bootstrap=None, *, gamma, lam, c_bar=1.0, q_targets=None, workspace=None, stream=None):
+    N, T = rewards.shape
+    out = _out(rewards, q_targets)
+    wp, wb = _ws(workspace)
+    _check(lib().rlcs_retrace(_ptr(rewards, "f32"), _ptr(q_sa, "f32", (N, T)), _ptr(expected_q, "f32", (N, T)),
+                              _ptr(log_rhos, "f32", (N, T)), _ptr(dones, "u8", (N, T)), _ptr(truncs, "u8", (N, T)),
+                              _ptr(trunc_bootstrap, "f32", (N, T)), _ptr(bootstrap, "f32", (N,)),
+                              _ptr(out, "f32", (N, T)), N, T, gamma, lam, c_bar, wp, wb, _stream(stream)))
+    return out
+
+
+def rlcs_td_lambda(rewards, values, dones, truncs=None, trunc_bootstrap=None, bootstrap=None, *, gamma, lam,
+                   returns=None, workspace=None, stream=None):
+    N, T = rewards.shape
+    out = _out(rewards, returns)
+    wp, wb = _ws(workspace)
+    _check(lib().rlcs_td_lambda(_ptr(rewards, "f32"), _ptr(values, "f32", (N, T)), _ptr(dones, "u8", (N, T)),
+                                _ptr(truncs, "u8", (N, T)), _ptr(trunc_bootstrap, "f32", (N, T)),
+                                _ptr(bootstrap, "f32", (N,)), _ptr(out, "f32", (N, T)), N, T, gamma, lam,
+                                wp, wb, _stream(stream)))
+    return out
+
+
+def rlcs_discounted_return(rewards, dones, truncs=None, trunc_bootstrap=None, bootstrap=None, *, gamma,
+                           returns=None, workspace=None, stream=None):
+    N, T = rewards.shape
+    out = _out(rewards, returns)
+    wp, wb = _ws(workspace)
+    _check(lib().rlcs_discounted_return(_ptr(rewards, "f32"), _ptr(dones, "u8", (N, T)), _ptr(truncs, "u8", (N, T)),
+                                        _ptr(trunc_bootstrap, "f32", (N, T)), _ptr(bootstrap, "f32", (N,)),
+                                        _ptr(out, "f32", (N, T)), N, T, gamma, wp, wb, _stream(stream)))
+    return out
+
+
+def rlcs_elig_trace(x, dones, *, gamma, lam, traces=None, workspace=None, stream=None):
+    N, T = x.shape
+    out = _out(x, traces)
+    wp, wb = _ws(workspace)
+    _check(lib().rlcs_elig_trace(_ptr(x, "f32"), _ptr(dones, "u8", (N, T)), _ptr(out, "f32", (N, T)), N, T,
+                                 gamma, lam, wp, wb, _stream(stream)))
+    return out
+
+
+def rlcs_episodic_prefix_sum(x, dones, *, starts_at=False, sums=None, workspace=None, stream=None):
+    N, T = x.shape
+    out = _out(x, sums)
+    wp, wb = _ws(workspace)
+    _check(lib().rlcs_episodic_prefix_sum(_ptr(x, "f32"), _ptr(dones, "u8", (N, T)), _ptr(out, "f32", (N, T)),
+                                          N, T, int(bool(starts_at)), wp, wb, _stream(stream)))
+    return out
+
+
+def rlcs_affine_scan(alpha, beta, *, forward=False, out=None, workspace=None, stream=None):
+    N, T = alpha.shape
+    out = _out(alpha, out)
+    wp, wb = _ws(workspace)
+    _check(lib().rlcs_affine_scan(_ptr(alpha, "f32"), _ptr(beta, "f32", (N, T)), _ptr(out, "f32", (N, T)), N, T,
+                                  int(bool(forward)), wp, wb, _stream(stream)))
+    return out
+
+
+def rlcs_debug_set_tile_variant(variant: int):
+    _check(lib().rlcs_debug_set_tile_variant(variant))
+
+
+def rlcs_debug_tile_elems(variant: int) -> int:
+    return int(lib().rlcs_debug_tile_elems(variant))
+
+
+def rlcs_debug_set_carry_fault(mute_tile: int = -1, spin_cap: int = 0):
+    _check(lib().rlcs_debug_set_carry_fault(mute_tile, spin_cap))

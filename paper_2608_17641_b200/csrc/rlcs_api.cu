@@ -1,0 +1,316 @@
+// C ABI of the library: argument validation, kernel selection, launch.  No allocation, no state
+// between calls apart from the two test hooks at the bottom.
+#include <cmath>
+#include <cstdint>
+
+#include "../../include/rlcs.h"
+#include "rlcs_launch.cuh"
+
+namespace {
+
+using rlcs::ScanParams;
+
+int g_variant = 0;               // test hook: tile variant
+long long g_mute_tile = -1;      // test hook: tile that does not publish
+long long g_spin_cap = 0;        // test hook: poll limit (0 = default)
+constexpr unsigned kDefaultSpinCap = 1u << 21;
+
+constexpr int64_t kMaxT = (int64_t(1) << 31) - 1;
+constexpr int64_t kMaxTotal = int64_t(1) << 40;
+
+inline bool aligned(const void* p, uintptr_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+inline bool unit_interval(float v) { return v >= 0.f && v <= 1.f; }   // false for NaN
+inline bool clip_ok(float v) { return v >= 0.f; }                       // false for NaN; +inf allowed
+
+int tile_elems(int variant) { return rlcs::kVariants[variant].threads * rlcs::kVariants[variant].items; }
+
+// size check common to every entry point; returns RLCS_OK with *total = 0 for empty problems
+int check_sizes(int64_t N, int64_t T, int64_t* total) {
+    *total = 0;
+    if (N < 0 || T < 0 || T > kMaxT) return RLCS_ERR_SIZE;
+    if (N == 0 || T == 0) return RLCS_OK;
+    if (N > kMaxTotal / T) return RLCS_ERR_SIZE;
+    *total = N * T;
+    return RLCS_OK;
+}
+
+struct Ptrs {
+    const void* f32[8];
+    int nf32 = 0;
+    const void* u8[2];
+    int nu8 = 0;
+    void add_f32(const void* p) { if (p) f32[nf32++] = p; }
+    void add_u8(const void* p) { if (p) u8[nu8++] = p; }
+};
+
+// RLCS_ERR_ALIGN if an fp32 pointer is not 4-byte aligned; *vec = all pointers allow vector access
+int check_alignment(const Ptrs& ps, bool* vec) {
+    *vec = true;
+    for (int i = 0; i < ps.nf32; ++i) {
+        if (!aligned(ps.f32[i], 4)) return RLCS_ERR_ALIGN;
+        if (!aligned(ps.f32[i], 16)) *vec = false;
+    }
+    for (int i = 0; i < ps.nu8; ++i)
+        if (!aligned(ps.u8[i], 16)) *vec = false;
+    return RLCS_OK;
+}
+
+// Fill the size / tiling / carry fields and validate the workspace for this call.
+int finish_params(ScanParams& p, int64_t total, int64_t T, void* workspace, size_t workspace_bytes) {
+    const int tile = tile_elems(g_variant);
+    p.total = total;
+    p.T = (unsigned)T;
+    p.num_tiles = (total + tile - 1) / tile;
+    p.idx32 = (total + tile) <= 0xffffffffLL;
+    p.carry_mode = (tile % T) != 0;          // T does not divide the tile: rows straddle tiles
+    p.header = nullptr;
+    p.records = nullptr;
+    p.mute_tile = g_mute_tile;
+    p.spin_cap = g_spin_cap > 0 ? (unsigned)g_spin_cap : kDefaultSpinCap;
+    if (p.carry_mode) {
+        const size_t need = sizeof(unsigned) * rlcs::kHeaderWords + sizeof(uint4) * (size_t)p.num_tiles;
+        if (workspace == nullptr || workspace_bytes < need) return RLCS_ERR_WORKSPACE;
+        if (!aligned(workspace, 16)) return RLCS_ERR_ALIGN;
+        p.header = static_cast<unsigned*>(workspace);
+        p.records = reinterpret_cast<uint4*>(p.header + rlcs::kHeaderWords);
+    }
+    return RLCS_OK;
+}
+
+typedef cudaError_t (*Launcher)(const ScanParams&, int, bool, bool, cudaStream_t);
+
+int run(Launcher fn, const ScanParams& p, bool trunc, bool vec, void* stream) {
+    return fn(p, g_variant, trunc, vec, static_cast<cudaStream_t>(stream)) == cudaSuccess ? RLCS_OK : RLCS_ERR_CUDA;
+}
+
+// shared front half of the five backward entry points
+int backward_common(ScanParams& p, Ptrs& ps, const uint8_t* dones, const uint8_t* truncs,
+                    const float* trunc_bootstrap, const float* bootstrap, int64_t N, int64_t T,
+                    int64_t* total, bool* vec) {
+    int st = check_sizes(N, T, total);
+    if (st != RLCS_OK || *total == 0) return st;
+    if (dones == nullptr || (truncs == nullptr) != (trunc_bootstrap == nullptr)) return RLCS_ERR_NULL;
+    ps.add_u8(dones);
+    ps.add_u8(truncs);
+    ps.add_f32(trunc_bootstrap);
+    ps.add_f32(bootstrap);
+    st = check_alignment(ps, vec);
+    if (st != RLCS_OK) return st;
+    p.dones = dones;
+    p.truncs = truncs;
+    p.trunc_boot = trunc_bootstrap;
+    p.boot = bootstrap;
+    return RLCS_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* rlcs_status_string(int status) {
+    switch (status) {
+        case RLCS_OK: return "RLCS_OK";
+        case RLCS_ERR_NULL: return "RLCS_ERR_NULL: required pointer is NULL (or only one of truncs/trunc_bootstrap given)";
+        case RLCS_ERR_SIZE: return "RLCS_ERR_SIZE: N or T negative or too large";
+        case RLCS_ERR_ARG: return "RLCS_ERR_ARG: gamma/lambda/clip out of range";
+        case RLCS_ERR_ALIGN: return "RLCS_ERR_ALIGN: misaligned pointer";
+        case RLCS_ERR_WORKSPACE: return "RLCS_ERR_WORKSPACE: workspace missing or too small";
+        case RLCS_ERR_CUDA: return "RLCS_ERR_CUDA: CUDA call failed";
+        case RLCS_ERR_TIMEOUT: return "RLCS_ERR_TIMEOUT: bounded carry wait gave up";
+        default: return "RLCS: unknown status";
+    }
+}
+
+size_t rlcs_workspace_bytes(int64_t N, int64_t T) {
+    int64_t total = 0;
+    if (check_sizes(N, T, &total) != RLCS_OK || total == 0) return 0;
+    if (rlcs::kMinTileElems % T == 0) return 0;     // T divides every tile size: no row straddles a tile
+    const int64_t tiles = (total + rlcs::kMinTileElems - 1) / rlcs::kMinTileElems;
+    return sizeof(unsigned) * rlcs::kHeaderWords + sizeof(uint4) * (size_t)tiles;
+}
+
+int rlcs_workspace_init(void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    if (workspace == nullptr) return workspace_bytes == 0 ? RLCS_OK : RLCS_ERR_NULL;
+    if (!aligned(workspace, 16)) return RLCS_ERR_ALIGN;
+    if (workspace_bytes < sizeof(unsigned) * rlcs::kHeaderWords) return RLCS_ERR_WORKSPACE;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    if (cudaMemsetAsync(workspace, 0, workspace_bytes, s) != cudaSuccess) return RLCS_ERR_CUDA;
+    // epoch starts at 1 so that zeroed records are never valid (byte pattern 0x01 0x00 0x00 0x00)
+    if (cudaMemsetAsync(workspace, 1, 1, s) != cudaSuccess) return RLCS_ERR_CUDA;
+    return RLCS_OK;
+}
+
+int rlcs_last_device_status(void* workspace, void* cuda_stream) {
+    if (workspace == nullptr) return RLCS_OK;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    unsigned status = 0;
+    unsigned* word = static_cast<unsigned*>(workspace) + 2;
+    if (cudaMemcpyAsync(&status, word, sizeof(status), cudaMemcpyDeviceToHost, s) != cudaSuccess) return RLCS_ERR_CUDA;
+    if (cudaMemsetAsync(word, 0, sizeof(status), s) != cudaSuccess) return RLCS_ERR_CUDA;
+    if (cudaStreamSynchronize(s) != cudaSuccess) return RLCS_ERR_CUDA;
+    return status == 0 ? RLCS_OK : (int)status;
+}
+
+int rlcs_gae(const float* rewards, const float* values, const uint8_t* dones, const uint8_t* truncs,
+             const float* trunc_bootstrap, const float* bootstrap, float* advantages, float* returns,
+             int64_t N, int64_t T, float gamma, float lambda, void* workspace, size_t workspace_bytes,
+             void* cuda_stream) {
+    ScanParams p = {};
+    Ptrs ps;
+    int64_t total;
+    bool vec;
+    if (!unit_interval(gamma) || !unit_interval(lambda)) return RLCS_ERR_ARG;
+    ps.add_f32(rewards); ps.add_f32(values); ps.add_f32(advantages); ps.add_f32(returns);
+    int st = backward_common(p, ps, dones, truncs, trunc_bootstrap, bootstrap, N, T, &total, &vec);
+    if (st != RLCS_OK || total == 0) return st;
+    if (!rewards || !values || !advantages) return RLCS_ERR_NULL;
+    p.f0 = rewards; p.f1 = values; p.out0 = advantages; p.out1 = returns;
+    p.gamma = gamma; p.decay = gamma * lambda;
+    st = finish_params(p, total, T, workspace, workspace_bytes);
+    if (st != RLCS_OK) return st;
+    return run(rlcs::launch_gae, p, truncs != nullptr, vec, cuda_stream);
+}
+
+int rlcs_vtrace(const float* rewards, const float* values, const float* log_rhos, const uint8_t* dones,
+                const uint8_t* truncs, const float* trunc_bootstrap, const float* bootstrap, float* vs,
+                float* pg_advantages, int64_t N, int64_t T, float gamma, float rho_bar, float c_bar,
+                void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    ScanParams p = {};
+    Ptrs ps;
+    int64_t total;
+    bool vec;
+    if (!unit_interval(gamma) || !clip_ok(rho_bar) || !clip_ok(c_bar)) return RLCS_ERR_ARG;
+    ps.add_f32(rewards); ps.add_f32(values); ps.add_f32(log_rhos); ps.add_f32(vs); ps.add_f32(pg_advantages);
+    int st = backward_common(p, ps, dones, truncs, trunc_bootstrap, bootstrap, N, T, &total, &vec);
+    if (st != RLCS_OK || total == 0) return st;
+    if (!rewards || !values || !log_rhos || !vs) return RLCS_ERR_NULL;
+    p.f0 = rewards; p.f1 = values; p.f3 = log_rhos; p.out0 = vs; p.out1 = pg_advantages;
+    p.gamma = gamma; p.rho_bar = rho_bar; p.c_bar = c_bar;
+    st = finish_params(p, total, T, workspace, workspace_bytes);
+    if (st != RLCS_OK) return st;
+    return run(rlcs::launch_vtrace, p, truncs != nullptr, vec, cuda_stream);
+}
+
+int rlcs_retrace(const float* rewards, const float* q_sa, const float* expected_q, const float* log_rhos,
+                 const uint8_t* dones, const uint8_t* truncs, const float* trunc_bootstrap,
+                 const float* bootstrap, float* q_targets, int64_t N, int64_t T, float gamma, float lambda,
+                 float c_bar, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    ScanParams p = {};
+    Ptrs ps;
+    int64_t total;
+    bool vec;
+    if (!unit_interval(gamma) || !unit_interval(lambda) || !clip_ok(c_bar)) return RLCS_ERR_ARG;
+    ps.add_f32(rewards); ps.add_f32(q_sa); ps.add_f32(expected_q); ps.add_f32(log_rhos); ps.add_f32(q_targets);
+    int st = backward_common(p, ps, dones, truncs, trunc_bootstrap, bootstrap, N, T, &total, &vec);
+    if (st != RLCS_OK || total == 0) return st;
+    if (!rewards || !q_sa || !expected_q || !log_rhos || !q_targets) return RLCS_ERR_NULL;
+    p.f0 = rewards; p.f1 = q_sa; p.f2 = expected_q; p.f3 = log_rhos; p.out0 = q_targets;
+    p.gamma = gamma; p.aux = lambda; p.c_bar = c_bar;
+    st = finish_params(p, total, T, workspace, workspace_bytes);
+    if (st != RLCS_OK) return st;
+    return run(rlcs::launch_retrace, p, truncs != nullptr, vec, cuda_stream);
+}
+
+int rlcs_td_lambda(const float* rewards, const float* values, const uint8_t* dones, const uint8_t* truncs,
+                   const float* trunc_bootstrap, const float* bootstrap, float* returns, int64_t N, int64_t T,
+                   float gamma, float lambda, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    ScanParams p = {};
+    Ptrs ps;
+    int64_t total;
+    bool vec;
+    if (!unit_interval(gamma) || !unit_interval(lambda)) return RLCS_ERR_ARG;
+    ps.add_f32(rewards); ps.add_f32(values); ps.add_f32(returns);
+    int st = backward_common(p, ps, dones, truncs, trunc_bootstrap, bootstrap, N, T, &total, &vec);
+    if (st != RLCS_OK || total == 0) return st;
+    if (!rewards || !values || !returns) return RLCS_ERR_NULL;
+    p.f0 = rewards; p.f1 = values; p.out0 = returns;
+    p.gamma = gamma; p.decay = gamma * lambda; p.aux = gamma * (1.f - lambda);
+    st = finish_params(p, total, T, workspace, workspace_bytes);
+    if (st != RLCS_OK) return st;
+    return run(rlcs::launch_td_lambda, p, truncs != nullptr, vec, cuda_stream);
+}
+
+int rlcs_discounted_return(const float* rewards, const uint8_t* dones, const uint8_t* truncs,
+                           const float* trunc_bootstrap, const float* bootstrap, float* returns, int64_t N,
+                           int64_t T, float gamma, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    ScanParams p = {};
+    Ptrs ps;
+    int64_t total;
+    bool vec;
+    if (!unit_interval(gamma)) return RLCS_ERR_ARG;
+    ps.add_f32(rewards); ps.add_f32(returns);
+    int st = backward_common(p, ps, dones, truncs, trunc_bootstrap, bootstrap, N, T, &total, &vec);
+    if (st != RLCS_OK || total == 0) return st;
+    if (!rewards || !returns) return RLCS_ERR_NULL;
+    p.f0 = rewards; p.out0 = returns;
+    p.gamma = gamma; p.decay = gamma;
+    st = finish_params(p, total, T, workspace, workspace_bytes);
+    if (st != RLCS_OK) return st;
+    return run(rlcs::launch_disc, p, truncs != nullptr, vec, cuda_stream);
+}
+
+static int forward_scan(rlcs::Algo algo, const float* x, const uint8_t* dones, float* out, int64_t N, int64_t T,
+                        float decay, int starts_at, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    ScanParams p = {};
+    Ptrs ps;
+    int64_t total;
+    bool vec;
+    int st = check_sizes(N, T, &total);
+    if (st != RLCS_OK || total == 0) return st;
+    if (!x || !dones || !out) return RLCS_ERR_NULL;
+    ps.add_f32(x); ps.add_f32(out); ps.add_u8(dones);
+    st = check_alignment(ps, &vec);
+    if (st != RLCS_OK) return st;
+    p.f0 = x; p.dones = dones; p.out0 = out; p.decay = decay; p.starts_at = starts_at != 0;
+    st = finish_params(p, total, T, workspace, workspace_bytes);
+    if (st != RLCS_OK) return st;
+    return run(algo == rlcs::kElig ? rlcs::launch_elig : rlcs::launch_prefix, p, false, vec, cuda_stream);
+}
+
+int rlcs_elig_trace(const float* x, const uint8_t* dones, float* traces, int64_t N, int64_t T, float gamma,
+                    float lambda, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    if (!unit_interval(gamma) || !unit_interval(lambda)) return RLCS_ERR_ARG;
+    return forward_scan(rlcs::kElig, x, dones, traces, N, T, gamma * lambda, 0, workspace, workspace_bytes, cuda_stream);
+}
+
+int rlcs_episodic_prefix_sum(const float* x, const uint8_t* dones, float* sums, int64_t N, int64_t T,
+                             int starts_at, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    return forward_scan(rlcs::kPrefix, x, dones, sums, N, T, 1.f, starts_at, workspace, workspace_bytes, cuda_stream);
+}
+
+int rlcs_affine_scan(const float* alpha, const float* beta, float* out, int64_t N, int64_t T, int forward,
+                     void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    ScanParams p = {};
+    Ptrs ps;
+    int64_t total;
+    bool vec;
+    int st = check_sizes(N, T, &total);
+    if (st != RLCS_OK || total == 0) return st;
+    if (!alpha || !beta || !out) return RLCS_ERR_NULL;
+    ps.add_f32(alpha); ps.add_f32(beta); ps.add_f32(out);
+    st = check_alignment(ps, &vec);
+    if (st != RLCS_OK) return st;
+    p.f0 = alpha; p.f1 = beta; p.out0 = out;
+    st = finish_params(p, total, T, workspace, workspace_bytes);
+    if (st != RLCS_OK) return st;
+    return run(forward ? rlcs::launch_affine_fwd : rlcs::launch_affine_bwd, p, false, vec, cuda_stream);
+}
+
+int rlcs_debug_set_tile_variant(int variant) {
+    if (variant < 0 || variant >= rlcs::kNumVariants) return RLCS_ERR_ARG;
+    g_variant = variant;
+    return RLCS_OK;
+}
+
+int rlcs_debug_tile_elems(int variant) {
+    if (variant < 0 || variant >= rlcs::kNumVariants) return 0;
+    return tile_elems(variant);
+}
+
+int rlcs_debug_set_carry_fault(int64_t mute_tile, int64_t spin_cap) {
+    g_mute_tile = mute_tile;
+    g_spin_cap = spin_cap;
+    return RLCS_OK;
+}
+
+}  // extern "C"

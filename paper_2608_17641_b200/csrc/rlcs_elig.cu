@@ -1,0 +1,6 @@
+// Kernel instantiations for one algorithm (see rlcs_scan.cuh for the kernel itself).
+#include "rlcs_launch.cuh"
+
+namespace rlcs {
+RLCS_DEFINE_LAUNCHER(launch_elig, kElig, false)
+}  // namespace rlcs

@@ -1,0 +1,139 @@
+"""Host-side checks that need no GPU: the library builds and loads, exports every symbol the
+header declares, and rejects bad arguments before anything is launched (no compute calls here)."""
+import ctypes
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+OK, E_NULL, E_SIZE, E_ARG, E_ALIGN, E_WS = 0, 1, 2, 3, 4, 5
+
+
+@pytest.fixture(scope="module")
+def L():
+    from paper_2608_17641_b200 import build, binding
+    build.build()
+    return binding.lib()
+
+
+def _declared_symbols():
+    text = open(os.path.join(ROOT, "include", "rlcs.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(rlcs_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_header_declares_the_seven_entry_points():
+    names = _declared_symbols()
+    for n in ("rlcs_gae", "rlcs_vtrace", "rlcs_retrace", "rlcs_td_lambda", "rlcs_discounted_return",
+              "rlcs_elig_trace", "rlcs_episodic_prefix_sum", "rlcs_workspace_bytes", "rlcs_workspace_init",
+              "rlcs_last_device_status", "rlcs_status_string"):
+        assert n in names
+
+
+def test_library_exports_every_declared_symbol(L):
+    from paper_2608_17641_b200 import binding
+    for name in _declared_symbols():
+        assert hasattr(L, name), f"{name} declared in rlcs.h but not exported"
+        assert name in binding.SIGNATURES, f"{name} has no binding signature"
+    for name in binding.SIGNATURES:
+        assert name in _declared_symbols(), f"binding knows {name} but rlcs.h does not declare it"
+
+
+def test_status_strings(L):
+    assert L.rlcs_status_string(0) == b"RLCS_OK"
+    for s in range(1, 8):
+        assert L.rlcs_status_string(s).startswith(b"RLCS_ERR_")
+    assert b"unknown" in L.rlcs_status_string(99)
+
+
+def test_workspace_bytes(L):
+    assert L.rlcs_workspace_bytes(0, 128) == 0 and L.rlcs_workspace_bytes(8, 0) == 0
+    assert L.rlcs_workspace_bytes(-1, 5) == 0
+    for T in (1, 2, 64, 128, 512):                      # T divides every tile: nothing straddles
+        assert L.rlcs_workspace_bytes(4096, T) == 0
+    assert L.rlcs_workspace_bytes(64, 16384) == 256 + 16 * (64 * 16384 // 512)
+    assert L.rlcs_workspace_bytes(3, 1000) == 256 + 16 * ((3000 + 511) // 512)
+
+
+# fake, never-dereferenced device addresses: every call below must return before any launch
+P = 0x7f0000000000
+Q = P + 4                                                # 4-byte but not 16-byte aligned
+ODD = P + 2                                              # not even 4-byte aligned
+
+
+def _gae(L, r=P, v=P, d=P, tr=None, bv=None, bt=None, adv=P, ret=None, N=4, T=8, g=0.99, l=0.95, ws=None, wsb=0):
+    return L.rlcs_gae(r, v, d, tr, bv, bt, adv, ret, N, T, g, l, ws, wsb, None)
+
+
+def test_empty_problem_is_ok_without_launch(L):
+    assert _gae(L, N=0) == OK and _gae(L, T=0) == OK
+    assert L.rlcs_elig_trace(None, None, None, 0, 5, 0.9, 0.9, None, 0, None) == OK
+
+
+def test_size_errors(L):
+    assert _gae(L, N=-1) == E_SIZE and _gae(L, T=-3) == E_SIZE
+    assert _gae(L, T=2 ** 31) == E_SIZE
+    assert _gae(L, N=2 ** 40, T=2 ** 20) == E_SIZE
+
+
+def test_parameter_errors(L):
+    for g, l in [(-0.1, 0.5), (1.1, 0.5), (0.5, -1e-3), (0.5, 1.5), (float("nan"), 0.5), (0.5, float("nan"))]:
+        assert _gae(L, g=g, l=l) == E_ARG
+    v = lambda rb, cb: L.rlcs_vtrace(P, P, P, P, None, None, None, P, None, 4, 8, 0.9, rb, cb, None, 0, None)
+    assert v(-1.0, 1.0) == E_ARG and v(1.0, float("nan")) == E_ARG
+    assert L.rlcs_retrace(P, P, P, P, P, None, None, None, P, 4, 8, 0.9, 2.0, 1.0, None, 0, None) == E_ARG
+    assert L.rlcs_discounted_return(P, P, None, None, None, P, 4, 8, 7.0, None, 0, None) == E_ARG
+    assert L.rlcs_elig_trace(P, P, P, 4, 8, 0.9, -0.5, None, 0, None) == E_ARG
+
+
+def test_null_pointer_errors(L):
+    assert _gae(L, r=None) == E_NULL and _gae(L, v=None) == E_NULL
+    assert _gae(L, d=None) == E_NULL and _gae(L, adv=None) == E_NULL
+    assert _gae(L, tr=P, bv=None) == E_NULL and _gae(L, tr=None, bv=P) == E_NULL
+    assert L.rlcs_episodic_prefix_sum(P, None, P, 4, 8, 0, None, 0, None) == E_NULL
+    assert L.rlcs_affine_scan(P, None, P, 4, 8, 0, None, 0, None) == E_NULL
+
+
+def test_alignment_errors(L):
+    assert _gae(L, r=ODD) == E_ALIGN
+    assert _gae(L, adv=ODD) == E_ALIGN
+    # rows straddle tiles at T = 1000: a workspace is required, 16-byte aligned, large enough
+    need = L.rlcs_workspace_bytes(4, 1000)
+    assert need > 0
+    assert _gae(L, N=4, T=1000) == E_WS
+    assert _gae(L, N=4, T=1000, ws=P, wsb=need - 16 * 8) == E_WS
+    assert _gae(L, N=4, T=1000, ws=Q, wsb=need) == E_ALIGN
+
+
+def test_workspace_init_argument_checks(L):
+    assert L.rlcs_workspace_init(None, 0, None) == OK
+    assert L.rlcs_workspace_init(None, 64, None) == E_NULL
+    assert L.rlcs_workspace_init(Q, 4096, None) == E_ALIGN
+    assert L.rlcs_workspace_init(P, 8, None) == E_WS
+    assert L.rlcs_last_device_status(None, None) == OK
+
+
+def test_debug_hooks_argument_checks(L):
+    assert L.rlcs_debug_set_tile_variant(99) == E_ARG and L.rlcs_debug_set_tile_variant(-1) == E_ARG
+    assert L.rlcs_debug_set_tile_variant(0) == OK
+    assert L.rlcs_debug_tile_elems(0) == 2048 and L.rlcs_debug_tile_elems(1) == 512
+    assert L.rlcs_debug_tile_elems(99) == 0
+
+
+def test_binding_rejects_cpu_tensors_and_wrong_dtypes():
+    import torch
+    from paper_2608_17641_b200 import binding
+    x = torch.zeros(2, 8)
+    d = torch.zeros(2, 8, dtype=torch.uint8)
+    with pytest.raises(TypeError):                       # no CPU path: CUDA tensors only
+        binding.rlcs_elig_trace(x, d, gamma=0.9, lam=0.9, traces=x.clone())
+
+
+def test_missing_library_fails_loudly(tmp_path, monkeypatch):
+    from paper_2608_17641_b200 import binding
+    monkeypatch.setattr(binding, "_lib", None)
+    monkeypatch.setattr(binding, "LIB_PATH", str(tmp_path / "nope.so"))
+    with pytest.raises(RuntimeError, match="no fallback"):
+        binding.lib()

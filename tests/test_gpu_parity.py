@@ -1,0 +1,309 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the fp64 CPU oracle on the same
+seeded inputs.  Bar: |gpu - ref| <= 1e-4 + 1e-5 |ref| element by element; segmentation exact."""
+import numpy as np
+import pytest
+
+from _util import ALL_ALGOS, Dev, assert_close, compare_all, run_gpu, run_oracle
+
+pytestmark = pytest.mark.gpu
+
+BACKWARD = ("gae", "vtrace", "retrace", "td_lambda", "discounted_return")
+
+
+@pytest.fixture(scope="module")
+def W():
+    from paper_2608_17641_b200 import workloads
+    return workloads
+
+
+@pytest.fixture(scope="module")
+def B():
+    import torch
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    from paper_2608_17641_b200 import binding
+    binding.lib()                      # fail loudly if the extension is missing
+    binding.rlcs_debug_set_tile_variant(0)
+    binding.rlcs_debug_set_carry_fault(-1, 0)
+    return binding
+
+
+# ------------------------------------------------------------------ the benchmark configurations
+def test_config1_gae_8x128(oracle, W, B):
+    compare_all(oracle, W.config1(), algos=("gae",))
+
+
+def test_config2_all_seven_4096x64(oracle, W, B):
+    compare_all(oracle, W.config2())
+
+
+@pytest.mark.parametrize("T", [32, 64, 128, 256, 512, 1024])
+@pytest.mark.parametrize("with_truncs", [False, True])
+def test_config3_sweep(oracle, W, B, T, with_truncs):
+    ro = W.config3(T, with_truncs)
+    compare_all(oracle, ro, algos=("gae", "vtrace"), use_truncs=with_truncs)
+
+
+def test_config4_long_rows(oracle, W, B):
+    ro = W.config4()
+    gpu, ref, _ = compare_all(oracle, ro, algos=("gae", "discounted_return"), use_truncs=False)
+    # gamma = 1 and rewards only at segment ends: adding zeros is exact in any association, so the
+    # GPU returns must equal the oracle's bit for bit (after rounding the oracle to fp32).
+    assert np.array_equal(gpu["discounted_return"], ref["discounted_return"].astype(np.float32))
+
+
+def test_config5_full_size_all_seven(oracle, W, B):
+    """16384 x 2048, truncation handling on: every element of every output against the oracle."""
+    ro = W.config5()
+    dev = Dev(ro)
+    for a in ALL_ALGOS:                       # one algorithm at a time keeps host memory bounded
+        gpu = run_gpu(dev, (a,))
+        ref = run_oracle(oracle, ro, (a,))
+        if isinstance(ref[a], tuple):
+            for i, (g, r) in enumerate(zip(gpu[a], ref[a])):
+                assert_close(f"{a}[{i}]", g, r)
+        else:
+            assert_close(a, gpu[a], ref[a])
+
+
+# ------------------------------------------------------------------ shape / flag matrix
+SHAPES = [(1, 1), (3, 1), (1, 2), (2, 3), (3, 4), (8, 5), (3, 7), (64, 8), (3, 9), (8, 31), (64, 32), (3, 33),
+          (8, 63), (2, 65), (3, 127), (8, 1000), (3, 2047), (2, 2048), (3, 2049), (2, 4097), (1, 20000)]
+
+
+@pytest.mark.parametrize("N,T", SHAPES)
+@pytest.mark.parametrize("p_flag", [0.0, 0.01, 0.5, 1.0])
+def test_shape_matrix(oracle, W, B, N, T, p_flag):
+    ro = W.make_rollout(90, N, T, p_done=p_flag, p_trunc=p_flag / 2, salt=N * 100003 + T)
+    compare_all(oracle, ro)
+
+
+@pytest.mark.parametrize("variant", [0, 1, 2, 3])
+@pytest.mark.parametrize("N,T", [(5, 700), (4097, 3), (2, 9000), (64, 513)])
+def test_tile_variants(oracle, W, B, variant, N, T):
+    B.rlcs_debug_set_tile_variant(variant)
+    try:
+        ro = W.make_rollout(91, N, T, p_done=0.01, p_trunc=0.005, salt=T)
+        compare_all(oracle, ro)
+    finally:
+        B.rlcs_debug_set_tile_variant(0)
+
+
+def test_long_row_without_resets_multi_window_lookback(oracle, W, B):
+    """T = 131073 with no flags: 65 tiles per row, so the look-back crosses its 32-record window."""
+    ro = W.make_rollout(92, 3, 131073, p_done=0.0, p_trunc=0.0)
+    ro.params["gamma"] = 1.0
+    ro.params["lam"] = 1.0
+    compare_all(oracle, ro, algos=("gae", "discounted_return", "elig_trace", "prefix_ends_at", "vtrace", "retrace"))
+    B.rlcs_debug_set_tile_variant(1)          # 512-step tiles: 257 tiles per row
+    try:
+        compare_all(oracle, ro, algos=("gae", "prefix_ends_at"))
+    finally:
+        B.rlcs_debug_set_tile_variant(0)
+
+
+# ------------------------------------------------------------------ boundary cases
+def _forced(W, N=6, T=300, salt=0):
+    ro = W.make_rollout(93, N, T, p_done=0.02, p_trunc=0.02, salt=salt)
+    ro.dones[0, 0] = 1                        # flags at both ends
+    ro.dones[0, -1] = 1
+    ro.truncs[1, 0] = 1
+    ro.truncs[1, -1] = 1                      # truncated last step
+    ro.dones[2, 17] = ro.truncs[2, 17] = 1    # both flags on one step
+    ro.dones[3, -1] = ro.truncs[3, -1] = 1
+    ro.dones[4, :] = 0
+    ro.truncs[4, :] = 0                       # a row without any flag
+    return ro
+
+
+def test_forced_boundary_flags(oracle, W, B):
+    compare_all(oracle, _forced(W))
+
+
+def test_null_bootstrap_and_null_truncs(oracle, W, B):
+    ro = _forced(W, salt=1)
+    compare_all(oracle, ro, algos=BACKWARD, use_bootstrap=False)
+    compare_all(oracle, ro, algos=BACKWARD, use_truncs=False)
+    compare_all(oracle, ro, algos=BACKWARD, use_truncs=False, use_bootstrap=False)
+
+
+@pytest.mark.parametrize("offset", [1, 2, 3])
+@pytest.mark.parametrize("N,T", [(5, 333), (3, 2048), (2, 5000)])
+def test_unaligned_pointers_take_elementwise_path(oracle, W, B, offset, N, T):
+    ro = W.make_rollout(94, N, T, salt=offset)
+    compare_all(oracle, ro, offset=offset)
+
+
+def test_optional_outputs_null(oracle, W, B):
+    ro = W.make_rollout(95, 7, 500)
+    dev = Dev(ro)
+    ws = B.Workspace(ro.N, ro.T)
+    p = ro.params
+    adv = B.rlcs_gae(dev.rewards, dev.values, dev.dones, dev.truncs, dev.trunc_bootstrap, dev.bootstrap,
+                     gamma=p["gamma"], lam=p["lam"], want_returns=False, workspace=ws)
+    vs = B.rlcs_vtrace(dev.rewards, dev.values, dev.log_rhos, dev.dones, dev.truncs, dev.trunc_bootstrap,
+                       dev.bootstrap, gamma=p["gamma"], want_advantages=False, workspace=ws)
+    ref = run_oracle(oracle, ro, ("gae", "vtrace"))
+    assert_close("adv", adv.cpu().numpy(), ref["gae"][0])
+    assert_close("vs", vs.cpu().numpy(), ref["vtrace"][0])
+
+
+def test_guard_bands_untouched(oracle, W, B):
+    """Outputs sit between NaN canaries; nothing outside [N*T) may be written."""
+    import torch
+    N, T, pad = 5, 1001, 64
+    ro = W.make_rollout(96, N, T)
+    dev = Dev(ro)
+    ws = B.Workspace(N, T)
+    p = ro.params
+
+    def guarded():
+        flat = torch.full((N * T + 2 * pad,), float("nan"), device="cuda")
+        return flat, flat[pad:pad + N * T].view(N, T)
+
+    f1, adv = guarded()
+    f2, ret = guarded()
+    f3, z = guarded()
+    B.rlcs_gae(dev.rewards, dev.values, dev.dones, dev.truncs, dev.trunc_bootstrap, dev.bootstrap, gamma=p["gamma"],
+               lam=p["lam"], advantages=adv, returns=ret, workspace=ws)
+    B.rlcs_elig_trace(dev.x, dev.any_done, gamma=p["gamma"], lam=p["lam"], traces=z, workspace=ws)
+    torch.cuda.synchronize()
+    for f in (f1, f2, f3):
+        assert torch.isnan(f[:pad]).all() and torch.isnan(f[-pad:]).all()
+        assert torch.isfinite(f[pad:-pad]).all()
+
+
+def test_nonbinary_flag_bytes(oracle, W, B):
+    ro = W.make_rollout(97, 4, 600, p_done=0.05, p_trunc=0.05)
+    ro.dones = (ro.dones * np.uint8(0x80)).astype(np.uint8)
+    ro.truncs = (ro.truncs * np.uint8(0x7f)).astype(np.uint8)
+    compare_all(oracle, ro)
+
+
+def test_gamma_lambda_extremes(oracle, W, B):
+    for g, l in [(0.0, 0.5), (1.0, 1.0), (0.5, 0.0), (1.0, 0.0)]:
+        ro = W.make_rollout(98, 6, 777, p_done=0.01, p_trunc=0.01)
+        ro.params.update(gamma=g, lam=l)
+        compare_all(oracle, ro)
+
+
+def test_clip_thresholds(oracle, W, B):
+    for rb, cb in [(0.0, 0.0), (0.5, 2.0), (float("inf"), float("inf")), (1.5, 0.0)]:
+        ro = W.make_rollout(99, 6, 555)
+        ro.params.update(rho_bar=rb, c_bar=cb)
+        compare_all(oracle, ro, algos=("vtrace", "retrace"))
+
+
+# ------------------------------------------------------------------ segmentation is exact
+def test_severed_steps_equal_alpha_exactly(oracle, W, B):
+    ro = W.make_rollout(100, 16, 3000, p_done=0.03, p_trunc=0.0, with_truncs=False)
+    gpu = run_gpu(Dev(ro), ("gae", "discounted_return"), use_truncs=False)
+    tm = ro.dones != 0
+    assert np.array_equal(gpu["discounted_return"][tm], ro.rewards[tm])
+    assert np.array_equal(gpu["gae"][0][tm], (ro.rewards - ro.values)[tm])
+
+
+def test_segment_isolation_bitwise(oracle, W, B):
+    """Overwriting everything after a terminated step leaves the outputs up to it bit-identical
+    (backward scans); overwriting everything before it leaves the later outputs bit-identical
+    (forward scans).  The cut at t = 5000 is inside a tile, rows span several tiles."""
+    ro = W.make_rollout(101, 3, 9000, p_done=0.0, p_trunc=0.0)
+    cut = 5000
+    ro.dones[:, cut] = 1
+    base = run_gpu(Dev(ro), ALL_ALGOS)
+    ro2 = W.make_rollout(101, 3, 9000, p_done=0.0, p_trunc=0.0, salt=7)
+    ro2.dones[:, cut] = 1
+    for k in ("rewards", "values", "q_sa", "expected_q", "log_rhos", "x", "trunc_bootstrap"):
+        a = getattr(ro, k).copy()
+        getattr(ro2, k)[:, :cut + 1] = a[:, :cut + 1]
+    other = run_gpu(Dev(ro2), BACKWARD)
+    for a in BACKWARD:
+        pairs = zip(base[a], other[a]) if isinstance(base[a], tuple) else [(base[a], other[a])]
+        for g0, g1 in pairs:
+            assert np.array_equal(g0[:, :cut + 1], g1[:, :cut + 1]), a
+            assert not np.array_equal(g0[:, cut + 1:], g1[:, cut + 1:]), a
+    ro3 = W.make_rollout(101, 3, 9000, p_done=0.0, p_trunc=0.0, salt=9)
+    ro3.dones[:, cut] = 1
+    ro3.x[:, cut + 1:] = ro.x[:, cut + 1:]
+    fwd = run_gpu(Dev(ro3), ("elig_trace", "prefix_ends_at"))
+    for a in ("elig_trace", "prefix_ends_at"):
+        assert np.array_equal(base[a][:, cut + 1:], fwd[a][:, cut + 1:]), a
+        assert not np.array_equal(base[a][:, :cut + 1], fwd[a][:, :cut + 1]), a
+
+
+def test_bootstrap_only_reaches_last_open_segment(oracle, W, B):
+    ro = W.make_rollout(102, 4, 5000, p_done=0.001, p_trunc=0.0)
+    base = run_gpu(Dev(ro), BACKWARD)
+    ro.bootstrap = ro.bootstrap + np.float32(3.0)
+    other = run_gpu(Dev(ro), BACKWARD)
+    for n in range(ro.N):
+        flagged = np.flatnonzero(ro.dones[n])
+        last_reset = flagged[-1] if len(flagged) else -1
+        for a in BACKWARD:
+            g0 = base[a][0] if isinstance(base[a], tuple) else base[a]
+            g1 = other[a][0] if isinstance(other[a], tuple) else other[a]
+            assert np.array_equal(g0[n, :last_reset + 1], g1[n, :last_reset + 1]), a
+
+
+def test_run_to_run_bit_identical(oracle, W, B):
+    ro = W.config4(N=16, T=16384)
+    dev = Dev(ro)
+    first = run_gpu(dev, ("gae", "discounted_return"), use_truncs=False)
+    for _ in range(5):
+        again = run_gpu(dev, ("gae", "discounted_return"), use_truncs=False)
+        assert np.array_equal(first["discounted_return"], again["discounted_return"])
+        assert np.array_equal(first["gae"][0], again["gae"][0]) and np.array_equal(first["gae"][1], again["gae"][1])
+
+
+def test_workspace_reuse_across_algorithms_and_shapes(oracle, W, B):
+    """One workspace, many calls of different entry points and shapes on one stream."""
+    big = B.Workspace(64, 5000)
+    for (N, T) in [(64, 5000), (3, 700), (64, 4999)]:
+        ro = W.make_rollout(103, N, T, salt=T)
+        compare_all(oracle, ro, workspace=big)
+
+
+# ------------------------------------------------------------------ test hooks
+def test_affine_scan_matches_generic_recurrence(oracle, W, B):
+    import torch
+    rng = np.random.default_rng(5)
+    N, T = 4, 3000
+    alpha = rng.standard_normal((N, T)).astype(np.float32)
+    beta = rng.uniform(0.0, 1.0, (N, T)).astype(np.float32)
+    beta[rng.random((N, T)) < 0.01] = 0.0
+    ws = B.Workspace(N, T)
+    for fwd in (False, True):
+        out = B.rlcs_affine_scan(torch.from_numpy(alpha).cuda(), torch.from_numpy(beta).cuda(), forward=fwd,
+                                 workspace=ws).cpu().numpy()
+        ref = np.stack([oracle.linear_recurrence(alpha[n].astype(np.float64), beta[n].astype(np.float64), 0.0,
+                                                 forward=fwd) for n in range(N)])
+        assert_close(f"affine fwd={fwd}", out, ref)
+
+
+def test_bounded_carry_wait_reports_timeout_and_returns(oracle, W, B):
+    """A tile that never publishes: its dependant's wait runs out of polls, the kernel finishes,
+    the status word says TIMEOUT, and the next call on the same workspace works again."""
+    import torch
+    ro = W.make_rollout(104, 1, 16384, p_done=0.0, p_trunc=0.0)
+    dev = Dev(ro)
+    ws = B.Workspace(ro.N, ro.T)
+    B.rlcs_debug_set_carry_fault(2, 64)
+    try:
+        B.rlcs_discounted_return(dev.rewards, dev.dones, gamma=0.99, workspace=ws)
+        torch.cuda.synchronize()
+        assert ws.device_status() == B.RLCS_ERR_TIMEOUT
+    finally:
+        B.rlcs_debug_set_carry_fault(-1, 0)
+    assert ws.device_status() == B.RLCS_OK            # cleared by the read
+    compare_all(oracle, ro, algos=("discounted_return",), workspace=ws)
+
+
+def test_missing_workspace_is_an_error_not_a_launch(oracle, W, B):
+    ro = W.make_rollout(105, 2, 3000)
+    dev = Dev(ro)
+    with pytest.raises(B.RlcsError) as e:
+        B.rlcs_discounted_return(dev.rewards, dev.dones, gamma=0.99, workspace=None)
+    assert e.value.status == B.RLCS_ERR_WORKSPACE
+    small = B.Workspace(2, 3000, nbytes=256)
+    with pytest.raises(B.RlcsError) as e:
+        B.rlcs_discounted_return(dev.rewards, dev.dones, gamma=0.99, workspace=small)
+    assert e.value.status == B.RLCS_ERR_WORKSPACE
