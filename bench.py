@@ -1,0 +1,491 @@
+#!/usr/bin/env python
+"""Benchmark of the fused credit-assignment scans on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--no-sweep]
+
+A "step" is one pass of the whole hot path over one synthetic batch: the seven algorithms (GAE,
+V-Trace, Retrace, TD(lambda), discounted returns, eligibility trace, episodic prefix sum), one fused
+kernel launch each, on the 16384 x 2048 bandwidth-saturating configuration with per-step truncation
+handling.  `value` counts N*T env-steps per algorithm pass, i.e. 7*N*T per step and per GPU.
+
+Rank 0 prints ONE JSON line.  With N > 1 (torchrun) every rank works on its own batch of the same
+shape (rows are independent: weak scaling, no collective on the data path); the time is the max
+over ranks.  `--impl reference` times the CPU oracle instead (rank 0 only).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+METRIC = "env-steps/s"
+ALGOS = ("gae", "vtrace", "retrace", "td_lambda", "discounted_return", "elig_trace", "episodic_prefix_sum")
+WORKLOAD = dict(N=16384, T=2048)
+FALLBACK_HBM_GBS = 6650.0
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel on the bench
+# workload, from the ncu capture summarised under profiles/ (None until a capture exists).
+NCU_TRAFFIC_BYTES = {}
+
+
+# --------------------------------------------------------------------------------------------- helpers
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as fh:
+            return float(json.load(fh)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+def algorithmic_bytes(ro, algo: str) -> int:
+    """Compulsory input + output bytes of one launch: every [N,T] input read once, every output
+    written once, the [N] bootstrap once, and of the 2-D truncation bootstrap only the 32-byte
+    sectors that hold a value the kernel must read (truncated and not terminated)."""
+    S = ro.N * ro.T
+    f32_in = {"gae": 2, "vtrace": 3, "retrace": 4, "td_lambda": 2, "discounted_return": 1,
+              "elig_trace": 1, "episodic_prefix_sum": 1}[algo]
+    f32_out = {"gae": 2, "vtrace": 2}.get(algo, 1)
+    b = 4 * S * (f32_in + f32_out) + S                      # fp32 tensors + the done mask
+    if algo not in ("elig_trace", "episodic_prefix_sum"):
+        b += 4 * ro.N                                       # window-edge bootstrap
+        if ro.truncs is not None:
+            b += S                                          # truncation mask
+            idx = np.flatnonzero((ro.truncs.ravel() != 0) & (ro.dones.ravel() == 0))
+            b += 32 * int(np.unique(idx // 8).size)
+    return int(b)
+
+
+class ClockSampler:
+    """Samples SM clock and clock-event reasons through NVML while the timed region runs."""
+
+    REASONS = {0x1: "gpu_idle", 0x2: "applications_clocks_setting", 0x4: "sw_power_cap", 0x8: "hw_slowdown",
+               0x10: "sync_boost", 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown",
+               0x80: "hw_power_brake_slowdown", 0x100: "display_clock_setting"}
+
+    def __init__(self, index: int, period_s: float = 0.002):
+        self.samples, self.reasons, self.power = [], set(), []
+        self.period, self._stop, self.max_mhz, self.ok = period_s, threading.Event(), None, False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+            self.ok = True
+        except Exception:
+            self.ok = False
+        self.t = threading.Thread(target=self._run, daemon=True)
+
+    def _once(self):
+        nv = self.nv
+        self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+        try:
+            mask = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.h))
+        except Exception:
+            mask = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+        for bit, name in self.REASONS.items():
+            if mask & bit and name != "gpu_idle":
+                self.reasons.add(name)
+        try:
+            self.power.append(nv.nvmlDeviceGetPowerUsage(self.h) / 1000.0)
+        except Exception:
+            pass
+
+    def _run(self):
+        while not self._stop.is_set():
+            try:
+                self._once()
+            except Exception:
+                break
+            time.sleep(self.period)
+
+    def __enter__(self):
+        if self.ok:
+            self.t.start()
+        return self
+
+    def __exit__(self, *exc):
+        self._stop.set()
+        if self.ok:
+            self.t.join(timeout=2)
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0}
+        return {"sm_mhz": int(statistics.median(self.samples)), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples),
+                "power_w_max": round(max(self.power), 1) if self.power else None}
+
+
+# --------------------------------------------------------------------------------------------- GPU arm
+class GpuBatch:
+    """Device-resident inputs, outputs and workspace of one batch, and the seven calls on them."""
+
+    def __init__(self, ro, device):
+        import torch
+        from paper_2608_17641_b200 import binding as B
+        self.B, self.ro, self.torch = B, ro, torch
+        up = lambda a: None if a is None else torch.from_numpy(a).to(device, non_blocking=False)
+        self.inp = {k: up(getattr(ro, k)) for k in ("rewards", "values", "q_sa", "expected_q", "log_rhos", "x",
+                                                    "dones", "truncs", "trunc_bootstrap", "bootstrap")}
+        self.inp["any_done"] = up(ro.any_done)
+        new = lambda: torch.empty((ro.N, ro.T), dtype=torch.float32, device=device)
+        self.out = {"gae": (new(), new()), "vtrace": (new(), new()), "retrace": new(), "td_lambda": new(),
+                    "discounted_return": new(), "elig_trace": new(), "episodic_prefix_sum": new()}
+        self.ws = B.Workspace(ro.N, ro.T, device=device)
+        self.launches = 0
+
+    def call(self, algo: str):
+        B, i, o, p, ws = self.B, self.inp, self.out, self.ro.params, self.ws
+        bw = (i["dones"], i["truncs"], i["trunc_bootstrap"], i["bootstrap"])
+        if algo == "gae":
+            B.rlcs_gae(i["rewards"], i["values"], *bw, gamma=p["gamma"], lam=p["lam"], advantages=o[algo][0],
+                       returns=o[algo][1], workspace=ws)
+        elif algo == "vtrace":
+            B.rlcs_vtrace(i["rewards"], i["values"], i["log_rhos"], *bw, gamma=p["gamma"], rho_bar=p["rho_bar"],
+                          c_bar=p["c_bar"], vs=o[algo][0], pg_advantages=o[algo][1], workspace=ws)
+        elif algo == "retrace":
+            B.rlcs_retrace(i["rewards"], i["q_sa"], i["expected_q"], i["log_rhos"], *bw, gamma=p["gamma"],
+                           lam=p["lam"], c_bar=p["c_bar"], q_targets=o[algo], workspace=ws)
+        elif algo == "td_lambda":
+            B.rlcs_td_lambda(i["rewards"], i["values"], *bw, gamma=p["gamma"], lam=p["lam"], returns=o[algo], workspace=ws)
+        elif algo == "discounted_return":
+            B.rlcs_discounted_return(i["rewards"], *bw, gamma=p["gamma"], returns=o[algo], workspace=ws)
+        elif algo == "elig_trace":
+            B.rlcs_elig_trace(i["x"], i["any_done"], gamma=p["gamma"], lam=p["lam"], traces=o[algo], workspace=ws)
+        elif algo == "episodic_prefix_sum":
+            B.rlcs_episodic_prefix_sum(i["x"], i["any_done"], sums=o[algo], workspace=ws)
+        else:
+            raise KeyError(algo)
+        self.launches += 1
+
+    def step(self, events=None):
+        torch = self.torch
+        for k, a in enumerate(ALGOS):
+            if events is not None:
+                events[k].record()
+            self.call(a)
+        if events is not None:
+            events[len(ALGOS)].record()
+
+
+def time_device(batch: GpuBatch, steps: int, warmup: int, dist):
+    """K timed steps with inputs resident in HBM; per-kernel durations from CUDA events recorded
+    on the launching stream between the launches."""
+    torch = batch.torch
+    for _ in range(warmup):
+        batch.step()
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(len(ALGOS) + 1)] for _ in range(steps)]
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    dist.barrier()
+    torch.cuda.synchronize()
+    launches0 = batch.launches
+    with ClockSampler(torch.cuda.current_device()) as clk:
+        start.record()
+        for k in range(steps):
+            batch.step(ev[k])
+        stop.record()
+        torch.cuda.synchronize()
+    dist.barrier()
+    total_ms = start.elapsed_time(stop)
+    per_algo_ms = {a: [ev[k][j].elapsed_time(ev[k][j + 1]) for k in range(steps)] for j, a in enumerate(ALGOS)}
+    assert batch.ws.device_status() == 0, "device reported a carry-wait timeout"
+    return total_ms, per_algo_ms, batch.launches - launches0, clk.summary()
+
+
+def time_e2e(batch: GpuBatch, steps: int, warmup: int, dist):
+    """The same step called with HOST buffers: every step copies that step's inputs from pinned
+    host memory to the device, runs the seven C-ABI calls, and reads all outputs back."""
+    torch, ro = batch.torch, batch.ro
+    pin = lambda t: torch.empty(t.shape, dtype=t.dtype).pin_memory().copy_(t.cpu())
+    h_in = {k: pin(v) for k, v in batch.inp.items() if v is not None}
+    h_out = {}
+    for a, v in batch.out.items():
+        h_out[a] = tuple(torch.empty(t.shape, dtype=t.dtype).pin_memory() for t in v) if isinstance(v, tuple) \
+            else torch.empty(v.shape, dtype=v.dtype).pin_memory()
+    h2d = sum(t.numel() * t.element_size() for t in h_in.values())
+    d2h = sum(t.numel() * t.element_size() for v in h_out.values() for t in (v if isinstance(v, tuple) else (v,)))
+
+    def one():
+        for k, t in h_in.items():
+            batch.inp[k].copy_(t, non_blocking=True)
+        batch.step()
+        for a, v in batch.out.items():
+            if isinstance(v, tuple):
+                for hv, dv in zip(h_out[a], v):
+                    hv.copy_(dv, non_blocking=True)
+            else:
+                h_out[a].copy_(v, non_blocking=True)
+
+    for _ in range(warmup):
+        one()
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    dist.barrier()
+    torch.cuda.synchronize()
+    start.record()
+    for _ in range(steps):
+        one()
+    stop.record()
+    torch.cuda.synchronize()
+    dist.barrier()
+    return start.elapsed_time(stop), h2d, d2h
+
+
+# --------------------------------------------------------------------------------------------- CPU oracle arm
+def oracle_pass(ro, rows: int, threads: int):
+    """All seven algorithms of the oracle, as it stands, on the first `rows` rows; returns seconds."""
+    import oracle
+    p = ro.params
+    s = slice(0, rows)
+    cut = lambda a: None if a is None else a[s]
+    bw2 = dict(dones=cut(ro.dones), truncs=cut(ro.truncs), trunc_bootstrap=cut(ro.trunc_bootstrap))
+    bw1 = dict(bootstrap=cut(ro.bootstrap))
+    d_fwd = cut(ro.any_done)
+    par = lambda fn, a2, a1, **kw: oracle.run_rows_parallel(fn, a2, a1, threads, **kw)
+    t0 = time.perf_counter()
+    par(oracle.gae, dict(rewards=cut(ro.rewards), values=cut(ro.values), **bw2), bw1, gamma=p["gamma"], lam=p["lam"])
+    par(oracle.vtrace, dict(rewards=cut(ro.rewards), values=cut(ro.values), log_rhos=cut(ro.log_rhos), **bw2), bw1,
+        gamma=p["gamma"], rho_bar=p["rho_bar"], c_bar=p["c_bar"])
+    par(oracle.retrace, dict(rewards=cut(ro.rewards), q_sa=cut(ro.q_sa), expected_q=cut(ro.expected_q),
+                             log_rhos=cut(ro.log_rhos), **bw2), bw1, gamma=p["gamma"], lam=p["lam"], c_bar=p["c_bar"])
+    par(oracle.td_lambda, dict(rewards=cut(ro.rewards), values=cut(ro.values), **bw2), bw1, gamma=p["gamma"], lam=p["lam"])
+    par(oracle.discounted_return, dict(rewards=cut(ro.rewards), **bw2), bw1, gamma=p["gamma"])
+    par(oracle.elig_trace, dict(x=cut(ro.x), dones=d_fwd), {}, gamma=p["gamma"], lam=p["lam"])
+    par(oracle.episodic_prefix_sum, dict(x=cut(ro.x), dones=d_fwd), {})
+    return time.perf_counter() - t0
+
+
+def cpu_baseline(ro, budget_s: float = 20.0):
+    import oracle
+    oracle.build()
+    threads = os.cpu_count() or 1
+    probe_rows = min(ro.N, 256)
+    t = oracle_pass(ro, probe_rows, threads)                          # calibration (also warms the library)
+    rows = int(min(ro.N, max(probe_rows, probe_rows * budget_s / max(t, 1e-6))))
+    secs = oracle_pass(ro, rows, threads)
+    return {"value": len(ALGOS) * rows * ro.T / secs, "unit": METRIC, "cores": threads, "kind": "oracle",
+            "sample": f"first {rows} of {ro.N} rows x T={ro.T}, all seven algorithms once, {secs:.2f} s, "
+                      f"fp64 sequential C oracle, rows split over {threads} host threads"}
+
+
+def reference_arm(args, world: int):
+    """The CPU oracle on the bench workload; each step is a bounded row sample of it."""
+    from paper_2608_17641_b200 import workloads
+    import oracle
+    oracle.build()
+    ro = workloads.config5(**WORKLOAD)
+    threads = os.cpu_count() or 1
+    probe = 128
+    t = oracle_pass(ro, probe, threads)
+    per_step_budget = 150.0 / max(1, args.steps + args.warmup)
+    rows = int(min(ro.N, max(16, probe * per_step_budget / max(t, 1e-6))))
+    for _ in range(args.warmup):
+        oracle_pass(ro, rows, threads)
+    times = [oracle_pass(ro, rows, threads) for _ in range(args.steps)]
+    total = sum(times)
+    value = len(ALGOS) * rows * ro.T * args.steps / total
+    sample = (f"each step = first {rows} of {ro.N} rows x T={ro.T}, all seven algorithms, fp64 sequential C oracle, "
+              f"rows split over {threads} host threads")
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": METRIC, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": f"all seven algorithms, num_envs={ro.N}, T={ro.T}, fp32 inputs, truncation handling on "
+                               f"(bounded row sample per step)", "rows_per_step": rows},
+        "cpu_baseline": {"value": value, "unit": METRIC, "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": METRIC, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# --------------------------------------------------------------------------------------------- sweeps (cold L2)
+def sweep_case(torch, B, ro, algo: str, use_truncs: bool, hbm_peak: float, l2_bytes: int, trials=5, target_bytes=None):
+    """Device time per call with a cold L2: the calls of one batch rotate over R distinct copies of
+    all inputs and outputs whose total footprint exceeds 3x the L2 capacity."""
+    keys = {"gae": ("rewards", "values"), "vtrace": ("rewards", "values", "log_rhos"),
+            "discounted_return": ("rewards",)}[algo]
+    base = {k: torch.from_numpy(getattr(ro, k)).cuda() for k in keys + ("dones", "bootstrap")}
+    if use_truncs:
+        base["truncs"] = torch.from_numpy(ro.truncs).cuda()
+        base["trunc_bootstrap"] = torch.from_numpy(ro.trunc_bootstrap).cuda()
+    n_out = 1 if algo == "discounted_return" else 2
+    set_bytes = sum(t.numel() * t.element_size() for t in base.values()) + n_out * 4 * ro.N * ro.T
+    R = int(min(512, max(4, -(-3 * l2_bytes // set_bytes))))
+    sets = [{k: v.clone() for k, v in base.items()} for _ in range(R)]
+    outs = [[torch.empty((ro.N, ro.T), dtype=torch.float32, device="cuda") for _ in range(n_out)] for _ in range(R)]
+    ws = B.Workspace(ro.N, ro.T)
+    p = ro.params
+
+    def call(i):
+        s, o = sets[i], outs[i]
+        tr, bv = (s["truncs"], s["trunc_bootstrap"]) if use_truncs else (None, None)
+        if algo == "gae":
+            B.rlcs_gae(s["rewards"], s["values"], s["dones"], tr, bv, s["bootstrap"], gamma=p["gamma"], lam=p["lam"],
+                       advantages=o[0], returns=o[1], workspace=ws)
+        elif algo == "vtrace":
+            B.rlcs_vtrace(s["rewards"], s["values"], s["log_rhos"], s["dones"], tr, bv, s["bootstrap"], gamma=p["gamma"],
+                          vs=o[0], pg_advantages=o[1], workspace=ws)
+        else:
+            B.rlcs_discounted_return(s["rewards"], s["dones"], tr, bv, s["bootstrap"], gamma=p["gamma"], returns=o[0],
+                                     workspace=ws)
+
+    for i in range(R):
+        call(i)
+    per_call_us = []
+    for _ in range(trials):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        for i in range(R):
+            call(i)
+        e1.record()
+        torch.cuda.synchronize()
+        per_call_us.append(1e3 * e0.elapsed_time(e1) / R)
+    ro_eff = ro if use_truncs else _without_truncs(ro)
+    algo_bytes = algorithmic_bytes(ro_eff, algo)
+    best = min(per_call_us)
+    gbs = algo_bytes / (best * 1e-6) / 1e9
+    return {"algo": algo, "N": ro.N, "T": ro.T, "truncs": use_truncs, "us_per_call": round(best, 3),
+            "us_per_call_median": round(statistics.median(per_call_us), 3), "env_steps_per_s": ro.N * ro.T / (best * 1e-6),
+            "algorithmic_bytes": algo_bytes, "gbs": round(gbs, 1), "frac_of_peak": round(gbs / hbm_peak, 4),
+            "rotating_sets": R, "l2": "cold (rotating buffer sets > 3x L2)"}
+
+
+def _without_truncs(ro):
+    import copy
+    r2 = copy.copy(ro)
+    r2.truncs = None
+    r2.trunc_bootstrap = None
+    return r2
+
+
+def run_sweeps(torch, hbm_peak):
+    from paper_2608_17641_b200 import binding as B, workloads
+    l2 = torch.cuda.get_device_properties(0).L2_cache_size
+    out = []
+    for T in (32, 64, 128, 256, 512, 1024):
+        for tr in (False, True):
+            ro = workloads.config3(T, True)
+            for algo in ("gae", "vtrace"):
+                out.append(sweep_case(torch, B, ro, algo, tr, hbm_peak, l2))
+    ro4 = workloads.config4()
+    for algo in ("gae", "discounted_return"):
+        out.append(sweep_case(torch, B, ro4, algo, False, hbm_peak, l2))
+    return out
+
+
+# --------------------------------------------------------------------------------------------- main
+class _NoDist:
+    rank, world = 0, 1
+
+    def barrier(self):
+        pass
+
+    def max(self, x: float) -> float:
+        return x
+
+    def sum(self, x: float) -> float:
+        return x
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", choices=("ours", "reference"), default="ours")
+    ap.add_argument("--no-sweep", action="store_true", help="skip the cold-L2 sweeps of the smaller configurations")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--rows", type=int, default=WORKLOAD["N"], help="num_envs of the bench batch (default: full size)")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    if args.gpus > 1 and world == 1:
+        # not under torchrun: relaunch one rank per GPU
+        os.execvp(sys.executable, [sys.executable, "-m", "torch.distributed.run", "--nnodes=1",
+                                   f"--nproc-per-node={args.gpus}", "--master-addr", "127.0.0.1", "--master-port",
+                                   os.environ.get("MASTER_PORT", "29517"), os.path.abspath(__file__), *sys.argv[1:]])
+
+    if args.impl == "reference":
+        if rank == 0:
+            reference_arm(args, world)
+        return
+
+    import torch
+    from paper_2608_17641_b200 import binding, workloads
+    from paper_2608_17641_b200.distributed import Dist
+    binding.lib()                                   # no library, no benchmark: there is no fallback
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device"
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dist = Dist.from_env(backend="nccl", device=torch.device("cuda", local)) if world > 1 else _NoDist()
+
+    N = args.rows
+    ro = workloads.config5(N=N, T=WORKLOAD["T"], salt=rank)        # every rank draws its own batch
+    batch = GpuBatch(ro, torch.device("cuda", local))
+    total_ms, per_algo_ms, launches, clocks = time_device(batch, args.steps, args.warmup, dist)
+    total_ms = dist.max(total_ms)
+    units_per_step = len(ALGOS) * ro.N * ro.T * world
+    value = units_per_step * args.steps / (total_ms * 1e-3)
+
+    peak, peak_kind = measured_peak()
+    per_algo = {}
+    for a in ALGOS:
+        ms = statistics.mean(per_algo_ms[a])
+        ab = algorithmic_bytes(ro, a)
+        gbs = ab / (ms * 1e-3) / 1e9
+        per_algo[a] = {"ms": round(ms, 5), "env_steps_per_s": ro.N * ro.T / (ms * 1e-3), "algorithmic_bytes": ab,
+                       "gbs": round(gbs, 1), "frac_of_peak": round(gbs / peak, 4)}
+    dom = max(ALGOS, key=lambda a: per_algo[a]["ms"])
+    roofline = {"bound": "hbm", "kernel": f"scan_kernel<{dom}, truncation handling, vectorised, 256 threads x 8 steps>",
+                "achieved": per_algo[dom]["gbs"], "peak": peak, "unit": "GB/s",
+                "frac": round(per_algo[dom]["gbs"] / peak, 4), "traffic": NCU_TRAFFIC_BYTES.get(dom),
+                "algorithmic_bytes_per_launch": per_algo[dom]["algorithmic_bytes"], "peak_source": f"of {peak_kind}",
+                "all_kernels_frac": round(sum(v["algorithmic_bytes"] for v in per_algo.values())
+                                          / (sum(v["ms"] for v in per_algo.values()) * 1e-3) / 1e9 / peak, 4)}
+
+    e2e_steps = max(1, min(args.steps, 5))
+    e2e_ms, h2d, d2h = time_e2e(batch, e2e_steps, 1, dist)
+    e2e_ms = dist.max(e2e_ms)
+    e2e = {"value": units_per_step * e2e_steps / (e2e_ms * 1e-3), "unit": METRIC, "h2d_bytes_per_step": h2d,
+           "d2h_bytes_per_step": d2h, "steps": e2e_steps, "ms_per_step": e2e_ms / e2e_steps,
+           "note": "pinned host buffers -> device, seven C-ABI calls, all outputs -> pinned host, one stream"}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": METRIC, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic",
+        "config": {"workload": f"all seven algorithms, num_envs={ro.N}, T={ro.T}, fp32, dones~Bern(0.02), "
+                               f"truncs~Bern(0.005) with per-step truncation handling, gamma=0.99, lambda=0.95",
+                   "env_steps_per_step_per_gpu": len(ALGOS) * ro.N * ro.T, "launches_per_step": len(ALGOS),
+                   "l2": "inputs larger than L2 (2.2 GB touched per step), no flush"},
+        "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "per_algorithm": per_algo,
+    }
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        line["cpu_baseline"] = cpu_baseline(ro)
+    if rank == 0 and world == 1 and not args.no_sweep:
+        del batch
+        torch.cuda.empty_cache()
+        line["sweeps"] = run_sweeps(torch, peak)
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.close()
+
+
+if __name__ == "__main__":
+    main()

@@ -62,6 +62,15 @@ int finish_params(ScanParams& p, int64_t total, int64_t T, void* workspace, size
     p.T = (unsigned)T;
     p.num_tiles = (total + tile - 1) / tile;
     p.idx32 = (total + tile) <= 0xffffffffLL;
+    {   // invariant division by T (see FastDiv)
+        int l = 0;
+        while ((int64_t(1) << l) < T) ++l;
+        p.div_T.mul = (unsigned)((((uint64_t(1) << 32) * ((uint64_t(1) << l) - (uint64_t)T)) / (uint64_t)T) + 1);
+        p.div_T.sh1 = l < 1 ? l : 1;
+        p.div_T.sh2 = l > 1 ? l - 1 : 0;
+    }
+    p.decay_pow = 1.f;                       // beta product of a chunk without resets
+    for (int i = 0; i < rlcs::kVariants[g_variant].items; ++i) p.decay_pow *= p.decay;
     p.carry_mode = (tile % T) != 0;          // T does not divide the tile: rows straddle tiles
     p.header = nullptr;
     p.records = nullptr;
@@ -205,7 +214,7 @@ int rlcs_retrace(const float* rewards, const float* q_sa, const float* expected_
     if (st != RLCS_OK || total == 0) return st;
     if (!rewards || !q_sa || !expected_q || !log_rhos || !q_targets) return RLCS_ERR_NULL;
     p.f0 = rewards; p.f1 = q_sa; p.f2 = expected_q; p.f3 = log_rhos; p.out0 = q_targets;
-    p.gamma = gamma; p.aux = lambda; p.c_bar = c_bar;
+    p.gamma = gamma; p.aux = gamma * lambda; p.c_bar = c_bar;
     st = finish_params(p, total, T, workspace, workspace_bytes);
     if (st != RLCS_OK) return st;
     return run(rlcs::launch_retrace, p, truncs != nullptr, vec, cuda_stream);

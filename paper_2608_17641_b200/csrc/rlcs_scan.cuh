@@ -15,6 +15,12 @@
 //      (returns = A + V, V-Trace targets and advantages, Retrace targets) and stores once.
 // Backward algorithms scan from high addresses to low ones; thread block s handles tile
 // num_tiles-1-s, so that a block only ever waits on blocks with a smaller block index.
+//
+// The kernel is bound by HBM traffic and, next, by integer/select issue slots, so the per-step
+// code is branch-free: flags stay packed as mask bytes (4 steps per 32-bit word), a reset is a
+// beta of exactly 0 (0 * finite = 0 severs exactly), and the rare cases -- a row edge inside a
+// thread's chunk, the ragged last chunk, rows shorter than a chunk -- patch the packed words in
+// short side paths.
 #pragma once
 
 #include <cuda_runtime.h>
@@ -29,11 +35,18 @@ enum Algo : int {
 
 __host__ __device__ constexpr bool is_forward(int a) { return a == kElig || a == kPrefix || a == kAffineFwd; }
 __host__ __device__ constexpr bool has_values(int a) { return a == kGae || a == kTdLambda || a == kVtrace; }
-__host__ __device__ constexpr bool const_decay(int a) { return a != kVtrace && a != kRetrace && a != kAffineBwd && a != kAffineFwd; }
+__host__ __device__ constexpr bool is_affine(int a) { return a == kAffineBwd || a == kAffineFwd; }
+__host__ __device__ constexpr bool const_decay(int a) { return a != kVtrace && a != kRetrace && !is_affine(a); }
 
 constexpr unsigned kDeviceTimeout = 7;   // RLCS_ERR_TIMEOUT
 constexpr int kHeaderWords = 64;         // workspace header: 256 bytes
 // header[0] = call counter (epoch), header[1] = finished-block counter, header[2] = status word
+
+// Division of a 32-bit index by the invariant row length T (Granlund-Montgomery, round-up form):
+// q = (hi + ((n - hi) >> sh1)) >> sh2 with hi = umulhi(mul, n).  Exact for every n < 2^32, T >= 1.
+struct FastDiv {
+    unsigned mul, sh1, sh2;
+};
 
 struct ScanParams {
     const float* f0;          // rewards | x | alpha
@@ -50,9 +63,11 @@ struct ScanParams {
     long long num_tiles;
     unsigned T;
     int idx32;                // total + tile fits in 32 bits: 32-bit row/time arithmetic
+    FastDiv div_T;
     float gamma;
     float decay;              // gamma*lambda | gamma | 1
-    float aux;                // TD(lambda): gamma*(1-lambda); Retrace: lambda
+    float decay_pow;          // decay^ITEMS: the beta product of a chunk without resets
+    float aux;                // TD(lambda): gamma*(1-lambda); Retrace: gamma*lambda
     float rho_bar, c_bar;
     int starts_at;
     int carry_mode;           // rows may straddle tiles: publish aggregates, look back
@@ -65,21 +80,15 @@ struct ScanParams {
 struct Pair { float a, b; };
 
 // `x` covers steps that come later in scan order than everything in `acc`:
-// result = x (+) acc = (x.a + x.b*acc.a, x.b*acc.b)  (Eq. 2).  A zero beta selects x.a outright,
-// so nothing from beyond a reset is ever touched.
+// result = x (+) acc = (x.a + x.b*acc.a, x.b*acc.b)  (Eq. 2).
 __device__ __forceinline__ Pair apply(Pair x, Pair acc) {
     Pair r;
-    r.a = (x.b != 0.f) ? fmaf(x.b, acc.a, x.a) : x.a;
+    r.a = fmaf(x.b, acc.a, x.a);
     r.b = x.b * acc.b;
     return r;
 }
 
-__device__ __forceinline__ unsigned nonzero_bytes_to_bits(unsigned w) {
-    // bit k of the result = (byte k of w != 0)
-    unsigned nz = ((((w & 0x7f7f7f7fu) + 0x7f7f7f7fu) | w) >> 7) & 0x01010101u;
-    return ((nz * 0x00204081u) >> 21) & 0xfu;
-}
-
+// ------------------------------------------------------------------------------------------ loads / stores
 template <int ITEMS, bool VEC>
 __device__ __forceinline__ void load_f32(const float* __restrict__ p, long long i0, int nvalid, float (&x)[ITEMS]) {
     if (VEC && nvalid == ITEMS) {
@@ -95,27 +104,28 @@ __device__ __forceinline__ void load_f32(const float* __restrict__ p, long long 
     }
 }
 
+// Mask bytes of ITEMS consecutive steps, packed 4 per word (byte j%4 of word j/4), values as stored
+// (any non-zero byte = true).
 template <int ITEMS, bool VEC>
-__device__ __forceinline__ unsigned load_mask(const uint8_t* __restrict__ p, long long i0, int nvalid) {
-    unsigned m = 0;
+__device__ __forceinline__ void load_mask(const uint8_t* __restrict__ p, long long i0, int nvalid, unsigned (&w)[ITEMS / 4]) {
     if (VEC && nvalid == ITEMS) {
         if constexpr (ITEMS == 4) {
-            m = nonzero_bytes_to_bits(__ldcs(reinterpret_cast<const unsigned*>(p + i0)));
+            w[0] = __ldcs(reinterpret_cast<const unsigned*>(p + i0));
         } else if constexpr (ITEMS == 8) {
             uint2 v = __ldcs(reinterpret_cast<const uint2*>(p + i0));
-            m = nonzero_bytes_to_bits(v.x) | (nonzero_bytes_to_bits(v.y) << 4);
+            w[0] = v.x; w[1] = v.y;
         } else {
             static_assert(ITEMS == 16, "ITEMS must be 4, 8 or 16");
             uint4 v = __ldcs(reinterpret_cast<const uint4*>(p + i0));
-            m = nonzero_bytes_to_bits(v.x) | (nonzero_bytes_to_bits(v.y) << 4) |
-                (nonzero_bytes_to_bits(v.z) << 8) | (nonzero_bytes_to_bits(v.w) << 12);
+            w[0] = v.x; w[1] = v.y; w[2] = v.z; w[3] = v.w;
         }
     } else {
 #pragma unroll
+        for (int k = 0; k < ITEMS / 4; ++k) w[k] = 0;
+#pragma unroll
         for (int j = 0; j < ITEMS; ++j)
-            if (j < nvalid && __ldcs(p + i0 + j) != 0) m |= 1u << j;
+            if (j < nvalid) w[j / 4] |= (unsigned)__ldcs(p + i0 + j) << (8 * (j % 4));
     }
-    return m;
 }
 
 template <int ITEMS, bool VEC>
@@ -132,6 +142,27 @@ __device__ __forceinline__ void store_f32(float* __restrict__ p, long long i0, i
     }
 }
 
+// ------------------------------------------------------------------------------------------ packed mask bytes
+__device__ __forceinline__ constexpr unsigned byte_mask(int j) { return 0xffu << (8 * (j % 4)); }
+
+template <int W>
+__device__ __forceinline__ bool test_byte(const unsigned (&w)[W], int j) {      // j is a compile-time constant after unrolling
+    return (w[j / 4] & byte_mask(j)) != 0;
+}
+template <int W>
+__device__ __forceinline__ void mark_byte_dyn(unsigned (&w)[W], unsigned j) {   // j known only at run time
+#pragma unroll
+    for (int k = 0; k < W; ++k) w[k] |= ((j >> 2) == (unsigned)k) ? (0xffu << ((j & 3u) * 8u)) : 0u;
+}
+template <int W>
+__device__ __forceinline__ bool test_byte_dyn(const unsigned (&w)[W], unsigned j) {
+    unsigned v = 0;
+#pragma unroll
+    for (int k = 0; k < W; ++k) v |= ((j >> 2) == (unsigned)k) ? w[k] : 0u;
+    return ((v >> ((j & 3u) * 8u)) & 0xffu) != 0;
+}
+
+// ------------------------------------------------------------------------------------------ tile records
 __device__ __forceinline__ uint4 ld_volatile_u4(const uint4* p) {
     uint4 v;
     asm volatile("ld.volatile.global.v4.u32 {%0,%1,%2,%3}, [%4];"
@@ -155,8 +186,8 @@ __device__ __forceinline__ unsigned ld_volatile_u32(const unsigned* p) {
 // timing.  One warp runs this; each lane polls one predecessor.  Each 16-byte record carries the
 // call's epoch next to each 4-byte payload word, so an 8-byte half is self-validating and no
 // fence is needed.  The wait is bounded: after `cap` polls the status word is set and 0 returned.
-__device__ __forceinline__ float lookback(const uint4* __restrict__ records, unsigned epoch, long long s,
-                                          unsigned cap, unsigned* status, int lane) {
+static __device__ __noinline__ float lookback(const uint4* __restrict__ records, unsigned epoch, long long s,
+                                       unsigned cap, unsigned* status, int lane) {
     Pair acc = {0.f, 1.f};
     long long base = s - 1;
     unsigned polls = 0;
@@ -183,14 +214,15 @@ __device__ __forceinline__ float lookback(const uint4* __restrict__ records, uns
             __nanosleep(32);
             continue;
         }
-        // fold lanes 0..min(z,31) in lane order (lane 0 = nearest tile)
+        // fold lanes 0..min(z,31) in lane order (lane 0 = nearest tile); a terminator's alpha is
+        // taken as is, nothing beyond it is touched
         Pair cur = (lane <= z) ? p : Pair{0.f, 1.f};
 #pragma unroll
         for (int d = 1; d < 32; d <<= 1) {
             Pair o;
             o.a = __shfl_down_sync(0xffffffffu, cur.a, d);
             o.b = __shfl_down_sync(0xffffffffu, cur.b, d);
-            if (lane + d < 32) cur = apply(cur, o);
+            if (lane + d < 32 && cur.b != 0.f) cur = apply(cur, o);
         }
         Pair w;
         w.a = __shfl_sync(0xffffffffu, cur.a, 0);
@@ -201,10 +233,12 @@ __device__ __forceinline__ float lookback(const uint4* __restrict__ records, uns
     }
 }
 
+// ------------------------------------------------------------------------------------------ the kernel
 template <int ALGO, bool TRUNC, bool VEC, int THREADS, int ITEMS, int MIN_BLOCKS>
 __global__ void __launch_bounds__(THREADS, MIN_BLOCKS) scan_kernel(const ScanParams p) {
     constexpr bool FWD = is_forward(ALGO);
     constexpr int NW = THREADS / 32;
+    constexpr int W = ITEMS / 4;
     constexpr int TILE = THREADS * ITEMS;
     constexpr unsigned FULL = 0xffffffffu;
     static_assert(NW <= 32 && ITEMS % 4 == 0, "bad tile shape");
@@ -226,19 +260,22 @@ __global__ void __launch_bounds__(THREADS, MIN_BLOCKS) scan_kernel(const ScanPar
     long long n0;
     unsigned t0;
     if (p.idx32) {
-        const unsigned q = (unsigned)i0 / p.T;
+        const unsigned n = (unsigned)i0;
+        const unsigned hi = __umulhi(p.div_T.mul, n);
+        const unsigned q = (hi + ((n - hi) >> p.div_T.sh1)) >> p.div_T.sh2;
         n0 = q;
-        t0 = (unsigned)i0 - q * p.T;
+        t0 = n - q * p.T;
     } else {
         n0 = i0 / (long long)p.T;
         t0 = (unsigned)(i0 - n0 * (long long)p.T);
     }
-    const unsigned Tm1 = p.T - 1;
 
     // ------------------------------------------------------------------ 1. loads (all issued up front)
-    unsigned dmask = 0, tmask = 0;
-    if constexpr (ALGO != kAffineBwd && ALGO != kAffineFwd) dmask = load_mask<ITEMS, VEC>(p.dones, i0, nvalid);
-    if constexpr (TRUNC) tmask = load_mask<ITEMS, VEC>(p.truncs, i0, nvalid);
+    unsigned dw[W], tw[W];
+#pragma unroll
+    for (int k = 0; k < W; ++k) { dw[k] = 0; tw[k] = 0; }
+    if constexpr (!is_affine(ALGO)) load_mask<ITEMS, VEC>(p.dones, i0, nvalid, dw);
+    if constexpr (TRUNC) load_mask<ITEMS, VEC>(p.truncs, i0, nvalid, tw);
 
     float alpha[ITEMS];            // rewards | x | alpha, then alpha_t, then the first output
     load_f32<ITEMS, VEC>(p.f0, i0, nvalid, alpha);
@@ -249,34 +286,89 @@ __global__ void __launch_bounds__(THREADS, MIN_BLOCKS) scan_kernel(const ScanPar
     float x3[ITEMS];               // log_rhos
     if constexpr (ALGO == kVtrace || ALGO == kRetrace) load_f32<ITEMS, VEC>(p.f3, i0, nvalid, x3);
 
-    // one-step halo beyond the thread's chunk, in time direction of the dependency
+    // one-step halo beyond the thread's chunk, in the direction of the dependency
     float halo = 0.f, halo_lr = 0.f;
     unsigned halo_d = 0;
     if constexpr (!FWD && (has_values(ALGO) || ALGO == kRetrace)) {
         const float* src = (ALGO == kRetrace) ? p.f2 : p.f1;
-        const bool edge = (lane == 31) && (rem > ITEMS);
-        if (edge) halo = __ldg(src + i0 + ITEMS);
-        if constexpr (ALGO == kRetrace) if (edge) halo_lr = __ldg(p.f3 + i0 + ITEMS);
+        const bool edge_lane = (lane == 31) && (rem > ITEMS);
+        if (edge_lane) halo = __ldg(src + i0 + ITEMS);
+        if constexpr (ALGO == kRetrace) if (edge_lane) halo_lr = __ldg(p.f3 + i0 + ITEMS);
     }
     if constexpr (ALGO == kElig || ALGO == kPrefix) {
-        if (lane == 0 && i0 > 0 && rem > 0) halo_d = (__ldg(p.dones + i0 - 1) != 0);
+        if (lane == 0 && i0 > 0 && rem > 0) halo_d = __ldg(p.dones + i0 - 1);
     }
 
-    // window-edge bootstrap of the first row edge inside the chunk (later edges only when T < ITEMS)
+    // Row edge inside the chunk.  Backward: the row's last step, at chunk offset T-1-t0; its
+    // window-edge bootstrap is fetched now.  Forward: the next row's first step, at offset T-t0
+    // (offset 0 when the chunk itself starts a row).
+    const unsigned edge = FWD ? (t0 == 0 ? 0u : p.T - t0) : (p.T - 1 - t0);
+    const bool has_edge = edge < (unsigned)ITEMS;
     float boot_first = 0.f;
-    const unsigned to_edge = Tm1 - t0;           // steps from the chunk start to its row's last step
-    if constexpr (!FWD && ALGO != kAffineBwd) {
-        if (p.boot != nullptr && to_edge < (unsigned)nvalid) boot_first = __ldg(p.boot + n0);
+    if constexpr (!FWD && !is_affine(ALGO)) {
+        if (p.boot != nullptr && edge < (unsigned)nvalid) boot_first = __ldg(p.boot + n0);
     }
 
-    // ------------------------------------------------------------------ 2. flags, sparse truncation values
-    if constexpr (TRUNC) {
-        tmask &= ~dmask;           // termination wins: trunc_bootstrap is not read there
-    }
-    float bv[ITEMS];
-    if constexpr (TRUNC) {
+    // ------------------------------------------------------------------ 2. reset words
+    // sev: byte j non-zero = the recurrence does NOT continue from step j to its scan-order
+    // predecessor (t+1 backward, t-1 forward): a flag, a row edge, or a step beyond the array.
+    unsigned sev[W];
+    if constexpr (FWD) {
+        if constexpr (ALGO == kAffineFwd) {
 #pragma unroll
-        for (int j = 0; j < ITEMS; ++j) bv[j] = ((tmask >> j) & 1u) ? __ldg(p.trunc_boot + i0 + j) : 0.f;
+            for (int k = 0; k < W; ++k) sev[k] = 0;
+        } else {
+            // ends_at: step j is cut off by the flag of step j-1 -> shift the bytes up by one step
+            const unsigned nb = __shfl_up_sync(FULL, dw[W - 1] >> 24, 1);
+            if (lane != 0) halo_d = nb;
+            if (ALGO == kPrefix && p.starts_at) {
+#pragma unroll
+                for (int k = 0; k < W; ++k) sev[k] = dw[k];
+            } else {
+#pragma unroll
+                for (int k = 0; k < W; ++k) sev[k] = (dw[k] << 8) | (k == 0 ? (halo_d & 0xffu) : (dw[(k + W - 1) % W] >> 24));
+            }
+        }
+    } else {
+#pragma unroll
+        for (int k = 0; k < W; ++k) sev[k] = dw[k] | tw[k];
+    }
+    if (has_edge) mark_byte_dyn(sev, edge);
+    if (p.T < (unsigned)ITEMS) {                // rows shorter than a chunk: several edges
+        for (unsigned e = edge + p.T; e < (unsigned)ITEMS; e += p.T) mark_byte_dyn(sev, e);
+    }
+    if (nvalid < ITEMS) {                       // ragged end of the array
+        for (unsigned j = nvalid; j < (unsigned)ITEMS; ++j) mark_byte_dyn(sev, j);
+    }
+
+    // ------------------------------------------------------------------ 3. successor values at resets
+    // ov[j]: successor value used where the recurrence is severed -- 0 after a termination, the
+    // supplied continuation value after a truncation, the window-edge bootstrap at a row's last
+    // step (Section 3.2).  Zero wherever the recurrence continues.
+    float ov[ITEMS];
+#pragma unroll
+    for (int j = 0; j < ITEMS; ++j) ov[j] = 0.f;
+    if constexpr (!FWD && !is_affine(ALGO)) {
+        if constexpr (TRUNC) {
+#pragma unroll
+            for (int j = 0; j < ITEMS; ++j)
+                if (test_byte(tw, j) && !test_byte(dw, j)) ov[j] = __ldg(p.trunc_boot + i0 + j);
+        }
+        if (has_edge && p.boot != nullptr) {
+            unsigned e = edge;
+            long long n = n0;
+            float b = boot_first;
+            for (;;) {
+                if (e < (unsigned)nvalid && !test_byte_dyn(dw, e) && !test_byte_dyn(tw, e)) {
+#pragma unroll
+                    for (int j = 0; j < ITEMS; ++j) if ((unsigned)j == e) ov[j] = b;
+                }
+                e += p.T;
+                ++n;
+                if (e >= (unsigned)nvalid) break;          // only when T < ITEMS
+                b = __ldg(p.boot + n);
+            }
+        }
     }
 
     // neighbour values through the warp
@@ -289,106 +381,72 @@ __global__ void __launch_bounds__(THREADS, MIN_BLOCKS) scan_kernel(const ScanPar
             if (lane != 31) halo_lr = nl;
         }
     }
-    if constexpr (ALGO == kElig || (ALGO == kPrefix)) {
-        const unsigned nb = __shfl_up_sync(FULL, (dmask >> (ITEMS - 1)) & 1u, 1);
-        if (lane != 0) halo_d = nb;
-    }
 
-    // ------------------------------------------------------------------ 3. coefficients
-    // contmask bit j: the recurrence continues from step j into its scan-order predecessor
-    // (t+1 for backward scans, t-1 for forward scans).
-    unsigned contmask = 0;
-    float beta[ITEMS];             // only for algorithms with a per-step decay
-    float grho[ITEMS];             // V-Trace: gamma*rho_t for the advantage epilogue
-    {
-        unsigned t = t0;
-        long long n = n0;
+    // ------------------------------------------------------------------ 4. coefficients (branch-free)
+    float beta[ITEMS];
+    float grho[ITEMS];             // V-Trace: cont * gamma * rho_t, for the advantage epilogue
 #pragma unroll
-        for (int j = 0; j < ITEMS; ++j) {
-            const bool valid = j < nvalid;
-            if constexpr (FWD) {
-                const bool first = (t == 0);
-                bool cont;
-                if constexpr (ALGO == kAffineFwd) {
-                    cont = !first;
-                    beta[j] = (cont && valid) ? x1[j] : 0.f;
-                } else {
-                    const unsigned dprev = (j == 0) ? halo_d : ((dmask >> (j - 1)) & 1u);
-                    const unsigned dsel = (ALGO == kPrefix && p.starts_at) ? ((dmask >> j) & 1u) : dprev;
-                    cont = !first && !dsel;
-                }
-                if (cont && valid) contmask |= 1u << j;
-            } else {
-                const bool last = (t == Tm1);
-                const bool term = (dmask >> j) & 1u;
-                const bool trunc = TRUNC ? ((tmask >> j) & 1u) : false;
-                const bool cont = valid && !term && !trunc && !last;
-                if (cont) contmask |= 1u << j;
-                if constexpr (ALGO == kAffineBwd) {
-                    beta[j] = cont ? x1[j] : 0.f;
-                } else {
-                    float bootv = 0.f;
-                    if (last && p.boot != nullptr && valid) bootv = ((unsigned)j == to_edge) ? boot_first : __ldg(p.boot + n);
-                    // successor value of Section 3.2
-                    float nextv = 0.f;
-                    if constexpr (has_values(ALGO)) nextv = (j + 1 < ITEMS) ? x1[(j + 1) % ITEMS] : halo;
-                    if constexpr (ALGO == kRetrace) nextv = (j + 1 < ITEMS) ? x2[(j + 1) % ITEMS] : halo;
-                    float xn = last ? bootv : nextv;
-                    if constexpr (TRUNC) xn = trunc ? bv[j] : xn;
-                    xn = term ? 0.f : xn;
-                    const float r = alpha[j];
-                    if constexpr (ALGO == kGae) {
-                        alpha[j] = fmaf(p.gamma, xn, r) - x1[j];
-                    } else if constexpr (ALGO == kTdLambda) {
-                        alpha[j] = fmaf(cont ? p.aux : p.gamma, xn, r);
-                    } else if constexpr (ALGO == kDisc) {
-                        alpha[j] = cont ? r : fmaf(p.gamma, xn, r);
-                    } else if constexpr (ALGO == kVtrace) {
-                        const float raw = expf(x3[j]);
-                        const float rho = fminf(p.rho_bar, raw);
-                        const float c = fminf(p.c_bar, raw);
-                        alpha[j] = rho * (fmaf(p.gamma, xn, r) - x1[j]);
-                        beta[j] = cont ? p.gamma * c : 0.f;
-                        grho[j] = p.gamma * rho;
-                    } else if constexpr (ALGO == kRetrace) {
-                        alpha[j] = fmaf(p.gamma, xn, r) - x1[j];
-                        const float lr_next = (j + 1 < ITEMS) ? x3[(j + 1) % ITEMS] : halo_lr;
-                        beta[j] = cont ? p.gamma * (p.aux * fminf(p.c_bar, expf(lr_next))) : 0.f;
-                    }
-                    if (!valid) alpha[j] = 0.f;
-                }
+    for (int j = 0; j < ITEMS; ++j) {
+        const bool cut = test_byte(sev, j);
+        if constexpr (FWD) {
+            if constexpr (ALGO == kAffineFwd) beta[j] = cut ? 0.f : x1[j];
+            else beta[j] = cut ? 0.f : p.decay;
+        } else if constexpr (ALGO == kAffineBwd) {
+            beta[j] = cut ? 0.f : x1[j];
+        } else {
+            const float c = cut ? 0.f : 1.f;
+            const float r = alpha[j];
+            float nextv = 0.f;
+            if constexpr (has_values(ALGO)) nextv = (j + 1 < ITEMS) ? x1[(j + 1) % ITEMS] : halo;
+            if constexpr (ALGO == kRetrace) nextv = (j + 1 < ITEMS) ? x2[(j + 1) % ITEMS] : halo;
+            if constexpr (ALGO == kGae) {
+                alpha[j] = fmaf(p.gamma, fmaf(c, nextv, ov[j]), r) - x1[j];
+                beta[j] = cut ? 0.f : p.decay;
+            } else if constexpr (ALGO == kTdLambda) {
+                // continuing: r + gamma(1-lambda) V_{t+1}; severed: r + gamma * successor value
+                alpha[j] = fmaf(p.gamma, ov[j], fmaf(cut ? 0.f : p.aux, nextv, r));
+                beta[j] = cut ? 0.f : p.decay;
+            } else if constexpr (ALGO == kDisc) {
+                alpha[j] = fmaf(p.gamma, ov[j], r);
+                beta[j] = cut ? 0.f : p.decay;
+            } else if constexpr (ALGO == kVtrace) {
+                const float raw = expf(x3[j]);
+                const float rho = fminf(p.rho_bar, raw);
+                const float cc = fminf(p.c_bar, raw);
+                alpha[j] = rho * (fmaf(p.gamma, fmaf(c, nextv, ov[j]), r) - x1[j]);
+                beta[j] = cut ? 0.f : p.gamma * cc;
+                grho[j] = cut ? 0.f : p.gamma * rho;
+            } else if constexpr (ALGO == kRetrace) {
+                alpha[j] = fmaf(p.gamma, fmaf(c, nextv, ov[j]), r) - x1[j];
+                const float lr_next = (j + 1 < ITEMS) ? x3[(j + 1) % ITEMS] : halo_lr;
+                beta[j] = cut ? 0.f : p.aux * fminf(p.c_bar, expf(lr_next));
             }
-            if (++t == p.T) { t = 0; ++n; }
         }
     }
-    auto beta_of = [&](int j) -> float {
-        if constexpr (const_decay(ALGO)) return ((contmask >> j) & 1u) ? p.decay : 0.f;
-        else return beta[j];
-    };
 
-    // ------------------------------------------------------------------ 4. thread aggregate (serial combine, Eq. 2)
+    // ------------------------------------------------------------------ 5. thread aggregate (serial combine, Eq. 2)
     Pair agg;
     if constexpr (FWD) {
         agg.a = alpha[0];
-        agg.b = beta_of(0);
 #pragma unroll
-        for (int j = 1; j < ITEMS; ++j) {
-            const float b = beta_of(j);
-            agg.a = (b != 0.f) ? fmaf(b, agg.a, alpha[j]) : alpha[j];
-            agg.b *= b;
-        }
+        for (int j = 1; j < ITEMS; ++j) agg.a = fmaf(beta[j], agg.a, alpha[j]);
     } else {
         agg.a = alpha[ITEMS - 1];
-        agg.b = beta_of(ITEMS - 1);
 #pragma unroll
-        for (int j = ITEMS - 2; j >= 0; --j) {
-            const float b = beta_of(j);
-            agg.a = (b != 0.f) ? fmaf(b, agg.a, alpha[j]) : alpha[j];
-            agg.b *= b;
-        }
+        for (int j = ITEMS - 2; j >= 0; --j) agg.a = fmaf(beta[j], agg.a, alpha[j]);
+    }
+    if constexpr (const_decay(ALGO)) {
+        unsigned any = 0;
+#pragma unroll
+        for (int k = 0; k < W; ++k) any |= sev[k];
+        agg.b = any ? 0.f : p.decay_pow;
+    } else {
+        agg.b = beta[0];
+#pragma unroll
+        for (int j = 1; j < ITEMS; ++j) agg.b *= beta[j];
     }
 
-    // ------------------------------------------------------------------ 5. warp scan in scan order
+    // ------------------------------------------------------------------ 6. warp scan in scan order
     // rank = position in scan order inside the warp: lane for forward scans, 31 - lane for backward.
     const int rank = FWD ? lane : 31 - lane;
     Pair incl = agg;
@@ -414,13 +472,12 @@ __global__ void __launch_bounds__(THREADS, MIN_BLOCKS) scan_kernel(const ScanPar
     }
     if (rank == 0) excl = Pair{0.f, 1.f};
 
-    // ------------------------------------------------------------------ 6. block carry through shared memory
+    // ------------------------------------------------------------------ 7. block carry through shared memory
     const int wrank = FWD ? warp : NW - 1 - warp;
     if (rank == 31) s_agg[wrank] = incl;
     if (wrank == 0 && rank == 0) {
         // the tile's first step in scan order: does the recurrence enter the tile from outside?
-        const int jfirst = FWD ? 0 : ITEMS - 1;
-        s_need = (int)((contmask >> jfirst) & 1u);
+        s_need = test_byte(sev, FWD ? 0 : ITEMS - 1) ? 0 : 1;
     }
     __syncthreads();
 
@@ -443,7 +500,7 @@ __global__ void __launch_bounds__(THREADS, MIN_BLOCKS) scan_kernel(const ScanPar
     }
     const Pair before = apply(excl, wcarry);   // everything earlier in scan order inside this tile
 
-    // ------------------------------------------------------------------ 7. carry between thread blocks
+    // ------------------------------------------------------------------ 8. carry between thread blocks
     float carry_in = 0.f;
     if (p.carry_mode) {
         unsigned epoch = 0;
@@ -465,29 +522,27 @@ __global__ void __launch_bounds__(THREADS, MIN_BLOCKS) scan_kernel(const ScanPar
         }
     }
     // value of the recurrence at the step just before this thread's chunk in scan order
-    float prev = (before.b != 0.f) ? fmaf(before.b, carry_in, before.a) : before.a;
+    float prev = fmaf(before.b, carry_in, before.a);
 
-    // ------------------------------------------------------------------ 8. replay, epilogue, store
+    // ------------------------------------------------------------------ 9. replay, epilogue, store
     float out1v[ITEMS];
     if constexpr (FWD) {
 #pragma unroll
         for (int j = 0; j < ITEMS; ++j) {
-            const float b = beta_of(j);
-            prev = (b != 0.f) ? fmaf(b, prev, alpha[j]) : alpha[j];
+            prev = fmaf(beta[j], prev, alpha[j]);
             alpha[j] = prev;
         }
     } else {
 #pragma unroll
         for (int j = ITEMS - 1; j >= 0; --j) {
-            const float b = beta_of(j);
-            const float d = (b != 0.f) ? fmaf(b, prev, alpha[j]) : alpha[j];
+            const float d = fmaf(beta[j], prev, alpha[j]);
             if constexpr (ALGO == kGae) {
                 alpha[j] = d;
                 out1v[j] = d + x1[j];
             } else if constexpr (ALGO == kVtrace) {
                 // A_t = rho_t (r_t + gamma v_{t+1} - V_t) = alpha_t + gamma rho_t Delta_{t+1} where the
                 // recurrence continues (v_{t+1} = V_{t+1} + Delta_{t+1}), alpha_t elsewhere.
-                out1v[j] = ((contmask >> j) & 1u) ? fmaf(grho[j], prev, alpha[j]) : alpha[j];
+                out1v[j] = fmaf(grho[j], prev, alpha[j]);
                 alpha[j] = x1[j] + d;
             } else if constexpr (ALGO == kRetrace) {
                 alpha[j] = x1[j] + d;
@@ -504,7 +559,7 @@ __global__ void __launch_bounds__(THREADS, MIN_BLOCKS) scan_kernel(const ScanPar
         }
     }
 
-    // ------------------------------------------------------------------ 9. close the call (carry mode)
+    // ------------------------------------------------------------------ 10. close the call (carry mode)
     // The last block to finish advances the epoch, so the records of this call can never be taken
     // for those of the next one and no per-call clearing is needed.
     if (p.carry_mode && tid == 0) {
