@@ -343,7 +343,23 @@ def sweep_case(torch, B, ro, algo: str, use_truncs: bool, hbm_peak: float, l2_by
 
     for i in range(R):
         call(i)
-    per_call_us = []
+    torch.cuda.synchronize()
+    # device time: the R launches replayed from a CUDA graph (no host launch cost between kernels)
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        for i in range(R):
+            call(i)
+    graph.replay()
+    per_call_us, full_call_us = [], []
+    for _ in range(trials):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        graph.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        per_call_us.append(1e3 * e0.elapsed_time(e1) / R)
+    # full call: the same launches issued one by one through the Python binding
     for _ in range(trials):
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         torch.cuda.synchronize()
@@ -352,15 +368,16 @@ def sweep_case(torch, B, ro, algo: str, use_truncs: bool, hbm_peak: float, l2_by
             call(i)
         e1.record()
         torch.cuda.synchronize()
-        per_call_us.append(1e3 * e0.elapsed_time(e1) / R)
+        full_call_us.append(1e3 * e0.elapsed_time(e1) / R)
     ro_eff = ro if use_truncs else _without_truncs(ro)
     algo_bytes = algorithmic_bytes(ro_eff, algo)
     best = min(per_call_us)
     gbs = algo_bytes / (best * 1e-6) / 1e9
     return {"algo": algo, "N": ro.N, "T": ro.T, "truncs": use_truncs, "us_per_call": round(best, 3),
-            "us_per_call_median": round(statistics.median(per_call_us), 3), "env_steps_per_s": ro.N * ro.T / (best * 1e-6),
+            "us_per_call_median": round(statistics.median(per_call_us), 3),
+            "full_call_us": round(min(full_call_us), 3), "env_steps_per_s": ro.N * ro.T / (best * 1e-6),
             "algorithmic_bytes": algo_bytes, "gbs": round(gbs, 1), "frac_of_peak": round(gbs / hbm_peak, 4),
-            "rotating_sets": R, "l2": "cold (rotating buffer sets > 3x L2)"}
+            "rotating_sets": R, "l2": "cold (rotating buffer sets > 3x L2)", "timing": "CUDA-graph replay of the rotating launches"}
 
 
 def _without_truncs(ro):
@@ -408,6 +425,8 @@ def main():
     ap.add_argument("--impl", choices=("ours", "reference"), default="ours")
     ap.add_argument("--no-sweep", action="store_true", help="skip the cold-L2 sweeps of the smaller configurations")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sweep-only", action="store_true", help="print only the cold-L2 sweeps (one JSON line)")
+    ap.add_argument("--variant", type=int, default=None, help="tile variant test hook (default: library default)")
     ap.add_argument("--rows", type=int, default=WORKLOAD["N"], help="num_envs of the bench batch (default: full size)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
@@ -429,10 +448,17 @@ def main():
     from paper_2608_17641_b200 import binding, workloads
     from paper_2608_17641_b200.distributed import Dist
     binding.lib()                                   # no library, no benchmark: there is no fallback
+    if args.variant is not None:
+        binding.rlcs_debug_set_tile_variant(args.variant)
     assert torch.cuda.is_available(), "bench.py needs a CUDA device"
     local = int(os.environ.get("LOCAL_RANK", "0"))
     torch.cuda.set_device(local)
     dist = Dist.from_env(backend="nccl", device=torch.device("cuda", local)) if world > 1 else _NoDist()
+
+    if args.sweep_only:
+        peak, _ = measured_peak()
+        print(json.dumps({"sweeps": run_sweeps(torch, peak)}), flush=True)
+        return
 
     N = args.rows
     ro = workloads.config5(N=N, T=WORKLOAD["T"], salt=rank)        # every rank draws its own batch

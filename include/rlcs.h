@@ -170,15 +170,16 @@ int rlcs_affine_scan(const float* alpha, const float* beta, float* out, int64_t 
                      void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
- * Test hook: choose the kernels' tile shape for subsequent calls in this process (not thread-safe).
- * variant 0 = default.  Other variants change threads per block / steps per thread, hence where
- * tiles and warps cut the rows; results must agree across variants to rounding and exactly at
- * severed steps.  Returns RLCS_ERR_ARG for an unknown variant.  rlcs_workspace_bytes is an upper
- * bound over all variants.
+ * Test hook: choose the kernel and tile shape for subsequent calls in this process (not
+ * thread-safe).  variant -1 = the library default.  Other variants change the kernel (persistent
+ * blocks with a bulk-copy ring, or one tile per block), threads per block and steps per thread,
+ * hence where tiles and warps cut the rows; results must agree across variants to rounding, and
+ * exactly at severed steps.  Returns RLCS_ERR_ARG for an unknown variant.  rlcs_workspace_bytes is
+ * an upper bound over all variants.
  */
 int rlcs_debug_set_tile_variant(int variant);
 
-/* Elements per tile of a variant (0 for an unknown variant). */
+/* Elements per tile of a variant (-1 = the default; 0 for an unknown variant). */
 int rlcs_debug_tile_elems(int variant);
 
 /*

@@ -10,7 +10,8 @@ namespace {
 
 using rlcs::ScanParams;
 
-int g_variant = 0;               // test hook: tile variant
+constexpr int kDefaultVariant = 0;
+int g_variant = kDefaultVariant; // test hook: tile variant
 long long g_mute_tile = -1;      // test hook: tile that does not publish
 long long g_spin_cap = 0;        // test hook: poll limit (0 = default)
 constexpr unsigned kDefaultSpinCap = 1u << 21;
@@ -74,6 +75,9 @@ int finish_params(ScanParams& p, int64_t total, int64_t T, void* workspace, size
     p.carry_mode = (tile % T) != 0;          // T does not divide the tile: rows straddle tiles
     p.header = nullptr;
     p.records = nullptr;
+    p.status = nullptr;
+    if (workspace != nullptr && workspace_bytes >= sizeof(unsigned) * rlcs::kHeaderWords && aligned(workspace, 16))
+        p.status = static_cast<unsigned*>(workspace) + 2;
     p.mute_tile = g_mute_tile;
     p.spin_cap = g_spin_cap > 0 ? (unsigned)g_spin_cap : kDefaultSpinCap;
     if (p.carry_mode) {
@@ -306,12 +310,13 @@ int rlcs_affine_scan(const float* alpha, const float* beta, float* out, int64_t 
 }
 
 int rlcs_debug_set_tile_variant(int variant) {
-    if (variant < 0 || variant >= rlcs::kNumVariants) return RLCS_ERR_ARG;
-    g_variant = variant;
+    if (variant < -1 || variant >= rlcs::kNumVariants) return RLCS_ERR_ARG;
+    g_variant = variant < 0 ? kDefaultVariant : variant;
     return RLCS_OK;
 }
 
 int rlcs_debug_tile_elems(int variant) {
+    if (variant == -1) variant = kDefaultVariant;
     if (variant < 0 || variant >= rlcs::kNumVariants) return 0;
     return tile_elems(variant);
 }

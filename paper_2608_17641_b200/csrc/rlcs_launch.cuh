@@ -1,39 +1,85 @@
-// Host-side dispatch from (tile variant, truncation handling, vector alignment) to one
-// instantiation of scan_kernel.  Each algorithm's translation unit instantiates its own kernels
-// through RLCS_DEFINE_LAUNCHER so that the build can compile them in parallel.
+// Host-side dispatch from (tile variant, truncation handling, pointer alignment) to one
+// instantiation of the scan kernels.  Each algorithm's translation unit instantiates its own
+// kernels through RLCS_DEFINE_LAUNCHER so that the build can compile them in parallel.
 #pragma once
 
 #include "rlcs_scan.cuh"
 
 namespace rlcs {
 
-struct TileVariant { int threads, items, min_blocks; };
-constexpr int kNumVariants = 4;
-// variant 0 is the default; the others exist for the tiling-invariance tests and for tuning.
+// stages == 0: scan_kernel (one tile per block).  stages > 0: scan_kernel_tma (persistent blocks,
+// bulk-copy ring of that many tiles; min_blocks = blocks per SM it is compiled and sized for).
+struct TileVariant { int threads, items, min_blocks, stages; };
+constexpr int kNumVariants = 14;
 constexpr TileVariant kVariants[kNumVariants] = {
-    {256, 8, 4},   // 2048 steps per tile
-    {128, 4, 8},   //  512
-    {512, 8, 2},   // 4096
-    {256, 4, 4},   // 1024
+    {256, 8, 4, 0},    //  0: 2048 steps per tile
+    {128, 4, 8, 0},    //  1:  512
+    {512, 8, 2, 0},    //  2: 4096
+    {256, 4, 4, 0},    //  3: 1024
+    {256, 16, 2, 0},   //  4: 4096
+    {128, 16, 4, 0},   //  5: 2048
+    {128, 8, 8, 0},    //  6: 1024
+    {512, 16, 1, 0},   //  7: 8192
+    {256, 8, 3, 3},    //  8: 2048, persistent, 3 stages
+    {256, 8, 2, 4},    //  9: 2048, persistent, 4 stages
+    {256, 8, 4, 2},    // 10: 2048, persistent, 2 stages
+    {128, 8, 6, 3},    // 11: 1024, persistent, 3 stages
+    {512, 8, 1, 3},    // 12: 4096, persistent, 3 stages
+    {256, 16, 2, 2},   // 13: 4096, persistent, 2 stages
 };
 constexpr int kMinTileElems = 512;
+constexpr int kMaxDevices = 64;
+
+template <int ALGO, bool TRUNC, int V>
+cudaError_t launch_persistent(const ScanParams& p, cudaStream_t stream) {
+    constexpr TileVariant tv = kVariants[V];
+    constexpr int STAGES = tv.stages > 0 ? tv.stages : 1;
+    using L = StageLayout<ALGO, TRUNC, tv.threads * tv.items>;
+    constexpr size_t kSmem = (size_t)STAGES * L::BYTES;
+    auto kernel = scan_kernel_tma<ALGO, TRUNC, tv.threads, tv.items, STAGES, tv.min_blocks>;
+    // Per-device launch configuration, found once: the grid must not exceed what is co-resident,
+    // because a block may wait for the tile record of any block with a smaller index.
+    static int s_blocks[kMaxDevices] = {};
+    int dev = 0;
+    cudaError_t err = cudaGetDevice(&dev);
+    if (err != cudaSuccess) return err;
+    if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    if (s_blocks[dev] == 0) {
+        err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmem);
+        if (err != cudaSuccess) return err;
+        int per_sm = 0, sms = 0;
+        err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, tv.threads, kSmem);
+        if (err != cudaSuccess) return err;
+        err = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        if (err != cudaSuccess) return err;
+        if (per_sm < 1 || sms < 1) return cudaErrorLaunchOutOfResources;
+        s_blocks[dev] = per_sm * sms;
+    }
+    const long long grid = p.num_tiles < s_blocks[dev] ? p.num_tiles : s_blocks[dev];
+    kernel<<<(unsigned)grid, tv.threads, kSmem, stream>>>(p);
+    return cudaGetLastError();
+}
 
 template <int ALGO, bool TRUNC, bool VEC, int V>
 cudaError_t launch_variant(const ScanParams& p, cudaStream_t stream) {
     constexpr TileVariant tv = kVariants[V];
-    scan_kernel<ALGO, TRUNC, VEC, tv.threads, tv.items, tv.min_blocks>
-        <<<(unsigned)p.num_tiles, tv.threads, 0, stream>>>(p);
-    return cudaGetLastError();
+    if constexpr (tv.stages > 0 && VEC) {
+        return launch_persistent<ALGO, TRUNC, V>(p, stream);
+    } else {
+        // bulk copies need 16-byte aligned pointers; otherwise the element-wise kernel of the same tile shape
+        scan_kernel<ALGO, TRUNC, VEC, tv.threads, tv.items, tv.min_blocks>
+            <<<(unsigned)p.num_tiles, tv.threads, 0, stream>>>(p);
+        return cudaGetLastError();
+    }
 }
 
-template <int ALGO, bool TRUNC, bool VEC>
+template <int ALGO, bool TRUNC, bool VEC, int V = 0>
 cudaError_t launch_tv(const ScanParams& p, int variant, cudaStream_t stream) {
-    switch (variant) {
-        case 0: return launch_variant<ALGO, TRUNC, VEC, 0>(p, stream);
-        case 1: return launch_variant<ALGO, TRUNC, VEC, 1>(p, stream);
-        case 2: return launch_variant<ALGO, TRUNC, VEC, 2>(p, stream);
-        case 3: return launch_variant<ALGO, TRUNC, VEC, 3>(p, stream);
-        default: return cudaErrorInvalidValue;
+    if constexpr (V >= kNumVariants) {
+        return cudaErrorInvalidValue;
+    } else {
+        if (variant == V) return launch_variant<ALGO, TRUNC, VEC, V>(p, stream);
+        return launch_tv<ALGO, TRUNC, VEC, V + 1>(p, variant, stream);
     }
 }
 

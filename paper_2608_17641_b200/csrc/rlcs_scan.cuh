@@ -1,26 +1,33 @@
 // Fused segmented affine scan over the flattened [N*T] rollout array (sm_100a).
 //
-// One kernel template serves all seven algorithms.  The row-major [N, T] tensors are treated as
-// one contiguous array of N*T steps that is cut into fixed tiles of THREADS*ITEMS steps, one
-// thread block per tile; a row edge is simply one more reset.  Per tile:
-//   1. every thread loads ITEMS consecutive steps of each input with 16-byte vector loads
-//      (masks: one ITEMS-byte load), plus a one-step halo of the successor value;
+// The row-major [N, T] tensors are treated as one contiguous array of N*T steps that is cut into
+// fixed tiles of THREADS*ITEMS steps; a row edge is simply one more reset.  Per tile a thread block
+//   1. brings ITEMS consecutive steps of each input per thread on chip, plus a one-step halo of the
+//      successor value;
 //   2. builds (alpha_t, beta_t) of Table 1 in registers, with the boundary rules of Section 3.2
 //      and the window-edge carry folded into alpha, so that every row scans with carry 0;
-//   3. folds its ITEMS pairs serially with the combine of Eq. 2, scans the per-thread aggregates
-//      with warp shuffles, and the per-warp aggregates through shared memory;
+//   3. folds each thread's ITEMS pairs serially with the combine of Eq. 2, scans the per-thread
+//      aggregates with warp shuffles, and the per-warp aggregates through shared memory;
 //   4. if the tile is entered in the middle of an episode, obtains the carry from the preceding
 //      tiles (in scan order) by a bounded, deterministic look-back over published tile aggregates;
 //   5. replays the recurrence over its ITEMS steps from the carry, applies the epilogue
 //      (returns = A + V, V-Trace targets and advantages, Retrace targets) and stores once.
-// Backward algorithms scan from high addresses to low ones; thread block s handles tile
-// num_tiles-1-s, so that a block only ever waits on blocks with a smaller block index.
+// Backward algorithms scan from high addresses to low ones: scan-order tile s is address tile
+// num_tiles-1-s, so a block only ever waits on tiles with a smaller scan-order index.
 //
-// The kernel is bound by HBM traffic and, next, by integer/select issue slots, so the per-step
-// code is branch-free: flags stay packed as mask bytes (4 steps per 32-bit word), a reset is a
-// beta of exactly 0 (0 * finite = 0 severs exactly), and the rare cases -- a row edge inside a
-// thread's chunk, the ragged last chunk, rows shorter than a chunk -- patch the packed words in
-// short side paths.
+// Two kernels share this per-tile code:
+//   scan_kernel_tma  persistent thread blocks (all co-resident); each walks tiles s, s+G, s+2G, ...
+//                    and keeps a ring of STAGES tiles in flight: one elected thread issues 1-D bulk
+//                    copies (cp.async.bulk, no multicast, no tensor map: tiles of the flat array are
+//                    contiguous) that complete on an mbarrier per stage.  Needs 16-byte aligned
+//                    pointers; the ragged last tile(s) are loaded with plain loads.
+//   scan_kernel      one tile per thread block, plain (vector or element-wise) global loads; used
+//                    for unaligned pointers and as the cross-check in the tests.
+//
+// The per-step code is branch-free: flags stay packed as mask bytes (4 steps per 32-bit word), a
+// reset is a beta of exactly 0, successor values at resets are selected (never multiplied), and
+// the rare cases -- a row edge inside a thread's chunk, the ragged last chunk, rows shorter than a
+// chunk -- patch the packed words in short side paths.
 #pragma once
 
 #include <cuda_runtime.h>
@@ -37,6 +44,12 @@ __host__ __device__ constexpr bool is_forward(int a) { return a == kElig || a ==
 __host__ __device__ constexpr bool has_values(int a) { return a == kGae || a == kTdLambda || a == kVtrace; }
 __host__ __device__ constexpr bool is_affine(int a) { return a == kAffineBwd || a == kAffineFwd; }
 __host__ __device__ constexpr bool const_decay(int a) { return a != kVtrace && a != kRetrace && !is_affine(a); }
+// a float input is read one step beyond the tile (successor value)
+__host__ __device__ constexpr bool float_halo(int a) { return has_values(a) || a == kRetrace; }
+__host__ __device__ constexpr bool uses_f1(int a) { return a != kDisc && a != kElig && a != kPrefix; }
+__host__ __device__ constexpr bool uses_f2(int a) { return a == kRetrace; }
+__host__ __device__ constexpr bool uses_f3(int a) { return a == kVtrace || a == kRetrace; }
+__host__ __device__ constexpr bool uses_dones(int a) { return !is_affine(a); }
 
 constexpr unsigned kDeviceTimeout = 7;   // RLCS_ERR_TIMEOUT
 constexpr int kHeaderWords = 64;         // workspace header: 256 bytes
@@ -71,7 +84,8 @@ struct ScanParams {
     float rho_bar, c_bar;
     int starts_at;
     int carry_mode;           // rows may straddle tiles: publish aggregates, look back
-    unsigned* header;
+    unsigned* header;         // workspace header (carry mode) or nullptr
+    unsigned* status;         // device status word, or nullptr when there is no workspace
     uint4* records;           // one 16-byte record per tile: {alpha_bits, epoch, beta_bits, epoch}
     long long mute_tile;      // test hook: this scan-order tile does not publish
     unsigned spin_cap;
@@ -88,7 +102,7 @@ __device__ __forceinline__ Pair apply(Pair x, Pair acc) {
     return r;
 }
 
-// ------------------------------------------------------------------------------------------ loads / stores
+// ------------------------------------------------------------------------------------------ global loads / stores
 template <int ITEMS, bool VEC>
 __device__ __forceinline__ void load_f32(const float* __restrict__ p, long long i0, int nvalid, float (&x)[ITEMS]) {
     if (VEC && nvalid == ITEMS) {
@@ -142,6 +156,29 @@ __device__ __forceinline__ void store_f32(float* __restrict__ p, long long i0, i
     }
 }
 
+// ------------------------------------------------------------------------------------------ shared-memory reads
+template <int ITEMS>
+__device__ __forceinline__ void lds_f32(const float* s, float (&x)[ITEMS]) {   // s is 16-byte aligned
+    const float4* q = reinterpret_cast<const float4*>(s);
+#pragma unroll
+    for (int k = 0; k < ITEMS / 4; ++k) {
+        float4 v = q[k];
+        x[4 * k + 0] = v.x; x[4 * k + 1] = v.y; x[4 * k + 2] = v.z; x[4 * k + 3] = v.w;
+    }
+}
+template <int ITEMS>
+__device__ __forceinline__ void lds_mask(const uint8_t* s, unsigned (&w)[ITEMS / 4]) {   // s is ITEMS-byte aligned
+    if constexpr (ITEMS == 4) {
+        w[0] = *reinterpret_cast<const unsigned*>(s);
+    } else if constexpr (ITEMS == 8) {
+        uint2 v = *reinterpret_cast<const uint2*>(s);
+        w[0] = v.x; w[1] = v.y;
+    } else {
+        uint4 v = *reinterpret_cast<const uint4*>(s);
+        w[0] = v.x; w[1] = v.y; w[2] = v.z; w[3] = v.w;
+    }
+}
+
 // ------------------------------------------------------------------------------------------ packed mask bytes
 __device__ __forceinline__ constexpr unsigned byte_mask(int j) { return 0xffu << (8 * (j % 4)); }
 
@@ -154,12 +191,23 @@ __device__ __forceinline__ void mark_byte_dyn(unsigned (&w)[W], unsigned j) {   
 #pragma unroll
     for (int k = 0; k < W; ++k) w[k] |= ((j >> 2) == (unsigned)k) ? (0xffu << ((j & 3u) * 8u)) : 0u;
 }
+// (Pure shift arithmetic on purpose: a select between array elements would let the compiler index
+// the array dynamically and move the whole chunk to local memory.)
 template <int W>
 __device__ __forceinline__ bool test_byte_dyn(const unsigned (&w)[W], unsigned j) {
-    unsigned v = 0;
-#pragma unroll
-    for (int k = 0; k < W; ++k) v |= ((j >> 2) == (unsigned)k) ? w[k] : 0u;
-    return ((v >> ((j & 3u) * 8u)) & 0xffu) != 0;
+    static_assert(W == 1 || W == 2 || W == 4, "unsupported chunk width");
+    if constexpr (W == 1) {
+        return ((w[0] >> (j * 8u)) & 0xffu) != 0;
+    } else if constexpr (W == 2) {
+        const unsigned long long v = ((unsigned long long)w[1] << 32) | w[0];
+        return ((v >> (j * 8u)) & 0xffull) != 0;
+    } else {
+        const unsigned long long lo = ((unsigned long long)w[1] << 32) | w[0];
+        const unsigned long long hi = ((unsigned long long)w[3] << 32) | w[2];
+        const unsigned long long m = 0ull - (unsigned long long)((j >> 3) & 1u);      // all ones for the upper half
+        const unsigned long long v = (hi & m) | (lo & ~m);
+        return ((v >> ((j & 7u) * 8u)) & 0xffull) != 0;
+    }
 }
 
 // ------------------------------------------------------------------------------------------ tile records
@@ -187,7 +235,7 @@ __device__ __forceinline__ unsigned ld_volatile_u32(const unsigned* p) {
 // call's epoch next to each 4-byte payload word, so an 8-byte half is self-validating and no
 // fence is needed.  The wait is bounded: after `cap` polls the status word is set and 0 returned.
 static __device__ __noinline__ float lookback(const uint4* __restrict__ records, unsigned epoch, long long s,
-                                       unsigned cap, unsigned* status, int lane) {
+                                              unsigned cap, unsigned* status, int lane) {
     Pair acc = {0.f, 1.f};
     long long base = s - 1;
     unsigned polls = 0;
@@ -233,207 +281,248 @@ static __device__ __noinline__ float lookback(const uint4* __restrict__ records,
     }
 }
 
-// ------------------------------------------------------------------------------------------ the kernel
-template <int ALGO, bool TRUNC, bool VEC, int THREADS, int ITEMS, int MIN_BLOCKS>
-__global__ void __launch_bounds__(THREADS, MIN_BLOCKS) scan_kernel(const ScanParams p) {
-    constexpr bool FWD = is_forward(ALGO);
-    constexpr int NW = THREADS / 32;
-    constexpr int W = ITEMS / 4;
-    constexpr int TILE = THREADS * ITEMS;
-    constexpr unsigned FULL = 0xffffffffu;
-    static_assert(NW <= 32 && ITEMS % 4 == 0, "bad tile shape");
+// ------------------------------------------------------------------------------------------ one thread's part of a tile
+// Flags and geometry of a thread's ITEMS consecutive steps: everything the coefficient stage needs
+// besides the float inputs.  The persistent kernel fetches this one tile ahead.
+template <int ALGO, bool TRUNC, int ITEMS>
+struct Chunk {
+    static constexpr int W = ITEMS / 4;
+    long long i0;            // flat index of the chunk's first step
+    long long n0;            // its row
+    unsigned edge;           // offset of the first row edge at or after the chunk start (see locate)
+    int nvalid;              // steps of the chunk inside the array
+    unsigned dw[W], tw[W];   // dones / truncs mask bytes
+    unsigned halo_d;         // forward scans: dones byte of the step before the chunk
+    float ov[ITEMS];         // successor value where the recurrence is severed (0 | trunc_bootstrap | bootstrap)
+    float boot_first;        // window-edge bootstrap of the row whose edge lies in the chunk
+};
 
-    __shared__ Pair s_agg[NW];     // warp aggregates, indexed by the warp's rank in scan order
-    __shared__ float s_carry;      // tile carry-in
-    __shared__ int s_need;         // the tile is entered mid-episode
+// The float inputs of the same steps.
+template <int ITEMS>
+struct Vals {
+    float a[ITEMS];          // rewards | x | alpha; then alpha_t; then the first output
+    float x1[ITEMS];         // values | q_sa | beta
+    float x2[ITEMS];         // expected_q
+    float x3[ITEMS];         // log_rhos
+    float halo, halo_lr;     // successor-side neighbour of the chunk's last step (values | expected_q, log_rhos)
+};
 
-    const int tid = threadIdx.x;
-    const int lane = tid & 31;
-    const int warp = tid >> 5;
-    const long long s = blockIdx.x;                       // tile index in scan order
-    const long long tile = FWD ? s : (p.num_tiles - 1 - s);
-    const long long i0 = tile * TILE + (long long)tid * ITEMS;
+// Row / timestep of flat index i0, and the chunk offset of the first row edge: for backward scans
+// the row's last step (offset T-1-t0); for forward scans the next row's first step (offset T-t0, or
+// 0 when the chunk itself starts a row).
+template <int ALGO, bool TRUNC, int ITEMS>
+__device__ __forceinline__ void locate(Chunk<ALGO, TRUNC, ITEMS>& c, const ScanParams& p, long long i0) {
+    c.i0 = i0;
     const long long rem = p.total - i0;
-    const int nvalid = rem >= ITEMS ? ITEMS : (rem > 0 ? (int)rem : 0);
-
-    // row and timestep of this thread's first step
-    long long n0;
+    c.nvalid = rem >= ITEMS ? ITEMS : (rem > 0 ? (int)rem : 0);
     unsigned t0;
     if (p.idx32) {
         const unsigned n = (unsigned)i0;
         const unsigned hi = __umulhi(p.div_T.mul, n);
         const unsigned q = (hi + ((n - hi) >> p.div_T.sh1)) >> p.div_T.sh2;
-        n0 = q;
+        c.n0 = q;
         t0 = n - q * p.T;
     } else {
-        n0 = i0 / (long long)p.T;
-        t0 = (unsigned)(i0 - n0 * (long long)p.T);
+        c.n0 = i0 / (long long)p.T;
+        t0 = (unsigned)(i0 - c.n0 * (long long)p.T);
     }
+    c.edge = is_forward(ALGO) ? (t0 == 0 ? 0u : p.T - t0) : (p.T - 1 - t0);
+}
 
-    // ------------------------------------------------------------------ 1. loads (all issued up front)
-    unsigned dw[W], tw[W];
+// Window-edge bootstrap of the first row edge inside the chunk (plain load, issued early).
+template <int ALGO, bool TRUNC, int ITEMS>
+__device__ __forceinline__ void issue_boot(Chunk<ALGO, TRUNC, ITEMS>& c, const ScanParams& p) {
+    c.boot_first = 0.f;
+    if constexpr (!is_forward(ALGO) && !is_affine(ALGO)) {
+        if (p.boot != nullptr && c.edge < (unsigned)c.nvalid) c.boot_first = __ldg(p.boot + c.n0);
+    }
+}
+
+// Mask bytes from global memory; forward scans also need the dones byte just before the chunk.
+template <int ALGO, bool TRUNC, int ITEMS, bool VEC>
+__device__ __forceinline__ void load_flags_global(Chunk<ALGO, TRUNC, ITEMS>& c, const ScanParams& p, int lane) {
+    constexpr int W = ITEMS / 4;
 #pragma unroll
-    for (int k = 0; k < W; ++k) { dw[k] = 0; tw[k] = 0; }
-    if constexpr (!is_affine(ALGO)) load_mask<ITEMS, VEC>(p.dones, i0, nvalid, dw);
-    if constexpr (TRUNC) load_mask<ITEMS, VEC>(p.truncs, i0, nvalid, tw);
-
-    float alpha[ITEMS];            // rewards | x | alpha, then alpha_t, then the first output
-    load_f32<ITEMS, VEC>(p.f0, i0, nvalid, alpha);
-    float x1[ITEMS];               // values | q_sa | beta
-    if constexpr (ALGO != kDisc && ALGO != kElig && ALGO != kPrefix) load_f32<ITEMS, VEC>(p.f1, i0, nvalid, x1);
-    float x2[ITEMS];               // expected_q
-    if constexpr (ALGO == kRetrace) load_f32<ITEMS, VEC>(p.f2, i0, nvalid, x2);
-    float x3[ITEMS];               // log_rhos
-    if constexpr (ALGO == kVtrace || ALGO == kRetrace) load_f32<ITEMS, VEC>(p.f3, i0, nvalid, x3);
-
-    // one-step halo beyond the thread's chunk, in the direction of the dependency
-    float halo = 0.f, halo_lr = 0.f;
-    unsigned halo_d = 0;
-    if constexpr (!FWD && (has_values(ALGO) || ALGO == kRetrace)) {
-        const float* src = (ALGO == kRetrace) ? p.f2 : p.f1;
-        const bool edge_lane = (lane == 31) && (rem > ITEMS);
-        if (edge_lane) halo = __ldg(src + i0 + ITEMS);
-        if constexpr (ALGO == kRetrace) if (edge_lane) halo_lr = __ldg(p.f3 + i0 + ITEMS);
-    }
+    for (int k = 0; k < W; ++k) { c.dw[k] = 0; c.tw[k] = 0; }
+    c.halo_d = 0;
     if constexpr (ALGO == kElig || ALGO == kPrefix) {
-        if (lane == 0 && i0 > 0 && rem > 0) halo_d = __ldg(p.dones + i0 - 1);
+        if (lane == 0 && c.i0 > 0 && c.nvalid > 0) c.halo_d = __ldg(p.dones + c.i0 - 1);
     }
-
-    // Row edge inside the chunk.  Backward: the row's last step, at chunk offset T-1-t0; its
-    // window-edge bootstrap is fetched now.  Forward: the next row's first step, at offset T-t0
-    // (offset 0 when the chunk itself starts a row).
-    const unsigned edge = FWD ? (t0 == 0 ? 0u : p.T - t0) : (p.T - 1 - t0);
-    const bool has_edge = edge < (unsigned)ITEMS;
-    float boot_first = 0.f;
-    if constexpr (!FWD && !is_affine(ALGO)) {
-        if (p.boot != nullptr && edge < (unsigned)nvalid) boot_first = __ldg(p.boot + n0);
+    if constexpr (uses_dones(ALGO)) load_mask<ITEMS, VEC>(p.dones, c.i0, c.nvalid, c.dw);
+    if constexpr (TRUNC) load_mask<ITEMS, VEC>(p.truncs, c.i0, c.nvalid, c.tw);
+    if constexpr (ALGO == kElig || ALGO == kPrefix) {
+        const unsigned nb = __shfl_up_sync(0xffffffffu, c.dw[W - 1] >> 24, 1);
+        if (lane != 0) c.halo_d = nb;
     }
+}
 
-    // ------------------------------------------------------------------ 2. reset words
-    // sev: byte j non-zero = the recurrence does NOT continue from step j to its scan-order
-    // predecessor (t+1 backward, t-1 forward): a flag, a row edge, or a step beyond the array.
+// Sparse truncation continuation values: only where truncs is set and dones is not.
+template <int ALGO, bool TRUNC, int ITEMS>
+__device__ __forceinline__ void issue_trunc_values(Chunk<ALGO, TRUNC, ITEMS>& c, const ScanParams& p) {
+#pragma unroll
+    for (int j = 0; j < ITEMS; ++j) c.ov[j] = 0.f;
+    if constexpr (TRUNC) {
+#pragma unroll
+        for (int j = 0; j < ITEMS; ++j)
+            if (test_byte(c.tw, j) && !test_byte(c.dw, j)) c.ov[j] = __ldg(p.trunc_boot + c.i0 + j);
+    }
+}
+
+// Float inputs from global memory, with the one-step halo (lane 31 loads it, the others take
+// their neighbour's first element).
+template <int ALGO, bool TRUNC, int ITEMS, bool VEC>
+__device__ __forceinline__ void load_values_global(const Chunk<ALGO, TRUNC, ITEMS>& c, Vals<ITEMS>& v, const ScanParams& p, int lane) {
+    load_f32<ITEMS, VEC>(p.f0, c.i0, c.nvalid, v.a);
+    if constexpr (uses_f1(ALGO)) load_f32<ITEMS, VEC>(p.f1, c.i0, c.nvalid, v.x1);
+    if constexpr (uses_f2(ALGO)) load_f32<ITEMS, VEC>(p.f2, c.i0, c.nvalid, v.x2);
+    if constexpr (uses_f3(ALGO)) load_f32<ITEMS, VEC>(p.f3, c.i0, c.nvalid, v.x3);
+    v.halo = 0.f;
+    v.halo_lr = 0.f;
+    if constexpr (float_halo(ALGO)) {
+        const float* src = (ALGO == kRetrace) ? p.f2 : p.f1;
+        const bool edge_lane = (lane == 31) && (p.total - c.i0 > ITEMS);
+        if (edge_lane) v.halo = __ldg(src + c.i0 + ITEMS);
+        if constexpr (ALGO == kRetrace) if (edge_lane) v.halo_lr = __ldg(p.f3 + c.i0 + ITEMS);
+        const float first = (ALGO == kRetrace) ? v.x2[0] : v.x1[0];
+        const float nb = __shfl_down_sync(0xffffffffu, first, 1);
+        if (lane != 31) v.halo = nb;
+        if constexpr (ALGO == kRetrace) {
+            const float nl = __shfl_down_sync(0xffffffffu, v.x3[0], 1);
+            if (lane != 31) v.halo_lr = nl;
+        }
+    }
+}
+
+// Shared-memory scratch of the block-level scan; double-buffered by tile parity in the persistent
+// kernel so that one barrier per tile suffices.
+template <int NW>
+struct ScanSmem {
+    Pair agg[2][NW];     // warp aggregates, indexed by the warp's rank in scan order
+    float carry[2];      // tile carry-in
+    int need[2];         // the tile is entered mid-episode
+};
+
+struct NoHook {
+    __device__ __forceinline__ void operator()() const {}
+};
+
+// Steps 2-5 of the header comment for one tile, given the thread's loaded Chunk.
+// `after_barrier` runs right after the block barrier (every thread has consumed its inputs).
+template <int ALGO, bool TRUNC, bool VEC, int THREADS, int ITEMS, class Hook>
+__device__ __forceinline__ void tile_compute(Chunk<ALGO, TRUNC, ITEMS>& c, Vals<ITEMS>& v, const ScanParams& p, long long s,
+                                             unsigned epoch, ScanSmem<THREADS / 32>& sm, int buf, Hook after_barrier) {
+    constexpr bool FWD = is_forward(ALGO);
+    constexpr int NW = THREADS / 32;
+    constexpr int W = ITEMS / 4;
+    constexpr unsigned FULL = 0xffffffffu;
+    const int tid = threadIdx.x;
+    const int lane = tid & 31;
+    const int warp = tid >> 5;
+    const bool has_edge = c.edge < (unsigned)ITEMS;
+
+    // ---- reset words: byte j non-zero = the recurrence does NOT continue from step j to its
+    // scan-order predecessor (t+1 backward, t-1 forward): a flag, a row edge, a step beyond the array
     unsigned sev[W];
     if constexpr (FWD) {
         if constexpr (ALGO == kAffineFwd) {
 #pragma unroll
             for (int k = 0; k < W; ++k) sev[k] = 0;
+        } else if (ALGO == kPrefix && p.starts_at) {
+#pragma unroll
+            for (int k = 0; k < W; ++k) sev[k] = c.dw[k];
         } else {
             // ends_at: step j is cut off by the flag of step j-1 -> shift the bytes up by one step
-            const unsigned nb = __shfl_up_sync(FULL, dw[W - 1] >> 24, 1);
-            if (lane != 0) halo_d = nb;
-            if (ALGO == kPrefix && p.starts_at) {
 #pragma unroll
-                for (int k = 0; k < W; ++k) sev[k] = dw[k];
-            } else {
-#pragma unroll
-                for (int k = 0; k < W; ++k) sev[k] = (dw[k] << 8) | (k == 0 ? (halo_d & 0xffu) : (dw[(k + W - 1) % W] >> 24));
-            }
+            for (int k = 0; k < W; ++k)
+                sev[k] = (c.dw[k] << 8) | (k == 0 ? (c.halo_d & 0xffu) : (c.dw[(k + W - 1) % W] >> 24));
         }
     } else {
 #pragma unroll
-        for (int k = 0; k < W; ++k) sev[k] = dw[k] | tw[k];
+        for (int k = 0; k < W; ++k) sev[k] = c.dw[k] | c.tw[k];
     }
-    if (has_edge) mark_byte_dyn(sev, edge);
+    if (has_edge) mark_byte_dyn(sev, c.edge);
     if (p.T < (unsigned)ITEMS) {                // rows shorter than a chunk: several edges
-        for (unsigned e = edge + p.T; e < (unsigned)ITEMS; e += p.T) mark_byte_dyn(sev, e);
+        for (unsigned e = c.edge + p.T; e < (unsigned)ITEMS; e += p.T) mark_byte_dyn(sev, e);
     }
-    if (nvalid < ITEMS) {                       // ragged end of the array
-        for (unsigned j = nvalid; j < (unsigned)ITEMS; ++j) mark_byte_dyn(sev, j);
+    if (c.nvalid < ITEMS) {                     // ragged end of the array
+        for (unsigned j = c.nvalid; j < (unsigned)ITEMS; ++j) mark_byte_dyn(sev, j);
     }
 
-    // ------------------------------------------------------------------ 3. successor values at resets
-    // ov[j]: successor value used where the recurrence is severed -- 0 after a termination, the
-    // supplied continuation value after a truncation, the window-edge bootstrap at a row's last
-    // step (Section 3.2).  Zero wherever the recurrence continues.
-    float ov[ITEMS];
-#pragma unroll
-    for (int j = 0; j < ITEMS; ++j) ov[j] = 0.f;
+    // ---- window-edge bootstrap into ov at the row's last step, unless that step carries a flag
+    // (static indexing only, so that ov stays in registers)
     if constexpr (!FWD && !is_affine(ALGO)) {
-        if constexpr (TRUNC) {
-#pragma unroll
-            for (int j = 0; j < ITEMS; ++j)
-                if (test_byte(tw, j) && !test_byte(dw, j)) ov[j] = __ldg(p.trunc_boot + i0 + j);
-        }
         if (has_edge && p.boot != nullptr) {
-            unsigned e = edge;
-            long long n = n0;
-            float b = boot_first;
-            for (;;) {
-                if (e < (unsigned)nvalid && !test_byte_dyn(dw, e) && !test_byte_dyn(tw, e)) {
+            if (p.T >= (unsigned)ITEMS) {       // at most one row edge in the chunk; its bootstrap was fetched early
+                const bool ok = c.edge < (unsigned)c.nvalid && !test_byte_dyn(c.dw, c.edge) && !test_byte_dyn(c.tw, c.edge);
 #pragma unroll
-                    for (int j = 0; j < ITEMS; ++j) if ((unsigned)j == e) ov[j] = b;
+                for (int j = 0; j < ITEMS; ++j) c.ov[j] = (ok && (unsigned)j == c.edge) ? c.boot_first : c.ov[j];
+            } else {                            // rows shorter than a chunk: walk the steps
+                unsigned e = c.edge;
+                long long n = c.n0;
+#pragma unroll
+                for (int j = 0; j < ITEMS; ++j) {
+                    if ((unsigned)j == e) {
+                        if (j < c.nvalid && !test_byte(c.dw, j) && !test_byte(c.tw, j)) c.ov[j] = __ldg(p.boot + n);
+                        e += p.T;
+                        ++n;
+                    }
                 }
-                e += p.T;
-                ++n;
-                if (e >= (unsigned)nvalid) break;          // only when T < ITEMS
-                b = __ldg(p.boot + n);
             }
         }
     }
 
-    // neighbour values through the warp
-    if constexpr (!FWD && (has_values(ALGO) || ALGO == kRetrace)) {
-        const float first = (ALGO == kRetrace) ? x2[0] : x1[0];
-        const float nb = __shfl_down_sync(FULL, first, 1);
-        if (lane != 31) halo = nb;
-        if constexpr (ALGO == kRetrace) {
-            const float nl = __shfl_down_sync(FULL, x3[0], 1);
-            if (lane != 31) halo_lr = nl;
-        }
-    }
-
-    // ------------------------------------------------------------------ 4. coefficients (branch-free)
+    // ---- coefficients (branch-free)
     float beta[ITEMS];
-    float grho[ITEMS];             // V-Trace: cont * gamma * rho_t, for the advantage epilogue
+    float grho[ITEMS];             // V-Trace: gamma * rho_t where the recurrence continues, for the advantage epilogue
 #pragma unroll
     for (int j = 0; j < ITEMS; ++j) {
         const bool cut = test_byte(sev, j);
         if constexpr (FWD) {
-            if constexpr (ALGO == kAffineFwd) beta[j] = cut ? 0.f : x1[j];
+            if constexpr (ALGO == kAffineFwd) beta[j] = cut ? 0.f : v.x1[j];
             else beta[j] = cut ? 0.f : p.decay;
         } else if constexpr (ALGO == kAffineBwd) {
-            beta[j] = cut ? 0.f : x1[j];
+            beta[j] = cut ? 0.f : v.x1[j];
         } else {
-            const float c = cut ? 0.f : 1.f;
-            const float r = alpha[j];
+            const float r = v.a[j];
             float nextv = 0.f;
-            if constexpr (has_values(ALGO)) nextv = (j + 1 < ITEMS) ? x1[(j + 1) % ITEMS] : halo;
-            if constexpr (ALGO == kRetrace) nextv = (j + 1 < ITEMS) ? x2[(j + 1) % ITEMS] : halo;
+            if constexpr (has_values(ALGO)) nextv = (j + 1 < ITEMS) ? v.x1[(j + 1) % ITEMS] : v.halo;
+            if constexpr (ALGO == kRetrace) nextv = (j + 1 < ITEMS) ? v.x2[(j + 1) % ITEMS] : v.halo;
+            const float xn = cut ? c.ov[j] : nextv;      // successor value of Section 3.2 (selected, never multiplied)
             if constexpr (ALGO == kGae) {
-                alpha[j] = fmaf(p.gamma, fmaf(c, nextv, ov[j]), r) - x1[j];
+                v.a[j] = fmaf(p.gamma, xn, r) - v.x1[j];
                 beta[j] = cut ? 0.f : p.decay;
             } else if constexpr (ALGO == kTdLambda) {
                 // continuing: r + gamma(1-lambda) V_{t+1}; severed: r + gamma * successor value
-                alpha[j] = fmaf(p.gamma, ov[j], fmaf(cut ? 0.f : p.aux, nextv, r));
+                v.a[j] = fmaf(cut ? p.gamma : p.aux, xn, r);
                 beta[j] = cut ? 0.f : p.decay;
             } else if constexpr (ALGO == kDisc) {
-                alpha[j] = fmaf(p.gamma, ov[j], r);
+                v.a[j] = fmaf(p.gamma, c.ov[j], r);
                 beta[j] = cut ? 0.f : p.decay;
             } else if constexpr (ALGO == kVtrace) {
-                const float raw = expf(x3[j]);
+                const float raw = expf(v.x3[j]);
                 const float rho = fminf(p.rho_bar, raw);
                 const float cc = fminf(p.c_bar, raw);
-                alpha[j] = rho * (fmaf(p.gamma, fmaf(c, nextv, ov[j]), r) - x1[j]);
+                v.a[j] = rho * (fmaf(p.gamma, xn, r) - v.x1[j]);
                 beta[j] = cut ? 0.f : p.gamma * cc;
                 grho[j] = cut ? 0.f : p.gamma * rho;
             } else if constexpr (ALGO == kRetrace) {
-                alpha[j] = fmaf(p.gamma, fmaf(c, nextv, ov[j]), r) - x1[j];
-                const float lr_next = (j + 1 < ITEMS) ? x3[(j + 1) % ITEMS] : halo_lr;
+                v.a[j] = fmaf(p.gamma, xn, r) - v.x1[j];
+                const float lr_next = (j + 1 < ITEMS) ? v.x3[(j + 1) % ITEMS] : v.halo_lr;
                 beta[j] = cut ? 0.f : p.aux * fminf(p.c_bar, expf(lr_next));
             }
         }
     }
 
-    // ------------------------------------------------------------------ 5. thread aggregate (serial combine, Eq. 2)
+    // ---- thread aggregate (serial combine, Eq. 2)
     Pair agg;
     if constexpr (FWD) {
-        agg.a = alpha[0];
+        agg.a = v.a[0];
 #pragma unroll
-        for (int j = 1; j < ITEMS; ++j) agg.a = fmaf(beta[j], agg.a, alpha[j]);
+        for (int j = 1; j < ITEMS; ++j) agg.a = fmaf(beta[j], agg.a, v.a[j]);
     } else {
-        agg.a = alpha[ITEMS - 1];
+        agg.a = v.a[ITEMS - 1];
 #pragma unroll
-        for (int j = ITEMS - 2; j >= 0; --j) agg.a = fmaf(beta[j], agg.a, alpha[j]);
+        for (int j = ITEMS - 2; j >= 0; --j) agg.a = fmaf(beta[j], agg.a, v.a[j]);
     }
     if constexpr (const_decay(ALGO)) {
         unsigned any = 0;
@@ -446,8 +535,7 @@ __global__ void __launch_bounds__(THREADS, MIN_BLOCKS) scan_kernel(const ScanPar
         for (int j = 1; j < ITEMS; ++j) agg.b *= beta[j];
     }
 
-    // ------------------------------------------------------------------ 6. warp scan in scan order
-    // rank = position in scan order inside the warp: lane for forward scans, 31 - lane for backward.
+    // ---- warp scan in scan order; rank = position in scan order inside the warp
     const int rank = FWD ? lane : 31 - lane;
     Pair incl = agg;
 #pragma unroll
@@ -472,19 +560,20 @@ __global__ void __launch_bounds__(THREADS, MIN_BLOCKS) scan_kernel(const ScanPar
     }
     if (rank == 0) excl = Pair{0.f, 1.f};
 
-    // ------------------------------------------------------------------ 7. block carry through shared memory
+    // ---- block carry through shared memory
     const int wrank = FWD ? warp : NW - 1 - warp;
-    if (rank == 31) s_agg[wrank] = incl;
+    if (rank == 31) sm.agg[buf][wrank] = incl;
     if (wrank == 0 && rank == 0) {
         // the tile's first step in scan order: does the recurrence enter the tile from outside?
-        s_need = test_byte(sev, FWD ? 0 : ITEMS - 1) ? 0 : 1;
+        sm.need[buf] = test_byte(sev, FWD ? 0 : ITEMS - 1) ? 0 : 1;
     }
     __syncthreads();
+    after_barrier();
 
     Pair wcarry = {0.f, 1.f};      // all warps earlier in scan order
     Pair tile_agg;
     {
-        Pair w = (lane < NW) ? s_agg[lane] : Pair{0.f, 1.f};
+        Pair w = (lane < NW) ? sm.agg[buf][lane] : Pair{0.f, 1.f};
 #pragma unroll
         for (int d = 1; d < NW; d <<= 1) {
             Pair o;
@@ -500,69 +589,66 @@ __global__ void __launch_bounds__(THREADS, MIN_BLOCKS) scan_kernel(const ScanPar
     }
     const Pair before = apply(excl, wcarry);   // everything earlier in scan order inside this tile
 
-    // ------------------------------------------------------------------ 8. carry between thread blocks
+    // ---- carry between thread blocks
     float carry_in = 0.f;
     if (p.carry_mode) {
-        unsigned epoch = 0;
-        if (warp == 0) {
-            epoch = ld_volatile_u32(p.header);
-            if (lane == 0 && s != p.mute_tile) {
-                st_volatile_u4(p.records + s, make_uint4(__float_as_uint(tile_agg.a), epoch,
-                                                         __float_as_uint(tile_agg.b), epoch));
-            }
+        if (warp == 0 && lane == 0 && s != p.mute_tile) {
+            st_volatile_u4(p.records + s, make_uint4(__float_as_uint(tile_agg.a), epoch,
+                                                     __float_as_uint(tile_agg.b), epoch));
         }
-        const int need = s_need;               // block-uniform
+        const int need = sm.need[buf];         // block-uniform
         if (need) {
             if (warp == 0) {
-                const float c = lookback(p.records, epoch, s, p.spin_cap, p.header + 2, lane);
-                if (lane == 0) s_carry = c;
+                const float cin = lookback(p.records, epoch, s, p.spin_cap, p.status, lane);
+                if (lane == 0) sm.carry[buf] = cin;
             }
             __syncthreads();
-            carry_in = s_carry;
+            carry_in = sm.carry[buf];
         }
     }
     // value of the recurrence at the step just before this thread's chunk in scan order
     float prev = fmaf(before.b, carry_in, before.a);
 
-    // ------------------------------------------------------------------ 9. replay, epilogue, store
+    // ---- replay, epilogue, store
     float out1v[ITEMS];
     if constexpr (FWD) {
 #pragma unroll
         for (int j = 0; j < ITEMS; ++j) {
-            prev = fmaf(beta[j], prev, alpha[j]);
-            alpha[j] = prev;
+            prev = fmaf(beta[j], prev, v.a[j]);
+            v.a[j] = prev;
         }
     } else {
 #pragma unroll
         for (int j = ITEMS - 1; j >= 0; --j) {
-            const float d = fmaf(beta[j], prev, alpha[j]);
+            const float d = fmaf(beta[j], prev, v.a[j]);
             if constexpr (ALGO == kGae) {
-                alpha[j] = d;
-                out1v[j] = d + x1[j];
+                v.a[j] = d;
+                out1v[j] = d + v.x1[j];
             } else if constexpr (ALGO == kVtrace) {
                 // A_t = rho_t (r_t + gamma v_{t+1} - V_t) = alpha_t + gamma rho_t Delta_{t+1} where the
                 // recurrence continues (v_{t+1} = V_{t+1} + Delta_{t+1}), alpha_t elsewhere.
-                out1v[j] = fmaf(grho[j], prev, alpha[j]);
-                alpha[j] = x1[j] + d;
+                out1v[j] = fmaf(grho[j], prev, v.a[j]);
+                v.a[j] = v.x1[j] + d;
             } else if constexpr (ALGO == kRetrace) {
-                alpha[j] = x1[j] + d;
+                v.a[j] = v.x1[j] + d;
             } else {
-                alpha[j] = d;
+                v.a[j] = d;
             }
             prev = d;
         }
     }
-    if (nvalid > 0) {
-        store_f32<ITEMS, VEC>(p.out0, i0, nvalid, alpha);
+    if (c.nvalid > 0) {
+        store_f32<ITEMS, VEC>(p.out0, c.i0, c.nvalid, v.a);
         if constexpr (ALGO == kGae || ALGO == kVtrace) {
-            if (p.out1 != nullptr) store_f32<ITEMS, VEC>(p.out1, i0, nvalid, out1v);
+            if (p.out1 != nullptr) store_f32<ITEMS, VEC>(p.out1, c.i0, c.nvalid, out1v);
         }
     }
+}
 
-    // ------------------------------------------------------------------ 10. close the call (carry mode)
-    // The last block to finish advances the epoch, so the records of this call can never be taken
-    // for those of the next one and no per-call clearing is needed.
-    if (p.carry_mode && tid == 0) {
+// The last block to finish advances the epoch, so the records of this call can never be taken for
+// those of the next one and no per-call clearing is needed.
+__device__ __forceinline__ void close_call(const ScanParams& p) {
+    if (p.carry_mode && threadIdx.x == 0) {
         __threadfence();
         const unsigned done = atomicAdd(p.header + 1, 1u);
         if (done == gridDim.x - 1) {
@@ -571,6 +657,280 @@ __global__ void __launch_bounds__(THREADS, MIN_BLOCKS) scan_kernel(const ScanPar
             p.header[0] = (e == 0xffffffffu) ? 1u : e + 1u;
         }
     }
+}
+
+// ------------------------------------------------------------------------------------------ kernel 1: one tile per block
+template <int ALGO, bool TRUNC, bool VEC, int THREADS, int ITEMS, int MIN_BLOCKS>
+__global__ void __launch_bounds__(THREADS, MIN_BLOCKS) scan_kernel(const ScanParams p) {
+    constexpr bool FWD = is_forward(ALGO);
+    constexpr int TILE = THREADS * ITEMS;
+    __shared__ ScanSmem<THREADS / 32> sm;
+
+    const int tid = threadIdx.x;
+    const int lane = tid & 31;
+    const long long s = blockIdx.x;                       // tile index in scan order
+    const long long tile = FWD ? s : (p.num_tiles - 1 - s);
+
+    Chunk<ALGO, TRUNC, ITEMS> c;
+    locate(c, p, tile * TILE + (long long)tid * ITEMS);
+    load_flags_global<ALGO, TRUNC, ITEMS, VEC>(c, p, lane);
+    Vals<ITEMS> v;
+    load_values_global<ALGO, TRUNC, ITEMS, VEC>(c, v, p, lane);
+    issue_boot(c, p);
+    issue_trunc_values(c, p);
+    unsigned epoch = 0;
+    if (p.carry_mode && tid < 32) epoch = ld_volatile_u32(p.header);
+    tile_compute<ALGO, TRUNC, VEC, THREADS, ITEMS>(c, v, p, s, epoch, sm, 0, NoHook{});
+    close_call(p);
+}
+
+// ------------------------------------------------------------------------------------------ mbarrier / bulk copy (PTX)
+__device__ __forceinline__ unsigned smem_u32(const void* ptr) { return (unsigned)__cvta_generic_to_shared(ptr); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, unsigned count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, unsigned bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, unsigned parity) {
+    unsigned ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+// 1-D bulk copy global -> this block's shared memory, completing `bytes` on `bar`.  No multicast.
+// dst, src 16-byte aligned; bytes a multiple of 16.
+__device__ __forceinline__ void bulk_load(void* dst, const void* src, unsigned bytes, uint64_t* bar) {
+    asm volatile("cp.async.bulk.shared::cta.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 :: "r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void fence_barrier_init() {
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void fence_proxy_async() {
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+
+// Shared-memory layout of one ring stage: the float arrays the algorithm reads (TILE + 4 floats
+// each: the tile plus the halo step) and its mask arrays (16 bytes of front pad, then TILE bytes;
+// forward scans copy the 16 bytes before the tile into the pad to get the preceding dones byte).
+template <int ALGO, bool TRUNC, int TILE>
+struct StageLayout {
+    static constexpr int NF = 1 + (uses_f1(ALGO) ? 1 : 0) + (uses_f2(ALGO) ? 1 : 0) + (uses_f3(ALGO) ? 1 : 0);
+    static constexpr int NM = (uses_dones(ALGO) ? 1 : 0) + (TRUNC ? 1 : 0);
+    static constexpr int F_BYTES = (TILE + 4) * 4;
+    static constexpr int M_BYTES = TILE + 16;
+    static constexpr int BYTES = ((NF * F_BYTES + NM * M_BYTES) + 127) / 128 * 128;
+    // slot of each array among the float arrays
+    static constexpr int SLOT_F1 = 1;
+    static constexpr int SLOT_F2 = 2;
+    static constexpr int SLOT_F3 = 1 + (uses_f1(ALGO) ? 1 : 0) + (uses_f2(ALGO) ? 1 : 0);
+    __device__ static float* f(unsigned char* stage, int slot) { return reinterpret_cast<float*>(stage + slot * F_BYTES); }
+    __device__ static uint8_t* m(unsigned char* stage, int slot) { return stage + NF * F_BYTES + slot * M_BYTES; }
+};
+
+// Wait until the ring stage of the cj-th bulk-fetched tile of this block has landed.  The wait is
+// bounded twice over (poll count and about a second of SM clock); when it gives up it records
+// RLCS_ERR_TIMEOUT in the status word and every later wait of this block returns at once.
+constexpr long long kWaitClockLimit = 2000000000ll;
+template <int STAGES>
+__device__ __forceinline__ void wait_stage(uint64_t* full_bar, unsigned cj, const ScanParams& p, bool& gave_up) {
+    uint64_t* bar = &full_bar[cj % STAGES];
+    const unsigned parity = (cj / STAGES) & 1u;
+    if (gave_up || mbar_try_wait(bar, parity)) return;
+    const long long t_start = clock64();
+    unsigned spins = 0;
+    while (!mbar_try_wait(bar, parity)) {
+        if (++spins > p.spin_cap || clock64() - t_start > kWaitClockLimit) {
+            if (p.status != nullptr) atomicExch(p.status, kDeviceTimeout);
+            gave_up = true;
+            return;
+        }
+    }
+}
+
+// Geometry, flags, window-edge bootstrap and sparse truncation values of address tile `tile`:
+// everything the coefficient stage needs besides the float inputs.  Called one tile ahead, so that
+// the dependent loads (bootstrap values) are in flight while the previous tile is being stored.
+template <int ALGO, bool TRUNC, int THREADS, int ITEMS, int STAGES>
+__device__ __forceinline__ void prefetch_flags(Chunk<ALGO, TRUNC, ITEMS>& c, const ScanParams& p, long long tile,
+                                               unsigned char* ring, uint64_t* full_bar, unsigned cj, bool& gave_up) {
+    constexpr int TILE = THREADS * ITEMS;
+    constexpr int HALO = float_halo(ALGO) ? 4 : 0;
+    constexpr int W = ITEMS / 4;
+    using L = StageLayout<ALGO, TRUNC, TILE>;
+    const int tid = threadIdx.x;
+    locate(c, p, tile * TILE + (long long)tid * ITEMS);
+    issue_boot(c, p);
+    if (tile * TILE + TILE + HALO <= p.total) {
+        wait_stage<STAGES>(full_bar, cj, p, gave_up);
+        unsigned char* stage = ring + (size_t)(cj % STAGES) * L::BYTES;
+#pragma unroll
+        for (int k = 0; k < W; ++k) { c.dw[k] = 0; c.tw[k] = 0; }
+        c.halo_d = 0;
+        if constexpr (uses_dones(ALGO)) {
+            const uint8_t* md = L::m(stage, 0) + 16 + tid * ITEMS;
+            lds_mask<ITEMS>(md, c.dw);
+            if constexpr (ALGO == kElig || ALGO == kPrefix) c.halo_d = md[-1];   // unused garbage for tile 0 (row start)
+        }
+        if constexpr (TRUNC) lds_mask<ITEMS>(L::m(stage, 1) + 16 + tid * ITEMS, c.tw);
+    } else {
+        load_flags_global<ALGO, TRUNC, ITEMS, true>(c, p, tid & 31);
+    }
+    issue_trunc_values(c, p);
+}
+
+// ------------------------------------------------------------------------------------------ kernel 2: persistent, bulk-copy ring
+// Per-block walk state of the persistent kernel.
+struct Walk {
+    long long G;             // grid size = stride of the walk in scan-order tiles
+    long long s;             // scan-order tile being processed
+    long long ps;            // producer (thread 0): next scan-order tile to fetch
+    unsigned pj;             // producer: tiles fetched so far
+    unsigned cj;             // bulk-fetched tiles consumed so far
+    unsigned epoch;
+    int buf;                 // parity of the block-scan scratch
+    bool gave_up;            // a bounded wait ran out: stop waiting, finish the walk
+};
+
+template <int ALGO, int TILE>
+__device__ __forceinline__ long long tile_of(const ScanParams& p, long long s) {
+    return is_forward(ALGO) ? s : (p.num_tiles - 1 - s);
+}
+// A tile can be fetched by bulk copies when it, and the halo step behind it, lie inside the array.
+template <int ALGO, int TILE>
+__device__ __forceinline__ bool bulk_ok(const ScanParams& p, long long tile) {
+    return tile * TILE + TILE + (float_halo(ALGO) ? 4 : 0) <= p.total;
+}
+
+// Thread 0: issue the bulk copies of this block's next fetchable tile into ring stage pj % STAGES.
+template <int ALGO, bool TRUNC, int TILE, int STAGES>
+__device__ __forceinline__ void produce_next(const ScanParams& p, Walk& w, unsigned char* ring, uint64_t* full_bar) {
+    constexpr bool FWD = is_forward(ALGO);
+    constexpr int HALO = float_halo(ALGO) ? 4 : 0;
+    using L = StageLayout<ALGO, TRUNC, TILE>;
+    while (w.ps < p.num_tiles) {
+        const long long tile = tile_of<ALGO, TILE>(p, w.ps);
+        w.ps += w.G;
+        if (!bulk_ok<ALGO, TILE>(p, tile)) continue;
+        unsigned char* stage = ring + (size_t)(w.pj % STAGES) * L::BYTES;
+        uint64_t* bar = &full_bar[w.pj % STAGES];
+        const long long e0 = tile * TILE;
+        // forward scans fetch the 16 mask bytes before the tile as well (the preceding step's flag)
+        const bool pre = FWD && uses_dones(ALGO) && e0 >= 16;
+        const unsigned dbytes = pre ? TILE + 16 : TILE;
+        mbar_expect_tx(bar, L::NF * (TILE + HALO) * 4 + (uses_dones(ALGO) ? dbytes : 0) + (TRUNC ? TILE : 0));
+        bulk_load(L::f(stage, 0), p.f0 + e0, (TILE + HALO) * 4, bar);
+        if constexpr (uses_f1(ALGO)) bulk_load(L::f(stage, L::SLOT_F1), p.f1 + e0, (TILE + HALO) * 4, bar);
+        if constexpr (uses_f2(ALGO)) bulk_load(L::f(stage, L::SLOT_F2), p.f2 + e0, (TILE + HALO) * 4, bar);
+        if constexpr (uses_f3(ALGO)) bulk_load(L::f(stage, L::SLOT_F3), p.f3 + e0, (TILE + HALO) * 4, bar);
+        if constexpr (uses_dones(ALGO))
+            bulk_load(L::m(stage, 0) + (pre ? 0 : 16), p.dones + e0 - (pre ? 16 : 0), dbytes, bar);
+        if constexpr (TRUNC) bulk_load(L::m(stage, 1) + 16, p.truncs + e0, TILE, bar);
+        ++w.pj;
+        return;
+    }
+}
+
+template <int ALGO, bool TRUNC, int TILE, int STAGES>
+struct Refill {
+    const ScanParams& p;
+    Walk& w;
+    unsigned char* ring;
+    uint64_t* full_bar;
+    bool active;
+    // After the block barrier every thread has read the current stage: thread 0 refills it.
+    __device__ __forceinline__ void operator()() const {
+        if (active && threadIdx.x == 0) {
+            fence_proxy_async();
+            produce_next<ALGO, TRUNC, TILE, STAGES>(p, w, ring, full_bar);
+        }
+    }
+};
+
+// One tile of the walk: `cur` holds the flags of tile w.s (fetched during the previous step), `nxt`
+// receives those of tile w.s + G now, so that its dependent loads (truncation and window-edge
+// bootstrap values) have a whole tile's time to arrive.
+template <int ALGO, bool TRUNC, int THREADS, int ITEMS, int STAGES>
+__device__ __forceinline__ void walk_step(Chunk<ALGO, TRUNC, ITEMS>& cur, Chunk<ALGO, TRUNC, ITEMS>& nxt,
+                                          const ScanParams& p, Walk& w, unsigned char* ring, uint64_t* full_bar,
+                                          ScanSmem<THREADS / 32>& sm) {
+    constexpr int TILE = THREADS * ITEMS;
+    using L = StageLayout<ALGO, TRUNC, TILE>;
+    const int tid = threadIdx.x;
+    const bool bulk = bulk_ok<ALGO, TILE>(p, tile_of<ALGO, TILE>(p, w.s));
+    if (w.s + w.G < p.num_tiles)
+        prefetch_flags<ALGO, TRUNC, THREADS, ITEMS, STAGES>(nxt, p, tile_of<ALGO, TILE>(p, w.s + w.G), ring, full_bar,
+                                                            w.cj + (bulk ? 1u : 0u), w.gave_up);
+    Vals<ITEMS> v;
+    if (bulk) {
+        unsigned char* stage = ring + (size_t)(w.cj % STAGES) * L::BYTES;     // landed: prefetch_flags waited for it
+        const int off = tid * ITEMS;
+        lds_f32<ITEMS>(L::f(stage, 0) + off, v.a);
+        if constexpr (uses_f1(ALGO)) lds_f32<ITEMS>(L::f(stage, L::SLOT_F1) + off, v.x1);
+        if constexpr (uses_f2(ALGO)) lds_f32<ITEMS>(L::f(stage, L::SLOT_F2) + off, v.x2);
+        if constexpr (uses_f3(ALGO)) lds_f32<ITEMS>(L::f(stage, L::SLOT_F3) + off, v.x3);
+        v.halo = 0.f;
+        v.halo_lr = 0.f;
+        if constexpr (has_values(ALGO)) v.halo = L::f(stage, L::SLOT_F1)[off + ITEMS];
+        if constexpr (ALGO == kRetrace) {
+            v.halo = L::f(stage, L::SLOT_F2)[off + ITEMS];
+            v.halo_lr = L::f(stage, L::SLOT_F3)[off + ITEMS];
+        }
+    } else {
+        load_values_global<ALGO, TRUNC, ITEMS, true>(cur, v, p, tid & 31);
+    }
+    tile_compute<ALGO, TRUNC, true, THREADS, ITEMS>(cur, v, p, w.s, w.epoch, sm, w.buf,
+                                                    Refill<ALGO, TRUNC, TILE, STAGES>{p, w, ring, full_bar, bulk});
+    if (bulk) ++w.cj;
+    w.s += w.G;
+    w.buf ^= 1;
+}
+
+template <int ALGO, bool TRUNC, int THREADS, int ITEMS, int STAGES, int MIN_BLOCKS>
+__global__ void __launch_bounds__(THREADS, MIN_BLOCKS) scan_kernel_tma(const ScanParams p) {
+    constexpr int TILE = THREADS * ITEMS;
+    using L = StageLayout<ALGO, TRUNC, TILE>;
+
+    extern __shared__ __align__(128) unsigned char ring[];          // STAGES * L::BYTES
+    __shared__ __align__(8) uint64_t full_bar[STAGES];
+    __shared__ ScanSmem<THREADS / 32> sm;
+
+    const int tid = threadIdx.x;
+    Walk w;
+    w.G = gridDim.x;
+    w.s = blockIdx.x;
+    w.ps = blockIdx.x;
+    w.pj = 0;
+    w.cj = 0;
+    w.epoch = 0;
+    w.buf = 0;
+    w.gave_up = false;
+
+    if (tid == 0) {
+#pragma unroll
+        for (int k = 0; k < STAGES; ++k) mbar_init(&full_bar[k], 1);
+        fence_barrier_init();
+        fence_proxy_async();
+    }
+    __syncthreads();
+    if (tid == 0) {
+#pragma unroll
+        for (int k = 0; k < STAGES; ++k) produce_next<ALGO, TRUNC, TILE, STAGES>(p, w, ring, full_bar);
+    }
+    if (p.carry_mode && tid < 32) w.epoch = ld_volatile_u32(p.header);
+
+    // Two flag sets alternate between "current" and "next" so that no register copies are needed.
+    Chunk<ALGO, TRUNC, ITEMS> fa, fb;
+    if (w.s < p.num_tiles)
+        prefetch_flags<ALGO, TRUNC, THREADS, ITEMS, STAGES>(fa, p, tile_of<ALGO, TILE>(p, w.s), ring, full_bar, w.cj, w.gave_up);
+    while (w.s < p.num_tiles) {
+        walk_step<ALGO, TRUNC, THREADS, ITEMS, STAGES>(fa, fb, p, w, ring, full_bar, sm);
+        if (w.s >= p.num_tiles) break;
+        walk_step<ALGO, TRUNC, THREADS, ITEMS, STAGES>(fb, fa, p, w, ring, full_bar, sm);
+    }
+    close_call(p);
 }
 
 }  // namespace rlcs

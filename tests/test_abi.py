@@ -116,7 +116,8 @@ def test_workspace_init_argument_checks(L):
 
 
 def test_debug_hooks_argument_checks(L):
-    assert L.rlcs_debug_set_tile_variant(99) == E_ARG and L.rlcs_debug_set_tile_variant(-1) == E_ARG
+    assert L.rlcs_debug_set_tile_variant(99) == E_ARG and L.rlcs_debug_set_tile_variant(-2) == E_ARG
+    assert L.rlcs_debug_set_tile_variant(-1) == OK
     assert L.rlcs_debug_set_tile_variant(0) == OK
     assert L.rlcs_debug_tile_elems(0) == 2048 and L.rlcs_debug_tile_elems(1) == 512
     assert L.rlcs_debug_tile_elems(99) == 0
