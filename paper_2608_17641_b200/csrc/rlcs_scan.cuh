@@ -287,8 +287,6 @@ static __device__ __noinline__ float lookback(const uint4* __restrict__ records,
 template <int ALGO, bool TRUNC, int ITEMS>
 struct Chunk {
     static constexpr int W = ITEMS / 4;
-    long long i0;            // flat index of the chunk's first step
-    long long n0;            // its row
     unsigned edge;           // offset of the first row edge at or after the chunk start (see locate)
     int nvalid;              // steps of the chunk inside the array
     unsigned dw[W], tw[W];   // dones / truncs mask bytes
@@ -311,45 +309,46 @@ struct Vals {
 // the row's last step (offset T-1-t0); for forward scans the next row's first step (offset T-t0, or
 // 0 when the chunk itself starts a row).
 template <int ALGO, bool TRUNC, int ITEMS>
-__device__ __forceinline__ void locate(Chunk<ALGO, TRUNC, ITEMS>& c, const ScanParams& p, long long i0) {
-    c.i0 = i0;
+__device__ __forceinline__ long long locate(Chunk<ALGO, TRUNC, ITEMS>& c, const ScanParams& p, long long i0) {
     const long long rem = p.total - i0;
     c.nvalid = rem >= ITEMS ? ITEMS : (rem > 0 ? (int)rem : 0);
     unsigned t0;
+    long long n0;
     if (p.idx32) {
         const unsigned n = (unsigned)i0;
         const unsigned hi = __umulhi(p.div_T.mul, n);
         const unsigned q = (hi + ((n - hi) >> p.div_T.sh1)) >> p.div_T.sh2;
-        c.n0 = q;
+        n0 = q;
         t0 = n - q * p.T;
     } else {
-        c.n0 = i0 / (long long)p.T;
-        t0 = (unsigned)(i0 - c.n0 * (long long)p.T);
+        n0 = i0 / (long long)p.T;
+        t0 = (unsigned)(i0 - n0 * (long long)p.T);
     }
     c.edge = is_forward(ALGO) ? (t0 == 0 ? 0u : p.T - t0) : (p.T - 1 - t0);
+    return n0;               // the row of step i0
 }
 
 // Window-edge bootstrap of the first row edge inside the chunk (plain load, issued early).
 template <int ALGO, bool TRUNC, int ITEMS>
-__device__ __forceinline__ void issue_boot(Chunk<ALGO, TRUNC, ITEMS>& c, const ScanParams& p) {
+__device__ __forceinline__ void issue_boot(Chunk<ALGO, TRUNC, ITEMS>& c, const ScanParams& p, long long n0) {
     c.boot_first = 0.f;
     if constexpr (!is_forward(ALGO) && !is_affine(ALGO)) {
-        if (p.boot != nullptr && c.edge < (unsigned)c.nvalid) c.boot_first = __ldg(p.boot + c.n0);
+        if (p.boot != nullptr && c.edge < (unsigned)c.nvalid) c.boot_first = __ldg(p.boot + n0);
     }
 }
 
 // Mask bytes from global memory; forward scans also need the dones byte just before the chunk.
 template <int ALGO, bool TRUNC, int ITEMS, bool VEC>
-__device__ __forceinline__ void load_flags_global(Chunk<ALGO, TRUNC, ITEMS>& c, const ScanParams& p, int lane) {
+__device__ __forceinline__ void load_flags_global(Chunk<ALGO, TRUNC, ITEMS>& c, const ScanParams& p, long long i0, int lane) {
     constexpr int W = ITEMS / 4;
 #pragma unroll
     for (int k = 0; k < W; ++k) { c.dw[k] = 0; c.tw[k] = 0; }
     c.halo_d = 0;
     if constexpr (ALGO == kElig || ALGO == kPrefix) {
-        if (lane == 0 && c.i0 > 0 && c.nvalid > 0) c.halo_d = __ldg(p.dones + c.i0 - 1);
+        if (lane == 0 && i0 > 0 && c.nvalid > 0) c.halo_d = __ldg(p.dones + i0 - 1);
     }
-    if constexpr (uses_dones(ALGO)) load_mask<ITEMS, VEC>(p.dones, c.i0, c.nvalid, c.dw);
-    if constexpr (TRUNC) load_mask<ITEMS, VEC>(p.truncs, c.i0, c.nvalid, c.tw);
+    if constexpr (uses_dones(ALGO)) load_mask<ITEMS, VEC>(p.dones, i0, c.nvalid, c.dw);
+    if constexpr (TRUNC) load_mask<ITEMS, VEC>(p.truncs, i0, c.nvalid, c.tw);
     if constexpr (ALGO == kElig || ALGO == kPrefix) {
         const unsigned nb = __shfl_up_sync(0xffffffffu, c.dw[W - 1] >> 24, 1);
         if (lane != 0) c.halo_d = nb;
@@ -358,31 +357,31 @@ __device__ __forceinline__ void load_flags_global(Chunk<ALGO, TRUNC, ITEMS>& c, 
 
 // Sparse truncation continuation values: only where truncs is set and dones is not.
 template <int ALGO, bool TRUNC, int ITEMS>
-__device__ __forceinline__ void issue_trunc_values(Chunk<ALGO, TRUNC, ITEMS>& c, const ScanParams& p) {
+__device__ __forceinline__ void issue_trunc_values(Chunk<ALGO, TRUNC, ITEMS>& c, const ScanParams& p, long long i0) {
 #pragma unroll
     for (int j = 0; j < ITEMS; ++j) c.ov[j] = 0.f;
     if constexpr (TRUNC) {
 #pragma unroll
         for (int j = 0; j < ITEMS; ++j)
-            if (test_byte(c.tw, j) && !test_byte(c.dw, j)) c.ov[j] = __ldg(p.trunc_boot + c.i0 + j);
+            if (test_byte(c.tw, j) && !test_byte(c.dw, j)) c.ov[j] = __ldg(p.trunc_boot + i0 + j);
     }
 }
 
 // Float inputs from global memory, with the one-step halo (lane 31 loads it, the others take
 // their neighbour's first element).
 template <int ALGO, bool TRUNC, int ITEMS, bool VEC>
-__device__ __forceinline__ void load_values_global(const Chunk<ALGO, TRUNC, ITEMS>& c, Vals<ITEMS>& v, const ScanParams& p, int lane) {
-    load_f32<ITEMS, VEC>(p.f0, c.i0, c.nvalid, v.a);
-    if constexpr (uses_f1(ALGO)) load_f32<ITEMS, VEC>(p.f1, c.i0, c.nvalid, v.x1);
-    if constexpr (uses_f2(ALGO)) load_f32<ITEMS, VEC>(p.f2, c.i0, c.nvalid, v.x2);
-    if constexpr (uses_f3(ALGO)) load_f32<ITEMS, VEC>(p.f3, c.i0, c.nvalid, v.x3);
+__device__ __forceinline__ void load_values_global(const Chunk<ALGO, TRUNC, ITEMS>& c, Vals<ITEMS>& v, const ScanParams& p, long long i0, int lane) {
+    load_f32<ITEMS, VEC>(p.f0, i0, c.nvalid, v.a);
+    if constexpr (uses_f1(ALGO)) load_f32<ITEMS, VEC>(p.f1, i0, c.nvalid, v.x1);
+    if constexpr (uses_f2(ALGO)) load_f32<ITEMS, VEC>(p.f2, i0, c.nvalid, v.x2);
+    if constexpr (uses_f3(ALGO)) load_f32<ITEMS, VEC>(p.f3, i0, c.nvalid, v.x3);
     v.halo = 0.f;
     v.halo_lr = 0.f;
     if constexpr (float_halo(ALGO)) {
         const float* src = (ALGO == kRetrace) ? p.f2 : p.f1;
-        const bool edge_lane = (lane == 31) && (p.total - c.i0 > ITEMS);
-        if (edge_lane) v.halo = __ldg(src + c.i0 + ITEMS);
-        if constexpr (ALGO == kRetrace) if (edge_lane) v.halo_lr = __ldg(p.f3 + c.i0 + ITEMS);
+        const bool edge_lane = (lane == 31) && (p.total - i0 > ITEMS);
+        if (edge_lane) v.halo = __ldg(src + i0 + ITEMS);
+        if constexpr (ALGO == kRetrace) if (edge_lane) v.halo_lr = __ldg(p.f3 + i0 + ITEMS);
         const float first = (ALGO == kRetrace) ? v.x2[0] : v.x1[0];
         const float nb = __shfl_down_sync(0xffffffffu, first, 1);
         if (lane != 31) v.halo = nb;
@@ -409,7 +408,7 @@ struct NoHook {
 // Steps 2-5 of the header comment for one tile, given the thread's loaded Chunk.
 // `after_barrier` runs right after the block barrier (every thread has consumed its inputs).
 template <int ALGO, bool TRUNC, bool VEC, int THREADS, int ITEMS, class Hook>
-__device__ __forceinline__ void tile_compute(Chunk<ALGO, TRUNC, ITEMS>& c, Vals<ITEMS>& v, const ScanParams& p, long long s,
+__device__ __forceinline__ void tile_compute(Chunk<ALGO, TRUNC, ITEMS>& c, Vals<ITEMS>& v, const ScanParams& p, long long i0, long long s,
                                              unsigned epoch, ScanSmem<THREADS / 32>& sm, int buf, Hook after_barrier) {
     constexpr bool FWD = is_forward(ALGO);
     constexpr int NW = THREADS / 32;
@@ -458,7 +457,7 @@ __device__ __forceinline__ void tile_compute(Chunk<ALGO, TRUNC, ITEMS>& c, Vals<
                 for (int j = 0; j < ITEMS; ++j) c.ov[j] = (ok && (unsigned)j == c.edge) ? c.boot_first : c.ov[j];
             } else {                            // rows shorter than a chunk: walk the steps
                 unsigned e = c.edge;
-                long long n = c.n0;
+                long long n = i0 / (long long)p.T;      // row of the chunk's first step
 #pragma unroll
                 for (int j = 0; j < ITEMS; ++j) {
                     if ((unsigned)j == e) {
@@ -638,9 +637,9 @@ __device__ __forceinline__ void tile_compute(Chunk<ALGO, TRUNC, ITEMS>& c, Vals<
         }
     }
     if (c.nvalid > 0) {
-        store_f32<ITEMS, VEC>(p.out0, c.i0, c.nvalid, v.a);
+        store_f32<ITEMS, VEC>(p.out0, i0, c.nvalid, v.a);
         if constexpr (ALGO == kGae || ALGO == kVtrace) {
-            if (p.out1 != nullptr) store_f32<ITEMS, VEC>(p.out1, c.i0, c.nvalid, out1v);
+            if (p.out1 != nullptr) store_f32<ITEMS, VEC>(p.out1, i0, c.nvalid, out1v);
         }
     }
 }
@@ -672,15 +671,16 @@ __global__ void __launch_bounds__(THREADS, MIN_BLOCKS) scan_kernel(const ScanPar
     const long long tile = FWD ? s : (p.num_tiles - 1 - s);
 
     Chunk<ALGO, TRUNC, ITEMS> c;
-    locate(c, p, tile * TILE + (long long)tid * ITEMS);
-    load_flags_global<ALGO, TRUNC, ITEMS, VEC>(c, p, lane);
+    const long long i0 = tile * TILE + (long long)tid * ITEMS;
+    const long long n0 = locate(c, p, i0);
+    load_flags_global<ALGO, TRUNC, ITEMS, VEC>(c, p, i0, lane);
     Vals<ITEMS> v;
-    load_values_global<ALGO, TRUNC, ITEMS, VEC>(c, v, p, lane);
-    issue_boot(c, p);
-    issue_trunc_values(c, p);
+    load_values_global<ALGO, TRUNC, ITEMS, VEC>(c, v, p, i0, lane);
+    issue_boot(c, p, n0);
+    issue_trunc_values(c, p, i0);
     unsigned epoch = 0;
     if (p.carry_mode && tid < 32) epoch = ld_volatile_u32(p.header);
-    tile_compute<ALGO, TRUNC, VEC, THREADS, ITEMS>(c, v, p, s, epoch, sm, 0, NoHook{});
+    tile_compute<ALGO, TRUNC, VEC, THREADS, ITEMS>(c, v, p, i0, s, epoch, sm, 0, NoHook{});
     close_call(p);
 }
 
@@ -761,8 +761,9 @@ __device__ __forceinline__ void prefetch_flags(Chunk<ALGO, TRUNC, ITEMS>& c, con
     constexpr int W = ITEMS / 4;
     using L = StageLayout<ALGO, TRUNC, TILE>;
     const int tid = threadIdx.x;
-    locate(c, p, tile * TILE + (long long)tid * ITEMS);
-    issue_boot(c, p);
+    const long long i0 = tile * TILE + (long long)tid * ITEMS;
+    const long long n0 = locate(c, p, i0);
+    issue_boot(c, p, n0);
     if (tile * TILE + TILE + HALO <= p.total) {
         wait_stage<STAGES>(full_bar, cj, p, gave_up);
         unsigned char* stage = ring + (size_t)(cj % STAGES) * L::BYTES;
@@ -776,22 +777,23 @@ __device__ __forceinline__ void prefetch_flags(Chunk<ALGO, TRUNC, ITEMS>& c, con
         }
         if constexpr (TRUNC) lds_mask<ITEMS>(L::m(stage, 1) + 16 + tid * ITEMS, c.tw);
     } else {
-        load_flags_global<ALGO, TRUNC, ITEMS, true>(c, p, tid & 31);
+        load_flags_global<ALGO, TRUNC, ITEMS, true>(c, p, i0, tid & 31);
     }
-    issue_trunc_values(c, p);
+    issue_trunc_values(c, p, i0);
 }
 
 // ------------------------------------------------------------------------------------------ kernel 2: persistent, bulk-copy ring
-// Per-block walk state of the persistent kernel.
+// Per-block walk state of the persistent kernel (scan-order tile indices fit 32 bits: the grid of
+// the one-tile-per-block kernel bounds num_tiles).  The producer's cursor lives in shared memory:
+// only thread 0 uses it.
 struct Walk {
-    long long G;             // grid size = stride of the walk in scan-order tiles
-    long long s;             // scan-order tile being processed
-    long long ps;            // producer (thread 0): next scan-order tile to fetch
-    unsigned pj;             // producer: tiles fetched so far
+    unsigned G;              // grid size = stride of the walk in scan-order tiles
+    unsigned s;              // scan-order tile being processed
     unsigned cj;             // bulk-fetched tiles consumed so far
     unsigned epoch;
     int buf;                 // parity of the block-scan scratch
     bool gave_up;            // a bounded wait ran out: stop waiting, finish the walk
+    unsigned* prod;          // shared: [0] = next scan-order tile to fetch, [1] = tiles fetched so far
 };
 
 template <int ALGO, int TILE>
@@ -810,12 +812,14 @@ __device__ __forceinline__ void produce_next(const ScanParams& p, Walk& w, unsig
     constexpr bool FWD = is_forward(ALGO);
     constexpr int HALO = float_halo(ALGO) ? 4 : 0;
     using L = StageLayout<ALGO, TRUNC, TILE>;
-    while (w.ps < p.num_tiles) {
-        const long long tile = tile_of<ALGO, TILE>(p, w.ps);
-        w.ps += w.G;
+    unsigned ps = w.prod[0];
+    const unsigned pj = w.prod[1];
+    while (ps < p.num_tiles) {
+        const long long tile = tile_of<ALGO, TILE>(p, ps);
+        ps += w.G;
         if (!bulk_ok<ALGO, TILE>(p, tile)) continue;
-        unsigned char* stage = ring + (size_t)(w.pj % STAGES) * L::BYTES;
-        uint64_t* bar = &full_bar[w.pj % STAGES];
+        unsigned char* stage = ring + (size_t)(pj % STAGES) * L::BYTES;
+        uint64_t* bar = &full_bar[pj % STAGES];
         const long long e0 = tile * TILE;
         // forward scans fetch the 16 mask bytes before the tile as well (the preceding step's flag)
         const bool pre = FWD && uses_dones(ALGO) && e0 >= 16;
@@ -828,41 +832,47 @@ __device__ __forceinline__ void produce_next(const ScanParams& p, Walk& w, unsig
         if constexpr (uses_dones(ALGO))
             bulk_load(L::m(stage, 0) + (pre ? 0 : 16), p.dones + e0 - (pre ? 16 : 0), dbytes, bar);
         if constexpr (TRUNC) bulk_load(L::m(stage, 1) + 16, p.truncs + e0, TILE, bar);
-        ++w.pj;
+        w.prod[0] = ps;
+        w.prod[1] = pj + 1;
         return;
     }
+    w.prod[0] = ps;
 }
 
-template <int ALGO, bool TRUNC, int TILE, int STAGES>
-struct Refill {
+// Runs right after the block barrier of a tile, when every thread has consumed the current ring
+// stage and its flags: thread 0 refills the stage, and every thread fetches the flags of the
+// block's next tile (mask bytes from the ring, truncation / window-edge bootstrap values from global
+// memory) so that those dependent loads are in flight during the rest of the current tile.
+template <int ALGO, bool TRUNC, int THREADS, int ITEMS, int STAGES>
+struct AfterBarrier {
     const ScanParams& p;
     Walk& w;
     unsigned char* ring;
     uint64_t* full_bar;
-    bool active;
-    // After the block barrier every thread has read the current stage: thread 0 refills it.
+    Chunk<ALGO, TRUNC, ITEMS>& nxt;
+    bool bulk;               // the current tile came through the ring
     __device__ __forceinline__ void operator()() const {
-        if (active && threadIdx.x == 0) {
+        constexpr int TILE = THREADS * ITEMS;
+        if (bulk && threadIdx.x == 0) {
             fence_proxy_async();
             produce_next<ALGO, TRUNC, TILE, STAGES>(p, w, ring, full_bar);
         }
+        if (w.s + w.G < p.num_tiles)
+            prefetch_flags<ALGO, TRUNC, THREADS, ITEMS, STAGES>(nxt, p, tile_of<ALGO, TILE>(p, w.s + w.G), ring, full_bar,
+                                                                w.cj + (bulk ? 1u : 0u), w.gave_up);
     }
 };
 
-// One tile of the walk: `cur` holds the flags of tile w.s (fetched during the previous step), `nxt`
-// receives those of tile w.s + G now, so that its dependent loads (truncation and window-edge
-// bootstrap values) have a whole tile's time to arrive.
+// One tile of the walk.  `cur` holds the flags of tile w.s (fetched during the previous tile).
 template <int ALGO, bool TRUNC, int THREADS, int ITEMS, int STAGES>
-__device__ __forceinline__ void walk_step(Chunk<ALGO, TRUNC, ITEMS>& cur, Chunk<ALGO, TRUNC, ITEMS>& nxt,
-                                          const ScanParams& p, Walk& w, unsigned char* ring, uint64_t* full_bar,
-                                          ScanSmem<THREADS / 32>& sm) {
+__device__ __forceinline__ void walk_step(Chunk<ALGO, TRUNC, ITEMS>& cur, const ScanParams& p, Walk& w,
+                                          unsigned char* ring, uint64_t* full_bar, ScanSmem<THREADS / 32>& sm) {
     constexpr int TILE = THREADS * ITEMS;
     using L = StageLayout<ALGO, TRUNC, TILE>;
     const int tid = threadIdx.x;
-    const bool bulk = bulk_ok<ALGO, TILE>(p, tile_of<ALGO, TILE>(p, w.s));
-    if (w.s + w.G < p.num_tiles)
-        prefetch_flags<ALGO, TRUNC, THREADS, ITEMS, STAGES>(nxt, p, tile_of<ALGO, TILE>(p, w.s + w.G), ring, full_bar,
-                                                            w.cj + (bulk ? 1u : 0u), w.gave_up);
+    const long long tile = tile_of<ALGO, TILE>(p, w.s);
+    const long long i0 = tile * TILE + (long long)tid * ITEMS;
+    const bool bulk = bulk_ok<ALGO, TILE>(p, tile);
     Vals<ITEMS> v;
     if (bulk) {
         unsigned char* stage = ring + (size_t)(w.cj % STAGES) * L::BYTES;     // landed: prefetch_flags waited for it
@@ -879,10 +889,12 @@ __device__ __forceinline__ void walk_step(Chunk<ALGO, TRUNC, ITEMS>& cur, Chunk<
             v.halo_lr = L::f(stage, L::SLOT_F3)[off + ITEMS];
         }
     } else {
-        load_values_global<ALGO, TRUNC, ITEMS, true>(cur, v, p, tid & 31);
+        load_values_global<ALGO, TRUNC, ITEMS, true>(cur, v, p, i0, tid & 31);
     }
-    tile_compute<ALGO, TRUNC, true, THREADS, ITEMS>(cur, v, p, w.s, w.epoch, sm, w.buf,
-                                                    Refill<ALGO, TRUNC, TILE, STAGES>{p, w, ring, full_bar, bulk});
+    Chunk<ALGO, TRUNC, ITEMS> nxt;
+    tile_compute<ALGO, TRUNC, true, THREADS, ITEMS>(cur, v, p, i0, w.s, w.epoch, sm, w.buf,
+                                                    AfterBarrier<ALGO, TRUNC, THREADS, ITEMS, STAGES>{p, w, ring, full_bar, nxt, bulk});
+    if (w.s + w.G < p.num_tiles) cur = nxt;
     if (bulk) ++w.cj;
     w.s += w.G;
     w.buf ^= 1;
@@ -898,17 +910,19 @@ __global__ void __launch_bounds__(THREADS, MIN_BLOCKS) scan_kernel_tma(const Sca
     __shared__ ScanSmem<THREADS / 32> sm;
 
     const int tid = threadIdx.x;
+    __shared__ unsigned prod[2];
     Walk w;
     w.G = gridDim.x;
     w.s = blockIdx.x;
-    w.ps = blockIdx.x;
-    w.pj = 0;
+    w.prod = prod;
     w.cj = 0;
     w.epoch = 0;
     w.buf = 0;
     w.gave_up = false;
 
     if (tid == 0) {
+        prod[0] = blockIdx.x;
+        prod[1] = 0;
 #pragma unroll
         for (int k = 0; k < STAGES; ++k) mbar_init(&full_bar[k], 1);
         fence_barrier_init();
@@ -921,15 +935,10 @@ __global__ void __launch_bounds__(THREADS, MIN_BLOCKS) scan_kernel_tma(const Sca
     }
     if (p.carry_mode && tid < 32) w.epoch = ld_volatile_u32(p.header);
 
-    // Two flag sets alternate between "current" and "next" so that no register copies are needed.
-    Chunk<ALGO, TRUNC, ITEMS> fa, fb;
+    Chunk<ALGO, TRUNC, ITEMS> cur;
     if (w.s < p.num_tiles)
-        prefetch_flags<ALGO, TRUNC, THREADS, ITEMS, STAGES>(fa, p, tile_of<ALGO, TILE>(p, w.s), ring, full_bar, w.cj, w.gave_up);
-    while (w.s < p.num_tiles) {
-        walk_step<ALGO, TRUNC, THREADS, ITEMS, STAGES>(fa, fb, p, w, ring, full_bar, sm);
-        if (w.s >= p.num_tiles) break;
-        walk_step<ALGO, TRUNC, THREADS, ITEMS, STAGES>(fb, fa, p, w, ring, full_bar, sm);
-    }
+        prefetch_flags<ALGO, TRUNC, THREADS, ITEMS, STAGES>(cur, p, tile_of<ALGO, TILE>(p, w.s), ring, full_bar, w.cj, w.gave_up);
+    while (w.s < p.num_tiles) walk_step<ALGO, TRUNC, THREADS, ITEMS, STAGES>(cur, p, w, ring, full_bar, sm);
     close_call(p);
 }
 
