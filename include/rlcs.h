@@ -67,7 +67,8 @@ typedef enum {
     RLCS_ERR_ALIGN = 4,      /* fp32 pointer not 4-byte aligned, workspace not 16-byte aligned */
     RLCS_ERR_WORKSPACE = 5,  /* workspace NULL or too small for this (N, T) */
     RLCS_ERR_CUDA = 6,       /* the launch itself failed (cudaGetLastError) */
-    RLCS_ERR_TIMEOUT = 7     /* device status: a bounded carry wait gave up */
+    RLCS_ERR_TIMEOUT = 7,    /* device status: a bounded carry wait gave up */
+    RLCS_ERR_LIMIT = 8       /* rlcs_gae_no_alloc: the problem needs more scratch than the built-in array holds */
 } rlcs_status_t;
 
 /* Human-readable name of a status code (static storage, never NULL). */
@@ -159,6 +160,37 @@ int rlcs_elig_trace(const float* x, const uint8_t* dones, float* traces, int64_t
  */
 int rlcs_episodic_prefix_sum(const float* x, const uint8_t* dones, float* sums, int64_t N, int64_t T,
                              int starts_at, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * GAE without any workspace argument, for callers that cannot allocate device memory.  (The paper
+ * has no counterpart: its library allocates through PyTorch.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- inside a stream capture or other
+ * region in which the driver refuses allocation, in a process whose memory was handed out
+ * completely to a pool up front, or in a real-time control loop that must not take the allocator's
+ * locks -- and that cannot carve a workspace for rlcs_gae out of memory it already owns.  Same
+ * arguments and results as rlcs_gae; the scratch for the carry between thread blocks lives in a
+ * fixed 1 MiB device array inside the library (rlcs_no_alloc_scratch_bytes()), which every GPU
+ * that loads the library holds until the process exits.  The call itself allocates nothing: no
+ * cudaMalloc, no cudaFree, no allocating library routine.
+ *
+ * Limit: rlcs_workspace_bytes(N, T) must not exceed that array, i.e. N*T <= 33.5 million steps
+ * (unlimited when T divides 512, where no scratch is used); larger problems return RLCS_ERR_LIMIT
+ * and launch nothing.
+ * First call on a device: looks up the array's device address (cudaGetSymbolAddress) and
+ * initialises it with two small memsets on `cuda_stream`; make this first call outside any stream
+ * capture, with the device current that later calls will use.
+ * Sharing: every call on a device uses the same array, which keeps what the last call left; the
+ * entry point re-zeroes the words that must start at zero.  Calls that can overlap on the GPU
+ * (different streams without ordering, several host threads) race on it and give wrong results:
+ * keep them ordered, or use rlcs_gae with separate workspaces.
+ */
+int rlcs_gae_no_alloc(const float* rewards, const float* values, const uint8_t* dones, const uint8_t* truncs,
+                      const float* trunc_bootstrap, const float* bootstrap, float* advantages, float* returns,
+                      int64_t N, int64_t T, float gamma, float lambda, void* cuda_stream);
+
+/* Size in bytes of the built-in scratch array used by rlcs_gae_no_alloc. */
+size_t rlcs_no_alloc_scratch_bytes(void);
 
 /*
  * Test hook: the bare scan of Eq. 1 / Eq. 2 on caller-supplied coefficients, every row with

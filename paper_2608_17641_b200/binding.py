@@ -15,7 +15,7 @@ LIB_PATH = os.path.join(_PKG, "librlcs.so")
 
 RLCS_OK = 0
 RLCS_ERR_NULL, RLCS_ERR_SIZE, RLCS_ERR_ARG, RLCS_ERR_ALIGN = 1, 2, 3, 4
-RLCS_ERR_WORKSPACE, RLCS_ERR_CUDA, RLCS_ERR_TIMEOUT = 5, 6, 7
+RLCS_ERR_WORKSPACE, RLCS_ERR_CUDA, RLCS_ERR_TIMEOUT, RLCS_ERR_LIMIT = 5, 6, 7, 8
 
 _vp, _i64, _f, _sz, _int = ctypes.c_void_p, ctypes.c_int64, ctypes.c_float, ctypes.c_size_t, ctypes.c_int
 _TAIL = [_vp, _sz, _vp]          # workspace, workspace_bytes, cuda_stream
@@ -33,6 +33,8 @@ SIGNATURES = {
     "rlcs_discounted_return": ([_vp] * 6 + [_i64, _i64, _f] + _TAIL, _int),
     "rlcs_elig_trace": ([_vp] * 3 + [_i64, _i64, _f, _f] + _TAIL, _int),
     "rlcs_episodic_prefix_sum": ([_vp] * 3 + [_i64, _i64, _int] + _TAIL, _int),
+    "rlcs_gae_no_alloc": ([_vp] * 8 + [_i64, _i64, _f, _f, _vp], _int),
+    "rlcs_no_alloc_scratch_bytes": ([], _sz),
     "rlcs_affine_scan": ([_vp] * 3 + [_i64, _i64, _int] + _TAIL, _int),
     "rlcs_debug_set_tile_variant": ([_int], _int),
     "rlcs_debug_tile_elems": ([_int], _int),
@@ -143,6 +145,22 @@ def rlcs_gae(rewards, values, dones, truncs=None, trunc_bootstrap=None, bootstra
                           _ptr(truncs, "u8", (N, T)), _ptr(trunc_bootstrap, "f32", (N, T)),
                           _ptr(bootstrap, "f32", (N,)), _ptr(adv, "f32", (N, T)), _ptr(ret, "f32", (N, T)),
                           N, T, gamma, lam, wp, wb, _stream(stream)))
+    return (adv, ret) if want_returns else adv
+
+
+def rlcs_gae_no_alloc(rewards, values, dones, truncs=None, trunc_bootstrap=None, bootstrap=None, *, gamma, lam,
+                      advantages=None, returns=None, want_returns=True, stream=None):
+    """GAE through the entry point that takes no workspace: the carry scratch is a fixed device
+    array inside the library, so this call path performs no device allocation (pass `advantages`
+    and `returns` to keep torch from allocating the outputs either).  Calls must not overlap on
+    the GPU; the first call on a device should happen outside stream capture."""
+    N, T = rewards.shape
+    adv = _out(rewards, advantages)
+    ret = (_out(rewards, returns) if want_returns else None)
+    _check(lib().rlcs_gae_no_alloc(_ptr(rewards, "f32"), _ptr(values, "f32", (N, T)), _ptr(dones, "u8", (N, T)),
+                                   _ptr(truncs, "u8", (N, T)), _ptr(trunc_bootstrap, "f32", (N, T)),
+                                   _ptr(bootstrap, "f32", (N,)), _ptr(adv, "f32", (N, T)), _ptr(ret, "f32", (N, T)),
+                                   N, T, gamma, lam, _stream(stream)))
     return (adv, ret) if want_returns else adv
 
 

@@ -130,6 +130,7 @@ const char* rlcs_status_string(int status) {
         case RLCS_ERR_WORKSPACE: return "RLCS_ERR_WORKSPACE: workspace missing or too small";
         case RLCS_ERR_CUDA: return "RLCS_ERR_CUDA: CUDA call failed";
         case RLCS_ERR_TIMEOUT: return "RLCS_ERR_TIMEOUT: bounded carry wait gave up";
+        case RLCS_ERR_LIMIT: return "RLCS_ERR_LIMIT: problem too large for the built-in scratch array of rlcs_gae_no_alloc";
         default: return "RLCS: unknown status";
     }
 }
