@@ -12,7 +12,8 @@
  *
  * Pointers.  Every pointer except `cuda_stream` is a DEVICE pointer.  The caller owns every
  *   buffer, including `workspace`; the library allocates nothing and keeps no state between
- *   calls.  Outputs must not overlap inputs or each other.
+ *   calls (apart from a per-device cache of launch configurations).  Outputs must not overlap
+ *   inputs or each other.
  * Layout.  Every [N, T] tensor is contiguous row-major: element (n, t) at index n*T + t.
  *   Floating-point tensors are fp32 (Section 4.4: the method is fp32-only).  Masks are uint8,
  *   zero = false, any non-zero value = true.
@@ -45,8 +46,9 @@
  *   before anything is launched.  The only device-side wait is the bounded carry wait between
  *   thread blocks; if it ever gives up, the kernel still terminates normally, the outputs of that
  *   call are unspecified, and rlcs_last_device_status reports RLCS_ERR_TIMEOUT.
- * Inputs are assumed finite.  Resets are applied by selection, not by multiplying with zero, so
- *   a non-finite value inside one episode cannot leak into a neighbouring episode.
+ * Inputs must be finite.  A reset is a decay of exactly 0 inside the scan (0 * finite severs
+ *   exactly); successor values at resets are selected, never multiplied.  A NaN or infinity in one
+ *   episode can therefore reach the flagged last step of the preceding episode, but nothing else.
  * Results are deterministic: the same inputs give bit-identical outputs on every call.
  */
 #ifndef RLCS_H_
