@@ -33,9 +33,9 @@
  * Sizes.  N >= 0, 0 <= T < 2^31, N*T < 2^40.  N == 0 or T == 0 returns RLCS_OK without a launch.
  * Parameters.  gamma and lambda must lie in [0, 1] (1 is valid); clip thresholds must be >= 0
  *   (+inf = no clipping).  NaN is rejected.
- * Alignment.  fp32 pointers must be 4-byte aligned.  When every fp32 pointer is 16-byte aligned
- *   and every mask pointer 8-byte aligned the vectorised kernels run; otherwise a slower
- *   element-wise variant of the same kernel is used (same results).
+ * Alignment.  fp32 pointers must be 4-byte aligned.  When every fp32 pointer is 32-byte aligned
+ *   and every mask pointer 16-byte aligned the vectorised kernels run (256-bit accesses, bulk
+ *   copies); otherwise a slower element-wise variant of the same kernel is used (same results).
  * Workspace.  Rows that straddle the kernels' tiles need a carry between thread blocks, passed
  *   through `workspace`: at least rlcs_workspace_bytes(N, T) bytes, 16-byte aligned, initialised
  *   once with rlcs_workspace_init and then reusable by any number of calls, of any of the entry

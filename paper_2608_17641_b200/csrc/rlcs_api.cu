@@ -49,7 +49,7 @@ int check_alignment(const Ptrs& ps, bool* vec) {
     *vec = true;
     for (int i = 0; i < ps.nf32; ++i) {
         if (!aligned(ps.f32[i], 4)) return RLCS_ERR_ALIGN;
-        if (!aligned(ps.f32[i], 16)) *vec = false;
+        if (!aligned(ps.f32[i], 32)) *vec = false;          // 256-bit vector accesses
     }
     for (int i = 0; i < ps.nu8; ++i)
         if (!aligned(ps.u8[i], 16)) *vec = false;

@@ -103,14 +103,39 @@ __device__ __forceinline__ Pair apply(Pair x, Pair acc) {
 }
 
 // ------------------------------------------------------------------------------------------ global loads / stores
+// 256-bit global accesses (sm_100): one instruction moves a thread's 8 consecutive fp32 values, so a
+// warp touches 1 KiB of whole 32-byte sectors per instruction.  32-byte aligned addresses only.
+__device__ __forceinline__ void ldg_v8(const float* p, float* x) {
+    asm volatile("ld.global.nc.L1::no_allocate.v8.f32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=f"(x[0]), "=f"(x[1]), "=f"(x[2]), "=f"(x[3]), "=f"(x[4]), "=f"(x[5]), "=f"(x[6]), "=f"(x[7])
+                 : "l"(p));
+}
+__device__ __forceinline__ void stg_v8(float* p, const float* x) {
+    asm volatile("st.global.cs.v8.f32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+                 :: "l"(p), "f"(x[0]), "f"(x[1]), "f"(x[2]), "f"(x[3]), "f"(x[4]), "f"(x[5]), "f"(x[6]), "f"(x[7])
+                 : "memory");
+}
+// Load *p if pred, else keep 0: a predicated load instead of a branch around a load.
+__device__ __forceinline__ float ldg_if(const float* p, bool pred) {
+    float v = 0.f;
+    asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.u32 q, %2, 0;\n\t@q ld.global.nc.f32 %0, [%1];\n\t}"
+                 : "+f"(v) : "l"(p), "r"((unsigned)pred));
+    return v;
+}
+
 template <int ITEMS, bool VEC>
 __device__ __forceinline__ void load_f32(const float* __restrict__ p, long long i0, int nvalid, float (&x)[ITEMS]) {
     if (VEC && nvalid == ITEMS) {
-        const float4* q = reinterpret_cast<const float4*>(p + i0);
+        if constexpr (ITEMS % 8 == 0) {
 #pragma unroll
-        for (int k = 0; k < ITEMS / 4; ++k) {
-            float4 v = __ldcs(q + k);
-            x[4 * k + 0] = v.x; x[4 * k + 1] = v.y; x[4 * k + 2] = v.z; x[4 * k + 3] = v.w;
+            for (int k = 0; k < ITEMS / 8; ++k) ldg_v8(p + i0 + 8 * k, &x[8 * k]);
+        } else {
+            const float4* q = reinterpret_cast<const float4*>(p + i0);
+#pragma unroll
+            for (int k = 0; k < ITEMS / 4; ++k) {
+                float4 v = __ldcs(q + k);
+                x[4 * k + 0] = v.x; x[4 * k + 1] = v.y; x[4 * k + 2] = v.z; x[4 * k + 3] = v.w;
+            }
         }
     } else {
 #pragma unroll
@@ -145,10 +170,15 @@ __device__ __forceinline__ void load_mask(const uint8_t* __restrict__ p, long lo
 template <int ITEMS, bool VEC>
 __device__ __forceinline__ void store_f32(float* __restrict__ p, long long i0, int nvalid, const float (&x)[ITEMS]) {
     if (VEC && nvalid == ITEMS) {
-        float4* q = reinterpret_cast<float4*>(p + i0);
+        if constexpr (ITEMS % 8 == 0) {
 #pragma unroll
-        for (int k = 0; k < ITEMS / 4; ++k)
-            __stcs(q + k, make_float4(x[4 * k + 0], x[4 * k + 1], x[4 * k + 2], x[4 * k + 3]));
+            for (int k = 0; k < ITEMS / 8; ++k) stg_v8(p + i0 + 8 * k, &x[8 * k]);
+        } else {
+            float4* q = reinterpret_cast<float4*>(p + i0);
+#pragma unroll
+            for (int k = 0; k < ITEMS / 4; ++k)
+                __stcs(q + k, make_float4(x[4 * k + 0], x[4 * k + 1], x[4 * k + 2], x[4 * k + 3]));
+        }
     } else {
 #pragma unroll
         for (int j = 0; j < ITEMS; ++j)
@@ -333,22 +363,23 @@ template <int ALGO, bool TRUNC, int ITEMS>
 __device__ __forceinline__ void issue_boot(Chunk<ALGO, TRUNC, ITEMS>& c, const ScanParams& p, long long n0) {
     c.boot_first = 0.f;
     if constexpr (!is_forward(ALGO) && !is_affine(ALGO)) {
-        if (p.boot != nullptr && c.edge < (unsigned)c.nvalid) c.boot_first = __ldg(p.boot + n0);
+        c.boot_first = ldg_if(p.boot + n0, p.boot != nullptr && c.edge < (unsigned)c.nvalid);
     }
 }
 
 // Mask bytes from global memory; forward scans also need the dones byte just before the chunk.
-template <int ALGO, bool TRUNC, int ITEMS, bool VEC>
+template <int ALGO, bool TRUNC, int ITEMS, bool VEC, bool FULL = false>
 __device__ __forceinline__ void load_flags_global(Chunk<ALGO, TRUNC, ITEMS>& c, const ScanParams& p, long long i0, int lane) {
     constexpr int W = ITEMS / 4;
+    const int nvalid = FULL ? ITEMS : c.nvalid;
 #pragma unroll
     for (int k = 0; k < W; ++k) { c.dw[k] = 0; c.tw[k] = 0; }
     c.halo_d = 0;
     if constexpr (ALGO == kElig || ALGO == kPrefix) {
-        if (lane == 0 && i0 > 0 && c.nvalid > 0) c.halo_d = __ldg(p.dones + i0 - 1);
+        if (lane == 0 && i0 > 0 && nvalid > 0) c.halo_d = __ldg(p.dones + i0 - 1);
     }
-    if constexpr (uses_dones(ALGO)) load_mask<ITEMS, VEC>(p.dones, i0, c.nvalid, c.dw);
-    if constexpr (TRUNC) load_mask<ITEMS, VEC>(p.truncs, i0, c.nvalid, c.tw);
+    if constexpr (uses_dones(ALGO)) load_mask<ITEMS, VEC>(p.dones, i0, nvalid, c.dw);
+    if constexpr (TRUNC) load_mask<ITEMS, VEC>(p.truncs, i0, nvalid, c.tw);
     if constexpr (ALGO == kElig || ALGO == kPrefix) {
         const unsigned nb = __shfl_up_sync(0xffffffffu, c.dw[W - 1] >> 24, 1);
         if (lane != 0) c.halo_d = nb;
@@ -363,25 +394,26 @@ __device__ __forceinline__ void issue_trunc_values(Chunk<ALGO, TRUNC, ITEMS>& c,
     if constexpr (TRUNC) {
 #pragma unroll
         for (int j = 0; j < ITEMS; ++j)
-            if (test_byte(c.tw, j) && !test_byte(c.dw, j)) c.ov[j] = __ldg(p.trunc_boot + i0 + j);
+            c.ov[j] = ldg_if(p.trunc_boot + i0 + j, test_byte(c.tw, j) && !test_byte(c.dw, j));
     }
 }
 
 // Float inputs from global memory, with the one-step halo (lane 31 loads it, the others take
 // their neighbour's first element).
-template <int ALGO, bool TRUNC, int ITEMS, bool VEC>
+template <int ALGO, bool TRUNC, int ITEMS, bool VEC, bool FULL = false>
 __device__ __forceinline__ void load_values_global(const Chunk<ALGO, TRUNC, ITEMS>& c, Vals<ITEMS>& v, const ScanParams& p, long long i0, int lane) {
-    load_f32<ITEMS, VEC>(p.f0, i0, c.nvalid, v.a);
-    if constexpr (uses_f1(ALGO)) load_f32<ITEMS, VEC>(p.f1, i0, c.nvalid, v.x1);
-    if constexpr (uses_f2(ALGO)) load_f32<ITEMS, VEC>(p.f2, i0, c.nvalid, v.x2);
-    if constexpr (uses_f3(ALGO)) load_f32<ITEMS, VEC>(p.f3, i0, c.nvalid, v.x3);
+    const int nvalid = FULL ? ITEMS : c.nvalid;
+    load_f32<ITEMS, VEC>(p.f0, i0, nvalid, v.a);
+    if constexpr (uses_f1(ALGO)) load_f32<ITEMS, VEC>(p.f1, i0, nvalid, v.x1);
+    if constexpr (uses_f2(ALGO)) load_f32<ITEMS, VEC>(p.f2, i0, nvalid, v.x2);
+    if constexpr (uses_f3(ALGO)) load_f32<ITEMS, VEC>(p.f3, i0, nvalid, v.x3);
     v.halo = 0.f;
     v.halo_lr = 0.f;
     if constexpr (float_halo(ALGO)) {
         const float* src = (ALGO == kRetrace) ? p.f2 : p.f1;
         const bool edge_lane = (lane == 31) && (p.total - i0 > ITEMS);
-        if (edge_lane) v.halo = __ldg(src + i0 + ITEMS);
-        if constexpr (ALGO == kRetrace) if (edge_lane) v.halo_lr = __ldg(p.f3 + i0 + ITEMS);
+        v.halo = ldg_if(src + i0 + ITEMS, edge_lane);
+        if constexpr (ALGO == kRetrace) v.halo_lr = ldg_if(p.f3 + i0 + ITEMS, edge_lane);
         const float first = (ALGO == kRetrace) ? v.x2[0] : v.x1[0];
         const float nb = __shfl_down_sync(0xffffffffu, first, 1);
         if (lane != 31) v.halo = nb;
@@ -407,17 +439,20 @@ struct NoHook {
 
 // Steps 2-5 of the header comment for one tile, given the thread's loaded Chunk.
 // `after_barrier` runs right after the block barrier (every thread has consumed its inputs).
-template <int ALGO, bool TRUNC, bool VEC, int THREADS, int ITEMS, class Hook>
+// FULL: the tile lies completely inside the array and rows are at least ITEMS long (block-uniform),
+// which removes the ragged-chunk and short-row side paths at compile time.
+template <int ALGO, bool TRUNC, bool VEC, int THREADS, int ITEMS, bool FULL, class Hook>
 __device__ __forceinline__ void tile_compute(Chunk<ALGO, TRUNC, ITEMS>& c, Vals<ITEMS>& v, const ScanParams& p, long long i0, long long s,
                                              unsigned epoch, ScanSmem<THREADS / 32>& sm, int buf, Hook after_barrier) {
     constexpr bool FWD = is_forward(ALGO);
     constexpr int NW = THREADS / 32;
     constexpr int W = ITEMS / 4;
-    constexpr unsigned FULL = 0xffffffffu;
+    constexpr unsigned ALL = 0xffffffffu;
     const int tid = threadIdx.x;
     const int lane = tid & 31;
     const int warp = tid >> 5;
     const bool has_edge = c.edge < (unsigned)ITEMS;
+    const int nvalid = FULL ? ITEMS : c.nvalid;
 
     // ---- reset words: byte j non-zero = the recurrence does NOT continue from step j to its
     // scan-order predecessor (t+1 backward, t-1 forward): a flag, a row edge, a step beyond the array
@@ -440,19 +475,21 @@ __device__ __forceinline__ void tile_compute(Chunk<ALGO, TRUNC, ITEMS>& c, Vals<
         for (int k = 0; k < W; ++k) sev[k] = c.dw[k] | c.tw[k];
     }
     if (has_edge) mark_byte_dyn(sev, c.edge);
-    if (p.T < (unsigned)ITEMS) {                // rows shorter than a chunk: several edges
-        for (unsigned e = c.edge + p.T; e < (unsigned)ITEMS; e += p.T) mark_byte_dyn(sev, e);
-    }
-    if (c.nvalid < ITEMS) {                     // ragged end of the array
-        for (unsigned j = c.nvalid; j < (unsigned)ITEMS; ++j) mark_byte_dyn(sev, j);
+    if constexpr (!FULL) {
+        if (p.T < (unsigned)ITEMS) {            // rows shorter than a chunk: several edges
+            for (unsigned e = c.edge + p.T; e < (unsigned)ITEMS; e += p.T) mark_byte_dyn(sev, e);
+        }
+        if (nvalid < ITEMS) {                   // ragged end of the array
+            for (unsigned j = nvalid; j < (unsigned)ITEMS; ++j) mark_byte_dyn(sev, j);
+        }
     }
 
     // ---- window-edge bootstrap into ov at the row's last step, unless that step carries a flag
     // (static indexing only, so that ov stays in registers)
     if constexpr (!FWD && !is_affine(ALGO)) {
         if (has_edge && p.boot != nullptr) {
-            if (p.T >= (unsigned)ITEMS) {       // at most one row edge in the chunk; its bootstrap was fetched early
-                const bool ok = c.edge < (unsigned)c.nvalid && !test_byte_dyn(c.dw, c.edge) && !test_byte_dyn(c.tw, c.edge);
+            if (FULL || p.T >= (unsigned)ITEMS) {   // at most one row edge in the chunk; its bootstrap was fetched early
+                const bool ok = c.edge < (unsigned)nvalid && !test_byte_dyn(c.dw, c.edge) && !test_byte_dyn(c.tw, c.edge);
 #pragma unroll
                 for (int j = 0; j < ITEMS; ++j) c.ov[j] = (ok && (unsigned)j == c.edge) ? c.boot_first : c.ov[j];
             } else {                            // rows shorter than a chunk: walk the steps
@@ -461,7 +498,7 @@ __device__ __forceinline__ void tile_compute(Chunk<ALGO, TRUNC, ITEMS>& c, Vals<
 #pragma unroll
                 for (int j = 0; j < ITEMS; ++j) {
                     if ((unsigned)j == e) {
-                        if (j < c.nvalid && !test_byte(c.dw, j) && !test_byte(c.tw, j)) c.ov[j] = __ldg(p.boot + n);
+                        if (j < nvalid && !test_byte(c.dw, j) && !test_byte(c.tw, j)) c.ov[j] = __ldg(p.boot + n);
                         e += p.T;
                         ++n;
                     }
@@ -541,21 +578,21 @@ __device__ __forceinline__ void tile_compute(Chunk<ALGO, TRUNC, ITEMS>& c, Vals<
     for (int d = 1; d < 32; d <<= 1) {
         Pair o;
         if constexpr (FWD) {
-            o.a = __shfl_up_sync(FULL, incl.a, d);
-            o.b = __shfl_up_sync(FULL, incl.b, d);
+            o.a = __shfl_up_sync(ALL, incl.a, d);
+            o.b = __shfl_up_sync(ALL, incl.b, d);
         } else {
-            o.a = __shfl_down_sync(FULL, incl.a, d);
-            o.b = __shfl_down_sync(FULL, incl.b, d);
+            o.a = __shfl_down_sync(ALL, incl.a, d);
+            o.b = __shfl_down_sync(ALL, incl.b, d);
         }
         if (rank >= d) incl = apply(incl, o);
     }
     Pair excl;     // everything earlier in scan order inside this warp
     if constexpr (FWD) {
-        excl.a = __shfl_up_sync(FULL, incl.a, 1);
-        excl.b = __shfl_up_sync(FULL, incl.b, 1);
+        excl.a = __shfl_up_sync(ALL, incl.a, 1);
+        excl.b = __shfl_up_sync(ALL, incl.b, 1);
     } else {
-        excl.a = __shfl_down_sync(FULL, incl.a, 1);
-        excl.b = __shfl_down_sync(FULL, incl.b, 1);
+        excl.a = __shfl_down_sync(ALL, incl.a, 1);
+        excl.b = __shfl_down_sync(ALL, incl.b, 1);
     }
     if (rank == 0) excl = Pair{0.f, 1.f};
 
@@ -576,14 +613,14 @@ __device__ __forceinline__ void tile_compute(Chunk<ALGO, TRUNC, ITEMS>& c, Vals<
 #pragma unroll
         for (int d = 1; d < NW; d <<= 1) {
             Pair o;
-            o.a = __shfl_up_sync(FULL, w.a, d);
-            o.b = __shfl_up_sync(FULL, w.b, d);
+            o.a = __shfl_up_sync(ALL, w.a, d);
+            o.b = __shfl_up_sync(ALL, w.b, d);
             if (lane >= d) w = apply(w, o);
         }
-        tile_agg.a = __shfl_sync(FULL, w.a, NW - 1);
-        tile_agg.b = __shfl_sync(FULL, w.b, NW - 1);
-        const float ca = __shfl_sync(FULL, w.a, (wrank + NW - 1) % NW);
-        const float cb = __shfl_sync(FULL, w.b, (wrank + NW - 1) % NW);
+        tile_agg.a = __shfl_sync(ALL, w.a, NW - 1);
+        tile_agg.b = __shfl_sync(ALL, w.b, NW - 1);
+        const float ca = __shfl_sync(ALL, w.a, (wrank + NW - 1) % NW);
+        const float cb = __shfl_sync(ALL, w.b, (wrank + NW - 1) % NW);
         if (wrank > 0) wcarry = Pair{ca, cb};
     }
     const Pair before = apply(excl, wcarry);   // everything earlier in scan order inside this tile
@@ -636,10 +673,10 @@ __device__ __forceinline__ void tile_compute(Chunk<ALGO, TRUNC, ITEMS>& c, Vals<
             prev = d;
         }
     }
-    if (c.nvalid > 0) {
-        store_f32<ITEMS, VEC>(p.out0, i0, c.nvalid, v.a);
+    if (nvalid > 0) {
+        store_f32<ITEMS, VEC>(p.out0, i0, nvalid, v.a);
         if constexpr (ALGO == kGae || ALGO == kVtrace) {
-            if (p.out1 != nullptr) store_f32<ITEMS, VEC>(p.out1, i0, c.nvalid, out1v);
+            if (p.out1 != nullptr) store_f32<ITEMS, VEC>(p.out1, i0, nvalid, out1v);
         }
     }
 }
@@ -659,6 +696,23 @@ __device__ __forceinline__ void close_call(const ScanParams& p) {
 }
 
 // ------------------------------------------------------------------------------------------ kernel 1: one tile per block
+template <int ALGO, bool TRUNC, bool VEC, int THREADS, int ITEMS, bool FULL>
+__device__ __forceinline__ void one_tile(const ScanParams& p, long long tile, long long s, unsigned epoch,
+                                         ScanSmem<THREADS / 32>& sm) {
+    constexpr int TILE = THREADS * ITEMS;
+    const int tid = threadIdx.x;
+    const int lane = tid & 31;
+    Chunk<ALGO, TRUNC, ITEMS> c;
+    const long long i0 = tile * TILE + (long long)tid * ITEMS;
+    const long long n0 = locate(c, p, i0);
+    load_flags_global<ALGO, TRUNC, ITEMS, VEC, FULL>(c, p, i0, lane);
+    Vals<ITEMS> v;
+    load_values_global<ALGO, TRUNC, ITEMS, VEC, FULL>(c, v, p, i0, lane);
+    issue_boot(c, p, n0);
+    issue_trunc_values(c, p, i0);
+    tile_compute<ALGO, TRUNC, VEC, THREADS, ITEMS, FULL>(c, v, p, i0, s, epoch, sm, 0, NoHook{});
+}
+
 template <int ALGO, bool TRUNC, bool VEC, int THREADS, int ITEMS, int MIN_BLOCKS>
 __global__ void __launch_bounds__(THREADS, MIN_BLOCKS) scan_kernel(const ScanParams p) {
     constexpr bool FWD = is_forward(ALGO);
@@ -670,17 +724,12 @@ __global__ void __launch_bounds__(THREADS, MIN_BLOCKS) scan_kernel(const ScanPar
     const long long s = blockIdx.x;                       // tile index in scan order
     const long long tile = FWD ? s : (p.num_tiles - 1 - s);
 
-    Chunk<ALGO, TRUNC, ITEMS> c;
-    const long long i0 = tile * TILE + (long long)tid * ITEMS;
-    const long long n0 = locate(c, p, i0);
-    load_flags_global<ALGO, TRUNC, ITEMS, VEC>(c, p, i0, lane);
-    Vals<ITEMS> v;
-    load_values_global<ALGO, TRUNC, ITEMS, VEC>(c, v, p, i0, lane);
-    issue_boot(c, p, n0);
-    issue_trunc_values(c, p, i0);
     unsigned epoch = 0;
     if (p.carry_mode && tid < 32) epoch = ld_volatile_u32(p.header);
-    tile_compute<ALGO, TRUNC, VEC, THREADS, ITEMS>(c, v, p, i0, s, epoch, sm, 0, NoHook{});
+    // block-uniform: the whole tile is inside the array and no row is shorter than a chunk
+    const bool full = (tile * TILE + TILE <= p.total) && (p.T >= (unsigned)ITEMS);
+    if (full) one_tile<ALGO, TRUNC, VEC, THREADS, ITEMS, true>(p, tile, s, epoch, sm);
+    else one_tile<ALGO, TRUNC, VEC, THREADS, ITEMS, false>(p, tile, s, epoch, sm);
     close_call(p);
 }
 
@@ -892,7 +941,7 @@ __device__ __forceinline__ void walk_step(Chunk<ALGO, TRUNC, ITEMS>& cur, const 
         load_values_global<ALGO, TRUNC, ITEMS, true>(cur, v, p, i0, tid & 31);
     }
     Chunk<ALGO, TRUNC, ITEMS> nxt;
-    tile_compute<ALGO, TRUNC, true, THREADS, ITEMS>(cur, v, p, i0, w.s, w.epoch, sm, w.buf,
+    tile_compute<ALGO, TRUNC, true, THREADS, ITEMS, false>(cur, v, p, i0, w.s, w.epoch, sm, w.buf,
                                                     AfterBarrier<ALGO, TRUNC, THREADS, ITEMS, STAGES>{p, w, ring, full_bar, nxt, bulk});
     if (w.s + w.G < p.num_tiles) cur = nxt;
     if (bulk) ++w.cj;
