@@ -427,6 +427,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sweep-only", action="store_true", help="print only the cold-L2 sweeps (one JSON line)")
     ap.add_argument("--variant", type=int, default=None, help="tile variant test hook (default: library default)")
+    ap.add_argument("--no-truncs", action="store_true", help="bench batch without per-step truncation handling")
     ap.add_argument("--rows", type=int, default=WORKLOAD["N"], help="num_envs of the bench batch (default: full size)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
@@ -462,6 +463,9 @@ def main():
 
     N = args.rows
     ro = workloads.config5(N=N, T=WORKLOAD["T"], salt=rank)        # every rank draws its own batch
+    if args.no_truncs:
+        ro.truncs = None
+        ro.trunc_bootstrap = None
     batch = GpuBatch(ro, torch.device("cuda", local))
     total_ms, per_algo_ms, launches, clocks = time_device(batch, args.steps, args.warmup, dist)
     total_ms = dist.max(total_ms)
@@ -477,7 +481,10 @@ def main():
         per_algo[a] = {"ms": round(ms, 5), "env_steps_per_s": ro.N * ro.T / (ms * 1e-3), "algorithmic_bytes": ab,
                        "gbs": round(gbs, 1), "frac_of_peak": round(gbs / peak, 4)}
     dom = max(ALGOS, key=lambda a: per_algo[a]["ms"])
-    roofline = {"bound": "hbm", "kernel": f"scan_kernel<{dom}, truncation handling, vectorised, 256 threads x 8 steps>",
+    vi = binding.rlcs_debug_variant_for(dom, ro.truncs is not None and dom not in ("elig_trace", "episodic_prefix_sum"), ro.N, ro.T)
+    kname = "scan_kernel_tma" if vi["ring_stages"] else "scan_kernel"
+    roofline = {"bound": "hbm", "kernel": f"{kname}<{dom}>, {vi['threads']} threads x {vi['steps_per_thread']} steps per tile "
+                                          f"(variant {vi['variant']})",
                 "achieved": per_algo[dom]["gbs"], "peak": peak, "unit": "GB/s",
                 "frac": round(per_algo[dom]["gbs"] / peak, 4), "traffic": NCU_TRAFFIC_BYTES.get(dom),
                 "algorithmic_bytes_per_launch": per_algo[dom]["algorithmic_bytes"], "peak_source": f"of {peak_kind}",

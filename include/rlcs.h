@@ -205,7 +205,7 @@ int rlcs_affine_scan(const float* alpha, const float* beta, float* out, int64_t 
 
 /*
  * Test hook: choose the kernel and tile shape for subsequent calls in this process (not
- * thread-safe).  variant -1 = the library default.  Other variants change the kernel (persistent
+ * thread-safe).  variant -1 = chosen per call from algorithm and problem size (the default).  Other variants change the kernel (persistent
  * blocks with a bulk-copy ring, or one tile per block), threads per block and steps per thread,
  * hence where tiles and warps cut the rows; results must agree across variants to rounding, and
  * exactly at severed steps.  Returns RLCS_ERR_ARG for an unknown variant.  rlcs_workspace_bytes is
@@ -213,8 +213,19 @@ int rlcs_affine_scan(const float* alpha, const float* beta, float* out, int64_t 
  */
 int rlcs_debug_set_tile_variant(int variant);
 
-/* Elements per tile of a variant (-1 = the default; 0 for an unknown variant). */
+/* Elements per tile of a variant (0 for an unknown variant). */
 int rlcs_debug_tile_elems(int variant);
+
+/*
+ * Which variant a call would use: algorithm 0 = GAE, 1 = TD(lambda), 2 = discounted return,
+ * 3 = V-Trace, 4 = Retrace, 5 = eligibility trace, 6 = prefix sum, 7 / 8 = rlcs_affine_scan backward /
+ * forward.  Honours rlcs_debug_set_tile_variant.  -1 for invalid arguments or an empty problem.
+ */
+int rlcs_debug_variant_for(int algorithm, int has_truncs, int64_t N, int64_t T);
+
+/* Shape of a variant: threads per block, steps per thread, blocks per SM it is compiled for, and
+ * ring stages (0 = the one-tile-per-block kernel).  Any output pointer may be NULL. */
+int rlcs_debug_variant_info(int variant, int* threads, int* steps_per_thread, int* blocks_per_sm, int* ring_stages);
 
 /*
  * Test hook for the bounded carry wait: for subsequent calls in this process, the thread block

@@ -39,6 +39,8 @@ SIGNATURES = {
     "rlcs_debug_set_tile_variant": ([_int], _int),
     "rlcs_debug_tile_elems": ([_int], _int),
     "rlcs_debug_set_carry_fault": ([_i64, _i64], _int),
+    "rlcs_debug_variant_for": ([_int, _int, _i64, _i64], _int),
+    "rlcs_debug_variant_info": ([_int] + [ctypes.POINTER(ctypes.c_int)] * 4, _int),
 }
 
 _lib = None
@@ -247,6 +249,19 @@ def rlcs_debug_set_tile_variant(variant: int):
 
 def rlcs_debug_tile_elems(variant: int) -> int:
     return int(lib().rlcs_debug_tile_elems(variant))
+
+
+ALGORITHM_IDS = {"gae": 0, "td_lambda": 1, "discounted_return": 2, "vtrace": 3, "retrace": 4, "elig_trace": 5,
+                 "episodic_prefix_sum": 6}
+
+
+def rlcs_debug_variant_for(algorithm: str, has_truncs: bool, N: int, T: int) -> dict:
+    """The kernel variant a call would use, as {variant, threads, steps_per_thread, blocks_per_sm, ring_stages}."""
+    v = int(lib().rlcs_debug_variant_for(ALGORITHM_IDS[algorithm], int(bool(has_truncs)), N, T))
+    out = [ctypes.c_int() for _ in range(4)]
+    _check(lib().rlcs_debug_variant_info(v, *[ctypes.byref(o) for o in out]))
+    return dict(variant=v, threads=out[0].value, steps_per_thread=out[1].value, blocks_per_sm=out[2].value,
+                ring_stages=out[3].value)
 
 
 def rlcs_debug_set_carry_fault(mute_tile: int = -1, spin_cap: int = 0):

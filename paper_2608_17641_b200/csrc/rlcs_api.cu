@@ -10,8 +10,7 @@ namespace {
 
 using rlcs::ScanParams;
 
-constexpr int kDefaultVariant = 0;
-int g_variant = kDefaultVariant; // test hook: tile variant
+int g_variant = -1;              // test hook: tile variant; -1 = chosen per call by choose_variant
 long long g_mute_tile = -1;      // test hook: tile that does not publish
 long long g_spin_cap = 0;        // test hook: poll limit (0 = default)
 constexpr unsigned kDefaultSpinCap = 1u << 21;
@@ -56,9 +55,29 @@ int check_alignment(const Ptrs& ps, bool* vec) {
     return RLCS_OK;
 }
 
+// Kernel and tile shape for one call, from measurements on B200 (see the tile-variant table in
+// rlcs_launch.cuh).  Large problems are bound by HBM: what matters is resident warps and bytes in
+// flight, so algorithms with few registers run more blocks per SM or 16 steps per thread.  Small
+// problems are bound by latency: smaller tiles spread them over more SMs, unless rows are long
+// enough for the inter-block carry to dominate.
+int choose_variant(int algo, bool trunc, int64_t total, int64_t T) {
+    if (g_variant >= 0) return g_variant;
+    if (total < (int64_t(1) << 23)) return T <= 2048 ? 6 : 0;
+    switch (algo) {
+        case rlcs::kGae: return trunc ? 16 : 0;
+        case rlcs::kVtrace: return trunc ? 18 : 0;
+        case rlcs::kRetrace: return 0;
+        case rlcs::kTdLambda: return trunc ? 17 : 0;
+        case rlcs::kDisc: return trunc ? 17 : 5;
+        case rlcs::kElig: return 18;
+        case rlcs::kPrefix: return 18;
+        default: return 0;
+    }
+}
+
 // Fill the size / tiling / carry fields and validate the workspace for this call.
-int finish_params(ScanParams& p, int64_t total, int64_t T, void* workspace, size_t workspace_bytes) {
-    const int tile = tile_elems(g_variant);
+int finish_params(ScanParams& p, int variant, int64_t total, int64_t T, void* workspace, size_t workspace_bytes) {
+    const int tile = tile_elems(variant);
     p.total = total;
     p.T = (unsigned)T;
     p.num_tiles = (total + tile - 1) / tile;
@@ -71,7 +90,7 @@ int finish_params(ScanParams& p, int64_t total, int64_t T, void* workspace, size
         p.div_T.sh2 = l > 1 ? l - 1 : 0;
     }
     p.decay_pow = 1.f;                       // beta product of a chunk without resets
-    for (int i = 0; i < rlcs::kVariants[g_variant].items; ++i) p.decay_pow *= p.decay;
+    for (int i = 0; i < rlcs::kVariants[variant].items; ++i) p.decay_pow *= p.decay;
     p.carry_mode = (tile % T) != 0;          // T does not divide the tile: rows straddle tiles
     p.header = nullptr;
     p.records = nullptr;
@@ -92,8 +111,8 @@ int finish_params(ScanParams& p, int64_t total, int64_t T, void* workspace, size
 
 typedef cudaError_t (*Launcher)(const ScanParams&, int, bool, bool, cudaStream_t);
 
-int run(Launcher fn, const ScanParams& p, bool trunc, bool vec, void* stream) {
-    return fn(p, g_variant, trunc, vec, static_cast<cudaStream_t>(stream)) == cudaSuccess ? RLCS_OK : RLCS_ERR_CUDA;
+int run(Launcher fn, const ScanParams& p, int variant, bool trunc, bool vec, void* stream) {
+    return fn(p, variant, trunc, vec, static_cast<cudaStream_t>(stream)) == cudaSuccess ? RLCS_OK : RLCS_ERR_CUDA;
 }
 
 // shared front half of the five backward entry points
@@ -180,9 +199,10 @@ int rlcs_gae(const float* rewards, const float* values, const uint8_t* dones, co
     if (!rewards || !values || !advantages) return RLCS_ERR_NULL;
     p.f0 = rewards; p.f1 = values; p.out0 = advantages; p.out1 = returns;
     p.gamma = gamma; p.decay = gamma * lambda;
-    st = finish_params(p, total, T, workspace, workspace_bytes);
+    const int variant = choose_variant(rlcs::kGae, truncs != nullptr, total, T);
+    st = finish_params(p, variant, total, T, workspace, workspace_bytes);
     if (st != RLCS_OK) return st;
-    return run(rlcs::launch_gae, p, truncs != nullptr, vec, cuda_stream);
+    return run(rlcs::launch_gae, p, variant, truncs != nullptr, vec, cuda_stream);
 }
 
 int rlcs_vtrace(const float* rewards, const float* values, const float* log_rhos, const uint8_t* dones,
@@ -200,9 +220,10 @@ int rlcs_vtrace(const float* rewards, const float* values, const float* log_rhos
     if (!rewards || !values || !log_rhos || !vs) return RLCS_ERR_NULL;
     p.f0 = rewards; p.f1 = values; p.f3 = log_rhos; p.out0 = vs; p.out1 = pg_advantages;
     p.gamma = gamma; p.rho_bar = rho_bar; p.c_bar = c_bar;
-    st = finish_params(p, total, T, workspace, workspace_bytes);
+    const int variant = choose_variant(rlcs::kVtrace, truncs != nullptr, total, T);
+    st = finish_params(p, variant, total, T, workspace, workspace_bytes);
     if (st != RLCS_OK) return st;
-    return run(rlcs::launch_vtrace, p, truncs != nullptr, vec, cuda_stream);
+    return run(rlcs::launch_vtrace, p, variant, truncs != nullptr, vec, cuda_stream);
 }
 
 int rlcs_retrace(const float* rewards, const float* q_sa, const float* expected_q, const float* log_rhos,
@@ -220,9 +241,10 @@ int rlcs_retrace(const float* rewards, const float* q_sa, const float* expected_
     if (!rewards || !q_sa || !expected_q || !log_rhos || !q_targets) return RLCS_ERR_NULL;
     p.f0 = rewards; p.f1 = q_sa; p.f2 = expected_q; p.f3 = log_rhos; p.out0 = q_targets;
     p.gamma = gamma; p.aux = gamma * lambda; p.c_bar = c_bar;
-    st = finish_params(p, total, T, workspace, workspace_bytes);
+    const int variant = choose_variant(rlcs::kRetrace, truncs != nullptr, total, T);
+    st = finish_params(p, variant, total, T, workspace, workspace_bytes);
     if (st != RLCS_OK) return st;
-    return run(rlcs::launch_retrace, p, truncs != nullptr, vec, cuda_stream);
+    return run(rlcs::launch_retrace, p, variant, truncs != nullptr, vec, cuda_stream);
 }
 
 int rlcs_td_lambda(const float* rewards, const float* values, const uint8_t* dones, const uint8_t* truncs,
@@ -239,9 +261,10 @@ int rlcs_td_lambda(const float* rewards, const float* values, const uint8_t* don
     if (!rewards || !values || !returns) return RLCS_ERR_NULL;
     p.f0 = rewards; p.f1 = values; p.out0 = returns;
     p.gamma = gamma; p.decay = gamma * lambda; p.aux = gamma * (1.f - lambda);
-    st = finish_params(p, total, T, workspace, workspace_bytes);
+    const int variant = choose_variant(rlcs::kTdLambda, truncs != nullptr, total, T);
+    st = finish_params(p, variant, total, T, workspace, workspace_bytes);
     if (st != RLCS_OK) return st;
-    return run(rlcs::launch_td_lambda, p, truncs != nullptr, vec, cuda_stream);
+    return run(rlcs::launch_td_lambda, p, variant, truncs != nullptr, vec, cuda_stream);
 }
 
 int rlcs_discounted_return(const float* rewards, const uint8_t* dones, const uint8_t* truncs,
@@ -258,9 +281,10 @@ int rlcs_discounted_return(const float* rewards, const uint8_t* dones, const uin
     if (!rewards || !returns) return RLCS_ERR_NULL;
     p.f0 = rewards; p.out0 = returns;
     p.gamma = gamma; p.decay = gamma;
-    st = finish_params(p, total, T, workspace, workspace_bytes);
+    const int variant = choose_variant(rlcs::kDisc, truncs != nullptr, total, T);
+    st = finish_params(p, variant, total, T, workspace, workspace_bytes);
     if (st != RLCS_OK) return st;
-    return run(rlcs::launch_disc, p, truncs != nullptr, vec, cuda_stream);
+    return run(rlcs::launch_disc, p, variant, truncs != nullptr, vec, cuda_stream);
 }
 
 static int forward_scan(rlcs::Algo algo, const float* x, const uint8_t* dones, float* out, int64_t N, int64_t T,
@@ -276,9 +300,10 @@ static int forward_scan(rlcs::Algo algo, const float* x, const uint8_t* dones, f
     st = check_alignment(ps, &vec);
     if (st != RLCS_OK) return st;
     p.f0 = x; p.dones = dones; p.out0 = out; p.decay = decay; p.starts_at = starts_at != 0;
-    st = finish_params(p, total, T, workspace, workspace_bytes);
+    const int variant = choose_variant(algo, false, total, T);
+    st = finish_params(p, variant, total, T, workspace, workspace_bytes);
     if (st != RLCS_OK) return st;
-    return run(algo == rlcs::kElig ? rlcs::launch_elig : rlcs::launch_prefix, p, false, vec, cuda_stream);
+    return run(algo == rlcs::kElig ? rlcs::launch_elig : rlcs::launch_prefix, p, variant, false, vec, cuda_stream);
 }
 
 int rlcs_elig_trace(const float* x, const uint8_t* dones, float* traces, int64_t N, int64_t T, float gamma,
@@ -305,21 +330,37 @@ int rlcs_affine_scan(const float* alpha, const float* beta, float* out, int64_t 
     st = check_alignment(ps, &vec);
     if (st != RLCS_OK) return st;
     p.f0 = alpha; p.f1 = beta; p.out0 = out;
-    st = finish_params(p, total, T, workspace, workspace_bytes);
+    const int variant = choose_variant(forward ? rlcs::kAffineFwd : rlcs::kAffineBwd, false, total, T);
+    st = finish_params(p, variant, total, T, workspace, workspace_bytes);
     if (st != RLCS_OK) return st;
-    return run(forward ? rlcs::launch_affine_fwd : rlcs::launch_affine_bwd, p, false, vec, cuda_stream);
+    return run(forward ? rlcs::launch_affine_fwd : rlcs::launch_affine_bwd, p, variant, false, vec, cuda_stream);
 }
 
 int rlcs_debug_set_tile_variant(int variant) {
     if (variant < -1 || variant >= rlcs::kNumVariants) return RLCS_ERR_ARG;
-    g_variant = variant < 0 ? kDefaultVariant : variant;
+    g_variant = variant;
     return RLCS_OK;
 }
 
 int rlcs_debug_tile_elems(int variant) {
-    if (variant == -1) variant = kDefaultVariant;
     if (variant < 0 || variant >= rlcs::kNumVariants) return 0;
     return tile_elems(variant);
+}
+
+int rlcs_debug_variant_for(int algorithm, int has_truncs, int64_t N, int64_t T) {
+    int64_t total = 0;
+    if (algorithm < 0 || algorithm > rlcs::kAffineFwd || check_sizes(N, T, &total) != RLCS_OK || total == 0) return -1;
+    return choose_variant(algorithm, has_truncs != 0, total, T);
+}
+
+int rlcs_debug_variant_info(int variant, int* threads, int* steps_per_thread, int* blocks_per_sm, int* ring_stages) {
+    if (variant < 0 || variant >= rlcs::kNumVariants) return RLCS_ERR_ARG;
+    const rlcs::TileVariant tv = rlcs::kVariants[variant];
+    if (threads) *threads = tv.threads;
+    if (steps_per_thread) *steps_per_thread = tv.items;
+    if (blocks_per_sm) *blocks_per_sm = tv.min_blocks;
+    if (ring_stages) *ring_stages = tv.stages;
+    return RLCS_OK;
 }
 
 int rlcs_debug_set_carry_fault(int64_t mute_tile, int64_t spin_cap) {

@@ -10,7 +10,7 @@ namespace rlcs {
 // stages == 0: scan_kernel (one tile per block).  stages > 0: scan_kernel_tma (persistent blocks,
 // bulk-copy ring of that many tiles; min_blocks = blocks per SM it is compiled and sized for).
 struct TileVariant { int threads, items, min_blocks, stages; };
-constexpr int kNumVariants = 16;
+constexpr int kNumVariants = 19;
 constexpr TileVariant kVariants[kNumVariants] = {
     {256, 8, 4, 0},    //  0: 2048 steps per tile
     {128, 4, 8, 0},    //  1:  512
@@ -28,6 +28,9 @@ constexpr TileVariant kVariants[kNumVariants] = {
     {256, 16, 2, 2},   // 13: 4096, persistent, 2 stages
     {256, 8, 3, 4},    // 14: 2048, persistent, 4 stages
     {256, 8, 3, 6},    // 15: 2048, persistent, 6 stages
+    {256, 8, 5, 0},    // 16: 2048, at most 48 registers
+    {256, 8, 6, 0},    // 17: 2048, at most 40 registers
+    {128, 16, 5, 0},   // 18: 2048, 16 steps per thread
 };
 constexpr int kMinTileElems = 512;
 constexpr int kMaxDevices = 64;

@@ -82,7 +82,7 @@ def test_shape_matrix(oracle, W, B, N, T, p_flag):
     compare_all(oracle, ro)
 
 
-@pytest.mark.parametrize("variant", list(range(16)))
+@pytest.mark.parametrize("variant", list(range(19)))
 @pytest.mark.parametrize("N,T", [(5, 700), (4097, 3), (2, 9000), (64, 513)])
 def test_tile_variants(oracle, W, B, variant, N, T):
     B.rlcs_debug_set_tile_variant(variant)
