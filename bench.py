@@ -35,7 +35,10 @@ FALLBACK_HBM_GBS = 6650.0
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel on the bench
 # workload, from the ncu capture summarised under profiles/ (None until a capture exists).
-NCU_TRAFFIC_BYTES = {}
+NCU_TRAFFIC_BYTES = {          # profiles/dram_traffic_16384x2048.md (full-size capture, read + write)
+    "gae": 576827904, "vtrace": 715524096, "retrace": 738515712, "td_lambda": 456696832,
+    "discounted_return": 312028672, "elig_trace": 255066880, "episodic_prefix_sum": 251662080,
+}
 
 
 # --------------------------------------------------------------------------------------------- helpers
@@ -486,7 +489,7 @@ def main():
     roofline = {"bound": "hbm", "kernel": f"{kname}<{dom}>, {vi['threads']} threads x {vi['steps_per_thread']} steps per tile "
                                           f"(variant {vi['variant']})",
                 "achieved": per_algo[dom]["gbs"], "peak": peak, "unit": "GB/s",
-                "frac": round(per_algo[dom]["gbs"] / peak, 4), "traffic": NCU_TRAFFIC_BYTES.get(dom),
+                "frac": round(per_algo[dom]["gbs"] / peak, 4), "traffic": NCU_TRAFFIC_BYTES.get(dom) if (ro.N, ro.T) == (WORKLOAD["N"], WORKLOAD["T"]) and ro.truncs is not None else None,
                 "algorithmic_bytes_per_launch": per_algo[dom]["algorithmic_bytes"], "peak_source": f"of {peak_kind}",
                 "all_kernels_frac": round(sum(v["algorithmic_bytes"] for v in per_algo.values())
                                           / (sum(v["ms"] for v in per_algo.values()) * 1e-3) / 1e9 / peak, 4)}
