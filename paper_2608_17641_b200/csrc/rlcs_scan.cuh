@@ -311,6 +311,23 @@ static __device__ __noinline__ float lookback(const uint4* __restrict__ records,
     }
 }
 
+// A block signs off from the carry protocol of this call once it has published its last record and
+// finished its last look-back: from then on it neither reads the epoch nor polls records.  The last
+// block to sign off advances the epoch, so the records of this call can never be taken for those
+// of the next one and no per-call clearing is needed.  (No fence: nothing but the protocol words
+// depends on it, and the next call starts only after this kernel has ended.)  Signing off before
+// the stores keeps this round trip off the tail of the kernel.
+__device__ __forceinline__ void sign_off(const ScanParams& p) {
+    if (threadIdx.x == 0) {
+        const unsigned done = atomicAdd(p.header + 1, 1u);
+        if (done == gridDim.x - 1) {
+            p.header[1] = 0;
+            const unsigned e = ld_volatile_u32(p.header);
+            p.header[0] = (e == 0xffffffffu) ? 1u : e + 1u;
+        }
+    }
+}
+
 // ------------------------------------------------------------------------------------------ one thread's part of a tile
 // Flags and geometry of a thread's ITEMS consecutive steps: everything the coefficient stage needs
 // besides the float inputs.  The persistent kernel fetches this one tile ahead.
@@ -441,7 +458,9 @@ struct NoHook {
 // `after_barrier` runs right after the block barrier (every thread has consumed its inputs).
 // FULL: the tile lies completely inside the array and rows are at least ITEMS long (block-uniform),
 // which removes the ragged-chunk and short-row side paths at compile time.
-template <int ALGO, bool TRUNC, bool VEC, int THREADS, int ITEMS, bool FULL, class Hook>
+// LAST: this is the block's last tile of the call; the block then signs off from the carry protocol
+// as soon as its own look-back is over (see sign_off) instead of after its stores.
+template <int ALGO, bool TRUNC, bool VEC, int THREADS, int ITEMS, bool FULL, bool LAST, class Hook>
 __device__ __forceinline__ void tile_compute(Chunk<ALGO, TRUNC, ITEMS>& c, Vals<ITEMS>& v, const ScanParams& p, long long i0, long long s,
                                              unsigned epoch, ScanSmem<THREADS / 32>& sm, int buf, Hook after_barrier) {
     constexpr bool FWD = is_forward(ALGO);
@@ -641,6 +660,7 @@ __device__ __forceinline__ void tile_compute(Chunk<ALGO, TRUNC, ITEMS>& c, Vals<
             __syncthreads();
             carry_in = sm.carry[buf];
         }
+        if constexpr (LAST) sign_off(p);
     }
     // value of the recurrence at the step just before this thread's chunk in scan order
     float prev = fmaf(before.b, carry_in, before.a);
@@ -681,20 +701,7 @@ __device__ __forceinline__ void tile_compute(Chunk<ALGO, TRUNC, ITEMS>& c, Vals<
     }
 }
 
-// The last block to finish advances the epoch, so the records of this call can never be taken for
-// those of the next one and no per-call clearing is needed.
-__device__ __forceinline__ void close_call(const ScanParams& p) {
-    if (p.carry_mode && threadIdx.x == 0) {
-        __threadfence();
-        const unsigned done = atomicAdd(p.header + 1, 1u);
-        if (done == gridDim.x - 1) {
-            p.header[1] = 0;
-            const unsigned e = ld_volatile_u32(p.header);
-            p.header[0] = (e == 0xffffffffu) ? 1u : e + 1u;
-        }
-    }
-}
-
+// ------------------------------------------------------------------------------------------ end of a call (carry mode)
 // ------------------------------------------------------------------------------------------ kernel 1: one tile per block
 template <int ALGO, bool TRUNC, bool VEC, int THREADS, int ITEMS, bool FULL>
 __device__ __forceinline__ void one_tile(const ScanParams& p, long long tile, long long s, unsigned epoch,
@@ -710,7 +717,7 @@ __device__ __forceinline__ void one_tile(const ScanParams& p, long long tile, lo
     load_values_global<ALGO, TRUNC, ITEMS, VEC, FULL>(c, v, p, i0, lane);
     issue_boot(c, p, n0);
     issue_trunc_values(c, p, i0);
-    tile_compute<ALGO, TRUNC, VEC, THREADS, ITEMS, FULL>(c, v, p, i0, s, epoch, sm, 0, NoHook{});
+    tile_compute<ALGO, TRUNC, VEC, THREADS, ITEMS, FULL, true>(c, v, p, i0, s, epoch, sm, 0, NoHook{});
 }
 
 template <int ALGO, bool TRUNC, bool VEC, int THREADS, int ITEMS, int MIN_BLOCKS>
@@ -730,7 +737,6 @@ __global__ void __launch_bounds__(THREADS, MIN_BLOCKS) scan_kernel(const ScanPar
     const bool full = (tile * TILE + TILE <= p.total) && (p.T >= (unsigned)ITEMS);
     if (full) one_tile<ALGO, TRUNC, VEC, THREADS, ITEMS, true>(p, tile, s, epoch, sm);
     else one_tile<ALGO, TRUNC, VEC, THREADS, ITEMS, false>(p, tile, s, epoch, sm);
-    close_call(p);
 }
 
 // ------------------------------------------------------------------------------------------ mbarrier / bulk copy (PTX)
@@ -941,7 +947,7 @@ __device__ __forceinline__ void walk_step(Chunk<ALGO, TRUNC, ITEMS>& cur, const 
         load_values_global<ALGO, TRUNC, ITEMS, true>(cur, v, p, i0, tid & 31);
     }
     Chunk<ALGO, TRUNC, ITEMS> nxt;
-    tile_compute<ALGO, TRUNC, true, THREADS, ITEMS, false>(cur, v, p, i0, w.s, w.epoch, sm, w.buf,
+    tile_compute<ALGO, TRUNC, true, THREADS, ITEMS, false, false>(cur, v, p, i0, w.s, w.epoch, sm, w.buf,
                                                     AfterBarrier<ALGO, TRUNC, THREADS, ITEMS, STAGES>{p, w, ring, full_bar, nxt, bulk});
     if (w.s + w.G < p.num_tiles) cur = nxt;
     if (bulk) ++w.cj;
@@ -988,7 +994,7 @@ __global__ void __launch_bounds__(THREADS, MIN_BLOCKS) scan_kernel_tma(const Sca
     if (w.s < p.num_tiles)
         prefetch_flags<ALGO, TRUNC, THREADS, ITEMS, STAGES>(cur, p, tile_of<ALGO, TILE>(p, w.s), ring, full_bar, w.cj, w.gave_up);
     while (w.s < p.num_tiles) walk_step<ALGO, TRUNC, THREADS, ITEMS, STAGES>(cur, p, w, ring, full_bar, sm);
-    close_call(p);
+    if (p.carry_mode) sign_off(p);
 }
 
 }  // namespace rlcs
