@@ -135,17 +135,28 @@ class ClockSampler:
 class GpuBatch:
     """Device-resident inputs, outputs and workspace of one batch, and the seven calls on them."""
 
-    def __init__(self, ro, device):
+    NEEDS = {"gae": ("rewards", "values"), "vtrace": ("rewards", "values", "log_rhos"),
+             "retrace": ("rewards", "q_sa", "expected_q", "log_rhos"), "td_lambda": ("rewards", "values"),
+             "discounted_return": ("rewards",), "elig_trace": ("x", "any_done"), "episodic_prefix_sum": ("x", "any_done")}
+    BACKWARD_COMMON = ("dones", "truncs", "trunc_bootstrap", "bootstrap")
+
+    def __init__(self, ro, device, only=None):
         import torch
         from paper_2608_17641_b200 import binding as B
         self.B, self.ro, self.torch = B, ro, torch
+        algos = ALGOS if only is None else (only,)
+        keys = set()
+        for a in algos:
+            keys.update(self.NEEDS[a])
+            if a not in ("elig_trace", "episodic_prefix_sum"):
+                keys.update(self.BACKWARD_COMMON)
+        src = lambda k: ro.any_done if k == "any_done" else getattr(ro, k)
         up = lambda a: None if a is None else torch.from_numpy(a).to(device, non_blocking=False)
-        self.inp = {k: up(getattr(ro, k)) for k in ("rewards", "values", "q_sa", "expected_q", "log_rhos", "x",
-                                                    "dones", "truncs", "trunc_bootstrap", "bootstrap")}
-        self.inp["any_done"] = up(ro.any_done)
+        self.inp = {k: (up(src(k)) if k in keys else None) for k in ("rewards", "values", "q_sa", "expected_q", "log_rhos",
+                                                                      "x", "dones", "truncs", "trunc_bootstrap", "bootstrap",
+                                                                      "any_done")}
         new = lambda: torch.empty((ro.N, ro.T), dtype=torch.float32, device=device)
-        self.out = {"gae": (new(), new()), "vtrace": (new(), new()), "retrace": new(), "td_lambda": new(),
-                    "discounted_return": new(), "elig_trace": new(), "episodic_prefix_sum": new()}
+        self.out = {a: ((new(), new()) if a in ("gae", "vtrace") else new()) for a in algos}
         self.ws = B.Workspace(ro.N, ro.T, device=device)
         self.launches = 0
 
@@ -209,7 +220,11 @@ def time_device(batch: GpuBatch, steps: int, warmup: int, dist):
 
 def time_e2e(batch: GpuBatch, steps: int, warmup: int, dist):
     """The same step called with HOST buffers: every step copies that step's inputs from pinned
-    host memory to the device, runs the seven C-ABI calls, and reads all outputs back."""
+    host memory to the device, runs the seven C-ABI calls, and reads all outputs back to pinned
+    host memory.  Three streams, as a caller would arrange them: copies in, kernels, copies out;
+    a kernel starts as soon as its own inputs have landed, and one step's read-back overlaps the
+    next step's upload (the link is full duplex).  Inputs and outputs are single-buffered on the
+    device, so uploads wait for the previous step's kernels and kernels for the previous read-back."""
     torch, ro = batch.torch, batch.ro
     pin = lambda t: torch.empty(t.shape, dtype=t.dtype).pin_memory().copy_(t.cpu())
     h_in = {k: pin(v) for k, v in batch.inp.items() if v is not None}
@@ -219,27 +234,59 @@ def time_e2e(batch: GpuBatch, steps: int, warmup: int, dist):
             else torch.empty(v.shape, dtype=v.dtype).pin_memory()
     h2d = sum(t.numel() * t.element_size() for t in h_in.values())
     d2h = sum(t.numel() * t.element_size() for v in h_out.values() for t in (v if isinstance(v, tuple) else (v,)))
+    s_in, s_k, s_out = torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.Stream()
+    # upload order and the algorithms that can start after each group
+    groups = [(("dones", "truncs", "bootstrap", "trunc_bootstrap", "rewards", "values"), ("gae", "td_lambda", "discounted_return")),
+              (("log_rhos",), ("vtrace",)), (("q_sa", "expected_q"), ("retrace",)),
+              (("x", "any_done"), ("elig_trace", "episodic_prefix_sum"))]
+    state = {"kernels_done": None, "readback_done": None}
 
     def one():
-        for k, t in h_in.items():
-            batch.inp[k].copy_(t, non_blocking=True)
-        batch.step()
-        for a, v in batch.out.items():
-            if isinstance(v, tuple):
-                for hv, dv in zip(h_out[a], v):
-                    hv.copy_(dv, non_blocking=True)
-            else:
-                h_out[a].copy_(v, non_blocking=True)
+        if state["kernels_done"] is not None:
+            s_in.wait_event(state["kernels_done"])          # the previous step still reads the inputs
+        if state["readback_done"] is not None:
+            s_k.wait_event(state["readback_done"])          # ... and its outputs are still being read back
+        for names, algos in groups:
+            with torch.cuda.stream(s_in):
+                for k in names:
+                    if k in h_in:
+                        batch.inp[k].copy_(h_in[k], non_blocking=True)
+                landed = torch.cuda.Event()
+                landed.record(s_in)
+            s_k.wait_event(landed)
+            for a in algos:
+                with torch.cuda.stream(s_k):
+                    batch.call(a)
+                    ran = torch.cuda.Event()
+                    ran.record(s_k)
+                s_out.wait_event(ran)
+                with torch.cuda.stream(s_out):
+                    v = batch.out[a]
+                    for hv, dv in zip(h_out[a] if isinstance(v, tuple) else (h_out[a],), v if isinstance(v, tuple) else (v,)):
+                        hv.copy_(dv, non_blocking=True)
+        state["kernels_done"] = torch.cuda.Event()
+        state["kernels_done"].record(s_k)
+        state["readback_done"] = torch.cuda.Event()
+        state["readback_done"].record(s_out)
 
+    cur = torch.cuda.current_stream()
+    for s in (s_in, s_k, s_out):
+        s.wait_stream(cur)
     for _ in range(warmup):
         one()
+    for s in (s_in, s_k, s_out):
+        cur.wait_stream(s)
     start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     dist.barrier()
     torch.cuda.synchronize()
-    start.record()
+    start.record(cur)
+    for s in (s_in, s_k, s_out):
+        s.wait_stream(cur)
     for _ in range(steps):
         one()
-    stop.record()
+    for s in (s_in, s_k, s_out):
+        cur.wait_stream(s)
+    stop.record(cur)
     torch.cuda.synchronize()
     dist.barrier()
     return start.elapsed_time(stop), h2d, d2h
@@ -314,36 +361,14 @@ def reference_arm(args, world: int):
 
 
 # --------------------------------------------------------------------------------------------- sweeps (cold L2)
-def sweep_case(torch, B, ro, algo: str, use_truncs: bool, hbm_peak: float, l2_bytes: int, trials=5, target_bytes=None):
+def sweep_case(torch, B, ro, algo: str, use_truncs: bool, hbm_peak: float, l2_bytes: int, trials=5):
     """Device time per call with a cold L2: the calls of one batch rotate over R distinct copies of
     all inputs and outputs whose total footprint exceeds 3x the L2 capacity."""
-    keys = {"gae": ("rewards", "values"), "vtrace": ("rewards", "values", "log_rhos"),
-            "discounted_return": ("rewards",)}[algo]
-    base = {k: torch.from_numpy(getattr(ro, k)).cuda() for k in keys + ("dones", "bootstrap")}
-    if use_truncs:
-        base["truncs"] = torch.from_numpy(ro.truncs).cuda()
-        base["trunc_bootstrap"] = torch.from_numpy(ro.trunc_bootstrap).cuda()
-    n_out = 1 if algo == "discounted_return" else 2
-    set_bytes = sum(t.numel() * t.element_size() for t in base.values()) + n_out * 4 * ro.N * ro.T
-    R = int(min(512, max(4, -(-3 * l2_bytes // set_bytes))))
-    sets = [{k: v.clone() for k, v in base.items()} for _ in range(R)]
-    outs = [[torch.empty((ro.N, ro.T), dtype=torch.float32, device="cuda") for _ in range(n_out)] for _ in range(R)]
-    ws = B.Workspace(ro.N, ro.T)
-    p = ro.params
-
-    def call(i):
-        s, o = sets[i], outs[i]
-        tr, bv = (s["truncs"], s["trunc_bootstrap"]) if use_truncs else (None, None)
-        if algo == "gae":
-            B.rlcs_gae(s["rewards"], s["values"], s["dones"], tr, bv, s["bootstrap"], gamma=p["gamma"], lam=p["lam"],
-                       advantages=o[0], returns=o[1], workspace=ws)
-        elif algo == "vtrace":
-            B.rlcs_vtrace(s["rewards"], s["values"], s["log_rhos"], s["dones"], tr, bv, s["bootstrap"], gamma=p["gamma"],
-                          vs=o[0], pg_advantages=o[1], workspace=ws)
-        else:
-            B.rlcs_discounted_return(s["rewards"], s["dones"], tr, bv, s["bootstrap"], gamma=p["gamma"], returns=o[0],
-                                     workspace=ws)
-
+    ro_eff = ro if use_truncs else _without_truncs(ro)
+    algo_bytes = algorithmic_bytes(ro_eff, algo)
+    R = int(min(512, max(4, -(-3 * l2_bytes // algo_bytes))))
+    sets = [GpuBatch(ro_eff, torch.device("cuda", torch.cuda.current_device()), only=algo) for _ in range(R)]
+    call = lambda i: sets[i].call(algo)
     for i in range(R):
         call(i)
     torch.cuda.synchronize()
@@ -372,8 +397,6 @@ def sweep_case(torch, B, ro, algo: str, use_truncs: bool, hbm_peak: float, l2_by
         e1.record()
         torch.cuda.synchronize()
         full_call_us.append(1e3 * e0.elapsed_time(e1) / R)
-    ro_eff = ro if use_truncs else _without_truncs(ro)
-    algo_bytes = algorithmic_bytes(ro_eff, algo)
     best = min(per_call_us)
     gbs = algo_bytes / (best * 1e-6) / 1e9
     return {"algo": algo, "N": ro.N, "T": ro.T, "truncs": use_truncs, "us_per_call": round(best, 3),
@@ -395,6 +418,10 @@ def run_sweeps(torch, hbm_peak):
     from paper_2608_17641_b200 import binding as B, workloads
     l2 = torch.cuda.get_device_properties(0).L2_cache_size
     out = []
+    out.append(sweep_case(torch, B, workloads.config1(), "gae", True, hbm_peak, l2))          # config 1: latency floor
+    ro2 = workloads.config2()
+    for algo in ALGOS:                                                                         # config 2: all seven
+        out.append(sweep_case(torch, B, ro2, algo, True, hbm_peak, l2))
     for T in (32, 64, 128, 256, 512, 1024):
         for tr in (False, True):
             ro = workloads.config3(T, True)
@@ -494,12 +521,13 @@ def main():
                 "all_kernels_frac": round(sum(v["algorithmic_bytes"] for v in per_algo.values())
                                           / (sum(v["ms"] for v in per_algo.values()) * 1e-3) / 1e9 / peak, 4)}
 
-    e2e_steps = max(1, min(args.steps, 5))
+    e2e_steps = max(1, min(args.steps, 8))
     e2e_ms, h2d, d2h = time_e2e(batch, e2e_steps, 1, dist)
     e2e_ms = dist.max(e2e_ms)
     e2e = {"value": units_per_step * e2e_steps / (e2e_ms * 1e-3), "unit": METRIC, "h2d_bytes_per_step": h2d,
            "d2h_bytes_per_step": d2h, "steps": e2e_steps, "ms_per_step": e2e_ms / e2e_steps,
-           "note": "pinned host buffers -> device, seven C-ABI calls, all outputs -> pinned host, one stream"}
+           "note": "pinned host buffers -> device, seven C-ABI calls, all outputs -> pinned host; upload, kernel and "
+                   "read-back streams chained by events"}
 
     line = {
         "metric": METRIC, "value": value, "unit": METRIC, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,

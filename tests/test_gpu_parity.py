@@ -131,7 +131,7 @@ def test_null_bootstrap_and_null_truncs(oracle, W, B):
     compare_all(oracle, ro, algos=BACKWARD, use_truncs=False, use_bootstrap=False)
 
 
-@pytest.mark.parametrize("offset", [1, 2, 3])
+@pytest.mark.parametrize("offset", [1, 2, 3, 4])       # 4 floats = 16-byte but not 32-byte aligned
 @pytest.mark.parametrize("N,T", [(5, 333), (3, 2048), (2, 5000)])
 def test_unaligned_pointers_take_elementwise_path(oracle, W, B, offset, N, T):
     ro = W.make_rollout(94, N, T, salt=offset)
@@ -181,6 +181,18 @@ def test_nonbinary_flag_bytes(oracle, W, B):
     ro = W.make_rollout(97, 4, 600, p_done=0.05, p_trunc=0.05)
     ro.dones = (ro.dones * np.uint8(0x80)).astype(np.uint8)
     ro.truncs = (ro.truncs * np.uint8(0x7f)).astype(np.uint8)
+    compare_all(oracle, ro)
+
+
+def test_large_problem_variants_with_carry(oracle, W, B):
+    """Above 2^23 steps the library picks per-algorithm tile shapes (more blocks per SM, 16 steps per
+    thread); T = 3000 makes rows straddle every one of them, so the inter-block carry runs too."""
+    ro = W.make_rollout(106, 2900, 3000, p_done=0.002, p_trunc=0.002)
+    assert ro.N * ro.T > 1 << 23
+    for a in ("gae", "vtrace", "td_lambda", "discounted_return", "elig_trace", "episodic_prefix_sum"):
+        name = a if a != "episodic_prefix_sum" else "episodic_prefix_sum"
+        info = B.rlcs_debug_variant_for(name, True, ro.N, ro.T)
+        assert BASE_VARIANT != -1 or info["variant"] not in (0, 6), (a, info)
     compare_all(oracle, ro)
 
 
