@@ -228,6 +228,13 @@ int rlcs_debug_variant_for(int algorithm, int has_truncs, int64_t N, int64_t T);
 int rlcs_debug_variant_info(int variant, int* threads, int* steps_per_thread, int* blocks_per_sm, int* ring_stages);
 
 /*
+ * Test hook: with on != 0, subsequent calls compute row and timestep of a step with the 64-bit
+ * arithmetic that problems of 2^32 steps and more need, whatever their size (the 32-bit path uses a
+ * multiply-shift division by T).  Results must be identical.
+ */
+int rlcs_debug_force_wide_index(int on);
+
+/*
  * Test hook for the bounded carry wait: for subsequent calls in this process, the thread block
  * whose scan-order index is `mute_tile` does not publish its tile record (negative = publish
  * normally), and the wait gives up after `spin_cap` polls (<= 0 = default).  A dependent block

@@ -11,6 +11,7 @@ namespace {
 using rlcs::ScanParams;
 
 int g_variant = -1;              // test hook: tile variant; -1 = chosen per call by choose_variant
+bool g_wide_index = false;       // test hook: use the 64-bit index path even when 32 bits would do
 long long g_mute_tile = -1;      // test hook: tile that does not publish
 long long g_spin_cap = 0;        // test hook: poll limit (0 = default)
 constexpr unsigned kDefaultSpinCap = 1u << 21;
@@ -81,7 +82,7 @@ int finish_params(ScanParams& p, int variant, int64_t total, int64_t T, void* wo
     p.total = total;
     p.T = (unsigned)T;
     p.num_tiles = (total + tile - 1) / tile;
-    p.idx32 = (total + tile) <= 0xffffffffLL;
+    p.idx32 = !g_wide_index && (total + tile) <= 0xffffffffLL;
     {   // invariant division by T (see FastDiv)
         int l = 0;
         while ((int64_t(1) << l) < T) ++l;
@@ -360,6 +361,11 @@ int rlcs_debug_variant_info(int variant, int* threads, int* steps_per_thread, in
     if (steps_per_thread) *steps_per_thread = tv.items;
     if (blocks_per_sm) *blocks_per_sm = tv.min_blocks;
     if (ring_stages) *ring_stages = tv.stages;
+    return RLCS_OK;
+}
+
+int rlcs_debug_force_wide_index(int on) {
+    g_wide_index = on != 0;
     return RLCS_OK;
 }
 

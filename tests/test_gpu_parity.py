@@ -196,6 +196,28 @@ def test_large_problem_variants_with_carry(oracle, W, B):
     compare_all(oracle, ro)
 
 
+def test_wide_index_path_gives_identical_results(oracle, W, B):
+    """The 64-bit row/timestep arithmetic (for 2^32 steps and more) against the 32-bit one, bit for
+    bit, on shapes whose T is and is not a power of two, in both kernels."""
+    for N, T in [(37, 1000), (5, 4096), (700, 7)]:
+        ro = W.make_rollout(107, N, T, salt=T)
+        dev = Dev(ro)
+        for variant in (BASE_VARIANT, 8):
+            B.rlcs_debug_set_tile_variant(variant)
+            try:
+                narrow = run_gpu(dev, ALL_ALGOS)
+                B.rlcs_debug_force_wide_index(True)
+                wide = run_gpu(dev, ALL_ALGOS)
+            finally:
+                B.rlcs_debug_force_wide_index(False)
+                B.rlcs_debug_set_tile_variant(BASE_VARIANT)
+            for a in ALL_ALGOS:
+                pairs = zip(narrow[a], wide[a]) if isinstance(narrow[a], tuple) else [(narrow[a], wide[a])]
+                for x, y in pairs:
+                    assert np.array_equal(x, y), (a, N, T, variant)
+        compare_all(oracle, ro)
+
+
 def test_gamma_lambda_extremes(oracle, W, B):
     for g, l in [(0.0, 0.5), (1.0, 1.0), (0.5, 0.0), (1.0, 0.0)]:
         ro = W.make_rollout(98, 6, 777, p_done=0.01, p_trunc=0.01)
