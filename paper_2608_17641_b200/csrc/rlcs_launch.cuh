@@ -69,7 +69,11 @@ template <int ALGO, bool TRUNC, bool VEC, int V>
 cudaError_t launch_variant(const ScanParams& p, cudaStream_t stream) {
     constexpr TileVariant tv = kVariants[V];
     if constexpr (tv.stages > 0 && VEC) {
-        return launch_persistent<ALGO, TRUNC, V>(p, stream);
+        // (rows shorter than a chunk go to the one-tile kernel: the persistent one assumes T >= ITEMS)
+        if (p.T >= (unsigned)tv.items) return launch_persistent<ALGO, TRUNC, V>(p, stream);
+        scan_kernel<ALGO, TRUNC, true, tv.threads, tv.items, tv.min_blocks>
+            <<<(unsigned)p.num_tiles, tv.threads, 0, stream>>>(p);
+        return cudaGetLastError();
     } else {
         // bulk copies need 16-byte aligned pointers; otherwise the element-wise kernel of the same tile shape
         scan_kernel<ALGO, TRUNC, VEC, tv.threads, tv.items, tv.min_blocks>

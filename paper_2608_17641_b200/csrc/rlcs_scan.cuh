@@ -947,8 +947,11 @@ __device__ __forceinline__ void walk_step(Chunk<ALGO, TRUNC, ITEMS>& cur, const 
         load_values_global<ALGO, TRUNC, ITEMS, true>(cur, v, p, i0, tid & 31);
     }
     Chunk<ALGO, TRUNC, ITEMS> nxt;
-    tile_compute<ALGO, TRUNC, true, THREADS, ITEMS, false, false>(cur, v, p, i0, w.s, w.epoch, sm, w.buf,
-                                                    AfterBarrier<ALGO, TRUNC, THREADS, ITEMS, STAGES>{p, w, ring, full_bar, nxt, bulk});
+    const AfterBarrier<ALGO, TRUNC, THREADS, ITEMS, STAGES> hook{p, w, ring, full_bar, nxt, bulk};
+    // A tile that came through the ring lies inside the array, and the host sends rows shorter
+    // than a chunk to the other kernel: the full-tile path applies.
+    if (bulk) tile_compute<ALGO, TRUNC, true, THREADS, ITEMS, true, false>(cur, v, p, i0, w.s, w.epoch, sm, w.buf, hook);
+    else tile_compute<ALGO, TRUNC, true, THREADS, ITEMS, false, false>(cur, v, p, i0, w.s, w.epoch, sm, w.buf, hook);
     if (w.s + w.G < p.num_tiles) cur = nxt;
     if (bulk) ++w.cj;
     w.s += w.G;
