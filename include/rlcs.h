@@ -228,6 +228,13 @@ int rlcs_debug_variant_for(int algorithm, int has_truncs, int64_t N, int64_t T);
 int rlcs_debug_variant_info(int variant, int* threads, int* steps_per_thread, int* blocks_per_sm, int* ring_stages);
 
 /*
+ * Test hook: rows that are exactly 2..8 tiles long are scanned by one thread-block cluster per row,
+ * with the carry between blocks in distributed shared memory (no workspace use).  on == 0 sends
+ * such calls through the workspace look-back instead.  Results must agree to rounding.
+ */
+int rlcs_debug_allow_cluster_carry(int on);
+
+/*
  * Test hook: with on != 0, subsequent calls compute row and timestep of a step with the 64-bit
  * arithmetic that problems of 2^32 steps and more need, whatever their size (the 32-bit path uses a
  * multiply-shift division by T).  Results must be identical.

@@ -40,6 +40,7 @@ SIGNATURES = {
     "rlcs_debug_tile_elems": ([_int], _int),
     "rlcs_debug_set_carry_fault": ([_i64, _i64], _int),
     "rlcs_debug_force_wide_index": ([_int], _int),
+    "rlcs_debug_allow_cluster_carry": ([_int], _int),
     "rlcs_debug_variant_for": ([_int, _int, _i64, _i64], _int),
     "rlcs_debug_variant_info": ([_int] + [ctypes.POINTER(ctypes.c_int)] * 4, _int),
 }
@@ -263,6 +264,10 @@ def rlcs_debug_variant_for(algorithm: str, has_truncs: bool, N: int, T: int) -> 
     _check(lib().rlcs_debug_variant_info(v, *[ctypes.byref(o) for o in out]))
     return dict(variant=v, threads=out[0].value, steps_per_thread=out[1].value, blocks_per_sm=out[2].value,
                 ring_stages=out[3].value)
+
+
+def rlcs_debug_allow_cluster_carry(on: bool):
+    _check(lib().rlcs_debug_allow_cluster_carry(int(bool(on))))
 
 
 def rlcs_debug_force_wide_index(on: bool):

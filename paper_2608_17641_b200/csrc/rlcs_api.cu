@@ -11,6 +11,7 @@ namespace {
 using rlcs::ScanParams;
 
 int g_variant = -1;              // test hook: tile variant; -1 = chosen per call by choose_variant
+bool g_cluster = true;           // test hook: allow the cluster carry
 bool g_wide_index = false;       // test hook: use the 64-bit index path even when 32 bits would do
 long long g_mute_tile = -1;      // test hook: tile that does not publish
 long long g_spin_cap = 0;        // test hook: poll limit (0 = default)
@@ -77,7 +78,7 @@ int choose_variant(int algo, bool trunc, int64_t total, int64_t T) {
 }
 
 // Fill the size / tiling / carry fields and validate the workspace for this call.
-int finish_params(ScanParams& p, int variant, int64_t total, int64_t T, void* workspace, size_t workspace_bytes) {
+int finish_params(ScanParams& p, int variant, int64_t total, int64_t T, void* workspace, size_t workspace_bytes, bool vec) {
     const int tile = tile_elems(variant);
     p.total = total;
     p.T = (unsigned)T;
@@ -93,6 +94,13 @@ int finish_params(ScanParams& p, int variant, int64_t total, int64_t T, void* wo
     p.decay_pow = 1.f;                       // beta product of a chunk without resets
     for (int i = 0; i < rlcs::kVariants[variant].items; ++i) p.decay_pow *= p.decay;
     p.carry_mode = (tile % T) != 0;          // T does not divide the tile: rows straddle tiles
+    // Rows of exactly 2..8 tiles: one thread-block cluster per row carries through distributed
+    // shared memory instead (needs the vectorised one-tile kernel; g_cluster = 0 turns it off).
+    p.cluster = 0;
+    if (g_cluster && vec && rlcs::kVariants[variant].stages == 0 && T % tile == 0 && T / tile >= 2 && T / tile <= 8) {
+        p.cluster = (int)(T / tile);
+        p.carry_mode = 0;
+    }
     p.header = nullptr;
     p.records = nullptr;
     p.status = nullptr;
@@ -201,7 +209,7 @@ int rlcs_gae(const float* rewards, const float* values, const uint8_t* dones, co
     p.f0 = rewards; p.f1 = values; p.out0 = advantages; p.out1 = returns;
     p.gamma = gamma; p.decay = gamma * lambda;
     const int variant = choose_variant(rlcs::kGae, truncs != nullptr, total, T);
-    st = finish_params(p, variant, total, T, workspace, workspace_bytes);
+    st = finish_params(p, variant, total, T, workspace, workspace_bytes, vec);
     if (st != RLCS_OK) return st;
     return run(rlcs::launch_gae, p, variant, truncs != nullptr, vec, cuda_stream);
 }
@@ -222,7 +230,7 @@ int rlcs_vtrace(const float* rewards, const float* values, const float* log_rhos
     p.f0 = rewards; p.f1 = values; p.f3 = log_rhos; p.out0 = vs; p.out1 = pg_advantages;
     p.gamma = gamma; p.rho_bar = rho_bar; p.c_bar = c_bar;
     const int variant = choose_variant(rlcs::kVtrace, truncs != nullptr, total, T);
-    st = finish_params(p, variant, total, T, workspace, workspace_bytes);
+    st = finish_params(p, variant, total, T, workspace, workspace_bytes, vec);
     if (st != RLCS_OK) return st;
     return run(rlcs::launch_vtrace, p, variant, truncs != nullptr, vec, cuda_stream);
 }
@@ -243,7 +251,7 @@ int rlcs_retrace(const float* rewards, const float* q_sa, const float* expected_
     p.f0 = rewards; p.f1 = q_sa; p.f2 = expected_q; p.f3 = log_rhos; p.out0 = q_targets;
     p.gamma = gamma; p.aux = gamma * lambda; p.c_bar = c_bar;
     const int variant = choose_variant(rlcs::kRetrace, truncs != nullptr, total, T);
-    st = finish_params(p, variant, total, T, workspace, workspace_bytes);
+    st = finish_params(p, variant, total, T, workspace, workspace_bytes, vec);
     if (st != RLCS_OK) return st;
     return run(rlcs::launch_retrace, p, variant, truncs != nullptr, vec, cuda_stream);
 }
@@ -263,7 +271,7 @@ int rlcs_td_lambda(const float* rewards, const float* values, const uint8_t* don
     p.f0 = rewards; p.f1 = values; p.out0 = returns;
     p.gamma = gamma; p.decay = gamma * lambda; p.aux = gamma * (1.f - lambda);
     const int variant = choose_variant(rlcs::kTdLambda, truncs != nullptr, total, T);
-    st = finish_params(p, variant, total, T, workspace, workspace_bytes);
+    st = finish_params(p, variant, total, T, workspace, workspace_bytes, vec);
     if (st != RLCS_OK) return st;
     return run(rlcs::launch_td_lambda, p, variant, truncs != nullptr, vec, cuda_stream);
 }
@@ -283,7 +291,7 @@ int rlcs_discounted_return(const float* rewards, const uint8_t* dones, const uin
     p.f0 = rewards; p.out0 = returns;
     p.gamma = gamma; p.decay = gamma;
     const int variant = choose_variant(rlcs::kDisc, truncs != nullptr, total, T);
-    st = finish_params(p, variant, total, T, workspace, workspace_bytes);
+    st = finish_params(p, variant, total, T, workspace, workspace_bytes, vec);
     if (st != RLCS_OK) return st;
     return run(rlcs::launch_disc, p, variant, truncs != nullptr, vec, cuda_stream);
 }
@@ -302,7 +310,7 @@ static int forward_scan(rlcs::Algo algo, const float* x, const uint8_t* dones, f
     if (st != RLCS_OK) return st;
     p.f0 = x; p.dones = dones; p.out0 = out; p.decay = decay; p.starts_at = starts_at != 0;
     const int variant = choose_variant(algo, false, total, T);
-    st = finish_params(p, variant, total, T, workspace, workspace_bytes);
+    st = finish_params(p, variant, total, T, workspace, workspace_bytes, vec);
     if (st != RLCS_OK) return st;
     return run(algo == rlcs::kElig ? rlcs::launch_elig : rlcs::launch_prefix, p, variant, false, vec, cuda_stream);
 }
@@ -332,7 +340,7 @@ int rlcs_affine_scan(const float* alpha, const float* beta, float* out, int64_t 
     if (st != RLCS_OK) return st;
     p.f0 = alpha; p.f1 = beta; p.out0 = out;
     const int variant = choose_variant(forward ? rlcs::kAffineFwd : rlcs::kAffineBwd, false, total, T);
-    st = finish_params(p, variant, total, T, workspace, workspace_bytes);
+    st = finish_params(p, variant, total, T, workspace, workspace_bytes, vec);
     if (st != RLCS_OK) return st;
     return run(forward ? rlcs::launch_affine_fwd : rlcs::launch_affine_bwd, p, variant, false, vec, cuda_stream);
 }
@@ -361,6 +369,11 @@ int rlcs_debug_variant_info(int variant, int* threads, int* steps_per_thread, in
     if (steps_per_thread) *steps_per_thread = tv.items;
     if (blocks_per_sm) *blocks_per_sm = tv.min_blocks;
     if (ring_stages) *ring_stages = tv.stages;
+    return RLCS_OK;
+}
+
+int rlcs_debug_allow_cluster_carry(int on) {
+    g_cluster = on != 0;
     return RLCS_OK;
 }
 

@@ -65,9 +65,31 @@ cudaError_t launch_persistent(const ScanParams& p, cudaStream_t stream) {
     return cudaGetLastError();
 }
 
+// One cluster per row (p.cluster = tiles per row, 2..8): carry through distributed shared memory.
+template <int ALGO, bool TRUNC, int V>
+cudaError_t launch_cluster(const ScanParams& p, cudaStream_t stream) {
+    constexpr TileVariant tv = kVariants[V];
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)p.num_tiles, 1, 1);
+    cfg.blockDim = dim3(tv.threads, 1, 1);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)p.cluster;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, scan_kernel_cluster<ALGO, TRUNC, tv.threads, tv.items, tv.min_blocks>, p);
+}
+
 template <int ALGO, bool TRUNC, bool VEC, int V>
 cudaError_t launch_variant(const ScanParams& p, cudaStream_t stream) {
     constexpr TileVariant tv = kVariants[V];
+    if constexpr (VEC && tv.stages == 0) {
+        if (p.cluster > 1) return launch_cluster<ALGO, TRUNC, V>(p, stream);
+    }
     if constexpr (tv.stages > 0 && VEC) {
         // (rows shorter than a chunk go to the one-tile kernel: the persistent one assumes T >= ITEMS)
         if (p.T >= (unsigned)tv.items) return launch_persistent<ALGO, TRUNC, V>(p, stream);

@@ -30,6 +30,7 @@
 // chunk -- patch the packed words in short side paths.
 #pragma once
 
+#include <cooperative_groups.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -84,6 +85,7 @@ struct ScanParams {
     float rho_bar, c_bar;
     int starts_at;
     int carry_mode;           // rows may straddle tiles: publish aggregates, look back
+    int cluster;              // > 1: rows are exactly this many tiles long, one thread-block cluster per row
     unsigned* header;         // workspace header (carry mode) or nullptr
     unsigned* status;         // device status word, or nullptr when there is no workspace
     uint4* records;           // one 16-byte record per tile: {alpha_bits, epoch, beta_bits, epoch}
@@ -448,7 +450,42 @@ struct ScanSmem {
     Pair agg[2][NW];     // warp aggregates, indexed by the warp's rank in scan order
     float carry[2];      // tile carry-in
     int need[2];         // the tile is entered mid-episode
+    Pair cl_agg;         // cluster carry: this tile's aggregate, read by the other blocks of the cluster
 };
+
+// Carry between the thread blocks of one cluster (rows that are exactly 2..8 tiles long: one
+// cluster per row, block rank = the tile's position in scan order inside the row).  Every block
+// leaves its tile aggregate in its own shared memory; after a cluster barrier one warp reads the
+// aggregates of the preceding tiles through distributed shared memory and folds them in the same
+// fixed order as the look-back (nearest first, cut at the first beta = 0).  No global scratch, no
+// polling.  Returns the arrival token of the second cluster barrier: a block must not exit before
+// every peer has finished reading its shared memory, so the caller waits on it at the very end.
+template <int NW>
+__device__ __forceinline__ float cluster_carry(Pair tile_agg, ScanSmem<NW>& sm, int buf) {
+    namespace cg = cooperative_groups;
+    cg::cluster_group cl = cg::this_cluster();
+    const unsigned r = cl.block_rank();
+    const int lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) sm.cl_agg = tile_agg;
+    cl.sync();
+    if (threadIdx.x < 32) {
+        Pair q = {0.f, 0.f};                                   // lanes >= r: terminators
+        if ((unsigned)lane < r) q = *cl.map_shared_rank(&sm.cl_agg, r - 1 - lane);
+        const unsigned zer = __ballot_sync(0xffffffffu, q.b == 0.f);
+        const int z = __ffs(zer) - 1;                          // exists: r <= 8 < 32
+        Pair cur = (lane <= z) ? q : Pair{0.f, 1.f};
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            Pair o;
+            o.a = __shfl_down_sync(0xffffffffu, cur.a, d);
+            o.b = __shfl_down_sync(0xffffffffu, cur.b, d);
+            if (lane + d < 32 && cur.b != 0.f) cur = apply(cur, o);
+        }
+        if (lane == 0) sm.carry[buf] = cur.a;
+    }
+    cl.sync();          // the carry is visible to the block, and nobody reads remote memory any more
+    return sm.carry[buf];
+}
 
 struct NoHook {
     __device__ __forceinline__ void operator()() const {}
@@ -460,7 +497,8 @@ struct NoHook {
 // which removes the ragged-chunk and short-row side paths at compile time.
 // LAST: this is the block's last tile of the call; the block then signs off from the carry protocol
 // as soon as its own look-back is over (see sign_off) instead of after its stores.
-template <int ALGO, bool TRUNC, bool VEC, int THREADS, int ITEMS, bool FULL, bool LAST, class Hook>
+// CLUSTER: the carry between blocks goes through distributed shared memory (cluster_carry).
+template <int ALGO, bool TRUNC, bool VEC, int THREADS, int ITEMS, bool FULL, bool LAST, class Hook, bool CLUSTER = false>
 __device__ __forceinline__ void tile_compute(Chunk<ALGO, TRUNC, ITEMS>& c, Vals<ITEMS>& v, const ScanParams& p, long long i0, long long s,
                                              unsigned epoch, ScanSmem<THREADS / 32>& sm, int buf, Hook after_barrier) {
     constexpr bool FWD = is_forward(ALGO);
@@ -646,7 +684,9 @@ __device__ __forceinline__ void tile_compute(Chunk<ALGO, TRUNC, ITEMS>& c, Vals<
 
     // ---- carry between thread blocks
     float carry_in = 0.f;
-    if (p.carry_mode) {
+    if constexpr (CLUSTER) {
+        carry_in = cluster_carry<NW>(tile_agg, sm, buf);
+    } else if (p.carry_mode) {
         if (warp == 0 && lane == 0 && s != p.mute_tile) {
             st_volatile_u4(p.records + s, make_uint4(__float_as_uint(tile_agg.a), epoch,
                                                      __float_as_uint(tile_agg.b), epoch));
@@ -737,6 +777,29 @@ __global__ void __launch_bounds__(THREADS, MIN_BLOCKS) scan_kernel(const ScanPar
     const bool full = (tile * TILE + TILE <= p.total) && (p.T >= (unsigned)ITEMS);
     if (full) one_tile<ALGO, TRUNC, VEC, THREADS, ITEMS, true>(p, tile, s, epoch, sm);
     else one_tile<ALGO, TRUNC, VEC, THREADS, ITEMS, false>(p, tile, s, epoch, sm);
+}
+
+// ------------------------------------------------------------------------------------------ kernel 1b: one tile per block, one cluster per row
+// For rows that are exactly 2..8 tiles long (T = k * TILE): launched with cluster size k, so a
+// cluster is a row and the carry stays on chip.  All tiles are full; 32-byte aligned pointers.
+template <int ALGO, bool TRUNC, int THREADS, int ITEMS, int MIN_BLOCKS>
+__global__ void __launch_bounds__(THREADS, MIN_BLOCKS) scan_kernel_cluster(const ScanParams p) {
+    constexpr bool FWD = is_forward(ALGO);
+    constexpr int TILE = THREADS * ITEMS;
+    __shared__ ScanSmem<THREADS / 32> sm;
+    const int tid = threadIdx.x;
+    const int lane = tid & 31;
+    const long long s = blockIdx.x;
+    const long long tile = FWD ? s : (p.num_tiles - 1 - s);
+    Chunk<ALGO, TRUNC, ITEMS> c;
+    const long long i0 = tile * TILE + (long long)tid * ITEMS;
+    const long long n0 = locate(c, p, i0);
+    load_flags_global<ALGO, TRUNC, ITEMS, true, true>(c, p, i0, lane);
+    Vals<ITEMS> v;
+    load_values_global<ALGO, TRUNC, ITEMS, true, true>(c, v, p, i0, lane);
+    issue_boot(c, p, n0);
+    issue_trunc_values(c, p, i0);
+    tile_compute<ALGO, TRUNC, true, THREADS, ITEMS, true, false, NoHook, true>(c, v, p, i0, s, 0u, sm, 0, NoHook{});
 }
 
 // ------------------------------------------------------------------------------------------ mbarrier / bulk copy (PTX)

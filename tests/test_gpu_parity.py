@@ -106,6 +106,31 @@ def test_long_row_without_resets_multi_window_lookback(oracle, W, B):
         B.rlcs_debug_set_tile_variant(BASE_VARIANT)
 
 
+def test_randomized_shapes_flags_and_options(oracle, W, B):
+    """Seeded fuzz over shapes, flag densities, kernel variants, pointer offsets and NULL options."""
+    rng = np.random.default_rng(20260817)
+    n_variants = 19
+    for case in range(60):
+        N = int(rng.integers(1, 200))
+        T = int(rng.choice([rng.integers(1, 40), rng.integers(40, 3000), rng.integers(3000, 12000)]))
+        if N * T > 600_000:
+            N = max(1, 600_000 // T)
+        p_done = float(rng.choice([0.0, 0.001, 0.02, 0.3]))
+        p_trunc = float(rng.choice([0.0, 0.005, 0.2]))
+        ro = W.make_rollout(108, N, T, p_done=p_done, p_trunc=p_trunc, salt=case)
+        ro.params.update(gamma=float(rng.choice([0.9, 0.99, 1.0])), lam=float(rng.choice([0.0, 0.5, 0.95, 1.0])),
+                         rho_bar=float(rng.choice([0.5, 1.0, 2.0])), c_bar=float(rng.choice([0.5, 1.0])))
+        variant = int(rng.choice([BASE_VARIANT, int(rng.integers(0, n_variants))]))
+        B.rlcs_debug_set_tile_variant(variant)
+        try:
+            compare_all(oracle, ro, offset=int(rng.choice([0, 0, 0, 1, 4, 8])),
+                        use_truncs=bool(rng.random() < 0.7), use_bootstrap=bool(rng.random() < 0.8))
+        except AssertionError as e:
+            raise AssertionError(f"case {case}: N={N} T={T} p_done={p_done} p_trunc={p_trunc} variant={variant}: {e}")
+        finally:
+            B.rlcs_debug_set_tile_variant(BASE_VARIANT)
+
+
 # ------------------------------------------------------------------ boundary cases
 def _forced(W, N=6, T=300, salt=0):
     ro = W.make_rollout(93, N, T, p_done=0.02, p_trunc=0.02, salt=salt)
@@ -194,6 +219,27 @@ def test_large_problem_variants_with_carry(oracle, W, B):
         info = B.rlcs_debug_variant_for(name, True, ro.N, ro.T)
         assert BASE_VARIANT != -1 or info["variant"] not in (0, 6), (a, info)
     compare_all(oracle, ro)
+
+
+@pytest.mark.parametrize("N,T,variant", [(5, 4096, 0), (3, 16384, 0), (64, 2048, 6), (7, 8192, 6), (9, 3072, 3), (2, 32768, 7)])
+def test_cluster_carry_for_rows_of_whole_tiles(oracle, W, B, N, T, variant):
+    """Rows of exactly 2..8 tiles: one thread-block cluster per row, carry in distributed shared
+    memory and no workspace.  Against the oracle and against the workspace look-back."""
+    tile = B.rlcs_debug_tile_elems(variant)
+    assert T % tile == 0 and 2 <= T // tile <= 8
+    ro = W.make_rollout(109, N, T, p_done=0.0005, p_trunc=0.0005, salt=T)
+    B.rlcs_debug_set_tile_variant(variant)
+    try:
+        gpu, ref, _ = compare_all(oracle, ro, workspace=None)          # no workspace needed on this path
+        B.rlcs_debug_allow_cluster_carry(False)
+        other = run_gpu(Dev(ro), ALL_ALGOS)
+    finally:
+        B.rlcs_debug_allow_cluster_carry(True)
+        B.rlcs_debug_set_tile_variant(BASE_VARIANT)
+    for a in ALL_ALGOS:
+        pairs = zip(gpu[a], other[a]) if isinstance(gpu[a], tuple) else [(gpu[a], other[a])]
+        for x, y in pairs:
+            np.testing.assert_allclose(x, y, rtol=1e-5, atol=1e-5, err_msg=a)
 
 
 def test_wide_index_path_gives_identical_results(oracle, W, B):
@@ -326,12 +372,14 @@ def test_bounded_carry_wait_reports_timeout_and_returns(oracle, W, B):
     dev = Dev(ro)
     ws = B.Workspace(ro.N, ro.T)
     B.rlcs_debug_set_carry_fault(2, 64)
+    B.rlcs_debug_allow_cluster_carry(False)           # this row length would otherwise carry on chip
     try:
         B.rlcs_discounted_return(dev.rewards, dev.dones, gamma=0.99, workspace=ws)
         torch.cuda.synchronize()
         assert ws.device_status() == B.RLCS_ERR_TIMEOUT
     finally:
         B.rlcs_debug_set_carry_fault(-1, 0)
+        B.rlcs_debug_allow_cluster_carry(True)
     assert ws.device_status() == B.RLCS_OK            # cleared by the read
     compare_all(oracle, ro, algos=("discounted_return",), workspace=ws)
 
