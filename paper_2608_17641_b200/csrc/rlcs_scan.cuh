@@ -458,8 +458,13 @@ struct ScanSmem {
 // leaves its tile aggregate in its own shared memory; after a cluster barrier one warp reads the
 // aggregates of the preceding tiles through distributed shared memory and folds them in the same
 // fixed order as the look-back (nearest first, cut at the first beta = 0).  No global scratch, no
-// polling.  Returns the arrival token of the second cluster barrier: a block must not exit before
-// every peer has finished reading its shared memory, so the caller waits on it at the very end.
+// polling.  A block must not exit before every peer has finished reading its shared memory: each
+// thread arrives at a second cluster barrier here, right after the remote reads, and the caller
+// waits on it (cluster_exit_wait) after its stores, so that wait overlaps the rest of the tile.
+__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_exit_wait() { cluster_wait(); }
+
 template <int NW>
 __device__ __forceinline__ float cluster_carry(Pair tile_agg, ScanSmem<NW>& sm, int buf) {
     namespace cg = cooperative_groups;
@@ -467,7 +472,8 @@ __device__ __forceinline__ float cluster_carry(Pair tile_agg, ScanSmem<NW>& sm, 
     const unsigned r = cl.block_rank();
     const int lane = threadIdx.x & 31;
     if (threadIdx.x == 0) sm.cl_agg = tile_agg;
-    cl.sync();
+    cluster_arrive();
+    cluster_wait();                                            // every block's aggregate is in place
     if (threadIdx.x < 32) {
         Pair q = {0.f, 0.f};                                   // lanes >= r: terminators
         if ((unsigned)lane < r) q = *cl.map_shared_rank(&sm.cl_agg, r - 1 - lane);
@@ -483,7 +489,8 @@ __device__ __forceinline__ float cluster_carry(Pair tile_agg, ScanSmem<NW>& sm, 
         }
         if (lane == 0) sm.carry[buf] = cur.a;
     }
-    cl.sync();          // the carry is visible to the block, and nobody reads remote memory any more
+    cluster_arrive();                                          // this thread reads no remote memory any more
+    __syncthreads();                                           // the carry is visible to the block
     return sm.carry[buf];
 }
 
@@ -739,6 +746,7 @@ __device__ __forceinline__ void tile_compute(Chunk<ALGO, TRUNC, ITEMS>& c, Vals<
             if (p.out1 != nullptr) store_f32<ITEMS, VEC>(p.out1, i0, nvalid, out1v);
         }
     }
+    if constexpr (CLUSTER) cluster_exit_wait();
 }
 
 // ------------------------------------------------------------------------------------------ end of a call (carry mode)
