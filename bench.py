@@ -218,6 +218,31 @@ def time_device(batch: GpuBatch, steps: int, warmup: int, dist):
     return total_ms, per_algo_ms, batch.launches - launches0, clk.summary()
 
 
+def time_gae_normalized(batch: GpuBatch, steps: int, peak: float):
+    """Extension beyond the seven kernels: GAE + advantage normalisation (three launches) on the
+    bench batch; algorithmic bytes = GAE's plus one read and one write of the advantages."""
+    torch, B, ro = batch.torch, batch.B, batch.ro
+    i, o, p = batch.inp, batch.out, ro.params
+    ws = B.Workspace(ro.N, ro.T, nbytes=int(B.lib().rlcs_gae_normalized_workspace_bytes(ro.N, ro.T)))
+    call = lambda: B.rlcs_gae_normalized(i["rewards"], i["values"], i["dones"], i["truncs"], i["trunc_bootstrap"],
+                                         i["bootstrap"], gamma=p["gamma"], lam=p["lam"], eps=1e-8, ddof=1,
+                                         advantages=o["gae"][0], returns=o["gae"][1], workspace=ws)
+    for _ in range(3):
+        call()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(steps):
+        call()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    ab = algorithmic_bytes(ro, "gae") + 8 * ro.N * ro.T
+    gbs = ab / (ms * 1e-3) / 1e9
+    return {"ms": round(ms, 5), "launches_per_call": 3, "env_steps_per_s": ro.N * ro.T / (ms * 1e-3),
+            "algorithmic_bytes": ab, "gbs": round(gbs, 1), "frac_of_peak": round(gbs / peak, 4)}
+
+
 def time_e2e(batch: GpuBatch, steps: int, warmup: int, dist):
     """The same step called with HOST buffers: every step copies that step's inputs from pinned
     host memory to the device, runs the seven C-ABI calls, and reads all outputs back to pinned
@@ -521,6 +546,7 @@ def main():
                 "all_kernels_frac": round(sum(v["algorithmic_bytes"] for v in per_algo.values())
                                           / (sum(v["ms"] for v in per_algo.values()) * 1e-3) / 1e9 / peak, 4)}
 
+    extensions = {"gae_normalized": time_gae_normalized(batch, max(3, min(args.steps, 50)), peak)}
     e2e_steps = max(1, min(args.steps, 8))
     e2e_ms, h2d, d2h = time_e2e(batch, e2e_steps, 1, dist)
     e2e_ms = dist.max(e2e_ms)
@@ -538,6 +564,7 @@ def main():
                    "env_steps_per_step_per_gpu": len(ALGOS) * ro.N * ro.T, "launches_per_step": len(ALGOS),
                    "l2": "inputs larger than L2 (2.2 GB touched per step), no flush"},
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "per_algorithm": per_algo,
+        "extensions": extensions,
     }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline(ro)

@@ -101,6 +101,26 @@ int rlcs_gae(const float* rewards, const float* values, const uint8_t* dones, co
              void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * GAE followed by advantage normalisation, the step directly downstream of GAE in PPO-style
+ * training.  Section 9.3 lists "fused advantage normalization" as a planned extension without
+ * defining it; the convention taken here is the usual one, over all N*T steps of the call:
+ *   advantages[n,t] = (A_t - mean(A)) / (std(A) + eps),   std = sqrt(sum (A - mean)^2 / (N*T - ddof)),
+ *   ddof = 0 (population) or 1 (sample; std = 0 when N*T = 1);   eps >= 0, finite
+ *   returns[n,t]    = A_t + values_t  from the un-normalised A_t  (may be NULL)
+ * Three launches: the GAE kernel (which also leaves per-tile sums of A and A^2), a one-block
+ * reduction to mean and 1/(std + eps), and an in-place rescale of `advantages` -- one read of A
+ * fewer than GAE, a statistics pass and a rescale.  Deterministic (fixed reduction order).
+ * `workspace`: at least rlcs_gae_normalized_workspace_bytes(N, T) bytes (always > 0), 16-byte
+ * aligned, initialised once with rlcs_workspace_init; same sharing rules as any workspace.
+ */
+int rlcs_gae_normalized(const float* rewards, const float* values, const uint8_t* dones, const uint8_t* truncs,
+                        const float* trunc_bootstrap, const float* bootstrap, float* advantages, float* returns,
+                        int64_t N, int64_t T, float gamma, float lambda, float eps, int ddof,
+                        void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+size_t rlcs_gae_normalized_workspace_bytes(int64_t N, int64_t T);
+
+/*
  * V-Trace -- Section 3.3.2, Table 1 row "V-Trace".  log_rhos[n,t] = log pi(a_t|s_t) - log mu(a_t|s_t).
  *   rho_t = min(rho_bar, exp(log_rhos_t));   c_t = min(c_bar, exp(log_rhos_t))
  *   Delta_t = rho_t*(rewards_t + gamma*values_next(t) - values_t) + (cont_t ? gamma*c_t*Delta_{t+1} : 0)

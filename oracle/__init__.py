@@ -123,6 +123,19 @@ def gae(rewards, values, dones, truncs=None, trunc_bootstrap=None, bootstrap=Non
     return (adv, ret) if want_returns else adv
 
 
+def gae_normalized(rewards, values, dones, truncs=None, trunc_bootstrap=None, bootstrap=None, *, gamma, lam,
+                   eps=1e-8, ddof=1):
+    """GAE, then (A - mean) / (std + eps) over all N*T steps; std with `ddof` (0 when N*T <= ddof).
+    The paper only names this step (planned extension, Section 9.3); this is the usual PPO convention.
+    Plain fp64 sums; returns (normalised advantages, returns = A + V from the raw A)."""
+    adv, ret = gae(rewards, values, dones, truncs, trunc_bootstrap, bootstrap, gamma=gamma, lam=lam)
+    n = adv.size
+    mean = adv.sum() / n
+    dev2 = ((adv - mean) ** 2).sum()
+    std = np.sqrt(dev2 / (n - ddof)) if n > ddof else 0.0
+    return (adv - mean) / (std + float(np.float32(eps))), ret
+
+
 def td_lambda(rewards, values, dones, truncs=None, trunc_bootstrap=None, bootstrap=None, *, gamma, lam):
     """TD(lambda) returns -- Section 3.3.4."""
     shape = _shape2(rewards)

@@ -27,6 +27,8 @@ SIGNATURES = {
     "rlcs_workspace_init": ([_vp, _sz, _vp], _int),
     "rlcs_last_device_status": ([_vp, _vp], _int),
     "rlcs_gae": ([_vp] * 8 + [_i64, _i64, _f, _f] + _TAIL, _int),
+    "rlcs_gae_normalized": ([_vp] * 8 + [_i64, _i64, _f, _f, _f, _int] + _TAIL, _int),
+    "rlcs_gae_normalized_workspace_bytes": ([_i64, _i64], _sz),
     "rlcs_vtrace": ([_vp] * 9 + [_i64, _i64, _f, _f, _f] + _TAIL, _int),
     "rlcs_retrace": ([_vp] * 9 + [_i64, _i64, _f, _f, _f] + _TAIL, _int),
     "rlcs_td_lambda": ([_vp] * 7 + [_i64, _i64, _f, _f] + _TAIL, _int),
@@ -149,6 +151,24 @@ def rlcs_gae(rewards, values, dones, truncs=None, trunc_bootstrap=None, bootstra
                           _ptr(truncs, "u8", (N, T)), _ptr(trunc_bootstrap, "f32", (N, T)),
                           _ptr(bootstrap, "f32", (N,)), _ptr(adv, "f32", (N, T)), _ptr(ret, "f32", (N, T)),
                           N, T, gamma, lam, wp, wb, _stream(stream)))
+    return (adv, ret) if want_returns else adv
+
+
+def rlcs_gae_normalized(rewards, values, dones, truncs=None, trunc_bootstrap=None, bootstrap=None, *, gamma, lam,
+                        eps=1e-8, ddof=1, advantages=None, returns=None, want_returns=True, workspace=None, stream=None):
+    """GAE + advantage normalisation over all N*T steps.  `workspace` must be a Workspace created with
+    nbytes=rlcs_gae_normalized_workspace_bytes(N, T) (one is made on the fly when omitted)."""
+    N, T = rewards.shape
+    adv = _out(rewards, advantages)
+    ret = (_out(rewards, returns) if want_returns else None)
+    if workspace is None:
+        workspace = Workspace(N, T, device=rewards.device, stream=stream,
+                              nbytes=int(lib().rlcs_gae_normalized_workspace_bytes(N, T)))
+    wp, wb = _ws(workspace)
+    _check(lib().rlcs_gae_normalized(_ptr(rewards, "f32"), _ptr(values, "f32", (N, T)), _ptr(dones, "u8", (N, T)),
+                                     _ptr(truncs, "u8", (N, T)), _ptr(trunc_bootstrap, "f32", (N, T)),
+                                     _ptr(bootstrap, "f32", (N,)), _ptr(adv, "f32", (N, T)), _ptr(ret, "f32", (N, T)),
+                                     N, T, gamma, lam, eps, ddof, wp, wb, _stream(stream)))
     return (adv, ret) if want_returns else adv
 
 

@@ -66,7 +66,8 @@ int choose_variant(int algo, bool trunc, int64_t total, int64_t T) {
     if (g_variant >= 0) return g_variant;
     if (total < (int64_t(1) << 23)) return T <= 2048 ? 6 : 0;
     switch (algo) {
-        case rlcs::kGae: return trunc ? 16 : 0;
+        case rlcs::kGae:
+        case rlcs::kGaeStats: return trunc ? 16 : 0;
         case rlcs::kVtrace: return trunc ? 18 : 0;
         case rlcs::kRetrace: return 0;
         case rlcs::kTdLambda: return trunc ? 17 : 0;
@@ -212,6 +213,49 @@ int rlcs_gae(const float* rewards, const float* values, const uint8_t* dones, co
     st = finish_params(p, variant, total, T, workspace, workspace_bytes, vec);
     if (st != RLCS_OK) return st;
     return run(rlcs::launch_gae, p, variant, truncs != nullptr, vec, cuda_stream);
+}
+
+// Layout of the workspace of rlcs_gae_normalized: the carry workspace of rlcs_workspace_bytes (rounded
+// up to 256 bytes), then {mean, 1/(std+eps)} in a 256-byte slot, then one {sum, sum of squares} pair per tile.
+static size_t norm_carry_bytes(int64_t N, int64_t T) { return (rlcs_workspace_bytes(N, T) + 255) / 256 * 256; }
+
+size_t rlcs_gae_normalized_workspace_bytes(int64_t N, int64_t T) {
+    int64_t total = 0;
+    if (check_sizes(N, T, &total) != RLCS_OK || total == 0) return 0;
+    const int64_t tiles = (total + rlcs::kMinTileElems - 1) / rlcs::kMinTileElems;
+    return norm_carry_bytes(N, T) + 256 + 2 * sizeof(float) * (size_t)tiles;
+}
+
+int rlcs_gae_normalized(const float* rewards, const float* values, const uint8_t* dones, const uint8_t* truncs,
+                        const float* trunc_bootstrap, const float* bootstrap, float* advantages, float* returns,
+                        int64_t N, int64_t T, float gamma, float lambda, float eps, int ddof, void* workspace,
+                        size_t workspace_bytes, void* cuda_stream) {
+    ScanParams p = {};
+    Ptrs ps;
+    int64_t total;
+    bool vec;
+    if (!unit_interval(gamma) || !unit_interval(lambda) || !(eps >= 0.f) || std::isinf(eps) || (ddof != 0 && ddof != 1))
+        return RLCS_ERR_ARG;
+    ps.add_f32(rewards); ps.add_f32(values); ps.add_f32(advantages); ps.add_f32(returns);
+    int st = backward_common(p, ps, dones, truncs, trunc_bootstrap, bootstrap, N, T, &total, &vec);
+    if (st != RLCS_OK || total == 0) return st;
+    if (!rewards || !values || !advantages) return RLCS_ERR_NULL;
+    if (workspace == nullptr || workspace_bytes < rlcs_gae_normalized_workspace_bytes(N, T)) return RLCS_ERR_WORKSPACE;
+    if (!aligned(workspace, 16)) return RLCS_ERR_ALIGN;
+    const size_t carry_bytes = norm_carry_bytes(N, T);
+    float* mean_rstd = reinterpret_cast<float*>(static_cast<unsigned char*>(workspace) + carry_bytes);
+    p.f0 = rewards; p.f1 = values; p.out0 = advantages; p.out1 = returns;
+    p.stats = mean_rstd + 64;
+    p.gamma = gamma; p.decay = gamma * lambda;
+    const int variant = choose_variant(rlcs::kGaeStats, truncs != nullptr, total, T);
+    st = finish_params(p, variant, total, T, carry_bytes ? workspace : nullptr, carry_bytes, vec);
+    if (st != RLCS_OK) return st;
+    st = run(rlcs::launch_gae_stats, p, variant, truncs != nullptr, vec, cuda_stream);
+    if (st != RLCS_OK) return st;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    if (rlcs::launch_norm_finalize(p.stats, p.num_tiles, (double)total, ddof, eps, mean_rstd, s) != cudaSuccess) return RLCS_ERR_CUDA;
+    if (rlcs::launch_norm_rescale(advantages, total, mean_rstd, vec, s) != cudaSuccess) return RLCS_ERR_CUDA;
+    return RLCS_OK;
 }
 
 int rlcs_vtrace(const float* rewards, const float* values, const float* log_rhos, const uint8_t* dones,

@@ -134,6 +134,10 @@ cudaError_t launch_elig(const ScanParams&, int variant, bool trunc, bool vec, cu
 cudaError_t launch_prefix(const ScanParams&, int variant, bool trunc, bool vec, cudaStream_t);
 cudaError_t launch_affine_bwd(const ScanParams&, int variant, bool trunc, bool vec, cudaStream_t);
 cudaError_t launch_affine_fwd(const ScanParams&, int variant, bool trunc, bool vec, cudaStream_t);
+cudaError_t launch_gae_stats(const ScanParams&, int variant, bool trunc, bool vec, cudaStream_t);
+cudaError_t launch_norm_finalize(const float* partial, long long num_tiles, double count, int ddof, float eps,
+                                 float* mean_rstd, cudaStream_t stream);
+cudaError_t launch_norm_rescale(float* adv, long long total, const float* mean_rstd, bool vec, cudaStream_t stream);
 
 #define RLCS_DEFINE_LAUNCHER(NAME, ALGO, HAS_TRUNC)                                                 \
     cudaError_t NAME(const ScanParams& p, int variant, bool trunc, bool vec, cudaStream_t stream) { \

@@ -38,11 +38,13 @@ namespace rlcs {
 
 enum Algo : int {
     kGae = 0, kTdLambda = 1, kDisc = 2, kVtrace = 3, kRetrace = 4, kElig = 5, kPrefix = 6,
-    kAffineBwd = 7, kAffineFwd = 8
+    kAffineBwd = 7, kAffineFwd = 8,
+    kGaeStats = 9     // GAE that also leaves per-tile sums of A and A^2 (for advantage normalisation)
 };
 
 __host__ __device__ constexpr bool is_forward(int a) { return a == kElig || a == kPrefix || a == kAffineFwd; }
-__host__ __device__ constexpr bool has_values(int a) { return a == kGae || a == kTdLambda || a == kVtrace; }
+__host__ __device__ constexpr bool is_gae(int a) { return a == kGae || a == kGaeStats; }
+__host__ __device__ constexpr bool has_values(int a) { return is_gae(a) || a == kTdLambda || a == kVtrace; }
 __host__ __device__ constexpr bool is_affine(int a) { return a == kAffineBwd || a == kAffineFwd; }
 __host__ __device__ constexpr bool const_decay(int a) { return a != kVtrace && a != kRetrace && !is_affine(a); }
 // a float input is read one step beyond the tile (successor value)
@@ -73,6 +75,7 @@ struct ScanParams {
     const float* boot;        // [N] or nullptr
     float* out0;
     float* out1;              // second output or nullptr
+    float* stats;             // kGaeStats: per scan-order tile {sum A, sum A^2}
     long long total;          // N*T
     long long num_tiles;
     unsigned T;
@@ -588,7 +591,7 @@ __device__ __forceinline__ void tile_compute(Chunk<ALGO, TRUNC, ITEMS>& c, Vals<
             if constexpr (has_values(ALGO)) nextv = (j + 1 < ITEMS) ? v.x1[(j + 1) % ITEMS] : v.halo;
             if constexpr (ALGO == kRetrace) nextv = (j + 1 < ITEMS) ? v.x2[(j + 1) % ITEMS] : v.halo;
             const float xn = cut ? c.ov[j] : nextv;      // successor value of Section 3.2 (selected, never multiplied)
-            if constexpr (ALGO == kGae) {
+            if constexpr (is_gae(ALGO)) {
                 v.a[j] = fmaf(p.gamma, xn, r) - v.x1[j];
                 beta[j] = cut ? 0.f : p.decay;
             } else if constexpr (ALGO == kTdLambda) {
@@ -724,7 +727,7 @@ __device__ __forceinline__ void tile_compute(Chunk<ALGO, TRUNC, ITEMS>& c, Vals<
 #pragma unroll
         for (int j = ITEMS - 1; j >= 0; --j) {
             const float d = fmaf(beta[j], prev, v.a[j]);
-            if constexpr (ALGO == kGae) {
+            if constexpr (is_gae(ALGO)) {
                 v.a[j] = d;
                 out1v[j] = d + v.x1[j];
             } else if constexpr (ALGO == kVtrace) {
@@ -742,8 +745,37 @@ __device__ __forceinline__ void tile_compute(Chunk<ALGO, TRUNC, ITEMS>& c, Vals<
     }
     if (nvalid > 0) {
         store_f32<ITEMS, VEC>(p.out0, i0, nvalid, v.a);
-        if constexpr (ALGO == kGae || ALGO == kVtrace) {
+        if constexpr (is_gae(ALGO) || ALGO == kVtrace) {
             if (p.out1 != nullptr) store_f32<ITEMS, VEC>(p.out1, i0, nvalid, out1v);
+        }
+    }
+    // ---- per-tile sums of A and A^2, in a fixed order (deterministic), for the normalisation pass
+    if constexpr (ALGO == kGaeStats) {
+        float s1 = 0.f, s2 = 0.f;
+#pragma unroll
+        for (int j = 0; j < ITEMS; ++j) {         // steps beyond the array hold A = 0
+            s1 += v.a[j];
+            s2 = fmaf(v.a[j], v.a[j], s2);
+        }
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) {
+            s1 += __shfl_xor_sync(ALL, s1, d);
+            s2 += __shfl_xor_sync(ALL, s2, d);
+        }
+        __syncthreads();                           // the scan's use of sm.agg is over
+        if (lane == 0) sm.agg[buf][warp] = Pair{s1, s2};
+        __syncthreads();
+        if (warp == 0) {
+            Pair w = (lane < NW) ? sm.agg[buf][lane] : Pair{0.f, 0.f};
+#pragma unroll
+            for (int d = 16; d > 0; d >>= 1) {
+                w.a += __shfl_xor_sync(ALL, w.a, d);
+                w.b += __shfl_xor_sync(ALL, w.b, d);
+            }
+            if (lane == 0) {
+                p.stats[2 * s] = w.a;
+                p.stats[2 * s + 1] = w.b;
+            }
         }
     }
     if constexpr (CLUSTER) cluster_exit_wait();

@@ -347,6 +347,43 @@ def test_workspace_reuse_across_algorithms_and_shapes(oracle, W, B):
         compare_all(oracle, ro, workspace=big)
 
 
+# ------------------------------------------------------------------ GAE + advantage normalisation
+@pytest.mark.parametrize("N,T", [(1, 1), (3, 7), (8, 128), (37, 1000), (64, 4096), (4096, 64), (5000, 2048)])
+@pytest.mark.parametrize("ddof", [0, 1])
+def test_gae_normalized(oracle, W, B, N, T, ddof):
+    ro = W.make_rollout(110, N, T, salt=T)
+    dev = Dev(ro)
+    p = ro.params
+    ws = B.Workspace(N, T, nbytes=B.lib().rlcs_gae_normalized_workspace_bytes(N, T))
+    for use_tr in (True, False):
+        tr, bv = (dev.truncs, dev.trunc_bootstrap) if use_tr else (None, None)
+        adv, ret = B.rlcs_gae_normalized(dev.rewards, dev.values, dev.dones, tr, bv, dev.bootstrap, gamma=p["gamma"],
+                                         lam=p["lam"], eps=1e-8, ddof=ddof, workspace=ws)
+        ref_adv, ref_ret = oracle.gae_normalized(ro.rewards, ro.values, ro.dones, ro.truncs if use_tr else None,
+                                                 ro.trunc_bootstrap if use_tr else None, ro.bootstrap,
+                                                 gamma=p["gamma"], lam=p["lam"], eps=1e-8, ddof=ddof)
+        assert ws.device_status() == 0
+        assert_close("normalised advantages", adv.cpu().numpy(), ref_adv)
+        assert_close("returns", ret.cpu().numpy(), ref_ret)
+    # deterministic: a second call gives the same bits
+    adv2, _ = B.rlcs_gae_normalized(dev.rewards, dev.values, dev.dones, None, None, dev.bootstrap, gamma=p["gamma"],
+                                    lam=p["lam"], eps=1e-8, ddof=ddof, workspace=ws)
+    assert np.array_equal(adv2.cpu().numpy(), adv.cpu().numpy())
+
+
+def test_gae_normalized_argument_checks(oracle, W, B):
+    ro = W.make_rollout(111, 4, 100)
+    dev = Dev(ro)
+    for kw in (dict(eps=-1.0), dict(eps=float("nan")), dict(eps=float("inf")), dict(ddof=2)):
+        with pytest.raises(B.RlcsError) as e:
+            B.rlcs_gae_normalized(dev.rewards, dev.values, dev.dones, gamma=0.99, lam=0.95, **kw)
+        assert e.value.status == B.RLCS_ERR_ARG
+    small = B.Workspace(4, 100, nbytes=256)
+    with pytest.raises(B.RlcsError) as e:
+        B.rlcs_gae_normalized(dev.rewards, dev.values, dev.dones, gamma=0.99, lam=0.95, workspace=small)
+    assert e.value.status == B.RLCS_ERR_WORKSPACE
+
+
 # ------------------------------------------------------------------ test hooks
 def test_affine_scan_matches_generic_recurrence(oracle, W, B):
     import torch

@@ -543,3 +543,49 @@ def test_rows_parallel_helper_matches_single_call(oracle):
         oracle.gae, dict(rewards=b["r"], values=b["V"], dones=b["term"], truncs=b["trunc"],
                          trunc_bootstrap=b["bv"]), dict(bootstrap=b["boot"]), threads=4, gamma=0.99, lam=0.95)
     assert np.array_equal(one[0], par[0]) and np.array_equal(one[1], par[1])
+
+
+# ----------------------------------------------------------------------------- advantage normalisation
+def test_normalised_advantages_hand_example(oracle):
+    """r = [1, 2, 3], V = 0, gamma = 0: A = r.  mean 2; population std sqrt(2/3), sample std 1."""
+    r = np.array([[1.0, 2.0, 3.0]], np.float32)
+    z = np.zeros((1, 3), np.float32)
+    d = np.zeros((1, 3), np.uint8)
+    a0, ret = oracle.gae_normalized(r, z, d, gamma=0.0, lam=0.9, eps=0.0, ddof=0)
+    np.testing.assert_allclose(a0[0], [-np.sqrt(1.5), 0.0, np.sqrt(1.5)], rtol=1e-14)
+    a1, _ = oracle.gae_normalized(r, z, d, gamma=0.0, lam=0.9, eps=0.0, ddof=1)
+    np.testing.assert_allclose(a1[0], [-1.0, 0.0, 1.0], rtol=1e-14)
+    np.testing.assert_array_equal(ret[0], [1.0, 2.0, 3.0])         # returns stay un-normalised
+
+
+def test_normalised_advantages_match_library_mean_and_std(oracle):
+    b = _batch(31, N=9, T=77)
+    for ddof in (0, 1):
+        for eps in (0.0, 1e-8, 0.5):
+            out, ret = oracle.gae_normalized(b["r"], b["V"], **_bk(b), gamma=0.99, lam=0.95, eps=eps, ddof=ddof)
+            adv, ret0 = oracle.gae(b["r"], b["V"], **_bk(b), gamma=0.99, lam=0.95)
+            want = (adv - np.mean(adv)) / (np.std(adv, ddof=ddof) + float(np.float32(eps)))
+            np.testing.assert_allclose(out, want, rtol=1e-12, atol=1e-12)
+            assert np.array_equal(ret, ret0)
+            if eps == 0.0:
+                assert abs(out.mean()) < 1e-12
+                np.testing.assert_allclose(out.std(ddof=ddof), 1.0, rtol=1e-12)
+
+
+def test_normalised_advantages_scale_invariance_and_degenerate_cases(oracle):
+    """GAE is linear in (rewards, values, bootstraps): scaling them by c > 0 leaves the normalised
+    advantages unchanged (eps = 0).  A constant advantage gives zeros; so does a single step."""
+    b = _batch(32, N=4, T=60)
+    base, _ = oracle.gae_normalized(b["r"], b["V"], **_bk(b), gamma=0.99, lam=0.95, eps=0.0, ddof=1)
+    kw = _bk(b)
+    kw["trunc_bootstrap"] = b["bv"] * np.float32(4.0)
+    kw["bootstrap"] = b["boot"] * np.float32(4.0)
+    scaled, _ = oracle.gae_normalized(b["r"] * np.float32(4.0), b["V"] * np.float32(4.0), **kw, gamma=0.99, lam=0.95,
+                                      eps=0.0, ddof=1)
+    np.testing.assert_allclose(scaled, base, rtol=1e-10, atol=1e-12)
+    ones = np.ones((3, 5), np.float32)
+    const, _ = oracle.gae_normalized(ones, np.zeros_like(ones), np.ones((3, 5), np.uint8), gamma=0.9, lam=0.9, eps=1e-8)
+    assert np.array_equal(const, np.zeros((3, 5)))
+    single, _ = oracle.gae_normalized(ones[:1, :1], ones[:1, :1] * 0, np.zeros((1, 1), np.uint8), gamma=0.9, lam=0.9,
+                                      eps=1e-8, ddof=1)
+    assert single[0, 0] == 0.0
