@@ -243,6 +243,36 @@ def time_gae_normalized(batch: GpuBatch, steps: int, peak: float):
             "algorithmic_bytes": ab, "gbs": round(gbs, 1), "frac_of_peak": round(gbs / peak, 4)}
 
 
+def time_retrace_probs(torch, B, steps: int, peak: float, N=16384, T=2048, A=4):
+    """Extension beyond the seven kernels: Retrace from [N,T,A] Q-values / action probabilities.
+    Algorithmic bytes per step: Q and pi rows (8A), one 32-byte sector of mu for the gathered
+    probability (min(32, 4A)), reward 4, action 4, two masks 2, output 4."""
+    from paper_2608_17641_b200 import workloads
+    ro = workloads.make_rollout(5, N, T, salt=1)
+    q, pi, mu, act = workloads.make_action_tensors(5, N, T, A)
+    up = lambda a: torch.from_numpy(a).cuda()
+    r, d, tr, bv, bt = up(ro.rewards), up(ro.dones), up(ro.truncs), up(ro.trunc_bootstrap), up(ro.bootstrap)
+    qd, pid, mud, actd = up(q), up(pi), up(mu), up(act)
+    out = torch.empty((N, T), dtype=torch.float32, device="cuda")
+    ws = B.Workspace(N, T)
+    call = lambda: B.rlcs_retrace_probs(r, qd, pid, mud, actd, d, tr, bv, bt, gamma=0.99, lam=0.95, c_bar=1.0,
+                                        q_targets=out, workspace=ws)
+    for _ in range(3):
+        call()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(steps):
+        call()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    ab = N * T * (8 * A + min(32, 4 * A) + 14) + 4 * N
+    gbs = ab / (ms * 1e-3) / 1e9
+    return {"ms": round(ms, 5), "N": N, "T": T, "A": A, "env_steps_per_s": N * T / (ms * 1e-3), "algorithmic_bytes": ab,
+            "gbs": round(gbs, 1), "frac_of_peak": round(gbs / peak, 4)}
+
+
 def time_e2e(batch: GpuBatch, steps: int, warmup: int, dist):
     """The same step called with HOST buffers: every step copies that step's inputs from pinned
     host memory to the device, runs the seven C-ABI calls, and reads all outputs back to pinned
@@ -571,6 +601,7 @@ def main():
     if rank == 0 and world == 1 and not args.no_sweep:
         del batch
         torch.cuda.empty_cache()
+        line["extensions"]["retrace_probs"] = time_retrace_probs(torch, binding, max(3, min(args.steps, 30)), peak)
         line["sweeps"] = run_sweeps(torch, peak)
     if rank == 0:
         print(json.dumps(line), flush=True)

@@ -147,6 +147,27 @@ int rlcs_retrace(const float* rewards, const float* q_sa, const float* expected_
                  float lambda, float c_bar, void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * Retrace(lambda) from the tensors a Q-learning agent holds -- Section 3.3.3 with the input form of
+ * Section 7.3 (the paper's fused kernel reads the [N,T,A] action-probability tensor; its exact
+ * signature is not given, this is the reading taken):
+ *   q_values[n,t,a]        = Q(s_t, a)              target_probs[n,t,a]    = pi(a | s_t)
+ *   behaviour_probs[n,t,a] = mu(a | s_t) (> 0 at the action taken)         actions[n,t] in [0, A), int32
+ *   Q(s_t,a_t) = q_values[n,t,actions[n,t]];   E_pi Q(s_t,.) = sum_a target_probs[n,t,a] * q_values[n,t,a];
+ *   c_t = lambda * min(c_bar, target_probs[n,t,a_t] / behaviour_probs[n,t,a_t])
+ * and then exactly rlcs_retrace's recurrence and boundary rules (bootstrap[n] = E_pi Q(s_T,.),
+ * trunc_bootstrap[n,t] = the continuation E_pi Q at a truncation).  [N,T,A] tensors are contiguous
+ * with a innermost.  Only three scalars per step stay on chip, so the kernel's register need does
+ * not depend on T.  Rows are read with 256-bit loads when A is 4, 8 or 16 and the three [N,T,A]
+ * pointers are 32-byte aligned (for A = 4 and 8 the mu rows are read whole as well: a gather would
+ * touch every sector anyway).  Actions outside [0, A) are clamped (for memory safety only).
+ */
+int rlcs_retrace_probs(const float* rewards, const float* q_values, const float* target_probs,
+                       const float* behaviour_probs, const int32_t* actions, const uint8_t* dones, const uint8_t* truncs,
+                       const float* trunc_bootstrap, const float* bootstrap, float* q_targets, int64_t N, int64_t T,
+                       int64_t A, float gamma, float lambda, float c_bar,
+                       void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
  * TD(lambda) returns -- Section 3.3.4, Table 1 row "TD(lambda)".
  *   G_t = rewards_t + gamma*[(1-lambda)*values_next(t) + lambda*G_{t+1}]     where cont_t,
  *   G_t = rewards_t + gamma*values_next(t)                                    elsewhere

@@ -54,6 +54,9 @@ def _load():
             lib.rlcs_oracle_discounted_return.argtypes = [_F, _U, _U, _F, _F, _D, _i64, _i64, _dbl]
             lib.rlcs_oracle_vtrace.argtypes = [_F, _F, _F, _U, _U, _F, _F, _D, _D, _i64, _i64, _dbl, _dbl, _dbl]
             lib.rlcs_oracle_retrace.argtypes = [_F, _F, _F, _F, _U, _U, _F, _F, _D, _i64, _i64, _dbl, _dbl, _dbl]
+            lib.rlcs_oracle_retrace_probs.argtypes = [_F, _F, _F, _F, ctypes.POINTER(ctypes.c_int32), _U, _U, _F, _F, _D,
+                                                      _i64, _i64, _i64, _dbl, _dbl, _dbl]
+            lib.rlcs_oracle_retrace_probs.restype = None
             lib.rlcs_oracle_elig_trace.argtypes = [_F, _U, _D, _i64, _i64, _dbl, _dbl]
             lib.rlcs_oracle_episodic_prefix_sum.argtypes = [_F, _U, _D, _i64, _i64, ctypes.c_int]
             lib.rlcs_oracle_linear_recurrence.argtypes = [_D, _D, _dbl, _D, _i64, ctypes.c_int]
@@ -191,6 +194,26 @@ def retrace(rewards, q_sa, expected_q, log_rhos, dones, truncs=None, trunc_boots
     _load().rlcs_oracle_retrace(_p(r, _F), _p(q, _F), _p(eq, _F), _p(lr, _F), _p(d, _U), _p(tr, _U),
                                 _p(bv, _F), _p(bt, _F), _p(out, _D), N, T, _s(gamma), _s(lam),
                                 _s(c_bar))
+    return out
+
+
+def retrace_probs(rewards, q_values, target_probs, behaviour_probs, actions, dones, truncs=None,
+                  trunc_bootstrap=None, bootstrap=None, *, gamma, lam, c_bar=1.0):
+    """Retrace(lambda) Q targets from [N,T,A] Q-values / policy probabilities and actions [N,T]."""
+    shape = _shape2(rewards)
+    N, T = shape
+    A = np.asarray(q_values).shape[2]
+    r, d = _f32(rewards, shape), _u8(dones, shape)
+    q, pi, mu = _f32(q_values, (N, T, A)), _f32(target_probs, (N, T, A)), _f32(behaviour_probs, (N, T, A))
+    act = np.ascontiguousarray(actions, dtype=np.int32)
+    if act.shape != shape or act.min() < 0 or act.max() >= A:
+        raise ValueError("actions must be [N, T] with values in [0, A)")
+    tr, bv = _trunc_args(truncs, trunc_bootstrap, shape)
+    bt = _f32(bootstrap, (N,))
+    out = np.empty(shape, np.float64)
+    _load().rlcs_oracle_retrace_probs(_p(r, _F), _p(q, _F), _p(pi, _F), _p(mu, _F),
+                                      act.ctypes.data_as(ctypes.POINTER(ctypes.c_int32)), _p(d, _U), _p(tr, _U),
+                                      _p(bv, _F), _p(bt, _F), _p(out, _D), N, T, A, _s(gamma), _s(lam), _s(c_bar))
     return out
 
 

@@ -187,6 +187,38 @@ void rlcs_oracle_retrace(const float* r, const float* q, const float* eq, const 
     }
 }
 
+/* Retrace(lambda) from [N,T,A] tensors (Section 3.3.3 with the input form of Section 7.3): per step
+ * Q(s_t,a_t) = Q[n,t,a_t], E_pi Q(s_t,.) = sum_a pi[n,t,a] Q[n,t,a], and the importance ratio
+ * pi[n,t,a_t] / mu[n,t,a_t]; then the same recurrence as rlcs_oracle_retrace, with the decay built
+ * from the NEXT step's ratio: c_{t+1} = lambda * min(c_bar, ratio_{t+1}). */
+void rlcs_oracle_retrace_probs(const float* r, const float* Q, const float* pi, const float* mu, const int32_t* act,
+                               const uint8_t* term, const uint8_t* trunc, const float* bv, const float* boot,
+                               double* target, int64_t N, int64_t T, int64_t A, double gamma, double lambda,
+                               double c_bar) {
+    for (int64_t n = 0; n < N; ++n) {
+        const int64_t o = n * T;
+        const double b = boot ? (double)boot[n] : 0.0;
+        double D_next = 0.0;
+        for (int64_t t = T - 1; t >= 0; --t) {
+            const int tm = flag(term, o + t), tr = flag(trunc, o + t), last = (t == T - 1);
+            double eq_next = 0.0;                       /* E_pi Q(s_{t+1}, .) */
+            if (!last)
+                for (int64_t a = 0; a < A; ++a) eq_next += (double)pi[(o + t + 1) * A + a] * (double)Q[(o + t + 1) * A + a];
+            const double x = successor(tm, tr, last, (tr && !tm) ? (double)bv[o + t] : 0.0, b, eq_next);
+            const int cont = !tm && !tr && !last;
+            const double q_sa = (double)Q[(o + t) * A + act[o + t]];
+            double D = (double)r[o + t] + gamma * x - q_sa;
+            if (cont) {
+                const int64_t an = act[o + t + 1];
+                const double raw = (double)pi[(o + t + 1) * A + an] / (double)mu[(o + t + 1) * A + an];
+                D += gamma * lambda * (raw < c_bar ? raw : c_bar) * D_next;
+            }
+            target[o + t] = q_sa + D;
+            D_next = D;
+        }
+    }
+}
+
 /* Eligibility trace, scalar form (Section 3.3.5), forward in time:
  * z_t = gamma*lambda*(1 - d_{t-1})*z_{t-1} + x_t, d_{-1} := 0, z_{-1} = 0.
  * `d` is the combined flag (term OR trunc), as the forward scans take it. */

@@ -31,6 +31,7 @@ SIGNATURES = {
     "rlcs_gae_normalized_workspace_bytes": ([_i64, _i64], _sz),
     "rlcs_vtrace": ([_vp] * 9 + [_i64, _i64, _f, _f, _f] + _TAIL, _int),
     "rlcs_retrace": ([_vp] * 9 + [_i64, _i64, _f, _f, _f] + _TAIL, _int),
+    "rlcs_retrace_probs": ([_vp] * 10 + [_i64, _i64, _i64, _f, _f, _f] + _TAIL, _int),
     "rlcs_td_lambda": ([_vp] * 7 + [_i64, _i64, _f, _f] + _TAIL, _int),
     "rlcs_discounted_return": ([_vp] * 6 + [_i64, _i64, _f] + _TAIL, _int),
     "rlcs_elig_trace": ([_vp] * 3 + [_i64, _i64, _f, _f] + _TAIL, _int),
@@ -212,6 +213,25 @@ def rlcs_retrace(rewards, q_sa, expected_q, log_rhos, dones, truncs=None, trunc_
                               _ptr(log_rhos, "f32", (N, T)), _ptr(dones, "u8", (N, T)), _ptr(truncs, "u8", (N, T)),
                               _ptr(trunc_bootstrap, "f32", (N, T)), _ptr(bootstrap, "f32", (N,)),
                               _ptr(out, "f32", (N, T)), N, T, gamma, lam, c_bar, wp, wb, _stream(stream)))
+    return out
+
+
+def rlcs_retrace_probs(rewards, q_values, target_probs, behaviour_probs, actions, dones, truncs=None,
+                       trunc_bootstrap=None, bootstrap=None, *, gamma, lam, c_bar=1.0, q_targets=None, workspace=None,
+                       stream=None):
+    """Retrace(lambda) from [N,T,A] Q-values / target / behaviour probabilities and int32 actions [N,T]."""
+    torch = _torch()
+    N, T = rewards.shape
+    A = q_values.shape[2]
+    if actions.dtype != torch.int32 or not actions.is_cuda or not actions.is_contiguous() or tuple(actions.shape) != (N, T):
+        raise TypeError("actions must be a contiguous CUDA int32 tensor of shape [N, T]")
+    out = _out(rewards, q_targets)
+    wp, wb = _ws(workspace)
+    _check(lib().rlcs_retrace_probs(_ptr(rewards, "f32"), _ptr(q_values, "f32", (N, T, A)),
+                                    _ptr(target_probs, "f32", (N, T, A)), _ptr(behaviour_probs, "f32", (N, T, A)),
+                                    actions.data_ptr(), _ptr(dones, "u8", (N, T)), _ptr(truncs, "u8", (N, T)),
+                                    _ptr(trunc_bootstrap, "f32", (N, T)), _ptr(bootstrap, "f32", (N,)),
+                                    _ptr(out, "f32", (N, T)), N, T, A, gamma, lam, c_bar, wp, wb, _stream(stream)))
     return out
 
 

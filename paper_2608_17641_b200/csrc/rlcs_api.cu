@@ -79,7 +79,8 @@ int choose_variant(int algo, bool trunc, int64_t total, int64_t T) {
 }
 
 // Fill the size / tiling / carry fields and validate the workspace for this call.
-int finish_params(ScanParams& p, int variant, int64_t total, int64_t T, void* workspace, size_t workspace_bytes, bool vec) {
+int finish_params(ScanParams& p, int variant, int64_t total, int64_t T, void* workspace, size_t workspace_bytes, bool vec,
+                  bool allow_cluster = true) {
     const int tile = tile_elems(variant);
     p.total = total;
     p.T = (unsigned)T;
@@ -98,7 +99,7 @@ int finish_params(ScanParams& p, int variant, int64_t total, int64_t T, void* wo
     // Rows of exactly 2..8 tiles: one thread-block cluster per row carries through distributed
     // shared memory instead (needs the vectorised one-tile kernel; g_cluster = 0 turns it off).
     p.cluster = 0;
-    if (g_cluster && vec && rlcs::kVariants[variant].stages == 0 && T % tile == 0 && T / tile >= 2 && T / tile <= 8) {
+    if (allow_cluster && g_cluster && vec && rlcs::kVariants[variant].stages == 0 && T % tile == 0 && T / tile >= 2 && T / tile <= 8) {
         p.cluster = (int)(T / tile);
         p.carry_mode = 0;
     }
@@ -298,6 +299,37 @@ int rlcs_retrace(const float* rewards, const float* q_sa, const float* expected_
     st = finish_params(p, variant, total, T, workspace, workspace_bytes, vec);
     if (st != RLCS_OK) return st;
     return run(rlcs::launch_retrace, p, variant, truncs != nullptr, vec, cuda_stream);
+}
+
+int rlcs_retrace_probs(const float* rewards, const float* q_values, const float* target_probs,
+                       const float* behaviour_probs, const int32_t* actions, const uint8_t* dones, const uint8_t* truncs,
+                       const float* trunc_bootstrap, const float* bootstrap, float* q_targets, int64_t N, int64_t T,
+                       int64_t A, float gamma, float lambda, float c_bar, void* workspace, size_t workspace_bytes,
+                       void* cuda_stream) {
+    ScanParams p = {};
+    Ptrs ps;
+    int64_t total;
+    bool vec;
+    if (!unit_interval(gamma) || !unit_interval(lambda) || !clip_ok(c_bar)) return RLCS_ERR_ARG;
+    if (A < 1 || A > (int64_t(1) << 20)) return RLCS_ERR_SIZE;
+    ps.add_f32(rewards); ps.add_f32(q_targets);
+    int st = backward_common(p, ps, dones, truncs, trunc_bootstrap, bootstrap, N, T, &total, &vec);
+    if (st != RLCS_OK || total == 0) return st;
+    if (total > kMaxTotal / A) return RLCS_ERR_SIZE;
+    if (!rewards || !q_values || !target_probs || !behaviour_probs || !actions || !q_targets) return RLCS_ERR_NULL;
+    if (!aligned(q_values, 4) || !aligned(target_probs, 4) || !aligned(behaviour_probs, 4) || !aligned(actions, 4))
+        return RLCS_ERR_ALIGN;
+    const bool vec_rows = (A % 4 == 0) && aligned(q_values, 32) && aligned(target_probs, 32) && aligned(behaviour_probs, 32);
+    p.f0 = rewards; p.f1 = q_values; p.pi = target_probs; p.mu = behaviour_probs; p.actions = actions; p.A = (int)A;
+    p.out0 = q_targets;
+    p.gamma = gamma; p.aux = gamma * lambda; p.c_bar = c_bar;
+    constexpr int kVariant = 3;      // 256 threads x 4 steps, the tile rlcs_retrace_probs.cu instantiates
+    static_assert(rlcs::kVariants[kVariant].threads == rlcs::kRetraceProbsThreads &&
+                  rlcs::kVariants[kVariant].items == rlcs::kRetraceProbsItems, "tile shape mismatch");
+    st = finish_params(p, kVariant, total, T, workspace, workspace_bytes, vec, false);
+    if (st != RLCS_OK) return st;
+    return rlcs::launch_retrace_probs(p, truncs != nullptr, vec, vec_rows, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess
+               ? RLCS_OK : RLCS_ERR_CUDA;
 }
 
 int rlcs_td_lambda(const float* rewards, const float* values, const uint8_t* dones, const uint8_t* truncs,

@@ -33,6 +33,7 @@ constexpr TileVariant kVariants[kNumVariants] = {
     {128, 16, 5, 0},   // 18: 2048, 16 steps per thread
 };
 constexpr int kMinTileElems = 512;
+constexpr int kRetraceProbsThreads = 256, kRetraceProbsItems = 4;      // tile of rlcs_retrace_probs
 constexpr int kMaxDevices = 64;
 
 template <int ALGO, bool TRUNC, int V>
@@ -134,6 +135,7 @@ cudaError_t launch_elig(const ScanParams&, int variant, bool trunc, bool vec, cu
 cudaError_t launch_prefix(const ScanParams&, int variant, bool trunc, bool vec, cudaStream_t);
 cudaError_t launch_affine_bwd(const ScanParams&, int variant, bool trunc, bool vec, cudaStream_t);
 cudaError_t launch_affine_fwd(const ScanParams&, int variant, bool trunc, bool vec, cudaStream_t);
+cudaError_t launch_retrace_probs(const ScanParams&, bool trunc, bool vec, bool vec_rows, cudaStream_t);
 cudaError_t launch_gae_stats(const ScanParams&, int variant, bool trunc, bool vec, cudaStream_t);
 cudaError_t launch_norm_finalize(const float* partial, long long num_tiles, double count, int ddof, float eps,
                                  float* mean_rstd, cudaStream_t stream);

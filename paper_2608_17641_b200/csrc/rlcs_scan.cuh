@@ -39,16 +39,18 @@ namespace rlcs {
 enum Algo : int {
     kGae = 0, kTdLambda = 1, kDisc = 2, kVtrace = 3, kRetrace = 4, kElig = 5, kPrefix = 6,
     kAffineBwd = 7, kAffineFwd = 8,
-    kGaeStats = 9     // GAE that also leaves per-tile sums of A and A^2 (for advantage normalisation)
+    kGaeStats = 9,    // GAE that also leaves per-tile sums of A and A^2 (for advantage normalisation)
+    kRetraceProbs = 10  // Retrace(lambda) from [N,T,A] Q-values and action probabilities
 };
 
 __host__ __device__ constexpr bool is_forward(int a) { return a == kElig || a == kPrefix || a == kAffineFwd; }
 __host__ __device__ constexpr bool is_gae(int a) { return a == kGae || a == kGaeStats; }
 __host__ __device__ constexpr bool has_values(int a) { return is_gae(a) || a == kTdLambda || a == kVtrace; }
 __host__ __device__ constexpr bool is_affine(int a) { return a == kAffineBwd || a == kAffineFwd; }
-__host__ __device__ constexpr bool const_decay(int a) { return a != kVtrace && a != kRetrace && !is_affine(a); }
+__host__ __device__ constexpr bool is_retrace(int a) { return a == kRetrace || a == kRetraceProbs; }
+__host__ __device__ constexpr bool const_decay(int a) { return a != kVtrace && !is_retrace(a) && !is_affine(a); }
 // a float input is read one step beyond the tile (successor value)
-__host__ __device__ constexpr bool float_halo(int a) { return has_values(a) || a == kRetrace; }
+__host__ __device__ constexpr bool float_halo(int a) { return has_values(a) || is_retrace(a); }
 __host__ __device__ constexpr bool uses_f1(int a) { return a != kDisc && a != kElig && a != kPrefix; }
 __host__ __device__ constexpr bool uses_f2(int a) { return a == kRetrace; }
 __host__ __device__ constexpr bool uses_f3(int a) { return a == kVtrace || a == kRetrace; }
@@ -69,6 +71,10 @@ struct ScanParams {
     const float* f1;          // values | q_sa | beta
     const float* f2;          // expected_q
     const float* f3;          // log_rhos
+    const float* pi;          // kRetraceProbs: target-policy probabilities [N,T,A]  (f1 = Q-values [N,T,A])
+    const float* mu;          // kRetraceProbs: behaviour-policy probabilities [N,T,A]
+    const int* actions;       // kRetraceProbs: actions taken [N,T]
+    int A;                    // kRetraceProbs: number of actions
     const uint8_t* dones;
     const uint8_t* truncs;
     const float* trunc_boot;  // [N,T]
@@ -446,6 +452,98 @@ __device__ __forceinline__ void load_values_global(const Chunk<ALGO, TRUNC, ITEM
     }
 }
 
+// Retrace from the [N,T,A] tensors: per step, Q(s_t,a_t), E_pi Q(s_t,.) = sum_a pi(a|s_t) Q(s_t,a) and the
+// importance ratio pi(a_t|s_t)/mu(a_t|s_t) are formed here from one dense read of the Q and pi rows
+// and three gathers, and only those three scalars per step stay in registers -- the tile never
+// holds whole [T, A] slabs, so the register need does not grow with T.  AV = A when known at
+// compile time (vector loads), 0 = any A.  Actions outside [0, A) are clamped (memory safety only).
+template <int AV>
+__device__ __forceinline__ void probs_step(const ScanParams& p, long long i, bool active, float& q_sa, float& eq, float& ratio) {
+    q_sa = 0.f; eq = 0.f; ratio = 0.f;
+    if (!active) return;
+    const int A = AV > 0 ? AV : p.A;
+    const float* __restrict__ qrow = p.f1 + i * A;
+    const float* __restrict__ prow = p.pi + i * A;
+    int act = __ldg(p.actions + i);
+    act = act < 0 ? 0 : (act >= A ? A - 1 : act);
+    float e = 0.f;
+    if constexpr (AV > 0 && AV % 8 == 0) {
+#pragma unroll
+        for (int k = 0; k < AV / 8; ++k) {
+            float a[8], b[8];
+            ldg_v8(qrow + 8 * k, a);
+            ldg_v8(prow + 8 * k, b);
+#pragma unroll
+            for (int x = 0; x < 8; ++x) e = fmaf(b[x], a[x], e);
+        }
+    } else {
+        for (int a = 0; a < A; ++a) e = fmaf(__ldcs(prow + a), __ldcs(qrow + a), e);
+    }
+    eq = e;
+    q_sa = __ldg(qrow + act);
+    ratio = __ldg(prow + act) / __ldg(p.mu + i * A + act);
+}
+
+// value of row[act] for a row held in registers (A small and known): a select chain, no second trip to memory
+template <int A>
+__device__ __forceinline__ float pick(const float* row, int act) {
+    float v = row[0];
+#pragma unroll
+    for (int a = 1; a < A; ++a) v = (act == a) ? row[a] : v;
+    return v;
+}
+
+template <int ALGO, bool TRUNC, int ITEMS, int AV>
+__device__ __forceinline__ void load_values_probs(const Chunk<ALGO, TRUNC, ITEMS>& c, Vals<ITEMS>& v, const ScanParams& p,
+                                                  long long i0, int lane, int nvalid) {
+    load_f32<ITEMS, false>(p.f0, i0, nvalid, v.a);               // rewards (element-wise: this kernel is bound by the 3-D reads)
+    if constexpr (AV == 4 || AV == 8) {
+        // Rows of 16 or 32 bytes: a gathered mu(a_t|s_t) would touch every 32-byte sector of mu anyway,
+        // so all three rows are read densely with 256-bit loads (no load depends on the action) and
+        // Q(s_t,a_t), pi(a_t|s_t), mu(a_t|s_t) are picked from registers.  Needs full chunks; the ragged
+        // tail falls through to the step-by-step path.
+        if (nvalid == ITEMS) {
+            constexpr int ROWS = 8 / AV;                         // rows per 256-bit load
+            int act[ITEMS];
+#pragma unroll
+            for (int j = 0; j < ITEMS; ++j) {
+                const int a = __ldg(p.actions + i0 + j);
+                act[j] = a < 0 ? 0 : (a >= AV ? AV - 1 : a);
+            }
+#pragma unroll
+            for (int j = 0; j < ITEMS; j += ROWS) {
+                float q[8], pr[8], m[8];
+                ldg_v8(p.f1 + (i0 + j) * AV, q);
+                ldg_v8(p.pi + (i0 + j) * AV, pr);
+                ldg_v8(p.mu + (i0 + j) * AV, m);
+#pragma unroll
+                for (int r = 0; r < ROWS; ++r) {
+                    float e = 0.f;
+#pragma unroll
+                    for (int a = 0; a < AV; ++a) e = fmaf(pr[r * AV + a], q[r * AV + a], e);
+                    v.x2[j + r] = e;
+                    v.x1[j + r] = pick<AV>(q + r * AV, act[j + r]);
+                    v.x3[j + r] = pick<AV>(pr + r * AV, act[j + r]) / pick<AV>(m + r * AV, act[j + r]);
+                }
+            }
+        } else {
+#pragma unroll
+            for (int j = 0; j < ITEMS; ++j) probs_step<0>(p, i0 + j, j < nvalid, v.x1[j], v.x2[j], v.x3[j]);
+        }
+    } else {
+#pragma unroll
+        for (int j = 0; j < ITEMS; ++j) probs_step<AV>(p, i0 + j, j < nvalid, v.x1[j], v.x2[j], v.x3[j]);
+    }
+    // successor-side neighbour: the next thread's first step, or one more step from memory at the warp edge
+    float hq, heq = 0.f, hr = 0.f;
+    const bool edge_lane = (lane == 31) && (p.total - i0 > ITEMS);
+    if (edge_lane) probs_step<0>(p, i0 + ITEMS, true, hq, heq, hr);
+    const float nb = __shfl_down_sync(0xffffffffu, v.x2[0], 1);
+    const float nr = __shfl_down_sync(0xffffffffu, v.x3[0], 1);
+    v.halo = (lane != 31) ? nb : heq;
+    v.halo_lr = (lane != 31) ? nr : hr;
+}
+
 // Shared-memory scratch of the block-level scan; double-buffered by tile parity in the persistent
 // kernel so that one barrier per tile suffices.
 template <int NW>
@@ -589,7 +687,7 @@ __device__ __forceinline__ void tile_compute(Chunk<ALGO, TRUNC, ITEMS>& c, Vals<
             const float r = v.a[j];
             float nextv = 0.f;
             if constexpr (has_values(ALGO)) nextv = (j + 1 < ITEMS) ? v.x1[(j + 1) % ITEMS] : v.halo;
-            if constexpr (ALGO == kRetrace) nextv = (j + 1 < ITEMS) ? v.x2[(j + 1) % ITEMS] : v.halo;
+            if constexpr (is_retrace(ALGO)) nextv = (j + 1 < ITEMS) ? v.x2[(j + 1) % ITEMS] : v.halo;
             const float xn = cut ? c.ov[j] : nextv;      // successor value of Section 3.2 (selected, never multiplied)
             if constexpr (is_gae(ALGO)) {
                 v.a[j] = fmaf(p.gamma, xn, r) - v.x1[j];
@@ -608,10 +706,12 @@ __device__ __forceinline__ void tile_compute(Chunk<ALGO, TRUNC, ITEMS>& c, Vals<
                 v.a[j] = rho * (fmaf(p.gamma, xn, r) - v.x1[j]);
                 beta[j] = cut ? 0.f : p.gamma * cc;
                 grho[j] = cut ? 0.f : p.gamma * rho;
-            } else if constexpr (ALGO == kRetrace) {
+            } else if constexpr (is_retrace(ALGO)) {
                 v.a[j] = fmaf(p.gamma, xn, r) - v.x1[j];
                 const float lr_next = (j + 1 < ITEMS) ? v.x3[(j + 1) % ITEMS] : v.halo_lr;
-                beta[j] = cut ? 0.f : p.aux * fminf(p.c_bar, expf(lr_next));
+                // x3 holds log(pi/mu) for the scalar-input form, the ratio pi/mu itself for the tensor form
+                const float ratio_next = (ALGO == kRetrace) ? expf(lr_next) : lr_next;
+                beta[j] = cut ? 0.f : p.aux * fminf(p.c_bar, ratio_next);
             }
         }
     }
@@ -735,7 +835,7 @@ __device__ __forceinline__ void tile_compute(Chunk<ALGO, TRUNC, ITEMS>& c, Vals<
                 // recurrence continues (v_{t+1} = V_{t+1} + Delta_{t+1}), alpha_t elsewhere.
                 out1v[j] = fmaf(grho[j], prev, v.a[j]);
                 v.a[j] = v.x1[j] + d;
-            } else if constexpr (ALGO == kRetrace) {
+            } else if constexpr (is_retrace(ALGO)) {
                 v.a[j] = v.x1[j] + d;
             } else {
                 v.a[j] = d;
@@ -817,6 +917,38 @@ __global__ void __launch_bounds__(THREADS, MIN_BLOCKS) scan_kernel(const ScanPar
     const bool full = (tile * TILE + TILE <= p.total) && (p.T >= (unsigned)ITEMS);
     if (full) one_tile<ALGO, TRUNC, VEC, THREADS, ITEMS, true>(p, tile, s, epoch, sm);
     else one_tile<ALGO, TRUNC, VEC, THREADS, ITEMS, false>(p, tile, s, epoch, sm);
+}
+
+// ------------------------------------------------------------------------------------------ kernel 1c: Retrace from [N,T,A] tensors
+template <bool TRUNC, bool VEC, int THREADS, int ITEMS, int AV, bool FULL>
+__device__ __forceinline__ void one_tile_probs(const ScanParams& p, long long tile, long long s, unsigned epoch,
+                                               ScanSmem<THREADS / 32>& sm) {
+    constexpr int ALGO = kRetraceProbs;
+    constexpr int TILE = THREADS * ITEMS;
+    const int tid = threadIdx.x;
+    const int lane = tid & 31;
+    Chunk<ALGO, TRUNC, ITEMS> c;
+    const long long i0 = tile * TILE + (long long)tid * ITEMS;
+    const long long n0 = locate(c, p, i0);
+    load_flags_global<ALGO, TRUNC, ITEMS, VEC, FULL>(c, p, i0, lane);
+    Vals<ITEMS> v;
+    load_values_probs<ALGO, TRUNC, ITEMS, AV>(c, v, p, i0, lane, FULL ? ITEMS : c.nvalid);
+    issue_boot(c, p, n0);
+    issue_trunc_values(c, p, i0);
+    tile_compute<ALGO, TRUNC, VEC, THREADS, ITEMS, FULL, true>(c, v, p, i0, s, epoch, sm, 0, NoHook{});
+}
+
+template <bool TRUNC, bool VEC, int THREADS, int ITEMS, int MIN_BLOCKS, int AV>
+__global__ void __launch_bounds__(THREADS, MIN_BLOCKS) scan_kernel_retrace_probs(const ScanParams p) {
+    constexpr int TILE = THREADS * ITEMS;
+    __shared__ ScanSmem<THREADS / 32> sm;
+    const long long s = blockIdx.x;
+    const long long tile = p.num_tiles - 1 - s;
+    unsigned epoch = 0;
+    if (p.carry_mode && threadIdx.x < 32) epoch = ld_volatile_u32(p.header);
+    const bool full = (tile * TILE + TILE <= p.total) && (p.T >= (unsigned)ITEMS);      // block-uniform
+    if (full) one_tile_probs<TRUNC, VEC, THREADS, ITEMS, AV, true>(p, tile, s, epoch, sm);
+    else one_tile_probs<TRUNC, VEC, THREADS, ITEMS, AV, false>(p, tile, s, epoch, sm);
 }
 
 // ------------------------------------------------------------------------------------------ kernel 1b: one tile per block, one cluster per row

@@ -119,3 +119,23 @@ def config4(N: int = 64, T: int = 16384, salt=0) -> Rollout:
 def config5(N: int = 16384, T: int = 2048, salt=0) -> Rollout:
     """Bandwidth-saturating batch: all seven algorithms, truncation handling on."""
     return make_rollout(5, N, T, salt=salt)
+
+
+def make_action_tensors(config: int, N: int, T: int, A: int, salt=0):
+    """[N,T,A] Q-values ~ N(0,1), target / behaviour action probabilities (softmax of N(0,1) logits; the
+    behaviour logits are the target logits plus N(0, 0.5^2) noise, so log pi - log mu has the spread
+    of the scalar-input configurations) and int32 actions [N,T] drawn from the behaviour policy."""
+    rng = np.random.default_rng(17641 * 1000 + 100 * config + 50 + 100000 * salt + 7 * A)
+    q = rng.standard_normal((N, T, A), dtype=np.float32)
+    logits = rng.standard_normal((N, T, A), dtype=np.float32)
+    blogits = logits + np.float32(0.5) * rng.standard_normal((N, T, A), dtype=np.float32)
+
+    def softmax(z):
+        z = z - z.max(axis=2, keepdims=True)
+        e = np.exp(z, dtype=np.float32)
+        return (e / e.sum(axis=2, keepdims=True)).astype(np.float32)
+
+    pi, mu = softmax(logits), softmax(blogits)
+    u = rng.random((N, T, 1), dtype=np.float32)
+    actions = np.minimum((np.cumsum(mu, axis=2) < u).sum(axis=2), A - 1).astype(np.int32)
+    return q, pi, mu, actions

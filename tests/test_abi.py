@@ -96,6 +96,17 @@ def test_null_pointer_errors(L):
     assert L.rlcs_affine_scan(P, None, P, 4, 8, 0, None, 0, None) == E_NULL
 
 
+def test_retrace_probs_argument_checks(L):
+    f = lambda **k: L.rlcs_retrace_probs(k.get("r", P), k.get("q", P), k.get("pi", P), k.get("mu", P), k.get("act", P), P,
+                                         None, None, None, P, k.get("N", 4), k.get("T", 8), k.get("A", 4), k.get("g", 0.9),
+                                         0.9, k.get("c", 1.0), None, 0, None)
+    assert f(A=0) == E_SIZE and f(A=2 ** 21) == E_SIZE and f(N=2 ** 30, T=2 ** 9, A=2 ** 10) == E_SIZE
+    assert f(g=1.5) == E_ARG and f(c=-1.0) == E_ARG
+    assert f(q=None) == E_NULL and f(pi=None) == E_NULL and f(mu=None) == E_NULL and f(act=None) == E_NULL
+    assert f(q=ODD) == E_ALIGN and f(act=ODD) == E_ALIGN
+    assert f(N=0) == OK
+
+
 def test_alignment_errors(L):
     assert _gae(L, r=ODD) == E_ALIGN
     assert _gae(L, adv=ODD) == E_ALIGN

@@ -384,6 +384,72 @@ def test_gae_normalized_argument_checks(oracle, W, B):
     assert e.value.status == B.RLCS_ERR_WORKSPACE
 
 
+# ------------------------------------------------------------------ Retrace from [N,T,A] tensors
+def _probs_gpu(B, ro, q, pi, mu, act, use_truncs=True, use_bootstrap=True, offset=0):
+    import torch
+    dev = Dev(ro, offset=offset)
+
+    def up3(a):
+        t = torch.from_numpy(a)
+        if offset == 0:
+            return t.cuda()
+        flat = torch.empty(t.numel() + offset, dtype=t.dtype, device="cuda")
+        view = flat[offset:].view(t.shape)
+        view.copy_(t)
+        return view
+
+    ws = B.Workspace(ro.N, ro.T)
+    p = ro.params
+    out = B.rlcs_retrace_probs(dev.rewards, up3(q), up3(pi), up3(mu), torch.from_numpy(act).cuda(), dev.dones,
+                               dev.truncs if use_truncs else None, dev.trunc_bootstrap if use_truncs else None,
+                               dev.bootstrap if use_bootstrap else None, gamma=p["gamma"], lam=p["lam"], c_bar=p["c_bar"],
+                               q_targets=dev.empty_out(), workspace=ws)
+    torch.cuda.synchronize()
+    assert ws.device_status() == 0
+    return out.cpu().numpy()
+
+
+@pytest.mark.parametrize("A", [1, 2, 3, 4, 5, 8, 16, 18])
+@pytest.mark.parametrize("N,T", [(1, 1), (3, 7), (8, 128), (5, 1000), (2, 4096), (300, 257)])
+def test_retrace_probs_matches_oracle(oracle, W, B, A, N, T):
+    ro = W.make_rollout(112, N, T, p_done=0.02, p_trunc=0.01, salt=A)
+    q, pi, mu, act = W.make_action_tensors(112, N, T, A, salt=T)
+    for use_tr, use_bt in ((True, True), (False, True), (True, False)):
+        got = _probs_gpu(B, ro, q, pi, mu, act, use_tr, use_bt)
+        ref = oracle.retrace_probs(ro.rewards, q, pi, mu, act, ro.dones, ro.truncs if use_tr else None,
+                                   ro.trunc_bootstrap if use_tr else None, ro.bootstrap if use_bt else None,
+                                   gamma=ro.params["gamma"], lam=ro.params["lam"], c_bar=ro.params["c_bar"])
+        assert_close(f"retrace_probs A={A}", got, ref)
+
+
+def test_retrace_probs_unaligned_and_long_rows(oracle, W, B):
+    """Pointers off 16-byte alignment (element-wise row reads), and T = 16384: the register need of the
+    tile does not depend on T (the paper's kernel spilled from T = 4096 on)."""
+    for (N, T, A, off) in [(4, 600, 4, 1), (3, 600, 8, 2), (2, 16384, 4, 0), (64, 16384, 4, 0)]:
+        ro = W.make_rollout(113, N, T, p_done=0.001, p_trunc=0.001, salt=A)
+        q, pi, mu, act = W.make_action_tensors(113, N, T, A, salt=off)
+        got = _probs_gpu(B, ro, q, pi, mu, act, offset=off)
+        ref = oracle.retrace_probs(ro.rewards, q, pi, mu, act, ro.dones, ro.truncs, ro.trunc_bootstrap, ro.bootstrap,
+                                   gamma=ro.params["gamma"], lam=ro.params["lam"], c_bar=ro.params["c_bar"])
+        assert_close(f"retrace_probs {N}x{T}x{A} offset {off}", got, ref)
+
+
+def test_retrace_probs_agrees_with_scalar_entry_point(oracle, W, B):
+    """The tensor form and rlcs_retrace on inputs derived from the tensors (gather, dot, log) agree."""
+    import torch
+    N, T, A = 16, 3000, 4
+    ro = W.make_rollout(114, N, T)
+    q, pi, mu, act = W.make_action_tensors(114, N, T, A)
+    got = _probs_gpu(B, ro, q, pi, mu, act)
+    idx = act[..., None].astype(np.int64)
+    ro.q_sa = np.take_along_axis(q, idx, axis=2)[..., 0].copy()
+    ro.expected_q = np.einsum("nta,nta->nt", pi.astype(np.float64), q.astype(np.float64)).astype(np.float32)
+    ro.log_rhos = np.log(np.take_along_axis(pi, idx, axis=2)[..., 0].astype(np.float64)
+                         / np.take_along_axis(mu, idx, axis=2)[..., 0].astype(np.float64)).astype(np.float32)
+    scalar = run_gpu(Dev(ro), ("retrace",))["retrace"]
+    np.testing.assert_allclose(got, scalar, rtol=3e-5, atol=3e-5)
+
+
 # ------------------------------------------------------------------ test hooks
 def test_affine_scan_matches_generic_recurrence(oracle, W, B):
     import torch

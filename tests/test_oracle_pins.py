@@ -589,3 +589,70 @@ def test_normalised_advantages_scale_invariance_and_degenerate_cases(oracle):
     single, _ = oracle.gae_normalized(ones[:1, :1], ones[:1, :1] * 0, np.zeros((1, 1), np.uint8), gamma=0.9, lam=0.9,
                                       eps=1e-8, ddof=1)
     assert single[0, 0] == 0.0
+
+
+# ----------------------------------------------------------------------------- Retrace from [N,T,A] tensors
+def _probs_case(seed, N=3, T=30, A=4, p=0.08):
+    from paper_2608_17641_b200 import workloads
+    b = _batch(seed, N=N, T=T, p=p)
+    q, pi, mu, act = workloads.make_action_tensors(70, N, T, A, salt=seed)
+    return b, q, pi, mu, act
+
+
+def test_retrace_probs_against_table1_explicit_sum(oracle):
+    """alpha_t = r_t + gamma (1 - term_t) E_pi Q(s_{t+1},.) - Q(s_t,a_t), beta_t = gamma c_{t+1} (1 - d_t) with
+    c_t = lambda min(c_bar, pi(a_t|s_t)/mu(a_t|s_t)), c_T = 0, carry 0 -- built literally from the tensors."""
+    for A in (2, 4, 5):
+        b, q, pi, mu, act = _probs_case(40 + A, N=2, T=25, A=A, p=0.1)
+        out = oracle.retrace_probs(b["r"], q, pi, mu, act, **_bk(b), gamma=0.99, lam=0.9, c_bar=1.0)
+        for n in range(2):
+            T = 25
+            q64, pi64, mu64 = q[n].astype(float), pi[n].astype(float), mu[n].astype(float)
+            eq = (pi64 * q64).sum(axis=1)
+            qsa = q64[np.arange(T), act[n]]
+            ratio = pi64[np.arange(T), act[n]] / mu64[np.arange(T), act[n]]
+            c = float(np.float32(0.9)) * np.minimum(1.0, ratio)
+            i = dict(r=b["r"][n], eq=eq, term=b["term"][n], trunc=b["trunc"][n], bv=b["bv"][n], boot=b["boot"][n])
+            d = np.maximum(i["term"], i["trunc"]).astype(float)
+            alpha = np.array([float(i["r"][t]) + G32 * _table1_successor(eq, i, t, T) - qsa[t] for t in range(T)])
+            beta = G32 * np.append(c[1:], 0.0) * (1.0 - d)
+            np.testing.assert_allclose(out[n], explicit_sum_backward(alpha, beta, 0.0) + qsa, rtol=1e-12, atol=1e-12)
+
+
+def test_retrace_probs_reduces_to_scalar_form(oracle):
+    """Feeding the scalar-input Retrace with Q(s,a), E_pi Q and log(pi/mu) derived with library routines
+    (gather, einsum, log) gives the same targets up to the fp32 rounding of those derived inputs."""
+    b, q, pi, mu, act = _probs_case(50, N=4, T=60, A=8)
+    out = oracle.retrace_probs(b["r"], q, pi, mu, act, **_bk(b), gamma=0.99, lam=0.95, c_bar=1.5)
+    idx = act[..., None].astype(np.int64)
+    q_sa = np.take_along_axis(q, idx, axis=2)[..., 0]
+    eq = np.einsum("nta,nta->nt", pi.astype(np.float64), q.astype(np.float64)).astype(np.float32)
+    lr = np.log(np.take_along_axis(pi, idx, axis=2)[..., 0].astype(np.float64)
+                / np.take_along_axis(mu, idx, axis=2)[..., 0].astype(np.float64)).astype(np.float32)
+    want = oracle.retrace(b["r"], q_sa, eq, lr, **_bk(b), gamma=0.99, lam=0.95, c_bar=1.5)
+    np.testing.assert_allclose(out, want, rtol=2e-5, atol=2e-5)
+
+
+def test_retrace_probs_structure(oracle):
+    b, q, pi, mu, act = _probs_case(51, N=3, T=40, A=4, p=0.0)
+    kw = dict(gamma=0.99, lam=0.9, c_bar=1.0)
+    base = oracle.retrace_probs(b["r"], q, pi, mu, act, **_bk(b), **kw)
+    # relabelling the actions consistently changes nothing
+    perm = np.array([2, 0, 3, 1])
+    inv = np.argsort(perm)
+    out = oracle.retrace_probs(b["r"], q[..., perm], pi[..., perm], mu[..., perm], inv[act].astype(np.int32), **_bk(b), **kw)
+    np.testing.assert_allclose(out, base, rtol=1e-13)
+    # index shift: the behaviour probabilities of the first step never matter, those of step 5 reach step 4
+    mu2 = mu.copy()
+    mu2[:, 0, :] = 0.25
+    assert np.array_equal(oracle.retrace_probs(b["r"], q, pi, mu2, act, **_bk(b), **kw), base)
+    mu3 = mu.copy()
+    mu3[:, 5, :] *= 3.0
+    out3 = oracle.retrace_probs(b["r"], q, pi, mu3, act, **_bk(b), **kw)
+    assert not np.array_equal(out3[:, 4], base[:, 4]) and np.array_equal(out3[:, 5:], base[:, 5:])
+    # action-independent Q = V, on-policy, c_bar = 1: target - V = GAE(lambda)
+    V = b["V"]
+    qv = np.repeat(V[..., None], 4, axis=2)
+    on = oracle.retrace_probs(b["r"], qv, pi, pi, act, **_bk(b), gamma=0.99, lam=0.95, c_bar=1.0)
+    adv, _ = oracle.gae(b["r"], V, **_bk(b), gamma=0.99, lam=0.95)
+    np.testing.assert_allclose(on - V, adv, rtol=1e-6, atol=1e-6)        # sum_a pi = 1 only to fp32 rounding
