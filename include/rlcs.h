@@ -197,6 +197,22 @@ int rlcs_elig_trace(const float* x, const uint8_t* dones, float* traces, int64_t
                     void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * Vector-valued eligibility trace -- Table 1, row "Elig. Traces" in its vector form (Section 3.3.5):
+ * x, traces: [N, T, D] contiguous with d innermost; one scalar decay per step, shared by all D
+ * components;  dones: [N, T], the combined flag as for rlcs_elig_trace.
+ *   z_t = x_t + ((t > 0 and not dones_{t-1}) ? gamma*lambda * z_{t-1} : 0)        (z_t, x_t in R^D)
+ * One pass over x when N*D is large enough to fill the GPU; otherwise the time axis is cut into
+ * chunks and x is read twice (chunk ends, ordered carry chain, rescan), which needs `workspace` of
+ * rlcs_elig_trace_vec_workspace_bytes(N, T, D) bytes (0 when no cut is needed; no initialisation
+ * required).  128-bit accesses when D is a multiple of 4 and x, traces are 16-byte aligned.
+ * Limits: T < 2^31, D <= 2^24, N*T*D < 2^40.
+ */
+int rlcs_elig_trace_vec(const float* x, const uint8_t* dones, float* traces, int64_t N, int64_t T, int64_t D,
+                        float gamma, float lambda, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+size_t rlcs_elig_trace_vec_workspace_bytes(int64_t N, int64_t T, int64_t D);
+
+/*
  * Episodic prefix sum, forward in time -- Section 3.3.6.
  *   starts_at == 0 ("ends_at", the flag closes a segment):  C_t = x_t + ((t>0 and not dones_{t-1}) ? C_{t-1} : 0)
  *   starts_at != 0 (the flag opens a segment):              C_t = x_t + ((t>0 and not dones_t)     ? C_{t-1} : 0)

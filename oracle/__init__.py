@@ -58,6 +58,8 @@ def _load():
                                                       _i64, _i64, _i64, _dbl, _dbl, _dbl]
             lib.rlcs_oracle_retrace_probs.restype = None
             lib.rlcs_oracle_elig_trace.argtypes = [_F, _U, _D, _i64, _i64, _dbl, _dbl]
+            lib.rlcs_oracle_elig_trace_vec.argtypes = [_F, _U, _D, _i64, _i64, _i64, _dbl, _dbl]
+            lib.rlcs_oracle_elig_trace_vec.restype = None
             lib.rlcs_oracle_episodic_prefix_sum.argtypes = [_F, _U, _D, _i64, _i64, ctypes.c_int]
             lib.rlcs_oracle_linear_recurrence.argtypes = [_D, _D, _dbl, _D, _i64, ctypes.c_int]
             lib.rlcs_oracle_combine.argtypes = [_dbl, _dbl, _dbl, _dbl, _D, _D]
@@ -224,6 +226,18 @@ def elig_trace(x, dones, *, gamma, lam):
     xx, d = _f32(x, shape), _u8(dones, shape)
     out = np.empty(shape, np.float64)
     _load().rlcs_oracle_elig_trace(_p(xx, _F), _p(d, _U), _p(out, _D), N, T, _s(gamma), _s(lam))
+    return out
+
+
+def elig_trace_vec(x, dones, *, gamma, lam):
+    """Vector-valued eligibility trace: x [N,T,D], dones [N,T] -- Table 1 (vector form), Section 3.3.5."""
+    xx = np.ascontiguousarray(x, dtype=np.float32)
+    if xx.ndim != 3:
+        raise ValueError("expected an [N, T, D] array")
+    N, T, D = xx.shape
+    d = _u8(dones, (N, T))
+    out = np.empty(xx.shape, np.float64)
+    _load().rlcs_oracle_elig_trace_vec(_p(xx, _F), _p(d, _U), _p(out, _D), N, T, D, _s(gamma), _s(lam))
     return out
 
 

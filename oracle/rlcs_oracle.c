@@ -236,6 +236,19 @@ void rlcs_oracle_elig_trace(const float* x, const uint8_t* d, double* z, int64_t
     }
 }
 
+/* Vector-valued eligibility trace (Table 1, vector form): x, z are [N,T,D]; one scalar decay per step. */
+void rlcs_oracle_elig_trace_vec(const float* x, const uint8_t* d, double* z, int64_t N, int64_t T, int64_t D,
+                                double gamma, double lambda) {
+    for (int64_t n = 0; n < N; ++n)
+        for (int64_t t = 0; t < T; ++t) {
+            const int carry = (t > 0) && !flag(d, n * T + t - 1);
+            for (int64_t c = 0; c < D; ++c) {
+                const int64_t i = (n * T + t) * D + c;
+                z[i] = carry ? (double)x[i] + gamma * lambda * z[i - D] : (double)x[i];
+            }
+        }
+}
+
 /* Episodic prefix sum (Section 3.3.6), forward in time.  ends_at (default):
  * C_t = x_t + (1 - d_{t-1})*C_{t-1}; starts_at: C_t = x_t + (1 - d_t)*C_{t-1}.
  * C_{-1} = 0 in both, so C_0 = x_0 whatever d_0 is. */

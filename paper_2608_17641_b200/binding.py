@@ -35,6 +35,8 @@ SIGNATURES = {
     "rlcs_td_lambda": ([_vp] * 7 + [_i64, _i64, _f, _f] + _TAIL, _int),
     "rlcs_discounted_return": ([_vp] * 6 + [_i64, _i64, _f] + _TAIL, _int),
     "rlcs_elig_trace": ([_vp] * 3 + [_i64, _i64, _f, _f] + _TAIL, _int),
+    "rlcs_elig_trace_vec": ([_vp] * 3 + [_i64, _i64, _i64, _f, _f] + _TAIL, _int),
+    "rlcs_elig_trace_vec_workspace_bytes": ([_i64, _i64, _i64], _sz),
     "rlcs_episodic_prefix_sum": ([_vp] * 3 + [_i64, _i64, _int] + _TAIL, _int),
     "rlcs_gae_no_alloc": ([_vp] * 8 + [_i64, _i64, _f, _f, _vp], _int),
     "rlcs_no_alloc_scratch_bytes": ([], _sz),
@@ -264,6 +266,20 @@ def rlcs_elig_trace(x, dones, *, gamma, lam, traces=None, workspace=None, stream
     wp, wb = _ws(workspace)
     _check(lib().rlcs_elig_trace(_ptr(x, "f32"), _ptr(dones, "u8", (N, T)), _ptr(out, "f32", (N, T)), N, T,
                                  gamma, lam, wp, wb, _stream(stream)))
+    return out
+
+
+def rlcs_elig_trace_vec(x, dones, *, gamma, lam, traces=None, workspace=None, stream=None):
+    """Vector-valued eligibility trace: x [N,T,D], dones [N,T].  A workspace is made on the fly when the
+    time axis has to be cut and none is given."""
+    N, T, D = x.shape
+    out = _out(x, traces)
+    if workspace is None:
+        nbytes = int(lib().rlcs_elig_trace_vec_workspace_bytes(N, T, D))
+        workspace = Workspace(N, T, device=x.device, stream=stream, nbytes=nbytes) if nbytes else None
+    wp, wb = _ws(workspace)
+    _check(lib().rlcs_elig_trace_vec(_ptr(x, "f32"), _ptr(dones, "u8", (N, T)), _ptr(out, "f32", (N, T, D)), N, T, D,
+                                     gamma, lam, wp, wb, _stream(stream)))
     return out
 
 

@@ -1,0 +1,202 @@
+// Vector-valued eligibility traces: x, z of shape [N, T, D] (d innermost), one scalar decay per
+// step shared by all D components (Table 1, row "Elig. Traces", in its vector form).
+//
+// The scan runs along T, which is the strided axis of this layout, so the mapping is the transpose of
+// the flat-tile kernels: a thread owns 4 (or 1) adjacent components d of one row n and walks the
+// timesteps in order -- z <- beta_t * z + x_t is one FMA per component -- while the 32 lanes of a
+// warp cover adjacent components, so every load and store is a fully used 512-byte (or 128-byte)
+// segment.  Addresses do not depend on the recurrence: UNROLL steps are loaded before the first
+// FMA, which keeps UNROLL x 16 bytes per thread in flight.
+//
+// Parallelism is N * D/4 threads.  When that cannot fill the GPU (few long rows) the time axis is cut
+// into chunks: pass 1 computes each chunk's end vector with carry 0 and its decay product, a small
+// pass chains the carries of a row's chunks in order, and pass 3 rescans every chunk from its carry
+// and writes the traces (x is then read twice).  Deterministic either way.
+#include <cstdint>
+
+#include "../../include/rlcs.h"
+#include "rlcs_scan.cuh"
+
+namespace {
+
+constexpr int kUnroll = 8;
+constexpr int kThreads = 256;
+
+struct VecParams {
+    const float* x;
+    const uint8_t* dones;
+    float* z;
+    long long N;
+    unsigned T, D;
+    unsigned groups;          // threads per row: ceil(D / V)
+    unsigned chunk;           // timesteps per chunk (== T when the time axis is not cut)
+    unsigned chunks;          // chunks per row
+    float decay;
+    float* ends;              // [N, chunks, D]: pass 1 chunk-end vectors, then (in place) the carries into each chunk
+    float* prods;             // [N, chunks]: decay product of each chunk
+};
+
+template <int V> struct Vec;
+template <> struct Vec<4> {
+    float4 v;
+    __device__ static Vec load(const float* p) { Vec r; r.v = __ldcs(reinterpret_cast<const float4*>(p)); return r; }
+    __device__ static Vec plain(const float* p) { Vec r; r.v = *reinterpret_cast<const float4*>(p); return r; }
+    __device__ void store(float* p) const { __stcs(reinterpret_cast<float4*>(p), v); }
+    __device__ void plain_store(float* p) const { *reinterpret_cast<float4*>(p) = v; }
+    __device__ static Vec zero() { Vec r; r.v = make_float4(0.f, 0.f, 0.f, 0.f); return r; }
+    __device__ void fma(float b, const Vec& x) {     // this <- b * this + x
+        v.x = fmaf(b, v.x, x.v.x); v.y = fmaf(b, v.y, x.v.y); v.z = fmaf(b, v.z, x.v.z); v.w = fmaf(b, v.w, x.v.w);
+    }
+};
+template <> struct Vec<1> {
+    float v;
+    __device__ static Vec load(const float* p) { Vec r; r.v = __ldcs(p); return r; }
+    __device__ static Vec plain(const float* p) { Vec r; r.v = *p; return r; }
+    __device__ void store(float* p) const { __stcs(p, v); }
+    __device__ void plain_store(float* p) const { *p = v; }
+    __device__ static Vec zero() { Vec r; r.v = 0.f; return r; }
+    __device__ void fma(float b, const Vec& x) { v = fmaf(b, v, x.v); }
+};
+
+// MODE 0: whole rows, write traces.  MODE 1: chunk ends and decay products only.  MODE 2: rescan
+// from the carry and write traces.
+template <int V, int MODE>
+__global__ void __launch_bounds__(kThreads) elig_vec_kernel(const VecParams p) {
+    const long long tid = (long long)blockIdx.x * kThreads + threadIdx.x;
+    const long long per_row = (long long)p.groups * p.chunks;
+    const long long n = tid / per_row;
+    if (n >= p.N) return;
+    const unsigned rest = (unsigned)(tid - n * per_row);
+    const unsigned k = rest / p.groups;                       // chunk of the row
+    const unsigned c = (rest - k * p.groups) * V;             // first component of this thread
+    const unsigned t_begin = k * p.chunk;
+    const unsigned t_end = min(p.T, t_begin + p.chunk);
+    const long long row = n * (long long)p.T;
+    const float* __restrict__ x = p.x + (row * p.D + c);
+    float* __restrict__ z = p.z + (row * p.D + c);
+    const uint8_t* __restrict__ d = p.dones + row;
+
+    Vec<V> acc = Vec<V>::zero();
+    if (MODE == 2 && k > 0) acc = Vec<V>::plain(p.ends + ((n * p.chunks + k) * (long long)p.D + c));
+    float prod = 1.f;
+    for (unsigned t0 = t_begin; t0 < t_end; t0 += kUnroll) {
+        Vec<V> xs[kUnroll];
+        float beta[kUnroll];
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+            const unsigned t = t0 + u;
+            if (t < t_end) {
+                xs[u] = Vec<V>::load(x + (long long)t * p.D);
+                // the carry into step t is severed by the flag of step t-1 (and at the row's first step)
+                beta[u] = (t == 0 || __ldg(d + t - 1) != 0) ? 0.f : p.decay;
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+            const unsigned t = t0 + u;
+            if (t < t_end) {
+                acc.fma(beta[u], xs[u]);
+                if (MODE == 1) prod *= beta[u];
+                else acc.store(z + (long long)t * p.D);
+            }
+        }
+    }
+    if (MODE == 1) {
+        acc.plain_store(p.ends + ((n * p.chunks + k) * (long long)p.D + c));
+        if (c == 0) p.prods[n * p.chunks + k] = prod;
+    }
+}
+
+// Chain the chunks of each row: carry into chunk k = end_{k-1} + prod_{k-1} * carry into chunk k-1,
+// in order, one thread per (row, component group).  Overwrites ends[n][k] with the carry into chunk k.
+template <int V>
+__global__ void __launch_bounds__(kThreads) elig_vec_chain_kernel(const VecParams p) {
+    const long long tid = (long long)blockIdx.x * kThreads + threadIdx.x;
+    const long long n = tid / p.groups;
+    if (n >= p.N) return;
+    const unsigned c = (unsigned)(tid - n * p.groups) * V;
+    float* e = p.ends + (n * p.chunks * (long long)p.D + c);
+    const float* pr = p.prods + n * p.chunks;
+    Vec<V> carry = Vec<V>::zero();
+    for (unsigned k = 0; k < p.chunks; ++k) {
+        const Vec<V> end_k = Vec<V>::plain(e + (long long)k * p.D);     // computed with carry 0
+        carry.plain_store(e + (long long)k * p.D);                      // carry into chunk k
+        carry.fma(pr[k], end_k);                                        // carry into chunk k+1
+    }
+}
+
+inline bool aligned(const void* p, uintptr_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+
+// chunking: cut the time axis only when N * groups threads cannot fill the GPU
+void plan(long long N, long long T, long long groups, unsigned* chunk, unsigned* chunks) {
+    // One pass needs enough threads to keep the memory system busy: each holds kUnroll x 16 bytes in
+    // flight, and ~40 K threads (5 MB) already saturate HBM; below that, cut -- but into chunks of
+    // at least 128 steps and at most 256 per row, so that the ordered carry chain stays short.
+    const long long want_threads = 148ll * 256;
+    long long k = 1;
+    if (N * groups < want_threads) k = (want_threads + N * groups - 1) / (N * groups);
+    if (k > 256) k = 256;
+    long long len = (T + k - 1) / k;
+    if (len < 128) len = 128;
+    len = (len + kUnroll - 1) / kUnroll * kUnroll;
+    if (len >= T) { *chunk = (unsigned)T; *chunks = 1; return; }
+    *chunk = (unsigned)len;
+    *chunks = (unsigned)((T + len - 1) / len);
+}
+
+template <int V>
+int run(VecParams p, cudaStream_t s) {
+    const long long threads = p.N * (long long)p.groups * p.chunks;
+    const unsigned blocks = (unsigned)((threads + kThreads - 1) / kThreads);
+    if (p.chunks == 1) {
+        elig_vec_kernel<V, 0><<<blocks, kThreads, 0, s>>>(p);
+    } else {
+        elig_vec_kernel<V, 1><<<blocks, kThreads, 0, s>>>(p);
+        const long long chain_threads = p.N * (long long)p.groups;
+        elig_vec_chain_kernel<V><<<(unsigned)((chain_threads + kThreads - 1) / kThreads), kThreads, 0, s>>>(p);
+        elig_vec_kernel<V, 2><<<blocks, kThreads, 0, s>>>(p);
+    }
+    return cudaGetLastError() == cudaSuccess ? RLCS_OK : RLCS_ERR_CUDA;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t rlcs_elig_trace_vec_workspace_bytes(int64_t N, int64_t T, int64_t D) {
+    if (N <= 0 || T <= 0 || D <= 0 || T > (int64_t(1) << 31) - 1 || D > (int64_t(1) << 24)) return 0;
+    unsigned chunk, chunks;
+    plan(N, T, (D + 3) / 4, &chunk, &chunks);
+    unsigned chunk1, chunks1;
+    plan(N, T, D, &chunk1, &chunks1);                         // the element-wise variant cuts differently
+    const size_t k = chunks > chunks1 ? chunks : chunks1;
+    if (k <= 1) return 0;
+    return sizeof(float) * (size_t)N * k * ((size_t)D + 1) + 256;
+}
+
+int rlcs_elig_trace_vec(const float* x, const uint8_t* dones, float* traces, int64_t N, int64_t T, int64_t D,
+                        float gamma, float lambda, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    if (!(gamma >= 0.f && gamma <= 1.f) || !(lambda >= 0.f && lambda <= 1.f)) return RLCS_ERR_ARG;
+    if (N < 0 || T < 0 || D < 0 || T > (int64_t(1) << 31) - 1 || D > (int64_t(1) << 24)) return RLCS_ERR_SIZE;
+    if (N == 0 || T == 0 || D == 0) return RLCS_OK;
+    if (N > (int64_t(1) << 40) / T || N * T > (int64_t(1) << 40) / D) return RLCS_ERR_SIZE;
+    if (!x || !dones || !traces) return RLCS_ERR_NULL;
+    if (!aligned(x, 4) || !aligned(traces, 4)) return RLCS_ERR_ALIGN;
+    const bool v4 = (D % 4 == 0) && aligned(x, 16) && aligned(traces, 16);
+    VecParams p = {};
+    p.x = x; p.dones = dones; p.z = traces; p.N = N; p.T = (unsigned)T; p.D = (unsigned)D;
+    p.groups = (unsigned)(v4 ? D / 4 : D);
+    p.decay = gamma * lambda;
+    plan(N, T, p.groups, &p.chunk, &p.chunks);
+    if (p.chunks > 1) {
+        const size_t need = sizeof(float) * (size_t)N * p.chunks * ((size_t)D + 1);
+        if (workspace == nullptr || workspace_bytes < need) return RLCS_ERR_WORKSPACE;
+        if (!aligned(workspace, 16)) return RLCS_ERR_ALIGN;
+        p.ends = static_cast<float*>(workspace);
+        p.prods = p.ends + (size_t)N * p.chunks * (size_t)D;
+    }
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    return v4 ? run<4>(p, s) : run<1>(p, s);
+}
+
+}  // extern "C"

@@ -450,6 +450,47 @@ def test_retrace_probs_agrees_with_scalar_entry_point(oracle, W, B):
     np.testing.assert_allclose(got, scalar, rtol=3e-5, atol=3e-5)
 
 
+# ------------------------------------------------------------------ vector-valued eligibility traces
+@pytest.mark.parametrize("N,T,D", [(1, 1, 1), (3, 7, 5), (8, 128, 64), (64, 257, 16), (4096, 40, 8), (2, 5000, 128),
+                                    (3, 16384, 32), (1, 70000, 4), (5, 999, 3), (7, 300, 130)])
+def test_vector_eligibility_trace(oracle, W, B, N, T, D):
+    import torch
+    rng = np.random.default_rng(N * 7919 + T * 31 + D)
+    x = rng.standard_normal((N, T, D)).astype(np.float32)
+    d = (rng.random((N, T)) < 0.02).astype(np.uint8)
+    d[:, 0] = rng.integers(0, 2, N)                      # a flag on the very first step
+    xd, dd = torch.from_numpy(x).cuda(), torch.from_numpy(d).cuda()
+    ref = oracle.elig_trace_vec(x, d, gamma=0.99, lam=0.95)
+    got = B.rlcs_elig_trace_vec(xd, dd, gamma=0.99, lam=0.95).cpu().numpy()
+    assert_close(f"vector trace {N}x{T}x{D}", got, ref)
+    again = B.rlcs_elig_trace_vec(xd, dd, gamma=0.99, lam=0.95).cpu().numpy()
+    assert np.array_equal(got, again)
+    # pointer off 16-byte alignment: element-wise variant
+    flat = torch.empty(x.size + 1, dtype=torch.float32, device="cuda")
+    xo = flat[1:].view(N, T, D)
+    xo.copy_(xd)
+    got1 = B.rlcs_elig_trace_vec(xo, dd, gamma=0.99, lam=0.95).cpu().numpy()
+    assert_close("vector trace, unaligned", got1, ref)
+    # against the scalar entry point, component by component
+    if N * T * D <= 200_000:
+        for c in range(min(D, 3)):
+            sc = B.rlcs_elig_trace(xd[:, :, c].contiguous(), dd, gamma=0.99, lam=0.95, workspace=B.Workspace(N, T))
+            np.testing.assert_allclose(got[:, :, c], sc.cpu().numpy(), rtol=1e-5, atol=1e-5)
+
+
+def test_vector_trace_argument_checks(oracle, W, B):
+    L = B.lib()
+    P = 0x7f0000000000
+    assert L.rlcs_elig_trace_vec(P, P, P, 4, 8, 0, 0.9, 0.9, None, 0, None) == B.RLCS_OK
+    assert L.rlcs_elig_trace_vec(P, P, P, 4, 8, -1, 0.9, 0.9, None, 0, None) == B.RLCS_ERR_SIZE
+    assert L.rlcs_elig_trace_vec(None, P, P, 4, 8, 4, 0.9, 0.9, None, 0, None) == B.RLCS_ERR_NULL
+    assert L.rlcs_elig_trace_vec(P, P, P, 4, 8, 4, 1.5, 0.9, None, 0, None) == B.RLCS_ERR_ARG
+    assert L.rlcs_elig_trace_vec(P + 2, P, P, 4, 8, 4, 0.9, 0.9, None, 0, None) == B.RLCS_ERR_ALIGN
+    need = L.rlcs_elig_trace_vec_workspace_bytes(2, 100000, 8)
+    assert need > 0 and L.rlcs_elig_trace_vec_workspace_bytes(100000, 64, 64) == 0
+    assert L.rlcs_elig_trace_vec(P, P, P, 2, 100000, 8, 0.9, 0.9, None, 0, None) == B.RLCS_ERR_WORKSPACE
+
+
 # ------------------------------------------------------------------ test hooks
 def test_affine_scan_matches_generic_recurrence(oracle, W, B):
     import torch

@@ -656,3 +656,20 @@ def test_retrace_probs_structure(oracle):
     on = oracle.retrace_probs(b["r"], qv, pi, pi, act, **_bk(b), gamma=0.99, lam=0.95, c_bar=1.0)
     adv, _ = oracle.gae(b["r"], V, **_bk(b), gamma=0.99, lam=0.95)
     np.testing.assert_allclose(on - V, adv, rtol=1e-6, atol=1e-6)        # sum_a pi = 1 only to fp32 rounding
+
+
+# ----------------------------------------------------------------------------- vector-valued traces
+def test_vector_trace_is_one_scalar_trace_per_component(oracle):
+    """Shared scalar decay: component d of the vector trace is the scalar trace of x[:, :, d], exactly."""
+    rng = np.random.default_rng(60)
+    N, T, D = 3, 50, 6
+    x = rng.standard_normal((N, T, D)).astype(np.float32)
+    d = (rng.random((N, T)) < 0.1).astype(np.uint8)
+    z = oracle.elig_trace_vec(x, d, gamma=0.99, lam=0.9)
+    for c in range(D):
+        assert np.array_equal(z[:, :, c], oracle.elig_trace(np.ascontiguousarray(x[:, :, c]), d, gamma=0.99, lam=0.9))
+    # closed form without flags: z_t = sum_k (gamma lambda)^(t-k) x_k
+    z0 = oracle.elig_trace_vec(x, np.zeros((N, T), np.uint8), gamma=0.5, lam=1.0)
+    w = 0.5 ** np.arange(T)
+    want = np.stack([[np.convolve(x[n, :, c].astype(float), w)[:T] for c in range(D)] for n in range(N)]).transpose(0, 2, 1)
+    np.testing.assert_allclose(z0, want, rtol=1e-12, atol=1e-12)
