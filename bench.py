@@ -33,9 +33,9 @@ ALGOS = ("gae", "vtrace", "retrace", "td_lambda", "discounted_return", "elig_tra
 WORKLOAD = dict(N=16384, T=2048)
 FALLBACK_HBM_GBS = 6650.0
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel on the bench
-# workload, from the ncu capture summarised under profiles/ (None until a capture exists).
-NCU_TRAFFIC_BYTES = {          # profiles/dram_traffic_16384x2048.md (full-size capture, read + write)
+# dram__bytes_read.sum + dram__bytes_write.sum per launch on the bench workload, from the committed
+# one-pass ncu capture of the full-size run (summarised under profiles/).
+NCU_TRAFFIC_BYTES = {
     "gae": 576827904, "vtrace": 715524096, "retrace": 738515712, "td_lambda": 456696832,
     "discounted_return": 312028672, "elig_trace": 255066880, "episodic_prefix_sum": 251662080,
 }
