@@ -252,6 +252,44 @@ int rlcs_gae_no_alloc(const float* rewards, const float* values, const uint8_t* 
 size_t rlcs_no_alloc_scratch_bytes(void);
 
 /*
+ * Time-major variants of the seven entry points: every [T, N] tensor has element (t, n) at t*N + n
+ * (step-major rollout storage); `bootstrap` stays [N].  Same definitions, flags, NULL conventions and
+ * parameter checks as the row-major entry points above; only the layout differs.  (The paper's API
+ * is row-major only; time-major buffers are what step-major collectors hold, cf. Section 9.1.)
+ * A lane per environment walks its timesteps in scan order.  When N is a multiple of 16 and the
+ * per-step inputs are 16-byte aligned each warp streams its 32 columns through a shared-memory ring
+ * of asynchronous copies; otherwise the same walk runs from registers (any N, 4-byte alignment).
+ * When N alone cannot fill the GPU the time axis is cut into chunks and the inputs are read twice
+ * (chunk aggregates, ordered carry chain, second walk), which needs `workspace` of
+ * rlcs_time_major_workspace_bytes(N, T) bytes (0 when no cut is needed; 4-byte aligned, no
+ * initialisation required).  The workspace carries no status word: nothing in these kernels waits.
+ */
+size_t rlcs_time_major_workspace_bytes(int64_t N, int64_t T);
+int rlcs_gae_time_major(const float* rewards, const float* values, const uint8_t* dones, const uint8_t* truncs,
+                        const float* trunc_bootstrap, const float* bootstrap, float* advantages, float* returns,
+                        int64_t N, int64_t T, float gamma, float lambda,
+                        void* workspace, size_t workspace_bytes, void* cuda_stream);
+int rlcs_vtrace_time_major(const float* rewards, const float* values, const float* log_rhos, const uint8_t* dones,
+                           const uint8_t* truncs, const float* trunc_bootstrap, const float* bootstrap, float* vs,
+                           float* pg_advantages, int64_t N, int64_t T, float gamma, float rho_bar, float c_bar,
+                           void* workspace, size_t workspace_bytes, void* cuda_stream);
+int rlcs_retrace_time_major(const float* rewards, const float* q_sa, const float* expected_q, const float* log_rhos,
+                            const uint8_t* dones, const uint8_t* truncs, const float* trunc_bootstrap,
+                            const float* bootstrap, float* q_targets, int64_t N, int64_t T, float gamma, float lambda,
+                            float c_bar, void* workspace, size_t workspace_bytes, void* cuda_stream);
+int rlcs_td_lambda_time_major(const float* rewards, const float* values, const uint8_t* dones, const uint8_t* truncs,
+                              const float* trunc_bootstrap, const float* bootstrap, float* returns, int64_t N,
+                              int64_t T, float gamma, float lambda,
+                              void* workspace, size_t workspace_bytes, void* cuda_stream);
+int rlcs_discounted_return_time_major(const float* rewards, const uint8_t* dones, const uint8_t* truncs,
+                                      const float* trunc_bootstrap, const float* bootstrap, float* returns, int64_t N,
+                                      int64_t T, float gamma, void* workspace, size_t workspace_bytes, void* cuda_stream);
+int rlcs_elig_trace_time_major(const float* x, const uint8_t* dones, float* traces, int64_t N, int64_t T, float gamma,
+                               float lambda, void* workspace, size_t workspace_bytes, void* cuda_stream);
+int rlcs_episodic_prefix_sum_time_major(const float* x, const uint8_t* dones, float* sums, int64_t N, int64_t T,
+                                        int starts_at, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
  * Test hook: the bare scan of Eq. 1 / Eq. 2 on caller-supplied coefficients, every row with
  * boundary carry 0 (the paper's generic kernel of Section 4.1).
  *   forward == 0:  out_t = alpha_t + (t < T-1 ? beta_t * out_{t+1} : 0)
@@ -306,6 +344,13 @@ int rlcs_debug_force_wide_index(int on);
  * word and finishes normally -- nothing hangs or faults.
  */
 int rlcs_debug_set_carry_fault(int64_t mute_tile, int64_t spin_cap);
+
+/*
+ * Test hook: path of the time-major entry points for subsequent calls in this process.  1 = the
+ * register walk whatever the alignment, any other value = the shared-memory ring wherever N and
+ * the pointers allow it (the default).  Results must be identical (same arithmetic, same order).
+ */
+void rlcs_debug_time_major_path(int path);
 
 #ifdef __cplusplus
 }

@@ -40,10 +40,19 @@ SIGNATURES = {
     "rlcs_episodic_prefix_sum": ([_vp] * 3 + [_i64, _i64, _int] + _TAIL, _int),
     "rlcs_gae_no_alloc": ([_vp] * 8 + [_i64, _i64, _f, _f, _vp], _int),
     "rlcs_no_alloc_scratch_bytes": ([], _sz),
+    "rlcs_time_major_workspace_bytes": ([_i64, _i64], _sz),
+    "rlcs_gae_time_major": ([_vp] * 8 + [_i64, _i64, _f, _f] + _TAIL, _int),
+    "rlcs_vtrace_time_major": ([_vp] * 9 + [_i64, _i64, _f, _f, _f] + _TAIL, _int),
+    "rlcs_retrace_time_major": ([_vp] * 9 + [_i64, _i64, _f, _f, _f] + _TAIL, _int),
+    "rlcs_td_lambda_time_major": ([_vp] * 7 + [_i64, _i64, _f, _f] + _TAIL, _int),
+    "rlcs_discounted_return_time_major": ([_vp] * 6 + [_i64, _i64, _f] + _TAIL, _int),
+    "rlcs_elig_trace_time_major": ([_vp] * 3 + [_i64, _i64, _f, _f] + _TAIL, _int),
+    "rlcs_episodic_prefix_sum_time_major": ([_vp] * 3 + [_i64, _i64, _int] + _TAIL, _int),
     "rlcs_affine_scan": ([_vp] * 3 + [_i64, _i64, _int] + _TAIL, _int),
     "rlcs_debug_set_tile_variant": ([_int], _int),
     "rlcs_debug_tile_elems": ([_int], _int),
     "rlcs_debug_set_carry_fault": ([_i64, _i64], _int),
+    "rlcs_debug_time_major_path": ([_int], None),
     "rlcs_debug_force_wide_index": ([_int], _int),
     "rlcs_debug_allow_cluster_carry": ([_int], _int),
     "rlcs_debug_variant_for": ([_int, _int, _i64, _i64], _int),
@@ -332,3 +341,106 @@ def rlcs_debug_force_wide_index(on: bool):
 
 def rlcs_debug_set_carry_fault(mute_tile: int = -1, spin_cap: int = 0):
     _check(lib().rlcs_debug_set_carry_fault(mute_tile, spin_cap))
+
+
+def rlcs_debug_time_major_path(path: int = 0):
+    """1 = register walk only; anything else = shared-memory ring wherever alignment allows (default)."""
+    lib().rlcs_debug_time_major_path(int(path))
+
+
+# ------------------------------------------------------------------------------------------ time-major [T, N] entry points
+def _tm_ws(T, N, like, workspace, stream):
+    if workspace is not None:
+        return _ws(workspace)
+    nbytes = int(lib().rlcs_time_major_workspace_bytes(N, T))
+    if not nbytes:
+        return None, 0
+    buf = _torch().empty(nbytes, dtype=_torch().uint8, device=like.device)     # needs no initialisation
+    _keep.append(buf)                     # keep the scratch alive until the enqueued work has run
+    del _keep[:-8]
+    return buf.data_ptr(), nbytes
+
+
+_keep: list = []
+
+
+def rlcs_gae_time_major(rewards, values, dones, truncs=None, trunc_bootstrap=None, bootstrap=None, *, gamma, lam,
+                        advantages=None, returns=None, want_returns=True, workspace=None, stream=None):
+    """GAE on [T, N] tensors (element (t, n) at t*N + n); bootstrap [N]."""
+    T, N = rewards.shape
+    adv = _out(rewards, advantages)
+    ret = (_out(rewards, returns) if want_returns else None)
+    wp, wb = _tm_ws(T, N, rewards, workspace, stream)
+    _check(lib().rlcs_gae_time_major(_ptr(rewards, "f32"), _ptr(values, "f32", (T, N)), _ptr(dones, "u8", (T, N)),
+                                     _ptr(truncs, "u8", (T, N)), _ptr(trunc_bootstrap, "f32", (T, N)),
+                                     _ptr(bootstrap, "f32", (N,)), _ptr(adv, "f32", (T, N)), _ptr(ret, "f32", (T, N)),
+                                     N, T, gamma, lam, wp, wb, _stream(stream)))
+    return (adv, ret) if want_returns else adv
+
+
+def rlcs_vtrace_time_major(rewards, values, log_rhos, dones, truncs=None, trunc_bootstrap=None, bootstrap=None, *,
+                           gamma, rho_bar=1.0, c_bar=1.0, vs=None, pg_advantages=None, workspace=None, stream=None):
+    T, N = rewards.shape
+    vs, adv = _out(rewards, vs), _out(rewards, pg_advantages)
+    wp, wb = _tm_ws(T, N, rewards, workspace, stream)
+    _check(lib().rlcs_vtrace_time_major(_ptr(rewards, "f32"), _ptr(values, "f32", (T, N)), _ptr(log_rhos, "f32", (T, N)),
+                                        _ptr(dones, "u8", (T, N)), _ptr(truncs, "u8", (T, N)),
+                                        _ptr(trunc_bootstrap, "f32", (T, N)), _ptr(bootstrap, "f32", (N,)),
+                                        _ptr(vs, "f32", (T, N)), _ptr(adv, "f32", (T, N)), N, T, gamma, rho_bar, c_bar,
+                                        wp, wb, _stream(stream)))
+    return vs, adv
+
+
+def rlcs_retrace_time_major(rewards, q_sa, expected_q, log_rhos, dones, truncs=None, trunc_bootstrap=None,
+                            bootstrap=None, *, gamma, lam, c_bar=1.0, q_targets=None, workspace=None, stream=None):
+    T, N = rewards.shape
+    out = _out(rewards, q_targets)
+    wp, wb = _tm_ws(T, N, rewards, workspace, stream)
+    _check(lib().rlcs_retrace_time_major(_ptr(rewards, "f32"), _ptr(q_sa, "f32", (T, N)), _ptr(expected_q, "f32", (T, N)),
+                                         _ptr(log_rhos, "f32", (T, N)), _ptr(dones, "u8", (T, N)),
+                                         _ptr(truncs, "u8", (T, N)), _ptr(trunc_bootstrap, "f32", (T, N)),
+                                         _ptr(bootstrap, "f32", (N,)), _ptr(out, "f32", (T, N)), N, T, gamma, lam, c_bar,
+                                         wp, wb, _stream(stream)))
+    return out
+
+
+def rlcs_td_lambda_time_major(rewards, values, dones, truncs=None, trunc_bootstrap=None, bootstrap=None, *, gamma, lam,
+                              returns=None, workspace=None, stream=None):
+    T, N = rewards.shape
+    out = _out(rewards, returns)
+    wp, wb = _tm_ws(T, N, rewards, workspace, stream)
+    _check(lib().rlcs_td_lambda_time_major(_ptr(rewards, "f32"), _ptr(values, "f32", (T, N)), _ptr(dones, "u8", (T, N)),
+                                           _ptr(truncs, "u8", (T, N)), _ptr(trunc_bootstrap, "f32", (T, N)),
+                                           _ptr(bootstrap, "f32", (N,)), _ptr(out, "f32", (T, N)), N, T, gamma, lam,
+                                           wp, wb, _stream(stream)))
+    return out
+
+
+def rlcs_discounted_return_time_major(rewards, dones, truncs=None, trunc_bootstrap=None, bootstrap=None, *, gamma,
+                                      returns=None, workspace=None, stream=None):
+    T, N = rewards.shape
+    out = _out(rewards, returns)
+    wp, wb = _tm_ws(T, N, rewards, workspace, stream)
+    _check(lib().rlcs_discounted_return_time_major(_ptr(rewards, "f32"), _ptr(dones, "u8", (T, N)),
+                                                   _ptr(truncs, "u8", (T, N)), _ptr(trunc_bootstrap, "f32", (T, N)),
+                                                   _ptr(bootstrap, "f32", (N,)), _ptr(out, "f32", (T, N)), N, T, gamma,
+                                                   wp, wb, _stream(stream)))
+    return out
+
+
+def rlcs_elig_trace_time_major(x, dones, *, gamma, lam, traces=None, workspace=None, stream=None):
+    T, N = x.shape
+    out = _out(x, traces)
+    wp, wb = _tm_ws(T, N, x, workspace, stream)
+    _check(lib().rlcs_elig_trace_time_major(_ptr(x, "f32"), _ptr(dones, "u8", (T, N)), _ptr(out, "f32", (T, N)), N, T,
+                                            gamma, lam, wp, wb, _stream(stream)))
+    return out
+
+
+def rlcs_episodic_prefix_sum_time_major(x, dones, *, starts_at=False, sums=None, workspace=None, stream=None):
+    T, N = x.shape
+    out = _out(x, sums)
+    wp, wb = _tm_ws(T, N, x, workspace, stream)
+    _check(lib().rlcs_episodic_prefix_sum_time_major(_ptr(x, "f32"), _ptr(dones, "u8", (T, N)), _ptr(out, "f32", (T, N)),
+                                                     N, T, int(bool(starts_at)), wp, wb, _stream(stream)))
+    return out

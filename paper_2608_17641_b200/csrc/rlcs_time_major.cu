@@ -1,0 +1,943 @@
+// Time-major entry points: every [T, N] tensor has element (t, n) at t*N + n, the layout rollout
+// buffers usually have (step-major storage of N parallel environments).
+//
+// The recurrence runs along t, the strided axis here, so the mapping is the transpose of the
+// flat-tile kernels: a lane owns one environment n and walks its timesteps in scan order, carrying
+// A_{t+1} (or A_{t-1}), the neighbouring value V(s_{t+1}) and, for Retrace, the next step's log-ratio
+// in registers; the 32 lanes of a warp are 32 adjacent environments, so every row of a warp is one
+// fully used 128-byte line.  The per-step arithmetic is the definition of Section 3.2 / 3.3 itself
+// (successor value selected by flag, the recurrence continued only where no flag is set): no scan,
+// no shuffles.
+//
+// Two kernels share that arithmetic:
+//   * tm_staged_kernel: each warp streams its 32 columns through a private ring of shared-memory
+//     stages filled by 16-byte asynchronous copies (cp.async), kRows timesteps per stage.  Load
+//     addresses do not depend on the recurrence, so S-1 stages are in flight per warp whatever the
+//     register budget; the host sizes S so that the whole grid keeps roughly 16 MB in flight.  Warps
+//     never synchronise with one another.  Needs N % 16 == 0 and 16-byte aligned inputs.
+//   * tm_kernel: the same walk with two alternating register blocks instead of the ring; any N and
+//     any 4-byte alignment.
+//
+// Parallelism is N/32 warps.  When that cannot fill the GPU the time axis is cut into chunks:
+// pass 1 walks every chunk with carry 0 and keeps only its aggregate (a, b) of Eq. 2, a small pass
+// chains the carries of an environment's chunks in scan order, and pass 3 walks every chunk again
+// from its carry and writes the outputs (inputs are then read twice, the second time mostly from
+// L2 at the sizes where a cut is needed).  Deterministic either way.
+#include <cmath>
+#include <cstdint>
+#include <type_traits>
+
+#include "../../include/rlcs.h"
+#include "rlcs_scan.cuh"
+
+namespace {
+
+using rlcs::kGae;
+using rlcs::kTdLambda;
+using rlcs::kDisc;
+using rlcs::kVtrace;
+using rlcs::kRetrace;
+using rlcs::kElig;
+using rlcs::kPrefix;
+
+constexpr int kRows = 8;         // timesteps per stage / per register block
+constexpr int kThreads = 128;    // register-path block; the staged path uses 32 * warps_per_block
+
+struct TmParams {
+    const float* f0;          // rewards | x
+    const float* f1;          // values | q_sa
+    const float* f2;          // expected_q
+    const float* f3;          // log_rhos
+    const uint8_t* dones;
+    const uint8_t* truncs;
+    const float* trunc_boot;  // [T,N]
+    const float* boot;        // [N] or nullptr
+    float* out0;
+    float* out1;
+    long long N;
+    unsigned T;
+    unsigned chunk, chunks;   // timesteps per chunk, chunks per environment (1 = time axis not cut)
+    float gamma, decay, aux, rho_bar, c_bar;
+    int starts_at;
+    int stages, warps_per_block;   // tm_block_kernel: ring depth and warps per thread block
+    float* agg_a;             // [chunks, N] pass 1: chunk aggregates; after the chain: carry into each chunk
+    float* agg_b;             // [chunks, N]
+};
+
+__host__ __device__ constexpr bool tm_forward(int a) { return a == kElig || a == kPrefix; }
+// float tensors that are read at every step, and mask tensors
+__host__ __device__ constexpr int tm_nf(int a) {
+    return a == kRetrace ? 4 : a == kVtrace ? 3 : (a == kGae || a == kTdLambda) ? 2 : 1;
+}
+__host__ __device__ constexpr int tm_row_bytes(int a, bool trunc) { return tm_nf(a) * 128 + (trunc ? 2 : 1) * 32; }
+
+// all ones where x != 0, else 0; written in PTX so that the flag reaches the arithmetic below as a
+// plain word, not as a condition the compiler could branch on
+__device__ __forceinline__ unsigned ones_if(unsigned x) {
+    unsigned m;
+    asm("{\n\t.reg .pred q;\n\tsetp.ne.u32 q, %1, 0;\n\tselp.u32 %0, 0xffffffff, 0, q;\n\t}" : "=r"(m) : "r"(x));
+    return m;
+}
+
+// predicated load: *ptr where m != 0 (the address is not touched otherwise), else 0
+__device__ __forceinline__ float ldg_if_mask(const float* ptr, unsigned m) {
+    float v = 0.f;
+    asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.u32 q, %2, 0;\n\t@q ld.global.nc.f32 %0, [%1];\n\t}" : "+f"(v) : "l"(ptr), "r"(m));
+    return v;
+}
+
+// m is all ones or all zero
+__device__ __forceinline__ float keep(unsigned m, float x) { return __uint_as_float(__float_as_uint(x) & m); }
+__device__ __forceinline__ float blend(unsigned m, float x1, float x0) {
+    return __uint_as_float((__float_as_uint(x1) & m) | (__float_as_uint(x0) & ~m));
+}
+
+struct StepIn {
+    float r, v1, v2, v3;   // the step's entries of f0..f3
+    float bv;              // truncation continuation value; 0 unless the step is a live truncation
+    unsigned dn, tr;       // mask bytes
+};
+
+struct BackState {
+    float carry;      // recurrence value at t+1
+    float prod;       // product of the betas walked so far (chunk aggregate)
+    float v_next;     // V(s_{t+1}) | E_pi Q(s_{t+1},.) as stored in the buffer
+    float lr_next;    // Retrace: log-ratio of step t+1
+};
+
+struct FwdState {
+    float carry;      // recurrence value at t-1
+    float prod;
+    unsigned d_prev;  // dones flag of step t-1 (1 at t = 0: nothing to carry)
+};
+
+// Coefficients of one step, A_t = alpha + beta * A_{t+-1} (Table 1), plus V-trace's policy-gradient
+// coefficient gamma * rho_t (0 where the step is cut).
+struct Coef {
+    float alpha, beta, pg;
+};
+
+// Backward algorithms, step t of one environment (Section 3.2 / 3.3).  Flags become all-ones /
+// all-zero words and every choice is a bitwise blend: the flags differ from lane to lane, and a
+// data-dependent branch would split the warp's 128-byte stores into partial ones.
+template <int ALGO, bool TRUNC>
+__device__ __forceinline__ Coef back_coef(const StepIn& in, const TmParams& p, unsigned last, float bootv, float v_next,
+                                          float lr_next) {
+    // last: all ones at the window's final step t = T-1, else 0
+    const unsigned term = ones_if(in.dn);
+    const unsigned trunc = TRUNC ? (ones_if(in.tr) & ~term) : 0u;
+    const unsigned cont = ~(term | trunc | last);
+    // successor value: 0 after a termination, the stored continuation value after a truncation, the
+    // bootstrap at the window edge, else the buffer's next entry
+    float succ = blend(last, bootv, v_next);
+    succ = __uint_as_float((__float_as_uint(succ) & ~(term | trunc)) | (TRUNC ? __float_as_uint(in.bv) : 0u));
+    Coef c;
+    c.pg = 0.f;
+    if constexpr (ALGO == kGae) {
+        c.alpha = fmaf(p.gamma, succ, in.r) - in.v1;
+        c.beta = keep(cont, p.decay);
+    } else if constexpr (ALGO == kTdLambda) {
+        c.alpha = fmaf(blend(cont, p.aux, p.gamma), succ, in.r);
+        c.beta = keep(cont, p.decay);
+    } else if constexpr (ALGO == kDisc) {
+        // a continued step has no successor term; succ is 0 there (no value tensor), so the blended
+        // coefficient only matters where the step is cut
+        c.alpha = fmaf(keep(~cont, p.gamma), succ, in.r);
+        c.beta = keep(cont, p.decay);
+    } else if constexpr (ALGO == kVtrace) {
+        const float raw = expf(in.v3);
+        const float rho = fminf(p.rho_bar, raw), cc = fminf(p.c_bar, raw);
+        c.alpha = rho * (fmaf(p.gamma, succ, in.r) - in.v1);
+        c.beta = keep(cont, p.gamma * cc);
+        c.pg = keep(cont, p.gamma * rho);
+    } else {   // kRetrace
+        c.alpha = fmaf(p.gamma, succ, in.r) - in.v1;
+        c.beta = keep(cont, p.aux * fminf(p.c_bar, expf(lr_next)));
+    }
+    return c;
+}
+
+// Forward algorithms (eligibility trace, episodic prefix sum): the carry into step t is severed by
+// the flag of step t-1, or by the step's own flag where dones marks episode starts.
+template <int ALGO>
+__device__ __forceinline__ Coef fwd_coef(float x, unsigned d, unsigned d_prev, const TmParams& p, unsigned t) {
+    const unsigned cutflag = (ALGO == kPrefix && p.starts_at) ? (t == 0 ? 1u : d) : d_prev;
+    Coef c;
+    c.alpha = x;
+    c.beta = keep(~ones_if(cutflag), p.decay);
+    c.pg = 0.f;
+    return c;
+}
+
+// Outputs of one step from its recurrence value `val` and the scan-order predecessor's `prev`.
+template <int ALGO>
+__device__ __forceinline__ void emit(const TmParams& p, long long i, float val, float prev, float v1, const Coef& c) {
+    if constexpr (ALGO == kGae) {
+        __stcs(p.out0 + i, val);
+        if (p.out1 != nullptr) __stcs(p.out1 + i, val + v1);
+    } else if constexpr (ALGO == kVtrace) {
+        __stcs(p.out0 + i, v1 + val);
+        if (p.out1 != nullptr) __stcs(p.out1 + i, fmaf(c.pg, prev, c.alpha));
+    } else if constexpr (ALGO == kRetrace) {
+        __stcs(p.out0 + i, v1 + val);
+    } else {
+        __stcs(p.out0 + i, val);
+    }
+}
+
+template <int ALGO, bool TRUNC, int MODE>
+__device__ __forceinline__ void back_step(const StepIn& in, const TmParams& p, unsigned t, long long i, float bootv,
+                                          bool write, BackState& st) {
+    const Coef c = back_coef<ALGO, TRUNC>(in, p, (t == p.T - 1) ? ~0u : 0u, bootv, st.v_next, st.lr_next);
+    const float val = fmaf(c.beta, st.carry, c.alpha);
+    if (MODE != 1 && write) emit<ALGO>(p, i, val, st.carry, in.v1, c);
+    st.carry = val;
+    if (MODE == 1) st.prod *= c.beta;
+    if constexpr (ALGO == kRetrace) {
+        st.v_next = in.v2;
+        st.lr_next = in.v3;
+    } else if constexpr (tm_nf(ALGO) >= 2) {
+        st.v_next = in.v1;
+    }
+}
+
+template <int ALGO, int MODE>
+__device__ __forceinline__ void fwd_step(float x, unsigned d, const TmParams& p, unsigned t, long long i, bool write,
+                                         FwdState& st) {
+    const Coef c = fwd_coef<ALGO>(x, d, st.d_prev, p, t);
+    const float val = fmaf(c.beta, st.carry, c.alpha);
+    if (MODE != 1 && write) emit<ALGO>(p, i, val, st.carry, 0.f, c);
+    st.carry = val;
+    if (MODE == 1) st.prod *= c.beta;
+    st.d_prev = d;
+}
+
+// successor-side neighbours of a chunk's last step, when they lie inside the buffer
+template <int ALGO>
+__device__ __forceinline__ void init_back(BackState& st, const TmParams& p, long long n, unsigned t_hi, float carry) {
+    st.carry = carry;
+    st.prod = 1.f;
+    st.v_next = 0.f;
+    st.lr_next = 0.f;
+    if (t_hi < p.T) {
+        if constexpr (ALGO == kGae || ALGO == kTdLambda || ALGO == kVtrace) st.v_next = __ldg(p.f1 + (long long)t_hi * p.N + n);
+        if constexpr (ALGO == kRetrace) {
+            st.v_next = __ldg(p.f2 + (long long)t_hi * p.N + n);
+            st.lr_next = __ldg(p.f3 + (long long)t_hi * p.N + n);
+        }
+    }
+}
+
+__device__ __forceinline__ void init_fwd(FwdState& st, const TmParams& p, long long n, unsigned t_lo, float carry) {
+    st.carry = carry;
+    st.prod = 1.f;
+    st.d_prev = 1;
+    if (t_lo > 0) st.d_prev = __ldg(p.dones + (long long)(t_lo - 1) * p.N + n);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Register path.  Steps of a chunk are numbered q = 0 .. len-1 in scan order.
+// ---------------------------------------------------------------------------------------------
+
+template <int ALGO, bool TRUNC>
+struct Blk {
+    StepIn s[kRows];
+};
+
+template <int ALGO>
+__device__ __forceinline__ unsigned step_t(unsigned t_lo, unsigned t_hi, unsigned q) {
+    return tm_forward(ALGO) ? t_lo + q : t_hi - 1 - q;
+}
+
+template <int ALGO, bool TRUNC>
+__device__ __forceinline__ void load_blk(Blk<ALGO, TRUNC>& k, const TmParams& p, long long n, unsigned q0, unsigned len,
+                                         unsigned t_lo, unsigned t_hi) {
+#pragma unroll
+    for (int u = 0; u < kRows; ++u) {
+        if (q0 + u < len) {
+            const long long i = (long long)step_t<ALGO>(t_lo, t_hi, q0 + u) * p.N + n;
+            k.s[u].dn = __ldcs(p.dones + i);
+            k.s[u].tr = TRUNC ? __ldcs(p.truncs + i) : 0u;
+            k.s[u].r = __ldcs(p.f0 + i);
+            if constexpr (tm_nf(ALGO) >= 2) k.s[u].v1 = __ldcs(p.f1 + i);
+            if constexpr (ALGO == kRetrace) k.s[u].v2 = __ldcs(p.f2 + i);
+            if constexpr (ALGO == kVtrace || ALGO == kRetrace) k.s[u].v3 = __ldcs(p.f3 + i);
+        }
+    }
+}
+
+// sparse truncation continuation values of a block whose masks have been loaded
+template <int ALGO, bool TRUNC>
+__device__ __forceinline__ void load_bv(Blk<ALGO, TRUNC>& k, const TmParams& p, long long n, unsigned q0, unsigned len,
+                                        unsigned t_lo, unsigned t_hi) {
+    if constexpr (TRUNC) {
+#pragma unroll
+        for (int u = 0; u < kRows; ++u) {
+            k.s[u].bv = 0.f;
+            if (q0 + u < len)
+                k.s[u].bv = rlcs::ldg_if(p.trunc_boot + (long long)step_t<ALGO>(t_lo, t_hi, q0 + u) * p.N + n,
+                                         k.s[u].tr != 0 && k.s[u].dn == 0);
+        }
+    }
+}
+
+template <int ALGO, bool TRUNC, int MODE>
+__device__ __forceinline__ void walk_blk(const Blk<ALGO, TRUNC>& k, const TmParams& p, long long n, unsigned q0,
+                                         unsigned len, unsigned t_lo, unsigned t_hi, float bootv, bool write,
+                                         BackState& bs, FwdState& fs) {
+#pragma unroll
+    for (int u = 0; u < kRows; ++u) {
+        if (q0 + u < len) {
+            const unsigned t = step_t<ALGO>(t_lo, t_hi, q0 + u);
+            const long long i = (long long)t * p.N + n;
+            if constexpr (tm_forward(ALGO)) fwd_step<ALGO, MODE>(k.s[u].r, k.s[u].dn, p, t, i, write, fs);
+            else back_step<ALGO, TRUNC, MODE>(k.s[u], p, t, i, bootv, write, bs);
+        }
+    }
+}
+
+// MODE 0: whole columns, write outputs.  MODE 1: chunk aggregates only.  MODE 2: walk from the
+// chained carry and write outputs.
+template <int ALGO, bool TRUNC, int MODE>
+__global__ void __launch_bounds__(kThreads) tm_kernel(const TmParams p) {
+    constexpr bool FWD = tm_forward(ALGO);
+    const long long n_raw = (long long)blockIdx.x * kThreads + threadIdx.x;
+    const bool write = n_raw < p.N;                          // lanes past N shadow the last column
+    const long long n = write ? n_raw : p.N - 1;
+    const unsigned k = blockIdx.y;
+    const unsigned t_lo = k * p.chunk;
+    const unsigned t_hi = min(p.T, t_lo + p.chunk);          // chunk = [t_lo, t_hi)
+    const unsigned len = t_hi - t_lo;
+    const float bootv = (!FWD && p.boot != nullptr) ? __ldg(p.boot + n) : 0.f;
+    const float carry0 = MODE == 2 ? p.agg_a[(long long)k * p.N + n] : 0.f;
+
+    BackState bs = {};
+    FwdState fs = {};
+    if constexpr (FWD) init_fwd(fs, p, n, t_lo, carry0);
+    else init_back<ALGO>(bs, p, n, t_hi, carry0);
+
+    // Two register sets alternate: while one block of kRows steps is walked, the loads of the next one
+    // are in flight, and its truncation values are requested as soon as its masks have arrived.  The
+    // __syncwarp() calls are there for speed, not for correctness: lanes that drift apart (the sparse
+    // predicated loads finish at different times) are not brought back together by the hardware, and
+    // a split warp turns every 128-byte row into several partial accesses.
+    Blk<ALGO, TRUNC> a, b;
+    unsigned q = 0;
+    load_blk<ALGO, TRUNC>(a, p, n, q, len, t_lo, t_hi);
+    load_bv<ALGO, TRUNC>(a, p, n, q, len, t_lo, t_hi);
+    for (;;) {
+        __syncwarp();
+        if (q + kRows < len) load_blk<ALGO, TRUNC>(b, p, n, q + kRows, len, t_lo, t_hi);
+        walk_blk<ALGO, TRUNC, MODE>(a, p, n, q, len, t_lo, t_hi, bootv, write, bs, fs);
+        q += kRows;
+        if (q >= len) break;
+        load_bv<ALGO, TRUNC>(b, p, n, q, len, t_lo, t_hi);
+        __syncwarp();
+        if (q + kRows < len) load_blk<ALGO, TRUNC>(a, p, n, q + kRows, len, t_lo, t_hi);
+        walk_blk<ALGO, TRUNC, MODE>(b, p, n, q, len, t_lo, t_hi, bootv, write, bs, fs);
+        q += kRows;
+        if (q >= len) break;
+        load_bv<ALGO, TRUNC>(a, p, n, q, len, t_lo, t_hi);
+    }
+    if (MODE == 1 && write) {
+        p.agg_a[(long long)k * p.N + n] = FWD ? fs.carry : bs.carry;
+        p.agg_b[(long long)k * p.N + n] = FWD ? fs.prod : bs.prod;
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Staged path: per-warp shared-memory ring filled by cp.async.
+// ---------------------------------------------------------------------------------------------
+
+// 16-byte asynchronous copy global -> shared through L2 only; bytes = 0 fills the 16 bytes with zeros
+__device__ __forceinline__ void cp_async16(void* dst_smem, const void* src, unsigned bytes) {
+    const unsigned d = (unsigned)__cvta_generic_to_shared(dst_smem);
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(d), "l"(src), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+// wait until at most `pending` of this thread's committed groups are still in flight
+__device__ __forceinline__ void cp_async_wait(int pending) {
+    switch (pending) {
+        case 0: asm volatile("cp.async.wait_group 0;" ::: "memory"); break;
+        case 1: asm volatile("cp.async.wait_group 1;" ::: "memory"); break;
+        case 2: asm volatile("cp.async.wait_group 2;" ::: "memory"); break;
+        case 3: asm volatile("cp.async.wait_group 3;" ::: "memory"); break;
+        case 4: asm volatile("cp.async.wait_group 4;" ::: "memory"); break;
+        case 5: asm volatile("cp.async.wait_group 5;" ::: "memory"); break;
+        case 6: asm volatile("cp.async.wait_group 6;" ::: "memory"); break;
+        case 7: asm volatile("cp.async.wait_group 7;" ::: "memory"); break;
+        case 8: asm volatile("cp.async.wait_group 8;" ::: "memory"); break;
+        case 9: asm volatile("cp.async.wait_group 9;" ::: "memory"); break;
+        case 10: asm volatile("cp.async.wait_group 10;" ::: "memory"); break;
+        case 11: asm volatile("cp.async.wait_group 11;" ::: "memory"); break;
+        case 12: asm volatile("cp.async.wait_group 12;" ::: "memory"); break;
+        case 13: asm volatile("cp.async.wait_group 13;" ::: "memory"); break;
+        case 14: asm volatile("cp.async.wait_group 14;" ::: "memory"); break;
+        case 15: asm volatile("cp.async.wait_group 15;" ::: "memory"); break;
+        default: asm volatile("cp.async.wait_group 0;" ::: "memory"); break;   // waits for more than asked: still correct
+    }
+}
+
+constexpr int kMaxStages = 16;
+constexpr int kMaxWarps = 8;
+
+// One stage of a thread block: R = kRows * warps rows of its 32 columns, row index = scan-order step
+// within the stage.  Floats and masks live in separate rings (the mask ring runs two stages ahead):
+// float tensor a at fbase[a][row][32 floats], mask tensor m at mbase[m][row][32 bytes].
+template <int ALGO, bool TRUNC, int W>
+struct StageView {
+    static constexpr int NF = tm_nf(ALGO);
+    static constexpr int NM = TRUNC ? 2 : 1;
+    static constexpr int R = kRows * W;
+    unsigned char* fbase;
+    unsigned char* mbase;
+    __device__ __forceinline__ float* f(int a, int row) const { return reinterpret_cast<float*>(fbase + (a * R + row) * 128); }
+    __device__ __forceinline__ uint8_t* m(int a, int row) const { return mbase + (a * R + row) * 32; }
+};
+
+// Per-thread bookkeeping for the copies of a stage.  Every float tensor has 8 R 16-byte pieces per
+// stage, two per thread (rows frow and frow + 4 W, piece = tid & 7); every mask tensor 2 R, one for
+// each of the first half of the threads.  Rows past the chunk and pieces past column N are
+// zero-filled (N is a multiple of 16 here, so a piece is never split by the edge).
+struct CopyPlan {
+    long long i_first;     // flat index of the chunk's scan-order step 0, column n0
+    long long rowstep;     // flat-index step between scan-order neighbours: +N forward, -N backward
+    unsigned len;          // steps in the chunk
+    int frow, fcol;        // first float row of this thread, column offset of its piece
+    bool fcol_ok;
+    int mrow, mcol;
+    bool m_on;
+};
+
+template <int ALGO, bool TRUNC, int W>
+__device__ __forceinline__ void issue_floats(const StageView<ALGO, TRUNC, W>& sv, const TmParams& p, const CopyPlan& cp, unsigned s) {
+    constexpr int R = kRows * W;
+    const float* const fsrc[4] = {p.f0, p.f1, p.f2, p.f3};
+    constexpr int fidx[4] = {0, 1, (ALGO == kVtrace) ? 3 : 2, 3};   // V-trace stages f0, f1, f3
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        const int row = cp.frow + h * 4 * W;
+        const unsigned q = s * R + row;
+        const bool ok = cp.fcol_ok && q < cp.len;
+        const long long off = ok ? cp.i_first + cp.rowstep * q + cp.fcol : 0;
+#pragma unroll
+        for (int a = 0; a < tm_nf(ALGO); ++a)
+            cp_async16(sv.f(a, row) + cp.fcol, fsrc[fidx[a]] + off, ok ? 16u : 0u);
+    }
+}
+
+template <int ALGO, bool TRUNC, int W>
+__device__ __forceinline__ void issue_masks(const StageView<ALGO, TRUNC, W>& sv, const TmParams& p, const CopyPlan& cp, unsigned s) {
+    if (cp.m_on) {
+        const unsigned q = s * (kRows * W) + cp.mrow;
+        const bool ok = q < cp.len;
+        const long long off = ok ? cp.i_first + cp.rowstep * q + cp.mcol : 0;
+        cp_async16(sv.m(0, cp.mrow) + cp.mcol, p.dones + off, ok ? 16u : 0u);
+        if constexpr (TRUNC) cp_async16(sv.m(1, cp.mrow) + cp.mcol, p.truncs + off, ok ? 16u : 0u);
+    }
+}
+
+// truncation continuation values of `nvalid` rows from row0 of a stage whose masks have landed;
+// i = flat index of the first of them for this lane
+template <int ALGO, bool TRUNC, int W>
+__device__ __forceinline__ void stage_bv(float (&bv)[kRows], const StageView<ALGO, TRUNC, W>& sv, const TmParams& p, long long i,
+                                         long long rowstep, int row0, int nvalid, int lane, unsigned write_mask) {
+    if (nvalid <= 0) return;                                 // past the chunk: the values are never used
+    if (nvalid >= kRows) {
+#pragma unroll
+        for (int u = 0; u < kRows; ++u) {
+            const unsigned tr = sv.m(1, row0 + u)[lane], dn = sv.m(0, row0 + u)[lane];
+            bv[u] = ldg_if_mask(p.trunc_boot + i, ones_if(tr) & ~ones_if(dn) & write_mask);
+            i += rowstep;
+        }
+    } else {
+#pragma unroll
+        for (int u = 0; u < kRows; ++u) {
+            const unsigned tr = sv.m(1, row0 + u)[lane], dn = sv.m(0, row0 + u)[lane];
+            bv[u] = ldg_if_mask(p.trunc_boot + i, ones_if(tr) & ~ones_if(dn) & write_mask & (u < nvalid ? ~0u : 0u));
+            i += rowstep;
+        }
+    }
+}
+
+__device__ __forceinline__ int wrap_next(int x, int n) { return x + 1 == n ? 0 : x + 1; }
+__device__ __forceinline__ int wrap_prev(int x, int n) { return x == 0 ? n - 1 : x - 1; }
+
+// A thread block owns 32 adjacent environments; its W warps split every stage of R = kRows * W
+// timesteps in time.  Per stage: each warp walks its kRows steps from carry 0, keeping per step the
+// value so far and the running product of betas (the step's affine map of the incoming carry,
+// Eq. 2); the W per-warp aggregates go through shared memory; every warp folds them in scan order
+// onto the block's carry (a few FMAs, redundantly in each warp) to get its own incoming carry, and
+// finishes its steps with one FMA each.  The inputs cross HBM once however the time axis is split.
+//
+// Copies are committed in groups {floats of stage s, masks of stage s+2}: when a stage's floats
+// have landed so have the masks two stages on, and the sparse truncation values they point at are
+// requested two stages before their use (registers bv1, bv2).
+// MODE as in tm_kernel.
+template <int ALGO, bool TRUNC, int MODE, int W>
+__global__ void __launch_bounds__(32 * W) tm_block_kernel(const TmParams p) {
+    constexpr bool FWD = tm_forward(ALGO);
+    using SV = StageView<ALGO, TRUNC, W>;
+    extern __shared__ __align__(16) unsigned char tm_smem[];
+    const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
+    constexpr int R = kRows * W;
+    const int S = p.stages, SM = S + 2;
+    constexpr int fstage = R * SV::NF * 128, mstage = R * SV::NM * 32;
+    unsigned char* const mring = tm_smem + (size_t)S * fstage;
+    float2* const agg = reinterpret_cast<float2*>(mring + (size_t)SM * mstage);         // [2][W][32]
+    float* const edge_v = reinterpret_cast<float*>(agg + 2 * W * 32);                   // [2][32]
+    float* const edge_x = edge_v + 64;                                                  // [2][32] log-ratio | dones flag
+
+    const long long n0 = (long long)blockIdx.x * 32;
+    const bool write = n0 + lane < p.N;                      // lanes past N read zero-filled columns
+    const unsigned write_mask = write ? ~0u : 0u;
+    const long long n = write ? n0 + lane : p.N - 1;
+    const unsigned k = blockIdx.y;
+    const unsigned t_lo = k * p.chunk;
+    const unsigned t_hi = min(p.T, t_lo + p.chunk);
+    const unsigned len = t_hi - t_lo;
+    const unsigned nst = (len + R - 1) / R;
+    const float bootv = (!FWD && p.boot != nullptr) ? __ldg(p.boot + n) : 0.f;
+    const unsigned edge_last = (!FWD && t_hi == p.T) ? ~0u : 0u;   // the chunk's first step in scan order is t = T-1
+
+    CopyPlan cp;
+    cp.rowstep = FWD ? p.N : -p.N;
+    cp.i_first = (long long)(FWD ? t_lo : t_hi - 1) * p.N + n0;
+    cp.len = len;
+    cp.frow = tid >> 3; cp.fcol = 4 * (tid & 7); cp.fcol_ok = n0 + cp.fcol < p.N;
+    cp.mrow = tid >> 1; cp.mcol = 16 * (tid & 1); cp.m_on = tid < 2 * R && n0 + cp.mcol < p.N;
+
+    // block state: the affine map of everything walked so far applied to the chunk's incoming carry
+    float A = MODE == 2 ? p.agg_a[(long long)k * p.N + n] : 0.f;
+    float P = 1.f;
+    // neighbours across the chunk's scan-order start
+    BackState b0 = {};
+    FwdState f0 = {};
+    if constexpr (FWD) init_fwd(f0, p, n, t_lo, 0.f);
+    else init_back<ALGO>(b0, p, n, t_hi, 0.f);
+
+    // A group is committed for every stage index, empty past the end, so that "all but the newest P
+    // groups" always names the same stages.  Floats of stage s sit in slot s mod S, masks in slot
+    // s mod (S + 2).
+    for (int s = 0; s + 1 < S; ++s) {
+        if (s == 0) {
+            if (0 < nst) issue_masks<ALGO, TRUNC>(SV{nullptr, mring}, p, cp, 0);
+            if (1 < nst) issue_masks<ALGO, TRUNC>(SV{nullptr, mring + mstage}, p, cp, 1);
+        }
+        if ((unsigned)s < nst) issue_floats<ALGO, TRUNC>(SV{tm_smem + s * fstage, nullptr}, p, cp, s);
+        if ((unsigned)s + 2 < nst) issue_masks<ALGO, TRUNC>(SV{nullptr, mring + (s + 2) * mstage}, p, cp, s + 2);
+        cp_async_commit();
+    }
+    float bvc[kRows], bv1[kRows], bv2[kRows];
+#pragma unroll
+    for (int u = 0; u < kRows; ++u) bvc[u] = bv1[u] = bv2[u] = 0.f;
+    const int row0 = kRows * w;
+    // this lane's flat index at its first row of the current stage, and rows it has there
+    long long iw = cp.i_first + cp.rowstep * row0 + lane;
+    int left = (int)len - row0;                              // steps from this warp's first row to the chunk's end
+    const long long stagestep = cp.rowstep * R;
+    if constexpr (TRUNC) {
+        cp_async_wait(S - 2);                                // stage 0 and the masks of stages 0..2 have landed
+        __syncthreads();
+        stage_bv<ALGO, TRUNC>(bvc, SV{nullptr, mring}, p, iw, cp.rowstep, row0, left, lane, write_mask);
+        stage_bv<ALGO, TRUNC>(bv1, SV{nullptr, mring + mstage}, p, iw + stagestep, cp.rowstep, row0, left - R, lane, write_mask);
+    }
+    int fs = 0, ms = 0;                                      // ring slots of stage j
+    for (unsigned j = 0; j < nst; ++j) {
+        const int par = j & 1;
+        cp_async_wait(S - 2);                                // this thread's pieces of stage j (masks: j+2)
+        __syncthreads();                                     // ... and everyone else's
+        const SV cur{tm_smem + fs * fstage, mring + ms * mstage};
+        const int nvalid = left < kRows ? (left < 0 ? 0 : left) : kRows;
+        if constexpr (TRUNC) {
+            const int ms2 = ms + 2 >= SM ? ms + 2 - SM : ms + 2;
+            stage_bv<ALGO, TRUNC>(bv2, SV{nullptr, mring + ms2 * mstage}, p, iw + 2 * stagestep, cp.rowstep, row0, left - 2 * R,
+                                  lane, write_mask);
+        }
+        // neighbour of this warp's first step: the row before it in the stage, the last row of the
+        // previous stage, or the chunk's outside neighbour
+        float v_next = 0.f, lr_next = 0.f;
+        unsigned d_prev = 0;
+        if (w > 0) {
+            if constexpr (FWD) d_prev = cur.m(0, row0 - 1)[lane];
+            else if constexpr (ALGO == kRetrace) { v_next = cur.f(2, row0 - 1)[lane]; lr_next = cur.f(3, row0 - 1)[lane]; }
+            else if constexpr (SV::NF >= 2) v_next = cur.f(1, row0 - 1)[lane];
+        } else if (j > 0) {
+            if constexpr (FWD) d_prev = __float_as_uint(edge_x[(par ^ 1) * 32 + lane]);
+            else { v_next = edge_v[(par ^ 1) * 32 + lane]; lr_next = edge_x[(par ^ 1) * 32 + lane]; }
+        } else {
+            v_next = b0.v_next; lr_next = b0.lr_next; d_prev = f0.d_prev;
+        }
+        // pass 1: from carry 0
+        float val0[kRows], pb[kRows], v1[kRows], pgc[kRows], alp[kRows];
+        float carry = 0.f, prod = 1.f;
+        // the per-row guards exist only in the instance that the chunk's ragged last stage takes
+        auto pass1 = [&](auto full) {
+        constexpr bool FULL = decltype(full)::value;
+#pragma unroll
+        for (int u = 0; u < kRows; ++u) {
+            v1[u] = 0.f; pgc[u] = 0.f; alp[u] = 0.f;
+            if (FULL || u < nvalid) {
+                Coef c;
+                if constexpr (FWD) {
+                    const unsigned d = cur.m(0, row0 + u)[lane];
+                    c = fwd_coef<ALGO>(cur.f(0, row0 + u)[lane], d, d_prev, p, (u == 0 && w == 0 && j == 0) ? t_lo : 1u);
+                    d_prev = d;
+                } else {
+                    StepIn in;
+                    in.r = cur.f(0, row0 + u)[lane];
+                    in.v1 = SV::NF >= 2 ? cur.f(1, row0 + u)[lane] : 0.f;
+                    in.v2 = ALGO == kRetrace ? cur.f(2, row0 + u)[lane] : 0.f;
+                    in.v3 = ALGO == kRetrace ? cur.f(3, row0 + u)[lane] : ALGO == kVtrace ? cur.f(2, row0 + u)[lane] : 0.f;
+                    in.dn = cur.m(0, row0 + u)[lane];
+                    in.tr = TRUNC ? cur.m(1, row0 + u)[lane] : 0u;
+                    in.bv = bvc[u];
+                    // only the block's very first row can be the window's final step
+                    const unsigned last = (u == 0 && w == 0 && j == 0) ? edge_last : 0u;
+                    c = back_coef<ALGO, TRUNC>(in, p, last, bootv, v_next, lr_next);
+                    v_next = ALGO == kRetrace ? in.v2 : in.v1;
+                    lr_next = in.v3;
+                    v1[u] = in.v1;
+                }
+                carry = fmaf(c.beta, carry, c.alpha);
+                prod *= c.beta;
+                pgc[u] = c.pg;
+                alp[u] = c.alpha;
+            }
+            val0[u] = carry;
+            pb[u] = prod;
+        }
+        };
+        if (nvalid == kRows) pass1(std::true_type{});
+        else pass1(std::false_type{});
+        agg[(par * W + w) * 32 + lane] = make_float2(carry, prod);
+        if (w == W - 1) {                                    // neighbours for the next stage's first warp
+            if constexpr (FWD) edge_x[par * 32 + lane] = __uint_as_float(d_prev);
+            else { edge_v[par * 32 + lane] = v_next; edge_x[par * 32 + lane] = lr_next; }
+        }
+        __syncthreads();
+        // fold the warps' aggregates in scan order onto the block state
+        float cin = A;
+#pragma unroll
+        for (int x = 0; x < W; ++x) {
+            const float2 ab = agg[(par * W + x) * 32 + lane];
+            if (x == w) cin = A;
+            A = fmaf(ab.y, A, ab.x);
+            P *= ab.y;
+        }
+        // pass 2: one FMA per step, then the outputs
+        if (MODE != 1) {
+            auto pass2 = [&](auto full) {
+                constexpr bool FULL = decltype(full)::value;
+                float prev = cin;
+                long long i = iw;
+#pragma unroll
+                for (int u = 0; u < kRows; ++u) {
+                    if ((FULL || u < nvalid) && write) {
+                        const float val = fmaf(pb[u], cin, val0[u]);
+                        Coef c;
+                        c.alpha = alp[u]; c.pg = pgc[u]; c.beta = 0.f;
+                        emit<ALGO>(p, i, val, prev, v1[u], c);
+                        prev = val;
+                    }
+                    i += cp.rowstep;
+                }
+            };
+            if (nvalid == kRows) pass2(std::true_type{});
+            else pass2(std::false_type{});
+        }
+        // everyone is past the barrier, hence done with stage j-1: refill its slots
+        {
+            const unsigned s = j + S - 1;
+            if (s < nst) issue_floats<ALGO, TRUNC>(SV{tm_smem + wrap_prev(fs, S) * fstage, nullptr}, p, cp, s);
+            if (s + 2 < nst) issue_masks<ALGO, TRUNC>(SV{nullptr, mring + wrap_prev(ms, SM) * mstage}, p, cp, s + 2);
+            cp_async_commit();
+        }
+#pragma unroll
+        for (int u = 0; u < kRows; ++u) { bvc[u] = bv1[u]; bv1[u] = bv2[u]; }
+        fs = wrap_next(fs, S);
+        ms = wrap_next(ms, SM);
+        iw += stagestep;
+        left -= R;
+    }
+    cp_async_wait(0);
+    if (MODE == 1 && write && w == 0) {
+        p.agg_a[(long long)k * p.N + n] = A;
+        p.agg_b[(long long)k * p.N + n] = P;
+    }
+}
+
+// Chain an environment's chunks in scan order: carry into chunk k = a_j + b_j * (carry into j) for the
+// scan-order predecessor j.  Overwrites agg_a[k] with the carry into chunk k.
+template <bool FWD>
+__global__ void __launch_bounds__(kThreads) tm_chain_kernel(const TmParams p) {
+    const long long n = (long long)blockIdx.x * kThreads + threadIdx.x;
+    if (n >= p.N) return;
+    float carry = 0.f;
+    for (unsigned s = 0; s < p.chunks; ++s) {
+        const unsigned k = FWD ? s : p.chunks - 1 - s;
+        const long long i = (long long)k * p.N + n;
+        const float a = p.agg_a[i], b = p.agg_b[i];
+        p.agg_a[i] = carry;
+        carry = fmaf(b, carry, a);
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Host side
+// ---------------------------------------------------------------------------------------------
+
+constexpr long long kSms = 148;
+constexpr size_t kSmemPerSm = 227 * 1024;        // usable by thread blocks; each resident block also costs 1 KB
+
+// How the time axis is cut.  Depends on N and T only, so that the workspace size does.
+void plan_chunks(long long N, long long T, unsigned* chunk, unsigned* chunks) {
+    // A thread block owns 32 columns.  From about two blocks for every three SMs upward whole columns
+    // are walked; with fewer the time axis is cut.  A cut costs a second read of the inputs whatever
+    // the number of chunks, so chunks are short (two blocks per SM in total), but not below 64 steps.
+    *chunk = (unsigned)T;
+    *chunks = 1;
+    const long long groups = (N + 31) / 32;
+    if (groups >= 96) return;
+    const long long k = (2 * kSms + groups - 1) / groups;
+    long long len = (T + k - 1) / k;
+    if (len < 64) len = 64;
+    len = (len + kRows - 1) / kRows * kRows;
+    if (len >= T) return;
+    *chunk = (unsigned)len;
+    *chunks = (unsigned)((T + len - 1) / len);
+}
+
+// Warps per block and ring depth for tm_block_kernel.  Eight warps when blocks are scarce, else four.
+// The kernel is bound by issue slots and dependent-ALU latency as much as by HBM, so resident warps
+// come first: the ring is as deep as still lets min(blocks per SM, 6) blocks share an SM, no deeper
+// than keeps about 16 MB in flight over the grid, and at least 3.
+size_t plan_block(TmParams& p, int row_bytes, bool trunc) {
+    const long long blocks = (p.N + 31) / 32 * p.chunks;
+    const int W = blocks < 2 * kSms ? 8 : 4;
+    const long long stage = (long long)kRows * W * row_bytes;
+    const long long mstage = (long long)kRows * W * (trunc ? 64 : 32);
+    const long long fixed = 2 * mstage + W * 512 + 512;      // mask ring's two extra slots, aggregates, edges
+    auto block_bytes = [&](long long S) { return S * stage + fixed; };
+    long long resident = (blocks + kSms - 1) / kSms;
+    if (resident > 6) resident = 6;
+    while (resident > 1 && resident * (block_bytes(3) + 1024) > (long long)kSmemPerSm) --resident;
+    long long S = 2 + ((16ll << 20) + blocks * stage - 1) / (blocks * stage);
+    const long long nst = ((long long)p.chunk + kRows * W - 1) / (kRows * W);
+    if (S > nst + 1) S = nst + 1;
+    if (S > kMaxStages) S = kMaxStages;
+    while (S > 3 && resident * (block_bytes(S) + 1024) > (long long)kSmemPerSm) --S;
+    if (S < 3) S = 3;
+    p.stages = (int)S;
+    p.warps_per_block = W;
+    return (size_t)block_bytes(S);
+}
+
+template <typename K>
+bool allow_smem(K kernel, size_t bytes) {
+    if (bytes <= 48 * 1024) return true;
+    return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kSmemPerSm - 1024)) == cudaSuccess;
+}
+
+template <int ALGO, bool TRUNC, int W>
+int launch_block(const TmParams& p, size_t smem, cudaStream_t s) {
+    const dim3 grid((unsigned)((p.N + 31) / 32), p.chunks);
+    if (p.chunks == 1) {
+        if (!allow_smem(tm_block_kernel<ALGO, TRUNC, 0, W>, smem)) return RLCS_ERR_CUDA;
+        tm_block_kernel<ALGO, TRUNC, 0, W><<<grid, 32 * W, smem, s>>>(p);
+    } else {
+        if (!allow_smem(tm_block_kernel<ALGO, TRUNC, 1, W>, smem) || !allow_smem(tm_block_kernel<ALGO, TRUNC, 2, W>, smem))
+            return RLCS_ERR_CUDA;
+        tm_block_kernel<ALGO, TRUNC, 1, W><<<grid, 32 * W, smem, s>>>(p);
+        tm_chain_kernel<tm_forward(ALGO)><<<(unsigned)((p.N + kThreads - 1) / kThreads), kThreads, 0, s>>>(p);
+        tm_block_kernel<ALGO, TRUNC, 2, W><<<grid, 32 * W, smem, s>>>(p);
+    }
+    return cudaGetLastError() == cudaSuccess ? RLCS_OK : RLCS_ERR_CUDA;
+}
+
+template <int ALGO, bool TRUNC>
+int launch(TmParams p, bool staged, cudaStream_t s) {
+    constexpr bool FWD = tm_forward(ALGO);
+    const unsigned gx_chain = (unsigned)((p.N + kThreads - 1) / kThreads);
+    if (staged) {
+        const size_t smem = plan_block(p, tm_row_bytes(ALGO, TRUNC), TRUNC);
+        return p.warps_per_block == 8 ? launch_block<ALGO, TRUNC, 8>(p, smem, s) : launch_block<ALGO, TRUNC, 4>(p, smem, s);
+    } else {
+        const dim3 grid(gx_chain, p.chunks);
+        if (p.chunks == 1) {
+            tm_kernel<ALGO, TRUNC, 0><<<grid, kThreads, 0, s>>>(p);
+        } else {
+            tm_kernel<ALGO, TRUNC, 1><<<grid, kThreads, 0, s>>>(p);
+            tm_chain_kernel<FWD><<<gx_chain, kThreads, 0, s>>>(p);
+            tm_kernel<ALGO, TRUNC, 2><<<grid, kThreads, 0, s>>>(p);
+        }
+    }
+    return cudaGetLastError() == cudaSuccess ? RLCS_OK : RLCS_ERR_CUDA;
+}
+
+inline bool aligned4(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 3u) == 0; }
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline bool unit(float v) { return v >= 0.f && v <= 1.f; }
+
+// the staged kernels copy 16-byte pieces of every per-step input
+bool can_stage(const TmParams& p) {
+    if (p.N % 16 != 0) return false;
+    const void* in[] = {p.f0, p.f1, p.f2, p.f3, p.dones, p.truncs};
+    for (const void* q : in)
+        if (q != nullptr && !aligned16(q)) return false;
+    return true;
+}
+
+int g_force_path = 0;   // test hook: 1 = register path only, 2 = staged wherever alignment allows (the default)
+
+// shared validation and workspace wiring; returns RLCS_OK with *skip = true for empty problems
+int prepare(TmParams& p, int64_t N, int64_t T, const void* const* f32, int nf32, const uint8_t* dones,
+            const uint8_t* truncs, const float* trunc_bootstrap, bool backward, void* workspace, size_t workspace_bytes,
+            bool* skip) {
+    *skip = false;
+    if (N < 0 || T < 0 || T > (int64_t(1) << 31) - 1) return RLCS_ERR_SIZE;
+    if (N == 0 || T == 0) { *skip = true; return RLCS_OK; }
+    if (N > (int64_t(1) << 40) / T) return RLCS_ERR_SIZE;
+    if (dones == nullptr) return RLCS_ERR_NULL;
+    if (backward && (truncs == nullptr) != (trunc_bootstrap == nullptr)) return RLCS_ERR_NULL;
+    for (int i = 0; i < nf32; ++i)
+        if (f32[i] != nullptr && !aligned4(f32[i])) return RLCS_ERR_ALIGN;
+    p.N = N;
+    p.T = (unsigned)T;
+    plan_chunks(N, T, &p.chunk, &p.chunks);
+    if (p.chunks > 1) {
+        const size_t need = 2 * sizeof(float) * (size_t)N * p.chunks;
+        if (workspace == nullptr || workspace_bytes < need) return RLCS_ERR_WORKSPACE;
+        if (!aligned4(workspace)) return RLCS_ERR_ALIGN;
+        p.agg_a = static_cast<float*>(workspace);
+        p.agg_b = p.agg_a + (size_t)N * p.chunks;
+    }
+    return RLCS_OK;
+}
+
+template <int ALGO, bool TRUNC>
+int run(const TmParams& p, void* cuda_stream) {
+    const bool staged = g_force_path != 1 && can_stage(p);
+    return launch<ALGO, TRUNC>(p, staged, static_cast<cudaStream_t>(cuda_stream));
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t rlcs_time_major_workspace_bytes(int64_t N, int64_t T) {
+    if (N <= 0 || T <= 0 || T > (int64_t(1) << 31) - 1) return 0;
+    unsigned chunk, chunks;
+    plan_chunks(N, T, &chunk, &chunks);
+    return chunks > 1 ? 2 * sizeof(float) * (size_t)N * chunks : 0;
+}
+
+void rlcs_debug_time_major_path(int path) { g_force_path = path; }
+
+int rlcs_gae_time_major(const float* rewards, const float* values, const uint8_t* dones, const uint8_t* truncs,
+                        const float* trunc_bootstrap, const float* bootstrap, float* advantages, float* returns,
+                        int64_t N, int64_t T, float gamma, float lambda, void* workspace, size_t workspace_bytes,
+                        void* cuda_stream) {
+    if (!unit(gamma) || !unit(lambda)) return RLCS_ERR_ARG;
+    TmParams p = {};
+    bool skip;
+    const void* f[] = {rewards, values, trunc_bootstrap, bootstrap, advantages, returns};
+    int st = prepare(p, N, T, f, 6, dones, truncs, trunc_bootstrap, true, workspace, workspace_bytes, &skip);
+    if (st != RLCS_OK || skip) return st;
+    if (!rewards || !values || !advantages) return RLCS_ERR_NULL;
+    p.f0 = rewards; p.f1 = values; p.dones = dones; p.truncs = truncs; p.trunc_boot = trunc_bootstrap; p.boot = bootstrap;
+    p.out0 = advantages; p.out1 = returns; p.gamma = gamma; p.decay = gamma * lambda;
+    return truncs ? run<kGae, true>(p, cuda_stream) : run<kGae, false>(p, cuda_stream);
+}
+
+int rlcs_vtrace_time_major(const float* rewards, const float* values, const float* log_rhos, const uint8_t* dones,
+                           const uint8_t* truncs, const float* trunc_bootstrap, const float* bootstrap, float* vs,
+                           float* pg_advantages, int64_t N, int64_t T, float gamma, float rho_bar, float c_bar,
+                           void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    if (!unit(gamma) || !(rho_bar >= 0.f) || !(c_bar >= 0.f)) return RLCS_ERR_ARG;
+    TmParams p = {};
+    bool skip;
+    const void* f[] = {rewards, values, log_rhos, trunc_bootstrap, bootstrap, vs, pg_advantages};
+    int st = prepare(p, N, T, f, 7, dones, truncs, trunc_bootstrap, true, workspace, workspace_bytes, &skip);
+    if (st != RLCS_OK || skip) return st;
+    if (!rewards || !values || !log_rhos || !vs) return RLCS_ERR_NULL;
+    p.f0 = rewards; p.f1 = values; p.f3 = log_rhos; p.dones = dones; p.truncs = truncs; p.trunc_boot = trunc_bootstrap;
+    p.boot = bootstrap; p.out0 = vs; p.out1 = pg_advantages; p.gamma = gamma; p.rho_bar = rho_bar; p.c_bar = c_bar;
+    return truncs ? run<kVtrace, true>(p, cuda_stream) : run<kVtrace, false>(p, cuda_stream);
+}
+
+int rlcs_retrace_time_major(const float* rewards, const float* q_sa, const float* expected_q, const float* log_rhos,
+                            const uint8_t* dones, const uint8_t* truncs, const float* trunc_bootstrap,
+                            const float* bootstrap, float* q_targets, int64_t N, int64_t T, float gamma, float lambda,
+                            float c_bar, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    if (!unit(gamma) || !unit(lambda) || !(c_bar >= 0.f)) return RLCS_ERR_ARG;
+    TmParams p = {};
+    bool skip;
+    const void* f[] = {rewards, q_sa, expected_q, log_rhos, trunc_bootstrap, bootstrap, q_targets};
+    int st = prepare(p, N, T, f, 7, dones, truncs, trunc_bootstrap, true, workspace, workspace_bytes, &skip);
+    if (st != RLCS_OK || skip) return st;
+    if (!rewards || !q_sa || !expected_q || !log_rhos || !q_targets) return RLCS_ERR_NULL;
+    p.f0 = rewards; p.f1 = q_sa; p.f2 = expected_q; p.f3 = log_rhos; p.dones = dones; p.truncs = truncs;
+    p.trunc_boot = trunc_bootstrap; p.boot = bootstrap; p.out0 = q_targets; p.gamma = gamma; p.aux = gamma * lambda;
+    p.c_bar = c_bar;
+    return truncs ? run<kRetrace, true>(p, cuda_stream) : run<kRetrace, false>(p, cuda_stream);
+}
+
+int rlcs_td_lambda_time_major(const float* rewards, const float* values, const uint8_t* dones, const uint8_t* truncs,
+                              const float* trunc_bootstrap, const float* bootstrap, float* returns, int64_t N,
+                              int64_t T, float gamma, float lambda, void* workspace, size_t workspace_bytes,
+                              void* cuda_stream) {
+    if (!unit(gamma) || !unit(lambda)) return RLCS_ERR_ARG;
+    TmParams p = {};
+    bool skip;
+    const void* f[] = {rewards, values, trunc_bootstrap, bootstrap, returns};
+    int st = prepare(p, N, T, f, 5, dones, truncs, trunc_bootstrap, true, workspace, workspace_bytes, &skip);
+    if (st != RLCS_OK || skip) return st;
+    if (!rewards || !values || !returns) return RLCS_ERR_NULL;
+    p.f0 = rewards; p.f1 = values; p.dones = dones; p.truncs = truncs; p.trunc_boot = trunc_bootstrap; p.boot = bootstrap;
+    p.out0 = returns; p.gamma = gamma; p.decay = gamma * lambda; p.aux = gamma * (1.f - lambda);
+    return truncs ? run<kTdLambda, true>(p, cuda_stream) : run<kTdLambda, false>(p, cuda_stream);
+}
+
+int rlcs_discounted_return_time_major(const float* rewards, const uint8_t* dones, const uint8_t* truncs,
+                                      const float* trunc_bootstrap, const float* bootstrap, float* returns, int64_t N,
+                                      int64_t T, float gamma, void* workspace, size_t workspace_bytes,
+                                      void* cuda_stream) {
+    if (!unit(gamma)) return RLCS_ERR_ARG;
+    TmParams p = {};
+    bool skip;
+    const void* f[] = {rewards, trunc_bootstrap, bootstrap, returns};
+    int st = prepare(p, N, T, f, 4, dones, truncs, trunc_bootstrap, true, workspace, workspace_bytes, &skip);
+    if (st != RLCS_OK || skip) return st;
+    if (!rewards || !returns) return RLCS_ERR_NULL;
+    p.f0 = rewards; p.dones = dones; p.truncs = truncs; p.trunc_boot = trunc_bootstrap; p.boot = bootstrap;
+    p.out0 = returns; p.gamma = gamma; p.decay = gamma;
+    return truncs ? run<kDisc, true>(p, cuda_stream) : run<kDisc, false>(p, cuda_stream);
+}
+
+int rlcs_elig_trace_time_major(const float* x, const uint8_t* dones, float* traces, int64_t N, int64_t T, float gamma,
+                               float lambda, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    if (!unit(gamma) || !unit(lambda)) return RLCS_ERR_ARG;
+    TmParams p = {};
+    bool skip;
+    const void* f[] = {x, traces};
+    int st = prepare(p, N, T, f, 2, dones, nullptr, nullptr, false, workspace, workspace_bytes, &skip);
+    if (st != RLCS_OK || skip) return st;
+    if (!x || !traces) return RLCS_ERR_NULL;
+    p.f0 = x; p.dones = dones; p.out0 = traces; p.decay = gamma * lambda;
+    return run<kElig, false>(p, cuda_stream);
+}
+
+int rlcs_episodic_prefix_sum_time_major(const float* x, const uint8_t* dones, float* sums, int64_t N, int64_t T,
+                                        int starts_at, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    TmParams p = {};
+    bool skip;
+    const void* f[] = {x, sums};
+    int st = prepare(p, N, T, f, 2, dones, nullptr, nullptr, false, workspace, workspace_bytes, &skip);
+    if (st != RLCS_OK || skip) return st;
+    if (!x || !sums) return RLCS_ERR_NULL;
+    p.f0 = x; p.dones = dones; p.out0 = sums; p.decay = 1.f; p.starts_at = starts_at != 0;
+    return run<kPrefix, false>(p, cuda_stream);
+}
+
+}  // extern "C"

@@ -491,6 +491,104 @@ def test_vector_trace_argument_checks(oracle, W, B):
     assert L.rlcs_elig_trace_vec(P, P, P, 2, 100000, 8, 0.9, 0.9, None, 0, None) == B.RLCS_ERR_WORKSPACE
 
 
+# ------------------------------------------------------------------ time-major [T, N] entry points
+def _tm(a):
+    import torch
+    return None if a is None else torch.from_numpy(np.ascontiguousarray(np.asarray(a).T)).cuda()
+
+
+@pytest.fixture
+def tm_path(B, request):
+    B.rlcs_debug_time_major_path(request.param)
+    yield request.param
+    B.rlcs_debug_time_major_path(0)
+
+
+@pytest.mark.parametrize("N,T", [(1, 1), (3, 7), (8, 128), (300, 65), (4096, 64), (64, 3000), (5, 20000), (40000, 33),
+                                 (16, 1), (48, 517), (4112, 70), (16, 20000), (20000, 9)])
+@pytest.mark.parametrize("p_flag", [0.0, 0.02, 0.5])
+@pytest.mark.parametrize("tm_path", [1, 2], indirect=True)
+def test_time_major_entry_points(oracle, W, B, N, T, p_flag, tm_path):
+    """All seven algorithms on [T, N] tensors against the oracle run on the transposed arrays; shapes
+    cover the single-pass walk (many environments), the cut time axis (few environments), both
+    kernels (register walk; shared-memory ring, which needs N % 16 == 0) and ragged last warps."""
+    if tm_path == 2 and N % 16 != 0:
+        pytest.skip("the ring needs N % 16 == 0; the register walk is covered by tm_path = 1")
+    ro = W.make_rollout(115, N, T, p_done=p_flag, p_trunc=p_flag / 2, salt=T)
+    p = ro.params
+    ref = run_oracle(oracle, ro, ALL_ALGOS)
+    r, v, d, tr, bv = _tm(ro.rewards), _tm(ro.values), _tm(ro.dones), _tm(ro.truncs), _tm(ro.trunc_bootstrap)
+    q, eq, lr, x, dany = _tm(ro.q_sa), _tm(ro.expected_q), _tm(ro.log_rhos), _tm(ro.x), _tm(ro.any_done)
+    import torch
+    bt = torch.from_numpy(ro.bootstrap).cuda()
+    back = lambda t: t.cpu().numpy().T
+    adv, ret = B.rlcs_gae_time_major(r, v, d, tr, bv, bt, gamma=p["gamma"], lam=p["lam"])
+    assert_close("gae adv", np.ascontiguousarray(back(adv)), ref["gae"][0])
+    assert_close("gae ret", np.ascontiguousarray(back(ret)), ref["gae"][1])
+    vs, pg = B.rlcs_vtrace_time_major(r, v, lr, d, tr, bv, bt, gamma=p["gamma"], rho_bar=p["rho_bar"], c_bar=p["c_bar"])
+    assert_close("vtrace vs", np.ascontiguousarray(back(vs)), ref["vtrace"][0])
+    assert_close("vtrace adv", np.ascontiguousarray(back(pg)), ref["vtrace"][1])
+    out = B.rlcs_retrace_time_major(r, q, eq, lr, d, tr, bv, bt, gamma=p["gamma"], lam=p["lam"], c_bar=p["c_bar"])
+    assert_close("retrace", np.ascontiguousarray(back(out)), ref["retrace"])
+    out = B.rlcs_td_lambda_time_major(r, v, d, tr, bv, bt, gamma=p["gamma"], lam=p["lam"])
+    assert_close("td_lambda", np.ascontiguousarray(back(out)), ref["td_lambda"])
+    out = B.rlcs_discounted_return_time_major(r, d, tr, bv, bt, gamma=p["gamma"])
+    assert_close("disc", np.ascontiguousarray(back(out)), ref["discounted_return"])
+    out = B.rlcs_elig_trace_time_major(x, dany, gamma=p["gamma"], lam=p["lam"])
+    assert_close("elig", np.ascontiguousarray(back(out)), ref["elig_trace"])
+    out = B.rlcs_episodic_prefix_sum_time_major(x, dany)
+    assert_close("prefix ends_at", np.ascontiguousarray(back(out)), ref["prefix_ends_at"])
+    out = B.rlcs_episodic_prefix_sum_time_major(x, dany, starts_at=True)
+    assert_close("prefix starts_at", np.ascontiguousarray(back(out)), ref["prefix_starts_at"])
+    # NULL truncs / bootstrap
+    ref2 = run_oracle(oracle, ro, ("gae", "discounted_return"), use_truncs=False, use_bootstrap=False)
+    adv2 = B.rlcs_gae_time_major(r, v, d, gamma=p["gamma"], lam=p["lam"], want_returns=False)
+    assert_close("gae no truncs", np.ascontiguousarray(back(adv2)), ref2["gae"][0])
+    out = B.rlcs_discounted_return_time_major(r, d, gamma=p["gamma"])
+    assert_close("disc no truncs", np.ascontiguousarray(back(out)), ref2["discounted_return"])
+
+
+def test_time_major_paths_agree_and_misaligned_inputs_fall_back(oracle, W, B):
+    """Block kernel (shared-memory ring, time split among warps) and register walk agree to rounding;
+    inputs that are only 4-byte aligned take the register walk silently, with identical bits."""
+    import torch
+    N, T = 4112, 300
+    ro = W.make_rollout(116, N, T, p_done=0.03, p_trunc=0.01)
+    p = ro.params
+    names = ("rewards", "values", "dones", "truncs", "trunc_bootstrap")
+    al = [_tm(getattr(ro, k)) for k in names]
+    bt = torch.from_numpy(ro.bootstrap).cuda()
+    outs = []
+    for path in (1, 2):
+        B.rlcs_debug_time_major_path(path)
+        try:
+            outs.append(B.rlcs_gae_time_major(*al, bt, gamma=p["gamma"], lam=p["lam"]))
+        finally:
+            B.rlcs_debug_time_major_path(0)
+    assert_close("adv ring vs walk", outs[1][0].cpu().numpy(), outs[0][0].cpu().numpy().astype(np.float64))
+    assert_close("ret ring vs walk", outs[1][1].cpu().numpy(), outs[0][1].cpu().numpy().astype(np.float64))
+    # the same tensors one element into a larger allocation: 4-byte (1-byte for masks) aligned only
+    mis = []
+    for a in al:
+        buf = torch.empty(a.numel() + 1, dtype=a.dtype, device=a.device)
+        buf[1:].copy_(a.reshape(-1))
+        mis.append(buf[1:].view(T, N))
+    out = B.rlcs_gae_time_major(*mis, bt, gamma=p["gamma"], lam=p["lam"])
+    assert torch.equal(out[0], outs[0][0]) and torch.equal(out[1], outs[0][1])
+
+
+def test_time_major_argument_checks(oracle, W, B):
+    L = B.lib()
+    P = 0x7f0000000000
+    g = lambda **k: L.rlcs_gae_time_major(k.get("r", P), P, k.get("d", P), k.get("tr"), k.get("bv"), None, P, None,
+                                          k.get("N", 4), k.get("T", 8), k.get("g", 0.9), 0.9, None, 0, None)
+    assert g(N=0) == B.RLCS_OK and g(N=-1) == B.RLCS_ERR_SIZE and g(g=2.0) == B.RLCS_ERR_ARG
+    assert g(r=None) == B.RLCS_ERR_NULL and g(d=None) == B.RLCS_ERR_NULL and g(tr=P) == B.RLCS_ERR_NULL
+    assert g(r=P + 2) == B.RLCS_ERR_ALIGN
+    assert L.rlcs_time_major_workspace_bytes(100000, 64) == 0 and L.rlcs_time_major_workspace_bytes(8, 4096) > 0
+    assert g(N=8, T=4096) == B.RLCS_ERR_WORKSPACE
+
+
 # ------------------------------------------------------------------ test hooks
 def test_affine_scan_matches_generic_recurrence(oracle, W, B):
     import torch
