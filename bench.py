@@ -350,6 +350,55 @@ def time_time_major(torch, B, steps: int, peak: float, N: int, T: int):
     return out
 
 
+def time_bf16(torch, B, steps: int, peak: float, N: int, T: int):
+    """Extension beyond the fp32 method: the seven algorithms on bfloat16 tensors (fp32 arithmetic on
+    chip).  Algorithmic bytes: 2 per float element read or written, 1 per mask byte, the bootstrap, and
+    of the truncation continuation values the 32-byte sectors (16 values) that hold one the kernel needs."""
+    g = torch.Generator(device="cuda").manual_seed(17641)
+    mk = lambda scale=1.0: (torch.randn((N, T), generator=g, device="cuda", dtype=torch.float32) * scale).to(torch.bfloat16)
+    r, v, q, eq, lr, x, bv = mk(), mk(), mk(), mk(), mk(0.3), mk(), mk()
+    d = (torch.rand((N, T), generator=g, device="cuda") < 0.02).to(torch.uint8)
+    tr = (torch.rand((N, T), generator=g, device="cuda") < 0.005).to(torch.uint8)
+    bt = torch.randn((N,), generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+    o1, o2 = torch.empty_like(r), torch.empty_like(r)
+    ws = B.Workspace(N, T)
+    S = N * T
+    sectors = int(((tr != 0) & (d == 0)).view(-1, 16).any(dim=1).sum().item())
+    back = lambda nin, nout: 2 * S * (nin + nout) + 2 * S + 2 * N + 32 * sectors
+    fwd = 2 * S * 2 + S
+    calls = {
+        "gae": (lambda: B.rlcs_gae_bf16(r, v, d, tr, bv, bt, gamma=0.99, lam=0.95, advantages=o1, returns=o2, workspace=ws), back(2, 2)),
+        "vtrace": (lambda: B.rlcs_vtrace_bf16(r, v, lr, d, tr, bv, bt, gamma=0.99, vs=o1, pg_advantages=o2, workspace=ws), back(3, 2)),
+        "retrace": (lambda: B.rlcs_retrace_bf16(r, q, eq, lr, d, tr, bv, bt, gamma=0.99, lam=0.95, q_targets=o1, workspace=ws), back(4, 1)),
+        "td_lambda": (lambda: B.rlcs_td_lambda_bf16(r, v, d, tr, bv, bt, gamma=0.99, lam=0.95, returns=o1, workspace=ws), back(2, 1)),
+        "discounted_return": (lambda: B.rlcs_discounted_return_bf16(r, d, tr, bv, bt, gamma=0.99, returns=o1, workspace=ws), back(1, 1)),
+        "elig_trace": (lambda: B.rlcs_elig_trace_bf16(x, d, gamma=0.99, lam=0.95, traces=o1, workspace=ws), fwd),
+        "episodic_prefix_sum": (lambda: B.rlcs_episodic_prefix_sum_bf16(x, d, sums=o1, workspace=ws), fwd),
+    }
+    out = {"N": N, "T": T, "per_algorithm": {}}
+    tot_ms = tot_b = 0.0
+    for name, (call, ab) in calls.items():
+        for _ in range(3):
+            call()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(steps):
+            call()
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / steps
+        gbs = ab / (ms * 1e-3) / 1e9
+        out["per_algorithm"][name] = {"ms": round(ms, 5), "algorithmic_bytes": ab, "gbs": round(gbs, 1),
+                                      "frac_of_peak": round(gbs / peak, 4)}
+        tot_ms += ms
+        tot_b += ab
+    out["ms_per_step"] = round(tot_ms, 5)
+    out["env_steps_per_s"] = round(len(calls) * S / (tot_ms * 1e-3), 1)
+    out["all_kernels_frac"] = round(tot_b / (tot_ms * 1e-3) / 1e9 / peak, 4)
+    return out
+
+
 def time_e2e(batch: GpuBatch, steps: int, warmup: int, dist):
     """The same step called with HOST buffers: every step copies that step's inputs from pinned
     host memory to the device, runs the seven C-ABI calls, and reads all outputs back to pinned
@@ -683,6 +732,8 @@ def main():
                                                 for shape in ((4096, 512, 64), (64, 16384, 64))]
         line["extensions"]["time_major"] = [time_time_major(torch, binding, max(3, min(args.steps, 20)), peak, *shape)
                                             for shape in ((WORKLOAD["N"], WORKLOAD["T"]), (65536, 512))]
+        torch.cuda.empty_cache()
+        line["extensions"]["bf16"] = time_bf16(torch, binding, max(3, min(args.steps, 20)), peak, WORKLOAD["N"], WORKLOAD["T"])
         torch.cuda.empty_cache()
         line["sweeps"] = run_sweeps(torch, peak)
     if rank == 0:

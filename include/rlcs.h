@@ -290,6 +290,39 @@ int rlcs_episodic_prefix_sum_time_major(const float* x, const uint8_t* dones, fl
                                         int starts_at, void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * bfloat16-tensor variants of the seven entry points (the paper's kernels are fp32-only; Section 9.1
+ * defers bfloat16, Section 9.2 plans it): every float tensor -- inputs, trunc_bootstrap, bootstrap
+ * and outputs -- holds bfloat16 bit patterns (uint16_t, row-major [N, T], 2-byte aligned; 32-byte
+ * alignment of all of them enables vector access), masks stay uint8.  Inputs are widened to fp32 on
+ * load (exact), all arithmetic and the carries between tiles are fp32, outputs are rounded to
+ * nearest-even once, on store.  Same definitions, flags, NULL conventions, parameter checks and
+ * workspace (rlcs_workspace_bytes, rlcs_workspace_init) as the fp32 entry points.
+ */
+int rlcs_gae_bf16(const uint16_t* rewards, const uint16_t* values, const uint8_t* dones, const uint8_t* truncs,
+                  const uint16_t* trunc_bootstrap, const uint16_t* bootstrap, uint16_t* advantages, uint16_t* returns,
+                  int64_t N, int64_t T, float gamma, float lambda,
+                  void* workspace, size_t workspace_bytes, void* cuda_stream);
+int rlcs_vtrace_bf16(const uint16_t* rewards, const uint16_t* values, const uint16_t* log_rhos, const uint8_t* dones,
+                     const uint8_t* truncs, const uint16_t* trunc_bootstrap, const uint16_t* bootstrap, uint16_t* vs,
+                     uint16_t* pg_advantages, int64_t N, int64_t T, float gamma, float rho_bar, float c_bar,
+                     void* workspace, size_t workspace_bytes, void* cuda_stream);
+int rlcs_retrace_bf16(const uint16_t* rewards, const uint16_t* q_sa, const uint16_t* expected_q, const uint16_t* log_rhos,
+                      const uint8_t* dones, const uint8_t* truncs, const uint16_t* trunc_bootstrap,
+                      const uint16_t* bootstrap, uint16_t* q_targets, int64_t N, int64_t T, float gamma, float lambda,
+                      float c_bar, void* workspace, size_t workspace_bytes, void* cuda_stream);
+int rlcs_td_lambda_bf16(const uint16_t* rewards, const uint16_t* values, const uint8_t* dones, const uint8_t* truncs,
+                        const uint16_t* trunc_bootstrap, const uint16_t* bootstrap, uint16_t* returns, int64_t N,
+                        int64_t T, float gamma, float lambda,
+                        void* workspace, size_t workspace_bytes, void* cuda_stream);
+int rlcs_discounted_return_bf16(const uint16_t* rewards, const uint8_t* dones, const uint8_t* truncs,
+                                const uint16_t* trunc_bootstrap, const uint16_t* bootstrap, uint16_t* returns, int64_t N,
+                                int64_t T, float gamma, void* workspace, size_t workspace_bytes, void* cuda_stream);
+int rlcs_elig_trace_bf16(const uint16_t* x, const uint8_t* dones, uint16_t* traces, int64_t N, int64_t T, float gamma,
+                         float lambda, void* workspace, size_t workspace_bytes, void* cuda_stream);
+int rlcs_episodic_prefix_sum_bf16(const uint16_t* x, const uint8_t* dones, uint16_t* sums, int64_t N, int64_t T,
+                                  int starts_at, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
  * Test hook: the bare scan of Eq. 1 / Eq. 2 on caller-supplied coefficients, every row with
  * boundary carry 0 (the paper's generic kernel of Section 4.1).
  *   forward == 0:  out_t = alpha_t + (t < T-1 ? beta_t * out_{t+1} : 0)

@@ -48,6 +48,13 @@ SIGNATURES = {
     "rlcs_discounted_return_time_major": ([_vp] * 6 + [_i64, _i64, _f] + _TAIL, _int),
     "rlcs_elig_trace_time_major": ([_vp] * 3 + [_i64, _i64, _f, _f] + _TAIL, _int),
     "rlcs_episodic_prefix_sum_time_major": ([_vp] * 3 + [_i64, _i64, _int] + _TAIL, _int),
+    "rlcs_gae_bf16": ([_vp] * 8 + [_i64, _i64, _f, _f] + _TAIL, _int),
+    "rlcs_vtrace_bf16": ([_vp] * 9 + [_i64, _i64, _f, _f, _f] + _TAIL, _int),
+    "rlcs_retrace_bf16": ([_vp] * 9 + [_i64, _i64, _f, _f, _f] + _TAIL, _int),
+    "rlcs_td_lambda_bf16": ([_vp] * 7 + [_i64, _i64, _f, _f] + _TAIL, _int),
+    "rlcs_discounted_return_bf16": ([_vp] * 6 + [_i64, _i64, _f] + _TAIL, _int),
+    "rlcs_elig_trace_bf16": ([_vp] * 3 + [_i64, _i64, _f, _f] + _TAIL, _int),
+    "rlcs_episodic_prefix_sum_bf16": ([_vp] * 3 + [_i64, _i64, _int] + _TAIL, _int),
     "rlcs_affine_scan": ([_vp] * 3 + [_i64, _i64, _int] + _TAIL, _int),
     "rlcs_debug_set_tile_variant": ([_int], _int),
     "rlcs_debug_tile_elems": ([_int], _int),
@@ -107,6 +114,9 @@ def _ptr(t, dtype_kind: str, shape=None):
     if dtype_kind == "f32":
         if t.dtype != torch.float32:
             raise TypeError(f"expected float32, got {t.dtype}")     # the method is fp32-only
+    elif dtype_kind == "bf16":
+        if t.dtype != torch.bfloat16:
+            raise TypeError(f"expected bfloat16, got {t.dtype}")
     elif t.dtype not in (torch.uint8, torch.bool):
         raise TypeError(f"expected a uint8/bool mask, got {t.dtype}")
     if not t.is_contiguous():
@@ -346,6 +356,94 @@ def rlcs_debug_set_carry_fault(mute_tile: int = -1, spin_cap: int = 0):
 def rlcs_debug_time_major_path(path: int = 0):
     """1 = register walk only; anything else = shared-memory ring wherever alignment allows (default)."""
     lib().rlcs_debug_time_major_path(int(path))
+
+
+# ------------------------------------------------------------------------------------------ bfloat16 tensors
+def _out16(like, out):
+    torch = _torch()
+    return torch.empty_like(like, dtype=torch.bfloat16) if out is None else out
+
+
+def rlcs_gae_bf16(rewards, values, dones, truncs=None, trunc_bootstrap=None, bootstrap=None, *, gamma, lam,
+                  advantages=None, returns=None, want_returns=True, workspace=None, stream=None):
+    """GAE on bfloat16 tensors (fp32 arithmetic on chip, outputs rounded to bfloat16 on store)."""
+    N, T = rewards.shape
+    adv = _out16(rewards, advantages)
+    ret = (_out16(rewards, returns) if want_returns else None)
+    wp, wb = _ws(workspace)
+    _check(lib().rlcs_gae_bf16(_ptr(rewards, "bf16"), _ptr(values, "bf16", (N, T)), _ptr(dones, "u8", (N, T)),
+                               _ptr(truncs, "u8", (N, T)), _ptr(trunc_bootstrap, "bf16", (N, T)),
+                               _ptr(bootstrap, "bf16", (N,)), _ptr(adv, "bf16", (N, T)), _ptr(ret, "bf16", (N, T)),
+                               N, T, gamma, lam, wp, wb, _stream(stream)))
+    return (adv, ret) if want_returns else adv
+
+
+def rlcs_vtrace_bf16(rewards, values, log_rhos, dones, truncs=None, trunc_bootstrap=None, bootstrap=None, *,
+                     gamma, rho_bar=1.0, c_bar=1.0, vs=None, pg_advantages=None, want_advantages=True,
+                     workspace=None, stream=None):
+    N, T = rewards.shape
+    vs = _out16(rewards, vs)
+    adv = (_out16(rewards, pg_advantages) if want_advantages else None)
+    wp, wb = _ws(workspace)
+    _check(lib().rlcs_vtrace_bf16(_ptr(rewards, "bf16"), _ptr(values, "bf16", (N, T)), _ptr(log_rhos, "bf16", (N, T)),
+                                  _ptr(dones, "u8", (N, T)), _ptr(truncs, "u8", (N, T)),
+                                  _ptr(trunc_bootstrap, "bf16", (N, T)), _ptr(bootstrap, "bf16", (N,)),
+                                  _ptr(vs, "bf16", (N, T)), _ptr(adv, "bf16", (N, T)), N, T, gamma, rho_bar, c_bar,
+                                  wp, wb, _stream(stream)))
+    return (vs, adv) if want_advantages else vs
+
+
+def rlcs_retrace_bf16(rewards, q_sa, expected_q, log_rhos, dones, truncs=None, trunc_bootstrap=None, bootstrap=None, *,
+                      gamma, lam, c_bar=1.0, q_targets=None, workspace=None, stream=None):
+    N, T = rewards.shape
+    out = _out16(rewards, q_targets)
+    wp, wb = _ws(workspace)
+    _check(lib().rlcs_retrace_bf16(_ptr(rewards, "bf16"), _ptr(q_sa, "bf16", (N, T)), _ptr(expected_q, "bf16", (N, T)),
+                                   _ptr(log_rhos, "bf16", (N, T)), _ptr(dones, "u8", (N, T)), _ptr(truncs, "u8", (N, T)),
+                                   _ptr(trunc_bootstrap, "bf16", (N, T)), _ptr(bootstrap, "bf16", (N,)),
+                                   _ptr(out, "bf16", (N, T)), N, T, gamma, lam, c_bar, wp, wb, _stream(stream)))
+    return out
+
+
+def rlcs_td_lambda_bf16(rewards, values, dones, truncs=None, trunc_bootstrap=None, bootstrap=None, *, gamma, lam,
+                        returns=None, workspace=None, stream=None):
+    N, T = rewards.shape
+    out = _out16(rewards, returns)
+    wp, wb = _ws(workspace)
+    _check(lib().rlcs_td_lambda_bf16(_ptr(rewards, "bf16"), _ptr(values, "bf16", (N, T)), _ptr(dones, "u8", (N, T)),
+                                     _ptr(truncs, "u8", (N, T)), _ptr(trunc_bootstrap, "bf16", (N, T)),
+                                     _ptr(bootstrap, "bf16", (N,)), _ptr(out, "bf16", (N, T)), N, T, gamma, lam,
+                                     wp, wb, _stream(stream)))
+    return out
+
+
+def rlcs_discounted_return_bf16(rewards, dones, truncs=None, trunc_bootstrap=None, bootstrap=None, *, gamma,
+                                returns=None, workspace=None, stream=None):
+    N, T = rewards.shape
+    out = _out16(rewards, returns)
+    wp, wb = _ws(workspace)
+    _check(lib().rlcs_discounted_return_bf16(_ptr(rewards, "bf16"), _ptr(dones, "u8", (N, T)), _ptr(truncs, "u8", (N, T)),
+                                             _ptr(trunc_bootstrap, "bf16", (N, T)), _ptr(bootstrap, "bf16", (N,)),
+                                             _ptr(out, "bf16", (N, T)), N, T, gamma, wp, wb, _stream(stream)))
+    return out
+
+
+def rlcs_elig_trace_bf16(x, dones, *, gamma, lam, traces=None, workspace=None, stream=None):
+    N, T = x.shape
+    out = _out16(x, traces)
+    wp, wb = _ws(workspace)
+    _check(lib().rlcs_elig_trace_bf16(_ptr(x, "bf16"), _ptr(dones, "u8", (N, T)), _ptr(out, "bf16", (N, T)), N, T,
+                                      gamma, lam, wp, wb, _stream(stream)))
+    return out
+
+
+def rlcs_episodic_prefix_sum_bf16(x, dones, *, starts_at=False, sums=None, workspace=None, stream=None):
+    N, T = x.shape
+    out = _out16(x, sums)
+    wp, wb = _ws(workspace)
+    _check(lib().rlcs_episodic_prefix_sum_bf16(_ptr(x, "bf16"), _ptr(dones, "u8", (N, T)), _ptr(out, "bf16", (N, T)),
+                                               N, T, int(bool(starts_at)), wp, wb, _stream(stream)))
+    return out
 
 
 # ------------------------------------------------------------------------------------------ time-major [T, N] entry points

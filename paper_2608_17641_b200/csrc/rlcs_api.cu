@@ -1,152 +1,14 @@
 // C ABI of the library: argument validation, kernel selection, launch.  No allocation, no state
 // between calls apart from the two test hooks at the bottom.
-#include <cmath>
-#include <cstdint>
+#include "rlcs_host.cuh"
 
-#include "../../include/rlcs.h"
-#include "rlcs_launch.cuh"
-
-namespace {
-
-using rlcs::ScanParams;
-
-int g_variant = -1;              // test hook: tile variant; -1 = chosen per call by choose_variant
-bool g_cluster = true;           // test hook: allow the cluster carry
-bool g_wide_index = false;       // test hook: use the 64-bit index path even when 32 bits would do
-long long g_mute_tile = -1;      // test hook: tile that does not publish
-long long g_spin_cap = 0;        // test hook: poll limit (0 = default)
-constexpr unsigned kDefaultSpinCap = 1u << 21;
-
-constexpr int64_t kMaxT = (int64_t(1) << 31) - 1;
-constexpr int64_t kMaxTotal = int64_t(1) << 40;
-
-inline bool aligned(const void* p, uintptr_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
-inline bool unit_interval(float v) { return v >= 0.f && v <= 1.f; }   // false for NaN
-inline bool clip_ok(float v) { return v >= 0.f; }                       // false for NaN; +inf allowed
-
-int tile_elems(int variant) { return rlcs::kVariants[variant].threads * rlcs::kVariants[variant].items; }
-
-// size check common to every entry point; returns RLCS_OK with *total = 0 for empty problems
-int check_sizes(int64_t N, int64_t T, int64_t* total) {
-    *total = 0;
-    if (N < 0 || T < 0 || T > kMaxT) return RLCS_ERR_SIZE;
-    if (N == 0 || T == 0) return RLCS_OK;
-    if (N > kMaxTotal / T) return RLCS_ERR_SIZE;
-    *total = N * T;
-    return RLCS_OK;
-}
-
-struct Ptrs {
-    const void* f32[8];
-    int nf32 = 0;
-    const void* u8[2];
-    int nu8 = 0;
-    void add_f32(const void* p) { if (p) f32[nf32++] = p; }
-    void add_u8(const void* p) { if (p) u8[nu8++] = p; }
-};
-
-// RLCS_ERR_ALIGN if an fp32 pointer is not 4-byte aligned; *vec = all pointers allow vector access
-int check_alignment(const Ptrs& ps, bool* vec) {
-    *vec = true;
-    for (int i = 0; i < ps.nf32; ++i) {
-        if (!aligned(ps.f32[i], 4)) return RLCS_ERR_ALIGN;
-        if (!aligned(ps.f32[i], 32)) *vec = false;          // 256-bit vector accesses
-    }
-    for (int i = 0; i < ps.nu8; ++i)
-        if (!aligned(ps.u8[i], 16)) *vec = false;
-    return RLCS_OK;
-}
-
-// Kernel and tile shape for one call, from measurements on B200 (see the tile-variant table in
-// rlcs_launch.cuh).  Large problems are bound by HBM: what matters is resident warps and bytes in
-// flight, so algorithms with few registers run more blocks per SM or 16 steps per thread.  Small
-// problems are bound by latency: smaller tiles spread them over more SMs, unless rows are long
-// enough for the inter-block carry to dominate.
-int choose_variant(int algo, bool trunc, int64_t total, int64_t T) {
-    if (g_variant >= 0) return g_variant;
-    if (total < (int64_t(1) << 23)) return T <= 2048 ? 6 : 0;
-    switch (algo) {
-        case rlcs::kGae:
-        case rlcs::kGaeStats: return trunc ? 16 : 0;
-        case rlcs::kVtrace: return trunc ? 18 : 0;
-        case rlcs::kRetrace: return 0;
-        case rlcs::kTdLambda: return trunc ? 17 : 0;
-        case rlcs::kDisc: return trunc ? 17 : 5;
-        case rlcs::kElig: return 18;
-        case rlcs::kPrefix: return 18;
-        default: return 0;
-    }
-}
-
-// Fill the size / tiling / carry fields and validate the workspace for this call.
-int finish_params(ScanParams& p, int variant, int64_t total, int64_t T, void* workspace, size_t workspace_bytes, bool vec,
-                  bool allow_cluster = true) {
-    const int tile = tile_elems(variant);
-    p.total = total;
-    p.T = (unsigned)T;
-    p.num_tiles = (total + tile - 1) / tile;
-    p.idx32 = !g_wide_index && (total + tile) <= 0xffffffffLL;
-    {   // invariant division by T (see FastDiv)
-        int l = 0;
-        while ((int64_t(1) << l) < T) ++l;
-        p.div_T.mul = (unsigned)((((uint64_t(1) << 32) * ((uint64_t(1) << l) - (uint64_t)T)) / (uint64_t)T) + 1);
-        p.div_T.sh1 = l < 1 ? l : 1;
-        p.div_T.sh2 = l > 1 ? l - 1 : 0;
-    }
-    p.decay_pow = 1.f;                       // beta product of a chunk without resets
-    for (int i = 0; i < rlcs::kVariants[variant].items; ++i) p.decay_pow *= p.decay;
-    p.carry_mode = (tile % T) != 0;          // T does not divide the tile: rows straddle tiles
-    // Rows of exactly 2..8 tiles: one thread-block cluster per row carries through distributed
-    // shared memory instead (needs the vectorised one-tile kernel; g_cluster = 0 turns it off).
-    p.cluster = 0;
-    if (allow_cluster && g_cluster && vec && rlcs::kVariants[variant].stages == 0 && T % tile == 0 && T / tile >= 2 && T / tile <= 8) {
-        p.cluster = (int)(T / tile);
-        p.carry_mode = 0;
-    }
-    p.header = nullptr;
-    p.records = nullptr;
-    p.status = nullptr;
-    if (workspace != nullptr && workspace_bytes >= sizeof(unsigned) * rlcs::kHeaderWords && aligned(workspace, 16))
-        p.status = static_cast<unsigned*>(workspace) + 2;
-    p.mute_tile = g_mute_tile;
-    p.spin_cap = g_spin_cap > 0 ? (unsigned)g_spin_cap : kDefaultSpinCap;
-    if (p.carry_mode) {
-        const size_t need = sizeof(unsigned) * rlcs::kHeaderWords + sizeof(uint4) * (size_t)p.num_tiles;
-        if (workspace == nullptr || workspace_bytes < need) return RLCS_ERR_WORKSPACE;
-        if (!aligned(workspace, 16)) return RLCS_ERR_ALIGN;
-        p.header = static_cast<unsigned*>(workspace);
-        p.records = reinterpret_cast<uint4*>(p.header + rlcs::kHeaderWords);
-    }
-    return RLCS_OK;
-}
-
-typedef cudaError_t (*Launcher)(const ScanParams&, int, bool, bool, cudaStream_t);
-
-int run(Launcher fn, const ScanParams& p, int variant, bool trunc, bool vec, void* stream) {
-    return fn(p, variant, trunc, vec, static_cast<cudaStream_t>(stream)) == cudaSuccess ? RLCS_OK : RLCS_ERR_CUDA;
-}
-
-// shared front half of the five backward entry points
-int backward_common(ScanParams& p, Ptrs& ps, const uint8_t* dones, const uint8_t* truncs,
-                    const float* trunc_bootstrap, const float* bootstrap, int64_t N, int64_t T,
-                    int64_t* total, bool* vec) {
-    int st = check_sizes(N, T, total);
-    if (st != RLCS_OK || *total == 0) return st;
-    if (dones == nullptr || (truncs == nullptr) != (trunc_bootstrap == nullptr)) return RLCS_ERR_NULL;
-    ps.add_u8(dones);
-    ps.add_u8(truncs);
-    ps.add_f32(trunc_bootstrap);
-    ps.add_f32(bootstrap);
-    st = check_alignment(ps, vec);
-    if (st != RLCS_OK) return st;
-    p.dones = dones;
-    p.truncs = truncs;
-    p.trunc_boot = trunc_bootstrap;
-    p.boot = bootstrap;
-    return RLCS_OK;
-}
-
-}  // namespace
+namespace rlcs_hooks {
+int g_variant = -1;
+bool g_cluster = true;
+bool g_wide_index = false;
+long long g_mute_tile = -1;
+long long g_spin_cap = 0;
+}  // namespace rlcs_hooks
 
 extern "C" {
 

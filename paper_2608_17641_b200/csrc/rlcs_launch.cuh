@@ -5,7 +5,7 @@
 
 #include "rlcs_scan.cuh"
 
-namespace rlcs {
+namespace RLCS_NS {
 
 // stages == 0: scan_kernel (one tile per block).  stages > 0: scan_kernel_tma (persistent blocks,
 // bulk-copy ring of that many tiles; min_blocks = blocks per SM it is compiled and sized for).
@@ -32,6 +32,8 @@ constexpr TileVariant kVariants[kNumVariants] = {
     {256, 8, 6, 0},    // 17: 2048, at most 40 registers
     {128, 16, 5, 0},   // 18: 2048, 16 steps per thread
 };
+// The bfloat16 build instantiates only these tile shapes (16 steps per thread = one 32-byte access).
+__host__ __device__ constexpr bool variant_built(int v) { return !kIoBf16 || v == 0 || v == 5 || v == 6 || v == 18; }
 constexpr int kMinTileElems = 512;
 constexpr int kRetraceProbsThreads = 256, kRetraceProbsItems = 4;      // tile of rlcs_retrace_probs
 constexpr int kMaxDevices = 64;
@@ -110,7 +112,9 @@ cudaError_t launch_tv(const ScanParams& p, int variant, cudaStream_t stream) {
     if constexpr (V >= kNumVariants) {
         return cudaErrorInvalidValue;
     } else {
-        if (variant == V) return launch_variant<ALGO, TRUNC, VEC, V>(p, stream);
+        if constexpr (variant_built(V)) {
+            if (variant == V) return launch_variant<ALGO, TRUNC, VEC, V>(p, stream);
+        }
         return launch_tv<ALGO, TRUNC, VEC, V + 1>(p, variant, stream);
     }
 }
@@ -146,4 +150,4 @@ cudaError_t launch_norm_rescale(float* adv, long long total, const float* mean_r
         return launch_algo<ALGO, HAS_TRUNC>(p, variant, trunc, vec, stream);                        \
     }
 
-}  // namespace rlcs
+}  // namespace RLCS_NS

@@ -34,7 +34,26 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
-namespace rlcs {
+// Element type of the float tensors in global memory.  A translation unit that defines
+// RLCS_IO_BF16 before including this header gets the same kernels with bfloat16 tensors (inputs
+// widened to fp32 on load -- exact -- and all arithmetic in fp32 registers, outputs rounded to
+// nearest-even on store) in a namespace of their own, so that both builds link into one library.
+#ifdef RLCS_IO_BF16
+#include <cuda_bf16.h>
+#define RLCS_NS rlcs_bf16
+namespace RLCS_NS {
+using io_t = __nv_bfloat16;
+constexpr bool kIoBf16 = true;
+}
+#else
+#define RLCS_NS rlcs
+namespace RLCS_NS {
+using io_t = float;
+constexpr bool kIoBf16 = false;
+}
+#endif
+
+namespace RLCS_NS {
 
 enum Algo : int {
     kGae = 0, kTdLambda = 1, kDisc = 2, kVtrace = 3, kRetrace = 4, kElig = 5, kPrefix = 6,
@@ -67,20 +86,20 @@ struct FastDiv {
 };
 
 struct ScanParams {
-    const float* f0;          // rewards | x | alpha
-    const float* f1;          // values | q_sa | beta
-    const float* f2;          // expected_q
-    const float* f3;          // log_rhos
+    const io_t* f0;           // rewards | x | alpha
+    const io_t* f1;           // values | q_sa | beta
+    const io_t* f2;           // expected_q
+    const io_t* f3;           // log_rhos
     const float* pi;          // kRetraceProbs: target-policy probabilities [N,T,A]  (f1 = Q-values [N,T,A])
     const float* mu;          // kRetraceProbs: behaviour-policy probabilities [N,T,A]
     const int* actions;       // kRetraceProbs: actions taken [N,T]
     int A;                    // kRetraceProbs: number of actions
     const uint8_t* dones;
     const uint8_t* truncs;
-    const float* trunc_boot;  // [N,T]
-    const float* boot;        // [N] or nullptr
-    float* out0;
-    float* out1;              // second output or nullptr
+    const io_t* trunc_boot;   // [N,T]
+    const io_t* boot;         // [N] or nullptr
+    io_t* out0;
+    io_t* out1;               // second output or nullptr
     float* stats;             // kGaeStats: per scan-order tile {sum A, sum A^2}
     long long total;          // N*T
     long long num_tiles;
@@ -196,6 +215,78 @@ __device__ __forceinline__ void store_f32(float* __restrict__ p, long long i0, i
             if (j < nvalid) __stcs(p + i0 + j, x[j]);
     }
 }
+
+#ifdef RLCS_IO_BF16
+// bfloat16 tensors: a 32-bit word holds two consecutive elements (low half first); widening is a
+// shift or a mask, narrowing is cvt.rn.bf16x2.f32 (round to nearest even).
+__device__ __forceinline__ void widen2(unsigned w, float& lo, float& hi) {
+    lo = __uint_as_float(w << 16);
+    hi = __uint_as_float(w & 0xffff0000u);
+}
+__device__ __forceinline__ unsigned narrow2(float lo, float hi) {
+    const __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<const unsigned*>(&h);
+}
+__device__ __forceinline__ float ld_io(const io_t* p) {
+    return __uint_as_float((unsigned)__ldg(reinterpret_cast<const unsigned short*>(p)) << 16);
+}
+__device__ __forceinline__ float ldg_if(const io_t* p, bool pred) {
+    unsigned short v = 0;
+    asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.u32 q, %2, 0;\n\t@q ld.global.nc.u16 %0, [%1];\n\t}"
+                 : "+h"(v) : "l"(p), "r"((unsigned)pred));
+    return __uint_as_float((unsigned)v << 16);
+}
+
+template <int ITEMS, bool VEC>
+__device__ __forceinline__ void load_f32(const io_t* __restrict__ p, long long i0, int nvalid, float (&x)[ITEMS]) {
+    if (VEC && nvalid == ITEMS) {
+        unsigned w[ITEMS / 2];
+        if constexpr (ITEMS == 16) {
+            asm volatile("ld.global.nc.L1::no_allocate.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                         : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]), "=r"(w[4]), "=r"(w[5]), "=r"(w[6]), "=r"(w[7])
+                         : "l"(p + i0));
+        } else if constexpr (ITEMS == 8) {
+            const uint4 v = __ldcs(reinterpret_cast<const uint4*>(p + i0));
+            w[0] = v.x; w[1] = v.y; w[2] = v.z; w[3] = v.w;
+        } else {
+            static_assert(ITEMS == 4, "ITEMS must be 4, 8 or 16");
+            const uint2 v = __ldcs(reinterpret_cast<const uint2*>(p + i0));
+            w[0] = v.x; w[1] = v.y;
+        }
+#pragma unroll
+        for (int k = 0; k < ITEMS / 2; ++k) widen2(w[k], x[2 * k], x[2 * k + 1]);
+    } else {
+        const unsigned short* q = reinterpret_cast<const unsigned short*>(p) + i0;
+#pragma unroll
+        for (int j = 0; j < ITEMS; ++j) x[j] = (j < nvalid) ? __uint_as_float((unsigned)__ldcs(q + j) << 16) : 0.f;
+    }
+}
+
+template <int ITEMS, bool VEC>
+__device__ __forceinline__ void store_f32(io_t* __restrict__ p, long long i0, int nvalid, const float (&x)[ITEMS]) {
+    if (VEC && nvalid == ITEMS) {
+        unsigned w[ITEMS / 2];
+#pragma unroll
+        for (int k = 0; k < ITEMS / 2; ++k) w[k] = narrow2(x[2 * k], x[2 * k + 1]);
+        if constexpr (ITEMS == 16) {
+            asm volatile("st.global.cs.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+                         :: "l"(p + i0), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7])
+                         : "memory");
+        } else if constexpr (ITEMS == 8) {
+            __stcs(reinterpret_cast<uint4*>(p + i0), make_uint4(w[0], w[1], w[2], w[3]));
+        } else {
+            __stcs(reinterpret_cast<uint2*>(p + i0), make_uint2(w[0], w[1]));
+        }
+    } else {
+        unsigned short* q = reinterpret_cast<unsigned short*>(p) + i0;
+#pragma unroll
+        for (int j = 0; j < ITEMS; ++j)
+            if (j < nvalid) __stcs(q + j, (unsigned short)(narrow2(x[j], 0.f) & 0xffffu));
+    }
+}
+#else
+__device__ __forceinline__ float ld_io(const io_t* p) { return __ldg(p); }
+#endif
 
 // ------------------------------------------------------------------------------------------ shared-memory reads
 template <int ITEMS>
@@ -438,7 +529,7 @@ __device__ __forceinline__ void load_values_global(const Chunk<ALGO, TRUNC, ITEM
     v.halo = 0.f;
     v.halo_lr = 0.f;
     if constexpr (float_halo(ALGO)) {
-        const float* src = (ALGO == kRetrace) ? p.f2 : p.f1;
+        const io_t* src = (ALGO == kRetrace) ? p.f2 : p.f1;
         const bool edge_lane = (lane == 31) && (p.total - i0 > ITEMS);
         v.halo = ldg_if(src + i0 + ITEMS, edge_lane);
         if constexpr (ALGO == kRetrace) v.halo_lr = ldg_if(p.f3 + i0 + ITEMS, edge_lane);
@@ -452,6 +543,7 @@ __device__ __forceinline__ void load_values_global(const Chunk<ALGO, TRUNC, ITEM
     }
 }
 
+#ifndef RLCS_IO_BF16   // the [N,T,A] form stays fp32
 // Retrace from the [N,T,A] tensors: per step, Q(s_t,a_t), E_pi Q(s_t,.) = sum_a pi(a|s_t) Q(s_t,a) and the
 // importance ratio pi(a_t|s_t)/mu(a_t|s_t) are formed here from one dense read of the Q and pi rows
 // and three gathers, and only those three scalars per step stay in registers -- the tile never
@@ -543,6 +635,8 @@ __device__ __forceinline__ void load_values_probs(const Chunk<ALGO, TRUNC, ITEMS
     v.halo = (lane != 31) ? nb : heq;
     v.halo_lr = (lane != 31) ? nr : hr;
 }
+
+#endif  // !RLCS_IO_BF16
 
 // Shared-memory scratch of the block-level scan; double-buffered by tile parity in the persistent
 // kernel so that one barrier per tile suffices.
@@ -663,7 +757,7 @@ __device__ __forceinline__ void tile_compute(Chunk<ALGO, TRUNC, ITEMS>& c, Vals<
 #pragma unroll
                 for (int j = 0; j < ITEMS; ++j) {
                     if ((unsigned)j == e) {
-                        if (j < nvalid && !test_byte(c.dw, j) && !test_byte(c.tw, j)) c.ov[j] = __ldg(p.boot + n);
+                        if (j < nvalid && !test_byte(c.dw, j) && !test_byte(c.tw, j)) c.ov[j] = ld_io(p.boot + n);
                         e += p.T;
                         ++n;
                     }
@@ -920,6 +1014,7 @@ __global__ void __launch_bounds__(THREADS, MIN_BLOCKS) scan_kernel(const ScanPar
 }
 
 // ------------------------------------------------------------------------------------------ kernel 1c: Retrace from [N,T,A] tensors
+#ifndef RLCS_IO_BF16
 template <bool TRUNC, bool VEC, int THREADS, int ITEMS, int AV, bool FULL>
 __device__ __forceinline__ void one_tile_probs(const ScanParams& p, long long tile, long long s, unsigned epoch,
                                                ScanSmem<THREADS / 32>& sm) {
@@ -950,6 +1045,8 @@ __global__ void __launch_bounds__(THREADS, MIN_BLOCKS) scan_kernel_retrace_probs
     if (full) one_tile_probs<TRUNC, VEC, THREADS, ITEMS, AV, true>(p, tile, s, epoch, sm);
     else one_tile_probs<TRUNC, VEC, THREADS, ITEMS, AV, false>(p, tile, s, epoch, sm);
 }
+
+#endif  // !RLCS_IO_BF16
 
 // ------------------------------------------------------------------------------------------ kernel 1b: one tile per block, one cluster per row
 // For rows that are exactly 2..8 tiles long (T = k * TILE): launched with cluster size k, so a
@@ -1235,4 +1332,4 @@ __global__ void __launch_bounds__(THREADS, MIN_BLOCKS) scan_kernel_tma(const Sca
     if (p.carry_mode) sign_off(p);
 }
 
-}  // namespace rlcs
+}  // namespace RLCS_NS

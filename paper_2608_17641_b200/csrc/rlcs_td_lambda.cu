@@ -1,6 +1,6 @@
 // Kernel instantiations for one algorithm (see rlcs_scan.cuh for the kernel itself).
 #include "rlcs_launch.cuh"
 
-namespace rlcs {
+namespace RLCS_NS {
 RLCS_DEFINE_LAUNCHER(launch_td_lambda, kTdLambda, true)
-}  // namespace rlcs
+}  // namespace RLCS_NS
