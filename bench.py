@@ -273,16 +273,23 @@ def time_retrace_probs(torch, B, steps: int, peak: float, N=16384, T=2048, A=4):
             "gbs": round(gbs, 1), "frac_of_peak": round(gbs / peak, 4)}
 
 
-def time_elig_trace_vec(torch, B, steps: int, peak: float, N: int, T: int, D: int):
-    """Extension beyond the seven kernels: vector-valued eligibility traces x[N,T,D] -> z[N,T,D].
-    Algorithmic bytes: one read of x, one write of z, the [N,T] flag."""
+def time_elig_trace_vec(torch, B, steps: int, peak: float, N: int, T: int, D: int, per_dim: bool = False):
+    """Extension beyond the seven kernels: vector-valued eligibility traces x[N,T,D] -> z[N,T,D], with
+    the shared scalar decay or (per_dim) a decay tensor beta[N,T,D] ~ U(0.5, 1).
+    Algorithmic bytes: one read of x (and beta), one write of z, the [N,T] flag."""
     g = torch.Generator(device="cuda").manual_seed(17641)
     x = torch.randn((N, T, D), generator=g, device="cuda", dtype=torch.float32)
     d = (torch.rand((N, T), generator=g, device="cuda") < 0.02).to(torch.uint8)
     out = torch.empty_like(x)
-    nbytes = int(B.lib().rlcs_elig_trace_vec_workspace_bytes(N, T, D))
-    ws = B.Workspace(N, T, nbytes=nbytes) if nbytes else None
-    call = lambda: B.rlcs_elig_trace_vec(x, d, gamma=0.99, lam=0.95, traces=out, workspace=ws)
+    if per_dim:
+        beta = torch.rand((N, T, D), generator=g, device="cuda", dtype=torch.float32) * 0.5 + 0.5
+        nbytes = int(B.lib().rlcs_elig_trace_vec_beta_workspace_bytes(N, T, D))
+        ws = B.Workspace(N, T, nbytes=nbytes) if nbytes else None
+        call = lambda: B.rlcs_elig_trace_vec_beta(x, beta, d, traces=out, workspace=ws)
+    else:
+        nbytes = int(B.lib().rlcs_elig_trace_vec_workspace_bytes(N, T, D))
+        ws = B.Workspace(N, T, nbytes=nbytes) if nbytes else None
+        call = lambda: B.rlcs_elig_trace_vec(x, d, gamma=0.99, lam=0.95, traces=out, workspace=ws)
     for _ in range(3):
         call()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -293,7 +300,7 @@ def time_elig_trace_vec(torch, B, steps: int, peak: float, N: int, T: int, D: in
     e1.record()
     torch.cuda.synchronize()
     ms = e0.elapsed_time(e1) / steps
-    ab = N * T * (8 * D + 1)
+    ab = N * T * ((12 if per_dim else 8) * D + 1)
     gbs = ab / (ms * 1e-3) / 1e9
     return {"ms": round(ms, 5), "N": N, "T": T, "D": D, "time_axis_cut": bool(nbytes), "algorithmic_bytes": ab,
             "gbs": round(gbs, 1), "frac_of_peak": round(gbs / peak, 4)}
@@ -730,6 +737,9 @@ def main():
         line["extensions"]["retrace_probs"] = time_retrace_probs(torch, binding, max(3, min(args.steps, 30)), peak)
         line["extensions"]["elig_trace_vec"] = [time_elig_trace_vec(torch, binding, max(3, min(args.steps, 30)), peak, *shape)
                                                 for shape in ((4096, 512, 64), (64, 16384, 64))]
+        line["extensions"]["elig_trace_vec_beta"] = [
+            time_elig_trace_vec(torch, binding, max(3, min(args.steps, 30)), peak, *shape, per_dim=True)
+            for shape in ((16384, 128, 64), (4096, 512, 64))]
         line["extensions"]["time_major"] = [time_time_major(torch, binding, max(3, min(args.steps, 20)), peak, *shape)
                                             for shape in ((WORKLOAD["N"], WORKLOAD["T"]), (65536, 512))]
         torch.cuda.empty_cache()

@@ -213,6 +213,19 @@ int rlcs_elig_trace_vec(const float* x, const uint8_t* dones, float* traces, int
 size_t rlcs_elig_trace_vec_workspace_bytes(int64_t N, int64_t T, int64_t D);
 
 /*
+ * Eligibility trace with a decay per component and step (the per-dimension beta_t that Section 9.1
+ * lists as unsupported by a scalar-beta kernel; Eq. 1 component by component):
+ *   z_t[c] = x_t[c] + ((t > 0 and not dones_{t-1}) ? beta_t[c] * z_{t-1}[c] : 0)
+ * x, beta, traces: [N, T, D] contiguous with d innermost (beta[n, 0, :] is never used); dones [N, T].
+ * Any finite beta is accepted (the caller folds gamma*lambda in).  Same kernel structure, workspace
+ * rules (rlcs_elig_trace_vec_beta_workspace_bytes), alignment rules and limits as rlcs_elig_trace_vec.
+ */
+int rlcs_elig_trace_vec_beta(const float* x, const float* beta, const uint8_t* dones, float* traces, int64_t N, int64_t T,
+                             int64_t D, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+size_t rlcs_elig_trace_vec_beta_workspace_bytes(int64_t N, int64_t T, int64_t D);
+
+/*
  * Episodic prefix sum, forward in time -- Section 3.3.6.
  *   starts_at == 0 ("ends_at", the flag closes a segment):  C_t = x_t + ((t>0 and not dones_{t-1}) ? C_{t-1} : 0)
  *   starts_at != 0 (the flag opens a segment):              C_t = x_t + ((t>0 and not dones_t)     ? C_{t-1} : 0)

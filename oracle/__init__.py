@@ -60,6 +60,8 @@ def _load():
             lib.rlcs_oracle_elig_trace.argtypes = [_F, _U, _D, _i64, _i64, _dbl, _dbl]
             lib.rlcs_oracle_elig_trace_vec.argtypes = [_F, _U, _D, _i64, _i64, _i64, _dbl, _dbl]
             lib.rlcs_oracle_elig_trace_vec.restype = None
+            lib.rlcs_oracle_elig_trace_vec_beta.argtypes = [_F, _F, _U, _D, _i64, _i64, _i64]
+            lib.rlcs_oracle_elig_trace_vec_beta.restype = None
             lib.rlcs_oracle_episodic_prefix_sum.argtypes = [_F, _U, _D, _i64, _i64, ctypes.c_int]
             lib.rlcs_oracle_linear_recurrence.argtypes = [_D, _D, _dbl, _D, _i64, ctypes.c_int]
             lib.rlcs_oracle_combine.argtypes = [_dbl, _dbl, _dbl, _dbl, _D, _D]
@@ -238,6 +240,22 @@ def elig_trace_vec(x, dones, *, gamma, lam):
     d = _u8(dones, (N, T))
     out = np.empty(xx.shape, np.float64)
     _load().rlcs_oracle_elig_trace_vec(_p(xx, _F), _p(d, _U), _p(out, _D), N, T, D, _s(gamma), _s(lam))
+    return out
+
+
+def elig_trace_vec_beta(x, beta, dones):
+    """Eligibility trace with a decay per component and step: x, beta [N,T,D], dones [N,T] -- Eq. 1
+    component by component (per-dimension beta, Section 9.1)."""
+    xx = np.ascontiguousarray(x, dtype=np.float32)
+    if xx.ndim != 3:
+        raise ValueError("expected an [N, T, D] array")
+    N, T, D = xx.shape
+    bb = np.ascontiguousarray(beta, dtype=np.float32)
+    if bb.shape != xx.shape:
+        raise ValueError("beta must have the shape of x")
+    d = _u8(dones, (N, T))
+    out = np.empty(xx.shape, np.float64)
+    _load().rlcs_oracle_elig_trace_vec_beta(_p(xx, _F), _p(bb, _F), _p(d, _U), _p(out, _D), N, T, D)
     return out
 
 

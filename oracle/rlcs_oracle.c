@@ -249,6 +249,20 @@ void rlcs_oracle_elig_trace_vec(const float* x, const uint8_t* d, double* z, int
         }
 }
 
+/* Eligibility trace with a decay per component and step (per-dimension beta_t, Section 9.1): Eq. 1
+ * component by component, z_t[c] = x_t[c] + beta_t[c] * z_{t-1}[c], the carry severed after a flag. */
+void rlcs_oracle_elig_trace_vec_beta(const float* x, const float* beta, const uint8_t* d, double* z, int64_t N, int64_t T,
+                                     int64_t D) {
+    for (int64_t n = 0; n < N; ++n)
+        for (int64_t t = 0; t < T; ++t) {
+            const int carry = (t > 0) && !flag(d, n * T + t - 1);
+            for (int64_t c = 0; c < D; ++c) {
+                const int64_t i = (n * T + t) * D + c;
+                z[i] = carry ? (double)x[i] + (double)beta[i] * z[i - D] : (double)x[i];
+            }
+        }
+}
+
 /* Episodic prefix sum (Section 3.3.6), forward in time.  ends_at (default):
  * C_t = x_t + (1 - d_{t-1})*C_{t-1}; starts_at: C_t = x_t + (1 - d_t)*C_{t-1}.
  * C_{-1} = 0 in both, so C_0 = x_0 whatever d_0 is. */

@@ -37,6 +37,8 @@ SIGNATURES = {
     "rlcs_elig_trace": ([_vp] * 3 + [_i64, _i64, _f, _f] + _TAIL, _int),
     "rlcs_elig_trace_vec": ([_vp] * 3 + [_i64, _i64, _i64, _f, _f] + _TAIL, _int),
     "rlcs_elig_trace_vec_workspace_bytes": ([_i64, _i64, _i64], _sz),
+    "rlcs_elig_trace_vec_beta": ([_vp] * 4 + [_i64, _i64, _i64] + _TAIL, _int),
+    "rlcs_elig_trace_vec_beta_workspace_bytes": ([_i64, _i64, _i64], _sz),
     "rlcs_episodic_prefix_sum": ([_vp] * 3 + [_i64, _i64, _int] + _TAIL, _int),
     "rlcs_gae_no_alloc": ([_vp] * 8 + [_i64, _i64, _f, _f, _vp], _int),
     "rlcs_no_alloc_scratch_bytes": ([], _sz),
@@ -299,6 +301,19 @@ def rlcs_elig_trace_vec(x, dones, *, gamma, lam, traces=None, workspace=None, st
     wp, wb = _ws(workspace)
     _check(lib().rlcs_elig_trace_vec(_ptr(x, "f32"), _ptr(dones, "u8", (N, T)), _ptr(out, "f32", (N, T, D)), N, T, D,
                                      gamma, lam, wp, wb, _stream(stream)))
+    return out
+
+
+def rlcs_elig_trace_vec_beta(x, beta, dones, *, traces=None, workspace=None, stream=None):
+    """Eligibility trace with a decay per component and step: x, beta [N,T,D], dones [N,T]."""
+    N, T, D = x.shape
+    out = _out(x, traces)
+    if workspace is None:
+        nbytes = int(lib().rlcs_elig_trace_vec_beta_workspace_bytes(N, T, D))
+        workspace = Workspace(N, T, device=x.device, stream=stream, nbytes=nbytes) if nbytes else None
+    wp, wb = _ws(workspace)
+    _check(lib().rlcs_elig_trace_vec_beta(_ptr(x, "f32"), _ptr(beta, "f32", (N, T, D)), _ptr(dones, "u8", (N, T)),
+                                          _ptr(out, "f32", (N, T, D)), N, T, D, wp, wb, _stream(stream)))
     return out
 
 

@@ -1,5 +1,7 @@
 // Vector-valued eligibility traces: x, z of shape [N, T, D] (d innermost), one scalar decay per
-// step shared by all D components (Table 1, row "Elig. Traces", in its vector form).
+// step shared by all D components (Table 1, row "Elig. Traces", in its vector form), or -- PERDIM --
+// a decay per component and step read from a [N, T, D] tensor (the per-dimension beta that true
+// online TD(lambda) needs and Section 9.1 lists as unsupported by a scalar-beta kernel).
 //
 // The scan runs along T, which is the strided axis of this layout, so the mapping is the transpose of
 // the flat-tile kernels: a thread owns 4 (or 1) adjacent components d of one row n and walks the
@@ -19,7 +21,8 @@
 
 namespace {
 
-constexpr int kUnroll = 8;
+constexpr int kBatch = 8;         // steps loaded before the first FMA
+constexpr int kBatchPerDim = 4;   // ... with a decay tensor beside x (twice the registers per step)
 constexpr int kThreads = 256;
 
 struct VecParams {
@@ -32,8 +35,9 @@ struct VecParams {
     unsigned chunk;           // timesteps per chunk (== T when the time axis is not cut)
     unsigned chunks;          // chunks per row
     float decay;
+    const float* beta;        // PERDIM: [N, T, D] decays; beta[n, t, :] multiplies z_{t-1} into step t
     float* ends;              // [N, chunks, D]: pass 1 chunk-end vectors, then (in place) the carries into each chunk
-    float* prods;             // [N, chunks]: decay product of each chunk
+    float* prods;             // [N, chunks]: decay product of each chunk; PERDIM: [N, chunks, D]
 };
 
 template <int V> struct Vec;
@@ -44,8 +48,19 @@ template <> struct Vec<4> {
     __device__ void store(float* p) const { __stcs(reinterpret_cast<float4*>(p), v); }
     __device__ void plain_store(float* p) const { *reinterpret_cast<float4*>(p) = v; }
     __device__ static Vec zero() { Vec r; r.v = make_float4(0.f, 0.f, 0.f, 0.f); return r; }
+    __device__ static Vec splat(float f) { Vec r; r.v = make_float4(f, f, f, f); return r; }
     __device__ void fma(float b, const Vec& x) {     // this <- b * this + x
         v.x = fmaf(b, v.x, x.v.x); v.y = fmaf(b, v.y, x.v.y); v.z = fmaf(b, v.z, x.v.z); v.w = fmaf(b, v.w, x.v.w);
+    }
+    __device__ void fma(const Vec& b, const Vec& x) {     // this <- b * this + x, component by component
+        v.x = fmaf(b.v.x, v.x, x.v.x); v.y = fmaf(b.v.y, v.y, x.v.y); v.z = fmaf(b.v.z, v.z, x.v.z); v.w = fmaf(b.v.w, v.w, x.v.w);
+    }
+    __device__ void mul(const Vec& b) { v.x *= b.v.x; v.y *= b.v.y; v.z *= b.v.z; v.w *= b.v.w; }
+    // zero unless on; bitwise, so that a flag that differs between the rows of a warp cannot become a branch
+    __device__ void keep(bool on) {
+        const unsigned m = on ? ~0u : 0u;
+        v.x = __uint_as_float(__float_as_uint(v.x) & m); v.y = __uint_as_float(__float_as_uint(v.y) & m);
+        v.z = __uint_as_float(__float_as_uint(v.z) & m); v.w = __uint_as_float(__float_as_uint(v.w) & m);
     }
 };
 template <> struct Vec<1> {
@@ -55,12 +70,16 @@ template <> struct Vec<1> {
     __device__ void store(float* p) const { __stcs(p, v); }
     __device__ void plain_store(float* p) const { *p = v; }
     __device__ static Vec zero() { Vec r; r.v = 0.f; return r; }
+    __device__ static Vec splat(float f) { Vec r; r.v = f; return r; }
     __device__ void fma(float b, const Vec& x) { v = fmaf(b, v, x.v); }
+    __device__ void fma(const Vec& b, const Vec& x) { v = fmaf(b.v, v, x.v); }
+    __device__ void mul(const Vec& b) { v *= b.v; }
+    __device__ void keep(bool on) { v = __uint_as_float(__float_as_uint(v) & (on ? ~0u : 0u)); }
 };
 
 // MODE 0: whole rows, write traces.  MODE 1: chunk ends and decay products only.  MODE 2: rescan
 // from the carry and write traces.
-template <int V, int MODE>
+template <int V, int MODE, bool PERDIM>
 __global__ void __launch_bounds__(kThreads) elig_vec_kernel(const VecParams p) {
     const long long tid = (long long)blockIdx.x * kThreads + threadIdx.x;
     const long long per_row = (long long)p.groups * p.chunks;
@@ -75,53 +94,72 @@ __global__ void __launch_bounds__(kThreads) elig_vec_kernel(const VecParams p) {
     const float* __restrict__ x = p.x + (row * p.D + c);
     float* __restrict__ z = p.z + (row * p.D + c);
     const uint8_t* __restrict__ d = p.dones + row;
+    const float* __restrict__ bsrc = PERDIM ? p.beta + (row * p.D + c) : nullptr;
 
     Vec<V> acc = Vec<V>::zero();
     if (MODE == 2 && k > 0) acc = Vec<V>::plain(p.ends + ((n * p.chunks + k) * (long long)p.D + c));
-    float prod = 1.f;
-    for (unsigned t0 = t_begin; t0 < t_end; t0 += kUnroll) {
-        Vec<V> xs[kUnroll];
-        float beta[kUnroll];
+    float prod = 1.f;                          // decay product of the chunk (scalar decay)
+    Vec<V> prodv = Vec<V>::splat(1.f);         // ... per component (PERDIM)
+
+    // (A software pipeline of two alternating register batches was measured and is slower: 0.60
+    // against 0.89 of the copy bandwidth for the shared-decay kernel.)
+    constexpr int KB = PERDIM ? kBatchPerDim : kBatch;
+    for (unsigned t0 = t_begin; t0 < t_end; t0 += KB) {
+        Vec<V> xs[KB], bs[KB];
+        float beta[KB];
 #pragma unroll
-        for (int u = 0; u < kUnroll; ++u) {
+        for (int u = 0; u < KB; ++u) {
             const unsigned t = t0 + u;
             if (t < t_end) {
                 xs[u] = Vec<V>::load(x + (long long)t * p.D);
                 // the carry into step t is severed by the flag of step t-1 (and at the row's first step)
-                beta[u] = (t == 0 || __ldg(d + t - 1) != 0) ? 0.f : p.decay;
+                const bool cut = (t == 0 || __ldg(d + t - 1) != 0);
+                if constexpr (PERDIM) {
+                    bs[u] = Vec<V>::load(bsrc + (long long)t * p.D);
+                    bs[u].keep(!cut);
+                } else {
+                    beta[u] = cut ? 0.f : p.decay;
+                }
             }
         }
 #pragma unroll
-        for (int u = 0; u < kUnroll; ++u) {
+        for (int u = 0; u < KB; ++u) {
             const unsigned t = t0 + u;
             if (t < t_end) {
-                acc.fma(beta[u], xs[u]);
-                if (MODE == 1) prod *= beta[u];
-                else acc.store(z + (long long)t * p.D);
+                if constexpr (PERDIM) {
+                    acc.fma(bs[u], xs[u]);
+                    if (MODE == 1) prodv.mul(bs[u]);
+                } else {
+                    acc.fma(beta[u], xs[u]);
+                    if (MODE == 1) prod *= beta[u];
+                }
+                if (MODE != 1) acc.store(z + (long long)t * p.D);
             }
         }
     }
     if (MODE == 1) {
         acc.plain_store(p.ends + ((n * p.chunks + k) * (long long)p.D + c));
-        if (c == 0) p.prods[n * p.chunks + k] = prod;
+        if constexpr (PERDIM) prodv.plain_store(p.prods + ((n * p.chunks + k) * (long long)p.D + c));
+        else if (c == 0) p.prods[n * p.chunks + k] = prod;
     }
 }
 
 // Chain the chunks of each row: carry into chunk k = end_{k-1} + prod_{k-1} * carry into chunk k-1,
 // in order, one thread per (row, component group).  Overwrites ends[n][k] with the carry into chunk k.
-template <int V>
+template <int V, bool PERDIM>
 __global__ void __launch_bounds__(kThreads) elig_vec_chain_kernel(const VecParams p) {
     const long long tid = (long long)blockIdx.x * kThreads + threadIdx.x;
     const long long n = tid / p.groups;
     if (n >= p.N) return;
     const unsigned c = (unsigned)(tid - n * p.groups) * V;
     float* e = p.ends + (n * p.chunks * (long long)p.D + c);
-    const float* pr = p.prods + n * p.chunks;
+    const float* pr = PERDIM ? p.prods + (n * p.chunks * (long long)p.D + c) : p.prods + n * p.chunks;
     Vec<V> carry = Vec<V>::zero();
     for (unsigned k = 0; k < p.chunks; ++k) {
         const Vec<V> end_k = Vec<V>::plain(e + (long long)k * p.D);     // computed with carry 0
         carry.plain_store(e + (long long)k * p.D);                      // carry into chunk k
-        carry.fma(pr[k], end_k);                                        // carry into chunk k+1
+        if constexpr (PERDIM) carry.fma(Vec<V>::plain(pr + (long long)k * p.D), end_k);
+        else carry.fma(pr[k], end_k);                                   // carry into chunk k+1
     }
 }
 
@@ -129,7 +167,7 @@ inline bool aligned(const void* p, uintptr_t a) { return (reinterpret_cast<uintp
 
 // chunking: cut the time axis only when N * groups threads cannot fill the GPU
 void plan(long long N, long long T, long long groups, unsigned* chunk, unsigned* chunks) {
-    // One pass needs enough threads to keep the memory system busy: each holds kUnroll x 16 bytes in
+    // One pass needs enough threads to keep the memory system busy: each holds kBatch x 16 bytes in
     // flight, and ~40 K threads (5 MB) already saturate HBM; below that, cut -- but into chunks of
     // at least 128 steps and at most 256 per row, so that the ordered carry chain stays short.
     const long long want_threads = 148ll * 256;
@@ -138,32 +176,51 @@ void plan(long long N, long long T, long long groups, unsigned* chunk, unsigned*
     if (k > 256) k = 256;
     long long len = (T + k - 1) / k;
     if (len < 128) len = 128;
-    len = (len + kUnroll - 1) / kUnroll * kUnroll;
+    len = (len + kBatch - 1) / kBatch * kBatch;
     if (len >= T) { *chunk = (unsigned)T; *chunks = 1; return; }
     *chunk = (unsigned)len;
     *chunks = (unsigned)((T + len - 1) / len);
 }
 
-template <int V>
+template <int V, bool PERDIM>
 int run(VecParams p, cudaStream_t s) {
     const long long threads = p.N * (long long)p.groups * p.chunks;
     const unsigned blocks = (unsigned)((threads + kThreads - 1) / kThreads);
     if (p.chunks == 1) {
-        elig_vec_kernel<V, 0><<<blocks, kThreads, 0, s>>>(p);
+        elig_vec_kernel<V, 0, PERDIM><<<blocks, kThreads, 0, s>>>(p);
     } else {
-        elig_vec_kernel<V, 1><<<blocks, kThreads, 0, s>>>(p);
+        elig_vec_kernel<V, 1, PERDIM><<<blocks, kThreads, 0, s>>>(p);
         const long long chain_threads = p.N * (long long)p.groups;
-        elig_vec_chain_kernel<V><<<(unsigned)((chain_threads + kThreads - 1) / kThreads), kThreads, 0, s>>>(p);
-        elig_vec_kernel<V, 2><<<blocks, kThreads, 0, s>>>(p);
+        elig_vec_chain_kernel<V, PERDIM><<<(unsigned)((chain_threads + kThreads - 1) / kThreads), kThreads, 0, s>>>(p);
+        elig_vec_kernel<V, 2, PERDIM><<<blocks, kThreads, 0, s>>>(p);
     }
     return cudaGetLastError() == cudaSuccess ? RLCS_OK : RLCS_ERR_CUDA;
 }
 
-}  // namespace
+// sizes, pointers and chunking common to both entry points; *skip = nothing to do
+int prepare(VecParams& p, const float* x, const float* beta, bool perdim, const uint8_t* dones, float* traces, int64_t N,
+            int64_t T, int64_t D, void* workspace, size_t workspace_bytes, bool* v4, bool* skip) {
+    *skip = false;
+    if (N < 0 || T < 0 || D < 0 || T > (int64_t(1) << 31) - 1 || D > (int64_t(1) << 24)) return RLCS_ERR_SIZE;
+    if (N == 0 || T == 0 || D == 0) { *skip = true; return RLCS_OK; }
+    if (N > (int64_t(1) << 40) / T || N * T > (int64_t(1) << 40) / D) return RLCS_ERR_SIZE;
+    if (!x || !dones || !traces || (perdim && !beta)) return RLCS_ERR_NULL;
+    if (!aligned(x, 4) || !aligned(traces, 4) || (perdim && !aligned(beta, 4))) return RLCS_ERR_ALIGN;
+    *v4 = (D % 4 == 0) && aligned(x, 16) && aligned(traces, 16) && (!perdim || aligned(beta, 16));
+    p.x = x; p.beta = beta; p.dones = dones; p.z = traces; p.N = N; p.T = (unsigned)T; p.D = (unsigned)D;
+    p.groups = (unsigned)(*v4 ? D / 4 : D);
+    plan(N, T, p.groups, &p.chunk, &p.chunks);
+    if (p.chunks > 1) {
+        const size_t need = sizeof(float) * (size_t)N * p.chunks * ((size_t)D + (perdim ? (size_t)D : 1));
+        if (workspace == nullptr || workspace_bytes < need) return RLCS_ERR_WORKSPACE;
+        if (!aligned(workspace, 16)) return RLCS_ERR_ALIGN;
+        p.ends = static_cast<float*>(workspace);
+        p.prods = p.ends + (size_t)N * p.chunks * (size_t)D;
+    }
+    return RLCS_OK;
+}
 
-extern "C" {
-
-size_t rlcs_elig_trace_vec_workspace_bytes(int64_t N, int64_t T, int64_t D) {
+size_t workspace_bytes(int64_t N, int64_t T, int64_t D, bool perdim) {
     if (N <= 0 || T <= 0 || D <= 0 || T > (int64_t(1) << 31) - 1 || D > (int64_t(1) << 24)) return 0;
     unsigned chunk, chunks;
     plan(N, T, (D + 3) / 4, &chunk, &chunks);
@@ -171,32 +228,37 @@ size_t rlcs_elig_trace_vec_workspace_bytes(int64_t N, int64_t T, int64_t D) {
     plan(N, T, D, &chunk1, &chunks1);                         // the element-wise variant cuts differently
     const size_t k = chunks > chunks1 ? chunks : chunks1;
     if (k <= 1) return 0;
-    return sizeof(float) * (size_t)N * k * ((size_t)D + 1) + 256;
+    return sizeof(float) * (size_t)N * k * ((size_t)D + (perdim ? (size_t)D : 1)) + 256;
 }
+
+}  // namespace
+
+extern "C" {
+
+size_t rlcs_elig_trace_vec_workspace_bytes(int64_t N, int64_t T, int64_t D) { return workspace_bytes(N, T, D, false); }
+
+size_t rlcs_elig_trace_vec_beta_workspace_bytes(int64_t N, int64_t T, int64_t D) { return workspace_bytes(N, T, D, true); }
 
 int rlcs_elig_trace_vec(const float* x, const uint8_t* dones, float* traces, int64_t N, int64_t T, int64_t D,
                         float gamma, float lambda, void* workspace, size_t workspace_bytes, void* cuda_stream) {
     if (!(gamma >= 0.f && gamma <= 1.f) || !(lambda >= 0.f && lambda <= 1.f)) return RLCS_ERR_ARG;
-    if (N < 0 || T < 0 || D < 0 || T > (int64_t(1) << 31) - 1 || D > (int64_t(1) << 24)) return RLCS_ERR_SIZE;
-    if (N == 0 || T == 0 || D == 0) return RLCS_OK;
-    if (N > (int64_t(1) << 40) / T || N * T > (int64_t(1) << 40) / D) return RLCS_ERR_SIZE;
-    if (!x || !dones || !traces) return RLCS_ERR_NULL;
-    if (!aligned(x, 4) || !aligned(traces, 4)) return RLCS_ERR_ALIGN;
-    const bool v4 = (D % 4 == 0) && aligned(x, 16) && aligned(traces, 16);
     VecParams p = {};
-    p.x = x; p.dones = dones; p.z = traces; p.N = N; p.T = (unsigned)T; p.D = (unsigned)D;
-    p.groups = (unsigned)(v4 ? D / 4 : D);
+    bool v4 = false, skip = false;
+    const int st = prepare(p, x, nullptr, false, dones, traces, N, T, D, workspace, workspace_bytes, &v4, &skip);
+    if (st != RLCS_OK || skip) return st;
     p.decay = gamma * lambda;
-    plan(N, T, p.groups, &p.chunk, &p.chunks);
-    if (p.chunks > 1) {
-        const size_t need = sizeof(float) * (size_t)N * p.chunks * ((size_t)D + 1);
-        if (workspace == nullptr || workspace_bytes < need) return RLCS_ERR_WORKSPACE;
-        if (!aligned(workspace, 16)) return RLCS_ERR_ALIGN;
-        p.ends = static_cast<float*>(workspace);
-        p.prods = p.ends + (size_t)N * p.chunks * (size_t)D;
-    }
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
-    return v4 ? run<4>(p, s) : run<1>(p, s);
+    return v4 ? run<4, false>(p, s) : run<1, false>(p, s);
+}
+
+int rlcs_elig_trace_vec_beta(const float* x, const float* beta, const uint8_t* dones, float* traces, int64_t N, int64_t T,
+                             int64_t D, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    VecParams p = {};
+    bool v4 = false, skip = false;
+    const int st = prepare(p, x, beta, true, dones, traces, N, T, D, workspace, workspace_bytes, &v4, &skip);
+    if (st != RLCS_OK || skip) return st;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    return v4 ? run<4, true>(p, s) : run<1, true>(p, s);
 }
 
 }  // extern "C"

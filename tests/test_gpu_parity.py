@@ -491,6 +491,39 @@ def test_vector_trace_argument_checks(oracle, W, B):
     assert L.rlcs_elig_trace_vec(P, P, P, 2, 100000, 8, 0.9, 0.9, None, 0, None) == B.RLCS_ERR_WORKSPACE
 
 
+@pytest.mark.parametrize("N,T,D", [(1, 1, 1), (3, 7, 5), (8, 128, 64), (64, 257, 16), (4096, 40, 8), (2, 5000, 128),
+                                    (3, 16384, 32), (5, 999, 3)])
+def test_per_dimension_beta_eligibility_trace(oracle, W, B, N, T, D):
+    import torch
+    rng = np.random.default_rng(N * 7919 + T * 31 + D + 1)
+    x = rng.standard_normal((N, T, D)).astype(np.float32)
+    beta = rng.uniform(0.5, 1.0, (N, T, D)).astype(np.float32)
+    d = (rng.random((N, T)) < 0.02).astype(np.uint8)
+    d[:, 0] = rng.integers(0, 2, N)
+    xd, bd, dd = torch.from_numpy(x).cuda(), torch.from_numpy(beta).cuda(), torch.from_numpy(d).cuda()
+    ref = oracle.elig_trace_vec_beta(x, beta, d)
+    got = B.rlcs_elig_trace_vec_beta(xd, bd, dd).cpu().numpy()
+    assert_close(f"per-dimension trace {N}x{T}x{D}", got, ref)
+    # pointers off 16-byte alignment: element-wise variant
+    off = lambda t: torch.cat([t.new_zeros(1), t.reshape(-1)])[1:].view(t.shape)
+    got1 = B.rlcs_elig_trace_vec_beta(off(xd), off(bd), dd).cpu().numpy()
+    assert_close("per-dimension trace, unaligned", got1, ref)
+    # a constant beta is the shared-scalar entry point, bit for bit (same FMA per step, same chunking)
+    const = torch.full_like(xd, 0.25)
+    same = B.rlcs_elig_trace_vec_beta(xd, const, dd)
+    assert torch.equal(same, B.rlcs_elig_trace_vec(xd, dd, gamma=0.5, lam=0.5))
+
+
+def test_per_dimension_beta_argument_checks(oracle, W, B):
+    L = B.lib()
+    P = 0x7f0000000000
+    assert L.rlcs_elig_trace_vec_beta(P, P, P, P, 4, 8, 0, None, 0, None) == B.RLCS_OK
+    assert L.rlcs_elig_trace_vec_beta(P, None, P, P, 4, 8, 4, None, 0, None) == B.RLCS_ERR_NULL
+    assert L.rlcs_elig_trace_vec_beta(P, P + 2, P, P, 4, 8, 4, None, 0, None) == B.RLCS_ERR_ALIGN
+    assert L.rlcs_elig_trace_vec_beta_workspace_bytes(2, 100000, 8) > L.rlcs_elig_trace_vec_workspace_bytes(2, 100000, 8)
+    assert L.rlcs_elig_trace_vec_beta(P, P, P, P, 2, 100000, 8, None, 0, None) == B.RLCS_ERR_WORKSPACE
+
+
 # ------------------------------------------------------------------ time-major [T, N] entry points
 def _tm(a):
     import torch

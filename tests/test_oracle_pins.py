@@ -673,3 +673,30 @@ def test_vector_trace_is_one_scalar_trace_per_component(oracle):
     w = 0.5 ** np.arange(T)
     want = np.stack([[np.convolve(x[n, :, c].astype(float), w)[:T] for c in range(D)] for n in range(N)]).transpose(0, 2, 1)
     np.testing.assert_allclose(z0, want, rtol=1e-12, atol=1e-12)
+
+
+def test_per_dimension_beta_trace_against_the_unrolled_sum(oracle):
+    """Eq. 1 unrolled: z_t[c] = sum_k x_k[c] * prod_{s=k+1..t} b_s[c] with b_s = beta_s where the carry into
+    s survives and 0 where the flag of step s-1 severs it -- written out with explicit products, no
+    recurrence.  Then the special cases: a constant beta reproduces the shared-scalar trace exactly,
+    and each component is the generic forward recurrence on its own coefficients."""
+    rng = np.random.default_rng(61)
+    N, T, D = 2, 12, 3
+    x = rng.standard_normal((N, T, D)).astype(np.float32)
+    beta = rng.uniform(0.2, 1.1, (N, T, D)).astype(np.float32)
+    d = (rng.random((N, T)) < 0.2).astype(np.uint8)
+    z = oracle.elig_trace_vec_beta(x, beta, d)
+    for n in range(N):
+        for c in range(D):
+            b = [0.0] + [0.0 if d[n, s - 1] else float(beta[n, s, c]) for s in range(1, T)]
+            for t in range(T):
+                want = sum(float(x[n, k, c]) * float(np.prod(b[k + 1:t + 1])) for k in range(t + 1))
+                assert abs(z[n, t, c] - want) <= 1e-12 * (1 + abs(want)), (n, t, c)
+            rec = oracle.linear_recurrence(x[n, :, c].astype(np.float64), np.array(b), 0.0, forward=True)
+            np.testing.assert_allclose(z[n, :, c], rec, rtol=1e-13, atol=1e-13)
+    const = np.full((N, T, D), 0.25, np.float32)                      # gamma * lambda = 0.5 * 0.5, exact in fp32
+    assert np.array_equal(oracle.elig_trace_vec_beta(x, const, d), oracle.elig_trace_vec(x, d, gamma=0.5, lam=0.5))
+    # beta at t = 0 is never read
+    beta2 = beta.copy()
+    beta2[:, 0, :] = np.nan
+    assert np.array_equal(oracle.elig_trace_vec_beta(x, beta2, d), z)
