@@ -393,8 +393,9 @@ int rlcs_debug_set_carry_fault(int64_t mute_tile, int64_t spin_cap);
 
 /*
  * Test hook: path of the time-major entry points for subsequent calls in this process.  1 = the
- * register walk whatever the alignment, any other value = the shared-memory ring wherever N and
- * the pointers allow it (the default).  Results must be identical (same arithmetic, same order).
+ * register walk whatever the alignment; 3 = the shared-memory ring with one column per lane whatever
+ * the size; any other value = the default (the ring wherever N and the pointers allow it, two
+ * columns per lane for large N).  Results must agree to rounding.
  */
 void rlcs_debug_time_major_path(int path);
 

@@ -59,7 +59,7 @@ struct TmParams {
     unsigned chunk, chunks;   // timesteps per chunk, chunks per environment (1 = time axis not cut)
     float gamma, decay, aux, rho_bar, c_bar;
     int starts_at;
-    int stages, warps_per_block;   // tm_block_kernel: ring depth and warps per thread block
+    int stages, warps_per_block, cols_per_lane;   // tm_block_kernel: ring depth, warps per block, columns per lane
     float* agg_a;             // [chunks, N] pass 1: chunk aggregates; after the chain: carry into each chunk
     float* agg_b;             // [chunks, N]
 };
@@ -381,26 +381,44 @@ __device__ __forceinline__ void cp_async_wait(int pending) {
 constexpr int kMaxStages = 16;
 constexpr int kMaxWarps = 8;
 
-// One stage of a thread block: R = kRows * warps rows of its 32 columns, row index = scan-order step
-// within the stage.  Floats and masks live in separate rings (the mask ring runs two stages ahead):
-// float tensor a at fbase[a][row][32 floats], mask tensor m at mbase[m][row][32 bytes].
-template <int ALGO, bool TRUNC, int W>
+// One stage of a thread block: R = kRows * warps rows of its 32 C columns (C columns per lane), row
+// index = scan-order step within the stage.  Floats and masks live in separate rings (the mask ring
+// runs two stages ahead): float tensor a at fbase[a][row][32 C floats], mask tensor m at
+// mbase[m][row][32 C bytes].
+template <int ALGO, bool TRUNC, int W, int C>
 struct StageView {
     static constexpr int NF = tm_nf(ALGO);
     static constexpr int NM = TRUNC ? 2 : 1;
     static constexpr int R = kRows * W;
     unsigned char* fbase;
     unsigned char* mbase;
-    __device__ __forceinline__ float* f(int a, int row) const { return reinterpret_cast<float*>(fbase + (a * R + row) * 128); }
-    __device__ __forceinline__ uint8_t* m(int a, int row) const { return mbase + (a * R + row) * 32; }
+    __device__ __forceinline__ float* f(int a, int row) const { return reinterpret_cast<float*>(fbase + (a * R + row) * (128 * C)); }
+    __device__ __forceinline__ uint8_t* m(int a, int row) const { return mbase + (a * R + row) * (32 * C); }
 };
 
-// Per-thread bookkeeping for the copies of a stage.  Every float tensor has 8 R 16-byte pieces per
-// stage, two per thread (rows frow and frow + 4 W, piece = tid & 7); every mask tensor 2 R, one for
-// each of the first half of the threads.  Rows past the chunk and pieces past column N are
-// zero-filled (N is a multiple of 16 here, so a piece is never split by the edge).
+// A lane's C adjacent values of one row
+template <int C>
+__device__ __forceinline__ void lds_f(const float* row, int lane, float (&x)[C]) {
+    if constexpr (C == 2) { const float2 v = *reinterpret_cast<const float2*>(row + 2 * lane); x[0] = v.x; x[1] = v.y; }
+    else x[0] = row[lane];
+}
+template <int C>
+__device__ __forceinline__ void lds_m(const uint8_t* row, int lane, unsigned (&x)[C]) {
+    if constexpr (C == 2) { const unsigned v = *reinterpret_cast<const unsigned short*>(row + 2 * lane); x[0] = v & 0xffu; x[1] = v >> 8; }
+    else x[0] = row[lane];
+}
+template <int C>
+__device__ __forceinline__ void stg_f(float* p, const float (&x)[C]) {
+    if constexpr (C == 2) __stcs(reinterpret_cast<float2*>(p), make_float2(x[0], x[1]));
+    else __stcs(p, x[0]);
+}
+
+// Per-thread bookkeeping for the copies of a stage.  A row of a float tensor is 8 C 16-byte pieces,
+// a row of a mask tensor 2 C; a thread moves the same piece of 2 C float rows and of one mask row
+// per stage.  Rows past the chunk and pieces past column N are zero-filled (N is a multiple of 16
+// here, so a piece is never split by the edge).
 struct CopyPlan {
-    long long i_first;     // flat index of the chunk's scan-order step 0, column n0
+    long long i_first;     // flat index of the chunk's scan-order step 0, first column of the block
     long long rowstep;     // flat-index step between scan-order neighbours: +N forward, -N backward
     unsigned len;          // steps in the chunk
     int frow, fcol;        // first float row of this thread, column offset of its piece
@@ -409,14 +427,14 @@ struct CopyPlan {
     bool m_on;
 };
 
-template <int ALGO, bool TRUNC, int W>
-__device__ __forceinline__ void issue_floats(const StageView<ALGO, TRUNC, W>& sv, const TmParams& p, const CopyPlan& cp, unsigned s) {
+template <int ALGO, bool TRUNC, int W, int C>
+__device__ __forceinline__ void issue_floats(const StageView<ALGO, TRUNC, W, C>& sv, const TmParams& p, const CopyPlan& cp, unsigned s) {
     constexpr int R = kRows * W;
     const float* const fsrc[4] = {p.f0, p.f1, p.f2, p.f3};
     constexpr int fidx[4] = {0, 1, (ALGO == kVtrace) ? 3 : 2, 3};   // V-trace stages f0, f1, f3
 #pragma unroll
-    for (int h = 0; h < 2; ++h) {
-        const int row = cp.frow + h * 4 * W;
+    for (int h = 0; h < 2 * C; ++h) {
+        const int row = cp.frow + h * (4 * W / C);
         const unsigned q = s * R + row;
         const bool ok = cp.fcol_ok && q < cp.len;
         const long long off = ok ? cp.i_first + cp.rowstep * q + cp.fcol : 0;
@@ -426,8 +444,8 @@ __device__ __forceinline__ void issue_floats(const StageView<ALGO, TRUNC, W>& sv
     }
 }
 
-template <int ALGO, bool TRUNC, int W>
-__device__ __forceinline__ void issue_masks(const StageView<ALGO, TRUNC, W>& sv, const TmParams& p, const CopyPlan& cp, unsigned s) {
+template <int ALGO, bool TRUNC, int W, int C>
+__device__ __forceinline__ void issue_masks(const StageView<ALGO, TRUNC, W, C>& sv, const TmParams& p, const CopyPlan& cp, unsigned s) {
     if (cp.m_on) {
         const unsigned q = s * (kRows * W) + cp.mrow;
         const bool ok = q < cp.len;
@@ -438,87 +456,97 @@ __device__ __forceinline__ void issue_masks(const StageView<ALGO, TRUNC, W>& sv,
 }
 
 // truncation continuation values of `nvalid` rows from row0 of a stage whose masks have landed;
-// i = flat index of the first of them for this lane
-template <int ALGO, bool TRUNC, int W>
-__device__ __forceinline__ void stage_bv(float (&bv)[kRows], const StageView<ALGO, TRUNC, W>& sv, const TmParams& p, long long i,
-                                         long long rowstep, int row0, int nvalid, int lane, unsigned write_mask) {
+// i = flat index of the first of them for this lane's first column
+template <int ALGO, bool TRUNC, int W, int C>
+__device__ __forceinline__ void stage_bv(float (&bv)[kRows][C], const StageView<ALGO, TRUNC, W, C>& sv, const TmParams& p,
+                                         long long i, long long rowstep, int row0, int nvalid, int lane, unsigned write_mask) {
     if (nvalid <= 0) return;                                 // past the chunk: the values are never used
-    if (nvalid >= kRows) {
+    auto rows = [&](auto full) {
+        constexpr bool FULL = decltype(full)::value;
 #pragma unroll
         for (int u = 0; u < kRows; ++u) {
-            const unsigned tr = sv.m(1, row0 + u)[lane], dn = sv.m(0, row0 + u)[lane];
-            bv[u] = ldg_if_mask(p.trunc_boot + i, ones_if(tr) & ~ones_if(dn) & write_mask);
-            i += rowstep;
-        }
-    } else {
+            unsigned tr[C], dn[C];
+            lds_m<C>(sv.m(1, row0 + u), lane, tr);
+            lds_m<C>(sv.m(0, row0 + u), lane, dn);
+            const unsigned rowmask = FULL ? write_mask : (write_mask & (u < nvalid ? ~0u : 0u));
 #pragma unroll
-        for (int u = 0; u < kRows; ++u) {
-            const unsigned tr = sv.m(1, row0 + u)[lane], dn = sv.m(0, row0 + u)[lane];
-            bv[u] = ldg_if_mask(p.trunc_boot + i, ones_if(tr) & ~ones_if(dn) & write_mask & (u < nvalid ? ~0u : 0u));
+            for (int c = 0; c < C; ++c) bv[u][c] = ldg_if_mask(p.trunc_boot + i + c, ones_if(tr[c]) & ~ones_if(dn[c]) & rowmask);
             i += rowstep;
         }
-    }
+    };
+    if (nvalid >= kRows) rows(std::true_type{});
+    else rows(std::false_type{});
 }
 
 __device__ __forceinline__ int wrap_next(int x, int n) { return x + 1 == n ? 0 : x + 1; }
 __device__ __forceinline__ int wrap_prev(int x, int n) { return x == 0 ? n - 1 : x - 1; }
 
-// A thread block owns 32 adjacent environments; its W warps split every stage of R = kRows * W
-// timesteps in time.  Per stage: each warp walks its kRows steps from carry 0, keeping per step the
-// value so far and the running product of betas (the step's affine map of the incoming carry,
-// Eq. 2); the W per-warp aggregates go through shared memory; every warp folds them in scan order
-// onto the block's carry (a few FMAs, redundantly in each warp) to get its own incoming carry, and
-// finishes its steps with one FMA each.  The inputs cross HBM once however the time axis is split.
+// A thread block owns 32 C adjacent environments (a lane C of them: with C = 2 every shared-memory
+// read, store and address computation serves two steps); its W warps split every stage of
+// R = kRows * W timesteps in time.  Per stage: each warp walks its kRows steps from carry 0, keeping
+// per step the value so far and the running product of betas (the step's affine map of the incoming
+// carry, Eq. 2); the W per-warp aggregates go through shared memory; every warp folds them in scan
+// order onto the block's carry (a few FMAs, redundantly in each warp) to get its own incoming
+// carry, and finishes its steps with one FMA each.  The inputs cross HBM once however the time
+// axis is split.
 //
 // Copies are committed in groups {floats of stage s, masks of stage s+2}: when a stage's floats
 // have landed so have the masks two stages on, and the sparse truncation values they point at are
 // requested two stages before their use (registers bv1, bv2).
 // MODE as in tm_kernel.
-template <int ALGO, bool TRUNC, int MODE, int W>
+template <int ALGO, bool TRUNC, int MODE, int W, int C>
 __global__ void __launch_bounds__(32 * W) tm_block_kernel(const TmParams p) {
     constexpr bool FWD = tm_forward(ALGO);
-    using SV = StageView<ALGO, TRUNC, W>;
+    using SV = StageView<ALGO, TRUNC, W, C>;
     extern __shared__ __align__(16) unsigned char tm_smem[];
     const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
     constexpr int R = kRows * W;
     const int S = p.stages, SM = S + 2;
-    constexpr int fstage = R * SV::NF * 128, mstage = R * SV::NM * 32;
+    constexpr int fstage = R * SV::NF * 128 * C, mstage = R * SV::NM * 32 * C;
     unsigned char* const mring = tm_smem + (size_t)S * fstage;
-    float2* const agg = reinterpret_cast<float2*>(mring + (size_t)SM * mstage);         // [2][W][32]
-    float* const edge_v = reinterpret_cast<float*>(agg + 2 * W * 32);                   // [2][32]
-    float* const edge_x = edge_v + 64;                                                  // [2][32] log-ratio | dones flag
+    float2* const agg = reinterpret_cast<float2*>(mring + (size_t)SM * mstage);         // [2][W][32 C]
+    float* const edge_v = reinterpret_cast<float*>(agg + 2 * W * 32 * C);               // [2][32 C]
+    float* const edge_x = edge_v + 64 * C;                                              // [2][32 C] log-ratio | dones flag
 
-    const long long n0 = (long long)blockIdx.x * 32;
-    const bool write = n0 + lane < p.N;                      // lanes past N read zero-filled columns
+    const long long n0 = (long long)blockIdx.x * (32 * C);
+    const bool write = n0 + C * lane < p.N;                  // lanes past N read zero-filled columns (N is even)
     const unsigned write_mask = write ? ~0u : 0u;
-    const long long n = write ? n0 + lane : p.N - 1;
     const unsigned k = blockIdx.y;
     const unsigned t_lo = k * p.chunk;
     const unsigned t_hi = min(p.T, t_lo + p.chunk);
     const unsigned len = t_hi - t_lo;
     const unsigned nst = (len + R - 1) / R;
-    const float bootv = (!FWD && p.boot != nullptr) ? __ldg(p.boot + n) : 0.f;
     const unsigned edge_last = (!FWD && t_hi == p.T) ? ~0u : 0u;   // the chunk's first step in scan order is t = T-1
 
     CopyPlan cp;
     cp.rowstep = FWD ? p.N : -p.N;
     cp.i_first = (long long)(FWD ? t_lo : t_hi - 1) * p.N + n0;
     cp.len = len;
-    cp.frow = tid >> 3; cp.fcol = 4 * (tid & 7); cp.fcol_ok = n0 + cp.fcol < p.N;
-    cp.mrow = tid >> 1; cp.mcol = 16 * (tid & 1); cp.m_on = tid < 2 * R && n0 + cp.mcol < p.N;
+    cp.frow = tid / (8 * C); cp.fcol = 4 * (tid % (8 * C)); cp.fcol_ok = n0 + cp.fcol < p.N;
+    cp.mrow = tid / (2 * C); cp.mcol = 16 * (tid % (2 * C)); cp.m_on = n0 + cp.mcol < p.N;
 
-    // block state: the affine map of everything walked so far applied to the chunk's incoming carry
-    float A = MODE == 2 ? p.agg_a[(long long)k * p.N + n] : 0.f;
-    float P = 1.f;
+    // block state per column: the affine map of everything walked so far applied to the chunk's incoming carry;
     // neighbours across the chunk's scan-order start
-    BackState b0 = {};
-    FwdState f0 = {};
-    if constexpr (FWD) init_fwd(f0, p, n, t_lo, 0.f);
-    else init_back<ALGO>(b0, p, n, t_hi, 0.f);
+    float A[C], P[C], bootv[C], v0[C], lr0[C];
+    unsigned d0[C];
+#pragma unroll
+    for (int c = 0; c < C; ++c) {
+        const long long n = write ? n0 + C * lane + c : p.N - 1;
+        A[c] = MODE == 2 ? p.agg_a[(long long)k * p.N + n] : 0.f;
+        P[c] = 1.f;
+        bootv[c] = (!FWD && p.boot != nullptr) ? __ldg(p.boot + n) : 0.f;
+        BackState b0 = {};
+        FwdState f0 = {};
+        if constexpr (FWD) init_fwd(f0, p, n, t_lo, 0.f);
+        else init_back<ALGO>(b0, p, n, t_hi, 0.f);
+        v0[c] = b0.v_next; lr0[c] = b0.lr_next; d0[c] = f0.d_prev;
+    }
 
     // A group is committed for every stage index, empty past the end, so that "all but the newest P
     // groups" always names the same stages.  Floats of stage s sit in slot s mod S, masks in slot
-    // s mod (S + 2).
+    // s mod (S + 2).  With C = 1 only the first half of the threads has a mask piece.
+    const bool mask_thread = C == 2 || tid < 2 * R;
+    cp.m_on = cp.m_on && mask_thread;
     for (int s = 0; s + 1 < S; ++s) {
         if (s == 0) {
             if (0 < nst) issue_masks<ALGO, TRUNC>(SV{nullptr, mring}, p, cp, 0);
@@ -528,12 +556,14 @@ __global__ void __launch_bounds__(32 * W) tm_block_kernel(const TmParams p) {
         if ((unsigned)s + 2 < nst) issue_masks<ALGO, TRUNC>(SV{nullptr, mring + (s + 2) * mstage}, p, cp, s + 2);
         cp_async_commit();
     }
-    float bvc[kRows], bv1[kRows], bv2[kRows];
+    float bvc[kRows][C], bv1[kRows][C], bv2[kRows][C];
 #pragma unroll
-    for (int u = 0; u < kRows; ++u) bvc[u] = bv1[u] = bv2[u] = 0.f;
+    for (int u = 0; u < kRows; ++u)
+#pragma unroll
+        for (int c = 0; c < C; ++c) bvc[u][c] = bv1[u][c] = bv2[u][c] = 0.f;
     const int row0 = kRows * w;
-    // this lane's flat index at its first row of the current stage, and rows it has there
-    long long iw = cp.i_first + cp.rowstep * row0 + lane;
+    // this lane's flat index (first column) at its first row of the current stage, and rows it has there
+    long long iw = cp.i_first + cp.rowstep * row0 + C * lane;
     int left = (int)len - row0;                              // steps from this warp's first row to the chunk's end
     const long long stagestep = cp.rowstep * R;
     if constexpr (TRUNC) {
@@ -556,89 +586,134 @@ __global__ void __launch_bounds__(32 * W) tm_block_kernel(const TmParams p) {
         }
         // neighbour of this warp's first step: the row before it in the stage, the last row of the
         // previous stage, or the chunk's outside neighbour
-        float v_next = 0.f, lr_next = 0.f;
-        unsigned d_prev = 0;
+        float v_next[C], lr_next[C];
+        unsigned d_prev[C];
+#pragma unroll
+        for (int c = 0; c < C; ++c) { v_next[c] = 0.f; lr_next[c] = 0.f; d_prev[c] = 0; }
         if (w > 0) {
-            if constexpr (FWD) d_prev = cur.m(0, row0 - 1)[lane];
-            else if constexpr (ALGO == kRetrace) { v_next = cur.f(2, row0 - 1)[lane]; lr_next = cur.f(3, row0 - 1)[lane]; }
-            else if constexpr (SV::NF >= 2) v_next = cur.f(1, row0 - 1)[lane];
+            if constexpr (FWD) lds_m<C>(cur.m(0, row0 - 1), lane, d_prev);
+            else if constexpr (ALGO == kRetrace) { lds_f<C>(cur.f(2, row0 - 1), lane, v_next); lds_f<C>(cur.f(3, row0 - 1), lane, lr_next); }
+            else if constexpr (SV::NF >= 2) lds_f<C>(cur.f(1, row0 - 1), lane, v_next);
         } else if (j > 0) {
-            if constexpr (FWD) d_prev = __float_as_uint(edge_x[(par ^ 1) * 32 + lane]);
-            else { v_next = edge_v[(par ^ 1) * 32 + lane]; lr_next = edge_x[(par ^ 1) * 32 + lane]; }
+            float t[C];
+            if constexpr (FWD) {
+                lds_f<C>(edge_x + (par ^ 1) * 32 * C, lane, t);
+#pragma unroll
+                for (int c = 0; c < C; ++c) d_prev[c] = __float_as_uint(t[c]);
+            } else {
+                lds_f<C>(edge_v + (par ^ 1) * 32 * C, lane, v_next);
+                lds_f<C>(edge_x + (par ^ 1) * 32 * C, lane, lr_next);
+            }
         } else {
-            v_next = b0.v_next; lr_next = b0.lr_next; d_prev = f0.d_prev;
+#pragma unroll
+            for (int c = 0; c < C; ++c) { v_next[c] = v0[c]; lr_next[c] = lr0[c]; d_prev[c] = d0[c]; }
         }
         // pass 1: from carry 0
-        float val0[kRows], pb[kRows], v1[kRows], pgc[kRows], alp[kRows];
-        float carry = 0.f, prod = 1.f;
+        float val0[kRows][C], pb[kRows][C], v1[kRows][C], pgc[kRows][C], alp[kRows][C];
+        float carry[C], prod[C];
+#pragma unroll
+        for (int c = 0; c < C; ++c) { carry[c] = 0.f; prod[c] = 1.f; }
         // the per-row guards exist only in the instance that the chunk's ragged last stage takes
         auto pass1 = [&](auto full) {
-        constexpr bool FULL = decltype(full)::value;
+            constexpr bool FULL = decltype(full)::value;
 #pragma unroll
-        for (int u = 0; u < kRows; ++u) {
-            v1[u] = 0.f; pgc[u] = 0.f; alp[u] = 0.f;
-            if (FULL || u < nvalid) {
-                Coef c;
-                if constexpr (FWD) {
-                    const unsigned d = cur.m(0, row0 + u)[lane];
-                    c = fwd_coef<ALGO>(cur.f(0, row0 + u)[lane], d, d_prev, p, (u == 0 && w == 0 && j == 0) ? t_lo : 1u);
-                    d_prev = d;
-                } else {
-                    StepIn in;
-                    in.r = cur.f(0, row0 + u)[lane];
-                    in.v1 = SV::NF >= 2 ? cur.f(1, row0 + u)[lane] : 0.f;
-                    in.v2 = ALGO == kRetrace ? cur.f(2, row0 + u)[lane] : 0.f;
-                    in.v3 = ALGO == kRetrace ? cur.f(3, row0 + u)[lane] : ALGO == kVtrace ? cur.f(2, row0 + u)[lane] : 0.f;
-                    in.dn = cur.m(0, row0 + u)[lane];
-                    in.tr = TRUNC ? cur.m(1, row0 + u)[lane] : 0u;
-                    in.bv = bvc[u];
-                    // only the block's very first row can be the window's final step
-                    const unsigned last = (u == 0 && w == 0 && j == 0) ? edge_last : 0u;
-                    c = back_coef<ALGO, TRUNC>(in, p, last, bootv, v_next, lr_next);
-                    v_next = ALGO == kRetrace ? in.v2 : in.v1;
-                    lr_next = in.v3;
-                    v1[u] = in.v1;
+            for (int u = 0; u < kRows; ++u) {
+#pragma unroll
+                for (int c = 0; c < C; ++c) { v1[u][c] = 0.f; pgc[u][c] = 0.f; alp[u][c] = 0.f; }
+                if (FULL || u < nvalid) {
+                    float r[C], x1[C], x2[C], x3[C];
+                    unsigned dn[C], tr[C];
+                    lds_f<C>(cur.f(0, row0 + u), lane, r);
+                    lds_m<C>(cur.m(0, row0 + u), lane, dn);
+                    if constexpr (!FWD) {
+                        if constexpr (SV::NF >= 2) lds_f<C>(cur.f(1, row0 + u), lane, x1);
+                        if constexpr (ALGO == kRetrace) { lds_f<C>(cur.f(2, row0 + u), lane, x2); lds_f<C>(cur.f(3, row0 + u), lane, x3); }
+                        if constexpr (ALGO == kVtrace) lds_f<C>(cur.f(2, row0 + u), lane, x3);
+                        if constexpr (TRUNC) lds_m<C>(cur.m(1, row0 + u), lane, tr);
+                    }
+#pragma unroll
+                    for (int c = 0; c < C; ++c) {
+                        Coef co;
+                        if constexpr (FWD) {
+                            co = fwd_coef<ALGO>(r[c], dn[c], d_prev[c], p, (u == 0 && w == 0 && j == 0) ? t_lo : 1u);
+                            d_prev[c] = dn[c];
+                        } else {
+                            StepIn in;
+                            in.r = r[c];
+                            in.v1 = SV::NF >= 2 ? x1[c] : 0.f;
+                            in.v2 = ALGO == kRetrace ? x2[c] : 0.f;
+                            in.v3 = (ALGO == kRetrace || ALGO == kVtrace) ? x3[c] : 0.f;
+                            in.dn = dn[c];
+                            in.tr = TRUNC ? tr[c] : 0u;
+                            in.bv = bvc[u][c];
+                            // only the block's very first row can be the window's final step
+                            const unsigned last = (u == 0 && w == 0 && j == 0) ? edge_last : 0u;
+                            co = back_coef<ALGO, TRUNC>(in, p, last, bootv[c], v_next[c], lr_next[c]);
+                            v_next[c] = ALGO == kRetrace ? in.v2 : in.v1;
+                            lr_next[c] = in.v3;
+                            v1[u][c] = in.v1;
+                        }
+                        carry[c] = fmaf(co.beta, carry[c], co.alpha);
+                        prod[c] *= co.beta;
+                        pgc[u][c] = co.pg;
+                        alp[u][c] = co.alpha;
+                    }
                 }
-                carry = fmaf(c.beta, carry, c.alpha);
-                prod *= c.beta;
-                pgc[u] = c.pg;
-                alp[u] = c.alpha;
+#pragma unroll
+                for (int c = 0; c < C; ++c) { val0[u][c] = carry[c]; pb[u][c] = prod[c]; }
             }
-            val0[u] = carry;
-            pb[u] = prod;
-        }
         };
         if (nvalid == kRows) pass1(std::true_type{});
         else pass1(std::false_type{});
-        agg[(par * W + w) * 32 + lane] = make_float2(carry, prod);
+#pragma unroll
+        for (int c = 0; c < C; ++c) agg[((par * W + w) * 32 + lane) * C + c] = make_float2(carry[c], prod[c]);
         if (w == W - 1) {                                    // neighbours for the next stage's first warp
-            if constexpr (FWD) edge_x[par * 32 + lane] = __uint_as_float(d_prev);
-            else { edge_v[par * 32 + lane] = v_next; edge_x[par * 32 + lane] = lr_next; }
+#pragma unroll
+            for (int c = 0; c < C; ++c) {
+                if constexpr (FWD) edge_x[par * 32 * C + C * lane + c] = __uint_as_float(d_prev[c]);
+                else { edge_v[par * 32 * C + C * lane + c] = v_next[c]; edge_x[par * 32 * C + C * lane + c] = lr_next[c]; }
+            }
         }
         __syncthreads();
         // fold the warps' aggregates in scan order onto the block state
-        float cin = A;
+        float cin[C];
+#pragma unroll
+        for (int c = 0; c < C; ++c) cin[c] = A[c];
 #pragma unroll
         for (int x = 0; x < W; ++x) {
-            const float2 ab = agg[(par * W + x) * 32 + lane];
-            if (x == w) cin = A;
-            A = fmaf(ab.y, A, ab.x);
-            P *= ab.y;
+#pragma unroll
+            for (int c = 0; c < C; ++c) {
+                const float2 ab = agg[((par * W + x) * 32 + lane) * C + c];
+                if (x == w) cin[c] = A[c];
+                A[c] = fmaf(ab.y, A[c], ab.x);
+                P[c] *= ab.y;
+            }
         }
         // pass 2: one FMA per step, then the outputs
         if (MODE != 1) {
             auto pass2 = [&](auto full) {
                 constexpr bool FULL = decltype(full)::value;
-                float prev = cin;
+                float prev[C];
+#pragma unroll
+                for (int c = 0; c < C; ++c) prev[c] = cin[c];
                 long long i = iw;
 #pragma unroll
                 for (int u = 0; u < kRows; ++u) {
                     if ((FULL || u < nvalid) && write) {
-                        const float val = fmaf(pb[u], cin, val0[u]);
-                        Coef c;
-                        c.alpha = alp[u]; c.pg = pgc[u]; c.beta = 0.f;
-                        emit<ALGO>(p, i, val, prev, v1[u], c);
-                        prev = val;
+                        float o0[C], o1[C];
+#pragma unroll
+                        for (int c = 0; c < C; ++c) {
+                            const float val = fmaf(pb[u][c], cin[c], val0[u][c]);
+                            if constexpr (ALGO == kGae) { o0[c] = val; o1[c] = val + v1[u][c]; }
+                            else if constexpr (ALGO == kVtrace) { o0[c] = v1[u][c] + val; o1[c] = fmaf(pgc[u][c], prev[c], alp[u][c]); }
+                            else if constexpr (ALGO == kRetrace) { o0[c] = v1[u][c] + val; o1[c] = 0.f; }
+                            else { o0[c] = val; o1[c] = 0.f; }
+                            prev[c] = val;
+                        }
+                        stg_f<C>(p.out0 + i, o0);
+                        if constexpr (ALGO == kGae || ALGO == kVtrace) {
+                            if (p.out1 != nullptr) stg_f<C>(p.out1 + i, o1);
+                        }
                     }
                     i += cp.rowstep;
                 }
@@ -654,7 +729,9 @@ __global__ void __launch_bounds__(32 * W) tm_block_kernel(const TmParams p) {
             cp_async_commit();
         }
 #pragma unroll
-        for (int u = 0; u < kRows; ++u) { bvc[u] = bv1[u]; bv1[u] = bv2[u]; }
+        for (int u = 0; u < kRows; ++u)
+#pragma unroll
+            for (int c = 0; c < C; ++c) { bvc[u][c] = bv1[u][c]; bv1[u][c] = bv2[u][c]; }
         fs = wrap_next(fs, S);
         ms = wrap_next(ms, SM);
         iw += stagestep;
@@ -662,8 +739,11 @@ __global__ void __launch_bounds__(32 * W) tm_block_kernel(const TmParams p) {
     }
     cp_async_wait(0);
     if (MODE == 1 && write && w == 0) {
-        p.agg_a[(long long)k * p.N + n] = A;
-        p.agg_b[(long long)k * p.N + n] = P;
+#pragma unroll
+        for (int c = 0; c < C; ++c) {
+            p.agg_a[(long long)k * p.N + n0 + C * lane + c] = A[c];
+            p.agg_b[(long long)k * p.N + n0 + C * lane + c] = P[c];
+        }
     }
 }
 
@@ -708,16 +788,19 @@ void plan_chunks(long long N, long long T, unsigned* chunk, unsigned* chunks) {
     *chunks = (unsigned)((T + len - 1) / len);
 }
 
-// Warps per block and ring depth for tm_block_kernel.  Eight warps when blocks are scarce, else four.
-// The kernel is bound by issue slots and dependent-ALU latency as much as by HBM, so resident warps
-// come first: the ring is as deep as still lets min(blocks per SM, 6) blocks share an SM, no deeper
-// than keeps about 16 MB in flight over the grid, and at least 3.
-size_t plan_block(TmParams& p, int row_bytes, bool trunc) {
-    const long long blocks = (p.N + 31) / 32 * p.chunks;
-    const int W = blocks < 2 * kSms ? 8 : 4;
-    const long long stage = (long long)kRows * W * row_bytes;
-    const long long mstage = (long long)kRows * W * (trunc ? 64 : 32);
-    const long long fixed = 2 * mstage + W * 512 + 512;      // mask ring's two extra slots, aggregates, edges
+// Columns per lane, warps per block and ring depth for tm_block_kernel.  Two columns per lane when
+// that still leaves two blocks per SM (and the outputs allow 8-byte stores); eight warps when blocks
+// are scarce, else four.  The kernel is bound by issue slots and dependent-ALU latency as much as by
+// HBM, so resident warps come first: the ring is as deep as still lets min(blocks per SM, 6) blocks
+// share an SM, no deeper than keeps about 16 MB in flight over the grid, and at least 3.
+size_t plan_block(TmParams& p, int row_bytes, bool trunc, bool wide_ok) {
+    int C = 1;
+    if (wide_ok && (p.N + 63) / 64 * p.chunks >= 2 * kSms) C = 2;
+    const long long blocks = (p.N + 32 * C - 1) / (32 * C) * p.chunks;
+    const int W = (C == 1 && blocks < 2 * kSms) ? 8 : 4;
+    const long long stage = (long long)kRows * W * row_bytes * C;
+    const long long mstage = (long long)kRows * W * (trunc ? 64 : 32) * C;
+    const long long fixed = 2 * mstage + (W * 512 + 512) * C;   // mask ring's two extra slots, aggregates, edges
     auto block_bytes = [&](long long S) { return S * stage + fixed; };
     long long resident = (blocks + kSms - 1) / kSms;
     if (resident > 6) resident = 6;
@@ -730,8 +813,13 @@ size_t plan_block(TmParams& p, int row_bytes, bool trunc) {
     if (S < 3) S = 3;
     p.stages = (int)S;
     p.warps_per_block = W;
+    p.cols_per_lane = C;
     return (size_t)block_bytes(S);
 }
+
+int g_force_cols = 0;    // test hook: 1 = one column per lane whatever the size
+
+inline bool aligned8(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 7u) == 0; }
 
 template <typename K>
 bool allow_smem(K kernel, size_t bytes) {
@@ -739,18 +827,18 @@ bool allow_smem(K kernel, size_t bytes) {
     return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kSmemPerSm - 1024)) == cudaSuccess;
 }
 
-template <int ALGO, bool TRUNC, int W>
+template <int ALGO, bool TRUNC, int W, int C>
 int launch_block(const TmParams& p, size_t smem, cudaStream_t s) {
-    const dim3 grid((unsigned)((p.N + 31) / 32), p.chunks);
+    const dim3 grid((unsigned)((p.N + 32 * C - 1) / (32 * C)), p.chunks);
     if (p.chunks == 1) {
-        if (!allow_smem(tm_block_kernel<ALGO, TRUNC, 0, W>, smem)) return RLCS_ERR_CUDA;
-        tm_block_kernel<ALGO, TRUNC, 0, W><<<grid, 32 * W, smem, s>>>(p);
+        if (!allow_smem(tm_block_kernel<ALGO, TRUNC, 0, W, C>, smem)) return RLCS_ERR_CUDA;
+        tm_block_kernel<ALGO, TRUNC, 0, W, C><<<grid, 32 * W, smem, s>>>(p);
     } else {
-        if (!allow_smem(tm_block_kernel<ALGO, TRUNC, 1, W>, smem) || !allow_smem(tm_block_kernel<ALGO, TRUNC, 2, W>, smem))
+        if (!allow_smem(tm_block_kernel<ALGO, TRUNC, 1, W, C>, smem) || !allow_smem(tm_block_kernel<ALGO, TRUNC, 2, W, C>, smem))
             return RLCS_ERR_CUDA;
-        tm_block_kernel<ALGO, TRUNC, 1, W><<<grid, 32 * W, smem, s>>>(p);
+        tm_block_kernel<ALGO, TRUNC, 1, W, C><<<grid, 32 * W, smem, s>>>(p);
         tm_chain_kernel<tm_forward(ALGO)><<<(unsigned)((p.N + kThreads - 1) / kThreads), kThreads, 0, s>>>(p);
-        tm_block_kernel<ALGO, TRUNC, 2, W><<<grid, 32 * W, smem, s>>>(p);
+        tm_block_kernel<ALGO, TRUNC, 2, W, C><<<grid, 32 * W, smem, s>>>(p);
     }
     return cudaGetLastError() == cudaSuccess ? RLCS_OK : RLCS_ERR_CUDA;
 }
@@ -760,8 +848,16 @@ int launch(TmParams p, bool staged, cudaStream_t s) {
     constexpr bool FWD = tm_forward(ALGO);
     const unsigned gx_chain = (unsigned)((p.N + kThreads - 1) / kThreads);
     if (staged) {
-        const size_t smem = plan_block(p, tm_row_bytes(ALGO, TRUNC), TRUNC);
-        return p.warps_per_block == 8 ? launch_block<ALGO, TRUNC, 8>(p, smem, s) : launch_block<ALGO, TRUNC, 4>(p, smem, s);
+        // Two columns per lane pay where registers allow it (measured: GAE and TD(lambda) without
+        // truncation handling, +4 %; with it, or with three or four float inputs, 128-168 registers
+        // per thread cost more occupancy than the shared addressing saves).
+        constexpr bool kWide = !TRUNC && (ALGO == kGae || ALGO == kTdLambda);
+        const bool wide_ok = kWide && g_force_cols != 1 && aligned8(p.out0) && aligned8(p.out1);
+        const size_t smem = plan_block(p, tm_row_bytes(ALGO, TRUNC), TRUNC, wide_ok);
+        if constexpr (kWide) {
+            if (p.cols_per_lane == 2) return launch_block<ALGO, TRUNC, 4, 2>(p, smem, s);
+        }
+        return p.warps_per_block == 8 ? launch_block<ALGO, TRUNC, 8, 1>(p, smem, s) : launch_block<ALGO, TRUNC, 4, 1>(p, smem, s);
     } else {
         const dim3 grid(gx_chain, p.chunks);
         if (p.chunks == 1) {
@@ -832,7 +928,10 @@ size_t rlcs_time_major_workspace_bytes(int64_t N, int64_t T) {
     return chunks > 1 ? 2 * sizeof(float) * (size_t)N * chunks : 0;
 }
 
-void rlcs_debug_time_major_path(int path) { g_force_path = path; }
+void rlcs_debug_time_major_path(int path) {
+    g_force_path = path == 3 ? 2 : path;
+    g_force_cols = path == 3 ? 1 : 0;
+}
 
 int rlcs_gae_time_major(const float* rewards, const float* values, const uint8_t* dones, const uint8_t* truncs,
                         const float* trunc_bootstrap, const float* bootstrap, float* advantages, float* returns,

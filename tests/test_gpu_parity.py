@@ -538,15 +538,19 @@ def tm_path(B, request):
 
 
 @pytest.mark.parametrize("N,T", [(1, 1), (3, 7), (8, 128), (300, 65), (4096, 64), (64, 3000), (5, 20000), (40000, 33),
-                                 (16, 1), (48, 517), (4112, 70), (16, 20000), (20000, 9)])
+                                 (16, 1), (48, 517), (4112, 70), (16, 20000), (20000, 9), (19024, 300)])
 @pytest.mark.parametrize("p_flag", [0.0, 0.02, 0.5])
-@pytest.mark.parametrize("tm_path", [1, 2], indirect=True)
+@pytest.mark.parametrize("tm_path", [1, 2, 3], indirect=True)
 def test_time_major_entry_points(oracle, W, B, N, T, p_flag, tm_path):
     """All seven algorithms on [T, N] tensors against the oracle run on the transposed arrays; shapes
     cover the single-pass walk (many environments), the cut time axis (few environments), both
-    kernels (register walk; shared-memory ring, which needs N % 16 == 0) and ragged last warps."""
-    if tm_path == 2 and N % 16 != 0:
+    kernels (register walk; shared-memory ring, which needs N % 16 == 0, with two columns per lane
+    where the library uses them -- GAE and TD(lambda) without truncations from 18944 environments up
+    -- and with one column per lane) and ragged last warps."""
+    if tm_path != 1 and N % 16 != 0:
         pytest.skip("the ring needs N % 16 == 0; the register walk is covered by tm_path = 1")
+    if tm_path == 3 and N < 18944:
+        pytest.skip("one column per lane is what tm_path = 2 already takes at this size")
     ro = W.make_rollout(115, N, T, p_done=p_flag, p_trunc=p_flag / 2, salt=T)
     p = ro.params
     ref = run_oracle(oracle, ro, ALL_ALGOS)
@@ -577,6 +581,11 @@ def test_time_major_entry_points(oracle, W, B, N, T, p_flag, tm_path):
     ref2 = run_oracle(oracle, ro, ("gae", "discounted_return"), use_truncs=False, use_bootstrap=False)
     adv2 = B.rlcs_gae_time_major(r, v, d, gamma=p["gamma"], lam=p["lam"], want_returns=False)
     assert_close("gae no truncs", np.ascontiguousarray(back(adv2)), ref2["gae"][0])
+    adv3, ret3 = B.rlcs_gae_time_major(r, v, d, gamma=p["gamma"], lam=p["lam"])
+    assert_close("gae no truncs, with returns", np.ascontiguousarray(back(ret3)), ref2["gae"][1])
+    ref3 = run_oracle(oracle, ro, ("td_lambda",), use_truncs=False)
+    out = B.rlcs_td_lambda_time_major(r, v, d, None, None, bt, gamma=p["gamma"], lam=p["lam"])
+    assert_close("td_lambda no truncs", np.ascontiguousarray(back(out)), ref3["td_lambda"])
     out = B.rlcs_discounted_return_time_major(r, d, gamma=p["gamma"])
     assert_close("disc no truncs", np.ascontiguousarray(back(out)), ref2["discounted_return"])
 
