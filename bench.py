@@ -647,6 +647,9 @@ def main():
     ap.add_argument("--variant", type=int, default=None, help="tile variant test hook (default: library default)")
     ap.add_argument("--no-truncs", action="store_true", help="bench batch without per-step truncation handling")
     ap.add_argument("--rows", type=int, default=WORKLOAD["N"], help="num_envs of the bench batch (default: full size)")
+    ap.add_argument("--only", choices=("time_major", "bf16"), default=None,
+                    help="time only that extension line on a --rows x --seq-len batch and print it (one JSON line)")
+    ap.add_argument("--seq-len", type=int, default=WORKLOAD["T"], help="T of the --only batch")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -677,6 +680,11 @@ def main():
     if args.sweep_only:
         peak, _ = measured_peak()
         print(json.dumps({"sweeps": run_sweeps(torch, peak)}), flush=True)
+        return
+    if args.only is not None:
+        peak, _ = measured_peak()
+        fn = time_time_major if args.only == "time_major" else time_bf16
+        print(json.dumps({args.only: fn(torch, binding, max(1, args.steps), peak, args.rows, args.seq_len)}), flush=True)
         return
 
     N = args.rows
