@@ -40,7 +40,7 @@ using rlcs::kRetrace;
 using rlcs::kElig;
 using rlcs::kPrefix;
 
-constexpr int kRows = 8;         // timesteps per stage / per register block
+constexpr int kRows = 8;         // timesteps per register block of tm_kernel; upper bound of tm_rows()
 constexpr int kThreads = 128;    // register-path block; the staged path uses 32 * warps_per_block
 
 struct TmParams {
@@ -69,6 +69,10 @@ __host__ __device__ constexpr bool tm_forward(int a) { return a == kElig || a ==
 __host__ __device__ constexpr int tm_nf(int a) {
     return a == kRetrace ? 4 : a == kVtrace ? 3 : (a == kGae || a == kTdLambda) ? 2 : 1;
 }
+// timesteps per warp and stage in tm_block_kernel: fewer for Retrace, whose four float inputs make a
+// row 576 bytes (measured: 0.84 -> 0.90 of the copy bandwidth with 4, while the lighter algorithms
+// lose 5-12 % to the doubled per-stage overhead)
+__host__ __device__ constexpr int tm_rows(int a) { return a == kRetrace ? 4 : 8; }
 __host__ __device__ constexpr int tm_row_bytes(int a, bool trunc) { return tm_nf(a) * 128 + (trunc ? 2 : 1) * 32; }
 
 // all ones where x != 0, else 0; written in PTX so that the flag reaches the arithmetic below as a
@@ -381,7 +385,7 @@ __device__ __forceinline__ void cp_async_wait(int pending) {
 constexpr int kMaxStages = 16;
 constexpr int kMaxWarps = 8;
 
-// One stage of a thread block: R = kRows * warps rows of its 32 C columns (C columns per lane), row
+// One stage of a thread block: R = KR * warps rows (KR = tm_rows(ALGO) timesteps per warp) of its 32 C columns (C columns per lane), row
 // index = scan-order step within the stage.  Floats and masks live in separate rings (the mask ring
 // runs two stages ahead): float tensor a at fbase[a][row][32 C floats], mask tensor m at
 // mbase[m][row][32 C bytes].
@@ -389,7 +393,8 @@ template <int ALGO, bool TRUNC, int W, int C>
 struct StageView {
     static constexpr int NF = tm_nf(ALGO);
     static constexpr int NM = TRUNC ? 2 : 1;
-    static constexpr int R = kRows * W;
+    static constexpr int KR = tm_rows(ALGO);
+    static constexpr int R = KR * W;
     unsigned char* fbase;
     unsigned char* mbase;
     __device__ __forceinline__ float* f(int a, int row) const { return reinterpret_cast<float*>(fbase + (a * R + row) * (128 * C)); }
@@ -429,11 +434,12 @@ struct CopyPlan {
 
 template <int ALGO, bool TRUNC, int W, int C>
 __device__ __forceinline__ void issue_floats(const StageView<ALGO, TRUNC, W, C>& sv, const TmParams& p, const CopyPlan& cp, unsigned s) {
-    constexpr int R = kRows * W;
+    constexpr int KR = tm_rows(ALGO);
+    constexpr int R = KR * W;
     const float* const fsrc[4] = {p.f0, p.f1, p.f2, p.f3};
     constexpr int fidx[4] = {0, 1, (ALGO == kVtrace) ? 3 : 2, 3};   // V-trace stages f0, f1, f3
 #pragma unroll
-    for (int h = 0; h < 2 * C; ++h) {
+    for (int h = 0; h < KR * C / 4; ++h) {
         const int row = cp.frow + h * (4 * W / C);
         const unsigned q = s * R + row;
         const bool ok = cp.fcol_ok && q < cp.len;
@@ -447,7 +453,7 @@ __device__ __forceinline__ void issue_floats(const StageView<ALGO, TRUNC, W, C>&
 template <int ALGO, bool TRUNC, int W, int C>
 __device__ __forceinline__ void issue_masks(const StageView<ALGO, TRUNC, W, C>& sv, const TmParams& p, const CopyPlan& cp, unsigned s) {
     if (cp.m_on) {
-        const unsigned q = s * (kRows * W) + cp.mrow;
+        const unsigned q = s * (tm_rows(ALGO) * W) + cp.mrow;
         const bool ok = q < cp.len;
         const long long off = ok ? cp.i_first + cp.rowstep * q + cp.mcol : 0;
         cp_async16(sv.m(0, cp.mrow) + cp.mcol, p.dones + off, ok ? 16u : 0u);
@@ -458,13 +464,14 @@ __device__ __forceinline__ void issue_masks(const StageView<ALGO, TRUNC, W, C>& 
 // truncation continuation values of `nvalid` rows from row0 of a stage whose masks have landed;
 // i = flat index of the first of them for this lane's first column
 template <int ALGO, bool TRUNC, int W, int C>
-__device__ __forceinline__ void stage_bv(float (&bv)[kRows][C], const StageView<ALGO, TRUNC, W, C>& sv, const TmParams& p,
+__device__ __forceinline__ void stage_bv(float (&bv)[tm_rows(ALGO)][C], const StageView<ALGO, TRUNC, W, C>& sv, const TmParams& p,
                                          long long i, long long rowstep, int row0, int nvalid, int lane, unsigned write_mask) {
+    constexpr int KR = tm_rows(ALGO);
     if (nvalid <= 0) return;                                 // past the chunk: the values are never used
     auto rows = [&](auto full) {
         constexpr bool FULL = decltype(full)::value;
 #pragma unroll
-        for (int u = 0; u < kRows; ++u) {
+        for (int u = 0; u < KR; ++u) {
             unsigned tr[C], dn[C];
             lds_m<C>(sv.m(1, row0 + u), lane, tr);
             lds_m<C>(sv.m(0, row0 + u), lane, dn);
@@ -474,7 +481,7 @@ __device__ __forceinline__ void stage_bv(float (&bv)[kRows][C], const StageView<
             i += rowstep;
         }
     };
-    if (nvalid >= kRows) rows(std::true_type{});
+    if (nvalid >= KR) rows(std::true_type{});
     else rows(std::false_type{});
 }
 
@@ -483,7 +490,7 @@ __device__ __forceinline__ int wrap_prev(int x, int n) { return x == 0 ? n - 1 :
 
 // A thread block owns 32 C adjacent environments (a lane C of them: with C = 2 every shared-memory
 // read, store and address computation serves two steps); its W warps split every stage of
-// R = kRows * W timesteps in time.  Per stage: each warp walks its kRows steps from carry 0, keeping
+// R = KR * W timesteps in time (KR = tm_rows).  Per stage: each warp walks its KR steps from carry 0, keeping
 // per step the value so far and the running product of betas (the step's affine map of the incoming
 // carry, Eq. 2); the W per-warp aggregates go through shared memory; every warp folds them in scan
 // order onto the block's carry (a few FMAs, redundantly in each warp) to get its own incoming
@@ -500,7 +507,8 @@ __global__ void __launch_bounds__(32 * W) tm_block_kernel(const TmParams p) {
     using SV = StageView<ALGO, TRUNC, W, C>;
     extern __shared__ __align__(16) unsigned char tm_smem[];
     const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
-    constexpr int R = kRows * W;
+    constexpr int KR = tm_rows(ALGO);
+    constexpr int R = KR * W;
     const int S = p.stages, SM = S + 2;
     constexpr int fstage = R * SV::NF * 128 * C, mstage = R * SV::NM * 32 * C;
     unsigned char* const mring = tm_smem + (size_t)S * fstage;
@@ -545,7 +553,7 @@ __global__ void __launch_bounds__(32 * W) tm_block_kernel(const TmParams p) {
     // A group is committed for every stage index, empty past the end, so that "all but the newest P
     // groups" always names the same stages.  Floats of stage s sit in slot s mod S, masks in slot
     // s mod (S + 2).  With C = 1 only the first half of the threads has a mask piece.
-    const bool mask_thread = C == 2 || tid < 2 * R;
+    const bool mask_thread = tid < 2 * C * R;
     cp.m_on = cp.m_on && mask_thread;
     for (int s = 0; s + 1 < S; ++s) {
         if (s == 0) {
@@ -556,12 +564,12 @@ __global__ void __launch_bounds__(32 * W) tm_block_kernel(const TmParams p) {
         if ((unsigned)s + 2 < nst) issue_masks<ALGO, TRUNC>(SV{nullptr, mring + (s + 2) * mstage}, p, cp, s + 2);
         cp_async_commit();
     }
-    float bvc[kRows][C], bv1[kRows][C], bv2[kRows][C];
+    float bvc[KR][C], bv1[KR][C], bv2[KR][C];
 #pragma unroll
-    for (int u = 0; u < kRows; ++u)
+    for (int u = 0; u < KR; ++u)
 #pragma unroll
         for (int c = 0; c < C; ++c) bvc[u][c] = bv1[u][c] = bv2[u][c] = 0.f;
-    const int row0 = kRows * w;
+    const int row0 = KR * w;
     // this lane's flat index (first column) at its first row of the current stage, and rows it has there
     long long iw = cp.i_first + cp.rowstep * row0 + C * lane;
     int left = (int)len - row0;                              // steps from this warp's first row to the chunk's end
@@ -578,7 +586,7 @@ __global__ void __launch_bounds__(32 * W) tm_block_kernel(const TmParams p) {
         cp_async_wait(S - 2);                                // this thread's pieces of stage j (masks: j+2)
         __syncthreads();                                     // ... and everyone else's
         const SV cur{tm_smem + fs * fstage, mring + ms * mstage};
-        const int nvalid = left < kRows ? (left < 0 ? 0 : left) : kRows;
+        const int nvalid = left < KR ? (left < 0 ? 0 : left) : KR;
         if constexpr (TRUNC) {
             const int ms2 = ms + 2 >= SM ? ms + 2 - SM : ms + 2;
             stage_bv<ALGO, TRUNC>(bv2, SV{nullptr, mring + ms2 * mstage}, p, iw + 2 * stagestep, cp.rowstep, row0, left - 2 * R,
@@ -609,7 +617,7 @@ __global__ void __launch_bounds__(32 * W) tm_block_kernel(const TmParams p) {
             for (int c = 0; c < C; ++c) { v_next[c] = v0[c]; lr_next[c] = lr0[c]; d_prev[c] = d0[c]; }
         }
         // pass 1: from carry 0
-        float val0[kRows][C], pb[kRows][C], v1[kRows][C], pgc[kRows][C], alp[kRows][C];
+        float val0[KR][C], pb[KR][C], v1[KR][C], pgc[KR][C], alp[KR][C];
         float carry[C], prod[C];
 #pragma unroll
         for (int c = 0; c < C; ++c) { carry[c] = 0.f; prod[c] = 1.f; }
@@ -617,7 +625,7 @@ __global__ void __launch_bounds__(32 * W) tm_block_kernel(const TmParams p) {
         auto pass1 = [&](auto full) {
             constexpr bool FULL = decltype(full)::value;
 #pragma unroll
-            for (int u = 0; u < kRows; ++u) {
+            for (int u = 0; u < KR; ++u) {
 #pragma unroll
                 for (int c = 0; c < C; ++c) { v1[u][c] = 0.f; pgc[u][c] = 0.f; alp[u][c] = 0.f; }
                 if (FULL || u < nvalid) {
@@ -663,7 +671,7 @@ __global__ void __launch_bounds__(32 * W) tm_block_kernel(const TmParams p) {
                 for (int c = 0; c < C; ++c) { val0[u][c] = carry[c]; pb[u][c] = prod[c]; }
             }
         };
-        if (nvalid == kRows) pass1(std::true_type{});
+        if (nvalid == KR) pass1(std::true_type{});
         else pass1(std::false_type{});
 #pragma unroll
         for (int c = 0; c < C; ++c) agg[((par * W + w) * 32 + lane) * C + c] = make_float2(carry[c], prod[c]);
@@ -698,7 +706,7 @@ __global__ void __launch_bounds__(32 * W) tm_block_kernel(const TmParams p) {
                 for (int c = 0; c < C; ++c) prev[c] = cin[c];
                 long long i = iw;
 #pragma unroll
-                for (int u = 0; u < kRows; ++u) {
+                for (int u = 0; u < KR; ++u) {
                     if ((FULL || u < nvalid) && write) {
                         float o0[C], o1[C];
 #pragma unroll
@@ -718,7 +726,7 @@ __global__ void __launch_bounds__(32 * W) tm_block_kernel(const TmParams p) {
                     i += cp.rowstep;
                 }
             };
-            if (nvalid == kRows) pass2(std::true_type{});
+            if (nvalid == KR) pass2(std::true_type{});
             else pass2(std::false_type{});
         }
         // everyone is past the barrier, hence done with stage j-1: refill its slots
@@ -729,7 +737,7 @@ __global__ void __launch_bounds__(32 * W) tm_block_kernel(const TmParams p) {
             cp_async_commit();
         }
 #pragma unroll
-        for (int u = 0; u < kRows; ++u)
+        for (int u = 0; u < KR; ++u)
 #pragma unroll
             for (int c = 0; c < C; ++c) { bvc[u][c] = bv1[u][c]; bv1[u][c] = bv2[u][c]; }
         fs = wrap_next(fs, S);
@@ -793,20 +801,20 @@ void plan_chunks(long long N, long long T, unsigned* chunk, unsigned* chunks) {
 // are scarce, else four.  The kernel is bound by issue slots and dependent-ALU latency as much as by
 // HBM, so resident warps come first: the ring is as deep as still lets min(blocks per SM, 6) blocks
 // share an SM, no deeper than keeps about 16 MB in flight over the grid, and at least 3.
-size_t plan_block(TmParams& p, int row_bytes, bool trunc, bool wide_ok) {
+size_t plan_block(TmParams& p, int rows, int row_bytes, bool trunc, bool wide_ok) {
     int C = 1;
     if (wide_ok && (p.N + 63) / 64 * p.chunks >= 2 * kSms) C = 2;
     const long long blocks = (p.N + 32 * C - 1) / (32 * C) * p.chunks;
     const int W = (C == 1 && blocks < 2 * kSms) ? 8 : 4;
-    const long long stage = (long long)kRows * W * row_bytes * C;
-    const long long mstage = (long long)kRows * W * (trunc ? 64 : 32) * C;
+    const long long stage = (long long)rows * W * row_bytes * C;
+    const long long mstage = (long long)rows * W * (trunc ? 64 : 32) * C;
     const long long fixed = 2 * mstage + (W * 512 + 512) * C;   // mask ring's two extra slots, aggregates, edges
     auto block_bytes = [&](long long S) { return S * stage + fixed; };
     long long resident = (blocks + kSms - 1) / kSms;
     if (resident > 6) resident = 6;
     while (resident > 1 && resident * (block_bytes(3) + 1024) > (long long)kSmemPerSm) --resident;
     long long S = 2 + ((16ll << 20) + blocks * stage - 1) / (blocks * stage);
-    const long long nst = ((long long)p.chunk + kRows * W - 1) / (kRows * W);
+    const long long nst = ((long long)p.chunk + rows * W - 1) / (rows * W);
     if (S > nst + 1) S = nst + 1;
     if (S > kMaxStages) S = kMaxStages;
     while (S > 3 && resident * (block_bytes(S) + 1024) > (long long)kSmemPerSm) --S;
@@ -853,7 +861,7 @@ int launch(TmParams p, bool staged, cudaStream_t s) {
         // per thread cost more occupancy than the shared addressing saves).
         constexpr bool kWide = !TRUNC && (ALGO == kGae || ALGO == kTdLambda);
         const bool wide_ok = kWide && g_force_cols != 1 && aligned8(p.out0) && aligned8(p.out1);
-        const size_t smem = plan_block(p, tm_row_bytes(ALGO, TRUNC), TRUNC, wide_ok);
+        const size_t smem = plan_block(p, tm_rows(ALGO), tm_row_bytes(ALGO, TRUNC), TRUNC, wide_ok);
         if constexpr (kWide) {
             if (p.cols_per_lane == 2) return launch_block<ALGO, TRUNC, 4, 2>(p, smem, s);
         }
