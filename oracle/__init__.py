@@ -58,6 +58,8 @@ def _load():
                                                       _i64, _i64, _i64, _dbl, _dbl, _dbl]
             lib.rlcs_oracle_retrace_probs.restype = None
             lib.rlcs_oracle_elig_trace.argtypes = [_F, _U, _D, _i64, _i64, _dbl, _dbl]
+            lib.rlcs_oracle_gae_skip.argtypes = [_F, _F, _U, _U, _F, _F, _U, _D, _D, _D, _i64, _i64, _dbl, _dbl]
+            lib.rlcs_oracle_gae_skip.restype = None
             lib.rlcs_oracle_elig_trace_vec.argtypes = [_F, _U, _D, _i64, _i64, _i64, _dbl, _dbl]
             lib.rlcs_oracle_elig_trace_vec.restype = None
             lib.rlcs_oracle_elig_trace_vec_beta.argtypes = [_F, _F, _U, _D, _i64, _i64, _i64]
@@ -128,6 +130,21 @@ def gae(rewards, values, dones, truncs=None, trunc_bootstrap=None, bootstrap=Non
     _load().rlcs_oracle_gae(_p(r, _F), _p(v, _F), _p(d, _U), _p(tr, _U), _p(bv, _F), _p(bt, _F),
                             _p(adv, _D), _p(ret, _D), N, T, _s(gamma), _s(lam))
     return (adv, ret) if want_returns else adv
+
+
+def gae_skip(rewards, values, dones, truncs=None, trunc_bootstrap=None, bootstrap=None, *, skip, gamma, lam):
+    """GAE with observation-skip masking (Section 9.2, planned): masked steps (skip != 0) are
+    transparent.  Returns (advantages, returns = A + W, filled values W)."""
+    shape = _shape2(rewards)
+    N, T = shape
+    r, v, d = _f32(rewards, shape), _f32(values, shape), _u8(dones, shape)
+    tr, bv = _trunc_args(truncs, trunc_bootstrap, shape)
+    bt = _f32(bootstrap, (N,))
+    sk = _u8(skip, shape)
+    adv, ret, fil = (np.empty(shape, np.float64) for _ in range(3))
+    _load().rlcs_oracle_gae_skip(_p(r, _F), _p(v, _F), _p(d, _U), _p(tr, _U), _p(bv, _F), _p(bt, _F), _p(sk, _U),
+                                 _p(adv, _D), _p(ret, _D), _p(fil, _D), N, T, _s(gamma), _s(lam))
+    return adv, ret, fil
 
 
 def gae_normalized(rewards, values, dones, truncs=None, trunc_bootstrap=None, bootstrap=None, *, gamma, lam,

@@ -74,6 +74,43 @@ void rlcs_oracle_gae(const float* r, const float* V, const uint8_t* term, const 
     }
 }
 
+/* GAE with observation-skip masking (planned in Section 9.2: the recurrence is carried across masked
+ * tokens with beta_t = 1).  Reading taken here: a masked step is transparent -- it adds no TD
+ * error and no discount, A_t = A_{t+1}, and the value that earlier steps see through it is the
+ * value of the next unmasked step, W_t = W_{t+1}; an unmasked step is the GAE step of Section 3.3.1
+ * with successor value W_{t+1}.  Termination and truncation flags sever the recurrence as in Section
+ * 3.2 wherever they stand: at a flagged masked step A_t = 0 and W_t is the flag's successor value.
+ * Outputs: adv = A, ret = A + W (optional), filled = W (optional).  Without flags on masked steps the
+ * result at the unmasked steps is plain GAE of the sequence with the masked steps deleted. */
+void rlcs_oracle_gae_skip(const float* r, const float* V, const uint8_t* term, const uint8_t* trunc,
+                          const float* bv, const float* boot, const uint8_t* skip, double* adv, double* ret,
+                          double* filled, int64_t N, int64_t T, double gamma, double lambda) {
+    for (int64_t n = 0; n < N; ++n) {
+        const int64_t o = n * T;
+        const double b = boot ? (double)boot[n] : 0.0;
+        double A_next = 0.0, W_next = 0.0;
+        for (int64_t t = T - 1; t >= 0; --t) {
+            const int tm = flag(term, o + t), tr = flag(trunc, o + t), last = (t == T - 1);
+            const double vn = successor(tm, tr, last, (tr && !tm) ? (double)bv[o + t] : 0.0, b, W_next);
+            const int cont = !tm && !tr && !last;
+            double A, W;
+            if (flag(skip, o + t)) {
+                A = cont ? A_next : 0.0;
+                W = vn;                                   /* cont: the next unmasked value, passed through */
+            } else {
+                const double delta = (double)r[o + t] + gamma * vn - (double)V[o + t];
+                A = cont ? delta + gamma * lambda * A_next : delta;
+                W = (double)V[o + t];
+            }
+            adv[o + t] = A;
+            if (ret) ret[o + t] = A + W;
+            if (filled) filled[o + t] = W;
+            A_next = A;
+            W_next = W;
+        }
+    }
+}
+
 /* TD(lambda) returns (Section 3.3.4):
  * G_t = r_t + gamma*[(1-lambda)*V(s_{t+1}) + lambda*G_{t+1}].  Where the
  * recurrence is severed (flag or window edge) the continuation G_{t+1} is the

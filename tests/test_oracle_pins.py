@@ -700,3 +700,64 @@ def test_per_dimension_beta_trace_against_the_unrolled_sum(oracle):
     beta2 = beta.copy()
     beta2[:, 0, :] = np.nan
     assert np.array_equal(oracle.elig_trace_vec_beta(x, beta2, d), z)
+
+
+# ----------------------------------------------------------------------------- observation-skip masking
+def test_skip_masked_gae_is_gae_of_the_sequence_with_masked_steps_deleted(oracle):
+    """The reading of Section 9.2's observation-skip masking: masked steps are transparent.  With no
+    flag on a masked step, the advantages at the unmasked steps equal plain GAE (an already pinned
+    routine) on the row with the masked steps deleted; a masked step repeats the advantage and the
+    value of the next unmasked step; the row's trailing masked steps see the window-edge bootstrap."""
+    rng = np.random.default_rng(62)
+    T = 60
+    for trial in range(20):
+        r = rng.standard_normal((1, T)).astype(np.float32)
+        V = rng.standard_normal((1, T)).astype(np.float32)
+        skip = (rng.random((1, T)) < 0.4).astype(np.uint8)
+        keep = skip[0] == 0
+        if not keep.any():
+            continue
+        d = ((rng.random((1, T)) < 0.1) & keep).astype(np.uint8)           # flags only on unmasked steps
+        tr = ((rng.random((1, T)) < 0.1) & keep).astype(np.uint8)
+        bv = rng.standard_normal((1, T)).astype(np.float32)
+        boot = rng.standard_normal((1,)).astype(np.float32)
+        adv, ret, fil = oracle.gae_skip(r, V, d, tr, bv, boot, skip=skip, gamma=0.97, lam=0.9)
+        c = lambda a: np.ascontiguousarray(a[:, keep])
+        # the compacted row ends where the original does: trailing masked steps pass the bootstrap through
+        want, want_ret = oracle.gae(c(r), c(V), c(d), c(tr), c(bv), boot, gamma=0.97, lam=0.9)
+        np.testing.assert_allclose(adv[:, keep], want, rtol=1e-12, atol=1e-12)
+        np.testing.assert_allclose(ret[:, keep], want_ret, rtol=1e-12, atol=1e-12)
+        np.testing.assert_array_equal(fil[:, keep], V[:, keep].astype(np.float64))
+        # masked steps repeat what follows them (advantage and value), or the edge values at the end
+        for t in range(T - 1, -1, -1):
+            if skip[0, t]:
+                nxt_a = adv[0, t + 1] if t + 1 < T else 0.0
+                nxt_w = fil[0, t + 1] if t + 1 < T else float(boot[0])
+                assert adv[0, t] == nxt_a and fil[0, t] == nxt_w and ret[0, t] == nxt_a + nxt_w
+
+
+def test_skip_masked_gae_special_cases(oracle):
+    rng = np.random.default_rng(63)
+    N, T = 3, 40
+    r, V, bv = (rng.standard_normal((N, T)).astype(np.float32) for _ in range(3))
+    d = (rng.random((N, T)) < 0.1).astype(np.uint8)
+    tr = (rng.random((N, T)) < 0.1).astype(np.uint8)
+    boot = rng.standard_normal((N,)).astype(np.float32)
+    # nothing masked: plain GAE, exactly
+    adv, ret, fil = oracle.gae_skip(r, V, d, tr, bv, boot, skip=np.zeros((N, T), np.uint8), gamma=0.99, lam=0.95)
+    a0, r0 = oracle.gae(r, V, d, tr, bv, boot, gamma=0.99, lam=0.95)
+    assert np.array_equal(adv, a0) and np.array_equal(ret, r0) and np.array_equal(fil, V.astype(np.float64))
+    # everything masked, no flags: nothing to estimate, the bootstrap shows through every step
+    z = np.zeros((N, T), np.uint8)
+    adv, ret, fil = oracle.gae_skip(r, V, z, None, None, boot, skip=np.ones((N, T), np.uint8), gamma=0.99, lam=0.95)
+    assert not adv.any() and np.array_equal(fil, np.repeat(boot.astype(np.float64)[:, None], T, axis=1))
+    # a flagged masked step severs the recurrence: hand-worked row  [u, m(term), u]
+    r1 = np.array([[1.0, 5.0, 2.0]], np.float32)
+    V1 = np.array([[0.5, 9.0, 0.25]], np.float32)
+    d1 = np.array([[0, 1, 0]], np.uint8)
+    s1 = np.array([[0, 1, 0]], np.uint8)
+    adv, ret, fil = oracle.gae_skip(r1, V1, d1, None, None, np.array([4.0], np.float32), skip=s1, gamma=0.5, lam=0.5)
+    # t=2: delta = 2 + 0.5*4 - 0.25 = 3.75 ; t=1 (masked, terminated): A = 0, W = 0 ; t=0: delta = 1 + 0.5*0 - 0.5 = 0.5,
+    # continues into the masked step: A = 0.5 + 0.25 * 0 = 0.5
+    np.testing.assert_allclose(adv, [[0.5, 0.0, 3.75]], rtol=0, atol=1e-15)
+    np.testing.assert_allclose(fil, [[0.5, 0.0, 0.25]], rtol=0, atol=1e-15)
