@@ -243,6 +243,38 @@ def time_gae_normalized(batch: GpuBatch, steps: int, peak: float):
             "algorithmic_bytes": ab, "gbs": round(gbs, 1), "frac_of_peak": round(gbs / peak, 4)}
 
 
+def time_gae_skip(batch: GpuBatch, steps: int, peak: float, p_skip: float = 0.3):
+    """Extension beyond the seven kernels: GAE with observation-skip masking (two launches) on the bench
+    batch with skip ~ Bernoulli(p_skip).  Algorithmic bytes = GAE's, plus the skip mask, plus one write
+    of the filled values W (an output of the call); the second scan's re-read of W and of the masks is
+    the method's own traffic and is not counted."""
+    torch, B, ro = batch.torch, batch.B, batch.ro
+    i, o, p = batch.inp, batch.out, ro.params
+    g = torch.Generator(device="cuda").manual_seed(17641)
+    skip = (torch.rand((ro.N, ro.T), generator=g, device="cuda") < p_skip).to(torch.uint8)
+    fil = torch.empty_like(i["values"])
+    ws = B.Workspace(ro.N, ro.T)
+    call = lambda: B.rlcs_gae_skip(i["rewards"], i["values"], i["dones"], i["truncs"], i["trunc_bootstrap"],
+                                   i["bootstrap"], skip=skip, gamma=p["gamma"], lam=p["lam"], values_filled=fil,
+                                   advantages=o["gae"][0], returns=o["gae"][1], workspace=ws)
+    for _ in range(3):
+        call()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(steps):
+        call()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    ab = algorithmic_bytes(ro, "gae") + 5 * ro.N * ro.T
+    moved = ab + (4 + 1 + (2 if ro.truncs is not None else 1)) * ro.N * ro.T      # W and the masks, read again by scan 2
+    gbs = ab / (ms * 1e-3) / 1e9
+    return {"ms": round(ms, 5), "launches_per_call": 2, "p_skip": p_skip, "env_steps_per_s": ro.N * ro.T / (ms * 1e-3),
+            "algorithmic_bytes": ab, "gbs": round(gbs, 1), "frac_of_peak": round(gbs / peak, 4),
+            "frac_of_peak_on_bytes_moved": round(moved / (ms * 1e-3) / 1e9 / peak, 4)}
+
+
 def time_retrace_probs(torch, B, steps: int, peak: float, N=16384, T=2048, A=4):
     """Extension beyond the seven kernels: Retrace from [N,T,A] Q-values / action probabilities.
     Algorithmic bytes per step: Q and pi rows (8A), one 32-byte sector of mu for the gathered
@@ -718,6 +750,8 @@ def main():
                                           / (sum(v["ms"] for v in per_algo.values()) * 1e-3) / 1e9 / peak, 4)}
 
     extensions = {"gae_normalized": time_gae_normalized(batch, max(3, min(args.steps, 50)), peak)}
+    if rank == 0 and world == 1 and not args.no_sweep:
+        extensions["gae_skip"] = time_gae_skip(batch, max(3, min(args.steps, 30)), peak)
     e2e_steps = max(1, min(args.steps, 8))
     e2e_ms, h2d, d2h = time_e2e(batch, e2e_steps, 1, dist)
     e2e_ms = dist.max(e2e_ms)

@@ -303,6 +303,25 @@ int rlcs_episodic_prefix_sum_time_major(const float* x, const uint8_t* dones, fl
                                         int starts_at, void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * GAE with observation-skip masking (planned in Section 9.2: "carries the recurrence across masked
+ * tokens (beta_t = 1)"; for token-level trajectories whose observation / tool tokens are not actions).
+ * skip [N, T] uint8, non-zero = masked.  Reading: a masked step is transparent --
+ *   masked t:    A_t = A_{t+1},  W_t = W_{t+1}                      (no TD error, no discount)
+ *   unmasked t:  A_t = r_t + gamma*W_{t+1} - V_t + gamma*lambda*A_{t+1},  W_t = V_t
+ * with A = 0 and W = bootstrap beyond the window, and termination / truncation flags severing both
+ * recurrences as in rlcs_gae wherever they stand (at a flagged masked step A_t = 0 and W_t is the
+ * flag's successor value).  Without flags on masked steps, the advantages at the unmasked steps are
+ * rlcs_gae of the rows with the masked steps deleted.
+ * Outputs: values_filled = W (required; also the scratch between the two scans), advantages = A,
+ * returns = A + W (optional).  Two launches: W by a backward scan, then the masked GAE scan on
+ * (rewards, W).  Same flags, NULL conventions, alignment rules and workspace as rlcs_gae.
+ */
+int rlcs_gae_skip(const float* rewards, const float* values, const uint8_t* dones, const uint8_t* truncs,
+                  const float* trunc_bootstrap, const float* bootstrap, const uint8_t* skip, float* values_filled,
+                  float* advantages, float* returns, int64_t N, int64_t T, float gamma, float lambda,
+                  void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
  * bfloat16-tensor variants of the seven entry points (the paper's kernels are fp32-only; Section 9.1
  * defers bfloat16, Section 9.2 plans it): every float tensor -- inputs, trunc_bootstrap, bootstrap
  * and outputs -- holds bfloat16 bit patterns (uint16_t, row-major [N, T], 2-byte aligned; 32-byte

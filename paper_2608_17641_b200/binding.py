@@ -40,6 +40,7 @@ SIGNATURES = {
     "rlcs_elig_trace_vec_beta": ([_vp] * 4 + [_i64, _i64, _i64] + _TAIL, _int),
     "rlcs_elig_trace_vec_beta_workspace_bytes": ([_i64, _i64, _i64], _sz),
     "rlcs_episodic_prefix_sum": ([_vp] * 3 + [_i64, _i64, _int] + _TAIL, _int),
+    "rlcs_gae_skip": ([_vp] * 10 + [_i64, _i64, _f, _f] + _TAIL, _int),
     "rlcs_gae_no_alloc": ([_vp] * 8 + [_i64, _i64, _f, _f, _vp], _int),
     "rlcs_no_alloc_scratch_bytes": ([], _sz),
     "rlcs_time_major_workspace_bytes": ([_i64, _i64], _sz),
@@ -194,6 +195,23 @@ def rlcs_gae_normalized(rewards, values, dones, truncs=None, trunc_bootstrap=Non
                                      _ptr(bootstrap, "f32", (N,)), _ptr(adv, "f32", (N, T)), _ptr(ret, "f32", (N, T)),
                                      N, T, gamma, lam, eps, ddof, wp, wb, _stream(stream)))
     return (adv, ret) if want_returns else adv
+
+
+def rlcs_gae_skip(rewards, values, dones, truncs=None, trunc_bootstrap=None, bootstrap=None, *, skip, gamma, lam,
+                  values_filled=None, advantages=None, returns=None, want_returns=True, workspace=None, stream=None):
+    """GAE with observation-skip masking (skip != 0: masked, transparent step).  Returns
+    (advantages, returns = A + W, values_filled = W), or (advantages, values_filled) without returns."""
+    N, T = rewards.shape
+    fil = _out(rewards, values_filled)
+    adv = _out(rewards, advantages)
+    ret = (_out(rewards, returns) if want_returns else None)
+    wp, wb = _ws(workspace)
+    _check(lib().rlcs_gae_skip(_ptr(rewards, "f32"), _ptr(values, "f32", (N, T)), _ptr(dones, "u8", (N, T)),
+                               _ptr(truncs, "u8", (N, T)), _ptr(trunc_bootstrap, "f32", (N, T)),
+                               _ptr(bootstrap, "f32", (N,)), _ptr(skip, "u8", (N, T)), _ptr(fil, "f32", (N, T)),
+                               _ptr(adv, "f32", (N, T)), _ptr(ret, "f32", (N, T)), N, T, gamma, lam, wp, wb,
+                               _stream(stream)))
+    return (adv, ret, fil) if want_returns else (adv, fil)
 
 
 def rlcs_gae_no_alloc(rewards, values, dones, truncs=None, trunc_bootstrap=None, bootstrap=None, *, gamma, lam,

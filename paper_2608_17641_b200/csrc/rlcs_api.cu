@@ -78,6 +78,38 @@ int rlcs_gae(const float* rewards, const float* values, const uint8_t* dones, co
     return run(rlcs::launch_gae, p, variant, truncs != nullptr, vec, cuda_stream);
 }
 
+int rlcs_gae_skip(const float* rewards, const float* values, const uint8_t* dones, const uint8_t* truncs,
+                  const float* trunc_bootstrap, const float* bootstrap, const uint8_t* skip, float* values_filled,
+                  float* advantages, float* returns, int64_t N, int64_t T, float gamma, float lambda, void* workspace,
+                  size_t workspace_bytes, void* cuda_stream) {
+    ScanParams p = {};
+    Ptrs ps;
+    int64_t total;
+    bool vec;
+    if (!unit_interval(gamma) || !unit_interval(lambda)) return RLCS_ERR_ARG;
+    ps.add_f32(rewards); ps.add_f32(values); ps.add_f32(values_filled); ps.add_f32(advantages); ps.add_f32(returns);
+    ps.add_u8(skip);
+    int st = backward_common(p, ps, dones, truncs, trunc_bootstrap, bootstrap, N, T, &total, &vec);
+    if (st != RLCS_OK || total == 0) return st;
+    if (!rewards || !values || !skip || !values_filled || !advantages) return RLCS_ERR_NULL;
+    p.skip = skip;
+    p.gamma = gamma; p.decay = gamma * lambda;
+    // scan 1: W = the value each step shows to its predecessors (V, or what lies behind a masked step)
+    ScanParams f = p;
+    f.f0 = values; f.out0 = values_filled;
+    int variant = choose_variant(rlcs::kFillSkip, truncs != nullptr, total, T);
+    st = finish_params(f, variant, total, T, workspace, workspace_bytes, vec);
+    if (st != RLCS_OK) return st;
+    st = run(rlcs::launch_fill_skip, f, variant, truncs != nullptr, vec, cuda_stream);
+    if (st != RLCS_OK) return st;
+    // scan 2: GAE on (rewards, W) with the masked steps as identities
+    p.f0 = rewards; p.f1 = values_filled; p.out0 = advantages; p.out1 = returns;
+    variant = choose_variant(rlcs::kGaeSkip, truncs != nullptr, total, T);
+    st = finish_params(p, variant, total, T, workspace, workspace_bytes, vec);
+    if (st != RLCS_OK) return st;
+    return run(rlcs::launch_gae_skip, p, variant, truncs != nullptr, vec, cuda_stream);
+}
+
 // Layout of the workspace of rlcs_gae_normalized: the carry workspace of rlcs_workspace_bytes (rounded
 // up to 256 bytes), then {mean, 1/(std+eps)} in a 256-byte slot, then one {sum, sum of squares} pair per tile.
 static size_t norm_carry_bytes(int64_t N, int64_t T) { return (rlcs_workspace_bytes(N, T) + 255) / 256 * 256; }

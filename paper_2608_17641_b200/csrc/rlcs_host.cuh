@@ -75,7 +75,7 @@ int check_alignment(const Ptrs& ps, bool* vec) {
 // problems are bound by latency: smaller tiles spread them over more SMs, unless rows are long
 // enough for the inter-block carry to dominate.
 int choose_variant(int algo, bool trunc, int64_t total, int64_t T) {
-    if (g_variant >= 0 && RLCS_NS::variant_built(g_variant)) return g_variant;
+    if (g_variant >= 0 && RLCS_NS::variant_built_for(algo, g_variant)) return g_variant;
     if (total < (int64_t(1) << 23)) return T <= 2048 ? 6 : 0;
     if (RLCS_NS::kIoBf16) return 18;                      // 16 steps per thread: one 32-byte access per tensor
     switch (algo) {
@@ -85,6 +85,8 @@ int choose_variant(int algo, bool trunc, int64_t total, int64_t T) {
         case RLCS_NS::kRetrace: return 0;
         case RLCS_NS::kTdLambda: return trunc ? 17 : 0;
         case RLCS_NS::kDisc: return trunc ? 17 : 5;
+        case RLCS_NS::kFillSkip: return 18;
+        case RLCS_NS::kGaeSkip: return 0;
         case RLCS_NS::kElig: return 18;
         case RLCS_NS::kPrefix: return 18;
         default: return 0;

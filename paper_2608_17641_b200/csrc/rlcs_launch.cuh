@@ -34,6 +34,10 @@ constexpr TileVariant kVariants[kNumVariants] = {
 };
 // The bfloat16 build instantiates only these tile shapes (16 steps per thread = one 32-byte access).
 __host__ __device__ constexpr bool variant_built(int v) { return !kIoBf16 || v == 0 || v == 5 || v == 6 || v == 18; }
+// ... and the observation-skip scans only these (the rest of the table is tuning history of the seven kernels).
+__host__ __device__ constexpr bool variant_built_for(int algo, int v) {
+    return variant_built(v) && (!uses_skip(algo) || v == 0 || v == 6 || v == 18);
+}
 constexpr int kMinTileElems = 512;
 constexpr int kRetraceProbsThreads = 256, kRetraceProbsItems = 4;      // tile of rlcs_retrace_probs
 constexpr int kMaxDevices = 64;
@@ -112,7 +116,7 @@ cudaError_t launch_tv(const ScanParams& p, int variant, cudaStream_t stream) {
     if constexpr (V >= kNumVariants) {
         return cudaErrorInvalidValue;
     } else {
-        if constexpr (variant_built(V)) {
+        if constexpr (variant_built_for(ALGO, V)) {
             if (variant == V) return launch_variant<ALGO, TRUNC, VEC, V>(p, stream);
         }
         return launch_tv<ALGO, TRUNC, VEC, V + 1>(p, variant, stream);
@@ -141,6 +145,8 @@ cudaError_t launch_affine_bwd(const ScanParams&, int variant, bool trunc, bool v
 cudaError_t launch_affine_fwd(const ScanParams&, int variant, bool trunc, bool vec, cudaStream_t);
 cudaError_t launch_retrace_probs(const ScanParams&, bool trunc, bool vec, bool vec_rows, cudaStream_t);
 cudaError_t launch_gae_stats(const ScanParams&, int variant, bool trunc, bool vec, cudaStream_t);
+cudaError_t launch_fill_skip(const ScanParams&, int variant, bool trunc, bool vec, cudaStream_t);
+cudaError_t launch_gae_skip(const ScanParams&, int variant, bool trunc, bool vec, cudaStream_t);
 cudaError_t launch_norm_finalize(const float* partial, long long num_tiles, double count, int ddof, float eps,
                                  float* mean_rstd, cudaStream_t stream);
 cudaError_t launch_norm_rescale(float* adv, long long total, const float* mean_rstd, bool vec, cudaStream_t stream);

@@ -59,18 +59,22 @@ enum Algo : int {
     kGae = 0, kTdLambda = 1, kDisc = 2, kVtrace = 3, kRetrace = 4, kElig = 5, kPrefix = 6,
     kAffineBwd = 7, kAffineFwd = 8,
     kGaeStats = 9,    // GAE that also leaves per-tile sums of A and A^2 (for advantage normalisation)
-    kRetraceProbs = 10  // Retrace(lambda) from [N,T,A] Q-values and action probabilities
+    kRetraceProbs = 10, // Retrace(lambda) from [N,T,A] Q-values and action probabilities
+    // Observation-skip masking (Section 9.2): masked steps are transparent.  Two scans:
+    kFillSkip = 11,     // W_t = V_t at unmasked steps, the successor's W (or the flag's successor value) at masked ones
+    kGaeSkip = 12       // GAE on rewards and W with alpha_t = 0, beta_t = 1 at masked steps
 };
 
 __host__ __device__ constexpr bool is_forward(int a) { return a == kElig || a == kPrefix || a == kAffineFwd; }
-__host__ __device__ constexpr bool is_gae(int a) { return a == kGae || a == kGaeStats; }
+__host__ __device__ constexpr bool is_gae(int a) { return a == kGae || a == kGaeStats || a == kGaeSkip; }
+__host__ __device__ constexpr bool uses_skip(int a) { return a == kFillSkip || a == kGaeSkip; }
 __host__ __device__ constexpr bool has_values(int a) { return is_gae(a) || a == kTdLambda || a == kVtrace; }
 __host__ __device__ constexpr bool is_affine(int a) { return a == kAffineBwd || a == kAffineFwd; }
 __host__ __device__ constexpr bool is_retrace(int a) { return a == kRetrace || a == kRetraceProbs; }
-__host__ __device__ constexpr bool const_decay(int a) { return a != kVtrace && !is_retrace(a) && !is_affine(a); }
+__host__ __device__ constexpr bool const_decay(int a) { return a != kVtrace && !is_retrace(a) && !is_affine(a) && !uses_skip(a); }
 // a float input is read one step beyond the tile (successor value)
 __host__ __device__ constexpr bool float_halo(int a) { return has_values(a) || is_retrace(a); }
-__host__ __device__ constexpr bool uses_f1(int a) { return a != kDisc && a != kElig && a != kPrefix; }
+__host__ __device__ constexpr bool uses_f1(int a) { return a != kDisc && a != kElig && a != kPrefix && a != kFillSkip; }
 __host__ __device__ constexpr bool uses_f2(int a) { return a == kRetrace; }
 __host__ __device__ constexpr bool uses_f3(int a) { return a == kVtrace || a == kRetrace; }
 __host__ __device__ constexpr bool uses_dones(int a) { return !is_affine(a); }
@@ -96,6 +100,7 @@ struct ScanParams {
     int A;                    // kRetraceProbs: number of actions
     const uint8_t* dones;
     const uint8_t* truncs;
+    const uint8_t* skip;      // kFillSkip, kGaeSkip: non-zero = masked step
     const io_t* trunc_boot;   // [N,T]
     const io_t* boot;         // [N] or nullptr
     io_t* out0;
@@ -439,6 +444,7 @@ struct Chunk {
     unsigned edge;           // offset of the first row edge at or after the chunk start (see locate)
     int nvalid;              // steps of the chunk inside the array
     unsigned dw[W], tw[W];   // dones / truncs mask bytes
+    unsigned kw[uses_skip(ALGO) ? W : 1];   // skip mask bytes (observation-skip masking)
     unsigned halo_d;         // forward scans: dones byte of the step before the chunk
     float ov[ITEMS];         // successor value where the recurrence is severed (0 | trunc_bootstrap | bootstrap)
     float boot_first;        // window-edge bootstrap of the row whose edge lies in the chunk
@@ -499,6 +505,7 @@ __device__ __forceinline__ void load_flags_global(Chunk<ALGO, TRUNC, ITEMS>& c, 
     }
     if constexpr (uses_dones(ALGO)) load_mask<ITEMS, VEC>(p.dones, i0, nvalid, c.dw);
     if constexpr (TRUNC) load_mask<ITEMS, VEC>(p.truncs, i0, nvalid, c.tw);
+    if constexpr (uses_skip(ALGO)) load_mask<ITEMS, VEC>(p.skip, i0, nvalid, c.kw);
     if constexpr (ALGO == kElig || ALGO == kPrefix) {
         const unsigned nb = __shfl_up_sync(0xffffffffu, c.dw[W - 1] >> 24, 1);
         if (lane != 0) c.halo_d = nb;
@@ -783,7 +790,18 @@ __device__ __forceinline__ void tile_compute(Chunk<ALGO, TRUNC, ITEMS>& c, Vals<
             if constexpr (has_values(ALGO)) nextv = (j + 1 < ITEMS) ? v.x1[(j + 1) % ITEMS] : v.halo;
             if constexpr (is_retrace(ALGO)) nextv = (j + 1 < ITEMS) ? v.x2[(j + 1) % ITEMS] : v.halo;
             const float xn = cut ? c.ov[j] : nextv;      // successor value of Section 3.2 (selected, never multiplied)
-            if constexpr (is_gae(ALGO)) {
+            if constexpr (ALGO == kFillSkip) {
+                // an unmasked step starts a new run with its own value; a masked one passes its
+                // successor's through, or takes the flag's successor value where it is severed
+                const bool masked = test_byte(c.kw, j);
+                v.a[j] = masked ? (cut ? c.ov[j] : 0.f) : r;
+                beta[j] = (masked && !cut) ? 1.f : 0.f;
+            } else if constexpr (ALGO == kGaeSkip) {
+                // x1 holds W (kFillSkip's output): V at unmasked steps, so delta is the usual one
+                const bool masked = test_byte(c.kw, j);
+                v.a[j] = masked ? 0.f : fmaf(p.gamma, xn, r) - v.x1[j];
+                beta[j] = cut ? 0.f : (masked ? 1.f : p.decay);
+            } else if constexpr (is_gae(ALGO)) {
                 v.a[j] = fmaf(p.gamma, xn, r) - v.x1[j];
                 beta[j] = cut ? 0.f : p.decay;
             } else if constexpr (ALGO == kTdLambda) {

@@ -524,6 +524,89 @@ def test_per_dimension_beta_argument_checks(oracle, W, B):
     assert L.rlcs_elig_trace_vec_beta(P, P, P, P, 2, 100000, 8, None, 0, None) == B.RLCS_ERR_WORKSPACE
 
 
+# ------------------------------------------------------------------ observation-skip masking
+def _skip_case(W, N, T, p_skip, p_flag, salt=0):
+    ro = W.make_rollout(130, N, T, p_done=p_flag, p_trunc=p_flag / 2, salt=salt + T)
+    rng = np.random.default_rng(N * 31 + T + salt)
+    skip = (rng.random((N, T)) < p_skip).astype(np.uint8)
+    # observation tokens come in runs: lengthen every masked step into a short span
+    for k in (1, 2):
+        skip[:, k:] |= skip[:, :-k] & (rng.random((N, T - k)) < 0.6).astype(np.uint8) if T > k else 0
+    return ro, skip
+
+
+@pytest.mark.parametrize("N,T", [(1, 1), (3, 7), (5, 1001), (64, 512), (4096, 64), (7, 5000), (2, 40000), (4, 2048)])
+@pytest.mark.parametrize("p_skip,p_flag", [(0.0, 0.02), (0.2, 0.0), (0.2, 0.02), (0.9, 0.05), (1.0, 0.0)])
+def test_gae_with_observation_skip_masking(oracle, W, B, N, T, p_skip, p_flag):
+    """Flags may sit on masked steps as well: the oracle defines that case too."""
+    import torch
+    ro, skip = _skip_case(W, N, T, p_skip, p_flag)
+    p = ro.params
+    dev = Dev(ro)
+    sk = torch.from_numpy(skip).cuda()
+    ws = B.Workspace(N, T)
+    adv, ret, fil = B.rlcs_gae_skip(dev.rewards, dev.values, dev.dones, dev.truncs, dev.trunc_bootstrap, dev.bootstrap,
+                                    skip=sk, gamma=p["gamma"], lam=p["lam"], workspace=ws)
+    torch.cuda.synchronize()
+    assert ws.device_status() == 0
+    ra, rr, rf = oracle.gae_skip(ro.rewards, ro.values, ro.dones, ro.truncs, ro.trunc_bootstrap, ro.bootstrap, skip=skip,
+                                 gamma=p["gamma"], lam=p["lam"])
+    assert np.array_equal(fil.cpu().numpy().astype(np.float64), rf)          # W is copied, never computed
+    assert_close("skip adv", adv.cpu().numpy(), ra)
+    assert_close("skip ret", ret.cpu().numpy(), rr)
+    if p_skip == 0.0:                                                        # nothing masked: rlcs_gae, bit for bit on the same tile shape
+        B.rlcs_debug_set_tile_variant(0)
+        try:
+            a0, _ = B.rlcs_gae(dev.rewards, dev.values, dev.dones, dev.truncs, dev.trunc_bootstrap, dev.bootstrap,
+                               gamma=p["gamma"], lam=p["lam"], workspace=ws)
+            a1, _, _ = B.rlcs_gae_skip(dev.rewards, dev.values, dev.dones, dev.truncs, dev.trunc_bootstrap, dev.bootstrap,
+                                       skip=sk, gamma=p["gamma"], lam=p["lam"], workspace=ws)
+        finally:
+            B.rlcs_debug_set_tile_variant(BASE_VARIANT)
+        assert torch.equal(a0, a1)
+
+
+def test_gae_skip_options_alignment_and_large_problem(oracle, W, B):
+    import torch
+    # no truncation tensors, no bootstrap, no returns; pointers off 16-byte alignment
+    ro, skip = _skip_case(W, 6, 900, 0.3, 0.03, salt=1)
+    p = ro.params
+    for offset in (0, 1):
+        dev = Dev(ro, offset=offset)
+        flat = torch.zeros(skip.size + offset, dtype=torch.uint8, device="cuda")
+        sk = flat[offset:].view(skip.shape)
+        sk.copy_(torch.from_numpy(skip))
+        adv, fil = B.rlcs_gae_skip(dev.rewards, dev.values, dev.dones, skip=sk, gamma=p["gamma"], lam=p["lam"],
+                                   values_filled=dev.empty_out(), advantages=dev.empty_out(), want_returns=False,
+                                   workspace=B.Workspace(ro.N, ro.T))
+        ra, _, rf = oracle.gae_skip(ro.rewards, ro.values, ro.dones, skip=skip, gamma=p["gamma"], lam=p["lam"])
+        assert_close(f"skip adv, offset {offset}", adv.cpu().numpy(), ra)
+        assert np.array_equal(fil.cpu().numpy().astype(np.float64), rf)
+    # above 2^23 steps (per-algorithm tile shapes), rows straddling tiles: look-back carries both scans
+    ro, skip = _skip_case(W, 2900, 3000, 0.3, 0.002, salt=2)
+    p = ro.params
+    dev = Dev(ro)
+    ws = B.Workspace(ro.N, ro.T)
+    adv, ret, fil = B.rlcs_gae_skip(dev.rewards, dev.values, dev.dones, dev.truncs, dev.trunc_bootstrap, dev.bootstrap,
+                                    skip=torch.from_numpy(skip).cuda(), gamma=p["gamma"], lam=p["lam"], workspace=ws)
+    ra, rr, rf = oracle.run_rows_parallel(
+        lambda **k: oracle.gae_skip(k["rewards"], k["values"], k["dones"], k["truncs"], k["trunc_bootstrap"], k["bootstrap"],
+                                    skip=k["skip"], gamma=p["gamma"], lam=p["lam"]),
+        dict(rewards=ro.rewards, values=ro.values, dones=ro.dones, truncs=ro.truncs, trunc_bootstrap=ro.trunc_bootstrap,
+             skip=skip), dict(bootstrap=ro.bootstrap), 8)
+    assert ws.device_status() == 0
+    assert_close("skip adv, large", adv.cpu().numpy(), ra)
+    assert_close("skip ret, large", ret.cpu().numpy(), rr)
+    assert np.array_equal(fil.cpu().numpy().astype(np.float64), rf)
+    # argument checks
+    L = B.lib()
+    P = 0x7f0000000000
+    g = lambda **k: L.rlcs_gae_skip(P, P, P, None, None, None, k.get("sk", P), k.get("fil", P), P, None, k.get("N", 4), 128,
+                                    k.get("g", 0.9), 0.9, None, 0, None)
+    assert g(N=0) == B.RLCS_OK and g(sk=None) == B.RLCS_ERR_NULL and g(fil=None) == B.RLCS_ERR_NULL
+    assert g(g=1.5) == B.RLCS_ERR_ARG and g(fil=P + 2) == B.RLCS_ERR_ALIGN
+
+
 # ------------------------------------------------------------------ time-major [T, N] entry points
 def _tm(a):
     import torch
