@@ -149,3 +149,39 @@ def test_missing_library_fails_loudly(tmp_path, monkeypatch):
     monkeypatch.setattr(binding, "LIB_PATH", str(tmp_path / "nope.so"))
     with pytest.raises(RuntimeError, match="no fallback"):
         binding.lib()
+
+
+# ------------------------------------------------------------------ the entry points beyond the paper's API
+def test_time_major_validation_and_workspace_plan(L):
+    tm = lambda **k: L.rlcs_gae_time_major(k.get("r", P), P, k.get("d", P), k.get("tr"), k.get("bv"), None, P, None,
+                                           k.get("N", 4), k.get("T", 8), k.get("g", 0.9), 0.9, None, 0, None)
+    assert tm(N=0) == OK and tm(N=-1) == E_SIZE and tm(T=2 ** 31) == E_SIZE and tm(g=2.0) == E_ARG
+    assert tm(r=None) == E_NULL and tm(d=None) == E_NULL and tm(tr=P) == E_NULL and tm(r=ODD) == E_ALIGN
+    # enough environments: whole columns, no workspace; few environments: the time axis is cut
+    assert L.rlcs_time_major_workspace_bytes(100000, 64) == 0 and L.rlcs_time_major_workspace_bytes(3072, 5000) == 0
+    need = L.rlcs_time_major_workspace_bytes(8, 4096)
+    assert need > 0 and need % (2 * 4 * 8) == 0            # two floats per chunk and environment
+    assert L.rlcs_time_major_workspace_bytes(8, 40) == 0   # chunks are at least 64 steps
+    assert tm(N=8, T=4096) == E_WS
+    assert L.rlcs_elig_trace_time_major(None, P, P, 4, 8, 0.9, 0.9, None, 0, None) == E_NULL
+    assert L.rlcs_episodic_prefix_sum_time_major(P, P, P, 0, 8, 0, None, 0, None) == OK
+
+
+def test_bf16_validation(L):
+    g = lambda **k: L.rlcs_gae_bf16(k.get("r", P), P, P, k.get("tr"), None, None, P, None, k.get("N", 4), k.get("T", 128),
+                                    k.get("g", 0.9), 0.9, None, 0, None)
+    assert g(N=0) == OK and g(N=-1) == E_SIZE and g(g=-0.1) == E_ARG and g(r=None) == E_NULL and g(tr=P) == E_NULL
+    assert g(r=P + 1) == E_ALIGN and g(N=3, T=3000) == E_WS
+    assert L.rlcs_retrace_bf16(P, P, None, P, P, None, None, None, P, 4, 128, 0.9, 0.9, 1.0, None, 0, None) == E_NULL
+    assert L.rlcs_vtrace_bf16(P, P, P, P, None, None, None, P, None, 4, 128, 0.9, -1.0, 1.0, None, 0, None) == E_ARG
+
+
+def test_vector_trace_and_skip_validation(L):
+    assert L.rlcs_elig_trace_vec_beta(P, P, P, P, 4, 8, 0, None, 0, None) == OK
+    assert L.rlcs_elig_trace_vec_beta(P, None, P, P, 4, 8, 4, None, 0, None) == E_NULL
+    assert L.rlcs_elig_trace_vec_beta(P, ODD, P, P, 4, 8, 4, None, 0, None) == E_ALIGN
+    assert L.rlcs_elig_trace_vec_beta_workspace_bytes(2, 100000, 8) > L.rlcs_elig_trace_vec_workspace_bytes(2, 100000, 8) > 0
+    assert L.rlcs_elig_trace_vec_beta(P, P, P, P, 2, 100000, 8, None, 0, None) == E_WS
+    sk = lambda **k: L.rlcs_gae_skip(P, P, P, None, None, None, k.get("sk", P), k.get("fil", P), P, None, k.get("N", 4), 128,
+                                     k.get("g", 0.9), 0.9, None, 0, None)
+    assert sk(N=0) == OK and sk(sk=None) == E_NULL and sk(fil=None) == E_NULL and sk(g=1.5) == E_ARG and sk(fil=ODD) == E_ALIGN
