@@ -77,14 +77,24 @@ int check_alignment(const Ptrs& ps, bool* vec) {
 int choose_variant(int algo, bool trunc, int64_t total, int64_t T) {
     if (g_variant >= 0 && RLCS_NS::variant_built_for(algo, g_variant)) return g_variant;
     if (total < (int64_t(1) << 23)) return T <= 2048 ? 6 : 0;
-    if (RLCS_NS::kIoBf16) return 18;                      // 16 steps per thread: one 32-byte access per tensor
+    if (RLCS_NS::kIoBf16) {
+        // 16 steps per thread (one 32-byte access per tensor); with half the bytes per step the kernels
+        // are bound by issue slots and latency, and more resident blocks pay even with a few spills
+        if (!trunc) return 18;
+        switch (algo) {
+            case RLCS_NS::kGae:
+            case RLCS_NS::kTdLambda:
+            case RLCS_NS::kDisc: return 20;
+            default: return 19;
+        }
+    }
     switch (algo) {
-        case RLCS_NS::kGae:
+        case RLCS_NS::kGae: return trunc ? 19 : 0;
         case RLCS_NS::kGaeStats: return trunc ? 16 : 0;
         case RLCS_NS::kVtrace: return trunc ? 18 : 0;
         case RLCS_NS::kRetrace: return 0;
-        case RLCS_NS::kTdLambda: return trunc ? 17 : 0;
-        case RLCS_NS::kDisc: return trunc ? 17 : 5;
+        case RLCS_NS::kTdLambda: return trunc ? 20 : 0;
+        case RLCS_NS::kDisc: return trunc ? 20 : 5;
         case RLCS_NS::kFillSkip: return 18;
         case RLCS_NS::kGaeSkip: return 0;
         case RLCS_NS::kElig: return 18;

@@ -10,7 +10,7 @@ namespace RLCS_NS {
 // stages == 0: scan_kernel (one tile per block).  stages > 0: scan_kernel_tma (persistent blocks,
 // bulk-copy ring of that many tiles; min_blocks = blocks per SM it is compiled and sized for).
 struct TileVariant { int threads, items, min_blocks, stages; };
-constexpr int kNumVariants = 19;
+constexpr int kNumVariants = 21;
 constexpr TileVariant kVariants[kNumVariants] = {
     {256, 8, 4, 0},    //  0: 2048 steps per tile
     {128, 4, 8, 0},    //  1:  512
@@ -31,9 +31,11 @@ constexpr TileVariant kVariants[kNumVariants] = {
     {256, 8, 5, 0},    // 16: 2048, at most 48 registers
     {256, 8, 6, 0},    // 17: 2048, at most 40 registers
     {128, 16, 5, 0},   // 18: 2048, 16 steps per thread
+    {128, 16, 6, 0},   // 19: 2048, 16 steps per thread, at most 80 registers
+    {128, 16, 8, 0},   // 20: 2048, 16 steps per thread, at most 64 registers
 };
 // The bfloat16 build instantiates only these tile shapes (16 steps per thread = one 32-byte access).
-__host__ __device__ constexpr bool variant_built(int v) { return !kIoBf16 || v == 0 || v == 5 || v == 6 || v == 18; }
+__host__ __device__ constexpr bool variant_built(int v) { return !kIoBf16 || v == 0 || v == 5 || v == 6 || v >= 18; }
 // ... and the observation-skip scans only these (the rest of the table is tuning history of the seven kernels).
 __host__ __device__ constexpr bool variant_built_for(int algo, int v) {
     return variant_built(v) && (!uses_skip(algo) || v == 0 || v == 6 || v == 18);

@@ -82,7 +82,7 @@ def test_shape_matrix(oracle, W, B, N, T, p_flag):
     compare_all(oracle, ro)
 
 
-@pytest.mark.parametrize("variant", list(range(19)))
+@pytest.mark.parametrize("variant", list(range(21)))
 @pytest.mark.parametrize("N,T", [(5, 700), (4097, 3), (2, 9000), (64, 513)])
 def test_tile_variants(oracle, W, B, variant, N, T):
     B.rlcs_debug_set_tile_variant(variant)
@@ -109,7 +109,7 @@ def test_long_row_without_resets_multi_window_lookback(oracle, W, B):
 def test_randomized_shapes_flags_and_options(oracle, W, B):
     """Seeded fuzz over shapes, flag densities, kernel variants, pointer offsets and NULL options."""
     rng = np.random.default_rng(20260817)
-    n_variants = 19
+    n_variants = 21
     for case in range(60):
         N = int(rng.integers(1, 200))
         T = int(rng.choice([rng.integers(1, 40), rng.integers(40, 3000), rng.integers(3000, 12000)]))
