@@ -90,13 +90,13 @@ int choose_variant(int algo, bool trunc, int64_t total, int64_t T) {
     }
     switch (algo) {
         case RLCS_NS::kGae: return trunc ? 19 : 0;
-        case RLCS_NS::kGaeStats: return trunc ? 16 : 0;
+        case RLCS_NS::kGaeStats: return trunc ? 19 : 0;
         case RLCS_NS::kVtrace: return trunc ? 18 : 0;
         case RLCS_NS::kRetrace: return 0;
         case RLCS_NS::kTdLambda: return trunc ? 20 : 0;
         case RLCS_NS::kDisc: return trunc ? 20 : 5;
-        case RLCS_NS::kFillSkip: return 18;
-        case RLCS_NS::kGaeSkip: return 0;
+        case RLCS_NS::kFillSkip: return 20;
+        case RLCS_NS::kGaeSkip: return 20;
         case RLCS_NS::kElig: return 18;
         case RLCS_NS::kPrefix: return 18;
         default: return 0;

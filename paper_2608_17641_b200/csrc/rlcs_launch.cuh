@@ -38,7 +38,7 @@ constexpr TileVariant kVariants[kNumVariants] = {
 __host__ __device__ constexpr bool variant_built(int v) { return !kIoBf16 || v == 0 || v == 5 || v == 6 || v >= 18; }
 // ... and the observation-skip scans only these (the rest of the table is tuning history of the seven kernels).
 __host__ __device__ constexpr bool variant_built_for(int algo, int v) {
-    return variant_built(v) && (!uses_skip(algo) || v == 0 || v == 6 || v == 18);
+    return variant_built(v) && (!uses_skip(algo) || v == 0 || v == 6 || v >= 18);
 }
 constexpr int kMinTileElems = 512;
 constexpr int kRetraceProbsThreads = 256, kRetraceProbsItems = 4;      // tile of rlcs_retrace_probs
