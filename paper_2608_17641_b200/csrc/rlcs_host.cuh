@@ -76,7 +76,12 @@ int check_alignment(const Ptrs& ps, bool* vec) {
 // enough for the inter-block carry to dominate.
 int choose_variant(int algo, bool trunc, int64_t total, int64_t T) {
     if (g_variant >= 0 && RLCS_NS::variant_built_for(algo, g_variant)) return g_variant;
-    if (total < (int64_t(1) << 23)) return T <= 2048 ? 6 : 0;
+    if (total < (int64_t(1) << 23)) {
+        // latency-bound sizes (cold-L2 sweeps): long rows want few carry hops (2048-step tiles, one
+        // cluster per row where that fits), the smallest problems want many small blocks
+        if (T > 2048) return 19;
+        return (total <= (int64_t(1) << 19) && RLCS_NS::variant_built_for(algo, 1)) ? 1 : 6;
+    }
     if (RLCS_NS::kIoBf16) {
         // 16 steps per thread (one 32-byte access per tensor); with half the bytes per step the kernels
         // are bound by issue slots and latency, and more resident blocks pay even with a few spills
