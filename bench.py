@@ -36,8 +36,8 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch on the bench workload, from the committed
 # one-pass ncu capture of the full-size run (summarised under profiles/).
 NCU_TRAFFIC_BYTES = {
-    "gae": 576827904, "vtrace": 715524096, "retrace": 738515712, "td_lambda": 456696832,
-    "discounted_return": 312028672, "elig_trace": 255066880, "episodic_prefix_sum": 251662080,
+    "gae": 575476736, "vtrace": 715139072, "retrace": 738443008, "td_lambda": 456630784,
+    "discounted_return": 310968064, "elig_trace": 255497472, "episodic_prefix_sum": 251432448,
 }
 
 
