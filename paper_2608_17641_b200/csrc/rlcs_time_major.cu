@@ -40,7 +40,7 @@ using rlcs::kRetrace;
 using rlcs::kElig;
 using rlcs::kPrefix;
 
-constexpr int kRows = 8;         // timesteps per register block of tm_kernel; upper bound of tm_rows()
+constexpr int kRows = 8;         // timesteps per register block of tm_kernel
 constexpr int kThreads = 128;    // register-path block; the staged path uses 32 * warps_per_block
 
 struct TmParams {
@@ -71,8 +71,9 @@ __host__ __device__ constexpr int tm_nf(int a) {
 }
 // timesteps per warp and stage in tm_block_kernel: fewer for Retrace, whose four float inputs make a
 // row 576 bytes (measured: 0.84 -> 0.90 of the copy bandwidth with 4, while the lighter algorithms
-// lose 5-12 % to the doubled per-stage overhead)
-__host__ __device__ constexpr int tm_rows(int a) { return a == kRetrace ? 4 : 8; }
+// lose 5-12 % to the doubled per-stage overhead); more for the discounted return, whose rows are
+// 160-192 bytes (0.52 -> 0.63 at 16384 environments with 16; the forward scans lose 1 % that way)
+__host__ __device__ constexpr int tm_rows(int a) { return a == kRetrace ? 4 : a == kDisc ? 16 : 8; }
 __host__ __device__ constexpr int tm_row_bytes(int a, bool trunc) { return tm_nf(a) * 128 + (trunc ? 2 : 1) * 32; }
 
 // all ones where x != 0, else 0; written in PTX so that the flag reaches the arithmetic below as a
