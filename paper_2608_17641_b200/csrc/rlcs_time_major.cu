@@ -384,7 +384,6 @@ __device__ __forceinline__ void cp_async_wait(int pending) {
 }
 
 constexpr int kMaxStages = 16;
-constexpr int kMaxWarps = 8;
 
 // One stage of a thread block: R = KR * warps rows (KR = tm_rows(ALGO) timesteps per warp) of its 32 C columns (C columns per lane), row
 // index = scan-order step within the stage.  Floats and masks live in separate rings (the mask ring
@@ -798,15 +797,15 @@ void plan_chunks(long long N, long long T, unsigned* chunk, unsigned* chunks) {
 }
 
 // Columns per lane, warps per block and ring depth for tm_block_kernel.  Two columns per lane when
-// that still leaves two blocks per SM (and the outputs allow 8-byte stores); eight warps when blocks
-// are scarce, else four.  The kernel is bound by issue slots and dependent-ALU latency as much as by
+// that still leaves two blocks per SM (and the outputs allow 8-byte stores); sixteen or eight warps when blocks
+// are scarce (fewer than one or two per SM), else four.  The kernel is bound by issue slots and dependent-ALU latency as much as by
 // HBM, so resident warps come first: the ring is as deep as still lets min(blocks per SM, 6) blocks
 // share an SM, no deeper than keeps about 16 MB in flight over the grid, and at least 3.
 size_t plan_block(TmParams& p, int rows, int row_bytes, bool trunc, bool wide_ok) {
     int C = 1;
     if (wide_ok && (p.N + 63) / 64 * p.chunks >= 2 * kSms) C = 2;
     const long long blocks = (p.N + 32 * C - 1) / (32 * C) * p.chunks;
-    const int W = (C == 1 && blocks < 2 * kSms) ? 8 : 4;
+    const int W = C == 2 ? 4 : blocks < kSms ? 16 : blocks < 2 * kSms ? 8 : 4;
     const long long stage = (long long)rows * W * row_bytes * C;
     const long long mstage = (long long)rows * W * (trunc ? 64 : 32) * C;
     const long long fixed = 2 * mstage + (W * 512 + 512) * C;   // mask ring's two extra slots, aggregates, edges
@@ -866,6 +865,7 @@ int launch(TmParams p, bool staged, cudaStream_t s) {
         if constexpr (kWide) {
             if (p.cols_per_lane == 2) return launch_block<ALGO, TRUNC, 4, 2>(p, smem, s);
         }
+        if (p.warps_per_block == 16) return launch_block<ALGO, TRUNC, 16, 1>(p, smem, s);
         return p.warps_per_block == 8 ? launch_block<ALGO, TRUNC, 8, 1>(p, smem, s) : launch_block<ALGO, TRUNC, 4, 1>(p, smem, s);
     } else {
         const dim3 grid(gx_chain, p.chunks);
