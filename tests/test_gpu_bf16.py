@@ -198,6 +198,28 @@ def test_bf16_equals_rounded_fp32_bit_for_bit(oracle, W, B, variant):
         assert torch.equal(g.view(torch.int16), r.to(torch.bfloat16).view(torch.int16)), name
 
 
+def test_bf16_randomized_shapes_flags_variants_and_options(oracle, W, B):
+    rng = np.random.default_rng(20260819)
+    for case in range(40):
+        N = int(rng.integers(1, 200))
+        T = int(rng.choice([rng.integers(1, 40), rng.integers(40, 3000), rng.integers(3000, 12000)]))
+        if N * T > 600_000:
+            N = max(1, 600_000 // T)
+        ro = W.make_rollout(126, N, T, p_done=float(rng.choice([0.0, 0.001, 0.02, 0.3])),
+                            p_trunc=float(rng.choice([0.0, 0.005, 0.2])), salt=case)
+        ro.params.update(gamma=float(rng.choice([0.9, 0.99, 1.0])), lam=float(rng.choice([0.0, 0.5, 0.95, 1.0])),
+                         rho_bar=float(rng.choice([0.5, 1.0, 2.0])), c_bar=float(rng.choice([0.5, 1.0])))
+        variant = int(rng.choice((-1,) + BUILT_VARIANTS))
+        B.rlcs_debug_set_tile_variant(variant)
+        try:
+            compare16(oracle, B, ro, offset=int(rng.choice([0, 0, 0, 1, 3, 16])),
+                      use_truncs=bool(rng.random() < 0.7), use_bootstrap=bool(rng.random() < 0.8))
+        except AssertionError as e:
+            raise AssertionError(f"case {case}: N={N} T={T} variant={variant}: {e}")
+        finally:
+            B.rlcs_debug_set_tile_variant(-1)
+
+
 def test_bf16_argument_checks(B):
     L = B.lib()
     P = 0x7f0000000000

@@ -714,6 +714,63 @@ def test_time_major_argument_checks(oracle, W, B):
     assert g(N=8, T=4096) == B.RLCS_ERR_WORKSPACE
 
 
+def test_randomized_time_major_and_skip(oracle, W, B):
+    """Seeded fuzz of the entry points beyond the paper's API: time-major (both kernels, every warp
+    count and chunking the planner picks), GAE with observation-skip masking."""
+    import torch
+    rng = np.random.default_rng(20260818)
+    for case in range(40):
+        N = int(rng.choice([rng.integers(1, 64), 16 * rng.integers(1, 40), 16 * rng.integers(200, 1300)]))
+        T = int(rng.choice([rng.integers(1, 40), rng.integers(40, 700), rng.integers(700, 5000)]))
+        if N * T > 1_500_000:
+            T = max(1, 1_500_000 // N)
+        p_done = float(rng.choice([0.0, 0.01, 0.3]))
+        ro = W.make_rollout(131, N, T, p_done=p_done, p_trunc=float(rng.choice([0.0, 0.01, 0.2])), salt=case)
+        ro.params.update(gamma=float(rng.choice([0.9, 0.99, 1.0])), lam=float(rng.choice([0.0, 0.5, 0.95, 1.0])))
+        p = ro.params
+        use_tr, use_bt = bool(rng.random() < 0.7), bool(rng.random() < 0.8)
+        ref = run_oracle(oracle, ro, ALL_ALGOS, use_truncs=use_tr, use_bootstrap=use_bt)
+        tm = lambda a: None if a is None else _tm(a)
+        r, v, d, q, eq, lr, x, dany = (tm(getattr(ro, k)) for k in ("rewards", "values", "dones", "q_sa", "expected_q", "log_rhos", "x", "any_done"))
+        tr, bv = (tm(ro.truncs), tm(ro.trunc_bootstrap)) if use_tr else (None, None)
+        bt = torch.from_numpy(ro.bootstrap).cuda() if use_bt else None
+        back = lambda t: np.ascontiguousarray(t.cpu().numpy().T)
+        path = int(rng.choice([0, 1, 3]))
+        B.rlcs_debug_time_major_path(path)
+        try:
+            adv, ret = B.rlcs_gae_time_major(r, v, d, tr, bv, bt, gamma=p["gamma"], lam=p["lam"])
+            vs, pg = B.rlcs_vtrace_time_major(r, v, lr, d, tr, bv, bt, gamma=p["gamma"], rho_bar=p["rho_bar"], c_bar=p["c_bar"])
+            qt = B.rlcs_retrace_time_major(r, q, eq, lr, d, tr, bv, bt, gamma=p["gamma"], lam=p["lam"], c_bar=p["c_bar"])
+            td = B.rlcs_td_lambda_time_major(r, v, d, tr, bv, bt, gamma=p["gamma"], lam=p["lam"])
+            dr = B.rlcs_discounted_return_time_major(r, d, tr, bv, bt, gamma=p["gamma"])
+            el = B.rlcs_elig_trace_time_major(x, dany, gamma=p["gamma"], lam=p["lam"])
+            ps = B.rlcs_episodic_prefix_sum_time_major(x, dany, starts_at=bool(case % 2))
+        finally:
+            B.rlcs_debug_time_major_path(0)
+        tag = f"case {case}: N={N} T={T} path={path} truncs={use_tr} boot={use_bt}"
+        for name, got, want in (("gae", adv, ref["gae"][0]), ("ret", ret, ref["gae"][1]), ("vs", vs, ref["vtrace"][0]),
+                                ("pg", pg, ref["vtrace"][1]), ("retrace", qt, ref["retrace"]), ("td", td, ref["td_lambda"]),
+                                ("disc", dr, ref["discounted_return"]), ("elig", el, ref["elig_trace"]),
+                                ("prefix", ps, ref["prefix_starts_at" if case % 2 else "prefix_ends_at"])):
+            assert_close(f"{tag} {name}", back(got), want)
+        # observation-skip masking on the same rollout (row-major)
+        skip = (rng.random((N, T)) < float(rng.choice([0.0, 0.3, 0.8]))).astype(np.uint8)
+        dev = Dev(ro, offset=int(rng.choice([0, 0, 1])))
+        flat = torch.zeros(skip.size + dev.offset, dtype=torch.uint8, device="cuda")
+        sk = flat[dev.offset:].view(skip.shape)
+        sk.copy_(torch.from_numpy(skip))
+        a, rt, fil = B.rlcs_gae_skip(dev.rewards, dev.values, dev.dones, dev.truncs if use_tr else None,
+                                     dev.trunc_bootstrap if use_tr else None, dev.bootstrap if use_bt else None, skip=sk,
+                                     gamma=p["gamma"], lam=p["lam"], values_filled=dev.empty_out(), advantages=dev.empty_out(),
+                                     returns=dev.empty_out(), workspace=B.Workspace(N, T))
+        ra, rr, rf = oracle.gae_skip(ro.rewards, ro.values, ro.dones, ro.truncs if use_tr else None,
+                                     ro.trunc_bootstrap if use_tr else None, ro.bootstrap if use_bt else None, skip=skip,
+                                     gamma=p["gamma"], lam=p["lam"])
+        assert_close(f"{tag} skip adv", a.cpu().numpy(), ra)
+        assert_close(f"{tag} skip ret", rt.cpu().numpy(), rr)
+        assert np.array_equal(fil.cpu().numpy().astype(np.float64), rf), tag
+
+
 # ------------------------------------------------------------------ test hooks
 def test_affine_scan_matches_generic_recurrence(oracle, W, B):
     import torch
