@@ -619,11 +619,45 @@ def sweep_case(torch, B, ro, algo: str, use_truncs: bool, hbm_peak: float, l2_by
         full_call_us.append(1e3 * e0.elapsed_time(e1) / R)
     best = min(per_call_us)
     gbs = algo_bytes / (best * 1e-6) / 1e9
+    del sets, graph
+    ceiling_us = copy_ceiling_us(torch, B, ro_eff, algo, algo_bytes, R, trials)
+    ceiling_gbs = algo_bytes / (ceiling_us * 1e-6) / 1e9
     return {"algo": algo, "N": ro.N, "T": ro.T, "truncs": use_truncs, "us_per_call": round(best, 3),
+            "copy_ceiling_us": round(ceiling_us, 3), "copy_ceiling_gbs": round(ceiling_gbs, 1),
+            "frac_of_copy_ceiling": round(gbs / ceiling_gbs, 4),
             "us_per_call_median": round(statistics.median(per_call_us), 3),
             "full_call_us": round(min(full_call_us), 3), "env_steps_per_s": ro.N * ro.T / (best * 1e-6),
             "algorithmic_bytes": algo_bytes, "gbs": round(gbs, 1), "frac_of_peak": round(gbs / hbm_peak, 4),
             "rotating_sets": R, "l2": "cold (rotating buffer sets > 3x L2)", "timing": "CUDA-graph replay of the rotating launches"}
+
+
+def copy_ceiling_us(torch, B, ro, algo: str, algo_bytes: int, R: int, trials: int) -> float:
+    """Device time of a plain streaming kernel at the same byte count, read:write ratio and cold-L2
+    rotation as one scan launch of this case: what the size itself allows."""
+    S = ro.N * ro.T
+    write_bytes = 4 * S * {"gae": 2, "vtrace": 2}.get(algo, 1)
+    read_bytes = max(32, algo_bytes - write_bytes)
+    rd = [torch.empty(read_bytes // 4 + 8, dtype=torch.float32, device="cuda").normal_() for _ in range(R)]
+    wr = [torch.empty(write_bytes // 4 + 8, dtype=torch.float32, device="cuda") for _ in range(R)]
+    call = lambda i: B.rlcs_debug_stream_copy(rd[i], wr[i], read_bytes, write_bytes)
+    for i in range(R):
+        call(i)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        for i in range(R):
+            call(i)
+    graph.replay()
+    times = []
+    for _ in range(trials):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        graph.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        times.append(1e3 * e0.elapsed_time(e1) / R)
+    return min(times)
 
 
 def _without_truncs(ro):

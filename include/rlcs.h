@@ -418,6 +418,15 @@ int rlcs_debug_set_carry_fault(int64_t mute_tile, int64_t spin_cap);
  */
 void rlcs_debug_time_major_path(int path);
 
+/*
+ * Measurement hook: a streaming kernel that reads read_bytes from src and writes write_bytes to dst
+ * (whole 32-byte pieces; both pointers 32-byte aligned, buffers at least that large; dst[0] may be
+ * written when write_bytes is 0), with the scan kernels' load / store instructions and one piece
+ * per thread.  bench.py times it at a scan launch's byte count and read:write ratio to report the
+ * bandwidth ceiling of that size next to the scan's own figure.
+ */
+int rlcs_debug_stream_copy(const float* src, float* dst, size_t read_bytes, size_t write_bytes, void* cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

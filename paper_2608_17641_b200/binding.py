@@ -63,6 +63,7 @@ SIGNATURES = {
     "rlcs_debug_tile_elems": ([_int], _int),
     "rlcs_debug_set_carry_fault": ([_i64, _i64], _int),
     "rlcs_debug_time_major_path": ([_int], None),
+    "rlcs_debug_stream_copy": ([_vp, _vp, _sz, _sz, _vp], _int),
     "rlcs_debug_force_wide_index": ([_int], _int),
     "rlcs_debug_allow_cluster_carry": ([_int], _int),
     "rlcs_debug_variant_for": ([_int, _int, _i64, _i64], _int),
@@ -143,6 +144,8 @@ class Workspace:
         self.nbytes = int(lib().rlcs_workspace_bytes(N, T)) if nbytes is None else int(nbytes)
         self.buf = torch.empty(max(self.nbytes, 16), dtype=torch.uint8, device=device) if self.nbytes else None
         if self.buf is not None:
+            if stream is not None:
+                self.buf.record_stream(stream)     # the caching allocator must not hand it out again before that stream is done
             _check(lib().rlcs_workspace_init(self.buf.data_ptr(), self.nbytes, _stream(stream)))
 
     @property
@@ -386,6 +389,11 @@ def rlcs_debug_set_carry_fault(mute_tile: int = -1, spin_cap: int = 0):
     _check(lib().rlcs_debug_set_carry_fault(mute_tile, spin_cap))
 
 
+def rlcs_debug_stream_copy(src, dst, read_bytes: int, write_bytes: int, stream=None):
+    """Streaming read of read_bytes from src and write of write_bytes to dst (measurement hook)."""
+    _check(lib().rlcs_debug_stream_copy(src.data_ptr(), dst.data_ptr(), int(read_bytes), int(write_bytes), _stream(stream)))
+
+
 def rlcs_debug_time_major_path(path: int = 0):
     """1 = register walk only; anything else = shared-memory ring wherever alignment allows (default)."""
     lib().rlcs_debug_time_major_path(int(path))
@@ -486,13 +494,15 @@ def _tm_ws(T, N, like, workspace, stream):
     nbytes = int(lib().rlcs_time_major_workspace_bytes(N, T))
     if not nbytes:
         return None, 0
-    buf = _torch().empty(nbytes, dtype=_torch().uint8, device=like.device)     # needs no initialisation
-    _keep.append(buf)                     # keep the scratch alive until the enqueued work has run
-    del _keep[:-8]
+    # Scratch for this one call; it needs no initialisation.  Freed memory goes back to torch's caching
+    # allocator, which reuses it in stream order on the allocating stream; a caller-chosen stream is
+    # recorded on the buffer so that the same holds there.
+    buf = _torch().empty(nbytes, dtype=_torch().uint8, device=like.device)
+    if stream is not None:
+        buf.record_stream(stream)
     return buf.data_ptr(), nbytes
 
 
-_keep: list = []
 
 
 def rlcs_gae_time_major(rewards, values, dones, truncs=None, trunc_bootstrap=None, bootstrap=None, *, gamma, lam,
