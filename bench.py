@@ -544,9 +544,24 @@ def cpu_baseline(ro, budget_s: float = 20.0):
     t = oracle_pass(ro, probe_rows, threads)                          # calibration (also warms the library)
     rows = int(min(ro.N, max(probe_rows, probe_rows * budget_s / max(t, 1e-6))))
     secs = oracle_pass(ro, rows, threads)
+    rows1 = max(16, rows // (4 * threads))                            # about a quarter of that time on one thread
+    secs1 = oracle_pass(ro, rows1, 1)
     return {"value": len(ALGOS) * rows * ro.T / secs, "unit": METRIC, "cores": threads, "kind": "oracle",
+            "single_thread_value": len(ALGOS) * rows1 * ro.T / secs1, "cpu_model": _cpu_model(),
             "sample": f"first {rows} of {ro.N} rows x T={ro.T}, all seven algorithms once, {secs:.2f} s, "
-                      f"fp64 sequential C oracle, rows split over {threads} host threads"}
+                      f"fp64 sequential C oracle, rows split over {threads} host threads "
+                      f"(single thread: first {rows1} rows, {secs1:.2f} s)"}
+
+
+def _cpu_model() -> str:
+    try:
+        with open("/proc/cpuinfo") as fh:
+            for line in fh:
+                if line.lower().startswith("model name"):
+                    return line.split(":", 1)[1].strip()
+    except OSError:
+        pass
+    return "unknown"
 
 
 def reference_arm(args, world: int):
