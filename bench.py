@@ -787,6 +787,11 @@ def main():
         gbs = ab / (ms * 1e-3) / 1e9
         per_algo[a] = {"ms": round(ms, 5), "env_steps_per_s": ro.N * ro.T / (ms * 1e-3), "algorithmic_bytes": ab,
                        "gbs": round(gbs, 1), "frac_of_peak": round(gbs / peak, 4)}
+        if ro.truncs is not None and a not in ("elig_trace", "episodic_prefix_sum"):
+            # the same time against the byte count of a kernel that would read trunc_bootstrap densely (context only)
+            dense = 4 * ro.N * ro.T * ({"gae": 4, "vtrace": 5, "retrace": 5, "td_lambda": 3, "discounted_return": 2}[a] + 1) \
+                + 2 * ro.N * ro.T + 4 * ro.N
+            per_algo[a]["gbs_dense_trunc_bootstrap_count"] = round(dense / (ms * 1e-3) / 1e9, 1)
     dom = max(ALGOS, key=lambda a: per_algo[a]["ms"])
     vi = binding.rlcs_debug_variant_for(dom, ro.truncs is not None and dom not in ("elig_trace", "episodic_prefix_sum"), ro.N, ro.T)
     kname = "scan_kernel_tma" if vi["ring_stages"] else "scan_kernel"
