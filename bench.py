@@ -244,10 +244,9 @@ def time_gae_normalized(batch: GpuBatch, steps: int, peak: float):
 
 
 def time_gae_skip(batch: GpuBatch, steps: int, peak: float, p_skip: float = 0.3):
-    """Extension beyond the seven kernels: GAE with observation-skip masking (two launches) on the bench
-    batch with skip ~ Bernoulli(p_skip).  Algorithmic bytes = GAE's, plus the skip mask, plus one write
-    of the filled values W (an output of the call); the second scan's re-read of W and of the masks is
-    the method's own traffic and is not counted."""
+    """Extension beyond the seven kernels: GAE with observation-skip masking (one launch, two scans per
+    tile) on the bench batch with skip ~ Bernoulli(p_skip).  Algorithmic bytes = GAE's, plus the skip
+    mask, plus one write of the filled values W (an output of the call)."""
     torch, B, ro = batch.torch, batch.B, batch.ro
     i, o, p = batch.inp, batch.out, ro.params
     g = torch.Generator(device="cuda").manual_seed(17641)
@@ -268,11 +267,9 @@ def time_gae_skip(batch: GpuBatch, steps: int, peak: float, p_skip: float = 0.3)
     torch.cuda.synchronize()
     ms = e0.elapsed_time(e1) / steps
     ab = algorithmic_bytes(ro, "gae") + 5 * ro.N * ro.T
-    moved = ab + (4 + 1 + (2 if ro.truncs is not None else 1)) * ro.N * ro.T      # W and the masks, read again by scan 2
     gbs = ab / (ms * 1e-3) / 1e9
-    return {"ms": round(ms, 5), "launches_per_call": 2, "p_skip": p_skip, "env_steps_per_s": ro.N * ro.T / (ms * 1e-3),
-            "algorithmic_bytes": ab, "gbs": round(gbs, 1), "frac_of_peak": round(gbs / peak, 4),
-            "frac_of_peak_on_bytes_moved": round(moved / (ms * 1e-3) / 1e9 / peak, 4)}
+    return {"ms": round(ms, 5), "launches_per_call": 1, "p_skip": p_skip, "env_steps_per_s": ro.N * ro.T / (ms * 1e-3),
+            "algorithmic_bytes": ab, "gbs": round(gbs, 1), "frac_of_peak": round(gbs / peak, 4)}
 
 
 def time_retrace_probs(torch, B, steps: int, peak: float, N=16384, T=2048, A=4):

@@ -312,9 +312,9 @@ int rlcs_episodic_prefix_sum_time_major(const float* x, const uint8_t* dones, fl
  * recurrences as in rlcs_gae wherever they stand (at a flagged masked step A_t = 0 and W_t is the
  * flag's successor value).  Without flags on masked steps, the advantages at the unmasked steps are
  * rlcs_gae of the rows with the masked steps deleted.
- * Outputs: values_filled = W (required; also the scratch between the two scans), advantages = A,
- * returns = A + W (optional).  Two launches: W by a backward scan, then the masked GAE scan on
- * (rewards, W).  Same flags, NULL conventions, alignment rules and workspace as rlcs_gae.
+ * Outputs: values_filled = W (required), advantages = A, returns = A + W (optional).  One launch:
+ * per tile, W by a backward scan and then the masked GAE scan on (rewards, W), each with its own
+ * carry between tiles.  Same flags, NULL conventions, alignment rules and workspace as rlcs_gae.
  */
 int rlcs_gae_skip(const float* rewards, const float* values, const uint8_t* dones, const uint8_t* truncs,
                   const float* trunc_bootstrap, const float* bootstrap, const uint8_t* skip, float* values_filled,

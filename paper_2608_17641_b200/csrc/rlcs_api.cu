@@ -31,8 +31,9 @@ size_t rlcs_workspace_bytes(int64_t N, int64_t T) {
     int64_t total = 0;
     if (check_sizes(N, T, &total) != RLCS_OK || total == 0) return 0;
     if (rlcs::kMinTileElems % T == 0) return 0;     // T divides every tile size: no row straddles a tile
+    // one record per 512-step tile, plus one: rlcs_gae_skip keeps two records per tile of >= 1024 steps
     const int64_t tiles = (total + rlcs::kMinTileElems - 1) / rlcs::kMinTileElems;
-    return sizeof(unsigned) * rlcs::kHeaderWords + sizeof(uint4) * (size_t)tiles;
+    return sizeof(unsigned) * rlcs::kHeaderWords + sizeof(uint4) * (size_t)(tiles + 1);
 }
 
 int rlcs_workspace_init(void* workspace, size_t workspace_bytes, void* cuda_stream) {
@@ -94,18 +95,12 @@ int rlcs_gae_skip(const float* rewards, const float* values, const uint8_t* done
     if (!rewards || !values || !skip || !values_filled || !advantages) return RLCS_ERR_NULL;
     p.skip = skip;
     p.gamma = gamma; p.decay = gamma * lambda;
-    // scan 1: W = the value each step shows to its predecessors (V, or what lies behind a masked step)
-    ScanParams f = p;
-    f.f0 = values; f.out0 = values_filled;
-    int variant = choose_variant(rlcs::kFillSkip, truncs != nullptr, total, T);
-    st = finish_params(f, variant, total, T, workspace, workspace_bytes, vec);
-    if (st != RLCS_OK) return st;
-    st = run(rlcs::launch_fill_skip, f, variant, truncs != nullptr, vec, cuda_stream);
-    if (st != RLCS_OK) return st;
-    // scan 2: GAE on (rewards, W) with the masked steps as identities
-    p.f0 = rewards; p.f1 = values_filled; p.out0 = advantages; p.out1 = returns;
-    variant = choose_variant(rlcs::kGaeSkip, truncs != nullptr, total, T);
-    st = finish_params(p, variant, total, T, workspace, workspace_bytes, vec);
+    p.f0 = rewards; p.f1 = values; p.out2 = values_filled; p.out0 = advantages; p.out1 = returns;
+    // One launch runs both scans per tile (value fill, then the masked GAE on its result); each scan has
+    // its own carry records.  These tile shapes have at least 1024 steps, so two records per tile still
+    // fit the workspace of rlcs_workspace_bytes (sized for 512-step tiles).  No cluster carry here.
+    const int variant = choose_variant(rlcs::kGaeSkip, truncs != nullptr, total, T);
+    st = finish_params(p, variant, total, T, workspace, workspace_bytes, vec, false, 2);
     if (st != RLCS_OK) return st;
     return run(rlcs::launch_gae_skip, p, variant, truncs != nullptr, vec, cuda_stream);
 }

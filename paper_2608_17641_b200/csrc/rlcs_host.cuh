@@ -100,8 +100,8 @@ int choose_variant(int algo, bool trunc, int64_t total, int64_t T) {
         case RLCS_NS::kRetrace: return 0;
         case RLCS_NS::kTdLambda: return trunc ? 20 : 0;
         case RLCS_NS::kDisc: return trunc ? 20 : 5;
-        case RLCS_NS::kFillSkip: return 20;
-        case RLCS_NS::kGaeSkip: return 20;
+        case RLCS_NS::kFillSkip:
+        case RLCS_NS::kGaeSkip: return 18;
         case RLCS_NS::kElig: return 18;
         case RLCS_NS::kPrefix: return 18;
         default: return 0;
@@ -110,7 +110,7 @@ int choose_variant(int algo, bool trunc, int64_t total, int64_t T) {
 
 // Fill the size / tiling / carry fields and validate the workspace for this call.
 int finish_params(ScanParams& p, int variant, int64_t total, int64_t T, void* workspace, size_t workspace_bytes, bool vec,
-                  bool allow_cluster = true) {
+                  bool allow_cluster = true, int records_per_tile = 1) {
     const int tile = tile_elems(variant);
     p.total = total;
     p.T = (unsigned)T;
@@ -141,7 +141,7 @@ int finish_params(ScanParams& p, int variant, int64_t total, int64_t T, void* wo
     p.mute_tile = g_mute_tile;
     p.spin_cap = g_spin_cap > 0 ? (unsigned)g_spin_cap : kDefaultSpinCap;
     if (p.carry_mode) {
-        const size_t need = sizeof(unsigned) * RLCS_NS::kHeaderWords + sizeof(uint4) * (size_t)p.num_tiles;
+        const size_t need = sizeof(unsigned) * RLCS_NS::kHeaderWords + sizeof(uint4) * (size_t)p.num_tiles * records_per_tile;
         if (workspace == nullptr || workspace_bytes < need) return RLCS_ERR_WORKSPACE;
         if (!aligned(workspace, 16)) return RLCS_ERR_ALIGN;
         p.header = static_cast<unsigned*>(workspace);

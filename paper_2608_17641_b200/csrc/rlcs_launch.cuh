@@ -147,7 +147,6 @@ cudaError_t launch_affine_bwd(const ScanParams&, int variant, bool trunc, bool v
 cudaError_t launch_affine_fwd(const ScanParams&, int variant, bool trunc, bool vec, cudaStream_t);
 cudaError_t launch_retrace_probs(const ScanParams&, bool trunc, bool vec, bool vec_rows, cudaStream_t);
 cudaError_t launch_gae_stats(const ScanParams&, int variant, bool trunc, bool vec, cudaStream_t);
-cudaError_t launch_fill_skip(const ScanParams&, int variant, bool trunc, bool vec, cudaStream_t);
 cudaError_t launch_gae_skip(const ScanParams&, int variant, bool trunc, bool vec, cudaStream_t);
 cudaError_t launch_norm_finalize(const float* partial, long long num_tiles, double count, int ddof, float eps,
                                  float* mean_rstd, cudaStream_t stream);

@@ -105,6 +105,7 @@ struct ScanParams {
     const io_t* boot;         // [N] or nullptr
     io_t* out0;
     io_t* out1;               // second output or nullptr
+    io_t* out2;               // scan_kernel_gae_skip: the filled values W
     float* stats;             // kGaeStats: per scan-order tile {sum A, sum A^2}
     long long total;          // N*T
     long long num_tiles;
@@ -709,7 +710,8 @@ struct NoHook {
 // CLUSTER: the carry between blocks goes through distributed shared memory (cluster_carry).
 template <int ALGO, bool TRUNC, bool VEC, int THREADS, int ITEMS, bool FULL, bool LAST, class Hook, bool CLUSTER = false>
 __device__ __forceinline__ void tile_compute(Chunk<ALGO, TRUNC, ITEMS>& c, Vals<ITEMS>& v, const ScanParams& p, long long i0, long long s,
-                                             unsigned epoch, ScanSmem<THREADS / 32>& sm, int buf, Hook after_barrier) {
+                                             unsigned epoch, ScanSmem<THREADS / 32>& sm, int buf, Hook after_barrier,
+                                             float* prev_out = nullptr) {
     constexpr bool FWD = is_forward(ALGO);
     constexpr int NW = THREADS / 32;
     constexpr int W = ITEMS / 4;
@@ -926,6 +928,7 @@ __device__ __forceinline__ void tile_compute(Chunk<ALGO, TRUNC, ITEMS>& c, Vals<
     }
     // value of the recurrence at the step just before this thread's chunk in scan order
     float prev = fmaf(before.b, carry_in, before.a);
+    if (prev_out != nullptr) *prev_out = prev;
 
     // ---- replay, epilogue, store
     float out1v[ITEMS];
@@ -1030,6 +1033,68 @@ __global__ void __launch_bounds__(THREADS, MIN_BLOCKS) scan_kernel(const ScanPar
     if (full) one_tile<ALGO, TRUNC, VEC, THREADS, ITEMS, true>(p, tile, s, epoch, sm);
     else one_tile<ALGO, TRUNC, VEC, THREADS, ITEMS, false>(p, tile, s, epoch, sm);
 }
+
+// ------------------------------------------------------------------------------------------ kernel 1b: GAE with observation-skip masking
+// Both scans of the masked GAE in one pass over the tile: first the fill scan (W = the value a step
+// shows to its predecessors), whose result stays in registers -- a thread's successor value W at
+// i0 + ITEMS is the fill recurrence's own incoming value -- then the masked GAE scan on (rewards, W).
+// Each scan has its own carry records (the second half of the record array) and shared-memory
+// buffers; the block signs off after the second.  p.f0 = rewards, p.f1 = values, p.out2 = W,
+// p.out0 / p.out1 = advantages / returns.
+#ifndef RLCS_IO_BF16
+template <bool TRUNC, bool VEC, int THREADS, int ITEMS, bool FULL>
+__device__ __forceinline__ void one_tile_gae_skip(const ScanParams& p, long long tile, long long s, unsigned epoch,
+                                                  ScanSmem<THREADS / 32>& sm) {
+    constexpr int TILE = THREADS * ITEMS;
+    const int tid = threadIdx.x;
+    const int lane = tid & 31;
+    const long long i0 = tile * TILE + (long long)tid * ITEMS;
+    Chunk<kFillSkip, TRUNC, ITEMS> cf;
+    const long long n0 = locate(cf, p, i0);
+    load_flags_global<kFillSkip, TRUNC, ITEMS, VEC, FULL>(cf, p, i0, lane);
+    const int nvalid = FULL ? ITEMS : cf.nvalid;
+    Vals<ITEMS> vf, vg;
+    load_f32<ITEMS, VEC>(p.f1, i0, nvalid, vf.a);            // values: the fill scan's input
+    load_f32<ITEMS, VEC>(p.f0, i0, nvalid, vg.a);            // rewards, for the second scan
+    vf.halo = 0.f; vf.halo_lr = 0.f;
+    issue_boot(cf, p, n0);
+    issue_trunc_values(cf, p, i0);
+    Chunk<kGaeSkip, TRUNC, ITEMS> cg;
+    cg.edge = cf.edge; cg.nvalid = cf.nvalid; cg.halo_d = 0; cg.boot_first = cf.boot_first;
+#pragma unroll
+    for (int k = 0; k < ITEMS / 4; ++k) { cg.dw[k] = cf.dw[k]; cg.tw[k] = cf.tw[k]; cg.kw[k] = cf.kw[k]; }
+#pragma unroll
+    for (int j = 0; j < ITEMS; ++j) cg.ov[j] = cf.ov[j];
+
+    ScanParams pf = p;
+    pf.out0 = p.out2;
+    pf.out1 = nullptr;
+    float w_next = 0.f;
+    tile_compute<kFillSkip, TRUNC, VEC, THREADS, ITEMS, FULL, false>(cf, vf, pf, i0, s, epoch, sm, 0, NoHook{}, &w_next);
+
+    ScanParams pg = p;
+    pg.records = p.records + p.num_tiles;
+#pragma unroll
+    for (int j = 0; j < ITEMS; ++j) vg.x1[j] = vf.a[j];      // W of this thread's steps
+    vg.halo = w_next;
+    vg.halo_lr = 0.f;
+    tile_compute<kGaeSkip, TRUNC, VEC, THREADS, ITEMS, FULL, true>(cg, vg, pg, i0, s, epoch, sm, 1, NoHook{});
+}
+
+template <bool TRUNC, bool VEC, int THREADS, int ITEMS, int MIN_BLOCKS>
+__global__ void __launch_bounds__(THREADS, MIN_BLOCKS) scan_kernel_gae_skip(const ScanParams p) {
+    constexpr int TILE = THREADS * ITEMS;
+    __shared__ ScanSmem<THREADS / 32> sm;
+    const int tid = threadIdx.x;
+    const long long s = blockIdx.x;
+    const long long tile = p.num_tiles - 1 - s;
+    unsigned epoch = 0;
+    if (p.carry_mode && tid < 32) epoch = ld_volatile_u32(p.header);
+    const bool full = (tile * TILE + TILE <= p.total) && (p.T >= (unsigned)ITEMS);
+    if (full) one_tile_gae_skip<TRUNC, VEC, THREADS, ITEMS, true>(p, tile, s, epoch, sm);
+    else one_tile_gae_skip<TRUNC, VEC, THREADS, ITEMS, false>(p, tile, s, epoch, sm);
+}
+#endif  // !RLCS_IO_BF16
 
 // ------------------------------------------------------------------------------------------ kernel 1c: Retrace from [N,T,A] tensors
 #ifndef RLCS_IO_BF16

@@ -53,8 +53,8 @@ def test_workspace_bytes(L):
     assert L.rlcs_workspace_bytes(-1, 5) == 0
     for T in (1, 2, 64, 128, 512):                      # T divides every tile: nothing straddles
         assert L.rlcs_workspace_bytes(4096, T) == 0
-    assert L.rlcs_workspace_bytes(64, 16384) == 256 + 16 * (64 * 16384 // 512)
-    assert L.rlcs_workspace_bytes(3, 1000) == 256 + 16 * ((3000 + 511) // 512)
+    assert L.rlcs_workspace_bytes(64, 16384) == 256 + 16 * (64 * 16384 // 512 + 1)
+    assert L.rlcs_workspace_bytes(3, 1000) == 256 + 16 * ((3000 + 511) // 512 + 1)
 
 
 # fake, never-dereferenced device addresses: every call below must return before any launch
