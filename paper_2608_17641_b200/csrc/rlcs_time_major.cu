@@ -60,21 +60,28 @@ struct TmParams {
     float gamma, decay, aux, rho_bar, c_bar;
     int starts_at;
     int stages, warps_per_block, cols_per_lane;   // tm_block_kernel: ring depth, warps per block, columns per lane
+    long long batch, batch_stride;                // kTmVec*: independent [T, N] problems (blockIdx.z), elements between them
     float* agg_a;             // [chunks, N] pass 1: chunk aggregates; after the chain: carry into each chunk
     float* agg_b;             // [chunks, N]
 };
 
-__host__ __device__ constexpr bool tm_forward(int a) { return a == kElig || a == kPrefix; }
+// Vector-valued eligibility traces x[n] : [T, D] are time-major problems with D columns per row n and
+// one flag per timestep shared by all columns (rlcs_elig_trace_vec / _beta use the block kernel for
+// few long rows): same kernel, the flag read per timestep instead of from a mask tile.
+constexpr int kTmVec = 101;        // shared scalar decay
+constexpr int kTmVecBeta = 102;    // decay per component and step in f1
+__host__ __device__ constexpr bool tm_row_mask(int a) { return a == kTmVec || a == kTmVecBeta; }
+__host__ __device__ constexpr bool tm_forward(int a) { return a == kElig || a == kPrefix || tm_row_mask(a); }
 // float tensors that are read at every step, and mask tensors
 __host__ __device__ constexpr int tm_nf(int a) {
-    return a == kRetrace ? 4 : a == kVtrace ? 3 : (a == kGae || a == kTdLambda) ? 2 : 1;
+    return a == kRetrace ? 4 : a == kVtrace ? 3 : (a == kGae || a == kTdLambda || a == kTmVecBeta) ? 2 : 1;
 }
 // timesteps per warp and stage in tm_block_kernel: fewer for Retrace, whose four float inputs make a
 // row 576 bytes (measured: 0.84 -> 0.90 of the copy bandwidth with 4, while the lighter algorithms
 // lose 5-12 % to the doubled per-stage overhead); more for the discounted return, whose rows are
 // 160-192 bytes (0.52 -> 0.63 at 16384 environments with 16; the forward scans lose 1 % that way)
 __host__ __device__ constexpr int tm_rows(int a) { return a == kRetrace ? 4 : a == kDisc ? 16 : 8; }
-__host__ __device__ constexpr int tm_row_bytes(int a, bool trunc) { return tm_nf(a) * 128 + (trunc ? 2 : 1) * 32; }
+__host__ __device__ constexpr int tm_row_bytes(int a, bool trunc) { return tm_nf(a) * 128 + (tm_row_mask(a) ? 0 : (trunc ? 2 : 1) * 32); }
 
 // all ones where x != 0, else 0; written in PTX so that the flag reaches the arithmetic below as a
 // plain word, not as a condition the compiler could branch on
@@ -392,7 +399,7 @@ constexpr int kMaxStages = 16;
 template <int ALGO, bool TRUNC, int W, int C>
 struct StageView {
     static constexpr int NF = tm_nf(ALGO);
-    static constexpr int NM = TRUNC ? 2 : 1;
+    static constexpr int NM = tm_row_mask(ALGO) ? 0 : (TRUNC ? 2 : 1);
     static constexpr int KR = tm_rows(ALGO);
     static constexpr int R = KR * W;
     unsigned char* fbase;
@@ -452,6 +459,7 @@ __device__ __forceinline__ void issue_floats(const StageView<ALGO, TRUNC, W, C>&
 
 template <int ALGO, bool TRUNC, int W, int C>
 __device__ __forceinline__ void issue_masks(const StageView<ALGO, TRUNC, W, C>& sv, const TmParams& p, const CopyPlan& cp, unsigned s) {
+    if constexpr (tm_row_mask(ALGO)) return;
     if (cp.m_on) {
         const unsigned q = s * (tm_rows(ALGO) * W) + cp.mrow;
         const bool ok = q < cp.len;
@@ -502,8 +510,17 @@ __device__ __forceinline__ int wrap_prev(int x, int n) { return x == 0 ? n - 1 :
 // requested two stages before their use (registers bv1, bv2).
 // MODE as in tm_kernel.
 template <int ALGO, bool TRUNC, int MODE, int W, int C>
-__global__ void __launch_bounds__(32 * W) tm_block_kernel(const TmParams p) {
+__global__ void __launch_bounds__(32 * W) tm_block_kernel(const TmParams p_in) {
     constexpr bool FWD = tm_forward(ALGO);
+    constexpr bool ROWMASK = tm_row_mask(ALGO);
+    TmParams p = p_in;
+    if constexpr (ROWMASK) {                                 // this block's row of the batch
+        const long long off = (long long)blockIdx.z * p_in.batch_stride;
+        p.f0 += off;
+        if constexpr (ALGO == kTmVecBeta) p.f1 += off;
+        p.out0 += off;
+        p.dones += (long long)blockIdx.z * p_in.T;
+    }
     using SV = StageView<ALGO, TRUNC, W, C>;
     extern __shared__ __align__(16) unsigned char tm_smem[];
     const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
@@ -545,7 +562,8 @@ __global__ void __launch_bounds__(32 * W) tm_block_kernel(const TmParams p) {
         bootv[c] = (!FWD && p.boot != nullptr) ? __ldg(p.boot + n) : 0.f;
         BackState b0 = {};
         FwdState f0 = {};
-        if constexpr (FWD) init_fwd(f0, p, n, t_lo, 0.f);
+        if constexpr (ROWMASK) f0.d_prev = 0;
+        else if constexpr (FWD) init_fwd(f0, p, n, t_lo, 0.f);
         else init_back<ALGO>(b0, p, n, t_hi, 0.f);
         v0[c] = b0.v_next; lr0[c] = b0.lr_next; d0[c] = f0.d_prev;
     }
@@ -598,7 +616,9 @@ __global__ void __launch_bounds__(32 * W) tm_block_kernel(const TmParams p) {
         unsigned d_prev[C];
 #pragma unroll
         for (int c = 0; c < C; ++c) { v_next[c] = 0.f; lr_next[c] = 0.f; d_prev[c] = 0; }
-        if (w > 0) {
+        if constexpr (ROWMASK) {
+            // the flag of step t-1 is read per step below
+        } else if (w > 0) {
             if constexpr (FWD) lds_m<C>(cur.m(0, row0 - 1), lane, d_prev);
             else if constexpr (ALGO == kRetrace) { lds_f<C>(cur.f(2, row0 - 1), lane, v_next); lds_f<C>(cur.f(3, row0 - 1), lane, lr_next); }
             else if constexpr (SV::NF >= 2) lds_f<C>(cur.f(1, row0 - 1), lane, v_next);
@@ -622,6 +642,15 @@ __global__ void __launch_bounds__(32 * W) tm_block_kernel(const TmParams p) {
 #pragma unroll
         for (int c = 0; c < C; ++c) { carry[c] = 0.f; prod[c] = 1.f; }
         // the per-row guards exist only in the instance that the chunk's ragged last stage takes
+        // one flag per timestep: the flags of the steps before this warp's rows (cut into step t <=> t == 0 or dones[t-1])
+        unsigned rowcut[KR];
+        if constexpr (ROWMASK) {
+#pragma unroll
+            for (int u = 0; u < KR; ++u) {
+                const unsigned t = t_lo + j * R + row0 + u;
+                rowcut[u] = (t == 0 || t > p.T) ? 1u : __ldg(p.dones + t - 1);
+            }
+        }
         auto pass1 = [&](auto full) {
             constexpr bool FULL = decltype(full)::value;
 #pragma unroll
@@ -632,7 +661,13 @@ __global__ void __launch_bounds__(32 * W) tm_block_kernel(const TmParams p) {
                     float r[C], x1[C], x2[C], x3[C];
                     unsigned dn[C], tr[C];
                     lds_f<C>(cur.f(0, row0 + u), lane, r);
-                    lds_m<C>(cur.m(0, row0 + u), lane, dn);
+                    if constexpr (ROWMASK) {
+                        if constexpr (ALGO == kTmVecBeta) lds_f<C>(cur.f(1, row0 + u), lane, x1);
+#pragma unroll
+                        for (int c = 0; c < C; ++c) dn[c] = 0;
+                    } else {
+                        lds_m<C>(cur.m(0, row0 + u), lane, dn);
+                    }
                     if constexpr (!FWD) {
                         if constexpr (SV::NF >= 2) lds_f<C>(cur.f(1, row0 + u), lane, x1);
                         if constexpr (ALGO == kRetrace) { lds_f<C>(cur.f(2, row0 + u), lane, x2); lds_f<C>(cur.f(3, row0 + u), lane, x3); }
@@ -642,7 +677,11 @@ __global__ void __launch_bounds__(32 * W) tm_block_kernel(const TmParams p) {
 #pragma unroll
                     for (int c = 0; c < C; ++c) {
                         Coef co;
-                        if constexpr (FWD) {
+                        if constexpr (ROWMASK) {
+                            co.alpha = r[c];
+                            co.beta = keep(~ones_if(rowcut[u]), ALGO == kTmVecBeta ? x1[c] : p.decay);
+                            co.pg = 0.f;
+                        } else if constexpr (FWD) {
                             co = fwd_coef<ALGO>(r[c], dn[c], d_prev[c], p, (u == 0 && w == 0 && j == 0) ? t_lo : 1u);
                             d_prev[c] = dn[c];
                         } else {
@@ -675,7 +714,7 @@ __global__ void __launch_bounds__(32 * W) tm_block_kernel(const TmParams p) {
         else pass1(std::false_type{});
 #pragma unroll
         for (int c = 0; c < C; ++c) agg[((par * W + w) * 32 + lane) * C + c] = make_float2(carry[c], prod[c]);
-        if (w == W - 1) {                                    // neighbours for the next stage's first warp
+        if (!ROWMASK && w == W - 1) {                        // neighbours for the next stage's first warp
 #pragma unroll
             for (int c = 0; c < C; ++c) {
                 if constexpr (FWD) edge_x[par * 32 * C + C * lane + c] = __uint_as_float(d_prev[c]);
@@ -803,8 +842,9 @@ void plan_chunks(long long N, long long T, unsigned* chunk, unsigned* chunks) {
 // share an SM, no deeper than keeps about 16 MB in flight over the grid, and at least 3.
 size_t plan_block(TmParams& p, int rows, int row_bytes, bool trunc, bool wide_ok) {
     int C = 1;
-    if (wide_ok && (p.N + 63) / 64 * p.chunks >= 2 * kSms) C = 2;
-    const long long blocks = (p.N + 32 * C - 1) / (32 * C) * p.chunks;
+    const long long batch = p.batch > 0 ? p.batch : 1;
+    if (wide_ok && (p.N + 63) / 64 * p.chunks * batch >= 2 * kSms) C = 2;
+    const long long blocks = (p.N + 32 * C - 1) / (32 * C) * p.chunks * batch;
     const int W = C == 2 ? 4 : blocks < kSms ? 16 : blocks < 2 * kSms ? 8 : 4;
     const long long stage = (long long)rows * W * row_bytes * C;
     const long long mstage = (long long)rows * W * (trunc ? 64 : 32) * C;
@@ -927,6 +967,47 @@ int run(const TmParams& p, void* cuda_stream) {
 }
 
 }  // namespace
+
+// Vector-valued eligibility traces for few long rows (called from rlcs_elig_vec.cu, today for the
+// per-component decay only): every row n is a time-major [T, D] problem with one flag per timestep;
+// one thread block per 32 components and row streams the row once through the shared-memory ring,
+// its warps splitting every stage in time.
+namespace rlcs_internal {
+
+// usable when every row of D floats can be copied in 16-byte pieces and rows alone give enough blocks
+bool vec_trace_block_usable(const float* x, const float* beta, int64_t N, int64_t T, int64_t D) {
+    if (g_force_path == 1) return false;
+    if (D % 4 != 0 || D < 32 || T < 64) return false;
+    if (!aligned16(x) || (beta != nullptr && !aligned16(beta))) return false;
+    return (D + 31) / 32 * N >= 96 && N <= 65535;
+}
+
+int vec_trace_block(const float* x, const float* beta, const uint8_t* dones, float* traces, int64_t N, int64_t T, int64_t D,
+                    float decay, void* cuda_stream) {
+    TmParams p = {};
+    p.f0 = x; p.f1 = beta; p.dones = dones; p.out0 = traces;
+    p.N = D; p.T = (unsigned)T; p.chunk = (unsigned)T; p.chunks = 1;
+    p.decay = decay;
+    p.batch = N; p.batch_stride = T * D;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    auto go = [&](auto algo_tag) {
+        constexpr int ALGO = decltype(algo_tag)::value;
+        const size_t smem = plan_block(p, tm_rows(ALGO), tm_row_bytes(ALGO, false), false, false);
+        const dim3 grid((unsigned)((D + 31) / 32), 1, (unsigned)N);
+        auto launch_w = [&](auto w_tag) {
+            constexpr int W = decltype(w_tag)::value;
+            if (!allow_smem(tm_block_kernel<ALGO, false, 0, W, 1>, smem)) return (int)RLCS_ERR_CUDA;
+            tm_block_kernel<ALGO, false, 0, W, 1><<<grid, 32 * W, smem, s>>>(p);
+            return cudaGetLastError() == cudaSuccess ? (int)RLCS_OK : (int)RLCS_ERR_CUDA;
+        };
+        if (p.warps_per_block == 16) return launch_w(std::integral_constant<int, 16>{});
+        if (p.warps_per_block == 8) return launch_w(std::integral_constant<int, 8>{});
+        return launch_w(std::integral_constant<int, 4>{});
+    };
+    return beta != nullptr ? go(std::integral_constant<int, kTmVecBeta>{}) : go(std::integral_constant<int, kTmVec>{});
+}
+
+}  // namespace rlcs_internal
 
 extern "C" {
 

@@ -452,7 +452,8 @@ def test_retrace_probs_agrees_with_scalar_entry_point(oracle, W, B):
 
 # ------------------------------------------------------------------ vector-valued eligibility traces
 @pytest.mark.parametrize("N,T,D", [(1, 1, 1), (3, 7, 5), (8, 128, 64), (64, 257, 16), (4096, 40, 8), (2, 5000, 128),
-                                    (3, 16384, 32), (1, 70000, 4), (5, 999, 3), (7, 300, 130)])
+                                    (3, 16384, 32), (1, 70000, 4), (5, 999, 3), (7, 300, 130),
+                                    (64, 4096, 64), (100, 3000, 32), (48, 2000, 96), (60, 1000, 36)])
 def test_vector_eligibility_trace(oracle, W, B, N, T, D):
     import torch
     rng = np.random.default_rng(N * 7919 + T * 31 + D)
@@ -492,7 +493,7 @@ def test_vector_trace_argument_checks(oracle, W, B):
 
 
 @pytest.mark.parametrize("N,T,D", [(1, 1, 1), (3, 7, 5), (8, 128, 64), (64, 257, 16), (4096, 40, 8), (2, 5000, 128),
-                                    (3, 16384, 32), (5, 999, 3)])
+                                    (3, 16384, 32), (5, 999, 3), (64, 4096, 64), (100, 3000, 32), (48, 2000, 96), (60, 1000, 36)])
 def test_per_dimension_beta_eligibility_trace(oracle, W, B, N, T, D):
     import torch
     rng = np.random.default_rng(N * 7919 + T * 31 + D + 1)
@@ -511,7 +512,11 @@ def test_per_dimension_beta_eligibility_trace(oracle, W, B, N, T, D):
     # a constant beta is the shared-scalar entry point, bit for bit (same FMA per step, same chunking)
     const = torch.full_like(xd, 0.25)
     same = B.rlcs_elig_trace_vec_beta(xd, const, dd)
-    assert torch.equal(same, B.rlcs_elig_trace_vec(xd, dd, gamma=0.5, lam=0.5))
+    scalar = B.rlcs_elig_trace_vec(xd, dd, gamma=0.5, lam=0.5)
+    if int(B.lib().rlcs_elig_trace_vec_beta_workspace_bytes(N, T, D)) == 0:
+        assert torch.equal(same, scalar)                   # one pass in both: same FMA per step
+    else:                                                   # few long rows: the block kernel splits time among warps
+        assert_close("constant beta vs shared decay", same.cpu().numpy(), scalar.cpu().numpy().astype(np.float64))
 
 
 def test_per_dimension_beta_argument_checks(oracle, W, B):
