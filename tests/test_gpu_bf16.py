@@ -170,6 +170,36 @@ def test_bf16_large_problem_with_carry(oracle, W, B):
     compare16(oracle, B, W.make_rollout(124, 2900, 3000, p_done=0.002, p_trunc=0.002), algos=("gae", "vtrace", "retrace"))
 
 
+def test_bf16_full_size_sampled_rows(oracle, W, B):
+    """16384 x 2048 with truncations, the configuration bench.py times: GAE, V-Trace and the discounted
+    return on bfloat16 tensors; every element of 192 sampled rows against the oracle."""
+    import copy
+    import torch
+    ro = to_bf16_values(W.config5())
+    p = ro.params
+    rows = np.unique(np.concatenate([[0, ro.N - 1], np.random.default_rng(7).integers(0, ro.N, 190)]))
+    small = copy.copy(ro)
+    for k in FLOAT_KEYS + ("dones", "truncs"):
+        a = getattr(ro, k)
+        setattr(small, k, None if a is None else np.ascontiguousarray(a[rows]))
+    small.N = len(rows)
+    ref = run_oracle(oracle, small, ("gae", "vtrace", "discounted_return"))
+    dev = Dev16(ro)
+    ws = B.Workspace(ro.N, ro.T)
+    idx = torch.from_numpy(rows).cuda()
+    adv, ret = B.rlcs_gae_bf16(dev.rewards, dev.values, dev.dones, dev.truncs, dev.trunc_bootstrap, dev.bootstrap,
+                               gamma=p["gamma"], lam=p["lam"], workspace=ws)
+    assert_close16("gae", adv[idx], ref["gae"][0]); assert_close16("ret", ret[idx], ref["gae"][1])
+    vs, pg = B.rlcs_vtrace_bf16(dev.rewards, dev.values, dev.log_rhos, dev.dones, dev.truncs, dev.trunc_bootstrap,
+                                dev.bootstrap, gamma=p["gamma"], rho_bar=p["rho_bar"], c_bar=p["c_bar"], workspace=ws)
+    assert_close16("vs", vs[idx], ref["vtrace"][0]); assert_close16("pg", pg[idx], ref["vtrace"][1])
+    out = B.rlcs_discounted_return_bf16(dev.rewards, dev.dones, dev.truncs, dev.trunc_bootstrap, dev.bootstrap,
+                                        gamma=p["gamma"], workspace=ws)
+    assert_close16("disc", out[idx], ref["discounted_return"])
+    torch.cuda.synchronize()
+    assert ws.device_status() == 0
+
+
 @pytest.mark.parametrize("variant", BUILT_VARIANTS)
 def test_bf16_equals_rounded_fp32_bit_for_bit(oracle, W, B, variant):
     """Same tile shape, same fp32 arithmetic: the only difference is the rounding on store, and torch's

@@ -70,6 +70,61 @@ def test_config5_full_size_all_seven(oracle, W, B):
             assert_close(a, gpu[a], ref[a])
 
 
+def test_config5_full_size_extension_entry_points(oracle, W, B):
+    """The entry points beyond the paper's API at the bench's full size, 16384 x 2048 with truncations,
+    in the configuration bench.py times: time-major (all seven), bfloat16 GAE, skip-masked GAE.  Rows are
+    independent, so the oracle checks every element of 192 sampled rows (first, last, and a seeded draw)."""
+    import torch
+    ro = W.config5()
+    p = ro.params
+    N, T = ro.N, ro.T
+    rng = np.random.default_rng(5)
+    rows = np.unique(np.concatenate([[0, 1, N - 2, N - 1], rng.integers(0, N, 188)]))
+    sub = lambda a: None if a is None else np.ascontiguousarray(a[rows])
+    import copy
+    small = copy.copy(ro)
+    for k in ("rewards", "values", "dones", "bootstrap", "truncs", "trunc_bootstrap", "q_sa", "expected_q", "log_rhos", "x"):
+        setattr(small, k, sub(getattr(ro, k)))
+    small.N = len(rows)
+    ref = run_oracle(oracle, small, ALL_ALGOS)
+    # time-major, all seven
+    r, v, d, tr, bv = _tm(ro.rewards), _tm(ro.values), _tm(ro.dones), _tm(ro.truncs), _tm(ro.trunc_bootstrap)
+    bt = torch.from_numpy(ro.bootstrap).cuda()
+    take = lambda t: np.ascontiguousarray(t[:, torch.from_numpy(rows).cuda()].cpu().numpy().T)
+    adv, ret = B.rlcs_gae_time_major(r, v, d, tr, bv, bt, gamma=p["gamma"], lam=p["lam"])
+    assert_close("tm gae", take(adv), ref["gae"][0]); assert_close("tm ret", take(ret), ref["gae"][1])
+    del adv, ret
+    out = B.rlcs_td_lambda_time_major(r, v, d, tr, bv, bt, gamma=p["gamma"], lam=p["lam"])
+    assert_close("tm td", take(out), ref["td_lambda"])
+    out = B.rlcs_discounted_return_time_major(r, d, tr, bv, bt, gamma=p["gamma"])
+    assert_close("tm disc", take(out), ref["discounted_return"])
+    lr = _tm(ro.log_rhos)
+    vs, pg = B.rlcs_vtrace_time_major(r, v, lr, d, tr, bv, bt, gamma=p["gamma"], rho_bar=p["rho_bar"], c_bar=p["c_bar"])
+    assert_close("tm vs", take(vs), ref["vtrace"][0]); assert_close("tm pg", take(pg), ref["vtrace"][1])
+    del vs, pg, v
+    q, eq = _tm(ro.q_sa), _tm(ro.expected_q)
+    out = B.rlcs_retrace_time_major(r, q, eq, lr, d, tr, bv, bt, gamma=p["gamma"], lam=p["lam"], c_bar=p["c_bar"])
+    assert_close("tm retrace", take(out), ref["retrace"])
+    del q, eq, lr, r, tr, bv, d
+    x, dany = _tm(ro.x), _tm(ro.any_done)
+    assert_close("tm elig", take(B.rlcs_elig_trace_time_major(x, dany, gamma=p["gamma"], lam=p["lam"])), ref["elig_trace"])
+    assert_close("tm prefix", take(B.rlcs_episodic_prefix_sum_time_major(x, dany)), ref["prefix_ends_at"])
+    del x, dany, out
+    torch.cuda.empty_cache()
+    # skip-masked GAE (row-major)
+    dev = Dev(ro)
+    skip = (np.random.default_rng(6).random((N, T)) < 0.3).astype(np.uint8)
+    ws = B.Workspace(N, T)
+    a, rt, fil = B.rlcs_gae_skip(dev.rewards, dev.values, dev.dones, dev.truncs, dev.trunc_bootstrap, dev.bootstrap,
+                                 skip=torch.from_numpy(skip).cuda(), gamma=p["gamma"], lam=p["lam"], workspace=ws)
+    ra, rr, rf = oracle.gae_skip(small.rewards, small.values, small.dones, small.truncs, small.trunc_bootstrap, small.bootstrap,
+                                 skip=np.ascontiguousarray(skip[rows]), gamma=p["gamma"], lam=p["lam"])
+    pick = lambda t: t[torch.from_numpy(rows).cuda()].cpu().numpy()
+    assert ws.device_status() == 0
+    assert_close("skip adv", pick(a), ra); assert_close("skip ret", pick(rt), rr)
+    assert np.array_equal(pick(fil).astype(np.float64), rf)
+
+
 # ------------------------------------------------------------------ shape / flag matrix
 SHAPES = [(1, 1), (3, 1), (1, 2), (2, 3), (3, 4), (8, 5), (3, 7), (64, 8), (3, 9), (8, 31), (64, 32), (3, 33),
           (8, 63), (2, 65), (3, 127), (8, 1000), (3, 2047), (2, 2048), (3, 2049), (2, 4097), (1, 20000)]
