@@ -18,7 +18,7 @@
 // Two kernels share this per-tile code:
 //   scan_kernel_tma  persistent thread blocks (all co-resident); each walks tiles s, s+G, s+2G, ...
 //                    and keeps a ring of STAGES tiles in flight: one elected thread issues 1-D bulk
-//                    copies (cp.async.bulk, no multicast, no tensor map: tiles of the flat array are
+//                    copies (cp.async.bulk into its own block's shared memory, no tensor map: tiles of the flat array are
 //                    contiguous) that complete on an mbarrier per stage.  Needs 16-byte aligned
 //                    pointers; the ragged last tile(s) are loaded with plain loads.
 //   scan_kernel      one tile per thread block, plain (vector or element-wise) global loads; used
@@ -1169,7 +1169,7 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, unsigned parity) {
                  : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
     return ok != 0;
 }
-// 1-D bulk copy global -> this block's shared memory, completing `bytes` on `bar`.  No multicast.
+// 1-D bulk copy global -> this block's shared memory only, completing `bytes` on `bar`.
 // dst, src 16-byte aligned; bytes a multiple of 16.
 __device__ __forceinline__ void bulk_load(void* dst, const void* src, unsigned bytes, uint64_t* bar) {
     asm volatile("cp.async.bulk.shared::cta.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
