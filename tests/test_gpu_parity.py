@@ -831,6 +831,65 @@ def test_randomized_time_major_and_skip(oracle, W, B):
         assert np.array_equal(fil.cpu().numpy().astype(np.float64), rf), tag
 
 
+def test_calls_can_be_captured_in_a_cuda_graph(oracle, W, B):
+    """No entry point allocates, synchronises or keeps host state a replay would miss: a graph that
+    captured one call of each family reproduces the eager results bit for bit, twice (the second
+    replay also proves that the carry workspace's per-call epoch advances inside the graph)."""
+    import torch
+    ro = W.make_rollout(132, 48, 3000, p_done=0.01, p_trunc=0.01)         # rows straddle tiles: look-back runs
+    p = ro.params
+    dev = Dev(ro)
+    r_tm, v_tm, d_tm = _tm(ro.rewards), _tm(ro.values), _tm(ro.dones)
+    tr_tm, bv_tm = _tm(ro.truncs), _tm(ro.trunc_bootstrap)
+    skip = (torch.rand((ro.N, ro.T), device="cuda") < 0.3).to(torch.uint8)
+    r16, v16 = dev.rewards.to(torch.bfloat16), dev.values.to(torch.bfloat16)
+    bv16, bt16 = dev.trunc_bootstrap.to(torch.bfloat16), dev.bootstrap.to(torch.bfloat16)
+    ws = B.Workspace(ro.N, ro.T)
+    wsn = B.Workspace(ro.N, ro.T, nbytes=int(B.lib().rlcs_gae_normalized_workspace_bytes(ro.N, ro.T)))
+    wtm = B.Workspace(ro.N, ro.T, nbytes=max(256, int(B.lib().rlcs_time_major_workspace_bytes(ro.N, ro.T))))
+    new = lambda like=dev.rewards, dt=None: torch.empty_like(like, dtype=dt or like.dtype)
+    outs = {k: new() for k in ("adv", "ret", "vs", "pg", "q", "nadv", "nret", "sadv", "sret", "fil", "el")}
+    outs.update(tadv=new(r_tm), tret=new(r_tm), badv=new(dt=torch.bfloat16), bret=new(dt=torch.bfloat16))
+
+    def run(s):
+        kw = dict(stream=s)
+        B.rlcs_gae(dev.rewards, dev.values, dev.dones, dev.truncs, dev.trunc_bootstrap, dev.bootstrap, gamma=p["gamma"],
+                   lam=p["lam"], advantages=outs["adv"], returns=outs["ret"], workspace=ws, **kw)
+        B.rlcs_vtrace(dev.rewards, dev.values, dev.log_rhos, dev.dones, dev.truncs, dev.trunc_bootstrap, dev.bootstrap,
+                      gamma=p["gamma"], vs=outs["vs"], pg_advantages=outs["pg"], workspace=ws, **kw)
+        B.rlcs_retrace(dev.rewards, dev.q_sa, dev.expected_q, dev.log_rhos, dev.dones, dev.truncs, dev.trunc_bootstrap,
+                       dev.bootstrap, gamma=p["gamma"], lam=p["lam"], q_targets=outs["q"], workspace=ws, **kw)
+        B.rlcs_elig_trace(dev.x, dev.any_done, gamma=p["gamma"], lam=p["lam"], traces=outs["el"], workspace=ws, **kw)
+        B.rlcs_gae_normalized(dev.rewards, dev.values, dev.dones, dev.truncs, dev.trunc_bootstrap, dev.bootstrap,
+                              gamma=p["gamma"], lam=p["lam"], advantages=outs["nadv"], returns=outs["nret"], workspace=wsn, **kw)
+        B.rlcs_gae_skip(dev.rewards, dev.values, dev.dones, dev.truncs, dev.trunc_bootstrap, dev.bootstrap, skip=skip,
+                        gamma=p["gamma"], lam=p["lam"], values_filled=outs["fil"], advantages=outs["sadv"],
+                        returns=outs["sret"], workspace=ws, **kw)
+        B.rlcs_gae_time_major(r_tm, v_tm, d_tm, tr_tm, bv_tm, dev.bootstrap, gamma=p["gamma"], lam=p["lam"],
+                              advantages=outs["tadv"], returns=outs["tret"], workspace=wtm, **kw)
+        B.rlcs_gae_bf16(r16, v16, dev.dones, dev.truncs, bv16, bt16, gamma=p["gamma"], lam=p["lam"],
+                        advantages=outs["badv"], returns=outs["bret"], workspace=ws, **kw)
+
+    s = torch.cuda.Stream()
+    with torch.cuda.stream(s):
+        run(s)                                                   # eager (also the warm-up before capture)
+        torch.cuda.synchronize()
+        eager = {k: v.clone() for k, v in outs.items()}
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=s):
+            run(s)
+        for _ in range(2):
+            for v in outs.values():
+                v.zero_()
+            graph.replay()
+            torch.cuda.synchronize()
+            for k, v in outs.items():
+                assert torch.equal(v.view(torch.int16 if v.dtype == torch.bfloat16 else torch.int32),
+                                   eager[k].view(torch.int16 if v.dtype == torch.bfloat16 else torch.int32)), k
+    assert ws.device_status() == 0 and wsn.device_status() == 0
+    assert_close("graph gae", outs["adv"].cpu().numpy(), run_oracle(oracle, ro, ("gae",))["gae"][0])
+
+
 # ------------------------------------------------------------------ test hooks
 def test_affine_scan_matches_generic_recurrence(oracle, W, B):
     import torch
