@@ -541,7 +541,7 @@ def cpu_baseline(ro, budget_s: float = 20.0):
     t = oracle_pass(ro, probe_rows, threads)                          # calibration (also warms the library)
     rows = int(min(ro.N, max(probe_rows, probe_rows * budget_s / max(t, 1e-6))))
     secs = oracle_pass(ro, rows, threads)
-    rows1 = max(16, rows // (4 * threads))                            # about a quarter of that time on one thread
+    rows1 = int(min(rows, max(64, rows * 3.0 / max(secs * threads, 1e-3))))   # about 3 CPU-seconds' worth of rows at the multi-thread rate
     secs1 = oracle_pass(ro, rows1, 1)
     return {"value": len(ALGOS) * rows * ro.T / secs, "unit": METRIC, "cores": threads, "kind": "oracle",
             "single_thread_value": len(ALGOS) * rows1 * ro.T / secs1, "cpu_model": _cpu_model(),
