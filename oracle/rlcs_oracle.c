@@ -33,7 +33,11 @@
  * Every function below is pinned by tests that do not use this file's
  * formulas: Table 1's literal (alpha, beta, carry) solved by the explicit
  * O(T^2) sum, closed forms, special cases (gamma=0, lambda=0, lambda=1),
- * cross-algorithm identities and the paper's 4-step expansion.
+ * cross-algorithm identities and the paper's 4-step expansion.  The routines
+ * beyond the seven (Retrace from [N,T,A] tensors, vector traces with a shared
+ * or a per-component decay, GAE with observation-skip masking) are pinned by
+ * reduction to the seven (gather / compaction / per-component equality) and by
+ * the unrolled sum of Eq. 1.  Nothing here is "parity unpinned".
  */
 #include <math.h>
 #include <stddef.h>
