@@ -680,22 +680,25 @@ def _without_truncs(ro):
     return r2
 
 
-def run_sweeps(torch, hbm_peak):
+def run_sweeps(torch, hbm_peak, pick=None, trials=5):
+    """The cold-L2 cases of configurations 1-4.  `pick` = (config, algo, T, truncs), None entries
+    matching anything, keeps only the matching cases (for a profiler run on one kernel)."""
     from paper_2608_17641_b200 import binding as B, workloads
     l2 = torch.cuda.get_device_properties(0).L2_cache_size
-    out = []
-    out.append(sweep_case(torch, B, workloads.config1(), "gae", True, hbm_peak, l2))          # config 1: latency floor
-    ro2 = workloads.config2()
-    for algo in ALGOS:                                                                         # config 2: all seven
-        out.append(sweep_case(torch, B, ro2, algo, True, hbm_peak, l2))
+    cases = [(1, lambda: workloads.config1(), "gae", True)]                                    # config 1: latency floor
+    cases += [(2, lambda: workloads.config2(), algo, True) for algo in ALGOS]                  # config 2: all seven
     for T in (32, 64, 128, 256, 512, 1024):
         for tr in (False, True):
-            ro = workloads.config3(T, True)
-            for algo in ("gae", "vtrace"):
-                out.append(sweep_case(torch, B, ro, algo, tr, hbm_peak, l2))
-    ro4 = workloads.config4()
-    for algo in ("gae", "discounted_return"):
-        out.append(sweep_case(torch, B, ro4, algo, False, hbm_peak, l2))
+            cases += [(3, (lambda T=T: workloads.config3(T, True)), algo, tr) for algo in ("gae", "vtrace")]
+    cases += [(4, lambda: workloads.config4(), algo, False) for algo in ("gae", "discounted_return")]
+    out = []
+    for cfg, make, algo, tr in cases:
+        if pick is not None and any(want is not None and want != got for want, got in zip(pick[:2], (cfg, algo))):
+            continue
+        ro = make()
+        if pick is not None and ((pick[2] is not None and pick[2] != ro.T) or (pick[3] is not None and pick[3] != tr)):
+            continue
+        out.append(sweep_case(torch, B, ro, algo, tr, hbm_peak, l2, trials=trials))
     return out
 
 
@@ -722,12 +725,17 @@ def main():
     ap.add_argument("--no-sweep", action="store_true", help="skip the cold-L2 sweeps of the smaller configurations")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sweep-only", action="store_true", help="print only the cold-L2 sweeps (one JSON line)")
+    ap.add_argument("--sweep-pick", default=None, metavar="CONFIG,ALGO,T,TRUNCS",
+                    help="with --sweep-only: keep the matching cases only, e.g. 3,vtrace,256,1 or 4,gae,, (empty = any)")
+    ap.add_argument("--sweep-trials", type=int, default=5)
     ap.add_argument("--variant", type=int, default=None, help="tile variant test hook (default: library default)")
     ap.add_argument("--no-truncs", action="store_true", help="bench batch without per-step truncation handling")
     ap.add_argument("--rows", type=int, default=WORKLOAD["N"], help="num_envs of the bench batch (default: full size)")
-    ap.add_argument("--only", choices=("time_major", "bf16"), default=None,
+    ap.add_argument("--only", choices=("time_major", "bf16", "retrace_probs", "elig_trace_vec", "elig_trace_vec_beta",
+                                       "gae_skip", "gae_normalized"), default=None,
                     help="time only that extension line on a --rows x --seq-len batch and print it (one JSON line)")
     ap.add_argument("--seq-len", type=int, default=WORKLOAD["T"], help="T of the --only batch")
+    ap.add_argument("--dim", type=int, default=64, help="D of the --only elig_trace_vec* batch, A of retrace_probs")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -757,12 +765,25 @@ def main():
 
     if args.sweep_only:
         peak, _ = measured_peak()
-        print(json.dumps({"sweeps": run_sweeps(torch, peak)}), flush=True)
+        pick = None
+        if args.sweep_pick is not None:
+            c, a, t, tr = (args.sweep_pick.split(",") + ["", "", "", ""])[:4]
+            pick = (int(c) if c else None, a or None, int(t) if t else None, bool(int(tr)) if tr else None)
+        print(json.dumps({"sweeps": run_sweeps(torch, peak, pick, max(1, args.sweep_trials))}), flush=True)
         return
     if args.only is not None:
         peak, _ = measured_peak()
-        fn = time_time_major if args.only == "time_major" else time_bf16
-        print(json.dumps({args.only: fn(torch, binding, max(1, args.steps), peak, args.rows, args.seq_len)}), flush=True)
+        k, N, T = max(1, args.steps), args.rows, args.seq_len
+        if args.only in ("time_major", "bf16"):
+            res = (time_time_major if args.only == "time_major" else time_bf16)(torch, binding, k, peak, N, T)
+        elif args.only == "retrace_probs":
+            res = time_retrace_probs(torch, binding, k, peak, N, T, args.dim)
+        elif args.only in ("elig_trace_vec", "elig_trace_vec_beta"):
+            res = time_elig_trace_vec(torch, binding, k, peak, N, T, args.dim, per_dim=args.only.endswith("beta"))
+        else:
+            batch = GpuBatch(workloads.config5(N=N, T=T, salt=rank), torch.device("cuda", local))
+            res = (time_gae_skip if args.only == "gae_skip" else time_gae_normalized)(batch, k, peak)
+        print(json.dumps({args.only: res}), flush=True)
         return
 
     N = args.rows

@@ -419,6 +419,17 @@ int rlcs_debug_set_carry_fault(int64_t mute_tile, int64_t spin_cap);
 void rlcs_debug_time_major_path(int path);
 
 /*
+ * Test hook: plan of the vector-trace entry points for subsequent calls in this process.  batch = 8,
+ * 16 or 32: the walk with one thread per component group and that many timesteps loaded ahead;
+ * batch = 1: the time-major block kernel wherever its copies can be issued; any other value: planned
+ * from N, T and D.  chunks > 0 (with the walk)
+ * cuts every row's time axis into that many chunks (capped by the minimum chunk length; 1 = never
+ * cut; <= 0: planned).  The *_workspace_bytes queries follow the forced plan.  Results must agree to
+ * rounding.
+ */
+void rlcs_debug_vec_trace_plan(int batch, int chunks);
+
+/*
  * Measurement hook: a streaming kernel that reads read_bytes from src and writes write_bytes to dst
  * (whole 32-byte pieces; both pointers 32-byte aligned, buffers at least that large; dst[0] may be
  * written when write_bytes is 0), with the scan kernels' load / store instructions and one piece

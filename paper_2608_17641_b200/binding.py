@@ -63,6 +63,7 @@ SIGNATURES = {
     "rlcs_debug_tile_elems": ([_int], _int),
     "rlcs_debug_set_carry_fault": ([_i64, _i64], _int),
     "rlcs_debug_time_major_path": ([_int], None),
+    "rlcs_debug_vec_trace_plan": ([_int, _int], None),
     "rlcs_debug_stream_copy": ([_vp, _vp, _sz, _sz, _vp], _int),
     "rlcs_debug_force_wide_index": ([_int], _int),
     "rlcs_debug_allow_cluster_carry": ([_int], _int),
@@ -392,6 +393,11 @@ def rlcs_debug_set_carry_fault(mute_tile: int = -1, spin_cap: int = 0):
 def rlcs_debug_stream_copy(src, dst, read_bytes: int, write_bytes: int, stream=None):
     """Streaming read of read_bytes from src and write of write_bytes to dst (measurement hook)."""
     _check(lib().rlcs_debug_stream_copy(src.data_ptr(), dst.data_ptr(), int(read_bytes), int(write_bytes), _stream(stream)))
+
+
+def rlcs_debug_vec_trace_plan(batch: int = 0, chunks: int = 0):
+    """Test hook: force the load-ahead depth (8/16/32) and the number of time chunks of the vector traces."""
+    lib().rlcs_debug_vec_trace_plan(int(batch), int(chunks))
 
 
 def rlcs_debug_time_major_path(path: int = 0):

@@ -28,9 +28,11 @@ int vec_trace_block(const float* x, const float* beta, const uint8_t* dones, flo
 
 namespace {
 
-constexpr int kBatch = 8;         // steps loaded before the first FMA
-constexpr int kBatchPerDim = 4;   // ... with a decay tensor beside x (twice the registers per step)
+constexpr int kBatch = 8;         // steps loaded before the first FMA (x 16 bytes per thread in flight) ...
+constexpr int kBatchMax = 32;     // ... up to this many when the threads are few
 constexpr int kThreads = 256;
+int g_force_batch = 0, g_force_chunks = 0;     // test hook: 0 = planned
+bool g_force_block = false;                    // test hook: the time-major block kernel wherever usable
 
 struct VecParams {
     const float* x;
@@ -40,6 +42,7 @@ struct VecParams {
     unsigned T, D;
     unsigned groups;          // threads per row: ceil(D / V)
     unsigned chunk;           // timesteps per chunk (== T when the time axis is not cut)
+    unsigned batch;           // steps loaded before the first FMA: 8, 16 or 32 (per-component decay: half)
     unsigned chunks;          // chunks per row
     float decay;
     const float* beta;        // PERDIM: [N, T, D] decays; beta[n, t, :] multiplies z_{t-1} into step t
@@ -86,9 +89,9 @@ template <> struct Vec<1> {
 
 // MODE 0: whole rows, write traces.  MODE 1: chunk ends and decay products only.  MODE 2: rescan
 // from the carry and write traces.
-template <int V, int MODE, bool PERDIM>
+template <int V, int MODE, bool PERDIM, int KB>
 __global__ void __launch_bounds__(kThreads) elig_vec_kernel(const VecParams p) {
-    const long long tid = (long long)blockIdx.x * kThreads + threadIdx.x;
+    const long long tid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     const long long per_row = (long long)p.groups * p.chunks;
     const long long n = tid / per_row;
     if (n >= p.N) return;
@@ -110,7 +113,6 @@ __global__ void __launch_bounds__(kThreads) elig_vec_kernel(const VecParams p) {
 
     // (A software pipeline of two alternating register batches was measured and is slower: 0.60
     // against 0.89 of the copy bandwidth for the shared-decay kernel.)
-    constexpr int KB = PERDIM ? kBatchPerDim : kBatch;
     for (unsigned t0 = t_begin; t0 < t_end; t0 += KB) {
         Vec<V> xs[KB], bs[KB];
         float beta[KB];
@@ -172,36 +174,57 @@ __global__ void __launch_bounds__(kThreads) elig_vec_chain_kernel(const VecParam
 
 inline bool aligned(const void* p, uintptr_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
 
-// chunking: cut the time axis only when N * groups threads cannot fill the GPU
-void plan(long long N, long long T, long long groups, unsigned* chunk, unsigned* chunks) {
-    // One pass needs enough threads to keep the memory system busy: each holds kBatch x 16 bytes in
-    // flight, and ~40 K threads (5 MB) already saturate HBM; below that, cut -- but into chunks of
-    // at least 128 steps and at most 256 per row, so that the ordered carry chain stays short.
-    const long long want_threads = 148ll * 256;
+// How deep each thread loads ahead, and whether the time axis is cut.  One pass keeps
+// threads x batch x 16 bytes in flight; about 300 K thread-steps (5 MB) saturate HBM with 8 steps per
+// thread.  With fewer threads the batch grows to 32 steps (0.49 -> 0.81 of the copy bandwidth at
+// 2048x512x64; 16 steps: 0.76); only when that is not enough is the time axis cut -- into chunks of
+// at least 128 steps and at most 256 per row, so that the ordered carry chain stays short.
+void plan(long long N, long long T, long long groups, bool perdim, unsigned* chunk, unsigned* chunks, unsigned* batch) {
+    const long long want = 148ll * 256 * kBatch;
+    const long long threads = N * groups;
+    unsigned kb = kBatch;
+    // (with a decay tensor the deeper batches measured slower: 0.87 -> 0.58 -> 0.38 at 16384x128x64)
+    if (!perdim && threads * kb < want) kb = kBatchMax;
+    if (g_force_batch) kb = (unsigned)g_force_batch;
     long long k = 1;
-    if (N * groups < want_threads) k = (want_threads + N * groups - 1) / (N * groups);
+    if (threads * kb < want) { kb = g_force_batch ? kb : kBatch; k = (want + threads * kb - 1) / (threads * kb); }
+    if (g_force_chunks) k = g_force_chunks;
     if (k > 256) k = 256;
     long long len = (T + k - 1) / k;
     if (len < 128) len = 128;
-    len = (len + kBatch - 1) / kBatch * kBatch;
+    len = (len + kBatchMax - 1) / kBatchMax * kBatchMax;
+    *batch = kb;
     if (len >= T) { *chunk = (unsigned)T; *chunks = 1; return; }
     *chunk = (unsigned)len;
     *chunks = (unsigned)((T + len - 1) / len);
 }
 
-template <int V, bool PERDIM>
-int run(VecParams p, cudaStream_t s) {
+template <int V, bool PERDIM, int KB>
+int run_batch(const VecParams& p, cudaStream_t s) {
     const long long threads = p.N * (long long)p.groups * p.chunks;
-    const unsigned blocks = (unsigned)((threads + kThreads - 1) / kThreads);
+    // few threads: smaller blocks, so that they spread over all SMs
+    const unsigned bt = threads < 148ll * kThreads * 2 ? 64 : kThreads;
+    const unsigned blocks = (unsigned)((threads + bt - 1) / bt);
     if (p.chunks == 1) {
-        elig_vec_kernel<V, 0, PERDIM><<<blocks, kThreads, 0, s>>>(p);
+        elig_vec_kernel<V, 0, PERDIM, KB><<<blocks, bt, 0, s>>>(p);
     } else {
-        elig_vec_kernel<V, 1, PERDIM><<<blocks, kThreads, 0, s>>>(p);
+        elig_vec_kernel<V, 1, PERDIM, KB><<<blocks, bt, 0, s>>>(p);
         const long long chain_threads = p.N * (long long)p.groups;
         elig_vec_chain_kernel<V, PERDIM><<<(unsigned)((chain_threads + kThreads - 1) / kThreads), kThreads, 0, s>>>(p);
-        elig_vec_kernel<V, 2, PERDIM><<<blocks, kThreads, 0, s>>>(p);
+        elig_vec_kernel<V, 2, PERDIM, KB><<<blocks, bt, 0, s>>>(p);
     }
     return cudaGetLastError() == cudaSuccess ? RLCS_OK : RLCS_ERR_CUDA;
+}
+
+// the per-component decay loads two tensors per step: half the steps for the same bytes in flight
+template <int V, bool PERDIM>
+int run(const VecParams& p, cudaStream_t s) {
+    constexpr int H = PERDIM ? 2 : 1;
+    switch (p.batch) {
+        case 32: return run_batch<V, PERDIM, 32 / H>(p, s);
+        case 16: return run_batch<V, PERDIM, 16 / H>(p, s);
+        default: return run_batch<V, PERDIM, 8 / H>(p, s);
+    }
 }
 
 // sizes, pointers and chunking common to both entry points; *skip = nothing to do
@@ -216,7 +239,7 @@ int prepare(VecParams& p, const float* x, const float* beta, bool perdim, const 
     *v4 = (D % 4 == 0) && aligned(x, 16) && aligned(traces, 16) && (!perdim || aligned(beta, 16));
     p.x = x; p.beta = beta; p.dones = dones; p.z = traces; p.N = N; p.T = (unsigned)T; p.D = (unsigned)D;
     p.groups = (unsigned)(*v4 ? D / 4 : D);
-    plan(N, T, p.groups, &p.chunk, &p.chunks);
+    plan(N, T, p.groups, perdim, &p.chunk, &p.chunks, &p.batch);
     if (p.chunks > 1) {
         const size_t need = sizeof(float) * (size_t)N * p.chunks * ((size_t)D + (perdim ? (size_t)D : 1));
         if (workspace == nullptr || workspace_bytes < need) return RLCS_ERR_WORKSPACE;
@@ -229,10 +252,10 @@ int prepare(VecParams& p, const float* x, const float* beta, bool perdim, const 
 
 size_t workspace_bytes(int64_t N, int64_t T, int64_t D, bool perdim) {
     if (N <= 0 || T <= 0 || D <= 0 || T > (int64_t(1) << 31) - 1 || D > (int64_t(1) << 24)) return 0;
-    unsigned chunk, chunks;
-    plan(N, T, (D + 3) / 4, &chunk, &chunks);
+    unsigned chunk, chunks, batch;
+    plan(N, T, (D + 3) / 4, perdim, &chunk, &chunks, &batch);
     unsigned chunk1, chunks1;
-    plan(N, T, D, &chunk1, &chunks1);                         // the element-wise variant cuts differently
+    plan(N, T, D, perdim, &chunk1, &chunks1, &batch);                         // the element-wise variant cuts differently
     const size_t k = chunks > chunks1 ? chunks : chunks1;
     if (k <= 1) return 0;
     return sizeof(float) * (size_t)N * k * ((size_t)D + (perdim ? (size_t)D : 1)) + 256;
@@ -254,10 +277,15 @@ int rlcs_elig_trace_vec(const float* x, const uint8_t* dones, float* traces, int
     const int st = prepare(p, x, nullptr, false, dones, traces, N, T, D, workspace, workspace_bytes, &v4, &skip);
     if (st != RLCS_OK || skip) return st;
     p.decay = gamma * lambda;
-    // (For few long rows the time-major block kernel, which reads x once, was measured against the
-    // chunked path below, which reads it twice: 0.32 against 0.41 of the copy bandwidth at 64x16384x64
-    // -- at 8 bytes per step that kernel is bound by issue slots.  It is used for the per-component
-    // decay only, where a step moves 12 bytes.)
+    // Between the sizes that fill the GPU with one thread per four components and the few long rows
+    // that need the time axis cut, the time-major block kernel (one block per row and 32 components,
+    // x read once) is faster: 0.56 -> 0.63 of the copy bandwidth at 1024x1024x64, 0.44 -> 0.62 at
+    // 512x2048x64.  With fewer than ~600 such blocks it is not (0.32 against 0.41 at 64x16384x64: at 8
+    // bytes per step a block is bound by its per-stage latency), and the chunked path below stays.
+    const long long blocks32 = (long long)N * ((D + 31) / 32);
+    const bool mid = (long long)N * p.groups < 32768 && blocks32 >= 4 * 148;
+    if ((mid || g_force_block) && !g_force_batch && !g_force_chunks && rlcs_internal::vec_trace_block_usable(x, nullptr, N, T, D))
+        return rlcs_internal::vec_trace_block(x, nullptr, dones, traces, N, T, D, p.decay, cuda_stream);
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
     return v4 ? run<4, false>(p, s) : run<1, false>(p, s);
 }
@@ -268,12 +296,20 @@ int rlcs_elig_trace_vec_beta(const float* x, const float* beta, const uint8_t* d
     bool v4 = false, skip = false;
     const int st = prepare(p, x, beta, true, dones, traces, N, T, D, workspace, workspace_bytes, &v4, &skip);
     if (st != RLCS_OK || skip) return st;
-    // few long rows: instead of cutting the time axis (x and beta read twice), stream each row once
-    // through the time-major block kernel (0.21 -> 0.47 of the copy bandwidth at 64x16384x64)
-    if (p.chunks > 1 && rlcs_internal::vec_trace_block_usable(x, beta, N, T, D))
+    // Wherever its copies can be issued (D a multiple of 4 and >= 32, 16-byte aligned tensors) the
+    // time-major block kernel streams each row once and is at least as fast as the thread-per-four-
+    // components walk: 0.87 -> 0.92 of the copy bandwidth at 16384x128x64, 0.63 -> 0.90 at 4096x512x64,
+    // 0.21 -> 0.47 at 64x16384x64 (where the walk would have to cut the time axis and read twice).
+    if (!g_force_batch && !g_force_chunks && rlcs_internal::vec_trace_block_usable(x, beta, N, T, D))
         return rlcs_internal::vec_trace_block(x, beta, dones, traces, N, T, D, 1.f, cuda_stream);
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
     return v4 ? run<4, true>(p, s) : run<1, true>(p, s);
+}
+
+void rlcs_debug_vec_trace_plan(int batch, int chunks) {
+    g_force_batch = (batch == 8 || batch == 16 || batch == 32) ? batch : 0;
+    g_force_block = batch == 1;
+    g_force_chunks = chunks > 0 ? chunks : 0;
 }
 
 }  // extern "C"

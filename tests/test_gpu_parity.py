@@ -564,14 +564,37 @@ def test_per_dimension_beta_eligibility_trace(oracle, W, B, N, T, D):
     off = lambda t: torch.cat([t.new_zeros(1), t.reshape(-1)])[1:].view(t.shape)
     got1 = B.rlcs_elig_trace_vec_beta(off(xd), off(bd), dd).cpu().numpy()
     assert_close("per-dimension trace, unaligned", got1, ref)
-    # a constant beta is the shared-scalar entry point, bit for bit (same FMA per step, same chunking)
+    # a constant beta is the shared-scalar entry point: bit for bit when both walk whole rows with one
+    # thread per component group (same FMA per step), to rounding under the planned kernels
     const = torch.full_like(xd, 0.25)
     same = B.rlcs_elig_trace_vec_beta(xd, const, dd)
     scalar = B.rlcs_elig_trace_vec(xd, dd, gamma=0.5, lam=0.5)
-    if int(B.lib().rlcs_elig_trace_vec_beta_workspace_bytes(N, T, D)) == 0:
-        assert torch.equal(same, scalar)                   # one pass in both: same FMA per step
-    else:                                                   # few long rows: the block kernel splits time among warps
-        assert_close("constant beta vs shared decay", same.cpu().numpy(), scalar.cpu().numpy().astype(np.float64))
+    assert_close("constant beta vs shared decay", same.cpu().numpy(), scalar.cpu().numpy().astype(np.float64))
+    B.rlcs_debug_vec_trace_plan(8, 1)
+    try:
+        assert torch.equal(B.rlcs_elig_trace_vec_beta(xd, const, dd), B.rlcs_elig_trace_vec(xd, dd, gamma=0.5, lam=0.5))
+    finally:
+        B.rlcs_debug_vec_trace_plan(0, 0)
+
+
+@pytest.mark.parametrize("plan", [(1, 0), (8, 1), (16, 1), (32, 1), (8, 3), (32, 2), (16, 7)])
+@pytest.mark.parametrize("N,T,D", [(8, 128, 64), (5, 999, 3), (48, 2000, 96), (3, 700, 36), (130, 300, 32)])
+def test_vector_trace_plans_agree(oracle, W, B, N, T, D, plan):
+    """Every load-ahead depth, forced time cuts and the block kernel give the oracle's traces."""
+    import torch
+    rng = np.random.default_rng(N * 7919 + T * 31 + D + 2)
+    x = rng.standard_normal((N, T, D)).astype(np.float32)
+    beta = rng.uniform(0.5, 1.0, (N, T, D)).astype(np.float32)
+    d = (rng.random((N, T)) < 0.02).astype(np.uint8)
+    xd, bd, dd = torch.from_numpy(x).cuda(), torch.from_numpy(beta).cuda(), torch.from_numpy(d).cuda()
+    B.rlcs_debug_vec_trace_plan(*plan)
+    try:
+        got = B.rlcs_elig_trace_vec(xd, dd, gamma=0.99, lam=0.95).cpu().numpy()
+        gotb = B.rlcs_elig_trace_vec_beta(xd, bd, dd).cpu().numpy()
+    finally:
+        B.rlcs_debug_vec_trace_plan(0, 0)
+    assert_close(f"vector trace, plan {plan}", got, oracle.elig_trace_vec(x, d, gamma=0.99, lam=0.95))
+    assert_close(f"per-dimension trace, plan {plan}", gotb, oracle.elig_trace_vec_beta(x, beta, d))
 
 
 def test_per_dimension_beta_argument_checks(oracle, W, B):
