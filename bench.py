@@ -735,6 +735,7 @@ def main():
                                        "gae_skip", "gae_normalized"), default=None,
                     help="time only that extension line on a --rows x --seq-len batch and print it (one JSON line)")
     ap.add_argument("--seq-len", type=int, default=WORKLOAD["T"], help="T of the --only batch")
+    ap.add_argument("--tm-path", type=int, default=0, help="time-major path test hook for --only runs (0 = library default)")
     ap.add_argument("--dim", type=int, default=64, help="D of the --only elig_trace_vec* batch, A of retrace_probs")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
@@ -773,6 +774,7 @@ def main():
         return
     if args.only is not None:
         peak, _ = measured_peak()
+        binding.rlcs_debug_time_major_path(args.tm_path)
         k, N, T = max(1, args.steps), args.rows, args.seq_len
         if args.only in ("time_major", "bf16"):
             res = (time_time_major if args.only == "time_major" else time_bf16)(torch, binding, k, peak, N, T)

@@ -272,10 +272,17 @@ size_t rlcs_no_alloc_scratch_bytes(void);
  * A lane per environment walks its timesteps in scan order.  When N is a multiple of 16 and the
  * per-step inputs are 16-byte aligned each warp streams its 32 columns through a shared-memory ring
  * of asynchronous copies; otherwise the same walk runs from registers (any N, 4-byte alignment).
- * When N alone cannot fill the GPU the time axis is cut into chunks and the inputs are read twice
- * (chunk aggregates, ordered carry chain, second walk), which needs `workspace` of
- * rlcs_time_major_workspace_bytes(N, T) bytes (0 when no cut is needed; 4-byte aligned, no
- * initialisation required).  The workspace carries no status word: nothing in these kernels waits.
+ * When N alone cannot fill the GPU the time axis is cut into chunks.  On the ring path one launch
+ * chains them: thread blocks take (column block, chunk) pairs in scan order from a ticket counter,
+ * walk their chunk for its aggregate, obtain the carry into it from the records of the chunks before
+ * (a bounded wait) and walk it again from L2 to write the outputs; on the register path three
+ * launches read the inputs twice (chunk aggregates, ordered carry chain, second walk).  Either way
+ * the result does not depend on timing.  Both need `workspace` of
+ * rlcs_time_major_workspace_bytes(N, T) bytes (0 when no cut is needed): 16-byte aligned; its
+ * contents need no initialisation for the results, but word 2 is a status word like that of the
+ * row-major workspaces (set to RLCS_ERR_TIMEOUT when a wait ran out, read and cleared by
+ * rlcs_last_device_status), so zero the first 256 bytes once -- rlcs_workspace_init does -- if you
+ * intend to query it.  Calls that may overlap on the GPU need separate workspaces.
  */
 size_t rlcs_time_major_workspace_bytes(int64_t N, int64_t T);
 int rlcs_gae_time_major(const float* rewards, const float* values, const uint8_t* dones, const uint8_t* truncs,
@@ -406,15 +413,20 @@ int rlcs_debug_force_wide_index(int on);
  * whose scan-order index is `mute_tile` does not publish its tile record (negative = publish
  * normally), and the wait gives up after `spin_cap` polls (<= 0 = default).  A dependent block
  * then runs out of polls within microseconds, records RLCS_ERR_TIMEOUT in the workspace status
- * word and finishes normally -- nothing hangs or faults.
+ * word and finishes normally -- nothing hangs or faults.  The chained time-major kernel (and the
+ * vector traces that use it) honours both: there `mute_tile` is the ticket of the block that
+ * publishes neither its chunk aggregate nor the value it carries out.
  */
 int rlcs_debug_set_carry_fault(int64_t mute_tile, int64_t spin_cap);
 
 /*
  * Test hook: path of the time-major entry points for subsequent calls in this process.  1 = the
  * register walk whatever the alignment; 3 = the shared-memory ring with one column per lane whatever
- * the size; any other value = the default (the ring wherever N and the pointers allow it, two
- * columns per lane for large N).  Results must agree to rounding.
+ * the size; 4 = a cut time axis always by three launches, never the chained kernel; 5 = the chained
+ * kernel whenever T exceeds one of its chunks, also where N alone would fill the GPU (the workspace
+ * query follows); any other value = the default (the ring wherever N and the pointers allow it, two
+ * columns per lane for large N, the chained kernel where the time axis is cut).  Results must agree
+ * to rounding.
  */
 void rlcs_debug_time_major_path(int path);
 

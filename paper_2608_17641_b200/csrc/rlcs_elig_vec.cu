@@ -22,8 +22,9 @@
 // the time-major block kernel, one [T, D] problem per row (rlcs_time_major.cu)
 namespace rlcs_internal {
 bool vec_trace_block_usable(const float* x, const float* beta, int64_t N, int64_t T, int64_t D);
+size_t vec_trace_block_workspace_bytes(int64_t N, int64_t T, int64_t D, bool perdim);
 int vec_trace_block(const float* x, const float* beta, const uint8_t* dones, float* traces, int64_t N, int64_t T, int64_t D,
-                    float decay, void* cuda_stream);
+                    float decay, void* workspace, size_t workspace_bytes, void* cuda_stream);
 }  // namespace rlcs_internal
 
 namespace {
@@ -257,8 +258,9 @@ size_t workspace_bytes(int64_t N, int64_t T, int64_t D, bool perdim) {
     unsigned chunk1, chunks1;
     plan(N, T, D, perdim, &chunk1, &chunks1, &batch);                         // the element-wise variant cuts differently
     const size_t k = chunks > chunks1 ? chunks : chunks1;
-    if (k <= 1) return 0;
-    return sizeof(float) * (size_t)N * k * ((size_t)D + (perdim ? (size_t)D : 1)) + 256;
+    const size_t walk = k <= 1 ? 0 : sizeof(float) * (size_t)N * k * ((size_t)D + (perdim ? (size_t)D : 1)) + 256;
+    const size_t block = rlcs_internal::vec_trace_block_workspace_bytes(N, T, D, perdim);   // the block kernel's chained chunks
+    return walk > block ? walk : block;
 }
 
 }  // namespace
@@ -277,15 +279,14 @@ int rlcs_elig_trace_vec(const float* x, const uint8_t* dones, float* traces, int
     const int st = prepare(p, x, nullptr, false, dones, traces, N, T, D, workspace, workspace_bytes, &v4, &skip);
     if (st != RLCS_OK || skip) return st;
     p.decay = gamma * lambda;
-    // Between the sizes that fill the GPU with one thread per four components and the few long rows
-    // that need the time axis cut, the time-major block kernel (one block per row and 32 components,
-    // x read once) is faster: 0.56 -> 0.63 of the copy bandwidth at 1024x1024x64, 0.44 -> 0.62 at
-    // 512x2048x64.  With fewer than ~600 such blocks it is not (0.32 against 0.41 at 64x16384x64: at 8
-    // bytes per step a block is bound by its per-stage latency), and the chunked path below stays.
-    const long long blocks32 = (long long)N * ((D + 31) / 32);
-    const bool mid = (long long)N * p.groups < 32768 && blocks32 >= 4 * 148;
+    // Below the sizes that fill the GPU with one thread per four components the time-major block kernel
+    // (one block per row and 32 components, x read from HBM once) is faster: 0.56 -> 0.63 of the copy
+    // bandwidth at 1024x1024x64, 0.44 -> 0.62 at 512x2048x64; for few long rows it cuts the time axis
+    // and chains the chunks in one launch (0.41 -> 0.46 at 64x16384x64, against the three-launch
+    // chunked walk below, which reads x twice and remains for shapes the block kernel cannot take).
+    const bool mid = (long long)N * p.groups < 32768;
     if ((mid || g_force_block) && !g_force_batch && !g_force_chunks && rlcs_internal::vec_trace_block_usable(x, nullptr, N, T, D))
-        return rlcs_internal::vec_trace_block(x, nullptr, dones, traces, N, T, D, p.decay, cuda_stream);
+        return rlcs_internal::vec_trace_block(x, nullptr, dones, traces, N, T, D, p.decay, workspace, workspace_bytes, cuda_stream);
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
     return v4 ? run<4, false>(p, s) : run<1, false>(p, s);
 }
@@ -301,7 +302,7 @@ int rlcs_elig_trace_vec_beta(const float* x, const float* beta, const uint8_t* d
     // components walk: 0.87 -> 0.92 of the copy bandwidth at 16384x128x64, 0.63 -> 0.90 at 4096x512x64,
     // 0.21 -> 0.47 at 64x16384x64 (where the walk would have to cut the time axis and read twice).
     if (!g_force_batch && !g_force_chunks && rlcs_internal::vec_trace_block_usable(x, beta, N, T, D))
-        return rlcs_internal::vec_trace_block(x, beta, dones, traces, N, T, D, 1.f, cuda_stream);
+        return rlcs_internal::vec_trace_block(x, beta, dones, traces, N, T, D, 1.f, workspace, workspace_bytes, cuda_stream);
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
     return v4 ? run<4, true>(p, s) : run<1, true>(p, s);
 }

@@ -9,26 +9,35 @@
 // (successor value selected by flag, the recurrence continued only where no flag is set): no scan,
 // no shuffles.
 //
-// Two kernels share that arithmetic:
-//   * tm_staged_kernel: each warp streams its 32 columns through a private ring of shared-memory
-//     stages filled by 16-byte asynchronous copies (cp.async), kRows timesteps per stage.  Load
-//     addresses do not depend on the recurrence, so S-1 stages are in flight per warp whatever the
-//     register budget; the host sizes S so that the whole grid keeps roughly 16 MB in flight.  Warps
-//     never synchronise with one another.  Needs N % 16 == 0 and 16-byte aligned inputs.
-//   * tm_kernel: the same walk with two alternating register blocks instead of the ring; any N and
-//     any 4-byte alignment.
+// Kernels that share that arithmetic:
+//   * tm_block_kernel: a thread block owns 32 (or 64) adjacent environments and streams their rows
+//     through a ring of shared-memory stages filled by 16-byte asynchronous copies (cp.async); its
+//     warps split every stage in time (per-warp walk from carry 0, aggregates through shared memory,
+//     fold, one FMA per step).  Load addresses do not depend on the recurrence, so S-1 stages are in
+//     flight per block whatever the register budget.  Needs N % 16 == 0 and 16-byte aligned inputs.
+//   * tm_kernel: a lane per environment walking from two alternating register blocks; any N and any
+//     4-byte alignment.
+//   * tm_block_chained_kernel: the block kernel over a cut time axis, in one launch (below).
 //
-// Parallelism is N/32 warps.  When that cannot fill the GPU the time axis is cut into chunks:
-// pass 1 walks every chunk with carry 0 and keeps only its aggregate (a, b) of Eq. 2, a small pass
-// chains the carries of an environment's chunks in scan order, and pass 3 walks every chunk again
-// from its carry and writes the outputs (inputs are then read twice, the second time mostly from
-// L2 at the sizes where a cut is needed).  Deterministic either way.
+// Parallelism is N/32 thread blocks.  When that cannot fill the GPU the time axis is cut into
+// chunks.  Ring path: one launch; blocks take (column block, chunk) pairs in scan order from a
+// ticket counter, walk their chunk for its aggregate (a, b) of Eq. 2, publish it, look back over
+// the records of the chunks before for the carry into their own, and walk the chunk again -- out of
+// L2 -- to write the outputs.  Register path: three launches (aggregates with carry 0, a small
+// kernel that chains an environment's chunks in scan order, second walk from the carry), the inputs
+// read twice.  Deterministic either way.
 #include <cmath>
 #include <cstdint>
 #include <type_traits>
 
 #include "../../include/rlcs.h"
 #include "rlcs_scan.cuh"
+
+// test hooks shared with the row-major entry points (rlcs_debug_set_carry_fault; defined in rlcs_api.cu)
+namespace rlcs_hooks {
+extern long long g_mute_tile;      // scan-order tile / block ticket that does not publish
+extern long long g_spin_cap;       // poll limit (0 = default)
+}  // namespace rlcs_hooks
 
 namespace {
 
@@ -63,6 +72,14 @@ struct TmParams {
     long long batch, batch_stride;                // kTmVec*: independent [T, N] problems (blockIdx.z), elements between them
     float* agg_a;             // [chunks, N] pass 1: chunk aggregates; after the chain: carry into each chunk
     float* agg_b;             // [chunks, N]
+    // tm_block_chained_kernel: header[63] = block ticket counter, header[2] = status word (both in the
+    // workspace's first 256 bytes), records[(z * chunks + scan-order chunk) * npad + column]
+    unsigned* header;
+    uint4* records;
+    unsigned colblocks;       // thread blocks across the columns
+    long long npad;           // colblocks * 32 * cols_per_lane
+    unsigned spin_cap;        // polls of one record before the kernel gives up
+    long long mute_ticket;    // test hook: the block with this ticket publishes nothing (-1: none)
 };
 
 // Vector-valued eligibility traces x[n] : [T, D] are time-major problems with D columns per row n and
@@ -509,18 +526,13 @@ __device__ __forceinline__ int wrap_prev(int x, int n) { return x == 0 ? n - 1 :
 // have landed so have the masks two stages on, and the sparse truncation values they point at are
 // requested two stages before their use (registers bv1, bv2).
 // MODE as in tm_kernel.
+// block_walk: chunk k of the block's 32 C columns from n0.  A: in, the carry into the chunk (MODE 0: 0;
+// MODE 1: 0); out, the recurrence value after the chunk's last step.  P: out, the product of the
+// chunk's betas.  Every thread returns the values of its own columns.
 template <int ALGO, bool TRUNC, int MODE, int W, int C>
-__global__ void __launch_bounds__(32 * W) tm_block_kernel(const TmParams p_in) {
+__device__ __forceinline__ void block_walk(const TmParams& p, const long long n0, const unsigned k, float (&A)[C], float (&P)[C]) {
     constexpr bool FWD = tm_forward(ALGO);
     constexpr bool ROWMASK = tm_row_mask(ALGO);
-    TmParams p = p_in;
-    if constexpr (ROWMASK) {                                 // this block's row of the batch
-        const long long off = (long long)blockIdx.z * p_in.batch_stride;
-        p.f0 += off;
-        if constexpr (ALGO == kTmVecBeta) p.f1 += off;
-        p.out0 += off;
-        p.dones += (long long)blockIdx.z * p_in.T;
-    }
     using SV = StageView<ALGO, TRUNC, W, C>;
     extern __shared__ __align__(16) unsigned char tm_smem[];
     const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
@@ -533,10 +545,8 @@ __global__ void __launch_bounds__(32 * W) tm_block_kernel(const TmParams p_in) {
     float* const edge_v = reinterpret_cast<float*>(agg + 2 * W * 32 * C);               // [2][32 C]
     float* const edge_x = edge_v + 64 * C;                                              // [2][32 C] log-ratio | dones flag
 
-    const long long n0 = (long long)blockIdx.x * (32 * C);
     const bool write = n0 + C * lane < p.N;                  // lanes past N read zero-filled columns (N is even)
     const unsigned write_mask = write ? ~0u : 0u;
-    const unsigned k = blockIdx.y;
     const unsigned t_lo = k * p.chunk;
     const unsigned t_hi = min(p.T, t_lo + p.chunk);
     const unsigned len = t_hi - t_lo;
@@ -552,12 +562,11 @@ __global__ void __launch_bounds__(32 * W) tm_block_kernel(const TmParams p_in) {
 
     // block state per column: the affine map of everything walked so far applied to the chunk's incoming carry;
     // neighbours across the chunk's scan-order start
-    float A[C], P[C], bootv[C], v0[C], lr0[C];
+    float bootv[C], v0[C], lr0[C];
     unsigned d0[C];
 #pragma unroll
     for (int c = 0; c < C; ++c) {
         const long long n = write ? n0 + C * lane + c : p.N - 1;
-        A[c] = MODE == 2 ? p.agg_a[(long long)k * p.N + n] : 0.f;
         P[c] = 1.f;
         bootv[c] = (!FWD && p.boot != nullptr) ? __ldg(p.boot + n) : 0.f;
         BackState b0 = {};
@@ -785,6 +794,33 @@ __global__ void __launch_bounds__(32 * W) tm_block_kernel(const TmParams p_in) {
         left -= R;
     }
     cp_async_wait(0);
+}
+
+// this block's problem of a batch (vector traces: row z)
+template <int ALGO>
+__device__ __forceinline__ TmParams batch_slice(const TmParams& p_in, unsigned z) {
+    TmParams p = p_in;
+    if constexpr (tm_row_mask(ALGO)) {
+        const long long off = (long long)z * p_in.batch_stride;
+        p.f0 += off;
+        if constexpr (ALGO == kTmVecBeta) p.f1 += off;
+        p.out0 += off;
+        p.dones += (long long)z * p_in.T;
+    }
+    return p;
+}
+
+template <int ALGO, bool TRUNC, int MODE, int W, int C>
+__global__ void __launch_bounds__(32 * W) tm_block_kernel(const TmParams p_in) {
+    const TmParams p = batch_slice<ALGO>(p_in, blockIdx.z);
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    const long long n0 = (long long)blockIdx.x * (32 * C);
+    const unsigned k = blockIdx.y;
+    const bool write = n0 + C * lane < p.N;
+    float A[C], P[C];
+#pragma unroll
+    for (int c = 0; c < C; ++c) A[c] = (MODE == 2 && write) ? p.agg_a[(long long)k * p.N + n0 + C * lane + c] : 0.f;
+    block_walk<ALGO, TRUNC, MODE, W, C>(p, n0, k, A, P);
     if (MODE == 1 && write && w == 0) {
 #pragma unroll
         for (int c = 0; c < C; ++c) {
@@ -792,6 +828,90 @@ __global__ void __launch_bounds__(32 * W) tm_block_kernel(const TmParams p_in) {
             p.agg_b[(long long)k * p.N + n0 + C * lane + c] = P[c];
         }
     }
+}
+
+// The time axis cut without a second read from HBM: one launch, every block takes a (column block,
+// chunk) pair from a ticket counter -- chunk index slowest, so that the scan-order predecessors of a
+// chunk hold lower tickets and are running or done when it starts -- walks its chunk for the
+// aggregate (A, P) = (value after the last step from carry 0, product of betas), publishes it, looks
+// back for the carry into its chunk, publishes the value it carries out, and walks the chunk again
+// to write the outputs.  The second walk reads what the first brought into L2 moments before (the
+// chunks of all resident blocks together are a fraction of the L2).
+//
+// Records are 16 bytes {value, kind, beta product, kind}, kind 0 = not yet (the call zeroes them),
+// 1 = aggregate, 2 = carried-out value; each 8-byte half carries the kind, so a record read while it
+// changes shows two different kinds and is read again.  The carry into chunk s is by definition the
+// left fold v_j = fma(P_j, v_{j-1}, A_j) over its predecessors; the look-back walks back to the
+// nearest record that fixes a value without its own predecessor (kind 2, P = 0, or chunk 0) and
+// re-applies the aggregates after it in that same order, so the result does not depend on timing.
+// Waits are bounded: after spin_cap polls of one record the status word is set and the carry taken as 0.
+constexpr int kLookbackDepth = 16;     // aggregates remembered before waiting for a carried-out value
+
+__device__ __forceinline__ float chained_carry(const TmParams& p, long long rec0, unsigned ks) {
+    // rec0: record of scan-order chunk 0 for this column; records of later chunks follow every npad
+    float sa[kLookbackDepth], sb[kLookbackDepth];
+    int n = 0;
+    long long j = (long long)ks - 1;
+    unsigned polls = 0;
+    float start = 0.f;
+    for (;;) {
+        const uint4 v = rlcs::ld_volatile_u4(p.records + rec0 + j * p.npad);
+        const float a = __uint_as_float(v.x), b = __uint_as_float(v.z);
+        const bool ready = v.y == v.w && v.y != 0;
+        if (ready && (v.y == 2 || b == 0.f || j == 0)) { start = a; break; }
+        if (ready && n < kLookbackDepth) { sa[n] = a; sb[n] = b; ++n; --j; polls = 0; continue; }
+        // not written yet, or enough aggregates remembered: wait for this record
+        if (++polls > p.spin_cap) {
+            atomicExch(p.header + 2, rlcs::kDeviceTimeout);
+            return 0.f;
+        }
+        __nanosleep(64);
+    }
+    for (int i = n - 1; i >= 0; --i) start = fmaf(sb[i], start, sa[i]);
+    return start;
+}
+
+template <int ALGO, bool TRUNC, int W, int C>
+__global__ void __launch_bounds__(32 * W) tm_block_chained_kernel(const TmParams p_in) {
+    constexpr bool FWD = tm_forward(ALGO);
+    __shared__ unsigned s_ticket;
+    __shared__ float s_carry[32 * C];
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    if (threadIdx.x == 0) s_ticket = atomicAdd(p_in.header + 63, 1u);
+    __syncthreads();
+    const unsigned chains = p_in.colblocks * (unsigned)p_in.batch;
+    const unsigned ks = s_ticket / chains;                   // chunk in scan order
+    const unsigned chain = s_ticket - ks * chains;
+    const unsigned z = chain / p_in.colblocks;
+    const unsigned xb = chain - z * p_in.colblocks;
+    if (ks >= p_in.chunks) return;
+    const TmParams p = batch_slice<ALGO>(p_in, z);
+    const unsigned k = FWD ? ks : p.chunks - 1 - ks;
+    const long long n0 = (long long)xb * (32 * C);
+    const bool write = n0 + C * lane < p.N;
+    float A[C], P[C];
+#pragma unroll
+    for (int c = 0; c < C; ++c) A[c] = 0.f;
+    block_walk<ALGO, TRUNC, 1, W, C>(p, n0, k, A, P);
+    if (w == 0) {
+        const long long rec0 = (long long)z * p.chunks * p.npad + n0 + C * lane;
+#pragma unroll
+        for (int c = 0; c < C; ++c) {
+            float carry = 0.f;
+            if (write && (long long)s_ticket != p.mute_ticket) {
+                uint4* mine = p.records + rec0 + c + (long long)ks * p.npad;
+                rlcs::st_volatile_u4(mine, make_uint4(__float_as_uint(A[c]), 1u, __float_as_uint(P[c]), 1u));
+                if (ks > 0) carry = chained_carry(p, rec0 + c, ks);
+                if (ks + 1 < p.chunks)
+                    rlcs::st_volatile_u4(mine, make_uint4(__float_as_uint(fmaf(P[c], carry, A[c])), 2u, 0u, 2u));
+            }
+            s_carry[C * lane + c] = carry;
+        }
+    }
+    __syncthreads();                                         // also: every warp is done with the ring
+#pragma unroll
+    for (int c = 0; c < C; ++c) A[c] = s_carry[C * lane + c];
+    block_walk<ALGO, TRUNC, 2, W, C>(p, n0, k, A, P);
 }
 
 // Chain an environment's chunks in scan order: carry into chunk k = a_j + b_j * (carry into j) for the
@@ -875,9 +995,45 @@ bool allow_smem(K kernel, size_t bytes) {
     return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kSmemPerSm - 1024)) == cudaSuccess;
 }
 
+// Chunks of the chained kernel: about 32 KB of inputs per block and chunk, so that the chunks of
+// all resident blocks stay in L2 between a block's two walks (measured with the profiler at
+// 64x8192x64, per-component decay: 270 MB read from DRAM for 268 MB of inputs; the kernel is bound
+// by issue slots, 70 % busy, not by HBM); a multiple of 64 steps (every stage size divides it), at
+// least 64.
+constexpr unsigned kChainedMinChunk = 64;
+unsigned chained_chunk_len(int row_bytes) {
+    unsigned len = (32768u / (unsigned)row_bytes) / 64u * 64u;
+    return len < kChainedMinChunk ? kChainedMinChunk : len;
+}
+// bytes of workspace that cover the records of any algorithm's chunking, plus the header
+size_t chained_ws_bytes(long long N, long long T, long long batch) {
+    const long long npad = (N + 63) / 64 * 64;
+    const long long chunks = (T + kChainedMinChunk - 1) / kChainedMinChunk;
+    return 256 + sizeof(uint4) * (size_t)(npad * chunks * batch);
+}
+
+int g_force_chained = 0;   // test hook: 1 = never the chained kernel, 2 = the chained kernel whenever T allows a cut
+
 template <int ALGO, bool TRUNC, int W, int C>
-int launch_block(const TmParams& p, size_t smem, cudaStream_t s) {
-    const dim3 grid((unsigned)((p.N + 32 * C - 1) / (32 * C)), p.chunks);
+int launch_block(const TmParams& p_in, size_t smem, cudaStream_t s) {
+    TmParams p = p_in;
+    const unsigned colblocks = (unsigned)((p.N + 32 * C - 1) / (32 * C));
+    const long long batch = p.batch > 0 ? p.batch : 1;
+    if (p.chunks > 1 && p.records != nullptr) {
+        p.colblocks = colblocks;
+        p.npad = (long long)colblocks * 32 * C;
+        p.batch = batch;
+        const long long blocks = (long long)colblocks * batch * p.chunks;
+        if (blocks > 0x7fffffffll) return RLCS_ERR_SIZE;
+        auto kernel = tm_block_chained_kernel<ALGO, TRUNC, W, C>;
+        if (!allow_smem(kernel, smem)) return RLCS_ERR_CUDA;
+        // the ticket counter (the header's last word) and the records behind it
+        const size_t clear = 4 + sizeof(uint4) * (size_t)(p.npad * p.chunks * batch);
+        if (cudaMemsetAsync(reinterpret_cast<unsigned char*>(p.header) + 252, 0, clear, s) != cudaSuccess) return RLCS_ERR_CUDA;
+        kernel<<<(unsigned)blocks, 32 * W, smem, s>>>(p);
+        return cudaGetLastError() == cudaSuccess ? RLCS_OK : RLCS_ERR_CUDA;
+    }
+    const dim3 grid(colblocks, p.chunks, (unsigned)batch);
     if (p.chunks == 1) {
         if (!allow_smem(tm_block_kernel<ALGO, TRUNC, 0, W, C>, smem)) return RLCS_ERR_CUDA;
         tm_block_kernel<ALGO, TRUNC, 0, W, C><<<grid, 32 * W, smem, s>>>(p);
@@ -901,6 +1057,15 @@ int launch(TmParams p, bool staged, cudaStream_t s) {
         // per thread cost more occupancy than the shared addressing saves).
         constexpr bool kWide = !TRUNC && (ALGO == kGae || ALGO == kTdLambda);
         const bool wide_ok = kWide && g_force_cols != 1 && aligned8(p.out0) && aligned8(p.out1);
+        if (p.header != nullptr && g_force_chained != 1 && (p.chunks > 1 || g_force_chained == 2)) {
+            // the time axis is cut: one launch with chained carries instead of three with a second read
+            const unsigned len = chained_chunk_len(tm_row_bytes(ALGO, TRUNC));
+            if (len < p.T) {
+                p.chunk = len;
+                p.chunks = (p.T + len - 1) / len;
+                p.records = reinterpret_cast<uint4*>(reinterpret_cast<unsigned char*>(p.header) + 256);
+            }
+        }
         const size_t smem = plan_block(p, tm_rows(ALGO), tm_row_bytes(ALGO, TRUNC), TRUNC, wide_ok);
         if constexpr (kWide) {
             if (p.cols_per_lane == 2) return launch_block<ALGO, TRUNC, 4, 2>(p, smem, s);
@@ -922,6 +1087,17 @@ int launch(TmParams p, bool staged, cudaStream_t s) {
 
 inline bool aligned4(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 3u) == 0; }
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+constexpr unsigned kDefaultSpinCap = 1u << 22;    // polls of one record (64 ns apart or more) before a chained kernel gives up
+unsigned spin_cap() { return rlcs_hooks::g_spin_cap > 0 ? (unsigned)rlcs_hooks::g_spin_cap : kDefaultSpinCap; }
+
+// workspace of the time-major entry points: 256-byte header, then whichever is larger of the chained
+// kernel's records and the three-launch path's two aggregate arrays
+size_t tm_ws_bytes(long long N, long long T, unsigned chunks) {
+    const size_t chained = chained_ws_bytes(N, T, 1);
+    const size_t three = 256 + 2 * sizeof(float) * (size_t)N * chunks;
+    return chained > three ? chained : three;
+}
 inline bool unit(float v) { return v >= 0.f && v <= 1.f; }
 
 // the staged kernels copy 16-byte pieces of every per-step input
@@ -950,11 +1126,15 @@ int prepare(TmParams& p, int64_t N, int64_t T, const void* const* f32, int nf32,
     p.N = N;
     p.T = (unsigned)T;
     plan_chunks(N, T, &p.chunk, &p.chunks);
-    if (p.chunks > 1) {
-        const size_t need = 2 * sizeof(float) * (size_t)N * p.chunks;
+    p.spin_cap = spin_cap();
+    p.mute_ticket = rlcs_hooks::g_mute_tile;
+    if (p.chunks > 1 || g_force_chained == 2) {
+        const size_t need = tm_ws_bytes(N, T, p.chunks);
         if (workspace == nullptr || workspace_bytes < need) return RLCS_ERR_WORKSPACE;
-        if (!aligned4(workspace)) return RLCS_ERR_ALIGN;
-        p.agg_a = static_cast<float*>(workspace);
+        if (!aligned16(workspace)) return RLCS_ERR_ALIGN;
+        // header (256 bytes), then either the chained kernel's records or the three-launch path's aggregates
+        p.header = static_cast<unsigned*>(workspace);
+        p.agg_a = reinterpret_cast<float*>(static_cast<unsigned char*>(workspace) + 256);
         p.agg_b = p.agg_a + (size_t)N * p.chunks;
     }
     return RLCS_OK;
@@ -974,37 +1154,58 @@ int run(const TmParams& p, void* cuda_stream) {
 // its warps splitting every stage in time.
 namespace rlcs_internal {
 
-// usable when every row of D floats can be copied in 16-byte pieces and rows alone give enough blocks
-bool vec_trace_block_usable(const float* x, const float* beta, int64_t N, int64_t T, int64_t D) {
+// usable when every row of D floats can be copied in 16-byte pieces and there are enough blocks
+bool vec_trace_block_shape_ok(int64_t N, int64_t T, int64_t D) {
     if (g_force_path == 1) return false;
     if (D % 4 != 0 || D < 32 || T < 64) return false;
-    if (!aligned16(x) || (beta != nullptr && !aligned16(beta))) return false;
     return (D + 31) / 32 * N >= 96 && N <= 65535;
+}
+bool vec_trace_block_usable(const float* x, const float* beta, int64_t N, int64_t T, int64_t D) {
+    return vec_trace_block_shape_ok(N, T, D) && aligned16(x) && (beta == nullptr || aligned16(beta));
+}
+
+// Few long rows: fewer than three or four blocks per SM from rows and components alone; the time axis
+// is then cut and the chunks chained inside one launch (measured, per-component decay: 0.47 -> 0.57
+// of the copy bandwidth at 64x16384x64 with 128 uncut blocks, 0.61 -> 0.57 at 256x4096x64 with 512;
+// shared decay: 0.43 -> 0.46 at 256x4096x64; chunks of 16-128 KB all within 0.05 of one another).
+bool vec_trace_block_cuts(int64_t N, int64_t T, int64_t D, bool perdim) {
+    if (g_force_chained == 1) return false;
+    const unsigned len = chained_chunk_len(tm_row_bytes(perdim ? kTmVecBeta : kTmVec, false));
+    if ((int64_t)len >= T) return false;
+    return g_force_chained == 2 || (D + 31) / 32 * N < (perdim ? 3 : 4) * kSms;
+}
+
+size_t vec_trace_block_workspace_bytes(int64_t N, int64_t T, int64_t D, bool perdim) {
+    return vec_trace_block_shape_ok(N, T, D) && vec_trace_block_cuts(N, T, D, perdim) ? chained_ws_bytes(D, T, N) : 0;
 }
 
 int vec_trace_block(const float* x, const float* beta, const uint8_t* dones, float* traces, int64_t N, int64_t T, int64_t D,
-                    float decay, void* cuda_stream) {
+                    float decay, void* workspace, size_t workspace_bytes, void* cuda_stream) {
     TmParams p = {};
     p.f0 = x; p.f1 = beta; p.dones = dones; p.out0 = traces;
     p.N = D; p.T = (unsigned)T; p.chunk = (unsigned)T; p.chunks = 1;
     p.decay = decay;
     p.batch = N; p.batch_stride = T * D;
+    p.spin_cap = spin_cap();
+    p.mute_ticket = rlcs_hooks::g_mute_tile;
+    const bool perdim = beta != nullptr;
+    if (vec_trace_block_cuts(N, T, D, perdim)) {
+        if (workspace == nullptr || workspace_bytes < chained_ws_bytes(D, T, N)) return RLCS_ERR_WORKSPACE;
+        if (!aligned16(workspace)) return RLCS_ERR_ALIGN;
+        p.header = static_cast<unsigned*>(workspace);
+        p.records = reinterpret_cast<uint4*>(static_cast<unsigned char*>(workspace) + 256);
+        p.chunk = chained_chunk_len(tm_row_bytes(perdim ? kTmVecBeta : kTmVec, false));
+        p.chunks = (p.T + p.chunk - 1) / p.chunk;
+    }
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
     auto go = [&](auto algo_tag) {
         constexpr int ALGO = decltype(algo_tag)::value;
         const size_t smem = plan_block(p, tm_rows(ALGO), tm_row_bytes(ALGO, false), false, false);
-        const dim3 grid((unsigned)((D + 31) / 32), 1, (unsigned)N);
-        auto launch_w = [&](auto w_tag) {
-            constexpr int W = decltype(w_tag)::value;
-            if (!allow_smem(tm_block_kernel<ALGO, false, 0, W, 1>, smem)) return (int)RLCS_ERR_CUDA;
-            tm_block_kernel<ALGO, false, 0, W, 1><<<grid, 32 * W, smem, s>>>(p);
-            return cudaGetLastError() == cudaSuccess ? (int)RLCS_OK : (int)RLCS_ERR_CUDA;
-        };
-        if (p.warps_per_block == 16) return launch_w(std::integral_constant<int, 16>{});
-        if (p.warps_per_block == 8) return launch_w(std::integral_constant<int, 8>{});
-        return launch_w(std::integral_constant<int, 4>{});
+        if (p.warps_per_block == 16) return launch_block<ALGO, false, 16, 1>(p, smem, s);
+        if (p.warps_per_block == 8) return launch_block<ALGO, false, 8, 1>(p, smem, s);
+        return launch_block<ALGO, false, 4, 1>(p, smem, s);
     };
-    return beta != nullptr ? go(std::integral_constant<int, kTmVecBeta>{}) : go(std::integral_constant<int, kTmVec>{});
+    return perdim ? go(std::integral_constant<int, kTmVecBeta>{}) : go(std::integral_constant<int, kTmVec>{});
 }
 
 }  // namespace rlcs_internal
@@ -1015,12 +1216,13 @@ size_t rlcs_time_major_workspace_bytes(int64_t N, int64_t T) {
     if (N <= 0 || T <= 0 || T > (int64_t(1) << 31) - 1) return 0;
     unsigned chunk, chunks;
     plan_chunks(N, T, &chunk, &chunks);
-    return chunks > 1 ? 2 * sizeof(float) * (size_t)N * chunks : 0;
+    return (chunks > 1 || g_force_chained == 2) ? tm_ws_bytes(N, T, chunks) : 0;
 }
 
 void rlcs_debug_time_major_path(int path) {
-    g_force_path = path == 3 ? 2 : path;
+    g_force_path = path == 1 ? 1 : 0;
     g_force_cols = path == 3 ? 1 : 0;
+    g_force_chained = path == 4 ? 1 : path == 5 ? 2 : 0;
 }
 
 int rlcs_gae_time_major(const float* rewards, const float* values, const uint8_t* dones, const uint8_t* truncs,

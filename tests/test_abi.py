@@ -160,7 +160,8 @@ def test_time_major_validation_and_workspace_plan(L):
     # enough environments: whole columns, no workspace; few environments: the time axis is cut
     assert L.rlcs_time_major_workspace_bytes(100000, 64) == 0 and L.rlcs_time_major_workspace_bytes(3072, 5000) == 0
     need = L.rlcs_time_major_workspace_bytes(8, 4096)
-    assert need > 0 and need % (2 * 4 * 8) == 0            # two floats per chunk and environment
+    # header, then the larger of: one 16-byte record per 64-step chunk and (padded) column, two floats per chunk and column
+    assert need == 256 + 16 * 64 * (4096 // 64)
     assert L.rlcs_time_major_workspace_bytes(8, 40) == 0   # chunks are at least 64 steps
     assert tm(N=8, T=4096) == E_WS
     assert L.rlcs_elig_trace_time_major(None, P, P, 4, 8, 0.9, 0.9, None, 0, None) == E_NULL

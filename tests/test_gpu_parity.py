@@ -577,7 +577,7 @@ def test_per_dimension_beta_eligibility_trace(oracle, W, B, N, T, D):
         B.rlcs_debug_vec_trace_plan(0, 0)
 
 
-@pytest.mark.parametrize("plan", [(1, 0), (8, 1), (16, 1), (32, 1), (8, 3), (32, 2), (16, 7)])
+@pytest.mark.parametrize("plan", [(1, 0), (8, 1), (16, 1), (32, 1), (8, 3), (32, 2), (16, 7), "chained", "unchained"])
 @pytest.mark.parametrize("N,T,D", [(8, 128, 64), (5, 999, 3), (48, 2000, 96), (3, 700, 36), (130, 300, 32)])
 def test_vector_trace_plans_agree(oracle, W, B, N, T, D, plan):
     """Every load-ahead depth, forced time cuts and the block kernel give the oracle's traces."""
@@ -587,12 +587,19 @@ def test_vector_trace_plans_agree(oracle, W, B, N, T, D, plan):
     beta = rng.uniform(0.5, 1.0, (N, T, D)).astype(np.float32)
     d = (rng.random((N, T)) < 0.02).astype(np.uint8)
     xd, bd, dd = torch.from_numpy(x).cuda(), torch.from_numpy(beta).cuda(), torch.from_numpy(d).cuda()
-    B.rlcs_debug_vec_trace_plan(*plan)
+    if isinstance(plan, str):            # the block kernel, its time axis always / never cut into chained chunks
+        B.rlcs_debug_vec_trace_plan(1, 0)
+        B.rlcs_debug_time_major_path(5 if plan == "chained" else 4)
+    else:
+        B.rlcs_debug_vec_trace_plan(*plan)
     try:
         got = B.rlcs_elig_trace_vec(xd, dd, gamma=0.99, lam=0.95).cpu().numpy()
         gotb = B.rlcs_elig_trace_vec_beta(xd, bd, dd).cpu().numpy()
+        if plan == "chained":
+            assert np.array_equal(gotb, B.rlcs_elig_trace_vec_beta(xd, bd, dd).cpu().numpy())
     finally:
         B.rlcs_debug_vec_trace_plan(0, 0)
+        B.rlcs_debug_time_major_path(0)
     assert_close(f"vector trace, plan {plan}", got, oracle.elig_trace_vec(x, d, gamma=0.99, lam=0.95))
     assert_close(f"per-dimension trace, plan {plan}", gotb, oracle.elig_trace_vec_beta(x, beta, d))
 
@@ -706,7 +713,7 @@ def tm_path(B, request):
 @pytest.mark.parametrize("N,T", [(1, 1), (3, 7), (8, 128), (300, 65), (4096, 64), (64, 3000), (5, 20000), (40000, 33),
                                  (16, 1), (48, 517), (4112, 70), (16, 20000), (20000, 9), (19024, 300)])
 @pytest.mark.parametrize("p_flag", [0.0, 0.02, 0.5])
-@pytest.mark.parametrize("tm_path", [1, 2, 3], indirect=True)
+@pytest.mark.parametrize("tm_path", [1, 2, 3, 4, 5], indirect=True)
 def test_time_major_entry_points(oracle, W, B, N, T, p_flag, tm_path):
     """All seven algorithms on [T, N] tensors against the oracle run on the transposed arrays; shapes
     cover the single-pass walk (many environments), the cut time axis (few environments), both
@@ -717,6 +724,10 @@ def test_time_major_entry_points(oracle, W, B, N, T, p_flag, tm_path):
         pytest.skip("the ring needs N % 16 == 0; the register walk is covered by tm_path = 1")
     if tm_path == 3 and N < 18944:
         pytest.skip("one column per lane is what tm_path = 2 already takes at this size")
+    if tm_path == 4 and (N >= 3072 or T <= 64):
+        pytest.skip("the time axis is not cut at this size: three launches against one chained launch is no choice here")
+    if tm_path == 5 and T <= 64:
+        pytest.skip("no chunk of the chained kernel is shorter than the whole window")
     ro = W.make_rollout(115, N, T, p_done=p_flag, p_trunc=p_flag / 2, salt=T)
     p = ro.params
     ref = run_oracle(oracle, ro, ALL_ALGOS)
@@ -783,6 +794,62 @@ def test_time_major_paths_agree_and_misaligned_inputs_fall_back(oracle, W, B):
         mis.append(buf[1:].view(T, N))
     out = B.rlcs_gae_time_major(*mis, bt, gamma=p["gamma"], lam=p["lam"])
     assert torch.equal(out[0], outs[0][0]) and torch.equal(out[1], outs[0][1])
+
+
+@pytest.mark.parametrize("N,T,p_flag", [(64, 3000, 0.0), (64, 3000, 0.01), (16, 20000, 0.0005), (2048, 700, 0.0)])
+def test_time_major_chained_kernel_is_reproducible_and_agrees_with_three_launches(oracle, W, B, N, T, p_flag):
+    """Cut time axis: the single chained launch gives the same bits run after run (its look-back
+    re-applies aggregates in a fixed order whatever the timing), and agrees to rounding with the
+    three-launch path.  Without flags every carry chain runs the whole window."""
+    import torch
+    ro = W.make_rollout(118, N, T, p_done=p_flag, p_trunc=p_flag / 2)
+    p = ro.params
+    al = [_tm(getattr(ro, k)) for k in ("rewards", "values", "dones", "truncs", "trunc_bootstrap")]
+    bt = torch.from_numpy(ro.bootstrap).cuda()
+    x, dany = _tm(ro.x), _tm(ro.any_done)
+    outs = {}
+    for path in (5, 5, 4):
+        B.rlcs_debug_time_major_path(path)
+        try:
+            need = int(B.lib().rlcs_time_major_workspace_bytes(N, T))
+            ws = B.Workspace(N, T, nbytes=need)
+            adv, ret = B.rlcs_gae_time_major(*al, bt, gamma=p["gamma"], lam=p["lam"], workspace=ws)
+            z = B.rlcs_elig_trace_time_major(x, dany, gamma=p["gamma"], lam=p["lam"], workspace=ws)
+            torch.cuda.synchronize()
+            assert ws.device_status() == B.RLCS_OK
+            outs.setdefault(path, []).append((adv, ret, z))
+        finally:
+            B.rlcs_debug_time_major_path(0)
+    for a, b in zip(outs[5][0], outs[5][1]):
+        assert torch.equal(a, b)
+    for a, b in zip(outs[5][0], outs[4][0]):
+        assert_close("chained vs three launches", a.cpu().numpy(), b.cpu().numpy().astype(np.float64))
+    ref = run_oracle(oracle, ro, ("gae", "elig_trace"))
+    assert_close("chained gae", np.ascontiguousarray(outs[5][0][0].cpu().numpy().T), ref["gae"][0])
+    assert_close("chained elig", np.ascontiguousarray(outs[5][0][2].cpu().numpy().T), ref["elig_trace"])
+
+
+def test_time_major_chained_wait_runs_out_and_reports_timeout(oracle, W, B):
+    """A block that never publishes its chunk: the waits of the chunks after it run out of polls,
+    the kernel finishes, the status word says TIMEOUT, and the next call on the workspace is right."""
+    import torch
+    N, T = 64, 4096
+    ro = W.make_rollout(119, N, T, p_done=0.0, p_trunc=0.0)
+    p = ro.params
+    r, d = _tm(ro.rewards), _tm(ro.dones)
+    ws = B.Workspace(N, T, nbytes=int(B.lib().rlcs_time_major_workspace_bytes(N, T)))
+    B.rlcs_debug_set_carry_fault(2, 50)
+    try:
+        B.rlcs_discounted_return_time_major(r, d, gamma=p["gamma"], workspace=ws)
+        torch.cuda.synchronize()
+        assert ws.device_status() == B.RLCS_ERR_TIMEOUT
+    finally:
+        B.rlcs_debug_set_carry_fault(-1, 0)
+    assert ws.device_status() == B.RLCS_OK
+    out = B.rlcs_discounted_return_time_major(r, d, gamma=p["gamma"], workspace=ws)
+    ref = run_oracle(oracle, ro, ("discounted_return",), use_truncs=False, use_bootstrap=False)
+    assert_close("after the timeout", np.ascontiguousarray(out.cpu().numpy().T), ref["discounted_return"])
+    assert ws.device_status() == B.RLCS_OK
 
 
 def test_time_major_argument_checks(oracle, W, B):
