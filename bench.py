@@ -857,7 +857,7 @@ def main():
             time_elig_trace_vec(torch, binding, max(3, min(args.steps, 30)), peak, *shape, per_dim=True)
             for shape in ((16384, 128, 64), (4096, 512, 64), (64, 16384, 64))]
         line["extensions"]["time_major"] = [time_time_major(torch, binding, max(3, min(args.steps, 20)), peak, *shape)
-                                            for shape in ((WORKLOAD["N"], WORKLOAD["T"]), (65536, 512))]
+                                            for shape in ((WORKLOAD["N"], WORKLOAD["T"]), (65536, 512), (2048, 2048))]
         torch.cuda.empty_cache()
         line["extensions"]["bf16"] = time_bf16(torch, binding, max(3, min(args.steps, 20)), peak, WORKLOAD["N"], WORKLOAD["T"])
         torch.cuda.empty_cache()

@@ -87,17 +87,24 @@ struct TmParams {
 // few long rows): same kernel, the flag read per timestep instead of from a mask tile.
 constexpr int kTmVec = 101;        // shared scalar decay
 constexpr int kTmVecBeta = 102;    // decay per component and step in f1
-__host__ __device__ constexpr bool tm_row_mask(int a) { return a == kTmVec || a == kTmVecBeta; }
+constexpr int kTmVecBeta16 = 103;  // the same with 16 timesteps per warp and stage (see tm_rows)
+__host__ __device__ constexpr bool tm_vec_beta(int a) { return a == kTmVecBeta || a == kTmVecBeta16; }
+__host__ __device__ constexpr bool tm_row_mask(int a) { return a == kTmVec || tm_vec_beta(a); }
 __host__ __device__ constexpr bool tm_forward(int a) { return a == kElig || a == kPrefix || tm_row_mask(a); }
 // float tensors that are read at every step, and mask tensors
 __host__ __device__ constexpr int tm_nf(int a) {
-    return a == kRetrace ? 4 : a == kVtrace ? 3 : (a == kGae || a == kTdLambda || a == kTmVecBeta) ? 2 : 1;
+    return a == kRetrace ? 4 : a == kVtrace ? 3 : (a == kGae || a == kTdLambda || tm_vec_beta(a)) ? 2 : 1;
 }
 // timesteps per warp and stage in tm_block_kernel: fewer for Retrace, whose four float inputs make a
 // row 576 bytes (measured: 0.84 -> 0.90 of the copy bandwidth with 4, while the lighter algorithms
 // lose 5-12 % to the doubled per-stage overhead); more for the discounted return, whose rows are
-// 160-192 bytes (0.52 -> 0.63 at 16384 environments with 16; the forward scans lose 1 % that way)
-__host__ __device__ constexpr int tm_rows(int a) { return a == kRetrace ? 4 : a == kDisc ? 16 : 8; }
+// 160-192 bytes (0.52 -> 0.63 at 16384 environments with 16; the forward scans lose 1 % that way),
+// and for the vector traces with the shared decay (128-byte rows; 0.63 -> 0.74 at 1024x1024x64 with
+// 16, 0.61 with 32).  With a decay tensor 16 pay only while all blocks are resident at once (0.59 ->
+// 0.76 at 512x2048x64, but 0.85 -> 0.77 at 1024x1024x64): two instances, chosen by the block count.
+__host__ __device__ constexpr int tm_rows(int a) {
+    return a == kRetrace ? 4 : (a == kDisc || a == kTmVec || a == kTmVecBeta16) ? 16 : 8;
+}
 __host__ __device__ constexpr int tm_row_bytes(int a, bool trunc) { return tm_nf(a) * 128 + (tm_row_mask(a) ? 0 : (trunc ? 2 : 1) * 32); }
 
 // all ones where x != 0, else 0; written in PTX so that the flag reaches the arithmetic below as a
@@ -671,7 +678,7 @@ __device__ __forceinline__ void block_walk(const TmParams& p, const long long n0
                     unsigned dn[C], tr[C];
                     lds_f<C>(cur.f(0, row0 + u), lane, r);
                     if constexpr (ROWMASK) {
-                        if constexpr (ALGO == kTmVecBeta) lds_f<C>(cur.f(1, row0 + u), lane, x1);
+                        if constexpr (tm_vec_beta(ALGO)) lds_f<C>(cur.f(1, row0 + u), lane, x1);
 #pragma unroll
                         for (int c = 0; c < C; ++c) dn[c] = 0;
                     } else {
@@ -688,7 +695,7 @@ __device__ __forceinline__ void block_walk(const TmParams& p, const long long n0
                         Coef co;
                         if constexpr (ROWMASK) {
                             co.alpha = r[c];
-                            co.beta = keep(~ones_if(rowcut[u]), ALGO == kTmVecBeta ? x1[c] : p.decay);
+                            co.beta = keep(~ones_if(rowcut[u]), tm_vec_beta(ALGO) ? x1[c] : p.decay);
                             co.pg = 0.f;
                         } else if constexpr (FWD) {
                             co = fwd_coef<ALGO>(r[c], dn[c], d_prev[c], p, (u == 0 && w == 0 && j == 0) ? t_lo : 1u);
@@ -803,7 +810,7 @@ __device__ __forceinline__ TmParams batch_slice(const TmParams& p_in, unsigned z
     if constexpr (tm_row_mask(ALGO)) {
         const long long off = (long long)z * p_in.batch_stride;
         p.f0 += off;
-        if constexpr (ALGO == kTmVecBeta) p.f1 += off;
+        if constexpr (tm_vec_beta(ALGO)) p.f1 += off;
         p.out0 += off;
         p.dones += (long long)z * p_in.T;
     }
@@ -965,11 +972,16 @@ size_t plan_block(TmParams& p, int rows, int row_bytes, bool trunc, bool wide_ok
     const long long batch = p.batch > 0 ? p.batch : 1;
     if (wide_ok && (p.N + 63) / 64 * p.chunks * batch >= 2 * kSms) C = 2;
     const long long blocks = (p.N + 32 * C - 1) / (32 * C) * p.chunks * batch;
-    const int W = C == 2 ? 4 : blocks < kSms ? 16 : blocks < 2 * kSms ? 8 : 4;
-    const long long stage = (long long)rows * W * row_bytes * C;
-    const long long mstage = (long long)rows * W * (trunc ? 64 : 32) * C;
-    const long long fixed = 2 * mstage + (W * 512 + 512) * C;   // mask ring's two extra slots, aggregates, edges
+    int W = C == 2 ? 4 : blocks < kSms ? 16 : blocks < 2 * kSms ? 8 : 4;
+    long long stage, mstage, fixed;
+    auto size = [&]() {
+        stage = (long long)rows * W * row_bytes * C;
+        mstage = (long long)rows * W * (trunc ? 64 : 32) * C;
+        fixed = 2 * mstage + (W * 512 + 512) * C;               // mask ring's two extra slots, aggregates, edges
+    };
     auto block_bytes = [&](long long S) { return S * stage + fixed; };
+    size();
+    while (W > 4 && block_bytes(3) + 1024 > (long long)kSmemPerSm) { W /= 2; size(); }   // the minimum ring must fit
     long long resident = (blocks + kSms - 1) / kSms;
     if (resident > 6) resident = 6;
     while (resident > 1 && resident * (block_bytes(3) + 1024) > (long long)kSmemPerSm) --resident;
@@ -1155,28 +1167,31 @@ int run(const TmParams& p, void* cuda_stream) {
 namespace rlcs_internal {
 
 // usable when every row of D floats can be copied in 16-byte pieces and there are enough blocks
-bool vec_trace_block_shape_ok(int64_t N, int64_t T, int64_t D) {
-    if (g_force_path == 1) return false;
-    if (D % 4 != 0 || D < 32 || T < 64) return false;
-    return (D + 31) / 32 * N >= 96 && N <= 65535;
-}
-bool vec_trace_block_usable(const float* x, const float* beta, int64_t N, int64_t T, int64_t D) {
-    return vec_trace_block_shape_ok(N, T, D) && aligned16(x) && (beta == nullptr || aligned16(beta));
-}
-
-// Few long rows: fewer than three or four blocks per SM from rows and components alone; the time axis
-// is then cut and the chunks chained inside one launch (measured, per-component decay: 0.47 -> 0.57
-// of the copy bandwidth at 64x16384x64 with 128 uncut blocks, 0.61 -> 0.57 at 256x4096x64 with 512;
-// shared decay: 0.43 -> 0.46 at 256x4096x64; chunks of 16-128 KB all within 0.05 of one another).
+// Few long rows: the time axis is cut and the chunks chained inside one launch.  Measured at D = 64
+// (fraction of the copy bandwidth, uncut -> chained): shared decay 0.46 -> 0.51 with 128 blocks,
+// 0.51 = 0.51 with 256, 0.55 -> 0.51 with 512; per-component decay 0.63 -> 0.57 with 128 blocks,
+// 0.74 -> 0.57 with 256.  So the shared decay cuts below two blocks per SM, the per-component decay
+// only where rows and components alone give too few blocks to run uncut at all (fewer than 96).
 bool vec_trace_block_cuts(int64_t N, int64_t T, int64_t D, bool perdim) {
     if (g_force_chained == 1) return false;
     const unsigned len = chained_chunk_len(tm_row_bytes(perdim ? kTmVecBeta : kTmVec, false));
     if ((int64_t)len >= T) return false;
-    return g_force_chained == 2 || (D + 31) / 32 * N < (perdim ? 3 : 4) * kSms;
+    return g_force_chained == 2 || (D + 31) / 32 * N < (perdim ? 96 : 2 * kSms);
+}
+
+// shapes the block kernel takes: rows of D floats copied in 16-byte pieces, and enough blocks -- from
+// rows and components alone, or from the chunks of a cut time axis
+bool vec_trace_block_shape_ok(int64_t N, int64_t T, int64_t D, bool perdim) {
+    if (g_force_path == 1) return false;
+    if (D % 4 != 0 || D < 32 || T < 64 || N > 65535) return false;
+    return (D + 31) / 32 * N >= 96 || vec_trace_block_cuts(N, T, D, perdim);
+}
+bool vec_trace_block_usable(const float* x, const float* beta, int64_t N, int64_t T, int64_t D) {
+    return vec_trace_block_shape_ok(N, T, D, beta != nullptr) && aligned16(x) && (beta == nullptr || aligned16(beta));
 }
 
 size_t vec_trace_block_workspace_bytes(int64_t N, int64_t T, int64_t D, bool perdim) {
-    return vec_trace_block_shape_ok(N, T, D) && vec_trace_block_cuts(N, T, D, perdim) ? chained_ws_bytes(D, T, N) : 0;
+    return vec_trace_block_shape_ok(N, T, D, perdim) && vec_trace_block_cuts(N, T, D, perdim) ? chained_ws_bytes(D, T, N) : 0;
 }
 
 int vec_trace_block(const float* x, const float* beta, const uint8_t* dones, float* traces, int64_t N, int64_t T, int64_t D,
@@ -1205,7 +1220,11 @@ int vec_trace_block(const float* x, const float* beta, const uint8_t* dones, flo
         if (p.warps_per_block == 8) return launch_block<ALGO, false, 8, 1>(p, smem, s);
         return launch_block<ALGO, false, 4, 1>(p, smem, s);
     };
-    return perdim ? go(std::integral_constant<int, kTmVecBeta>{}) : go(std::integral_constant<int, kTmVec>{});
+    if (!perdim) return go(std::integral_constant<int, kTmVec>{});
+    // deeper stages while every block is resident at once (up to ten 128-thread blocks per SM)
+    const long long blocks = (D + 31) / 32 * N * p.chunks;
+    return (p.chunks == 1 && blocks < 10 * kSms) ? go(std::integral_constant<int, kTmVecBeta16>{})
+                                                 : go(std::integral_constant<int, kTmVecBeta>{});
 }
 
 }  // namespace rlcs_internal
