@@ -331,7 +331,7 @@ def time_elig_trace_vec(torch, B, steps: int, peak: float, N: int, T: int, D: in
     ms = e0.elapsed_time(e1) / steps
     ab = N * T * ((12 if per_dim else 8) * D + 1)
     gbs = ab / (ms * 1e-3) / 1e9
-    return {"ms": round(ms, 5), "N": N, "T": T, "D": D, "time_axis_cut": bool(nbytes), "algorithmic_bytes": ab,
+    return {"ms": round(ms, 5), "N": N, "T": T, "D": D, "workspace_bytes": nbytes, "algorithmic_bytes": ab,
             "gbs": round(gbs, 1), "frac_of_peak": round(gbs / peak, 4)}
 
 
@@ -852,10 +852,10 @@ def main():
         torch.cuda.empty_cache()
         line["extensions"]["retrace_probs"] = time_retrace_probs(torch, binding, max(3, min(args.steps, 30)), peak)
         line["extensions"]["elig_trace_vec"] = [time_elig_trace_vec(torch, binding, max(3, min(args.steps, 30)), peak, *shape)
-                                                for shape in ((4096, 512, 64), (64, 16384, 64))]
+                                                for shape in ((4096, 512, 64), (1024, 1024, 64), (64, 16384, 64), (16, 65536, 64))]
         line["extensions"]["elig_trace_vec_beta"] = [
             time_elig_trace_vec(torch, binding, max(3, min(args.steps, 30)), peak, *shape, per_dim=True)
-            for shape in ((16384, 128, 64), (4096, 512, 64), (64, 16384, 64))]
+            for shape in ((16384, 128, 64), (4096, 512, 64), (64, 16384, 64), (16, 65536, 64))]
         line["extensions"]["time_major"] = [time_time_major(torch, binding, max(3, min(args.steps, 20)), peak, *shape)
                                             for shape in ((WORKLOAD["N"], WORKLOAD["T"]), (65536, 512), (2048, 2048))]
         torch.cuda.empty_cache()
