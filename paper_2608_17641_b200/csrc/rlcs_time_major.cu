@@ -115,6 +115,13 @@ __device__ __forceinline__ unsigned ones_if(unsigned x) {
     return m;
 }
 
+// all ones where bit `pos` of x is set, else 0 (bfe.s32 sign-extends the one-bit field)
+__device__ __forceinline__ unsigned bit_mask(unsigned x, int pos) {
+    int m;
+    asm("bfe.s32 %0, %1, %2, 1;" : "=r"(m) : "r"((int)x), "r"(pos));
+    return (unsigned)m;
+}
+
 // predicated load: *ptr where m != 0 (the address is not touched otherwise), else 0
 __device__ __forceinline__ float ldg_if_mask(const float* ptr, unsigned m) {
     float v = 0.f;
@@ -659,13 +666,14 @@ __device__ __forceinline__ void block_walk(const TmParams& p, const long long n0
         for (int c = 0; c < C; ++c) { carry[c] = 0.f; prod[c] = 1.f; }
         // the per-row guards exist only in the instance that the chunk's ragged last stage takes
         // one flag per timestep: the flags of the steps before this warp's rows (cut into step t <=> t == 0 or dones[t-1])
-        unsigned rowcut[KR];
+        // bit u: the carry into this warp's row u is cut.  Lane u reads the flag; one ballot shares them.
+        unsigned cutbits = 0;
         if constexpr (ROWMASK) {
-#pragma unroll
-            for (int u = 0; u < KR; ++u) {
-                const unsigned t = t_lo + j * R + row0 + u;
-                rowcut[u] = (t == 0 || t > p.T) ? 1u : __ldg(p.dones + t - 1);
-            }
+            static_assert(KR <= 32, "one lane per row of the warp");
+            const unsigned t = t_lo + j * R + row0 + lane;
+            unsigned f = 1u;
+            if (lane < KR && t != 0 && t <= p.T) f = __ldg(p.dones + t - 1);
+            cutbits = __ballot_sync(0xffffffffu, f != 0);
         }
         auto pass1 = [&](auto full) {
             constexpr bool FULL = decltype(full)::value;
@@ -695,7 +703,7 @@ __device__ __forceinline__ void block_walk(const TmParams& p, const long long n0
                         Coef co;
                         if constexpr (ROWMASK) {
                             co.alpha = r[c];
-                            co.beta = keep(~ones_if(rowcut[u]), tm_vec_beta(ALGO) ? x1[c] : p.decay);
+                            co.beta = keep(~bit_mask(cutbits, u), tm_vec_beta(ALGO) ? x1[c] : p.decay);
                             co.pg = 0.f;
                         } else if constexpr (FWD) {
                             co = fwd_coef<ALGO>(r[c], dn[c], d_prev[c], p, (u == 0 && w == 0 && j == 0) ? t_lo : 1u);
@@ -1168,15 +1176,17 @@ namespace rlcs_internal {
 
 // usable when every row of D floats can be copied in 16-byte pieces and there are enough blocks
 // Few long rows: the time axis is cut and the chunks chained inside one launch.  Measured at D = 64
-// (fraction of the copy bandwidth, uncut -> chained): shared decay 0.46 -> 0.51 with 128 blocks,
-// 0.51 = 0.51 with 256, 0.55 -> 0.51 with 512; per-component decay 0.63 -> 0.57 with 128 blocks,
-// 0.74 -> 0.57 with 256.  So the shared decay cuts below two blocks per SM, the per-component decay
-// only where rows and components alone give too few blocks to run uncut at all (fewer than 96).
+// (fraction of the copy bandwidth, uncut -> chained): shared decay 0.49 -> 0.59 with 128 blocks,
+// 0.56 -> 0.59 with 256, 0.58 -> 0.59 with 512, 0.81 -> 0.59 with 1024; per-component decay 0.67 ->
+// 0.59 with 128 blocks, 0.75 -> 0.59 with 256.  So the shared decay cuts below four blocks per SM, the
+// per-component decay only where rows and components alone give too few blocks to run uncut at all
+// (fewer than 96).  (More warps per block than plan_block gives lose with either decay; fewer lose
+// below two blocks per SM.)
 bool vec_trace_block_cuts(int64_t N, int64_t T, int64_t D, bool perdim) {
     if (g_force_chained == 1) return false;
     const unsigned len = chained_chunk_len(tm_row_bytes(perdim ? kTmVecBeta : kTmVec, false));
     if ((int64_t)len >= T) return false;
-    return g_force_chained == 2 || (D + 31) / 32 * N < (perdim ? 96 : 2 * kSms);
+    return g_force_chained == 2 || (D + 31) / 32 * N < (perdim ? 96 : 4 * kSms);
 }
 
 // shapes the block kernel takes: rows of D floats copied in 16-byte pieces, and enough blocks -- from
