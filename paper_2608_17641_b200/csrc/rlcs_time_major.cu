@@ -1200,8 +1200,15 @@ bool vec_trace_block_usable(const float* x, const float* beta, int64_t N, int64_
     return vec_trace_block_shape_ok(N, T, D, beta != nullptr) && aligned16(x) && (beta == nullptr || aligned16(beta));
 }
 
+// header plus one record per row, chunk and (padded) component; the vector kernels use one column per lane
+size_t vec_chained_ws_bytes(int64_t N, int64_t T, int64_t D, bool perdim) {
+    const long long len = chained_chunk_len(tm_row_bytes(perdim ? kTmVecBeta : kTmVec, false));
+    const long long npad = (D + 31) / 32 * 32, chunks = (T + len - 1) / len;
+    return 256 + sizeof(uint4) * (size_t)(npad * chunks * N);
+}
+
 size_t vec_trace_block_workspace_bytes(int64_t N, int64_t T, int64_t D, bool perdim) {
-    return vec_trace_block_shape_ok(N, T, D, perdim) && vec_trace_block_cuts(N, T, D, perdim) ? chained_ws_bytes(D, T, N) : 0;
+    return vec_trace_block_shape_ok(N, T, D, perdim) && vec_trace_block_cuts(N, T, D, perdim) ? vec_chained_ws_bytes(N, T, D, perdim) : 0;
 }
 
 int vec_trace_block(const float* x, const float* beta, const uint8_t* dones, float* traces, int64_t N, int64_t T, int64_t D,
@@ -1215,7 +1222,7 @@ int vec_trace_block(const float* x, const float* beta, const uint8_t* dones, flo
     p.mute_ticket = rlcs_hooks::g_mute_tile;
     const bool perdim = beta != nullptr;
     if (vec_trace_block_cuts(N, T, D, perdim)) {
-        if (workspace == nullptr || workspace_bytes < chained_ws_bytes(D, T, N)) return RLCS_ERR_WORKSPACE;
+        if (workspace == nullptr || workspace_bytes < vec_chained_ws_bytes(N, T, D, perdim)) return RLCS_ERR_WORKSPACE;
         if (!aligned16(workspace)) return RLCS_ERR_ALIGN;
         p.header = static_cast<unsigned*>(workspace);
         p.records = reinterpret_cast<uint4*>(static_cast<unsigned char*>(workspace) + 256);
