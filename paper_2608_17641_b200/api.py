@@ -148,6 +148,11 @@ def compute_eligibility_traces(x, dones, *, gamma=0.99, lam=0.95, beta=None, tim
     if x.dim() == 3:
         if time_major:
             raise ValueError("vector traces take [N, T, D] tensors")
+        N, T, D = x.shape
+        query = _B.lib().rlcs_elig_trace_vec_workspace_bytes if beta is None else _B.lib().rlcs_elig_trace_vec_beta_workspace_bytes
+        nbytes = int(query(N, T, D))
+        if workspace is None and nbytes:                       # few long rows: chunk records, cached like the others
+            workspace = _workspace(x, N, T, nbytes)
         if beta is not None:
             return _B.rlcs_elig_trace_vec_beta(x, beta, _mask(dones), workspace=workspace, stream=stream)
         return _B.rlcs_elig_trace_vec(x, _mask(dones), gamma=gamma, lam=lam, workspace=workspace, stream=stream)

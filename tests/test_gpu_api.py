@@ -64,6 +64,16 @@ def test_front_end_matches_binding_and_oracle(oracle, env):
     dv = torch.rand((6, 200), device="cuda") < 0.05
     assert_close("vector trace", api.compute_eligibility_traces(xv, dv, **g).cpu().numpy(),
                  oracle.elig_trace_vec(xv.cpu().numpy(), dv.cpu().numpy().astype(np.uint8), **g))
+    # few long rows: the time axis is cut, the chunk records live in a cached workspace
+    xl = torch.randn((4, 3000, 64), device="cuda")
+    bl = torch.rand((4, 3000, 64), device="cuda") * 0.5 + 0.5
+    dl = torch.rand((4, 3000), device="cuda") < 0.002
+    dl8 = dl.cpu().numpy().astype(np.uint8)
+    for _ in range(2):
+        assert_close("long vector trace", api.compute_eligibility_traces(xl, dl, **g).cpu().numpy(),
+                     oracle.elig_trace_vec(xl.cpu().numpy(), dl8, **g))
+        assert_close("long vector trace, per-component decay", api.compute_eligibility_traces(xl, dl, beta=bl).cpu().numpy(),
+                     oracle.elig_trace_vec_beta(xl.cpu().numpy(), bl.cpu().numpy(), dl8))
     # repeated calls reuse one workspace per shape
     before = len(api._workspaces)
     api.compute_gae(r, v, d, tr, bv, bt, **g)
