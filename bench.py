@@ -8,7 +8,9 @@ V-Trace, Retrace, TD(lambda), discounted returns, eligibility trace, episodic pr
 kernel launch each, on the 16384 x 2048 bandwidth-saturating configuration with per-step truncation
 handling.  `value` counts N*T env-steps per algorithm pass, i.e. 7*N*T per step and per GPU.
 
-Rank 0 prints ONE JSON line.  With N > 1 (torchrun) every rank works on its own batch of the same
+Rank 0 prints one JSON line per detail record (per-algorithm figures, extension entry points, the
+cold-L2 cases of the smaller configurations) and LAST the headline line, which is kept below 2 KB and
+holds every key of the bench contract (value, roofline, cpu_baseline, e2e, clocks).  With N > 1 (torchrun) every rank works on its own batch of the same
 shape (rows are independent: weak scaling, no collective on the data path); the time is the max
 over ranks.  `--impl reference` times the CPU oracle instead (rank 0 only).
 """
@@ -33,12 +35,11 @@ ALGOS = ("gae", "vtrace", "retrace", "td_lambda", "discounted_return", "elig_tra
 WORKLOAD = dict(N=16384, T=2048)
 FALLBACK_HBM_GBS = 6650.0
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch on the bench workload, from the committed
-# one-pass ncu capture of the full-size run (summarised under profiles/).
-NCU_TRAFFIC_BYTES = {
-    "gae": 575476736, "vtrace": 715139072, "retrace": 738443008, "td_lambda": 456630784,
-    "discounted_return": 310968064, "elig_trace": 255497472, "episodic_prefix_sum": 251432448,
-}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch on the bench workload come from a committed
+# one-pass ncu capture of the full-size run: `--traffic-from-ncu` turns ncu's CSV log into this file,
+# keyed by algorithm with the kernel instance beside each figure.
+TRAFFIC_JSON = os.path.join(ROOT, "profiles", "dram_traffic_16384x2048.json")
+HEADLINE_LIMIT = 2048        # the headline (last stdout line) stays below this many bytes
 
 
 # --------------------------------------------------------------------------------------------- helpers
@@ -67,6 +68,111 @@ def algorithmic_bytes(ro, algo: str) -> int:
             idx = np.flatnonzero((ro.truncs.ravel() != 0) & (ro.dones.ravel() == 0))
             b += 32 * int(np.unique(idx // 8).size)
     return int(b)
+
+
+def kernel_instance(binding, algo: str, has_truncs: bool, N: int, T: int) -> str:
+    """Name of the kernel instance a call takes, as ncu prints it: template arguments are
+    (algorithm id, truncation handling, vector accesses, threads, steps per thread, blocks per SM)."""
+    tr = bool(has_truncs) and algo not in ("elig_trace", "episodic_prefix_sum")
+    vi = binding.rlcs_debug_variant_for(algo, tr, N, T)
+    kname = "scan_kernel_tma" if vi["ring_stages"] else "scan_kernel"
+    return f"{kname}<{binding.ALGORITHM_IDS[algo]},{int(tr)},1,{vi['threads']},{vi['steps_per_thread']},{vi['blocks_per_sm']}>"
+
+
+def load_traffic(path: str = TRAFFIC_JSON) -> dict:
+    try:
+        with open(path) as fh:
+            return json.load(fh).get("kernels", {})
+    except Exception:
+        return {}
+
+
+def traffic_for(algo: str, instance: str, table: dict):
+    """Captured DRAM bytes per launch of `algo`, or None when the capture was taken on another kernel
+    instance than the one that runs now (a stale figure is worse than none)."""
+    rec = table.get(algo)
+    if not rec or rec.get("kernel") != instance:
+        return None
+    return int(rec["dram_bytes_per_launch"])
+
+
+def traffic_from_ncu(csv_path: str, out_path: str = TRAFFIC_JSON, command: str = "") -> dict:
+    """Turn the CSV log of `ncu --metrics dram__bytes_read.sum,dram__bytes_write.sum --csv` over the
+    bench command into the committed traffic table: per algorithm the kernel instance and the mean of
+    read + write bytes over its captured launches."""
+    import csv
+    ids = {0: "gae", 1: "td_lambda", 2: "discounted_return", 3: "vtrace", 4: "retrace", 5: "elig_trace",
+           6: "episodic_prefix_sum"}
+    unit = {"byte": 1.0, "Kbyte": 1e3, "Mbyte": 1e6, "Gbyte": 1e9}
+    with open(csv_path, newline="") as fh:
+        lines = [ln for ln in fh if ln.startswith('"')]
+    per_launch = {}                                   # launch id -> [kernel, bytes]
+    for row in csv.DictReader(lines):
+        name = row["Kernel Name"]
+        if "dram__bytes" not in row["Metric Name"]:
+            continue
+        val = float(row["Metric Value"].replace(",", "")) * unit.get(row["Metric Unit"], 1.0)
+        rec = per_launch.setdefault(row["ID"], [name, 0.0])
+        rec[1] += val
+    by_kernel = {}
+    for name, b in per_launch.values():
+        by_kernel.setdefault(name, []).append(b)
+    kernels = {}
+    for name, vals in by_kernel.items():
+        short = name.split("(")[0].split("::")[-1].replace(" ", "")
+        if not short.startswith("scan_kernel<") and not short.startswith("scan_kernel_tma<"):
+            continue
+        algo = ids.get(int(short.split("<")[1].split(",")[0]))
+        if algo is None:
+            continue
+        if "(bool)" in short or "true" in short or "false" in short:      # ncu may print bools as words
+            short = short.replace("(bool)1", "1").replace("(bool)0", "0").replace("true", "1").replace("false", "0")
+        short = short.replace("(rlcs::Algo)", "").replace("(int)", "")
+        kernels[algo] = {"kernel": short, "launches": len(vals), "dram_bytes_per_launch": int(round(sum(vals) / len(vals)))}
+    doc = {"workload": f"num_envs={WORKLOAD['N']}, T={WORKLOAD['T']}, truncation handling on", "command": command,
+           "metrics": "dram__bytes_read.sum + dram__bytes_write.sum, mean over the captured launches", "kernels": kernels}
+    with open(out_path, "w") as fh:
+        json.dump(doc, fh, indent=1)
+        fh.write("\n")
+    return doc
+
+
+def build_headline(*, value, world, steps, warmup, ms_per_step, workload, clocks, e2e, launches, roofline,
+                   cpu_baseline=None, per_algorithm_frac=None, small_frac=None, detail_file=None) -> dict:
+    """The last stdout line: every key the bench contract names and nothing bulky.  Per-algorithm,
+    extension and sweep figures are printed before it, one JSON line each."""
+    line = {
+        "metric": METRIC, "value": value, "unit": METRIC, "n_gpus": world, "steps": steps, "warmup": warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic", "config": {"workload": workload, "l2": "inputs larger than L2, no flush"},
+        "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline,
+    }
+    if cpu_baseline is not None:
+        line["cpu_baseline"] = cpu_baseline
+    if per_algorithm_frac:
+        line["frac_of_peak"] = per_algorithm_frac
+    if small_frac:
+        line["small_configs_frac_of_peak"] = small_frac
+    if detail_file:
+        line["detail_file"] = detail_file
+    return line
+
+
+def emit(details: list, headline: dict, detail_file=None):
+    """Detail lines first, the headline last and alone on the final line."""
+    text = json.dumps(headline)
+    for drop in ("small_configs_frac_of_peak", "frac_of_peak"):        # never let the headline outgrow the limit
+        if len(text) < HEADLINE_LIMIT:
+            break
+        headline.pop(drop, None)
+        text = json.dumps(headline)
+    assert len(text) < HEADLINE_LIMIT, f"headline line is {len(text)} bytes"
+    if detail_file:
+        with open(detail_file, "w") as fh:
+            json.dump({"headline": headline, "details": details}, fh, indent=1)
+    for d in details:
+        print(json.dumps(d), flush=True)
+    print(text, flush=True)
 
 
 class ClockSampler:
@@ -680,6 +786,17 @@ def _without_truncs(ro):
     return r2
 
 
+def small_config_summary(sweeps) -> dict:
+    """frac_of_peak of the cold-L2 cases the bandwidth target names: N=4096 with T >= 256, and the
+    long-row configuration (64 x 16384).  Keys: <algo>_<T>[t]; t = with truncation handling."""
+    short = {"gae": "gae", "vtrace": "vtr", "discounted_return": "disc"}
+    out = {}
+    for c in sweeps:
+        if (c["N"] == 4096 and c["T"] >= 256) or c["T"] == 16384:
+            out[f"{short.get(c['algo'], c['algo'])}_{c['T']}{'t' if c['truncs'] else ''}"] = round(c["frac_of_peak"], 3)
+    return out
+
+
 def run_sweeps(torch, hbm_peak, pick=None, trials=5):
     """The cold-L2 cases of configurations 1-4.  `pick` = (config, algo, T, truncs), None entries
     matching anything, keeps only the matching cases (for a profiler run on one kernel)."""
@@ -736,9 +853,17 @@ def main():
                     help="time only that extension line on a --rows x --seq-len batch and print it (one JSON line)")
     ap.add_argument("--seq-len", type=int, default=WORKLOAD["T"], help="T of the --only batch")
     ap.add_argument("--tm-path", type=int, default=0, help="time-major path test hook for --only runs (0 = library default)")
+    ap.add_argument("--detail-file", default=None, help="also write headline + detail lines to this JSON file")
+    ap.add_argument("--traffic-from-ncu", default=None, metavar="CSV",
+                    help="no benchmark: turn ncu's CSV log of the DRAM byte counters into profiles/dram_traffic_16384x2048.json")
+    ap.add_argument("--traffic-command", default="", help="with --traffic-from-ncu: the ncu command line, recorded in the file")
     ap.add_argument("--dim", type=int, default=64, help="D of the --only elig_trace_vec* batch, A of retrace_probs")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    if args.traffic_from_ncu is not None:
+        print(json.dumps(traffic_from_ncu(args.traffic_from_ncu, command=args.traffic_command)))
+        return
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -813,57 +938,62 @@ def main():
                 + 2 * ro.N * ro.T + 4 * ro.N
             per_algo[a]["gbs_dense_trunc_bootstrap_count"] = round(dense / (ms * 1e-3) / 1e9, 1)
     dom = max(ALGOS, key=lambda a: per_algo[a]["ms"])
-    vi = binding.rlcs_debug_variant_for(dom, ro.truncs is not None and dom not in ("elig_trace", "episodic_prefix_sum"), ro.N, ro.T)
-    kname = "scan_kernel_tma" if vi["ring_stages"] else "scan_kernel"
-    roofline = {"bound": "hbm", "kernel": f"{kname}<{dom}>, {vi['threads']} threads x {vi['steps_per_thread']} steps per tile "
-                                          f"(variant {vi['variant']})",
+    full_size = (ro.N, ro.T) == (WORKLOAD["N"], WORKLOAD["T"]) and ro.truncs is not None
+    traffic_table = load_traffic() if full_size else {}
+    for a in ALGOS:
+        per_algo[a]["kernel"] = kernel_instance(binding, a, ro.truncs is not None, ro.N, ro.T)
+        per_algo[a]["ncu_dram_bytes"] = traffic_for(a, per_algo[a]["kernel"], traffic_table)
+    roofline = {"bound": "hbm", "kernel": f"{per_algo[dom]['kernel']} ({dom})",
                 "achieved": per_algo[dom]["gbs"], "peak": peak, "unit": "GB/s",
-                "frac": round(per_algo[dom]["gbs"] / peak, 4), "traffic": NCU_TRAFFIC_BYTES.get(dom) if (ro.N, ro.T) == (WORKLOAD["N"], WORKLOAD["T"]) and ro.truncs is not None else None,
+                "frac": round(per_algo[dom]["gbs"] / peak, 4), "traffic": per_algo[dom]["ncu_dram_bytes"],
                 "algorithmic_bytes_per_launch": per_algo[dom]["algorithmic_bytes"], "peak_source": f"of {peak_kind}",
                 "all_kernels_frac": round(sum(v["algorithmic_bytes"] for v in per_algo.values())
                                           / (sum(v["ms"] for v in per_algo.values()) * 1e-3) / 1e9 / peak, 4)}
+    details = [{"detail": "per_algorithm", "N": ro.N, "T": ro.T, "truncs": ro.truncs is not None, "per_algorithm": per_algo}]
 
-    extensions = {"gae_normalized": time_gae_normalized(batch, max(3, min(args.steps, 50)), peak)}
+    ext = lambda name, res: details.append({"detail": "extension", "name": name, "result": res})
+    ext("gae_normalized", time_gae_normalized(batch, max(3, min(args.steps, 50)), peak))
     if rank == 0 and world == 1 and not args.no_sweep:
-        extensions["gae_skip"] = time_gae_skip(batch, max(3, min(args.steps, 30)), peak)
+        ext("gae_skip", time_gae_skip(batch, max(3, min(args.steps, 30)), peak))
     e2e_steps = max(1, min(args.steps, 8))
     e2e_ms, h2d, d2h = time_e2e(batch, e2e_steps, 1, dist)
     e2e_ms = dist.max(e2e_ms)
     e2e = {"value": units_per_step * e2e_steps / (e2e_ms * 1e-3), "unit": METRIC, "h2d_bytes_per_step": h2d,
-           "d2h_bytes_per_step": d2h, "steps": e2e_steps, "ms_per_step": e2e_ms / e2e_steps,
-           "note": "pinned host buffers -> device, seven C-ABI calls, all outputs -> pinned host; upload, kernel and "
-                   "read-back streams chained by events"}
+           "d2h_bytes_per_step": d2h, "steps": e2e_steps, "ms_per_step": round(e2e_ms / e2e_steps, 4),
+           "note": "pinned host -> device, seven C-ABI calls, all outputs -> pinned host; three streams"}
 
-    line = {
-        "metric": METRIC, "value": value, "unit": METRIC, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-        "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "f32", "data": "synthetic",
-        "config": {"workload": f"all seven algorithms, num_envs={ro.N}, T={ro.T}, fp32, dones~Bern(0.02), "
-                               f"truncs~Bern(0.005) with per-step truncation handling, gamma=0.99, lambda=0.95",
-                   "env_steps_per_step_per_gpu": len(ALGOS) * ro.N * ro.T, "launches_per_step": len(ALGOS),
-                   "l2": "inputs larger than L2 (2.2 GB touched per step), no flush"},
-        "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "per_algorithm": per_algo,
-        "extensions": extensions,
-    }
+    cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        line["cpu_baseline"] = cpu_baseline(ro)
+        cpu = cpu_baseline(ro)
+        details.append({"detail": "cpu_baseline", **cpu})
+        cpu = {k: cpu[k] for k in ("value", "unit", "cores", "kind", "sample")}
+    small = None
     if rank == 0 and world == 1 and not args.no_sweep:
         del batch
         torch.cuda.empty_cache()
-        line["extensions"]["retrace_probs"] = time_retrace_probs(torch, binding, max(3, min(args.steps, 30)), peak)
-        line["extensions"]["elig_trace_vec"] = [time_elig_trace_vec(torch, binding, max(3, min(args.steps, 30)), peak, *shape)
-                                                for shape in ((4096, 512, 64), (1024, 1024, 64), (64, 16384, 64), (16, 65536, 64))]
-        line["extensions"]["elig_trace_vec_beta"] = [
-            time_elig_trace_vec(torch, binding, max(3, min(args.steps, 30)), peak, *shape, per_dim=True)
-            for shape in ((16384, 128, 64), (4096, 512, 64), (64, 16384, 64), (16, 65536, 64))]
-        line["extensions"]["time_major"] = [time_time_major(torch, binding, max(3, min(args.steps, 20)), peak, *shape)
-                                            for shape in ((WORKLOAD["N"], WORKLOAD["T"]), (65536, 512), (2048, 2048))]
+        k30, k20 = max(3, min(args.steps, 30)), max(3, min(args.steps, 20))
+        ext("retrace_probs", time_retrace_probs(torch, binding, k30, peak))
+        ext("elig_trace_vec", [time_elig_trace_vec(torch, binding, k30, peak, *shape)
+                               for shape in ((4096, 512, 64), (1024, 1024, 64), (64, 16384, 64), (16, 65536, 64))])
+        ext("elig_trace_vec_beta", [time_elig_trace_vec(torch, binding, k30, peak, *shape, per_dim=True)
+                                    for shape in ((16384, 128, 64), (4096, 512, 64), (64, 16384, 64), (16, 65536, 64))])
+        for shape in ((WORKLOAD["N"], WORKLOAD["T"]), (65536, 512), (2048, 2048)):
+            ext("time_major", time_time_major(torch, binding, k20, peak, *shape))
         torch.cuda.empty_cache()
-        line["extensions"]["bf16"] = time_bf16(torch, binding, max(3, min(args.steps, 20)), peak, WORKLOAD["N"], WORKLOAD["T"])
+        ext("bf16", time_bf16(torch, binding, k20, peak, WORKLOAD["N"], WORKLOAD["T"]))
         torch.cuda.empty_cache()
-        line["sweeps"] = run_sweeps(torch, peak)
+        sweeps = run_sweeps(torch, peak)
+        details += [{"detail": "sweep", **c} for c in sweeps]
+        small = small_config_summary(sweeps)
     if rank == 0:
-        print(json.dumps(line), flush=True)
+        workload = (f"config 5: all seven algorithms, num_envs={ro.N}, T={ro.T}, fp32, dones~Bern(0.02), truncs~Bern(0.005) "
+                    f"with per-step truncation handling, gamma=0.99, lambda=0.95; {len(ALGOS)} launches per step")
+        headline = build_headline(value=value, world=world, steps=args.steps, warmup=args.warmup,
+                                  ms_per_step=round(total_ms / args.steps, 5), workload=workload, clocks=clocks, e2e=e2e,
+                                  launches=launches, roofline=roofline, cpu_baseline=cpu,
+                                  per_algorithm_frac={a: per_algo[a]["frac_of_peak"] for a in ALGOS}, small_frac=small,
+                                  detail_file=args.detail_file)
+        emit(details, headline, args.detail_file)
     if world > 1:
         dist.close()
 
