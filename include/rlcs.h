@@ -70,7 +70,8 @@ typedef enum {
     RLCS_ERR_WORKSPACE = 5,  /* workspace NULL or too small for this (N, T) */
     RLCS_ERR_CUDA = 6,       /* the launch itself failed (cudaGetLastError) */
     RLCS_ERR_TIMEOUT = 7,    /* device status: a bounded carry wait gave up */
-    RLCS_ERR_LIMIT = 8       /* rlcs_gae_no_alloc: the problem needs more scratch than the built-in array holds */
+    RLCS_ERR_LIMIT = 8,      /* rlcs_gae_no_alloc: the problem needs more scratch than the built-in array holds */
+    RLCS_ERR_CAPTURE = 9     /* rlcs_gae_no_alloc: a device's first call was made while its stream was capturing */
 } rlcs_status_t;
 
 /* Human-readable name of a status code (static storage, never NULL). */
@@ -246,20 +247,37 @@ int rlcs_episodic_prefix_sum(const float* x, const uint8_t* dones, float* sums, 
  * that loads the library holds until the process exits.  The call itself allocates nothing: no
  * cudaMalloc, no cudaFree, no allocating library routine.
  *
- * Limit: rlcs_workspace_bytes(N, T) must not exceed that array, i.e. N*T <= 33.5 million steps
- * (unlimited when T divides 512, where no scratch is used); larger problems return RLCS_ERR_LIMIT
- * and launch nothing.
+ * Limit: the carry scratch this call would use, rlcs_gae_carry_bytes(N, T, truncs != NULL, all
+ * pointers aligned for vector access), must not exceed that array.  That always holds for
+ * N*T <= 33 545 728 steps (65 520 tile records of at least 512 steps), and for any size when no
+ * row straddles a tile (T divides the tile, e.g. 16384 x 2048) or the tiles of a row form one
+ * thread-block cluster.  Larger problems return RLCS_ERR_LIMIT and launch nothing.
  * First call on a device: looks up the array's device address (cudaGetSymbolAddress) and
  * initialises it with two small memsets on `cuda_stream`; make this first call outside any stream
- * capture, with the device current that later calls will use.
+ * capture (it returns RLCS_ERR_CAPTURE otherwise, since the memsets would be recorded instead of
+ * run), with the device current that later calls will use.  Concurrent first calls from several
+ * host threads are serialised by a lock; later calls take it only to read the cached address.
  * Sharing: every call on a device uses the same array, which keeps what the last call left; the
- * entry point re-zeroes the words that must start at zero.  Calls that can overlap on the GPU
+ * entry point re-zeroes the word that must start at zero.  Calls that can overlap on the GPU
  * (different streams without ordering, several host threads) race on it and give wrong results:
  * keep them ordered, or use rlcs_gae with separate workspaces.
+ * Device status: a bounded carry wait that gave up leaves RLCS_ERR_TIMEOUT in the array's status
+ * word, where it stays until rlcs_no_alloc_last_device_status reads and clears it.
  */
 int rlcs_gae_no_alloc(const float* rewards, const float* values, const uint8_t* dones, const uint8_t* truncs,
                       const float* trunc_bootstrap, const float* bootstrap, float* advantages, float* returns,
                       int64_t N, int64_t T, float gamma, float lambda, void* cuda_stream);
+
+/* Device status of the rlcs_gae_no_alloc calls on the current device, like rlcs_last_device_status
+ * for a workspace: synchronises `cuda_stream`, returns RLCS_OK or RLCS_ERR_TIMEOUT and clears the
+ * word.  RLCS_OK when rlcs_gae_no_alloc has not run on this device yet.  (No counterpart in the paper.) */
+int rlcs_no_alloc_last_device_status(void* cuda_stream);
+
+/* Bytes of carry workspace one rlcs_gae call with these sizes would read or write: 0 when no row
+ * straddles a tile or a row's tiles form one thread-block cluster (needs `vector_access`: every fp32
+ * pointer 32-byte and every mask pointer 16-byte aligned); never more than rlcs_workspace_bytes(N, T),
+ * which stays the size to allocate for a workspace shared by all entry points. */
+size_t rlcs_gae_carry_bytes(int64_t N, int64_t T, int has_truncs, int vector_access);
 
 /* Size in bytes of the built-in scratch array used by rlcs_gae_no_alloc. */
 size_t rlcs_no_alloc_scratch_bytes(void);

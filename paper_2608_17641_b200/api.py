@@ -1,7 +1,9 @@
 """Call-by-name front end over the C-ABI binding, with the argument names of the paper's
 ``compute_*`` functions (Section 6.1): picks the entry point from dtype and layout, keeps one carry
-workspace per (device, shape) so that repeated calls allocate nothing, and accepts ``torch.bool``
-masks.  Argument marshalling only -- every step runs in the CUDA kernels, there is no CPU path.
+workspace per (device, stream, shape) so that repeated calls allocate nothing, and accepts
+``torch.bool`` masks.  Workspace sharing rule: calls that use the same cached workspace are those
+issued on the same stream, which orders them; calls on different streams get different workspaces.
+A caller that passes ``workspace=`` itself must keep the calls sharing it ordered on the GPU.  Argument marshalling only -- every step runs in the CUDA kernels, there is no CPU path.
 
     adv, ret = compute_gae(rewards, values, dones, truncateds, bootstrap_values, bootstrap,
                            gamma=0.99, lam=0.95)
@@ -31,13 +33,15 @@ def _mask(m):
     return m.view(torch.uint8) if m.dtype == torch.bool else m
 
 
-def _workspace(like, N: int, T: int, nbytes: int | None = None):
-    """One initialised workspace per (device, N, T, size), reused by every later call on that shape.
-    Calls that may overlap on the GPU (different streams without ordering) must pass their own."""
-    key = (like.device, N, T, nbytes)
+def _workspace(like, N: int, T: int, nbytes: int | None = None, stream=None):
+    """One initialised workspace per (device, stream, N, T, size), reused by every later call on that
+    shape and stream.  The stream is part of the key because two calls share carry records and a
+    call counter in the workspace: only calls ordered on one stream may share one."""
+    s = _torch().cuda.current_stream(like.device) if stream is None else stream
+    key = (like.device, int(s.cuda_stream), N, T, nbytes)
     ws = _workspaces.get(key)
     if ws is None:
-        ws = _B.Workspace(N, T, device=like.device, nbytes=nbytes)
+        ws = _B.Workspace(N, T, device=like.device, stream=s, nbytes=nbytes)
         _workspaces[key] = ws
     return ws
 
@@ -59,13 +63,13 @@ def _shape(t, time_major: bool):
     return (t.shape[1], t.shape[0]) if time_major else (t.shape[0], t.shape[1])
 
 
-def _ws_for(kind: str, like, N: int, T: int, workspace):
+def _ws_for(kind: str, like, N: int, T: int, workspace, stream=None):
     if workspace is not None:
         return workspace
     if kind == "tm":
         nbytes = int(_B.lib().rlcs_time_major_workspace_bytes(N, T))
-        return _workspace(like, N, T, max(nbytes, 256)) if nbytes else None
-    return _workspace(like, N, T)
+        return _workspace(like, N, T, max(nbytes, 256), stream=stream) if nbytes else None
+    return _workspace(like, N, T, stream=stream)
 
 
 def compute_gae(rewards, values, dones, truncateds=None, bootstrap_values=None, bootstrap=None, *, gamma=0.99,
@@ -80,10 +84,11 @@ def compute_gae(rewards, values, dones, truncateds=None, bootstrap_values=None, 
         if kind != "f32" or (normalize and skip_mask is not None):
             raise ValueError("normalize / skip_mask take row-major float32 tensors, one of the two at a time")
     if normalize:
-        ws = workspace or _workspace(rewards, N, T, int(_B.lib().rlcs_gae_normalized_workspace_bytes(N, T)))
+        ws = workspace if workspace is not None else _workspace(
+            rewards, N, T, int(_B.lib().rlcs_gae_normalized_workspace_bytes(N, T)), stream=stream)
         return _B.rlcs_gae_normalized(rewards, values, dones, truncateds, bootstrap_values, bootstrap, gamma=gamma, lam=lam,
                                       eps=eps, workspace=ws, stream=stream)
-    ws = _ws_for(kind, rewards, N, T, workspace)
+    ws = _ws_for(kind, rewards, N, T, workspace, stream)
     if skip_mask is not None:
         return _B.rlcs_gae_skip(rewards, values, dones, truncateds, bootstrap_values, bootstrap, skip=skip_mask, gamma=gamma,
                                 lam=lam, workspace=ws, stream=stream)
@@ -98,7 +103,7 @@ def compute_vtrace(rewards, values, log_rhos, dones, truncateds=None, bootstrap_
     N, T = _shape(rewards, time_major)
     fn = {"f32": _B.rlcs_vtrace, "bf16": _B.rlcs_vtrace_bf16, "tm": _B.rlcs_vtrace_time_major}[kind]
     return fn(rewards, values, log_rhos, _mask(dones), _mask(truncateds), bootstrap_values, bootstrap, gamma=gamma,
-              rho_bar=rho_bar, c_bar=c_bar, workspace=_ws_for(kind, rewards, N, T, workspace), stream=stream)
+              rho_bar=rho_bar, c_bar=c_bar, workspace=_ws_for(kind, rewards, N, T, workspace, stream), stream=stream)
 
 
 def compute_retrace(rewards, q_sa, expected_q, log_rhos, dones, truncateds=None, bootstrap_values=None, bootstrap=None, *,
@@ -108,7 +113,7 @@ def compute_retrace(rewards, q_sa, expected_q, log_rhos, dones, truncateds=None,
     N, T = _shape(rewards, time_major)
     fn = {"f32": _B.rlcs_retrace, "bf16": _B.rlcs_retrace_bf16, "tm": _B.rlcs_retrace_time_major}[kind]
     return fn(rewards, q_sa, expected_q, log_rhos, _mask(dones), _mask(truncateds), bootstrap_values, bootstrap, gamma=gamma,
-              lam=lam, c_bar=c_bar, workspace=_ws_for(kind, rewards, N, T, workspace), stream=stream)
+              lam=lam, c_bar=c_bar, workspace=_ws_for(kind, rewards, N, T, workspace, stream), stream=stream)
 
 
 def compute_retrace_from_probs(rewards, q_values, target_probs, behaviour_probs, actions, dones, truncateds=None,
@@ -118,7 +123,8 @@ def compute_retrace_from_probs(rewards, q_values, target_probs, behaviour_probs,
     N, T = rewards.shape
     return _B.rlcs_retrace_probs(rewards, q_values, target_probs, behaviour_probs, actions, _mask(dones), _mask(truncateds),
                                  bootstrap_values, bootstrap, gamma=gamma, lam=lam, c_bar=c_bar,
-                                 workspace=workspace or _workspace(rewards, N, T), stream=stream)
+                                 workspace=workspace if workspace is not None else _workspace(rewards, N, T, stream=stream),
+                                 stream=stream)
 
 
 def compute_td_lambda_returns(rewards, values, dones, truncateds=None, bootstrap_values=None, bootstrap=None, *, gamma=0.99,
@@ -128,7 +134,7 @@ def compute_td_lambda_returns(rewards, values, dones, truncateds=None, bootstrap
     N, T = _shape(rewards, time_major)
     fn = {"f32": _B.rlcs_td_lambda, "bf16": _B.rlcs_td_lambda_bf16, "tm": _B.rlcs_td_lambda_time_major}[kind]
     return fn(rewards, values, _mask(dones), _mask(truncateds), bootstrap_values, bootstrap, gamma=gamma, lam=lam,
-              workspace=_ws_for(kind, rewards, N, T, workspace), stream=stream)
+              workspace=_ws_for(kind, rewards, N, T, workspace, stream), stream=stream)
 
 
 def compute_discounted_returns(rewards, dones, truncateds=None, bootstrap_values=None, bootstrap=None, *, gamma=0.99,
@@ -139,7 +145,7 @@ def compute_discounted_returns(rewards, dones, truncateds=None, bootstrap_values
     fn = {"f32": _B.rlcs_discounted_return, "bf16": _B.rlcs_discounted_return_bf16,
           "tm": _B.rlcs_discounted_return_time_major}[kind]
     return fn(rewards, _mask(dones), _mask(truncateds), bootstrap_values, bootstrap, gamma=gamma,
-              workspace=_ws_for(kind, rewards, N, T, workspace), stream=stream)
+              workspace=_ws_for(kind, rewards, N, T, workspace, stream), stream=stream)
 
 
 def compute_eligibility_traces(x, dones, *, gamma=0.99, lam=0.95, beta=None, time_major=False, workspace=None, stream=None):
@@ -152,7 +158,7 @@ def compute_eligibility_traces(x, dones, *, gamma=0.99, lam=0.95, beta=None, tim
         query = _B.lib().rlcs_elig_trace_vec_workspace_bytes if beta is None else _B.lib().rlcs_elig_trace_vec_beta_workspace_bytes
         nbytes = int(query(N, T, D))
         if workspace is None and nbytes:                       # few long rows: chunk records, cached like the others
-            workspace = _workspace(x, N, T, nbytes)
+            workspace = _workspace(x, N, T, nbytes, stream=stream)
         if beta is not None:
             return _B.rlcs_elig_trace_vec_beta(x, beta, _mask(dones), workspace=workspace, stream=stream)
         return _B.rlcs_elig_trace_vec(x, _mask(dones), gamma=gamma, lam=lam, workspace=workspace, stream=stream)
@@ -161,7 +167,7 @@ def compute_eligibility_traces(x, dones, *, gamma=0.99, lam=0.95, beta=None, tim
     kind = _kind(x, time_major)
     N, T = _shape(x, time_major)
     fn = {"f32": _B.rlcs_elig_trace, "bf16": _B.rlcs_elig_trace_bf16, "tm": _B.rlcs_elig_trace_time_major}[kind]
-    return fn(x, _mask(dones), gamma=gamma, lam=lam, workspace=_ws_for(kind, x, N, T, workspace), stream=stream)
+    return fn(x, _mask(dones), gamma=gamma, lam=lam, workspace=_ws_for(kind, x, N, T, workspace, stream), stream=stream)
 
 
 def compute_episodic_prefix_sum(x, dones, *, boundary="ends_at", time_major=False, workspace=None, stream=None):
@@ -172,4 +178,4 @@ def compute_episodic_prefix_sum(x, dones, *, boundary="ends_at", time_major=Fals
     N, T = _shape(x, time_major)
     fn = {"f32": _B.rlcs_episodic_prefix_sum, "bf16": _B.rlcs_episodic_prefix_sum_bf16,
           "tm": _B.rlcs_episodic_prefix_sum_time_major}[kind]
-    return fn(x, _mask(dones), starts_at=(boundary == "starts_at"), workspace=_ws_for(kind, x, N, T, workspace), stream=stream)
+    return fn(x, _mask(dones), starts_at=(boundary == "starts_at"), workspace=_ws_for(kind, x, N, T, workspace, stream), stream=stream)

@@ -15,7 +15,7 @@ LIB_PATH = os.path.join(_PKG, "librlcs.so")
 
 RLCS_OK = 0
 RLCS_ERR_NULL, RLCS_ERR_SIZE, RLCS_ERR_ARG, RLCS_ERR_ALIGN = 1, 2, 3, 4
-RLCS_ERR_WORKSPACE, RLCS_ERR_CUDA, RLCS_ERR_TIMEOUT, RLCS_ERR_LIMIT = 5, 6, 7, 8
+RLCS_ERR_WORKSPACE, RLCS_ERR_CUDA, RLCS_ERR_TIMEOUT, RLCS_ERR_LIMIT, RLCS_ERR_CAPTURE = 5, 6, 7, 8, 9
 
 _vp, _i64, _f, _sz, _int = ctypes.c_void_p, ctypes.c_int64, ctypes.c_float, ctypes.c_size_t, ctypes.c_int
 _TAIL = [_vp, _sz, _vp]          # workspace, workspace_bytes, cuda_stream
@@ -43,6 +43,8 @@ SIGNATURES = {
     "rlcs_gae_skip": ([_vp] * 10 + [_i64, _i64, _f, _f] + _TAIL, _int),
     "rlcs_gae_no_alloc": ([_vp] * 8 + [_i64, _i64, _f, _f, _vp], _int),
     "rlcs_no_alloc_scratch_bytes": ([], _sz),
+    "rlcs_no_alloc_last_device_status": ([_vp], _int),
+    "rlcs_gae_carry_bytes": ([_i64, _i64, _int, _int], _sz),
     "rlcs_time_major_workspace_bytes": ([_i64, _i64], _sz),
     "rlcs_gae_time_major": ([_vp] * 8 + [_i64, _i64, _f, _f] + _TAIL, _int),
     "rlcs_vtrace_time_major": ([_vp] * 9 + [_i64, _i64, _f, _f, _f] + _TAIL, _int),
@@ -109,6 +111,19 @@ def _torch():
     return torch
 
 
+def _current_device() -> int:
+    return _torch().cuda.current_device()
+
+
+def _require_current_device(t, what: str = "tensor"):
+    """The library launches on the current device and the current stream of that device: a tensor
+    (or workspace) that lives on another GPU would hand the kernel a pointer it must not touch."""
+    index, cur = t.device.index, _current_device()
+    if index is not None and index != cur:
+        raise ValueError(f"{what} is on cuda:{index} but the current device is cuda:{cur}; "
+                         f"call under torch.cuda.device({index})")
+
+
 def _ptr(t, dtype_kind: str, shape=None):
     """Device pointer of a tensor (None -> NULL) after dtype / device / layout checks."""
     if t is None:
@@ -116,6 +131,7 @@ def _ptr(t, dtype_kind: str, shape=None):
     torch = _torch()
     if not t.is_cuda:
         raise TypeError("rlcs takes CUDA tensors (device pointers); there is no CPU path")
+    _require_current_device(t)
     if dtype_kind == "f32":
         if t.dtype != torch.float32:
             raise TypeError(f"expected float32, got {t.dtype}")     # the method is fp32-only
@@ -131,6 +147,12 @@ def _ptr(t, dtype_kind: str, shape=None):
     return t.data_ptr()
 
 
+def _alloc(shape, dtype, device):
+    """Device memory for outputs and workspaces the binding creates itself (torch's allocator).  A
+    module-level function so that a test harness can substitute an allocator that adds guard bands."""
+    return _torch().empty(shape, dtype=dtype, device=device)
+
+
 def _stream(stream=None):
     torch = _torch()
     s = torch.cuda.current_stream() if stream is None else stream
@@ -143,7 +165,7 @@ class Workspace:
     def __init__(self, N: int, T: int, device="cuda", stream=None, nbytes: int | None = None):
         torch = _torch()
         self.nbytes = int(lib().rlcs_workspace_bytes(N, T)) if nbytes is None else int(nbytes)
-        self.buf = torch.empty(max(self.nbytes, 16), dtype=torch.uint8, device=device) if self.nbytes else None
+        self.buf = _alloc((max(self.nbytes, 16),), torch.uint8, device) if self.nbytes else None
         if self.buf is not None:
             if stream is not None:
                 self.buf.record_stream(stream)     # the caching allocator must not hand it out again before that stream is done
@@ -162,12 +184,16 @@ def workspace_bytes(N: int, T: int) -> int:
 
 
 def _ws(ws: Workspace | None):
-    return (None, 0) if ws is None else (ws.ptr, ws.nbytes)
+    if ws is None:
+        return (None, 0)
+    if ws.buf is not None:
+        _require_current_device(ws.buf, "workspace")
+    return (ws.ptr, ws.nbytes)
 
 
 def _out(like, out):
     torch = _torch()
-    return torch.empty_like(like, dtype=torch.float32) if out is None else out
+    return _alloc(tuple(like.shape), torch.float32, like.device) if out is None else out
 
 
 def rlcs_gae(rewards, values, dones, truncs=None, trunc_bootstrap=None, bootstrap=None, *, gamma, lam,
@@ -232,6 +258,12 @@ def rlcs_gae_no_alloc(rewards, values, dones, truncs=None, trunc_bootstrap=None,
                                    _ptr(bootstrap, "f32", (N,)), _ptr(adv, "f32", (N, T)), _ptr(ret, "f32", (N, T)),
                                    N, T, gamma, lam, _stream(stream)))
     return (adv, ret) if want_returns else adv
+
+
+def rlcs_no_alloc_last_device_status(stream=None) -> int:
+    """Device status of the rlcs_gae_no_alloc calls on the current device (synchronises the stream,
+    clears the word): RLCS_OK or RLCS_ERR_TIMEOUT."""
+    return int(lib().rlcs_no_alloc_last_device_status(_stream(stream)))
 
 
 def rlcs_vtrace(rewards, values, log_rhos, dones, truncs=None, trunc_bootstrap=None, bootstrap=None, *,
@@ -408,7 +440,7 @@ def rlcs_debug_time_major_path(path: int = 0):
 # ------------------------------------------------------------------------------------------ bfloat16 tensors
 def _out16(like, out):
     torch = _torch()
-    return torch.empty_like(like, dtype=torch.bfloat16) if out is None else out
+    return _alloc(tuple(like.shape), torch.bfloat16, like.device) if out is None else out
 
 
 def rlcs_gae_bf16(rewards, values, dones, truncs=None, trunc_bootstrap=None, bootstrap=None, *, gamma, lam,

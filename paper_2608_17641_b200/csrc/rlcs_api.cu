@@ -23,6 +23,7 @@ const char* rlcs_status_string(int status) {
         case RLCS_ERR_CUDA: return "RLCS_ERR_CUDA: CUDA call failed";
         case RLCS_ERR_TIMEOUT: return "RLCS_ERR_TIMEOUT: bounded carry wait gave up";
         case RLCS_ERR_LIMIT: return "RLCS_ERR_LIMIT: problem too large for the built-in scratch array of rlcs_gae_no_alloc";
+        case RLCS_ERR_CAPTURE: return "RLCS_ERR_CAPTURE: first rlcs_gae_no_alloc call on a device made during stream capture";
         default: return "RLCS: unknown status";
     }
 }
@@ -77,6 +78,13 @@ int rlcs_gae(const float* rewards, const float* values, const uint8_t* dones, co
     st = finish_params(p, variant, total, T, workspace, workspace_bytes, vec);
     if (st != RLCS_OK) return st;
     return run(rlcs::launch_gae, p, variant, truncs != nullptr, vec, cuda_stream);
+}
+
+size_t rlcs_gae_carry_bytes(int64_t N, int64_t T, int has_truncs, int vector_access) {
+    int64_t total = 0;
+    if (check_sizes(N, T, &total) != RLCS_OK || total == 0) return 0;
+    const int variant = choose_variant(rlcs::kGae, has_truncs != 0, total, T);
+    return plan_carry(variant, total, T, vector_access != 0, true, 1).bytes;
 }
 
 int rlcs_gae_skip(const float* rewards, const float* values, const uint8_t* dones, const uint8_t* truncs,

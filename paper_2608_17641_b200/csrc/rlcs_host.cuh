@@ -108,6 +108,29 @@ int choose_variant(int algo, bool trunc, int64_t total, int64_t T) {
     }
 }
 
+// How the carry between thread blocks travels for one call, and the workspace bytes it needs.
+struct CarryPlan {
+    int carry_mode;      // rows straddle tiles: tile records in the workspace, look-back
+    int cluster;         // > 1: one thread-block cluster of this many tiles per row, no workspace
+    size_t bytes;        // workspace bytes this call reads or writes (0 when it needs none)
+};
+
+CarryPlan plan_carry(int variant, int64_t total, int64_t T, bool vec, bool allow_cluster, int records_per_tile) {
+    const int tile = tile_elems(variant);
+    const int64_t num_tiles = (total + tile - 1) / tile;
+    CarryPlan plan = {(tile % T) != 0 ? 1 : 0, 0, 0};       // T does not divide the tile: rows straddle tiles
+    // Rows of exactly 2..8 tiles: one thread-block cluster per row carries through distributed
+    // shared memory instead (needs the vectorised one-tile kernel; g_cluster = 0 turns it off).
+    if (allow_cluster && g_cluster && vec && RLCS_NS::kVariants[variant].stages == 0 && T % tile == 0 && T / tile >= 2 &&
+        T / tile <= 8) {
+        plan.cluster = (int)(T / tile);
+        plan.carry_mode = 0;
+    }
+    if (plan.carry_mode)
+        plan.bytes = sizeof(unsigned) * RLCS_NS::kHeaderWords + sizeof(uint4) * (size_t)num_tiles * records_per_tile;
+    return plan;
+}
+
 // Fill the size / tiling / carry fields and validate the workspace for this call.
 int finish_params(ScanParams& p, int variant, int64_t total, int64_t T, void* workspace, size_t workspace_bytes, bool vec,
                   bool allow_cluster = true, int records_per_tile = 1) {
@@ -125,14 +148,9 @@ int finish_params(ScanParams& p, int variant, int64_t total, int64_t T, void* wo
     }
     p.decay_pow = 1.f;                       // beta product of a chunk without resets
     for (int i = 0; i < RLCS_NS::kVariants[variant].items; ++i) p.decay_pow *= p.decay;
-    p.carry_mode = (tile % T) != 0;          // T does not divide the tile: rows straddle tiles
-    // Rows of exactly 2..8 tiles: one thread-block cluster per row carries through distributed
-    // shared memory instead (needs the vectorised one-tile kernel; g_cluster = 0 turns it off).
-    p.cluster = 0;
-    if (allow_cluster && g_cluster && vec && RLCS_NS::kVariants[variant].stages == 0 && T % tile == 0 && T / tile >= 2 && T / tile <= 8) {
-        p.cluster = (int)(T / tile);
-        p.carry_mode = 0;
-    }
+    const CarryPlan plan = plan_carry(variant, total, T, vec, allow_cluster, records_per_tile);
+    p.carry_mode = plan.carry_mode;
+    p.cluster = plan.cluster;
     p.header = nullptr;
     p.records = nullptr;
     p.status = nullptr;
@@ -141,8 +159,7 @@ int finish_params(ScanParams& p, int variant, int64_t total, int64_t T, void* wo
     p.mute_tile = g_mute_tile;
     p.spin_cap = g_spin_cap > 0 ? (unsigned)g_spin_cap : kDefaultSpinCap;
     if (p.carry_mode) {
-        const size_t need = sizeof(unsigned) * RLCS_NS::kHeaderWords + sizeof(uint4) * (size_t)p.num_tiles * records_per_tile;
-        if (workspace == nullptr || workspace_bytes < need) return RLCS_ERR_WORKSPACE;
+        if (workspace == nullptr || workspace_bytes < plan.bytes) return RLCS_ERR_WORKSPACE;
         if (!aligned(workspace, 16)) return RLCS_ERR_ALIGN;
         p.header = static_cast<unsigned*>(workspace);
         p.records = reinterpret_cast<uint4*>(p.header + RLCS_NS::kHeaderWords);

@@ -25,36 +25,75 @@ def assert_close(name, gpu, ref):
     return float(err.max())
 
 
+# ---------------------------------------------------------------------------------------------- guard bands
+# Every device tensor the tests hand to the library sits between two bands of 0xFF bytes (a NaN
+# pattern for fp32 and bfloat16, 255 for masks, -1 for int32).  A kernel that writes outside a
+# tensor -- before it, behind it, or into an input -- lands in a band; the bands of all live
+# allocations are compared after every run_gpu() and at the end of every GPU test (conftest.py).
+GUARD = 64                       # elements on each side
+_live = []                       # (flat uint8 view, first payload byte, one-past-last payload byte, label)
+
+
+def guarded_empty(shape, dtype, offset: int = 0, label: str = ""):
+    """Uninitialised device tensor of `shape` inside guard bands; `offset` shifts it by that many
+    elements from the (512-byte aligned) allocation start + GUARD elements, to break alignment."""
+    import torch
+    n = 1
+    for d in (shape if isinstance(shape, (tuple, list, torch.Size)) else (shape,)):
+        n *= int(d)
+    flat = torch.empty(GUARD + offset + n + GUARD, dtype=dtype, device="cuda")
+    raw = flat.view(torch.uint8)
+    raw.fill_(0xFF)
+    es = flat.element_size()
+    _live.append((raw, (GUARD + offset) * es, (GUARD + offset + n) * es, label or str(tuple(shape) if hasattr(shape, "__len__") else shape)))
+    return flat[GUARD + offset:GUARD + offset + n].view(shape)
+
+
+def guarded_upload(a, offset: int = 0, dtype=None, label: str = ""):
+    """Device copy of a numpy array (or CPU tensor) inside guard bands; None stays None."""
+    import torch
+    if a is None:
+        return None
+    t = a if isinstance(a, torch.Tensor) else torch.from_numpy(np.ascontiguousarray(a))
+    if dtype is not None:
+        t = t.to(dtype)
+    out = guarded_empty(tuple(t.shape), t.dtype, offset, label)
+    out.copy_(t)
+    return out
+
+
+def check_guards(clear: bool = False):
+    """Assert that no guard band of a live allocation has been written."""
+    import torch
+    if _live and torch.cuda.is_available():
+        torch.cuda.synchronize()
+        for raw, lo, hi, label in _live:
+            ok = bool(raw[:lo].eq(0xFF).all().item()) and bool(raw[hi:].eq(0xFF).all().item())
+            if not ok:
+                front = int((raw[:lo] != 0xFF).sum().item())
+                back = int((raw[hi:] != 0xFF).sum().item())
+                if clear:
+                    _live.clear()
+                raise AssertionError(f"guard band overwritten around tensor {label}: {front} bytes before it, {back} bytes behind it")
+    if clear:
+        _live.clear()
+
+
 class Dev:
-    """Device copies of a Rollout's arrays (torch tensors); `offset` shifts every tensor by that
-    many elements from its allocation start to break 16-byte alignment."""
+    """Device copies of a Rollout's arrays (torch tensors), each inside guard bands; `offset` shifts
+    every tensor by that many elements from its aligned position to break 16-byte alignment."""
 
     def __init__(self, ro, offset: int = 0):
-        import torch
         self.ro = ro
         self.offset = offset
-
-        def up(a):
-            if a is None:
-                return None
-            t = torch.from_numpy(np.ascontiguousarray(a))
-            if offset == 0:
-                return t.cuda()
-            flat = torch.empty(t.numel() + offset, dtype=t.dtype, device="cuda")
-            view = flat[offset:].view(t.shape)
-            view.copy_(t)
-            return view
-
         for k in ("rewards", "values", "dones", "bootstrap", "truncs", "trunc_bootstrap", "q_sa", "expected_q",
                   "log_rhos", "x"):
-            setattr(self, k, up(getattr(ro, k)))
-        self.any_done = up(ro.any_done)
+            setattr(self, k, guarded_upload(getattr(ro, k), offset, label=k))
+        self.any_done = guarded_upload(ro.any_done, offset, label="any_done")
 
     def empty_out(self):
         import torch
-        n = self.ro.N * self.ro.T
-        flat = torch.empty(n + self.offset, dtype=torch.float32, device="cuda")
-        return flat[self.offset:].view(self.ro.N, self.ro.T)
+        return guarded_empty((self.ro.N, self.ro.T), torch.float32, self.offset, label="output")
 
 
 def run_gpu(dev: Dev, algos=ALL_ALGOS, workspace="auto", use_truncs=True, use_bootstrap=True):
@@ -96,6 +135,7 @@ def run_gpu(dev: Dev, algos=ALL_ALGOS, workspace="auto", use_truncs=True, use_bo
             raise KeyError(a)
     import torch
     torch.cuda.synchronize()
+    check_guards()
     if ws is not None:
         assert ws.device_status() == 0, "device reported a carry-wait timeout"
     to_np = lambda v: tuple(t.cpu().numpy() for t in v) if isinstance(v, tuple) else v.cpu().numpy()

@@ -17,3 +17,21 @@ def oracle():
     import oracle as _oracle
     _oracle.build()
     return _oracle
+
+
+@pytest.fixture(autouse=True)
+def _guard_bands(request):
+    """After every GPU test: no kernel wrote outside the tensors it was given (see tests/_util.py)."""
+    if request.node.get_closest_marker("gpu") is None:
+        yield
+        return
+    from _util import check_guards, guarded_empty
+    from paper_2608_17641_b200 import binding
+    plain = binding._alloc
+    # outputs and workspaces that the binding allocates itself get bands too
+    binding._alloc = lambda shape, dtype, device: guarded_empty(shape, dtype, label="allocated by the binding")
+    try:
+        yield
+        check_guards(clear=True)
+    finally:
+        binding._alloc = plain

@@ -41,6 +41,21 @@ def test_library_exports_every_declared_symbol(L):
         assert name in _declared_symbols(), f"binding knows {name} but rlcs.h does not declare it"
 
 
+def test_no_alloc_limit_is_decided_on_the_scratch_a_call_uses(L):
+    cap = L.rlcs_no_alloc_scratch_bytes()
+    assert cap == 1 << 20
+    assert L.rlcs_gae_carry_bytes(0, 5, 0, 1) == 0 and L.rlcs_gae_carry_bytes(-1, 5, 0, 1) == 0
+    for N, T in ((96, 1000), (8, 128), (4096, 1000), (33545, 1000)):
+        for tr in (0, 1):
+            for vec in (0, 1):
+                assert L.rlcs_gae_carry_bytes(N, T, tr, vec) <= L.rlcs_workspace_bytes(N, T)
+    assert L.rlcs_gae_carry_bytes(16384, 2048, 1, 1) == 0 and L.rlcs_gae_carry_bytes(64, 16384, 0, 1) == 0
+    assert L.rlcs_gae_carry_bytes(33545, 1000, 1, 1) <= cap < L.rlcs_gae_carry_bytes(140000, 1000, 0, 1)
+    # beyond the array: refused on the host, before anything touches a device
+    assert L.rlcs_gae_no_alloc(P, P, P, None, None, None, P, None, 140000, 1000, 0.99, 0.95, None) == 8
+    assert b"scratch" in L.rlcs_status_string(8) and b"capture" in L.rlcs_status_string(9)
+
+
 def test_status_strings(L):
     assert L.rlcs_status_string(0) == b"RLCS_OK"
     for s in range(1, 8):
@@ -141,6 +156,67 @@ def test_binding_rejects_cpu_tensors_and_wrong_dtypes():
     d = torch.zeros(2, 8, dtype=torch.uint8)
     with pytest.raises(TypeError):                       # no CPU path: CUDA tensors only
         binding.rlcs_elig_trace(x, d, gamma=0.9, lam=0.9, traces=x.clone())
+
+
+class _FakeDevice:
+    def __init__(self, index):
+        self.index = index
+
+
+class _FakeTensor:
+    """Stands in for a CUDA tensor on a chosen device (no GPU is needed to check the host-side rule)."""
+
+    def __init__(self, index, dtype=None, shape=(2, 8)):
+        import torch
+        self.is_cuda, self.device, self.dtype, self.shape = True, _FakeDevice(index), dtype or torch.float32, shape
+
+    def is_contiguous(self):
+        return True
+
+    def data_ptr(self):
+        return 0x7f0000000000 + 4096 * (self.device.index or 0)
+
+
+def test_binding_rejects_tensors_and_workspaces_of_another_device(monkeypatch):
+    """The library launches on the current device: a tensor or workspace of another GPU is refused
+    on the host instead of reaching a kernel as a foreign pointer."""
+    from paper_2608_17641_b200 import binding
+    monkeypatch.setattr(binding, "_current_device", lambda: 0)
+    assert binding._ptr(_FakeTensor(0), "f32", (2, 8)) == 0x7f0000000000
+    with pytest.raises(ValueError, match="cuda:1 but the current device is cuda:0"):
+        binding._ptr(_FakeTensor(1), "f32", (2, 8))
+    ws = binding.Workspace.__new__(binding.Workspace)
+    ws.nbytes, ws.buf = 1024, _FakeTensor(1)
+    with pytest.raises(ValueError, match="workspace is on cuda:1"):
+        binding._ws(ws)
+    ws.buf = _FakeTensor(0)
+    assert binding._ws(ws) == (ws.buf.data_ptr(), 1024)
+    monkeypatch.setattr(binding, "_current_device", lambda: 1)
+    with pytest.raises(ValueError):
+        binding._ptr(_FakeTensor(0), "f32")
+
+
+def test_front_end_keeps_one_workspace_per_stream(monkeypatch):
+    """Calls on different streams must not share carry records: the cache key holds the stream."""
+    from paper_2608_17641_b200 import api
+
+    class FakeStream:
+        def __init__(self, handle):
+            self.cuda_stream = handle
+
+    made = []
+
+    class FakeWorkspace:
+        def __init__(self, N, T, device=None, stream=None, nbytes=None):
+            made.append((N, T, stream.cuda_stream, nbytes))
+
+    monkeypatch.setattr(api._B, "Workspace", FakeWorkspace)
+    monkeypatch.setattr(api, "_workspaces", {})
+    like = _FakeTensor(0)
+    a = api._workspace(like, 4, 1000, stream=FakeStream(11))
+    b = api._workspace(like, 4, 1000, stream=FakeStream(11))
+    c = api._workspace(like, 4, 1000, stream=FakeStream(22))
+    assert a is b and a is not c and [m[2] for m in made] == [11, 22]
 
 
 def test_missing_library_fails_loudly(tmp_path, monkeypatch):

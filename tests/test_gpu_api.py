@@ -3,7 +3,7 @@ for, bit for bit, and the oracle's result to the parity tolerance."""
 import numpy as np
 import pytest
 
-from _util import assert_close, run_oracle
+from _util import assert_close, guarded_upload, run_oracle
 
 pytestmark = pytest.mark.gpu
 
@@ -22,7 +22,7 @@ def test_front_end_matches_binding_and_oracle(oracle, env):
     api, B, W, torch = env
     ro = W.make_rollout(140, 24, 1500, p_done=0.02, p_trunc=0.01)
     p = ro.params
-    up = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()
+    up = lambda a: guarded_upload(np.ascontiguousarray(a))
     r, v, q, eq, lr, x, bv, bt = (up(getattr(ro, k)) for k in ("rewards", "values", "q_sa", "expected_q", "log_rhos", "x",
                                                                 "trunc_bootstrap", "bootstrap"))
     d, tr, dany = up(ro.dones).bool(), up(ro.truncs).bool(), up(ro.any_done).bool()      # bool masks are accepted

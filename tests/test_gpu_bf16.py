@@ -13,7 +13,7 @@ rounded to bfloat16 by torch, bit for bit.
 import numpy as np
 import pytest
 
-from _util import ALL_ALGOS, ATOL, RTOL, run_oracle
+from _util import ALL_ALGOS, ATOL, RTOL, guarded_empty, guarded_upload, run_oracle
 
 pytestmark = pytest.mark.gpu
 
@@ -60,13 +60,7 @@ class Dev16:
         def up(a, bf16):
             if a is None:
                 return None
-            t = torch.from_numpy(np.ascontiguousarray(a))
-            if bf16:
-                t = t.to(torch.bfloat16)
-            flat = torch.empty(t.numel() + offset, dtype=t.dtype, device="cuda")
-            view = flat[offset:].view(t.shape)
-            view.copy_(t)
-            return view
+            return guarded_upload(a, offset, dtype=torch.bfloat16 if bf16 else None)
 
         for k in FLOAT_KEYS:
             setattr(self, k, up(getattr(ro, k), True))
@@ -74,8 +68,7 @@ class Dev16:
 
     def out(self):
         import torch
-        flat = torch.empty(self.ro.N * self.ro.T + self.offset, dtype=torch.bfloat16, device="cuda")
-        return flat[self.offset:].view(self.ro.N, self.ro.T)
+        return guarded_empty((self.ro.N, self.ro.T), torch.bfloat16, self.offset, label="bf16 output")
 
 
 def run_gpu16(B, dev, algos=ALL_ALGOS, use_truncs=True, use_bootstrap=True):
@@ -186,7 +179,7 @@ def test_bf16_full_size_sampled_rows(oracle, W, B):
     ref = run_oracle(oracle, small, ("gae", "vtrace", "discounted_return"))
     dev = Dev16(ro)
     ws = B.Workspace(ro.N, ro.T)
-    idx = torch.from_numpy(rows).cuda()
+    idx = guarded_upload(rows)
     adv, ret = B.rlcs_gae_bf16(dev.rewards, dev.values, dev.dones, dev.truncs, dev.trunc_bootstrap, dev.bootstrap,
                                gamma=p["gamma"], lam=p["lam"], workspace=ws)
     assert_close16("gae", adv[idx], ref["gae"][0]); assert_close16("ret", ret[idx], ref["gae"][1])

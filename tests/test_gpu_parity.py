@@ -5,7 +5,8 @@ import os
 import numpy as np
 import pytest
 
-from _util import ALL_ALGOS, Dev, assert_close, compare_all, run_gpu, run_oracle
+from _util import (ALL_ALGOS, Dev, assert_close, check_guards, compare_all, guarded_empty, guarded_upload, run_gpu,
+                   run_oracle)
 
 pytestmark = pytest.mark.gpu
 
@@ -89,8 +90,8 @@ def test_config5_full_size_extension_entry_points(oracle, W, B):
     ref = run_oracle(oracle, small, ALL_ALGOS)
     # time-major, all seven
     r, v, d, tr, bv = _tm(ro.rewards), _tm(ro.values), _tm(ro.dones), _tm(ro.truncs), _tm(ro.trunc_bootstrap)
-    bt = torch.from_numpy(ro.bootstrap).cuda()
-    take = lambda t: np.ascontiguousarray(t[:, torch.from_numpy(rows).cuda()].cpu().numpy().T)
+    bt = guarded_upload(ro.bootstrap)
+    take = lambda t: np.ascontiguousarray(t[:, guarded_upload(rows)].cpu().numpy().T)
     adv, ret = B.rlcs_gae_time_major(r, v, d, tr, bv, bt, gamma=p["gamma"], lam=p["lam"])
     assert_close("tm gae", take(adv), ref["gae"][0]); assert_close("tm ret", take(ret), ref["gae"][1])
     del adv, ret
@@ -116,10 +117,10 @@ def test_config5_full_size_extension_entry_points(oracle, W, B):
     skip = (np.random.default_rng(6).random((N, T)) < 0.3).astype(np.uint8)
     ws = B.Workspace(N, T)
     a, rt, fil = B.rlcs_gae_skip(dev.rewards, dev.values, dev.dones, dev.truncs, dev.trunc_bootstrap, dev.bootstrap,
-                                 skip=torch.from_numpy(skip).cuda(), gamma=p["gamma"], lam=p["lam"], workspace=ws)
+                                 skip=guarded_upload(skip), gamma=p["gamma"], lam=p["lam"], workspace=ws)
     ra, rr, rf = oracle.gae_skip(small.rewards, small.values, small.dones, small.truncs, small.trunc_bootstrap, small.bootstrap,
                                  skip=np.ascontiguousarray(skip[rows]), gamma=p["gamma"], lam=p["lam"])
-    pick = lambda t: t[torch.from_numpy(rows).cuda()].cpu().numpy()
+    pick = lambda t: t[guarded_upload(rows)].cpu().numpy()
     assert ws.device_status() == 0
     assert_close("skip adv", pick(a), ra); assert_close("skip ret", pick(rt), rr)
     assert np.array_equal(pick(fil).astype(np.float64), rf)
@@ -444,18 +445,11 @@ def _probs_gpu(B, ro, q, pi, mu, act, use_truncs=True, use_bootstrap=True, offse
     import torch
     dev = Dev(ro, offset=offset)
 
-    def up3(a):
-        t = torch.from_numpy(a)
-        if offset == 0:
-            return t.cuda()
-        flat = torch.empty(t.numel() + offset, dtype=t.dtype, device="cuda")
-        view = flat[offset:].view(t.shape)
-        view.copy_(t)
-        return view
+    up3 = lambda a: guarded_upload(a, offset)
 
     ws = B.Workspace(ro.N, ro.T)
     p = ro.params
-    out = B.rlcs_retrace_probs(dev.rewards, up3(q), up3(pi), up3(mu), torch.from_numpy(act).cuda(), dev.dones,
+    out = B.rlcs_retrace_probs(dev.rewards, up3(q), up3(pi), up3(mu), guarded_upload(act), dev.dones,
                                dev.truncs if use_truncs else None, dev.trunc_bootstrap if use_truncs else None,
                                dev.bootstrap if use_bootstrap else None, gamma=p["gamma"], lam=p["lam"], c_bar=p["c_bar"],
                                q_targets=dev.empty_out(), workspace=ws)
@@ -515,16 +509,14 @@ def test_vector_eligibility_trace(oracle, W, B, N, T, D):
     x = rng.standard_normal((N, T, D)).astype(np.float32)
     d = (rng.random((N, T)) < 0.02).astype(np.uint8)
     d[:, 0] = rng.integers(0, 2, N)                      # a flag on the very first step
-    xd, dd = torch.from_numpy(x).cuda(), torch.from_numpy(d).cuda()
+    xd, dd = guarded_upload(x), guarded_upload(d)
     ref = oracle.elig_trace_vec(x, d, gamma=0.99, lam=0.95)
     got = B.rlcs_elig_trace_vec(xd, dd, gamma=0.99, lam=0.95).cpu().numpy()
     assert_close(f"vector trace {N}x{T}x{D}", got, ref)
     again = B.rlcs_elig_trace_vec(xd, dd, gamma=0.99, lam=0.95).cpu().numpy()
     assert np.array_equal(got, again)
     # pointer off 16-byte alignment: element-wise variant
-    flat = torch.empty(x.size + 1, dtype=torch.float32, device="cuda")
-    xo = flat[1:].view(N, T, D)
-    xo.copy_(xd)
+    xo = guarded_upload(x, 1)
     got1 = B.rlcs_elig_trace_vec(xo, dd, gamma=0.99, lam=0.95).cpu().numpy()
     assert_close("vector trace, unaligned", got1, ref)
     # against the scalar entry point, component by component
@@ -556,7 +548,7 @@ def test_per_dimension_beta_eligibility_trace(oracle, W, B, N, T, D):
     beta = rng.uniform(0.5, 1.0, (N, T, D)).astype(np.float32)
     d = (rng.random((N, T)) < 0.02).astype(np.uint8)
     d[:, 0] = rng.integers(0, 2, N)
-    xd, bd, dd = torch.from_numpy(x).cuda(), torch.from_numpy(beta).cuda(), torch.from_numpy(d).cuda()
+    xd, bd, dd = guarded_upload(x), guarded_upload(beta), guarded_upload(d)
     ref = oracle.elig_trace_vec_beta(x, beta, d)
     got = B.rlcs_elig_trace_vec_beta(xd, bd, dd).cpu().numpy()
     assert_close(f"per-dimension trace {N}x{T}x{D}", got, ref)
@@ -586,7 +578,7 @@ def test_vector_trace_plans_agree(oracle, W, B, N, T, D, plan):
     x = rng.standard_normal((N, T, D)).astype(np.float32)
     beta = rng.uniform(0.5, 1.0, (N, T, D)).astype(np.float32)
     d = (rng.random((N, T)) < 0.02).astype(np.uint8)
-    xd, bd, dd = torch.from_numpy(x).cuda(), torch.from_numpy(beta).cuda(), torch.from_numpy(d).cuda()
+    xd, bd, dd = guarded_upload(x), guarded_upload(beta), guarded_upload(d)
     if isinstance(plan, str):            # the block kernel, its time axis always / never cut into chained chunks
         B.rlcs_debug_vec_trace_plan(1, 0)
         B.rlcs_debug_time_major_path(5 if plan == "chained" else 4)
@@ -633,7 +625,7 @@ def test_gae_with_observation_skip_masking(oracle, W, B, N, T, p_skip, p_flag):
     ro, skip = _skip_case(W, N, T, p_skip, p_flag)
     p = ro.params
     dev = Dev(ro)
-    sk = torch.from_numpy(skip).cuda()
+    sk = guarded_upload(skip)
     ws = B.Workspace(N, T)
     adv, ret, fil = B.rlcs_gae_skip(dev.rewards, dev.values, dev.dones, dev.truncs, dev.trunc_bootstrap, dev.bootstrap,
                                     skip=sk, gamma=p["gamma"], lam=p["lam"], workspace=ws)
@@ -663,9 +655,7 @@ def test_gae_skip_options_alignment_and_large_problem(oracle, W, B):
     p = ro.params
     for offset in (0, 1):
         dev = Dev(ro, offset=offset)
-        flat = torch.zeros(skip.size + offset, dtype=torch.uint8, device="cuda")
-        sk = flat[offset:].view(skip.shape)
-        sk.copy_(torch.from_numpy(skip))
+        sk = guarded_upload(skip, offset)
         adv, fil = B.rlcs_gae_skip(dev.rewards, dev.values, dev.dones, skip=sk, gamma=p["gamma"], lam=p["lam"],
                                    values_filled=dev.empty_out(), advantages=dev.empty_out(), want_returns=False,
                                    workspace=B.Workspace(ro.N, ro.T))
@@ -678,7 +668,7 @@ def test_gae_skip_options_alignment_and_large_problem(oracle, W, B):
     dev = Dev(ro)
     ws = B.Workspace(ro.N, ro.T)
     adv, ret, fil = B.rlcs_gae_skip(dev.rewards, dev.values, dev.dones, dev.truncs, dev.trunc_bootstrap, dev.bootstrap,
-                                    skip=torch.from_numpy(skip).cuda(), gamma=p["gamma"], lam=p["lam"], workspace=ws)
+                                    skip=guarded_upload(skip), gamma=p["gamma"], lam=p["lam"], workspace=ws)
     ra, rr, rf = oracle.run_rows_parallel(
         lambda **k: oracle.gae_skip(k["rewards"], k["values"], k["dones"], k["truncs"], k["trunc_bootstrap"], k["bootstrap"],
                                     skip=k["skip"], gamma=p["gamma"], lam=p["lam"]),
@@ -700,7 +690,7 @@ def test_gae_skip_options_alignment_and_large_problem(oracle, W, B):
 # ------------------------------------------------------------------ time-major [T, N] entry points
 def _tm(a):
     import torch
-    return None if a is None else torch.from_numpy(np.ascontiguousarray(np.asarray(a).T)).cuda()
+    return None if a is None else guarded_upload(np.ascontiguousarray(np.asarray(a).T))
 
 
 @pytest.fixture
@@ -734,7 +724,7 @@ def test_time_major_entry_points(oracle, W, B, N, T, p_flag, tm_path):
     r, v, d, tr, bv = _tm(ro.rewards), _tm(ro.values), _tm(ro.dones), _tm(ro.truncs), _tm(ro.trunc_bootstrap)
     q, eq, lr, x, dany = _tm(ro.q_sa), _tm(ro.expected_q), _tm(ro.log_rhos), _tm(ro.x), _tm(ro.any_done)
     import torch
-    bt = torch.from_numpy(ro.bootstrap).cuda()
+    bt = guarded_upload(ro.bootstrap)
     back = lambda t: t.cpu().numpy().T
     adv, ret = B.rlcs_gae_time_major(r, v, d, tr, bv, bt, gamma=p["gamma"], lam=p["lam"])
     assert_close("gae adv", np.ascontiguousarray(back(adv)), ref["gae"][0])
@@ -776,7 +766,7 @@ def test_time_major_paths_agree_and_misaligned_inputs_fall_back(oracle, W, B):
     p = ro.params
     names = ("rewards", "values", "dones", "truncs", "trunc_bootstrap")
     al = [_tm(getattr(ro, k)) for k in names]
-    bt = torch.from_numpy(ro.bootstrap).cuda()
+    bt = guarded_upload(ro.bootstrap)
     outs = []
     for path in (1, 2):
         B.rlcs_debug_time_major_path(path)
@@ -789,9 +779,7 @@ def test_time_major_paths_agree_and_misaligned_inputs_fall_back(oracle, W, B):
     # the same tensors one element into a larger allocation: 4-byte (1-byte for masks) aligned only
     mis = []
     for a in al:
-        buf = torch.empty(a.numel() + 1, dtype=a.dtype, device=a.device)
-        buf[1:].copy_(a.reshape(-1))
-        mis.append(buf[1:].view(T, N))
+        mis.append(guarded_upload(a.cpu(), 1))
     out = B.rlcs_gae_time_major(*mis, bt, gamma=p["gamma"], lam=p["lam"])
     assert torch.equal(out[0], outs[0][0]) and torch.equal(out[1], outs[0][1])
 
@@ -805,7 +793,7 @@ def test_time_major_chained_kernel_is_reproducible_and_agrees_with_three_launche
     ro = W.make_rollout(118, N, T, p_done=p_flag, p_trunc=p_flag / 2)
     p = ro.params
     al = [_tm(getattr(ro, k)) for k in ("rewards", "values", "dones", "truncs", "trunc_bootstrap")]
-    bt = torch.from_numpy(ro.bootstrap).cuda()
+    bt = guarded_upload(ro.bootstrap)
     x, dany = _tm(ro.x), _tm(ro.any_done)
     outs = {}
     for path in (5, 5, 4):
@@ -883,7 +871,7 @@ def test_randomized_time_major_and_skip(oracle, W, B):
         tm = lambda a: None if a is None else _tm(a)
         r, v, d, q, eq, lr, x, dany = (tm(getattr(ro, k)) for k in ("rewards", "values", "dones", "q_sa", "expected_q", "log_rhos", "x", "any_done"))
         tr, bv = (tm(ro.truncs), tm(ro.trunc_bootstrap)) if use_tr else (None, None)
-        bt = torch.from_numpy(ro.bootstrap).cuda() if use_bt else None
+        bt = guarded_upload(ro.bootstrap) if use_bt else None
         back = lambda t: np.ascontiguousarray(t.cpu().numpy().T)
         path = int(rng.choice([0, 1, 3]))
         B.rlcs_debug_time_major_path(path)
@@ -906,9 +894,7 @@ def test_randomized_time_major_and_skip(oracle, W, B):
         # observation-skip masking on the same rollout (row-major)
         skip = (rng.random((N, T)) < float(rng.choice([0.0, 0.3, 0.8]))).astype(np.uint8)
         dev = Dev(ro, offset=int(rng.choice([0, 0, 1])))
-        flat = torch.zeros(skip.size + dev.offset, dtype=torch.uint8, device="cuda")
-        sk = flat[dev.offset:].view(skip.shape)
-        sk.copy_(torch.from_numpy(skip))
+        sk = guarded_upload(skip, dev.offset)
         a, rt, fil = B.rlcs_gae_skip(dev.rewards, dev.values, dev.dones, dev.truncs if use_tr else None,
                                      dev.trunc_bootstrap if use_tr else None, dev.bootstrap if use_bt else None, skip=sk,
                                      gamma=p["gamma"], lam=p["lam"], values_filled=dev.empty_out(), advantages=dev.empty_out(),
@@ -937,7 +923,7 @@ def test_calls_can_be_captured_in_a_cuda_graph(oracle, W, B):
     ws = B.Workspace(ro.N, ro.T)
     wsn = B.Workspace(ro.N, ro.T, nbytes=int(B.lib().rlcs_gae_normalized_workspace_bytes(ro.N, ro.T)))
     wtm = B.Workspace(ro.N, ro.T, nbytes=max(256, int(B.lib().rlcs_time_major_workspace_bytes(ro.N, ro.T))))
-    new = lambda like=dev.rewards, dt=None: torch.empty_like(like, dtype=dt or like.dtype)
+    new = lambda like=dev.rewards, dt=None: guarded_empty(tuple(like.shape), dt or like.dtype)
     outs = {k: new() for k in ("adv", "ret", "vs", "pg", "q", "nadv", "nret", "sadv", "sret", "fil", "el")}
     outs.update(tadv=new(r_tm), tret=new(r_tm), badv=new(dt=torch.bfloat16), bret=new(dt=torch.bfloat16))
 
@@ -990,7 +976,7 @@ def test_affine_scan_matches_generic_recurrence(oracle, W, B):
     beta[rng.random((N, T)) < 0.01] = 0.0
     ws = B.Workspace(N, T)
     for fwd in (False, True):
-        out = B.rlcs_affine_scan(torch.from_numpy(alpha).cuda(), torch.from_numpy(beta).cuda(), forward=fwd,
+        out = B.rlcs_affine_scan(guarded_upload(alpha), guarded_upload(beta), forward=fwd,
                                  workspace=ws).cpu().numpy()
         ref = np.stack([oracle.linear_recurrence(alpha[n].astype(np.float64), beta[n].astype(np.float64), 0.0,
                                                  forward=fwd) for n in range(N)])
