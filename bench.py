@@ -182,7 +182,7 @@ class ClockSampler:
                0x10: "sync_boost", 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown",
                0x80: "hw_power_brake_slowdown", 0x100: "display_clock_setting"}
 
-    def __init__(self, index: int, period_s: float = 0.002):
+    def __init__(self, index: int, period_s: float = 0.0005):
         self.samples, self.reasons, self.power = [], set(), []
         self.period, self._stop, self.max_mhz, self.ok = period_s, threading.Event(), None, False
         try:
@@ -290,23 +290,30 @@ class GpuBatch:
             raise KeyError(algo)
         self.launches += 1
 
-    def step(self, events=None):
-        torch = self.torch
+    def step(self, timed=None, events=None):
+        """One pass of the seven calls.  `timed` = index of the one call of this step that is
+        bracketed by the two CUDA events in `events` (on the launching stream)."""
         for k, a in enumerate(ALGOS):
-            if events is not None:
-                events[k].record()
+            if k == timed:
+                events[0].record()
             self.call(a)
-        if events is not None:
-            events[len(ALGOS)].record()
+            if k == timed:
+                events[1].record()
 
 
 def time_device(batch: GpuBatch, steps: int, warmup: int, dist):
-    """K timed steps with inputs resident in HBM; per-kernel durations from CUDA events recorded
-    on the launching stream between the launches."""
+    """K timed steps with inputs resident in HBM.  Per-kernel durations come from CUDA events on the
+    launching stream inside the timed region: every step brackets ONE of its seven launches (step k
+    the launch k mod 7), so each kernel is sampled about K/7 times while the other six launches of
+    a step run back to back as a caller would issue them -- an event between every pair of launches
+    costs several per cent of a step by itself.  When K < 7 the kernels that the timed region did not
+    reach are sampled in extra, untimed steps."""
     torch = batch.torch
     for _ in range(warmup):
         batch.step()
-    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(len(ALGOS) + 1)] for _ in range(steps)]
+    n = len(ALGOS)
+    extra = max(0, n - steps)
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps + extra)]
     start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     dist.barrier()
     torch.cuda.synchronize()
@@ -314,14 +321,18 @@ def time_device(batch: GpuBatch, steps: int, warmup: int, dist):
     with ClockSampler(torch.cuda.current_device()) as clk:
         start.record()
         for k in range(steps):
-            batch.step(ev[k])
+            batch.step(k % n, ev[k])
         stop.record()
         torch.cuda.synchronize()
     dist.barrier()
+    launches = batch.launches - launches0
+    for k in range(steps, steps + extra):
+        batch.step(k % n, ev[k])
+    torch.cuda.synchronize()
     total_ms = start.elapsed_time(stop)
-    per_algo_ms = {a: [ev[k][j].elapsed_time(ev[k][j + 1]) for k in range(steps)] for j, a in enumerate(ALGOS)}
+    per_algo_ms = {a: [ev[k][0].elapsed_time(ev[k][1]) for k in range(steps + extra) if k % n == j] for j, a in enumerate(ALGOS)}
     assert batch.ws.device_status() == 0, "device reported a carry-wait timeout"
-    return total_ms, per_algo_ms, batch.launches - launches0, clk.summary()
+    return total_ms, per_algo_ms, launches, clk.summary()
 
 
 def time_gae_normalized(batch: GpuBatch, steps: int, peak: float):
@@ -740,8 +751,10 @@ def sweep_case(torch, B, ro, algo: str, use_truncs: bool, hbm_peak: float, l2_by
     del sets, graph
     ceiling_us = copy_ceiling_us(torch, B, ro_eff, algo, algo_bytes, R, trials)
     ceiling_gbs = algo_bytes / (ceiling_us * 1e-6) / 1e9
+    memcpy_us = memcpy_ceiling_us(torch, algo_bytes, R, trials)
     return {"algo": algo, "N": ro.N, "T": ro.T, "truncs": use_truncs, "us_per_call": round(best, 3),
             "copy_ceiling_us": round(ceiling_us, 3), "copy_ceiling_gbs": round(ceiling_gbs, 1),
+            "memcpy_ceiling_us": round(memcpy_us, 3), "frac_of_memcpy_ceiling": round(memcpy_us / best, 4),
             "frac_of_copy_ceiling": round(gbs / ceiling_gbs, 4),
             "us_per_call_median": round(statistics.median(per_call_us), 3),
             "full_call_us": round(min(full_call_us), 3), "env_steps_per_s": ro.N * ro.T / (best * 1e-6),
@@ -765,6 +778,33 @@ def copy_ceiling_us(torch, B, ro, algo: str, algo_bytes: int, R: int, trials: in
     with torch.cuda.graph(graph):
         for i in range(R):
             call(i)
+    graph.replay()
+    times = []
+    for _ in range(trials):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        graph.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        times.append(1e3 * e0.elapsed_time(e1) / R)
+    return min(times)
+
+
+def memcpy_ceiling_us(torch, algo_bytes: int, R: int, trials: int) -> float:
+    """A second, independent ceiling: the driver's own device-to-device copy (cudaMemcpyAsync through
+    torch's copy_) moving the same total of bytes -- half of them read, half written -- in the same
+    cold-L2 rotation and CUDA-graph replay as the scan launches."""
+    n = -(-(algo_bytes // 2 // 4) // 4096) * 4096          # whole 16 KB pieces: odd sizes take a slower copy path
+    rd = [torch.empty(n, dtype=torch.float32, device="cuda").normal_() for _ in range(R)]
+    wr = [torch.empty(n, dtype=torch.float32, device="cuda") for _ in range(R)]
+    for i in range(R):
+        wr[i].copy_(rd[i])
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        for i in range(R):
+            wr[i].copy_(rd[i])
     graph.replay()
     times = []
     for _ in range(trials):
@@ -845,7 +885,11 @@ def main():
     ap.add_argument("--sweep-pick", default=None, metavar="CONFIG,ALGO,T,TRUNCS",
                     help="with --sweep-only: keep the matching cases only, e.g. 3,vtrace,256,1 or 4,gae,, (empty = any)")
     ap.add_argument("--sweep-trials", type=int, default=5)
+    ap.add_argument("--sweep-shape", default=None, metavar="N,T,ALGO,TRUNCS[,P_TRUNC]",
+                    help="with --sweep-only: one cold-L2 case on a dense-reward batch of this shape instead of the configurations")
     ap.add_argument("--variant", type=int, default=None, help="tile variant test hook (default: library default)")
+    ap.add_argument("--no-dependent-launch", action="store_true",
+                    help="measurement hook: launch the scan kernels without programmatic stream serialisation")
     ap.add_argument("--no-truncs", action="store_true", help="bench batch without per-step truncation handling")
     ap.add_argument("--rows", type=int, default=WORKLOAD["N"], help="num_envs of the bench batch (default: full size)")
     ap.add_argument("--only", choices=("time_major", "bf16", "retrace_probs", "elig_trace_vec", "elig_trace_vec_beta",
@@ -884,6 +928,8 @@ def main():
     binding.lib()                                   # no library, no benchmark: there is no fallback
     if args.variant is not None:
         binding.rlcs_debug_set_tile_variant(args.variant)
+    if args.no_dependent_launch:
+        binding.rlcs_debug_set_dependent_launch(False)
     assert torch.cuda.is_available(), "bench.py needs a CUDA device"
     local = int(os.environ.get("LOCAL_RANK", "0"))
     torch.cuda.set_device(local)
@@ -891,11 +937,19 @@ def main():
 
     if args.sweep_only:
         peak, _ = measured_peak()
+        if args.sweep_shape is not None:
+            n, t, a, tr, *rest = args.sweep_shape.split(",")
+            ro = workloads.make_rollout(3, int(n), int(t), with_truncs=True, p_trunc=float(rest[0]) if rest else 0.005)
+            case = sweep_case(torch, binding, ro, a, bool(int(tr)), peak, torch.cuda.get_device_properties(0).L2_cache_size,
+                              trials=max(1, args.sweep_trials))
+            print(json.dumps({"detail": "sweep", **case}), flush=True)
+            return
         pick = None
         if args.sweep_pick is not None:
             c, a, t, tr = (args.sweep_pick.split(",") + ["", "", "", ""])[:4]
             pick = (int(c) if c else None, a or None, int(t) if t else None, bool(int(tr)) if tr else None)
-        print(json.dumps({"sweeps": run_sweeps(torch, peak, pick, max(1, args.sweep_trials))}), flush=True)
+        for case in run_sweeps(torch, peak, pick, max(1, args.sweep_trials)):
+            print(json.dumps({"detail": "sweep", **case}), flush=True)
         return
     if args.only is not None:
         peak, _ = measured_peak()

@@ -42,10 +42,17 @@
  *   points, that are ordered on one stream.  Two calls that may run concurrently need two
  *   workspaces.  When rlcs_workspace_bytes(N, T) is 0 the workspace may be NULL.
  * Execution.  Work is enqueued on `cuda_stream` (a cudaStream_t passed as void*; NULL = the
- *   default stream) and the call returns without synchronising.  Argument errors are returned
- *   before anything is launched.  The only device-side wait is the bounded carry wait between
- *   thread blocks; if it ever gives up, the kernel still terminates normally, the outputs of that
- *   call are unspecified, and rlcs_last_device_status reports RLCS_ERR_TIMEOUT.
+ *   default stream) and the call returns without synchronising.  The row-major scan kernels are
+ *   launched with programmatic stream serialisation: their thread blocks may be placed on the GPU
+ *   while the preceding kernel of the stream drains, but they wait for that kernel's completion
+ *   (and the visibility of its writes) before their first access to global memory -- caller
+ *   tensors and workspace alike -- so the stream's ordering guarantees are unchanged.  Argument
+ *   errors are returned before anything is launched.  The only device-side wait is the bounded
+ *   carry wait between thread blocks.  A block only ever waits for tiles that precede its own in
+ *   scan order, and tiles are assigned by launch index: the look-back relies on the hardware
+ *   starting thread blocks in index order, as every current GPU does but CUDA does not promise.
+ *   Should a block ever wait for one that has not been started, nothing hangs: the wait runs out
+ *   of polls, the kernel still terminates normally, the outputs of that call are unspecified, and rlcs_last_device_status reports RLCS_ERR_TIMEOUT.
  * Inputs must be finite.  A reset is a decay of exactly 0 inside the scan (0 * finite severs
  *   exactly); successor values at resets are selected, never multiplied.  A NaN or infinity in one
  *   episode can therefore reach the flagged last step of the preceding episode, but nothing else.
@@ -108,8 +115,12 @@ int rlcs_gae(const float* rewards, const float* values, const uint8_t* dones, co
  *   advantages[n,t] = (A_t - mean(A)) / (std(A) + eps),   std = sqrt(sum (A - mean)^2 / (N*T - ddof)),
  *   ddof = 0 (population) or 1 (sample; std = 0 when N*T = 1);   eps >= 0, finite
  *   returns[n,t]    = A_t + values_t  from the un-normalised A_t  (may be NULL)
- * Three launches: the GAE kernel (which also leaves per-tile sums of A and A^2), a one-block
- * reduction to mean and 1/(std + eps), and an in-place rescale of `advantages` -- one read of A
+ *   With eps = 0 and std = 0 (all advantages equal) the quotient is 0/0 and the advantages come out
+ *   non-finite, as the formula says; pass eps > 0 to get zeros there.
+ * Three launches: the GAE kernel (which also leaves, per tile, the sum of A and the sum of squared
+ * deviations from the tile's own mean), a one-block reduction in double to mean and 1/(std + eps)
+ * (tile statistics are merged as q_i + n_i (m_i - mean)^2, so a mean much larger than the spread
+ * does not cancel the variance away), and an in-place rescale of `advantages` -- one read of A
  * fewer than GAE, a statistics pass and a rescale.  Deterministic (fixed reduction order).
  * `workspace`: at least rlcs_gae_normalized_workspace_bytes(N, T) bytes (always > 0), 16-byte
  * aligned, initialised once with rlcs_workspace_init; same sharing rules as any workspace.
@@ -397,6 +408,10 @@ int rlcs_affine_scan(const float* alpha, const float* beta, float* out, int64_t 
  * an upper bound over all variants.
  */
 int rlcs_debug_set_tile_variant(int variant);
+/* 1 if that tile variant is compiled into this build (the default build holds the shapes the
+ * selection can return plus two bulk-copy ring shapes; -DRLCS_ALL_VARIANTS compiles the whole table),
+ * else 0.  rlcs_debug_set_tile_variant returns RLCS_ERR_ARG for a variant that is not compiled. */
+int rlcs_debug_variant_built(int variant);
 
 /* Elements per tile of a variant (0 for an unknown variant). */
 int rlcs_debug_tile_elems(int variant);
@@ -411,6 +426,10 @@ int rlcs_debug_variant_for(int algorithm, int has_truncs, int64_t N, int64_t T);
 /* Shape of a variant: threads per block, steps per thread, blocks per SM it is compiled for, and
  * ring stages (0 = the one-tile-per-block kernel).  Any output pointer may be NULL. */
 int rlcs_debug_variant_info(int variant, int* threads, int* steps_per_thread, int* blocks_per_sm, int* ring_stages);
+
+/* Test / measurement hook: 0 launches the row-major scan kernels without programmatic stream
+ * serialisation (see "Execution" above), 1 (default) with it.  Results are identical. */
+int rlcs_debug_set_dependent_launch(int on);
 
 /*
  * Test hook: rows that are exactly 2..8 tiles long are scanned by one thread-block cluster per row,

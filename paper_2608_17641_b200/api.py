@@ -37,6 +37,8 @@ def _workspace(like, N: int, T: int, nbytes: int | None = None, stream=None):
     """One initialised workspace per (device, stream, N, T, size), reused by every later call on that
     shape and stream.  The stream is part of the key because two calls share carry records and a
     call counter in the workspace: only calls ordered on one stream may share one."""
+    if not like.is_cuda:
+        raise TypeError("rlcs takes CUDA tensors (device pointers); there is no CPU path")
     s = _torch().cuda.current_stream(like.device) if stream is None else stream
     key = (like.device, int(s.cuda_stream), N, T, nbytes)
     ws = _workspaces.get(key)

@@ -69,7 +69,9 @@ SIGNATURES = {
     "rlcs_debug_stream_copy": ([_vp, _vp, _sz, _sz, _vp], _int),
     "rlcs_debug_force_wide_index": ([_int], _int),
     "rlcs_debug_allow_cluster_carry": ([_int], _int),
+    "rlcs_debug_set_dependent_launch": ([_int], _int),
     "rlcs_debug_variant_for": ([_int, _int, _i64, _i64], _int),
+    "rlcs_debug_variant_built": ([_int], _int),
     "rlcs_debug_variant_info": ([_int] + [ctypes.POINTER(ctypes.c_int)] * 4, _int),
 }
 
@@ -408,6 +410,16 @@ def rlcs_debug_variant_for(algorithm: str, has_truncs: bool, N: int, T: int) -> 
     _check(lib().rlcs_debug_variant_info(v, *[ctypes.byref(o) for o in out]))
     return dict(variant=v, threads=out[0].value, steps_per_thread=out[1].value, blocks_per_sm=out[2].value,
                 ring_stages=out[3].value)
+
+
+def rlcs_debug_variant_built(variant: int) -> bool:
+    """Whether that tile variant is compiled into the loaded library."""
+    return bool(lib().rlcs_debug_variant_built(int(variant)))
+
+
+def rlcs_debug_set_dependent_launch(on: bool):
+    """Measurement hook: launch the row-major scan kernels with (default) or without programmatic stream serialisation."""
+    _check(lib().rlcs_debug_set_dependent_launch(int(bool(on))))
 
 
 def rlcs_debug_allow_cluster_carry(on: bool):

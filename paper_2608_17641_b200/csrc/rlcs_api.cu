@@ -8,6 +8,7 @@ bool g_cluster = true;
 bool g_wide_index = false;
 long long g_mute_tile = -1;
 long long g_spin_cap = 0;
+bool g_pdl = true;
 }  // namespace rlcs_hooks
 
 extern "C" {
@@ -43,8 +44,10 @@ int rlcs_workspace_init(void* workspace, size_t workspace_bytes, void* cuda_stre
     if (workspace_bytes < sizeof(unsigned) * rlcs::kHeaderWords) return RLCS_ERR_WORKSPACE;
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
     if (cudaMemsetAsync(workspace, 0, workspace_bytes, s) != cudaSuccess) return RLCS_ERR_CUDA;
-    // epoch starts at 1 so that zeroed records are never valid (byte pattern 0x01 0x00 0x00 0x00)
-    if (cudaMemsetAsync(workspace, 1, 1, s) != cudaSuccess) return RLCS_ERR_CUDA;
+    // the call counter starts at 256 (byte pattern 0x00 0x01 0x00 0x00): zeroed records are never
+    // valid, and neither are the small record tags (0, 1, 2) that the time-major kernels leave in the
+    // same area when a workspace is shared between the two families of entry points
+    if (cudaMemsetAsync(static_cast<unsigned char*>(workspace) + 1, 1, 1, s) != cudaSuccess) return RLCS_ERR_CUDA;
     return RLCS_OK;
 }
 
@@ -151,7 +154,7 @@ int rlcs_gae_normalized(const float* rewards, const float* values, const uint8_t
     st = run(rlcs::launch_gae_stats, p, variant, truncs != nullptr, vec, cuda_stream);
     if (st != RLCS_OK) return st;
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
-    if (rlcs::launch_norm_finalize(p.stats, p.num_tiles, (double)total, ddof, eps, mean_rstd, s) != cudaSuccess) return RLCS_ERR_CUDA;
+    if (rlcs::launch_norm_finalize(p.stats, p.num_tiles, total, tile_elems(variant), ddof, eps, mean_rstd, s) != cudaSuccess) return RLCS_ERR_CUDA;
     if (rlcs::launch_norm_rescale(advantages, total, mean_rstd, vec, s) != cudaSuccess) return RLCS_ERR_CUDA;
     return RLCS_OK;
 }
@@ -320,8 +323,13 @@ int rlcs_affine_scan(const float* alpha, const float* beta, float* out, int64_t 
 
 int rlcs_debug_set_tile_variant(int variant) {
     if (variant < -1 || variant >= rlcs::kNumVariants) return RLCS_ERR_ARG;
+    if (variant >= 0 && !rlcs::variant_built(variant)) return RLCS_ERR_ARG;      // not compiled into this build
     g_variant = variant;
     return RLCS_OK;
+}
+
+int rlcs_debug_variant_built(int variant) {
+    return variant >= 0 && variant < rlcs::kNumVariants && rlcs::variant_built(variant) ? 1 : 0;
 }
 
 int rlcs_debug_tile_elems(int variant) {
@@ -342,6 +350,11 @@ int rlcs_debug_variant_info(int variant, int* threads, int* steps_per_thread, in
     if (steps_per_thread) *steps_per_thread = tv.items;
     if (blocks_per_sm) *blocks_per_sm = tv.min_blocks;
     if (ring_stages) *ring_stages = tv.stages;
+    return RLCS_OK;
+}
+
+int rlcs_debug_set_dependent_launch(int on) {
+    rlcs_hooks::g_pdl = on != 0;
     return RLCS_OK;
 }
 

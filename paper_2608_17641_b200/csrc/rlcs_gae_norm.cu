@@ -6,31 +6,44 @@ namespace rlcs {
 
 RLCS_DEFINE_LAUNCHER(launch_gae_stats, kGaeStats, true)
 
-// One block: per-tile partial sums -> {mean, 1/(std + eps)}.  Each thread adds its strided share in
-// double, then a shared-memory tree in a fixed order: the result does not depend on timing.
+// One block: per-tile {sum, sum of squared deviations from the tile mean} -> {mean, 1/(std + eps)}.
+// Two strided passes in double, each followed by a shared-memory tree in a fixed order (the result
+// does not depend on timing): first the mean, then
+//     sum (A - mean)^2 = sum over tiles of [ q_i + n_i (m_i - mean)^2 ],   m_i = s_i / n_i,
+// which is exact algebra and never subtracts two large numbers.  Tile i of the scan order holds
+// `tile` steps except the one at the array's end (scan-order tile 0 of this backward scan).
 __global__ void __launch_bounds__(1024) norm_finalize_kernel(const float* __restrict__ partial, long long num_tiles,
-                                                             double count, int ddof, float eps, float* __restrict__ out) {
-    __shared__ double sh1[1024], sh2[1024];
-    double s1 = 0.0, s2 = 0.0;
-    for (long long i = threadIdx.x; i < num_tiles; i += 1024) {
-        s1 += (double)partial[2 * i];
-        s2 += (double)partial[2 * i + 1];
-    }
-    sh1[threadIdx.x] = s1;
-    sh2[threadIdx.x] = s2;
+                                                             long long total, int tile, int ddof, float eps,
+                                                             float* __restrict__ out) {
+    __shared__ double sh[1024];
+    __shared__ double mean_sh;
+    double acc = 0.0;
+    for (long long i = threadIdx.x; i < num_tiles; i += 1024) acc += (double)partial[2 * i];
+    sh[threadIdx.x] = acc;
     __syncthreads();
     for (int d = 512; d > 0; d >>= 1) {
-        if ((int)threadIdx.x < d) {
-            sh1[threadIdx.x] += sh1[threadIdx.x + d];
-            sh2[threadIdx.x] += sh2[threadIdx.x + d];
-        }
+        if ((int)threadIdx.x < d) sh[threadIdx.x] += sh[threadIdx.x + d];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) mean_sh = sh[0] / (double)total;
+    __syncthreads();
+    const double mean = mean_sh;
+    const long long last = total - (num_tiles - 1) * (long long)tile;      // steps in the ragged tile
+    acc = 0.0;
+    for (long long i = threadIdx.x; i < num_tiles; i += 1024) {
+        const double n = (double)(i == 0 ? last : (long long)tile);
+        const double dm = (double)partial[2 * i] / n - mean;
+        acc += (double)partial[2 * i + 1] + n * dm * dm;
+    }
+    sh[threadIdx.x] = acc;
+    __syncthreads();
+    for (int d = 512; d > 0; d >>= 1) {
+        if ((int)threadIdx.x < d) sh[threadIdx.x] += sh[threadIdx.x + d];
         __syncthreads();
     }
     if (threadIdx.x == 0) {
-        const double mean = sh1[0] / count;
-        const double denom = count - (double)ddof;
-        double var = denom > 0.0 ? (sh2[0] - sh1[0] * mean) / denom : 0.0;     // sum (A - mean)^2 = sum A^2 - mean * sum A
-        if (var < 0.0) var = 0.0;
+        const double denom = (double)total - (double)ddof;
+        const double var = denom > 0.0 ? sh[0] / denom : 0.0;
         out[0] = (float)mean;
         out[1] = (float)(1.0 / (sqrt(var) + (double)eps));
     }
@@ -55,9 +68,9 @@ __global__ void __launch_bounds__(256) norm_rescale_kernel(float* __restrict__ a
     }
 }
 
-cudaError_t launch_norm_finalize(const float* partial, long long num_tiles, double count, int ddof, float eps,
+cudaError_t launch_norm_finalize(const float* partial, long long num_tiles, long long total, int tile, int ddof, float eps,
                                  float* mean_rstd, cudaStream_t stream) {
-    norm_finalize_kernel<<<1, 1024, 0, stream>>>(partial, num_tiles, count, ddof, eps, mean_rstd);
+    norm_finalize_kernel<<<1, 1024, 0, stream>>>(partial, num_tiles, total, tile, ddof, eps, mean_rstd);
     return cudaGetLastError();
 }
 

@@ -7,8 +7,8 @@ namespace rlcs {
 template <bool TRUNC, bool VEC, int V>
 cudaError_t launch_skip_variant(const ScanParams& p, cudaStream_t stream) {
     constexpr TileVariant tv = kVariants[V];
-    scan_kernel_gae_skip<TRUNC, VEC, tv.threads, tv.items, tv.min_blocks><<<(unsigned)p.num_tiles, tv.threads, 0, stream>>>(p);
-    return cudaGetLastError();
+    return launch_scan(scan_kernel_gae_skip<TRUNC, VEC, tv.threads, tv.items, tv.min_blocks>, (unsigned)p.num_tiles, tv.threads, 0,
+                       stream, 0, p);
 }
 
 template <bool TRUNC, bool VEC>

@@ -74,13 +74,12 @@ int check_alignment(const Ptrs& ps, bool* vec) {
 // flight, so algorithms with few registers run more blocks per SM or 16 steps per thread.  Small
 // problems are bound by latency: smaller tiles spread them over more SMs, unless rows are long
 // enough for the inter-block carry to dominate.
-int choose_variant(int algo, bool trunc, int64_t total, int64_t T) {
-    if (g_variant >= 0 && RLCS_NS::variant_built_for(algo, g_variant)) return g_variant;
+int choose_variant_unchecked(int algo, bool trunc, int64_t total, int64_t T) {
     if (total < (int64_t(1) << 23)) {
         // latency-bound sizes (cold-L2 sweeps): long rows want few carry hops (2048-step tiles, one
         // cluster per row where that fits), the smallest problems want many small blocks
         if (T > 2048) return 19;
-        return (total <= (int64_t(1) << 19) && RLCS_NS::variant_built_for(algo, 1)) ? 1 : 6;
+        return total <= (int64_t(1) << 19) ? 1 : 6;
     }
     if (RLCS_NS::kIoBf16) {
         // 16 steps per thread (one 32-byte access per tensor); with half the bytes per step the kernels
@@ -106,6 +105,14 @@ int choose_variant(int algo, bool trunc, int64_t total, int64_t T) {
         case RLCS_NS::kPrefix: return 18;
         default: return 0;
     }
+}
+
+int choose_variant(int algo, bool trunc, int64_t total, int64_t T) {
+    if (g_variant >= 0 && RLCS_NS::variant_built_for(algo, g_variant)) return g_variant;
+    const int v = choose_variant_unchecked(algo, trunc, total, T);
+    if (RLCS_NS::variant_built_for(algo, v)) return v;
+    // not compiled for this algorithm / element type: the nearest shape that every build has
+    return (total < (int64_t(1) << 23) && T <= 2048) ? 6 : 0;
 }
 
 // How the carry between thread blocks travels for one call, and the workspace bytes it needs.

@@ -5,7 +5,42 @@
 
 #include "rlcs_scan.cuh"
 
+namespace rlcs_hooks {
+extern bool g_pdl;                 // launch with programmatic stream serialisation (default on)
+}
+
 namespace RLCS_NS {
+
+// Every scan kernel goes through this launch: grid/block/shared memory, an optional thread-block
+// cluster size, and programmatic stream serialisation, which lets the blocks of this launch be
+// placed while the previous kernel of the stream drains (the kernels call grid_dependency_wait()
+// before they touch global memory, so ordering on the stream is unchanged).
+template <class Kernel>
+cudaError_t launch_scan(Kernel kernel, unsigned grid, unsigned block, size_t smem, cudaStream_t stream, int cluster,
+                        const ScanParams& p) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid, 1, 1);
+    cfg.blockDim = dim3(block, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[2];
+    unsigned n = 0;
+    if (cluster > 1) {
+        attr[n].id = cudaLaunchAttributeClusterDimension;
+        attr[n].val.clusterDim.x = (unsigned)cluster;
+        attr[n].val.clusterDim.y = 1;
+        attr[n].val.clusterDim.z = 1;
+        ++n;
+    }
+    if (rlcs_hooks::g_pdl) {
+        attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[n].val.programmaticStreamSerializationAllowed = 1;
+        ++n;
+    }
+    cfg.attrs = attr;
+    cfg.numAttrs = n;
+    return cudaLaunchKernelEx(&cfg, kernel, p);
+}
 
 // stages == 0: scan_kernel (one tile per block).  stages > 0: scan_kernel_tma (persistent blocks,
 // bulk-copy ring of that many tiles; min_blocks = blocks per SM it is compiled and sized for).
@@ -34,11 +69,27 @@ constexpr TileVariant kVariants[kNumVariants] = {
     {128, 16, 6, 0},   // 19: 2048, 16 steps per thread, at most 80 registers
     {128, 16, 8, 0},   // 20: 2048, 16 steps per thread, at most 64 registers
 };
-// The bfloat16 build instantiates only these tile shapes (16 steps per thread = one 32-byte access).
-__host__ __device__ constexpr bool variant_built(int v) { return !kIoBf16 || v == 0 || v == 5 || v == 6 || v >= 18; }
-// ... and the observation-skip scans only these (the rest of the table is tuning history of the seven kernels).
+// Which rows of the table are compiled.  The default build holds the shapes the selection in
+// choose_variant() can return (0, 1, 5, 6, 18, 19, 20) and two persistent bulk-copy ring shapes (8, 11)
+// that the tests cross-check against; the rest of the table is tuning history and is compiled only
+// with -DRLCS_ALL_VARIANTS.  The bfloat16 build instantiates 16-steps-per-thread shapes (one 32-byte
+// access) and the two 8-step ones; the observation-skip scans and the bare affine scan (a test
+// hook) fewer still.
+#ifdef RLCS_ALL_VARIANTS
+constexpr bool kAllVariants = true;
+#else
+constexpr bool kAllVariants = false;
+#endif
+__host__ __device__ constexpr bool variant_built(int v) {
+    if (kIoBf16) return v == 0 || v == 5 || v == 6 || v >= 18;
+    return kAllVariants || v == 0 || v == 1 || v == 5 || v == 6 || v == 8 || v == 11 || v >= 18;
+}
 __host__ __device__ constexpr bool variant_built_for(int algo, int v) {
-    return variant_built(v) && (!uses_skip(algo) || v == 0 || v == 6 || v >= 18);
+    if (!variant_built(v)) return false;
+    if (uses_skip(algo)) return v == 0 || v == 6 || v >= 18;
+    if (is_affine(algo)) return kAllVariants || v == 0 || v == 6;
+    if (algo == kGaeStats) return kAllVariants || v == 0 || v == 1 || v == 6 || v == 19;
+    return true;
 }
 constexpr int kMinTileElems = 512;
 constexpr int kRetraceProbsThreads = 256, kRetraceProbsItems = 4;      // tile of rlcs_retrace_probs
@@ -70,27 +121,15 @@ cudaError_t launch_persistent(const ScanParams& p, cudaStream_t stream) {
         s_blocks[dev] = per_sm * sms;
     }
     const long long grid = p.num_tiles < s_blocks[dev] ? p.num_tiles : s_blocks[dev];
-    kernel<<<(unsigned)grid, tv.threads, kSmem, stream>>>(p);
-    return cudaGetLastError();
+    return launch_scan(kernel, (unsigned)grid, tv.threads, kSmem, stream, 0, p);
 }
 
 // One cluster per row (p.cluster = tiles per row, 2..8): carry through distributed shared memory.
 template <int ALGO, bool TRUNC, int V>
 cudaError_t launch_cluster(const ScanParams& p, cudaStream_t stream) {
     constexpr TileVariant tv = kVariants[V];
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)p.num_tiles, 1, 1);
-    cfg.blockDim = dim3(tv.threads, 1, 1);
-    cfg.dynamicSmemBytes = 0;
-    cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = (unsigned)p.cluster;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, scan_kernel_cluster<ALGO, TRUNC, tv.threads, tv.items, tv.min_blocks>, p);
+    return launch_scan(scan_kernel_cluster<ALGO, TRUNC, tv.threads, tv.items, tv.min_blocks>, (unsigned)p.num_tiles, tv.threads, 0,
+                       stream, p.cluster, p);
 }
 
 template <int ALGO, bool TRUNC, bool VEC, int V>
@@ -102,14 +141,12 @@ cudaError_t launch_variant(const ScanParams& p, cudaStream_t stream) {
     if constexpr (tv.stages > 0 && VEC) {
         // (rows shorter than a chunk go to the one-tile kernel: the persistent one assumes T >= ITEMS)
         if (p.T >= (unsigned)tv.items) return launch_persistent<ALGO, TRUNC, V>(p, stream);
-        scan_kernel<ALGO, TRUNC, true, tv.threads, tv.items, tv.min_blocks>
-            <<<(unsigned)p.num_tiles, tv.threads, 0, stream>>>(p);
-        return cudaGetLastError();
+        return launch_scan(scan_kernel<ALGO, TRUNC, true, tv.threads, tv.items, tv.min_blocks>, (unsigned)p.num_tiles, tv.threads,
+                           0, stream, 0, p);
     } else {
         // bulk copies need 16-byte aligned pointers; otherwise the element-wise kernel of the same tile shape
-        scan_kernel<ALGO, TRUNC, VEC, tv.threads, tv.items, tv.min_blocks>
-            <<<(unsigned)p.num_tiles, tv.threads, 0, stream>>>(p);
-        return cudaGetLastError();
+        return launch_scan(scan_kernel<ALGO, TRUNC, VEC, tv.threads, tv.items, tv.min_blocks>, (unsigned)p.num_tiles, tv.threads,
+                           0, stream, 0, p);
     }
 }
 
@@ -148,7 +185,7 @@ cudaError_t launch_affine_fwd(const ScanParams&, int variant, bool trunc, bool v
 cudaError_t launch_retrace_probs(const ScanParams&, bool trunc, bool vec, bool vec_rows, cudaStream_t);
 cudaError_t launch_gae_stats(const ScanParams&, int variant, bool trunc, bool vec, cudaStream_t);
 cudaError_t launch_gae_skip(const ScanParams&, int variant, bool trunc, bool vec, cudaStream_t);
-cudaError_t launch_norm_finalize(const float* partial, long long num_tiles, double count, int ddof, float eps,
+cudaError_t launch_norm_finalize(const float* partial, long long num_tiles, long long total, int tile, int ddof, float eps,
                                  float* mean_rstd, cudaStream_t stream);
 cudaError_t launch_norm_rescale(float* adv, long long total, const float* mean_rstd, bool vec, cudaStream_t stream);
 

@@ -70,9 +70,9 @@ int rlcs_gae_no_alloc(const float* rewards, const float* values, const uint8_t* 
     if (st != RLCS_OK) return st;
     // The array keeps whatever the previous call left.  Tile records need no clearing: a call tags
     // its records with the call counter, which the last block of every completed call advances.
-    // The finished-block counter must start at zero even if an earlier launch was refused half way.
-    // The status word is left alone: it holds RLCS_ERR_TIMEOUT from an earlier call until
-    // rlcs_no_alloc_last_device_status reads and clears it.
+    // The finished-block counter (second header word) must start at zero even if an earlier launch
+    // was refused half way.  The status word after it is left alone: it holds RLCS_ERR_TIMEOUT from
+    // an earlier call until rlcs_no_alloc_last_device_status reads and clears it.
     if (cudaMemsetAsync(static_cast<unsigned char*>(scratch) + 4, 0, 4, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
         return RLCS_ERR_CUDA;
     st = rlcs_gae(rewards, values, dones, truncs, trunc_bootstrap, bootstrap, advantages, returns, N, T, gamma,

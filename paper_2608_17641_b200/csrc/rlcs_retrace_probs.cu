@@ -7,9 +7,8 @@ namespace rlcs {
 
 template <bool TRUNC, bool VEC, int AV>
 static cudaError_t launch_one(const ScanParams& p, cudaStream_t stream) {
-    scan_kernel_retrace_probs<TRUNC, VEC, kRetraceProbsThreads, kRetraceProbsItems, 4, AV>
-        <<<(unsigned)p.num_tiles, kRetraceProbsThreads, 0, stream>>>(p);
-    return cudaGetLastError();
+    return launch_scan(scan_kernel_retrace_probs<TRUNC, VEC, kRetraceProbsThreads, kRetraceProbsItems, 4, AV>,
+                       (unsigned)p.num_tiles, kRetraceProbsThreads, 0, stream, 0, p);
 }
 
 template <bool TRUNC, bool VEC>

@@ -58,7 +58,7 @@ namespace RLCS_NS {
 enum Algo : int {
     kGae = 0, kTdLambda = 1, kDisc = 2, kVtrace = 3, kRetrace = 4, kElig = 5, kPrefix = 6,
     kAffineBwd = 7, kAffineFwd = 8,
-    kGaeStats = 9,    // GAE that also leaves per-tile sums of A and A^2 (for advantage normalisation)
+    kGaeStats = 9,    // GAE that also leaves per-tile sums of A and of its squared deviations (for advantage normalisation)
     kRetraceProbs = 10, // Retrace(lambda) from [N,T,A] Q-values and action probabilities
     // Observation-skip masking (Section 9.2): masked steps are transparent.  Two scans:
     kFillSkip = 11,     // W_t = V_t at unmasked steps, the successor's W (or the flag's successor value) at masked ones
@@ -106,7 +106,7 @@ struct ScanParams {
     io_t* out0;
     io_t* out1;               // second output or nullptr
     io_t* out2;               // scan_kernel_gae_skip: the filled values W
-    float* stats;             // kGaeStats: per scan-order tile {sum A, sum A^2}
+    float* stats;             // kGaeStats: per scan-order tile {sum A, sum (A - tile mean)^2}
     long long total;          // N*T
     long long num_tiles;
     unsigned T;
@@ -137,6 +137,18 @@ __device__ __forceinline__ Pair apply(Pair x, Pair acc) {
     r.b = x.b * acc.b;
     return r;
 }
+
+// ------------------------------------------------------------------------------------------ programmatic dependent launch
+// The kernels are launched with programmatic stream serialisation: the blocks of a launch may be
+// placed on the SMs while the previous kernel of the stream is still draining, so that launch
+// latency and block set-up overlap that kernel's tail.  grid_dependency_wait() returns once the
+// previous kernel has completed and its writes are visible; NOTHING in global memory -- caller
+// tensors, the workspace header, tile records -- is read or written before it.
+// grid_dependency_launch() tells the scheduler that the next launch's blocks may be placed; it is
+// given first thing, because a later kernel still waits for this one's completion at its own
+// grid_dependency_wait().  Both are no-ops for a launch without the attribute.
+__device__ __forceinline__ void grid_dependency_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
 // ------------------------------------------------------------------------------------------ global loads / stores
 // 256-bit global accesses (sm_100): one instruction moves a thread's 8 consecutive fp32 values, so a
@@ -431,7 +443,7 @@ __device__ __forceinline__ void sign_off(const ScanParams& p) {
         if (done == gridDim.x - 1) {
             p.header[1] = 0;
             const unsigned e = ld_volatile_u32(p.header);
-            p.header[0] = (e == 0xffffffffu) ? 1u : e + 1u;
+            p.header[0] = (e == 0xffffffffu) ? 256u : e + 1u;      // never 0..255 (see rlcs_workspace_init)
         }
     }
 }
@@ -655,6 +667,15 @@ struct ScanSmem {
     int need[2];         // the tile is entered mid-episode
     Pair cl_agg;         // cluster carry: this tile's aggregate, read by the other blocks of the cluster
 };
+
+// Scan-order tile of this block, and the call's epoch when the carry goes through the workspace.
+// Tiles are taken in launch-index order: a block waits only for the records of tiles with smaller
+// indices, whose blocks the hardware has dispatched before it.  Call after grid_dependency_wait().
+__device__ __forceinline__ long long take_tile(const ScanParams& p, unsigned& epoch) {
+    epoch = 0;
+    if (p.carry_mode && threadIdx.x < 32) epoch = ld_volatile_u32(p.header);
+    return blockIdx.x;
+}
 
 // Carry between the thread blocks of one cluster (rows that are exactly 2..8 tiles long: one
 // cluster per row, block rank = the tile's position in scan order inside the row).  Every block
@@ -964,33 +985,43 @@ __device__ __forceinline__ void tile_compute(Chunk<ALGO, TRUNC, ITEMS>& c, Vals<
             if (p.out1 != nullptr) store_f32<ITEMS, VEC>(p.out1, i0, nvalid, out1v);
         }
     }
-    // ---- per-tile sums of A and A^2, in a fixed order (deterministic), for the normalisation pass
+    // ---- per-tile statistics of A for the normalisation pass, in a fixed order (deterministic):
+    // the tile's sum, and its sum of squared deviations from the tile's own mean.  Squares are
+    // taken around the tile mean so that a mean far from zero does not swallow the variance in
+    // fp32 (sum A^2 - mean * sum A cancels catastrophically there).
     if constexpr (ALGO == kGaeStats) {
-        float s1 = 0.f, s2 = 0.f;
+        constexpr int TILE = THREADS * ITEMS;
+        float s1 = 0.f;
 #pragma unroll
-        for (int j = 0; j < ITEMS; ++j) {         // steps beyond the array hold A = 0
-            s1 += v.a[j];
-            s2 = fmaf(v.a[j], v.a[j], s2);
-        }
+        for (int j = 0; j < ITEMS; ++j) s1 += v.a[j];         // steps beyond the array hold A = 0
 #pragma unroll
-        for (int d = 16; d > 0; d >>= 1) {
-            s1 += __shfl_xor_sync(ALL, s1, d);
-            s2 += __shfl_xor_sync(ALL, s2, d);
-        }
+        for (int d = 16; d > 0; d >>= 1) s1 += __shfl_xor_sync(ALL, s1, d);
         __syncthreads();                           // the scan's use of sm.agg is over
-        if (lane == 0) sm.agg[buf][warp] = Pair{s1, s2};
+        if (lane == 0) sm.agg[buf][warp].a = s1;
         __syncthreads();
-        if (warp == 0) {
-            Pair w = (lane < NW) ? sm.agg[buf][lane] : Pair{0.f, 0.f};
+        float tile_sum = 0.f;
 #pragma unroll
-            for (int d = 16; d > 0; d >>= 1) {
-                w.a += __shfl_xor_sync(ALL, w.a, d);
-                w.b += __shfl_xor_sync(ALL, w.b, d);
-            }
-            if (lane == 0) {
-                p.stats[2 * s] = w.a;
-                p.stats[2 * s + 1] = w.b;
-            }
+        for (int w = 0; w < NW; ++w) tile_sum += sm.agg[buf][w].a;      // same order in every thread
+        const long long tile_start = i0 - (long long)tid * ITEMS;
+        const long long left = p.total - tile_start;
+        const float count = (float)(left < TILE ? left : TILE);
+        const float mean = tile_sum / count;
+        float q = 0.f;
+#pragma unroll
+        for (int j = 0; j < ITEMS; ++j) {
+            const float d = v.a[j] - mean;
+            q = (j < nvalid) ? fmaf(d, d, q) : q;
+        }
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) q += __shfl_xor_sync(ALL, q, d);
+        if (lane == 0) sm.agg[buf][warp].b = q;
+        __syncthreads();
+        if (tid == 0) {
+            float tile_q = 0.f;
+#pragma unroll
+            for (int w = 0; w < NW; ++w) tile_q += sm.agg[buf][w].b;
+            p.stats[2 * s] = tile_sum;
+            p.stats[2 * s + 1] = tile_q;
         }
     }
     if constexpr (CLUSTER) cluster_exit_wait();
@@ -1021,13 +1052,11 @@ __global__ void __launch_bounds__(THREADS, MIN_BLOCKS) scan_kernel(const ScanPar
     constexpr int TILE = THREADS * ITEMS;
     __shared__ ScanSmem<THREADS / 32> sm;
 
-    const int tid = threadIdx.x;
-    const int lane = tid & 31;
-    const long long s = blockIdx.x;                       // tile index in scan order
+    grid_dependency_launch();
+    grid_dependency_wait();
+    unsigned epoch;
+    const long long s = take_tile(p, epoch);          // tile index in scan order
     const long long tile = FWD ? s : (p.num_tiles - 1 - s);
-
-    unsigned epoch = 0;
-    if (p.carry_mode && tid < 32) epoch = ld_volatile_u32(p.header);
     // block-uniform: the whole tile is inside the array and no row is shorter than a chunk
     const bool full = (tile * TILE + TILE <= p.total) && (p.T >= (unsigned)ITEMS);
     if (full) one_tile<ALGO, TRUNC, VEC, THREADS, ITEMS, true>(p, tile, s, epoch, sm);
@@ -1085,11 +1114,11 @@ template <bool TRUNC, bool VEC, int THREADS, int ITEMS, int MIN_BLOCKS>
 __global__ void __launch_bounds__(THREADS, MIN_BLOCKS) scan_kernel_gae_skip(const ScanParams p) {
     constexpr int TILE = THREADS * ITEMS;
     __shared__ ScanSmem<THREADS / 32> sm;
-    const int tid = threadIdx.x;
-    const long long s = blockIdx.x;
+    grid_dependency_launch();
+    grid_dependency_wait();
+    unsigned epoch;
+    const long long s = take_tile(p, epoch);
     const long long tile = p.num_tiles - 1 - s;
-    unsigned epoch = 0;
-    if (p.carry_mode && tid < 32) epoch = ld_volatile_u32(p.header);
     const bool full = (tile * TILE + TILE <= p.total) && (p.T >= (unsigned)ITEMS);
     if (full) one_tile_gae_skip<TRUNC, VEC, THREADS, ITEMS, true>(p, tile, s, epoch, sm);
     else one_tile_gae_skip<TRUNC, VEC, THREADS, ITEMS, false>(p, tile, s, epoch, sm);
@@ -1120,10 +1149,11 @@ template <bool TRUNC, bool VEC, int THREADS, int ITEMS, int MIN_BLOCKS, int AV>
 __global__ void __launch_bounds__(THREADS, MIN_BLOCKS) scan_kernel_retrace_probs(const ScanParams p) {
     constexpr int TILE = THREADS * ITEMS;
     __shared__ ScanSmem<THREADS / 32> sm;
-    const long long s = blockIdx.x;
+    grid_dependency_launch();
+    grid_dependency_wait();
+    unsigned epoch;
+    const long long s = take_tile(p, epoch);
     const long long tile = p.num_tiles - 1 - s;
-    unsigned epoch = 0;
-    if (p.carry_mode && threadIdx.x < 32) epoch = ld_volatile_u32(p.header);
     const bool full = (tile * TILE + TILE <= p.total) && (p.T >= (unsigned)ITEMS);      // block-uniform
     if (full) one_tile_probs<TRUNC, VEC, THREADS, ITEMS, AV, true>(p, tile, s, epoch, sm);
     else one_tile_probs<TRUNC, VEC, THREADS, ITEMS, AV, false>(p, tile, s, epoch, sm);
@@ -1143,9 +1173,11 @@ __global__ void __launch_bounds__(THREADS, MIN_BLOCKS) scan_kernel_cluster(const
     const int lane = tid & 31;
     const long long s = blockIdx.x;
     const long long tile = FWD ? s : (p.num_tiles - 1 - s);
+    grid_dependency_launch();
     Chunk<ALGO, TRUNC, ITEMS> c;
     const long long i0 = tile * TILE + (long long)tid * ITEMS;
     const long long n0 = locate(c, p, i0);
+    grid_dependency_wait();
     load_flags_global<ALGO, TRUNC, ITEMS, true, true>(c, p, i0, lane);
     Vals<ITEMS> v;
     load_values_global<ALGO, TRUNC, ITEMS, true, true>(c, v, p, i0, lane);
@@ -1401,7 +1433,9 @@ __global__ void __launch_bounds__(THREADS, MIN_BLOCKS) scan_kernel_tma(const Sca
         fence_barrier_init();
         fence_proxy_async();
     }
+    grid_dependency_launch();
     __syncthreads();
+    grid_dependency_wait();
     if (tid == 0) {
 #pragma unroll
         for (int k = 0; k < STAGES; ++k) produce_next<ALGO, TRUNC, TILE, STAGES>(p, w, ring, full_bar);

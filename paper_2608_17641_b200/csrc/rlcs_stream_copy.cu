@@ -8,11 +8,17 @@
 #include "../../include/rlcs.h"
 #include "rlcs_scan.cuh"
 
+namespace rlcs_hooks {
+extern bool g_pdl;
+}
+
 namespace {
 
 __global__ void __launch_bounds__(256) stream_copy_kernel(const float* __restrict__ src, float* __restrict__ dst,
                                                           long long read_pieces, long long write_pieces) {
     const long long c = (long long)blockIdx.x * 256 + threadIdx.x;
+    rlcs::grid_dependency_launch();      // launched like the scan kernels (see rlcs_scan.cuh), so that it is a fair ceiling
+    rlcs::grid_dependency_wait();
     float v[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
     if (c < read_pieces) rlcs::ldg_v8(src + 8 * c, v);
     if (c < write_pieces) {
@@ -35,6 +41,14 @@ extern "C" int rlcs_debug_stream_copy(const float* src, float* dst, size_t read_
     const long long n = rp > wp ? rp : wp;
     if (n == 0) return RLCS_OK;
     if (n > (1ll << 31) * 256 - 256) return RLCS_ERR_SIZE;
-    stream_copy_kernel<<<(unsigned)((n + 255) / 256), 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(src, dst, rp, wp);
-    return cudaGetLastError() == cudaSuccess ? RLCS_OK : RLCS_ERR_CUDA;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)((n + 255) / 256), 1, 1);
+    cfg.blockDim = dim3(256, 1, 1);
+    cfg.stream = static_cast<cudaStream_t>(cuda_stream);
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = rlcs_hooks::g_pdl ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, stream_copy_kernel, src, dst, rp, wp) == cudaSuccess ? RLCS_OK : RLCS_ERR_CUDA;
 }

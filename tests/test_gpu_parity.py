@@ -141,6 +141,8 @@ def test_shape_matrix(oracle, W, B, N, T, p_flag):
 @pytest.mark.parametrize("variant", list(range(21)))
 @pytest.mark.parametrize("N,T", [(5, 700), (4097, 3), (2, 9000), (64, 513)])
 def test_tile_variants(oracle, W, B, variant, N, T):
+    if not B.rlcs_debug_variant_built(variant):
+        pytest.skip("tile variant not in this build (python -m paper_2608_17641_b200.build --all-variants compiles it)")
     B.rlcs_debug_set_tile_variant(variant)
     try:
         ro = W.make_rollout(91, N, T, p_done=0.01, p_trunc=0.005, salt=T)
@@ -177,6 +179,8 @@ def test_randomized_shapes_flags_and_options(oracle, W, B):
         ro.params.update(gamma=float(rng.choice([0.9, 0.99, 1.0])), lam=float(rng.choice([0.0, 0.5, 0.95, 1.0])),
                          rho_bar=float(rng.choice([0.5, 1.0, 2.0])), c_bar=float(rng.choice([0.5, 1.0])))
         variant = int(rng.choice([BASE_VARIANT, int(rng.integers(0, n_variants))]))
+        if variant >= 0 and not B.rlcs_debug_variant_built(variant):
+            variant = BASE_VARIANT
         B.rlcs_debug_set_tile_variant(variant)
         try:
             compare_all(oracle, ro, offset=int(rng.choice([0, 0, 0, 1, 4, 8])),
@@ -277,7 +281,8 @@ def test_large_problem_variants_with_carry(oracle, W, B):
     compare_all(oracle, ro)
 
 
-@pytest.mark.parametrize("N,T,variant", [(5, 4096, 0), (3, 16384, 0), (64, 2048, 6), (7, 8192, 6), (9, 3072, 3), (2, 32768, 7)])
+@pytest.mark.parametrize("N,T,variant", [(5, 4096, 0), (3, 16384, 0), (64, 2048, 6), (7, 8192, 6), (9, 3072, 6), (2, 16384, 5),
+                                              (3, 4096, 19)])
 def test_cluster_carry_for_rows_of_whole_tiles(oracle, W, B, N, T, variant):
     """Rows of exactly 2..8 tiles: one thread-block cluster per row, carry in distributed shared
     memory and no workspace.  Against the oracle and against the workspace look-back."""
@@ -425,6 +430,35 @@ def test_gae_normalized(oracle, W, B, N, T, ddof):
     adv2, _ = B.rlcs_gae_normalized(dev.rewards, dev.values, dev.dones, None, None, dev.bootstrap, gamma=p["gamma"],
                                     lam=p["lam"], eps=1e-8, ddof=ddof, workspace=ws)
     assert np.array_equal(adv2.cpu().numpy(), adv.cpu().numpy())
+
+
+def test_gae_normalized_with_a_mean_far_from_zero(oracle, W, B):
+    """Rewards ~ N(100, 0.1^2), small values, lambda = 0.1, no flags: every advantage is close to
+    100 with a spread of about 0.1, so |mean| is a thousand times the standard deviation -- the case
+    in which single-precision sums of squares (sum A^2 - mean * sum A) lose the variance."""
+    N, T, g, lam = 64, 1000, 0.99, 0.1
+    ro = W.make_rollout(113, N, T, p_done=0.0, p_trunc=0.0, gamma=g, lam=lam)
+    ro.rewards = (100.0 + 0.1 * ro.rewards).astype(np.float32)
+    ro.values = (0.01 * ro.values).astype(np.float32)
+    dev = Dev(ro)
+    ws = B.Workspace(N, T, nbytes=B.lib().rlcs_gae_normalized_workspace_bytes(N, T))
+    for ddof in (0, 1):
+        adv, _ = B.rlcs_gae_normalized(dev.rewards, dev.values, dev.dones, None, None, None, gamma=g, lam=lam,
+                                       eps=1e-8, ddof=ddof, workspace=ws)
+        raw, _ = B.rlcs_gae(dev.rewards, dev.values, dev.dones, None, None, None, gamma=g, lam=lam, workspace=B.Workspace(N, T))
+        ref_adv, _ = oracle.gae_normalized(ro.rewards, ro.values, ro.dones, None, None, None, gamma=g, lam=lam, eps=1e-8, ddof=ddof)
+        got = adv.cpu().numpy().astype(np.float64)
+        assert np.isfinite(got).all()
+        # against the fp64 statistics of the GPU's own raw advantages: what is left is the rounding of
+        # the mean to fp32 (half an ulp of 100, divided by the spread) and of the rescale itself
+        a = raw.cpu().numpy().astype(np.float64)
+        mean, std = a.mean(), a.std(ddof=ddof)
+        cond = np.abs(a).max() / std
+        assert cond > 200, cond
+        np.testing.assert_allclose(got, (a - mean) / (std + 1e-8), rtol=1e-5, atol=2e-4)
+        # and against the oracle: an fp32 rounding error of A is magnified by 1/std in the normalised value
+        err = np.abs(got - ref_adv)
+        assert err.max() <= 1e-4 + 1e-5 * np.abs(ref_adv).max() + 8 * 6e-8 * cond, (err.max(), cond)
 
 
 def test_gae_normalized_argument_checks(oracle, W, B):

@@ -31,13 +31,15 @@ def test_no_alloc_entry_matches_workspace_entry_twice(oracle):
         ret.fill_(float("nan"))
         torch.cuda.synchronize()
         # the point of the entry point: with the outputs provided, the call takes no device memory --
-        # neither from torch's caching allocator nor from the driver (free bytes as cudaMemGetInfo
-        # reports them; the first call on a device only looks up the built-in array's address)
-        held, reserved, free = torch.cuda.memory_allocated(), torch.cuda.memory_reserved(), torch.cuda.mem_get_info()[0]
+        # neither from torch's caching allocator (its counters of allocation requests and of segments
+        # obtained from the driver) nor from the driver directly (free bytes as cudaMemGetInfo reports
+        # them; the first call on a device only looks up the built-in array's address)
+        count = lambda: tuple(torch.cuda.memory_stats().get(k, 0) for k in ("allocation.all.allocated", "segment.all.allocated"))
+        before, free = count(), torch.cuda.mem_get_info()[0]
         B.rlcs_gae_no_alloc(dev.rewards, dev.values, dev.dones, dev.truncs, dev.trunc_bootstrap, dev.bootstrap,
                             gamma=p["gamma"], lam=p["lam"], advantages=adv, returns=ret)
         torch.cuda.synchronize()
-        assert torch.cuda.memory_allocated() == held and torch.cuda.memory_reserved() == reserved, f"call {call} allocated"
+        assert count() == before, f"call {call} allocated device memory"
         if call == 1:
             assert torch.cuda.mem_get_info()[0] == free, "second call changed the driver's free memory"
         assert B.rlcs_no_alloc_last_device_status() == B.RLCS_OK
