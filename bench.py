@@ -303,34 +303,39 @@ class GpuBatch:
 
 def time_device(batch: GpuBatch, steps: int, warmup: int, dist):
     """K timed steps with inputs resident in HBM.  Per-kernel durations come from CUDA events on the
-    launching stream inside the timed region: every step brackets ONE of its seven launches (step k
-    the launch k mod 7), so each kernel is sampled about K/7 times while the other six launches of
-    a step run back to back as a caller would issue them -- an event between every pair of launches
-    costs several per cent of a step by itself.  When K < 7 the kernels that the timed region did not
-    reach are sampled in extra, untimed steps."""
+    launching stream inside the timed region: every step but the first brackets ONE of its seven
+    launches (step k the launch (k-1) mod 7), so each kernel is sampled about K/7 times while the other
+    six launches of a step run back to back as a caller would issue them -- an event between every pair
+    of launches costs several per cent of a step by itself.  The first step brackets nothing: the
+    stream is empty when the region starts, so an event recorded there would also time the host's
+    launch latency.  Kernels that the timed region did not reach (K < 8) are sampled in extra, untimed
+    steps.  The per-kernel figure is the median of its samples; a bracketed launch overlaps neither
+    the kernel before it nor the one after it, so the figure includes its whole ramp-up and tail."""
     torch = batch.torch
     for _ in range(warmup):
         batch.step()
     n = len(ALGOS)
-    extra = max(0, n - steps)
+    extra = max(0, n + 1 - steps)
     ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps + extra)]
     start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    which = lambda k: (k - 1) % n if k > 0 else None
     dist.barrier()
     torch.cuda.synchronize()
     launches0 = batch.launches
     with ClockSampler(torch.cuda.current_device()) as clk:
         start.record()
         for k in range(steps):
-            batch.step(k % n, ev[k])
+            batch.step(which(k), ev[k])
         stop.record()
         torch.cuda.synchronize()
     dist.barrier()
     launches = batch.launches - launches0
     for k in range(steps, steps + extra):
-        batch.step(k % n, ev[k])
+        batch.step(which(k), ev[k])
     torch.cuda.synchronize()
     total_ms = start.elapsed_time(stop)
-    per_algo_ms = {a: [ev[k][0].elapsed_time(ev[k][1]) for k in range(steps + extra) if k % n == j] for j, a in enumerate(ALGOS)}
+    per_algo_ms = {a: [ev[k][0].elapsed_time(ev[k][1]) for k in range(1, steps + extra) if which(k) == j]
+                   for j, a in enumerate(ALGOS)}
     assert batch.ws.device_status() == 0, "device reported a carry-wait timeout"
     return total_ms, per_algo_ms, launches, clk.summary()
 
@@ -710,7 +715,7 @@ def reference_arm(args, world: int):
 
 
 # --------------------------------------------------------------------------------------------- sweeps (cold L2)
-def sweep_case(torch, B, ro, algo: str, use_truncs: bool, hbm_peak: float, l2_bytes: int, trials=5):
+def sweep_case(torch, B, ro, algo: str, use_truncs: bool, hbm_peak: float, l2_bytes: int, trials=5, ceilings=True):
     """Device time per call with a cold L2: the calls of one batch rotate over R distinct copies of
     all inputs and outputs whose total footprint exceeds 3x the L2 capacity."""
     ro_eff = ro if use_truncs else _without_truncs(ro)
@@ -749,6 +754,11 @@ def sweep_case(torch, B, ro, algo: str, use_truncs: bool, hbm_peak: float, l2_by
     best = min(per_call_us)
     gbs = algo_bytes / (best * 1e-6) / 1e9
     del sets, graph
+    if not ceilings:
+        return {"algo": algo, "N": ro.N, "T": ro.T, "truncs": use_truncs, "us_per_call": round(best, 3),
+                "us_per_call_median": round(statistics.median(per_call_us), 3), "algorithmic_bytes": algo_bytes,
+                "gbs": round(gbs, 1), "frac_of_peak": round(gbs / hbm_peak, 4), "rotating_sets": R,
+                "timing": "CUDA-graph replay of launches rotating over buffer sets > 3x L2"}
     ceiling_us = copy_ceiling_us(torch, B, ro_eff, algo, algo_bytes, R, trials)
     ceiling_gbs = algo_bytes / (ceiling_us * 1e-6) / 1e9
     memcpy_us = memcpy_ceiling_us(torch, algo_bytes, R, trials)
@@ -890,6 +900,7 @@ def main():
     ap.add_argument("--variant", type=int, default=None, help="tile variant test hook (default: library default)")
     ap.add_argument("--no-dependent-launch", action="store_true",
                     help="measurement hook: launch the scan kernels without programmatic stream serialisation")
+    ap.add_argument("--no-row-tiles", action="store_true", help="measurement hook: no row-aligned tiling (short rows use the look-back)")
     ap.add_argument("--no-truncs", action="store_true", help="bench batch without per-step truncation handling")
     ap.add_argument("--rows", type=int, default=WORKLOAD["N"], help="num_envs of the bench batch (default: full size)")
     ap.add_argument("--only", choices=("time_major", "bf16", "retrace_probs", "elig_trace_vec", "elig_trace_vec_beta",
@@ -930,6 +941,8 @@ def main():
         binding.rlcs_debug_set_tile_variant(args.variant)
     if args.no_dependent_launch:
         binding.rlcs_debug_set_dependent_launch(False)
+    if args.no_row_tiles:
+        binding.rlcs_debug_allow_row_tiles(False)
     assert torch.cuda.is_available(), "bench.py needs a CUDA device"
     local = int(os.environ.get("LOCAL_RANK", "0"))
     torch.cuda.set_device(local)
@@ -981,7 +994,7 @@ def main():
     peak, peak_kind = measured_peak()
     per_algo = {}
     for a in ALGOS:
-        ms = statistics.mean(per_algo_ms[a])
+        ms = statistics.median(per_algo_ms[a])
         ab = algorithmic_bytes(ro, a)
         gbs = ab / (ms * 1e-3) / 1e9
         per_algo[a] = {"ms": round(ms, 5), "env_steps_per_s": ro.N * ro.T / (ms * 1e-3), "algorithmic_bytes": ab,
@@ -1035,6 +1048,12 @@ def main():
             ext("time_major", time_time_major(torch, binding, k20, peak, *shape))
         torch.cuda.empty_cache()
         ext("bf16", time_bf16(torch, binding, k20, peak, WORKLOAD["N"], WORKLOAD["T"]))
+        torch.cuda.empty_cache()
+        # the seven kernels of the headline workload launched back to back (no event between launches):
+        # what each sustains when its ramp-up and tail overlap its neighbours', as they do in a step
+        l2 = torch.cuda.get_device_properties(0).L2_cache_size
+        details += [{"detail": "back_to_back", **sweep_case(torch, binding, ro, a, ro.truncs is not None, peak, l2, trials=3, ceilings=False)}
+                    for a in ALGOS]
         torch.cuda.empty_cache()
         sweeps = run_sweeps(torch, peak)
         details += [{"detail": "sweep", **c} for c in sweeps]

@@ -36,7 +36,11 @@
  * Alignment.  fp32 pointers must be 4-byte aligned.  When every fp32 pointer is 32-byte aligned
  *   and every mask pointer 16-byte aligned the vectorised kernels run (256-bit accesses, bulk
  *   copies); otherwise a slower element-wise variant of the same kernel is used (same results).
- * Workspace.  Rows that straddle the kernels' tiles need a carry between thread blocks, passed
+ * Workspace.  The kernels cut the flattened [N*T] array into tiles of 512 to 2048 steps, one per
+ *   thread block.  When T divides the tile, or a whole number of rows nearly fills it (at least 70 %,
+ *   with every thread still holding a whole chunk: T = 1000, 2000, 500, 250, 200, 100, ...), tiles
+ *   are aligned to rows and blocks are independent.  Otherwise rows straddle tiles and need a carry
+ *   between thread blocks, passed
  *   through `workspace`: at least rlcs_workspace_bytes(N, T) bytes, 16-byte aligned, initialised
  *   once with rlcs_workspace_init and then reusable by any number of calls, of any of the entry
  *   points, that are ordered on one stream.  Two calls that may run concurrently need two
@@ -426,6 +430,11 @@ int rlcs_debug_variant_for(int algorithm, int has_truncs, int64_t N, int64_t T);
 /* Shape of a variant: threads per block, steps per thread, blocks per SM it is compiled for, and
  * ring stages (0 = the one-tile-per-block kernel).  Any output pointer may be NULL. */
 int rlcs_debug_variant_info(int variant, int* threads, int* steps_per_thread, int* blocks_per_sm, int* ring_stages);
+
+/* Test / measurement hook: 0 turns row-aligned tiling off (see "Workspace" above: rows shorter than a
+ * tile that do not divide it are then carried between thread blocks through the workspace, as rows
+ * longer than a tile always are), 1 (default) allows it.  Results agree to rounding. */
+int rlcs_debug_allow_row_tiles(int on);
 
 /* Test / measurement hook: 0 launches the row-major scan kernels without programmatic stream
  * serialisation (see "Execution" above), 1 (default) with it.  Results are identical. */

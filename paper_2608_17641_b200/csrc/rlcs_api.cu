@@ -9,6 +9,7 @@ bool g_wide_index = false;
 long long g_mute_tile = -1;
 long long g_spin_cap = 0;
 bool g_pdl = true;
+bool g_row_tiles = true;
 }  // namespace rlcs_hooks
 
 extern "C" {
@@ -111,7 +112,7 @@ int rlcs_gae_skip(const float* rewards, const float* values, const uint8_t* done
     // its own carry records.  These tile shapes have at least 1024 steps, so two records per tile still
     // fit the workspace of rlcs_workspace_bytes (sized for 512-step tiles).  No cluster carry here.
     const int variant = choose_variant(rlcs::kGaeSkip, truncs != nullptr, total, T);
-    st = finish_params(p, variant, total, T, workspace, workspace_bytes, vec, false, 2);
+    st = finish_params(p, variant, total, T, workspace, workspace_bytes, vec, false, 2, false);
     if (st != RLCS_OK) return st;
     return run(rlcs::launch_gae_skip, p, variant, truncs != nullptr, vec, cuda_stream);
 }
@@ -154,7 +155,7 @@ int rlcs_gae_normalized(const float* rewards, const float* values, const uint8_t
     st = run(rlcs::launch_gae_stats, p, variant, truncs != nullptr, vec, cuda_stream);
     if (st != RLCS_OK) return st;
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
-    if (rlcs::launch_norm_finalize(p.stats, p.num_tiles, total, tile_elems(variant), ddof, eps, mean_rstd, s) != cudaSuccess) return RLCS_ERR_CUDA;
+    if (rlcs::launch_norm_finalize(p.stats, p.num_tiles, total, (int)p.tile_steps, ddof, eps, mean_rstd, s) != cudaSuccess) return RLCS_ERR_CUDA;
     if (rlcs::launch_norm_rescale(advantages, total, mean_rstd, vec, s) != cudaSuccess) return RLCS_ERR_CUDA;
     return RLCS_OK;
 }
@@ -226,7 +227,7 @@ int rlcs_retrace_probs(const float* rewards, const float* q_values, const float*
     constexpr int kVariant = 3;      // 256 threads x 4 steps, the tile rlcs_retrace_probs.cu instantiates
     static_assert(rlcs::kVariants[kVariant].threads == rlcs::kRetraceProbsThreads &&
                   rlcs::kVariants[kVariant].items == rlcs::kRetraceProbsItems, "tile shape mismatch");
-    st = finish_params(p, kVariant, total, T, workspace, workspace_bytes, vec, false);
+    st = finish_params(p, kVariant, total, T, workspace, workspace_bytes, vec, false, 1, false);
     if (st != RLCS_OK) return st;
     return rlcs::launch_retrace_probs(p, truncs != nullptr, vec, vec_rows, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess
                ? RLCS_OK : RLCS_ERR_CUDA;
@@ -350,6 +351,11 @@ int rlcs_debug_variant_info(int variant, int* threads, int* steps_per_thread, in
     if (steps_per_thread) *steps_per_thread = tv.items;
     if (blocks_per_sm) *blocks_per_sm = tv.min_blocks;
     if (ring_stages) *ring_stages = tv.stages;
+    return RLCS_OK;
+}
+
+int rlcs_debug_allow_row_tiles(int on) {
+    rlcs_hooks::g_row_tiles = on != 0;
     return RLCS_OK;
 }
 

@@ -17,6 +17,7 @@
 #include <cstdint>
 
 #include "../../include/rlcs.h"
+#include "rlcs_device.cuh"
 #include "rlcs_scan.cuh"
 
 // the time-major block kernel, one [T, D] problem per row (rlcs_time_major.cu)
@@ -181,7 +182,7 @@ inline bool aligned(const void* p, uintptr_t a) { return (reinterpret_cast<uintp
 // 2048x512x64; 16 steps: 0.76); only when that is not enough is the time axis cut -- into chunks of
 // at least 128 steps and at most 256 per row, so that the ordered carry chain stays short.
 void plan(long long N, long long T, long long groups, bool perdim, unsigned* chunk, unsigned* chunks, unsigned* batch) {
-    const long long want = 148ll * 256 * kBatch;
+    const long long want = rlcs_device::limits().sms * 256 * kBatch;
     const long long threads = N * groups;
     unsigned kb = kBatch;
     // (with a decay tensor the deeper batches measured slower: 0.87 -> 0.58 -> 0.38 at 16384x128x64)
@@ -204,7 +205,7 @@ template <int V, bool PERDIM, int KB>
 int run_batch(const VecParams& p, cudaStream_t s) {
     const long long threads = p.N * (long long)p.groups * p.chunks;
     // few threads: smaller blocks, so that they spread over all SMs
-    const unsigned bt = threads < 148ll * kThreads * 2 ? 64 : kThreads;
+    const unsigned bt = threads < rlcs_device::limits().sms * kThreads * 2 ? 64 : kThreads;
     const unsigned blocks = (unsigned)((threads + bt - 1) / bt);
     if (p.chunks == 1) {
         elig_vec_kernel<V, 0, PERDIM, KB><<<blocks, bt, 0, s>>>(p);

@@ -16,6 +16,7 @@ extern bool g_cluster;             // allow the cluster carry
 extern bool g_wide_index;          // use the 64-bit index path even when 32 bits would do
 extern long long g_mute_tile;      // tile that does not publish
 extern long long g_spin_cap;       // poll limit (0 = default)
+extern bool g_row_tiles;           // allow row-aligned tiling (default on)
 }  // namespace rlcs_hooks
 
 namespace {
@@ -120,12 +121,37 @@ struct CarryPlan {
     int carry_mode;      // rows straddle tiles: tile records in the workspace, look-back
     int cluster;         // > 1: one thread-block cluster of this many tiles per row, no workspace
     size_t bytes;        // workspace bytes this call reads or writes (0 when it needs none)
+    int tile_steps;      // steps per thread block: the tile, or less with row-aligned tiling
 };
 
-CarryPlan plan_carry(int variant, int64_t total, int64_t T, bool vec, bool allow_cluster, int records_per_tile) {
+// Row-aligned tiling: when rows are shorter than a tile but do not divide it, a block can take the
+// largest whole number of rows that fits (k*T steps) instead of a full tile, provided every thread
+// still gets either a whole chunk or nothing (k*T a multiple of the steps per thread) and few
+// threads idle (at least 70 % of the tile used).  No row straddles a tile then, so there is no
+// carry between blocks at all: no workspace traffic, no waiting on other blocks.  T = 1000 on
+// 1024-step tiles idles 3 threads of 128; T = 2000, 500, 250, 200, 100 fit 2048-step tiles the same way.
+int row_aligned_steps(int variant, int64_t T) {
+    const int tile = tile_elems(variant), items = RLCS_NS::kVariants[variant].items;
+    if (!rlcs_hooks::g_row_tiles || RLCS_NS::kVariants[variant].stages != 0 || T > tile || tile % T == 0) return 0;
+    if (T < items) return 0;
+    for (int64_t rows = tile / T; rows * T * 10 >= (int64_t)tile * 7; --rows)      // fewer rows if the most that fit do not split into whole chunks
+        if ((rows * T) % items == 0) return (int)(rows * T);
+    return 0;
+}
+
+CarryPlan plan_carry(int variant, int64_t total, int64_t T, bool vec, bool allow_cluster, int records_per_tile,
+                     bool allow_row_tiles = true) {
     const int tile = tile_elems(variant);
     const int64_t num_tiles = (total + tile - 1) / tile;
-    CarryPlan plan = {(tile % T) != 0 ? 1 : 0, 0, 0};       // T does not divide the tile: rows straddle tiles
+    CarryPlan plan = {(tile % T) != 0 ? 1 : 0, 0, 0, tile};       // T does not divide the tile: rows straddle tiles
+    if (plan.carry_mode && allow_row_tiles) {
+        const int steps = row_aligned_steps(variant, T);
+        if (steps > 0) {
+            plan.carry_mode = 0;
+            plan.tile_steps = steps;
+            return plan;
+        }
+    }
     // Rows of exactly 2..8 tiles: one thread-block cluster per row carries through distributed
     // shared memory instead (needs the vectorised one-tile kernel; g_cluster = 0 turns it off).
     if (allow_cluster && g_cluster && vec && RLCS_NS::kVariants[variant].stages == 0 && T % tile == 0 && T / tile >= 2 &&
@@ -140,11 +166,13 @@ CarryPlan plan_carry(int variant, int64_t total, int64_t T, bool vec, bool allow
 
 // Fill the size / tiling / carry fields and validate the workspace for this call.
 int finish_params(ScanParams& p, int variant, int64_t total, int64_t T, void* workspace, size_t workspace_bytes, bool vec,
-                  bool allow_cluster = true, int records_per_tile = 1) {
+                  bool allow_cluster = true, int records_per_tile = 1, bool allow_row_tiles = true) {
     const int tile = tile_elems(variant);
+    const CarryPlan plan = plan_carry(variant, total, T, vec, allow_cluster, records_per_tile, allow_row_tiles);
     p.total = total;
     p.T = (unsigned)T;
-    p.num_tiles = (total + tile - 1) / tile;
+    p.tile_steps = (unsigned)plan.tile_steps;
+    p.num_tiles = (total + plan.tile_steps - 1) / plan.tile_steps;
     p.idx32 = !g_wide_index && (total + tile) <= 0xffffffffLL;
     {   // invariant division by T (see FastDiv)
         int l = 0;
@@ -155,7 +183,6 @@ int finish_params(ScanParams& p, int variant, int64_t total, int64_t T, void* wo
     }
     p.decay_pow = 1.f;                       // beta product of a chunk without resets
     for (int i = 0; i < RLCS_NS::kVariants[variant].items; ++i) p.decay_pow *= p.decay;
-    const CarryPlan plan = plan_carry(variant, total, T, vec, allow_cluster, records_per_tile);
     p.carry_mode = plan.carry_mode;
     p.cluster = plan.cluster;
     p.header = nullptr;

@@ -109,6 +109,8 @@ struct ScanParams {
     float* stats;             // kGaeStats: per scan-order tile {sum A, sum (A - tile mean)^2}
     long long total;          // N*T
     long long num_tiles;
+    unsigned tile_steps;      // steps a thread block covers: THREADS*ITEMS, or a whole number of rows that is a little
+                              // less (row-aligned tiling: the last few threads idle, but no row straddles a tile)
     unsigned T;
     int idx32;                // total + tile fits in 32 bits: 32-bit row/time arithmetic
     FastDiv div_T;
@@ -171,8 +173,17 @@ __device__ __forceinline__ float ldg_if(const float* p, bool pred) {
     return v;
 }
 
-template <int ITEMS, bool VEC>
+// ALLORNONE (with VEC): the chunk is either whole or empty (an idle thread of a row-aligned tile),
+// so there is no element-wise path to compile.
+template <int ITEMS, bool VEC, bool ALLORNONE = false>
 __device__ __forceinline__ void load_f32(const float* __restrict__ p, long long i0, int nvalid, float (&x)[ITEMS]) {
+    if constexpr (VEC && ALLORNONE) {
+        if (nvalid != ITEMS) {
+#pragma unroll
+            for (int j = 0; j < ITEMS; ++j) x[j] = 0.f;
+            return;
+        }
+    }
     if (VEC && nvalid == ITEMS) {
         if constexpr (ITEMS % 8 == 0) {
 #pragma unroll
@@ -193,8 +204,15 @@ __device__ __forceinline__ void load_f32(const float* __restrict__ p, long long 
 
 // Mask bytes of ITEMS consecutive steps, packed 4 per word (byte j%4 of word j/4), values as stored
 // (any non-zero byte = true).
-template <int ITEMS, bool VEC>
+template <int ITEMS, bool VEC, bool ALLORNONE = false>
 __device__ __forceinline__ void load_mask(const uint8_t* __restrict__ p, long long i0, int nvalid, unsigned (&w)[ITEMS / 4]) {
+    if constexpr (VEC && ALLORNONE) {
+        if (nvalid != ITEMS) {
+#pragma unroll
+            for (int k = 0; k < ITEMS / 4; ++k) w[k] = 0;
+            return;
+        }
+    }
     if (VEC && nvalid == ITEMS) {
         if constexpr (ITEMS == 4) {
             w[0] = __ldcs(reinterpret_cast<const unsigned*>(p + i0));
@@ -255,8 +273,15 @@ __device__ __forceinline__ float ldg_if(const io_t* p, bool pred) {
     return __uint_as_float((unsigned)v << 16);
 }
 
-template <int ITEMS, bool VEC>
+template <int ITEMS, bool VEC, bool ALLORNONE = false>
 __device__ __forceinline__ void load_f32(const io_t* __restrict__ p, long long i0, int nvalid, float (&x)[ITEMS]) {
+    if constexpr (VEC && ALLORNONE) {
+        if (nvalid != ITEMS) {
+#pragma unroll
+            for (int j = 0; j < ITEMS; ++j) x[j] = 0.f;
+            return;
+        }
+    }
     if (VEC && nvalid == ITEMS) {
         unsigned w[ITEMS / 2];
         if constexpr (ITEMS == 16) {
@@ -477,8 +502,8 @@ struct Vals {
 // the row's last step (offset T-1-t0); for forward scans the next row's first step (offset T-t0, or
 // 0 when the chunk itself starts a row).
 template <int ALGO, bool TRUNC, int ITEMS>
-__device__ __forceinline__ long long locate(Chunk<ALGO, TRUNC, ITEMS>& c, const ScanParams& p, long long i0) {
-    const long long rem = p.total - i0;
+__device__ __forceinline__ long long locate(Chunk<ALGO, TRUNC, ITEMS>& c, const ScanParams& p, long long i0, long long end) {
+    const long long rem = end - i0;            // `end`: the array's end, or this tile's end when it comes first
     c.nvalid = rem >= ITEMS ? ITEMS : (rem > 0 ? (int)rem : 0);
     unsigned t0;
     long long n0;
@@ -495,6 +520,10 @@ __device__ __forceinline__ long long locate(Chunk<ALGO, TRUNC, ITEMS>& c, const 
     c.edge = is_forward(ALGO) ? (t0 == 0 ? 0u : p.T - t0) : (p.T - 1 - t0);
     return n0;               // the row of step i0
 }
+template <int ALGO, bool TRUNC, int ITEMS>
+__device__ __forceinline__ long long locate(Chunk<ALGO, TRUNC, ITEMS>& c, const ScanParams& p, long long i0) {
+    return locate(c, p, i0, p.total);
+}
 
 // Window-edge bootstrap of the first row edge inside the chunk (plain load, issued early).
 template <int ALGO, bool TRUNC, int ITEMS>
@@ -506,19 +535,20 @@ __device__ __forceinline__ void issue_boot(Chunk<ALGO, TRUNC, ITEMS>& c, const S
 }
 
 // Mask bytes from global memory; forward scans also need the dones byte just before the chunk.
-template <int ALGO, bool TRUNC, int ITEMS, bool VEC, bool FULL = false>
+// IDLE (with FULL): row-aligned tiling -- every thread of the block has a whole chunk or none at all.
+template <int ALGO, bool TRUNC, int ITEMS, bool VEC, bool FULL = false, bool IDLE = false>
 __device__ __forceinline__ void load_flags_global(Chunk<ALGO, TRUNC, ITEMS>& c, const ScanParams& p, long long i0, int lane) {
     constexpr int W = ITEMS / 4;
-    const int nvalid = FULL ? ITEMS : c.nvalid;
+    const int nvalid = (FULL && !IDLE) ? ITEMS : c.nvalid;
 #pragma unroll
     for (int k = 0; k < W; ++k) { c.dw[k] = 0; c.tw[k] = 0; }
     c.halo_d = 0;
     if constexpr (ALGO == kElig || ALGO == kPrefix) {
         if (lane == 0 && i0 > 0 && nvalid > 0) c.halo_d = __ldg(p.dones + i0 - 1);
     }
-    if constexpr (uses_dones(ALGO)) load_mask<ITEMS, VEC>(p.dones, i0, nvalid, c.dw);
-    if constexpr (TRUNC) load_mask<ITEMS, VEC>(p.truncs, i0, nvalid, c.tw);
-    if constexpr (uses_skip(ALGO)) load_mask<ITEMS, VEC>(p.skip, i0, nvalid, c.kw);
+    if constexpr (uses_dones(ALGO)) load_mask<ITEMS, VEC, IDLE>(p.dones, i0, nvalid, c.dw);
+    if constexpr (TRUNC) load_mask<ITEMS, VEC, IDLE>(p.truncs, i0, nvalid, c.tw);
+    if constexpr (uses_skip(ALGO)) load_mask<ITEMS, VEC, IDLE>(p.skip, i0, nvalid, c.kw);
     if constexpr (ALGO == kElig || ALGO == kPrefix) {
         const unsigned nb = __shfl_up_sync(0xffffffffu, c.dw[W - 1] >> 24, 1);
         if (lane != 0) c.halo_d = nb;
@@ -539,13 +569,13 @@ __device__ __forceinline__ void issue_trunc_values(Chunk<ALGO, TRUNC, ITEMS>& c,
 
 // Float inputs from global memory, with the one-step halo (lane 31 loads it, the others take
 // their neighbour's first element).
-template <int ALGO, bool TRUNC, int ITEMS, bool VEC, bool FULL = false>
+template <int ALGO, bool TRUNC, int ITEMS, bool VEC, bool FULL = false, bool IDLE = false>
 __device__ __forceinline__ void load_values_global(const Chunk<ALGO, TRUNC, ITEMS>& c, Vals<ITEMS>& v, const ScanParams& p, long long i0, int lane) {
-    const int nvalid = FULL ? ITEMS : c.nvalid;
-    load_f32<ITEMS, VEC>(p.f0, i0, nvalid, v.a);
-    if constexpr (uses_f1(ALGO)) load_f32<ITEMS, VEC>(p.f1, i0, nvalid, v.x1);
-    if constexpr (uses_f2(ALGO)) load_f32<ITEMS, VEC>(p.f2, i0, nvalid, v.x2);
-    if constexpr (uses_f3(ALGO)) load_f32<ITEMS, VEC>(p.f3, i0, nvalid, v.x3);
+    const int nvalid = (FULL && !IDLE) ? ITEMS : c.nvalid;
+    load_f32<ITEMS, VEC, IDLE>(p.f0, i0, nvalid, v.a);
+    if constexpr (uses_f1(ALGO)) load_f32<ITEMS, VEC, IDLE>(p.f1, i0, nvalid, v.x1);
+    if constexpr (uses_f2(ALGO)) load_f32<ITEMS, VEC, IDLE>(p.f2, i0, nvalid, v.x2);
+    if constexpr (uses_f3(ALGO)) load_f32<ITEMS, VEC, IDLE>(p.f3, i0, nvalid, v.x3);
     v.halo = 0.f;
     v.halo_lr = 0.f;
     if constexpr (float_halo(ALGO)) {
@@ -726,10 +756,13 @@ struct NoHook {
 // `after_barrier` runs right after the block barrier (every thread has consumed its inputs).
 // FULL: the tile lies completely inside the array and rows are at least ITEMS long (block-uniform),
 // which removes the ragged-chunk and short-row side paths at compile time.
+// IDLE (with FULL): row-aligned tiling -- the block's last threads may have no steps at all; they
+// read zeros, store nothing and take part in the scan as resets.
 // LAST: this is the block's last tile of the call; the block then signs off from the carry protocol
 // as soon as its own look-back is over (see sign_off) instead of after its stores.
 // CLUSTER: the carry between blocks goes through distributed shared memory (cluster_carry).
-template <int ALGO, bool TRUNC, bool VEC, int THREADS, int ITEMS, bool FULL, bool LAST, class Hook, bool CLUSTER = false>
+template <int ALGO, bool TRUNC, bool VEC, int THREADS, int ITEMS, bool FULL, bool LAST, class Hook, bool CLUSTER = false,
+          bool IDLE = false>
 __device__ __forceinline__ void tile_compute(Chunk<ALGO, TRUNC, ITEMS>& c, Vals<ITEMS>& v, const ScanParams& p, long long i0, long long s,
                                              unsigned epoch, ScanSmem<THREADS / 32>& sm, int buf, Hook after_barrier,
                                              float* prev_out = nullptr) {
@@ -741,7 +774,8 @@ __device__ __forceinline__ void tile_compute(Chunk<ALGO, TRUNC, ITEMS>& c, Vals<
     const int lane = tid & 31;
     const int warp = tid >> 5;
     const bool has_edge = c.edge < (unsigned)ITEMS;
-    const int nvalid = FULL ? ITEMS : c.nvalid;
+    // IDLE (row-aligned tiling, with FULL): c.nvalid is ITEMS, or 0 for the block's idle last threads
+    const int nvalid = (FULL && !IDLE) ? ITEMS : c.nvalid;
 
     // ---- reset words: byte j non-zero = the recurrence does NOT continue from step j to its
     // scan-order predecessor (t+1 backward, t-1 forward): a flag, a row edge, a step beyond the array
@@ -764,6 +798,11 @@ __device__ __forceinline__ void tile_compute(Chunk<ALGO, TRUNC, ITEMS>& c, Vals<
         for (int k = 0; k < W; ++k) sev[k] = c.dw[k] | c.tw[k];
     }
     if (has_edge) mark_byte_dyn(sev, c.edge);
+    if constexpr (IDLE) {                       // an idle thread: all its steps are resets with alpha = 0 (its inputs read as zeros)
+        const unsigned idle = nvalid == 0 ? 0xffffffffu : 0u;
+#pragma unroll
+        for (int k = 0; k < W; ++k) sev[k] |= idle;
+    }
     if constexpr (!FULL) {
         if (p.T < (unsigned)ITEMS) {            // rows shorter than a chunk: several edges
             for (unsigned e = c.edge + p.T; e < (unsigned)ITEMS; e += p.T) mark_byte_dyn(sev, e);
@@ -990,7 +1029,6 @@ __device__ __forceinline__ void tile_compute(Chunk<ALGO, TRUNC, ITEMS>& c, Vals<
     // taken around the tile mean so that a mean far from zero does not swallow the variance in
     // fp32 (sum A^2 - mean * sum A cancels catastrophically there).
     if constexpr (ALGO == kGaeStats) {
-        constexpr int TILE = THREADS * ITEMS;
         float s1 = 0.f;
 #pragma unroll
         for (int j = 0; j < ITEMS; ++j) s1 += v.a[j];         // steps beyond the array hold A = 0
@@ -1004,7 +1042,7 @@ __device__ __forceinline__ void tile_compute(Chunk<ALGO, TRUNC, ITEMS>& c, Vals<
         for (int w = 0; w < NW; ++w) tile_sum += sm.agg[buf][w].a;      // same order in every thread
         const long long tile_start = i0 - (long long)tid * ITEMS;
         const long long left = p.total - tile_start;
-        const float count = (float)(left < TILE ? left : TILE);
+        const float count = (float)(left < (long long)p.tile_steps ? left : (long long)p.tile_steps);
         const float mean = tile_sum / count;
         float q = 0.f;
 #pragma unroll
@@ -1029,21 +1067,23 @@ __device__ __forceinline__ void tile_compute(Chunk<ALGO, TRUNC, ITEMS>& c, Vals<
 
 // ------------------------------------------------------------------------------------------ end of a call (carry mode)
 // ------------------------------------------------------------------------------------------ kernel 1: one tile per block
-template <int ALGO, bool TRUNC, bool VEC, int THREADS, int ITEMS, bool FULL>
+template <int ALGO, bool TRUNC, bool VEC, int THREADS, int ITEMS, bool FULL, bool IDLE = false>
 __device__ __forceinline__ void one_tile(const ScanParams& p, long long tile, long long s, unsigned epoch,
                                          ScanSmem<THREADS / 32>& sm) {
-    constexpr int TILE = THREADS * ITEMS;
     const int tid = threadIdx.x;
     const int lane = tid & 31;
     Chunk<ALGO, TRUNC, ITEMS> c;
-    const long long i0 = tile * TILE + (long long)tid * ITEMS;
-    const long long n0 = locate(c, p, i0);
-    load_flags_global<ALGO, TRUNC, ITEMS, VEC, FULL>(c, p, i0, lane);
+    // a tile covers p.tile_steps steps: THREADS*ITEMS, or (row-aligned tiling) a whole number of rows
+    // that is a little less, in which case the last threads of the block have nothing to do
+    const long long i0 = tile * p.tile_steps + (long long)tid * ITEMS;
+    const long long tile_end = (tile + 1) * p.tile_steps;
+    const long long n0 = locate(c, p, i0, tile_end < p.total ? tile_end : p.total);
+    load_flags_global<ALGO, TRUNC, ITEMS, VEC, FULL, IDLE>(c, p, i0, lane);
     Vals<ITEMS> v;
-    load_values_global<ALGO, TRUNC, ITEMS, VEC, FULL>(c, v, p, i0, lane);
+    load_values_global<ALGO, TRUNC, ITEMS, VEC, FULL, IDLE>(c, v, p, i0, lane);
     issue_boot(c, p, n0);
     issue_trunc_values(c, p, i0);
-    tile_compute<ALGO, TRUNC, VEC, THREADS, ITEMS, FULL, true>(c, v, p, i0, s, epoch, sm, 0, NoHook{});
+    tile_compute<ALGO, TRUNC, VEC, THREADS, ITEMS, FULL, true, NoHook, false, IDLE>(c, v, p, i0, s, epoch, sm, 0, NoHook{});
 }
 
 template <int ALGO, bool TRUNC, bool VEC, int THREADS, int ITEMS, int MIN_BLOCKS>
@@ -1057,10 +1097,20 @@ __global__ void __launch_bounds__(THREADS, MIN_BLOCKS) scan_kernel(const ScanPar
     unsigned epoch;
     const long long s = take_tile(p, epoch);          // tile index in scan order
     const long long tile = FWD ? s : (p.num_tiles - 1 - s);
-    // block-uniform: the whole tile is inside the array and no row is shorter than a chunk
-    const bool full = (tile * TILE + TILE <= p.total) && (p.T >= (unsigned)ITEMS);
-    if (full) one_tile<ALGO, TRUNC, VEC, THREADS, ITEMS, true>(p, tile, s, epoch, sm);
-    else one_tile<ALGO, TRUNC, VEC, THREADS, ITEMS, false>(p, tile, s, epoch, sm);
+    // block-uniform: every thread has a whole chunk (the tile is a full one inside the array) and no row is shorter than a chunk
+    const bool full = (p.tile_steps == (unsigned)TILE) && (tile * TILE + TILE <= p.total) && (p.T >= (unsigned)ITEMS);
+    if (full) {
+        one_tile<ALGO, TRUNC, VEC, THREADS, ITEMS, true>(p, tile, s, epoch, sm);
+        return;
+    }
+    if constexpr (VEC) {
+        // row-aligned tiling, tile inside the array: whole chunks in the first threads, none in the last few
+        if (p.tile_steps != (unsigned)TILE && (tile + 1) * (long long)p.tile_steps <= p.total && p.T >= (unsigned)ITEMS) {
+            one_tile<ALGO, TRUNC, VEC, THREADS, ITEMS, true, true>(p, tile, s, epoch, sm);
+            return;
+        }
+    }
+    one_tile<ALGO, TRUNC, VEC, THREADS, ITEMS, false>(p, tile, s, epoch, sm);
 }
 
 // ------------------------------------------------------------------------------------------ kernel 1b: GAE with observation-skip masking

@@ -31,6 +31,7 @@
 #include <type_traits>
 
 #include "../../include/rlcs.h"
+#include "rlcs_device.cuh"
 #include "rlcs_scan.cuh"
 
 // test hooks shared with the row-major entry points (rlcs_debug_set_carry_fault; defined in rlcs_api.cu)
@@ -949,8 +950,10 @@ __global__ void __launch_bounds__(kThreads) tm_chain_kernel(const TmParams p) {
 // Host side
 // ---------------------------------------------------------------------------------------------
 
-constexpr long long kSms = 148;
-constexpr size_t kSmemPerSm = 227 * 1024;        // usable by thread blocks; each resident block also costs 1 KB
+// SM count and shared memory per SM of the current device (usable by thread blocks; each resident
+// block also costs 1 KB), see rlcs_device.cuh
+inline long long sm_count() { return rlcs_device::limits().sms; }
+inline long long smem_per_sm() { return (long long)rlcs_device::limits().smem_per_sm; }
 
 // How the time axis is cut.  Depends on N and T only, so that the workspace size does.
 void plan_chunks(long long N, long long T, unsigned* chunk, unsigned* chunks) {
@@ -961,7 +964,7 @@ void plan_chunks(long long N, long long T, unsigned* chunk, unsigned* chunks) {
     *chunks = 1;
     const long long groups = (N + 31) / 32;
     if (groups >= 96) return;
-    const long long k = (2 * kSms + groups - 1) / groups;
+    const long long k = (2 * sm_count() + groups - 1) / groups;
     long long len = (T + k - 1) / k;
     if (len < 64) len = 64;
     len = (len + kRows - 1) / kRows * kRows;
@@ -978,9 +981,10 @@ void plan_chunks(long long N, long long T, unsigned* chunk, unsigned* chunks) {
 size_t plan_block(TmParams& p, int rows, int row_bytes, bool trunc, bool wide_ok) {
     int C = 1;
     const long long batch = p.batch > 0 ? p.batch : 1;
-    if (wide_ok && (p.N + 63) / 64 * p.chunks * batch >= 2 * kSms) C = 2;
+    if (wide_ok && (p.N + 63) / 64 * p.chunks * batch >= 2 * sm_count()) C = 2;
     const long long blocks = (p.N + 32 * C - 1) / (32 * C) * p.chunks * batch;
-    int W = C == 2 ? 4 : blocks < kSms ? 16 : blocks < 2 * kSms ? 8 : 4;
+    const long long sms = sm_count(), smem = smem_per_sm();
+    int W = C == 2 ? 4 : blocks < sms ? 16 : blocks < 2 * sms ? 8 : 4;
     long long stage, mstage, fixed;
     auto size = [&]() {
         stage = (long long)rows * W * row_bytes * C;
@@ -989,15 +993,15 @@ size_t plan_block(TmParams& p, int rows, int row_bytes, bool trunc, bool wide_ok
     };
     auto block_bytes = [&](long long S) { return S * stage + fixed; };
     size();
-    while (W > 4 && block_bytes(3) + 1024 > (long long)kSmemPerSm) { W /= 2; size(); }   // the minimum ring must fit
-    long long resident = (blocks + kSms - 1) / kSms;
+    while (W > 4 && block_bytes(3) + 1024 > smem) { W /= 2; size(); }   // the minimum ring must fit
+    long long resident = (blocks + sms - 1) / sms;
     if (resident > 6) resident = 6;
-    while (resident > 1 && resident * (block_bytes(3) + 1024) > (long long)kSmemPerSm) --resident;
+    while (resident > 1 && resident * (block_bytes(3) + 1024) > smem) --resident;
     long long S = 2 + ((16ll << 20) + blocks * stage - 1) / (blocks * stage);
     const long long nst = ((long long)p.chunk + rows * W - 1) / (rows * W);
     if (S > nst + 1) S = nst + 1;
     if (S > kMaxStages) S = kMaxStages;
-    while (S > 3 && resident * (block_bytes(S) + 1024) > (long long)kSmemPerSm) --S;
+    while (S > 3 && resident * (block_bytes(S) + 1024) > smem) --S;
     if (S < 3) S = 3;
     p.stages = (int)S;
     p.warps_per_block = W;
@@ -1012,7 +1016,7 @@ inline bool aligned8(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 7
 template <typename K>
 bool allow_smem(K kernel, size_t bytes) {
     if (bytes <= 48 * 1024) return true;
-    return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kSmemPerSm - 1024)) == cudaSuccess;
+    return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(smem_per_sm() - 1024)) == cudaSuccess;
 }
 
 // Chunks of the chained kernel: about 32 KB of inputs per block and chunk, so that the chunks of
@@ -1186,7 +1190,7 @@ bool vec_trace_block_cuts(int64_t N, int64_t T, int64_t D, bool perdim) {
     if (g_force_chained == 1) return false;
     const unsigned len = chained_chunk_len(tm_row_bytes(perdim ? kTmVecBeta : kTmVec, false));
     if ((int64_t)len >= T) return false;
-    return g_force_chained == 2 || (D + 31) / 32 * N < (perdim ? 96 : 4 * kSms);
+    return g_force_chained == 2 || (D + 31) / 32 * N < (perdim ? 96 : 4 * sm_count());
 }
 
 // shapes the block kernel takes: rows of D floats copied in 16-byte pieces, and enough blocks -- from
@@ -1240,7 +1244,7 @@ int vec_trace_block(const float* x, const float* beta, const uint8_t* dones, flo
     if (!perdim) return go(std::integral_constant<int, kTmVec>{});
     // deeper stages while every block is resident at once (up to ten 128-thread blocks per SM)
     const long long blocks = (D + 31) / 32 * N * p.chunks;
-    return (p.chunks == 1 && blocks < 10 * kSms) ? go(std::integral_constant<int, kTmVecBeta16>{})
+    return (p.chunks == 1 && blocks < 10 * sm_count()) ? go(std::integral_constant<int, kTmVecBeta16>{})
                                                  : go(std::integral_constant<int, kTmVecBeta>{});
 }
 

@@ -45,15 +45,29 @@ def test_no_alloc_limit_is_decided_on_the_scratch_a_call_uses(L):
     cap = L.rlcs_no_alloc_scratch_bytes()
     assert cap == 1 << 20
     assert L.rlcs_gae_carry_bytes(0, 5, 0, 1) == 0 and L.rlcs_gae_carry_bytes(-1, 5, 0, 1) == 0
-    for N, T in ((96, 1000), (8, 128), (4096, 1000), (33545, 1000)):
+    for N, T in ((96, 999), (8, 128), (4096, 999), (33545, 999)):
         for tr in (0, 1):
             for vec in (0, 1):
                 assert L.rlcs_gae_carry_bytes(N, T, tr, vec) <= L.rlcs_workspace_bytes(N, T)
     assert L.rlcs_gae_carry_bytes(16384, 2048, 1, 1) == 0 and L.rlcs_gae_carry_bytes(64, 16384, 0, 1) == 0
-    assert L.rlcs_gae_carry_bytes(33545, 1000, 1, 1) <= cap < L.rlcs_gae_carry_bytes(140000, 1000, 0, 1)
+    assert L.rlcs_gae_carry_bytes(33545, 999, 1, 1) <= cap < L.rlcs_gae_carry_bytes(140000, 999, 0, 1)
     # beyond the array: refused on the host, before anything touches a device
-    assert L.rlcs_gae_no_alloc(P, P, P, None, None, None, P, None, 140000, 1000, 0.99, 0.95, None) == 8
+    assert L.rlcs_gae_no_alloc(P, P, P, None, None, None, P, None, 140000, 999, 0.99, 0.95, None) == 8
     assert b"scratch" in L.rlcs_status_string(8) and b"capture" in L.rlcs_status_string(9)
+
+
+def test_row_aligned_tiling_needs_no_carry_workspace(L):
+    """Short rows that nearly fill a tile with a whole number of rows are tiled by rows: no carry."""
+    try:
+        for N, T in ((4096, 1000), (16384, 2000), (4096, 500), (4096, 250), (64, 200)):
+            assert L.rlcs_gae_carry_bytes(N, T, 1, 1) == 0, (N, T)
+        assert L.rlcs_gae_carry_bytes(4096, 999, 1, 1) > 0          # 999 steps do not split into whole chunks
+        assert L.rlcs_gae_carry_bytes(4096, 600, 1, 1) > 0          # one row would leave 41 % of the tile idle
+        assert L.rlcs_gae_carry_bytes(64, 3000, 1, 1) > 0           # rows longer than a tile
+        assert L.rlcs_debug_allow_row_tiles(0) == OK
+        assert L.rlcs_gae_carry_bytes(4096, 1000, 1, 1) > 0
+    finally:
+        L.rlcs_debug_allow_row_tiles(1)
 
 
 def test_status_strings(L):

@@ -138,6 +138,28 @@ def test_shape_matrix(oracle, W, B, N, T, p_flag):
     compare_all(oracle, ro)
 
 
+@pytest.mark.parametrize("variant", [-1, 0, 5, 6, 19])
+@pytest.mark.parametrize("N,T", [(37, 1000), (9, 2000), (130, 500), (64, 250), (301, 200), (1000, 100), (3, 1800), (700, 96)])
+def test_row_aligned_tiles_and_look_back_agree(oracle, W, B, variant, N, T):
+    """Rows shorter than a tile that do not divide it: with row-aligned tiling (a block takes a whole
+    number of rows, its last threads idle) and without it (fixed tiles, carry through the workspace)
+    the results match the oracle, and each other to rounding."""
+    ro = W.make_rollout(93, N, T, p_done=0.004, p_trunc=0.004, salt=T)
+    B.rlcs_debug_set_tile_variant(variant)
+    try:
+        gpu_on, _, _ = compare_all(oracle, ro)
+        B.rlcs_debug_allow_row_tiles(False)
+        gpu_off, _, _ = compare_all(oracle, ro)
+    finally:
+        B.rlcs_debug_allow_row_tiles(True)
+        B.rlcs_debug_set_tile_variant(BASE_VARIANT)
+    for a in gpu_on:
+        for x, y in zip(gpu_on[a] if isinstance(gpu_on[a], tuple) else (gpu_on[a],), gpu_off[a] if isinstance(gpu_off[a], tuple) else (gpu_off[a],)):
+            np.testing.assert_allclose(x, y, rtol=1e-5, atol=1e-4)
+    # unaligned pointers take the element-wise instantiation of the same tiling
+    compare_all(oracle, ro, offset=1)
+
+
 @pytest.mark.parametrize("variant", list(range(21)))
 @pytest.mark.parametrize("N,T", [(5, 700), (4097, 3), (2, 9000), (64, 513)])
 def test_tile_variants(oracle, W, B, variant, N, T):

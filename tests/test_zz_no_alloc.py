@@ -14,8 +14,8 @@ def test_no_alloc_entry_matches_workspace_entry_twice(oracle):
     from paper_2608_17641_b200 import binding as B, workloads
     assert torch.cuda.is_available()
     B.lib()
-    # rows of 1000 steps straddle the tiles, so the scratch (tile records, call counter) is really used
-    ro = workloads.make_rollout(60, 96, 1000, p_done=0.002, p_trunc=0.002)
+    # rows of 999 steps straddle the tiles, so the scratch (tile records, call counter) is really used
+    ro = workloads.make_rollout(60, 96, 999, p_done=0.002, p_trunc=0.002)
     dev = Dev(ro)
     p = ro.params
     ws = B.Workspace(ro.N, ro.T)
@@ -82,7 +82,7 @@ def test_no_alloc_entry_serves_any_size_that_needs_no_scratch():
     L = B.lib()
     assert L.rlcs_gae_carry_bytes(16384, 2048, 1, 1) == 0          # T is a whole number of tiles
     assert L.rlcs_workspace_bytes(16384, 2048) > L.rlcs_no_alloc_scratch_bytes()
-    assert 0 < L.rlcs_gae_carry_bytes(96, 1000, 1, 1) <= L.rlcs_workspace_bytes(96, 1000)
+    assert 0 < L.rlcs_gae_carry_bytes(96, 999, 1, 1) <= L.rlcs_workspace_bytes(96, 999)
     assert L.rlcs_gae_carry_bytes(64, 16384, 0, 1) == 0            # one thread-block cluster per row
     assert L.rlcs_gae_carry_bytes(64, 16384, 0, 0) > 0             # ... which needs vector access
 
@@ -92,7 +92,7 @@ def test_no_alloc_entry_rejects_problems_beyond_its_scratch():
     L = B.lib()
     cap = L.rlcs_no_alloc_scratch_bytes()
     assert cap == 1 << 20
-    N, T = 140000, 1000                          # 140 M steps in rows that straddle tiles: more records than the array holds
+    N, T = 140000, 999                          # 140 M steps in rows that straddle tiles: more records than the array holds
     assert L.rlcs_gae_carry_bytes(N, T, 0, 1) > cap
     fake = 0x7f0000000000                        # never dereferenced: the call must fail before any launch
     st = L.rlcs_gae_no_alloc(fake, fake, fake, None, None, None, fake, None, N, T, 0.99, 0.95, None)
