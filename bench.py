@@ -900,6 +900,7 @@ def main():
     ap.add_argument("--variant", type=int, default=None, help="tile variant test hook (default: library default)")
     ap.add_argument("--no-dependent-launch", action="store_true",
                     help="measurement hook: launch the scan kernels without programmatic stream serialisation")
+    ap.add_argument("--row-blocks", type=int, default=None, help="measurement hook: one thread block per row (0 never, 1 whenever legal)")
     ap.add_argument("--no-row-tiles", action="store_true", help="measurement hook: no row-aligned tiling (short rows use the look-back)")
     ap.add_argument("--no-truncs", action="store_true", help="bench batch without per-step truncation handling")
     ap.add_argument("--rows", type=int, default=WORKLOAD["N"], help="num_envs of the bench batch (default: full size)")
@@ -943,6 +944,8 @@ def main():
         binding.rlcs_debug_set_dependent_launch(False)
     if args.no_row_tiles:
         binding.rlcs_debug_allow_row_tiles(False)
+    if args.row_blocks is not None:
+        binding.rlcs_debug_set_row_blocks(args.row_blocks)
     assert torch.cuda.is_available(), "bench.py needs a CUDA device"
     local = int(os.environ.get("LOCAL_RANK", "0"))
     torch.cuda.set_device(local)
@@ -997,7 +1000,8 @@ def main():
         ms = statistics.median(per_algo_ms[a])
         ab = algorithmic_bytes(ro, a)
         gbs = ab / (ms * 1e-3) / 1e9
-        per_algo[a] = {"ms": round(ms, 5), "env_steps_per_s": ro.N * ro.T / (ms * 1e-3), "algorithmic_bytes": ab,
+        per_algo[a] = {"ms": round(ms, 5), "samples_ms": [round(x, 4) for x in per_algo_ms[a]],
+                       "env_steps_per_s": ro.N * ro.T / (ms * 1e-3), "algorithmic_bytes": ab,
                        "gbs": round(gbs, 1), "frac_of_peak": round(gbs / peak, 4)}
         if ro.truncs is not None and a not in ("elig_trace", "episodic_prefix_sum"):
             # the same time against the byte count of a kernel that would read trunc_bootstrap densely (context only)

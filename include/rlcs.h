@@ -431,6 +431,11 @@ int rlcs_debug_variant_for(int algorithm, int has_truncs, int64_t N, int64_t T);
  * ring stages (0 = the one-tile-per-block kernel).  Any output pointer may be NULL. */
 int rlcs_debug_variant_info(int variant, int* threads, int* steps_per_thread, int* blocks_per_sm, int* ring_stages);
 
+/* Test / measurement hook for the one-thread-block-per-row kernel (rows longer than a tile, T a
+ * multiple of the steps per thread): -1 = used when there are at least as many rows as thread
+ * blocks fit on the GPU (default), 0 = never, 1 = whenever legal.  Results agree to rounding. */
+int rlcs_debug_set_row_blocks(int mode);
+
 /* Test / measurement hook: 0 turns row-aligned tiling off (see "Workspace" above: rows shorter than a
  * tile that do not divide it are then carried between thread blocks through the workspace, as rows
  * longer than a tile always are), 1 (default) allows it.  Results agree to rounding. */

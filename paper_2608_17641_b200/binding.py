@@ -71,6 +71,7 @@ SIGNATURES = {
     "rlcs_debug_allow_cluster_carry": ([_int], _int),
     "rlcs_debug_set_dependent_launch": ([_int], _int),
     "rlcs_debug_allow_row_tiles": ([_int], _int),
+    "rlcs_debug_set_row_blocks": ([_int], _int),
     "rlcs_debug_variant_for": ([_int, _int, _i64, _i64], _int),
     "rlcs_debug_variant_built": ([_int], _int),
     "rlcs_debug_variant_info": ([_int] + [ctypes.POINTER(ctypes.c_int)] * 4, _int),
@@ -411,6 +412,11 @@ def rlcs_debug_variant_for(algorithm: str, has_truncs: bool, N: int, T: int) -> 
     _check(lib().rlcs_debug_variant_info(v, *[ctypes.byref(o) for o in out]))
     return dict(variant=v, threads=out[0].value, steps_per_thread=out[1].value, blocks_per_sm=out[2].value,
                 ring_stages=out[3].value)
+
+
+def rlcs_debug_set_row_blocks(mode: int = -1):
+    """Test hook: one thread block per row: -1 = when there are enough rows (default), 0 = never, 1 = whenever legal."""
+    _check(lib().rlcs_debug_set_row_blocks(int(mode)))
 
 
 def rlcs_debug_allow_row_tiles(on: bool):

@@ -10,6 +10,7 @@ long long g_mute_tile = -1;
 long long g_spin_cap = 0;
 bool g_pdl = true;
 bool g_row_tiles = true;
+int g_row_blocks = -1;
 }  // namespace rlcs_hooks
 
 extern "C" {
@@ -351,6 +352,11 @@ int rlcs_debug_variant_info(int variant, int* threads, int* steps_per_thread, in
     if (steps_per_thread) *steps_per_thread = tv.items;
     if (blocks_per_sm) *blocks_per_sm = tv.min_blocks;
     if (ring_stages) *ring_stages = tv.stages;
+    return RLCS_OK;
+}
+
+int rlcs_debug_set_row_blocks(int mode) {
+    rlcs_hooks::g_row_blocks = mode;
     return RLCS_OK;
 }
 

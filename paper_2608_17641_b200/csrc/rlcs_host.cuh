@@ -7,6 +7,7 @@
 #include <cstdint>
 
 #include "../../include/rlcs.h"
+#include "rlcs_device.cuh"
 #include "rlcs_launch.cuh"
 
 // test hooks, set through the rlcs_debug_* entry points (defined in rlcs_api.cu)
@@ -17,6 +18,7 @@ extern bool g_wide_index;          // use the 64-bit index path even when 32 bit
 extern long long g_mute_tile;      // tile that does not publish
 extern long long g_spin_cap;       // poll limit (0 = default)
 extern bool g_row_tiles;           // allow row-aligned tiling (default on)
+extern int g_row_blocks;           // one thread block per row: -1 = when there are enough rows (default), 0 = never, 1 = whenever legal
 }  // namespace rlcs_hooks
 
 namespace {
@@ -108,9 +110,28 @@ int choose_variant_unchecked(int algo, bool trunc, int64_t total, int64_t T) {
     }
 }
 
+// A row longer than the variant's tile splits into whole chunks and fills its tiles to at least 70 %:
+// what the one-thread-block-per-row kernel needs of (variant, T).
+bool row_fits(int variant, int64_t T) {
+    const RLCS_NS::TileVariant tv = RLCS_NS::kVariants[variant];
+    const int64_t tile = (int64_t)tv.threads * tv.items;
+    if (tv.stages != 0 || T <= tile || T % tv.items != 0) return false;
+    const int64_t tiles = (T + tile - 1) / tile;
+    return T * 10 >= tiles * tile * 7;
+}
+
 int choose_variant(int algo, bool trunc, int64_t total, int64_t T) {
     if (g_variant >= 0 && RLCS_NS::variant_built_for(algo, g_variant)) return g_variant;
-    const int v = choose_variant_unchecked(algo, trunc, total, T);
+    int v = choose_variant_unchecked(algo, trunc, total, T);
+    // Long rows, enough of them for one thread block per row: if the preferred shape does not suit the
+    // row length (T not a multiple of its 16 steps per thread, or a mostly empty last tile), an 8-step
+    // shape that does is worth more than the preferred shape with a carry between blocks.
+    if (rlcs_hooks::g_row_blocks != 0 && RLCS_NS::variant_built_for(algo, v) && T > tile_elems(v) &&
+        total / T >= 3 * rlcs_device::limits().sms && !row_fits(v, T)) {
+        const int alternatives[2] = {0, 6};          // 256 x 8 (2048 steps), 128 x 8 (1024 steps)
+        for (int alt : alternatives)
+            if (RLCS_NS::variant_built_for(algo, alt) && row_fits(alt, T)) { v = alt; break; }
+    }
     if (RLCS_NS::variant_built_for(algo, v)) return v;
     // not compiled for this algorithm / element type: the nearest shape that every build has
     return (total < (int64_t(1) << 23) && T <= 2048) ? 6 : 0;
@@ -122,6 +143,7 @@ struct CarryPlan {
     int cluster;         // > 1: one thread-block cluster of this many tiles per row, no workspace
     size_t bytes;        // workspace bytes this call reads or writes (0 when it needs none)
     int tile_steps;      // steps per thread block: the tile, or less with row-aligned tiling
+    int row_blocks;      // one thread block per row, walking the row's tiles (no carry between blocks)
 };
 
 // Row-aligned tiling: when rows are shorter than a tile but do not divide it, a block can take the
@@ -139,11 +161,30 @@ int row_aligned_steps(int variant, int64_t T) {
     return 0;
 }
 
+// One thread block per row: rows longer than a tile, T a multiple of the steps per thread (every
+// chunk whole and aligned), vector access, the row's tiles at least 70 % used, and at least three
+// rows per SM (with fewer rows too many SMs idle: those go to the cluster carry or the look-back;
+// measured cross-over at T = 16384: 384 rows 0.70 against 0.73, 512 rows 0.84 against 0.70).
+bool row_blocks_ok(int variant, int64_t total, int64_t T, bool vec) {
+    const RLCS_NS::TileVariant tv = RLCS_NS::kVariants[variant];
+    const int tile = tv.threads * tv.items;
+    if (rlcs_hooks::g_row_blocks == 0 || !vec || tv.stages != 0 || T <= tile || T % tv.items != 0) return false;
+    const int64_t tiles = (T + tile - 1) / tile;
+    if (T * 10 < tiles * tile * 7) return false;
+    if (rlcs_hooks::g_row_blocks > 0) return true;
+    return total / T >= 3 * rlcs_device::limits().sms;        // measured cross-over against the cluster carry: about 3 rows per SM
+}
+
 CarryPlan plan_carry(int variant, int64_t total, int64_t T, bool vec, bool allow_cluster, int records_per_tile,
                      bool allow_row_tiles = true) {
     const int tile = tile_elems(variant);
     const int64_t num_tiles = (total + tile - 1) / tile;
-    CarryPlan plan = {(tile % T) != 0 ? 1 : 0, 0, 0, tile};       // T does not divide the tile: rows straddle tiles
+    CarryPlan plan = {(tile % T) != 0 ? 1 : 0, 0, 0, tile, 0};    // T does not divide the tile: rows straddle tiles
+    if (allow_row_tiles && row_blocks_ok(variant, total, T, vec)) {
+        plan.carry_mode = 0;
+        plan.row_blocks = 1;
+        return plan;
+    }
     if (plan.carry_mode && allow_row_tiles) {
         const int steps = row_aligned_steps(variant, T);
         if (steps > 0) {
@@ -172,7 +213,8 @@ int finish_params(ScanParams& p, int variant, int64_t total, int64_t T, void* wo
     p.total = total;
     p.T = (unsigned)T;
     p.tile_steps = (unsigned)plan.tile_steps;
-    p.num_tiles = (total + plan.tile_steps - 1) / plan.tile_steps;
+    p.num_tiles = plan.row_blocks ? total / T : (total + plan.tile_steps - 1) / plan.tile_steps;      // = the grid
+    p.row_blocks = plan.row_blocks;
     p.idx32 = !g_wide_index && (total + tile) <= 0xffffffffLL;
     {   // invariant division by T (see FastDiv)
         int l = 0;

@@ -132,9 +132,23 @@ cudaError_t launch_cluster(const ScanParams& p, cudaStream_t stream) {
                        stream, p.cluster, p);
 }
 
+// One thread block per row (p.row_blocks; rows longer than a tile, many rows): grid = number of rows.
+template <int ALGO, bool TRUNC, int V>
+cudaError_t launch_rows(const ScanParams& p, cudaStream_t stream) {
+    constexpr TileVariant tv = kVariants[V];
+    return launch_scan(scan_kernel_rows<ALGO, TRUNC, tv.threads, tv.items, tv.min_blocks>, (unsigned)p.num_tiles, tv.threads, 0,
+                       stream, 0, p);
+}
+
+// algorithms that have the one-block-per-row kernel (the seven of the paper and the bare affine scan)
+__host__ __device__ constexpr bool has_row_blocks(int algo) { return algo <= kAffineFwd; }
+
 template <int ALGO, bool TRUNC, bool VEC, int V>
 cudaError_t launch_variant(const ScanParams& p, cudaStream_t stream) {
     constexpr TileVariant tv = kVariants[V];
+    if constexpr (VEC && tv.stages == 0 && has_row_blocks(ALGO)) {
+        if (p.row_blocks) return launch_rows<ALGO, TRUNC, V>(p, stream);
+    }
     if constexpr (VEC && tv.stages == 0) {
         if (p.cluster > 1) return launch_cluster<ALGO, TRUNC, V>(p, stream);
     }

@@ -122,6 +122,7 @@ struct ScanParams {
     int starts_at;
     int carry_mode;           // rows may straddle tiles: publish aggregates, look back
     int cluster;              // > 1: rows are exactly this many tiles long, one thread-block cluster per row
+    int row_blocks;           // != 0: one thread block per row walks the row's tiles in scan order (scan_kernel_rows)
     unsigned* header;         // workspace header (carry mode) or nullptr
     unsigned* status;         // device status word, or nullptr when there is no workspace
     uint4* records;           // one 16-byte record per tile: {alpha_bits, epoch, beta_bits, epoch}
@@ -765,7 +766,7 @@ template <int ALGO, bool TRUNC, bool VEC, int THREADS, int ITEMS, bool FULL, boo
           bool IDLE = false>
 __device__ __forceinline__ void tile_compute(Chunk<ALGO, TRUNC, ITEMS>& c, Vals<ITEMS>& v, const ScanParams& p, long long i0, long long s,
                                              unsigned epoch, ScanSmem<THREADS / 32>& sm, int buf, Hook after_barrier,
-                                             float* prev_out = nullptr) {
+                                             float* prev_out = nullptr, float* row_carry = nullptr) {
     constexpr bool FWD = is_forward(ALGO);
     constexpr int NW = THREADS / 32;
     constexpr int W = ITEMS / 4;
@@ -968,7 +969,12 @@ __device__ __forceinline__ void tile_compute(Chunk<ALGO, TRUNC, ITEMS>& c, Vals<
 
     // ---- carry between thread blocks
     float carry_in = 0.f;
-    if constexpr (CLUSTER) {
+    if (row_carry != nullptr) {
+        // one block walks the whole row: the carry stays in a register (every thread holds the same
+        // tile aggregate, so every thread updates its own copy -- no barrier, no memory traffic)
+        carry_in = *row_carry;
+        *row_carry = fmaf(tile_agg.b, carry_in, tile_agg.a);
+    } else if constexpr (CLUSTER) {
         carry_in = cluster_carry<NW>(tile_agg, sm, buf);
     } else if (p.carry_mode) {
         if (warp == 0 && lane == 0 && s != p.mute_tile) {
@@ -1234,6 +1240,51 @@ __global__ void __launch_bounds__(THREADS, MIN_BLOCKS) scan_kernel_cluster(const
     issue_boot(c, p, n0);
     issue_trunc_values(c, p, i0);
     tile_compute<ALGO, TRUNC, true, THREADS, ITEMS, true, false, NoHook, true>(c, v, p, i0, s, 0u, sm, 0, NoHook{});
+}
+
+// ------------------------------------------------------------------------------------------ kernel 1e: one thread block per row
+// For rows longer than a tile when there are at least as many rows as thread blocks fit on the GPU:
+// block n walks the tiles of row n in scan order and carries the recurrence from tile to tile in a
+// register.  Blocks never wait for one another and nothing goes through global memory; the other
+// blocks resident on the SM keep the memory system busy while one block is between its loads and
+// its stores, exactly as with one tile per block.  The row's last tile (in address order) may be
+// short: its tail threads idle (T must be a multiple of the steps per thread, which also keeps every
+// chunk aligned for 256-bit accesses).  Vector accesses only.
+template <int ALGO, bool TRUNC, int THREADS, int ITEMS, bool IDLE>
+__device__ __forceinline__ void row_tile(const ScanParams& p, long long tile_start, long long row_end, float& carry,
+                                         ScanSmem<THREADS / 32>& sm, int buf) {
+    const int tid = threadIdx.x;
+    const int lane = tid & 31;
+    Chunk<ALGO, TRUNC, ITEMS> c;
+    const long long i0 = tile_start + (long long)tid * ITEMS;
+    const long long n0 = locate(c, p, i0, row_end);
+    load_flags_global<ALGO, TRUNC, ITEMS, true, true, IDLE>(c, p, i0, lane);
+    Vals<ITEMS> v;
+    load_values_global<ALGO, TRUNC, ITEMS, true, true, IDLE>(c, v, p, i0, lane);
+    issue_boot(c, p, n0);
+    issue_trunc_values(c, p, i0);
+    tile_compute<ALGO, TRUNC, true, THREADS, ITEMS, true, false, NoHook, false, IDLE>(c, v, p, i0, 0, 0u, sm, buf, NoHook{}, nullptr,
+                                                                                     &carry);
+}
+
+template <int ALGO, bool TRUNC, int THREADS, int ITEMS, int MIN_BLOCKS>
+__global__ void __launch_bounds__(THREADS, MIN_BLOCKS) scan_kernel_rows(const ScanParams p) {
+    constexpr bool FWD = is_forward(ALGO);
+    constexpr int TILE = THREADS * ITEMS;
+    __shared__ ScanSmem<THREADS / 32> sm;
+    grid_dependency_launch();
+    grid_dependency_wait();
+    const long long row_start = (long long)blockIdx.x * p.T;
+    const long long row_end = row_start + p.T;
+    const unsigned tiles = (p.T + TILE - 1) / TILE;
+    float carry = 0.f;                                        // the row's boundary carry is folded into alpha at its edge
+    for (unsigned k = 0; k < tiles; ++k) {
+        const unsigned m = FWD ? k : tiles - 1 - k;           // k-th tile in scan order
+        const long long tile_start = row_start + (long long)m * TILE;
+        // shared scratch alternates by tile parity, so one barrier per tile suffices (as in the persistent kernel)
+        if (tile_start + TILE <= row_end) row_tile<ALGO, TRUNC, THREADS, ITEMS, false>(p, tile_start, row_end, carry, sm, k & 1);
+        else row_tile<ALGO, TRUNC, THREADS, ITEMS, true>(p, tile_start, row_end, carry, sm, k & 1);
+    }
 }
 
 // ------------------------------------------------------------------------------------------ mbarrier / bulk copy (PTX)

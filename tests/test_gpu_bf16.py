@@ -158,6 +158,17 @@ def test_bf16_rows_of_whole_tiles_use_the_cluster_carry(oracle, W, B, N, T):
     compare16(oracle, B, W.make_rollout(123, N, T, p_done=0.001, p_trunc=0.001), algos=("gae", "discounted_return", "elig_trace"))
 
 
+@pytest.mark.parametrize("N,T", [(6, 6016), (3, 16384), (40, 2000), (9, 1000)])
+def test_bf16_row_kernels(oracle, W, B, N, T):
+    """The layouts without a carry between blocks on bfloat16 tensors: one thread block per row (forced
+    here, few rows) and row-aligned tiles."""
+    B.rlcs_debug_set_row_blocks(1)
+    try:
+        compare16(oracle, B, W.make_rollout(127, N, T, p_done=0.002, p_trunc=0.002))
+    finally:
+        B.rlcs_debug_set_row_blocks(-1)
+
+
 def test_bf16_large_problem_with_carry(oracle, W, B):
     """Above 2^23 steps the 16-steps-per-thread tile is chosen; T = 3000 makes rows straddle tiles."""
     compare16(oracle, B, W.make_rollout(124, 2900, 3000, p_done=0.002, p_trunc=0.002), algos=("gae", "vtrace", "retrace"))

@@ -160,6 +160,39 @@ def test_row_aligned_tiles_and_look_back_agree(oracle, W, B, variant, N, T):
     compare_all(oracle, ro, offset=1)
 
 
+@pytest.mark.parametrize("variant", [-1, 0, 6, 19])
+@pytest.mark.parametrize("N,T", [(7, 3008), (5, 4096), (3, 16384), (11, 6000), (2, 40000), (300, 2512), (6, 2064)])
+def test_one_block_per_row_agrees_with_the_carry_between_blocks(oracle, W, B, variant, N, T):
+    """Rows longer than a tile: one thread block walking the whole row (carry in a register) against
+    the carries between blocks (cluster / look-back).  Both match the oracle, and each other to
+    rounding; where the row kernel does not apply (T not a multiple of the steps per thread, or a
+    mostly empty last tile) the hook changes nothing."""
+    ro = W.make_rollout(94, N, T, p_done=0.001, p_trunc=0.001, salt=T)
+    B.rlcs_debug_set_tile_variant(variant)
+    try:
+        B.rlcs_debug_set_row_blocks(1)
+        gpu_on, _, _ = compare_all(oracle, ro)
+        B.rlcs_debug_set_row_blocks(0)
+        gpu_off, _, _ = compare_all(oracle, ro)
+    finally:
+        B.rlcs_debug_set_row_blocks(-1)
+        B.rlcs_debug_set_tile_variant(BASE_VARIANT)
+    for a in gpu_on:
+        for x, y in zip(gpu_on[a] if isinstance(gpu_on[a], tuple) else (gpu_on[a],), gpu_off[a] if isinstance(gpu_off[a], tuple) else (gpu_off[a],)):
+            np.testing.assert_allclose(x, y, rtol=1e-5, atol=1e-4)
+
+
+def test_one_block_per_row_is_the_default_with_many_rows(oracle, W, B):
+    """Enough rows to fill the GPU: the row kernel is what runs (no carry workspace is needed)."""
+    N, T = 1200, 2064                                     # 2048 + one chunk of 16: no tile shape is filled to 70 % by such rows
+    assert B.lib().rlcs_gae_carry_bytes(N, T, 1, 1) > 0   # ... so these rows are carried between blocks
+    assert B.lib().rlcs_gae_carry_bytes(1200, 4112, 1, 1) == 0      # 4112 = 5 tiles of 1024 at 80 %: the 1024-step shape is taken
+    N, T = 1200, 6000
+    ro = W.make_rollout(95, N, T, p_done=0.0005, p_trunc=0.0005)
+    assert B.lib().rlcs_gae_carry_bytes(N, T, 1, 1) == 0
+    compare_all(oracle, ro, algos=("gae", "vtrace", "discounted_return", "elig_trace"), workspace=None)
+
+
 @pytest.mark.parametrize("variant", list(range(21)))
 @pytest.mark.parametrize("N,T", [(5, 700), (4097, 3), (2, 9000), (64, 513)])
 def test_tile_variants(oracle, W, B, variant, N, T):
@@ -296,11 +329,18 @@ def test_large_problem_variants_with_carry(oracle, W, B):
     thread); T = 3000 makes rows straddle every one of them, so the inter-block carry runs too."""
     ro = W.make_rollout(106, 2900, 3000, p_done=0.002, p_trunc=0.002)
     assert ro.N * ro.T > 1 << 23
-    for a in ("gae", "vtrace", "td_lambda", "discounted_return", "elig_trace", "episodic_prefix_sum"):
-        name = a if a != "episodic_prefix_sum" else "episodic_prefix_sum"
-        info = B.rlcs_debug_variant_for(name, True, ro.N, ro.T)
-        assert BASE_VARIANT != -1 or info["variant"] not in (0, 6), (a, info)
-    compare_all(oracle, ro)
+    B.rlcs_debug_set_row_blocks(0)              # (with many rows the default would be one thread block per row)
+    try:
+        for a in ("gae", "vtrace", "td_lambda", "discounted_return", "elig_trace", "episodic_prefix_sum"):
+            info = B.rlcs_debug_variant_for(a, True, ro.N, ro.T)
+            assert BASE_VARIANT != -1 or info["variant"] not in (0, 6), (a, info)
+        compare_all(oracle, ro)
+    finally:
+        B.rlcs_debug_set_row_blocks(-1)
+    # the default for this shape: an 8-step tile shape that splits rows of 3000 into whole chunks, one block per row
+    info = B.rlcs_debug_variant_for("gae", True, ro.N, ro.T)
+    assert BASE_VARIANT != -1 or info["steps_per_thread"] == 8, info
+    compare_all(oracle, ro, workspace=None)
 
 
 @pytest.mark.parametrize("N,T,variant", [(5, 4096, 0), (3, 16384, 0), (64, 2048, 6), (7, 8192, 6), (9, 3072, 6), (2, 16384, 5),
