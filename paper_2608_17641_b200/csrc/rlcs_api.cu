@@ -151,7 +151,9 @@ int rlcs_gae_normalized(const float* rewards, const float* values, const uint8_t
     p.stats = mean_rstd + 64;
     p.gamma = gamma; p.decay = gamma * lambda;
     const int variant = choose_variant(rlcs::kGaeStats, truncs != nullptr, total, T);
-    st = finish_params(p, variant, total, T, carry_bytes ? workspace : nullptr, carry_bytes, vec);
+    // (the statistics flavour keeps fixed tiles: its per-tile sums are laid out for them, and it has no
+    // one-block-per-row instantiation)
+    st = finish_params(p, variant, total, T, carry_bytes ? workspace : nullptr, carry_bytes, vec, true, 1, false, false);
     if (st != RLCS_OK) return st;
     st = run(rlcs::launch_gae_stats, p, variant, truncs != nullptr, vec, cuda_stream);
     if (st != RLCS_OK) return st;

@@ -176,11 +176,11 @@ bool row_blocks_ok(int variant, int64_t total, int64_t T, bool vec) {
 }
 
 CarryPlan plan_carry(int variant, int64_t total, int64_t T, bool vec, bool allow_cluster, int records_per_tile,
-                     bool allow_row_tiles = true) {
+                     bool allow_row_tiles = true, bool allow_row_blocks = true) {
     const int tile = tile_elems(variant);
     const int64_t num_tiles = (total + tile - 1) / tile;
     CarryPlan plan = {(tile % T) != 0 ? 1 : 0, 0, 0, tile, 0};    // T does not divide the tile: rows straddle tiles
-    if (allow_row_tiles && row_blocks_ok(variant, total, T, vec)) {
+    if (allow_row_tiles && allow_row_blocks && row_blocks_ok(variant, total, T, vec)) {
         plan.carry_mode = 0;
         plan.row_blocks = 1;
         return plan;
@@ -205,11 +205,14 @@ CarryPlan plan_carry(int variant, int64_t total, int64_t T, bool vec, bool allow
     return plan;
 }
 
-// Fill the size / tiling / carry fields and validate the workspace for this call.
+// Fill the size / tiling / carry fields and validate the workspace for this call.  Callers whose
+// kernels have no row-aligned / one-block-per-row instantiation (has_row_blocks() in rlcs_launch.cuh:
+// the statistics flavour of GAE, the observation-skip scans, Retrace from [N,T,A] tensors) pass
+// allow_row_tiles = false.
 int finish_params(ScanParams& p, int variant, int64_t total, int64_t T, void* workspace, size_t workspace_bytes, bool vec,
-                  bool allow_cluster = true, int records_per_tile = 1, bool allow_row_tiles = true) {
+                  bool allow_cluster = true, int records_per_tile = 1, bool allow_row_tiles = true, bool allow_row_blocks = true) {
     const int tile = tile_elems(variant);
-    const CarryPlan plan = plan_carry(variant, total, T, vec, allow_cluster, records_per_tile, allow_row_tiles);
+    const CarryPlan plan = plan_carry(variant, total, T, vec, allow_cluster, records_per_tile, allow_row_tiles, allow_row_blocks);
     p.total = total;
     p.T = (unsigned)T;
     p.tile_steps = (unsigned)plan.tile_steps;

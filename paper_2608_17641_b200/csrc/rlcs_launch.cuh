@@ -158,6 +158,12 @@ cudaError_t launch_variant(const ScanParams& p, cudaStream_t stream) {
         return launch_scan(scan_kernel<ALGO, TRUNC, true, tv.threads, tv.items, tv.min_blocks>, (unsigned)p.num_tiles, tv.threads,
                            0, stream, 0, p);
     } else {
+        if constexpr (has_row_blocks(ALGO)) {
+            // row-aligned tiling has an instantiation of its own (idle tail threads, tile length at run time)
+            if (p.tile_steps != (unsigned)(tv.threads * tv.items))
+                return launch_scan(scan_kernel<ALGO, TRUNC, VEC, tv.threads, tv.items, tv.min_blocks, true>, (unsigned)p.num_tiles,
+                                   tv.threads, 0, stream, 0, p);
+        }
         // bulk copies need 16-byte aligned pointers; otherwise the element-wise kernel of the same tile shape
         return launch_scan(scan_kernel<ALGO, TRUNC, VEC, tv.threads, tv.items, tv.min_blocks>, (unsigned)p.num_tiles, tv.threads,
                            0, stream, 0, p);

@@ -1073,17 +1073,24 @@ __device__ __forceinline__ void tile_compute(Chunk<ALGO, TRUNC, ITEMS>& c, Vals<
 
 // ------------------------------------------------------------------------------------------ end of a call (carry mode)
 // ------------------------------------------------------------------------------------------ kernel 1: one tile per block
-template <int ALGO, bool TRUNC, bool VEC, int THREADS, int ITEMS, bool FULL, bool IDLE = false>
+template <int ALGO, bool TRUNC, bool VEC, int THREADS, int ITEMS, bool FULL, bool IDLE = false, bool ROWTILES = false>
 __device__ __forceinline__ void one_tile(const ScanParams& p, long long tile, long long s, unsigned epoch,
                                          ScanSmem<THREADS / 32>& sm) {
+    constexpr int TILE = THREADS * ITEMS;
     const int tid = threadIdx.x;
     const int lane = tid & 31;
     Chunk<ALGO, TRUNC, ITEMS> c;
-    // a tile covers p.tile_steps steps: THREADS*ITEMS, or (row-aligned tiling) a whole number of rows
-    // that is a little less, in which case the last threads of the block have nothing to do
-    const long long i0 = tile * p.tile_steps + (long long)tid * ITEMS;
-    const long long tile_end = (tile + 1) * p.tile_steps;
-    const long long n0 = locate(c, p, i0, tile_end < p.total ? tile_end : p.total);
+    long long i0, n0;
+    if constexpr (ROWTILES) {
+        // row-aligned tiling: a tile covers p.tile_steps steps, a whole number of rows that is a little
+        // less than THREADS*ITEMS, and the last threads of the block have nothing to do
+        i0 = tile * p.tile_steps + (long long)tid * ITEMS;
+        const long long tile_end = (tile + 1) * p.tile_steps;
+        n0 = locate(c, p, i0, tile_end < p.total ? tile_end : p.total);
+    } else {
+        i0 = tile * TILE + (long long)tid * ITEMS;
+        n0 = locate(c, p, i0);
+    }
     load_flags_global<ALGO, TRUNC, ITEMS, VEC, FULL, IDLE>(c, p, i0, lane);
     Vals<ITEMS> v;
     load_values_global<ALGO, TRUNC, ITEMS, VEC, FULL, IDLE>(c, v, p, i0, lane);
@@ -1092,7 +1099,9 @@ __device__ __forceinline__ void one_tile(const ScanParams& p, long long tile, lo
     tile_compute<ALGO, TRUNC, VEC, THREADS, ITEMS, FULL, true, NoHook, false, IDLE>(c, v, p, i0, s, epoch, sm, 0, NoHook{});
 }
 
-template <int ALGO, bool TRUNC, bool VEC, int THREADS, int ITEMS, int MIN_BLOCKS>
+// ROWTILES: the instantiation for row-aligned tiling (p.tile_steps < THREADS*ITEMS), kept apart so that
+// the kernel for whole tiles stays exactly as lean as it is without that feature.
+template <int ALGO, bool TRUNC, bool VEC, int THREADS, int ITEMS, int MIN_BLOCKS, bool ROWTILES = false>
 __global__ void __launch_bounds__(THREADS, MIN_BLOCKS) scan_kernel(const ScanParams p) {
     constexpr bool FWD = is_forward(ALGO);
     constexpr int TILE = THREADS * ITEMS;
@@ -1103,20 +1112,17 @@ __global__ void __launch_bounds__(THREADS, MIN_BLOCKS) scan_kernel(const ScanPar
     unsigned epoch;
     const long long s = take_tile(p, epoch);          // tile index in scan order
     const long long tile = FWD ? s : (p.num_tiles - 1 - s);
-    // block-uniform: every thread has a whole chunk (the tile is a full one inside the array) and no row is shorter than a chunk
-    const bool full = (p.tile_steps == (unsigned)TILE) && (tile * TILE + TILE <= p.total) && (p.T >= (unsigned)ITEMS);
-    if (full) {
-        one_tile<ALGO, TRUNC, VEC, THREADS, ITEMS, true>(p, tile, s, epoch, sm);
-        return;
+    if constexpr (ROWTILES) {
+        // tile inside the array: whole chunks in the first threads, none in the last few (block-uniform)
+        if (VEC && (tile + 1) * (long long)p.tile_steps <= p.total && p.T >= (unsigned)ITEMS)
+            one_tile<ALGO, TRUNC, VEC, THREADS, ITEMS, true, true, true>(p, tile, s, epoch, sm);
+        else one_tile<ALGO, TRUNC, VEC, THREADS, ITEMS, false, false, true>(p, tile, s, epoch, sm);
+    } else {
+        // block-uniform: the whole tile is inside the array and no row is shorter than a chunk
+        const bool full = (tile * TILE + TILE <= p.total) && (p.T >= (unsigned)ITEMS);
+        if (full) one_tile<ALGO, TRUNC, VEC, THREADS, ITEMS, true>(p, tile, s, epoch, sm);
+        else one_tile<ALGO, TRUNC, VEC, THREADS, ITEMS, false>(p, tile, s, epoch, sm);
     }
-    if constexpr (VEC) {
-        // row-aligned tiling, tile inside the array: whole chunks in the first threads, none in the last few
-        if (p.tile_steps != (unsigned)TILE && (tile + 1) * (long long)p.tile_steps <= p.total && p.T >= (unsigned)ITEMS) {
-            one_tile<ALGO, TRUNC, VEC, THREADS, ITEMS, true, true>(p, tile, s, epoch, sm);
-            return;
-        }
-    }
-    one_tile<ALGO, TRUNC, VEC, THREADS, ITEMS, false>(p, tile, s, epoch, sm);
 }
 
 // ------------------------------------------------------------------------------------------ kernel 1b: GAE with observation-skip masking
