@@ -19,6 +19,7 @@ from __future__ import annotations
 import argparse
 import json
 import os
+import re
 import statistics
 import sys
 import threading
@@ -71,12 +72,13 @@ def algorithmic_bytes(ro, algo: str) -> int:
 
 
 def kernel_instance(binding, algo: str, has_truncs: bool, N: int, T: int) -> str:
-    """Name of the kernel instance a call takes, as ncu prints it: template arguments are
-    (algorithm id, truncation handling, vector accesses, threads, steps per thread, blocks per SM)."""
+    """Name of the kernel instance a call on whole tiles takes, as ncu prints it: template arguments are
+    (algorithm id, truncation handling, vector accesses, threads, steps per thread, blocks per SM, row-aligned tiling)."""
     tr = bool(has_truncs) and algo not in ("elig_trace", "episodic_prefix_sum")
     vi = binding.rlcs_debug_variant_for(algo, tr, N, T)
     kname = "scan_kernel_tma" if vi["ring_stages"] else "scan_kernel"
-    return f"{kname}<{binding.ALGORITHM_IDS[algo]},{int(tr)},1,{vi['threads']},{vi['steps_per_thread']},{vi['blocks_per_sm']}>"
+    args = f"{binding.ALGORITHM_IDS[algo]},{int(tr)},1,{vi['threads']},{vi['steps_per_thread']},{vi['blocks_per_sm']}"
+    return f"{kname}<{args}>" if vi["ring_stages"] else f"{kname}<{args},0>"       # last argument: not the row-aligned instantiation
 
 
 def load_traffic(path: str = TRAFFIC_JSON) -> dict:
@@ -119,15 +121,15 @@ def traffic_from_ncu(csv_path: str, out_path: str = TRAFFIC_JSON, command: str =
         by_kernel.setdefault(name, []).append(b)
     kernels = {}
     for name, vals in by_kernel.items():
-        short = name.split("(")[0].split("::")[-1].replace(" ", "")
-        if not short.startswith("scan_kernel<") and not short.startswith("scan_kernel_tma<"):
+        m = re.search(r"(scan_kernel\w*)\s*<([^>]*)>", name)
+        if m is None or m.group(1) not in ("scan_kernel", "scan_kernel_tma"):
             continue
-        algo = ids.get(int(short.split("<")[1].split(",")[0]))
+        targs = [a.strip().replace("(rlcs::Algo)", "").replace("(bool)", "").replace("(int)", "") for a in m.group(2).split(",")]
+        targs = ["1" if a == "true" else "0" if a == "false" else a for a in targs]
+        algo = ids.get(int(targs[0]))
         if algo is None:
             continue
-        if "(bool)" in short or "true" in short or "false" in short:      # ncu may print bools as words
-            short = short.replace("(bool)1", "1").replace("(bool)0", "0").replace("true", "1").replace("false", "0")
-        short = short.replace("(rlcs::Algo)", "").replace("(int)", "")
+        short = f"{m.group(1)}<{','.join(targs)}>"
         kernels[algo] = {"kernel": short, "launches": len(vals), "dram_bytes_per_launch": int(round(sum(vals) / len(vals)))}
     doc = {"workload": f"num_envs={WORKLOAD['N']}, T={WORKLOAD['T']}, truncation handling on", "command": command,
            "metrics": "dram__bytes_read.sum + dram__bytes_write.sum, mean over the captured launches", "kernels": kernels}

@@ -81,7 +81,9 @@ int choose_variant_unchecked(int algo, bool trunc, int64_t total, int64_t T) {
     if (total < (int64_t(1) << 23)) {
         // latency-bound sizes (cold-L2 sweeps): long rows want few carry hops (2048-step tiles, one
         // cluster per row where that fits), the smallest problems want many small blocks
-        if (T > 2048) return 19;
+        // (the 16-step shape at 80 registers spills for the algorithms with three or four float inputs:
+        // V-trace takes it at 96 registers, Retrace the 8-step shape of the same tile length)
+        if (T > 2048) return algo == RLCS_NS::kRetrace ? 0 : algo == RLCS_NS::kVtrace ? 18 : 19;
         return total <= (int64_t(1) << 19) ? 1 : 6;
     }
     if (RLCS_NS::kIoBf16) {

@@ -81,16 +81,16 @@ def test_traffic_table_from_an_ncu_log(tmp_path):
         '==PROF== Connected to process 1\n'
         '"ID","Process ID","Process Name","Host Name","Kernel Name","Context","Stream","Block Size","Grid Size","Device","CC",'
         '"Section Name","Metric Name","Metric Unit","Metric Value"\n'
-        '"0","1","python","h","void rlcs::scan_kernel<4, 1, 1, 256, 8, 4>(rlcs::ScanParams)","1","7","(256, 1, 1)","(16384, 1, 1)","0","10.0",'
+        '"0","1","python","h","void scan_kernel<4, 1, 1, 256, 8, 4, 0>(ScanParams)","1","7","(256, 1, 1)","(16384, 1, 1)","0","10.0",'
         '"Command line profiler metrics","dram__bytes_read.sum","Mbyte","623.6"\n'
-        '"0","1","python","h","void rlcs::scan_kernel<4, 1, 1, 256, 8, 4>(rlcs::ScanParams)","1","7","(256, 1, 1)","(16384, 1, 1)","0","10.0",'
+        '"0","1","python","h","void scan_kernel<4, 1, 1, 256, 8, 4, 0>(ScanParams)","1","7","(256, 1, 1)","(16384, 1, 1)","0","10.0",'
         '"Command line profiler metrics","dram__bytes_write.sum","Mbyte","114.8"\n'
-        '"1","1","python","h","void rlcs::scan_kernel<0, 1, 1, 128, 16, 6>(rlcs::ScanParams)","1","7","(128, 1, 1)","(16384, 1, 1)","0","10.0",'
+        '"1","1","python","h","void rlcs::scan_kernel<0, true, true, 128, 16, 6, false>(rlcs::ScanParams)","1","7","(128, 1, 1)","(16384, 1, 1)","0","10.0",'
         '"Command line profiler metrics","dram__bytes_read.sum","byte","1,000"\n'
-        '"1","1","python","h","void rlcs::scan_kernel<0, 1, 1, 128, 16, 6>(rlcs::ScanParams)","1","7","(128, 1, 1)","(16384, 1, 1)","0","10.0",'
+        '"1","1","python","h","void rlcs::scan_kernel<0, true, true, 128, 16, 6, false>(rlcs::ScanParams)","1","7","(128, 1, 1)","(16384, 1, 1)","0","10.0",'
         '"Command line profiler metrics","dram__bytes_write.sum","byte","24"\n')
     out = tmp_path / "t.json"
     doc = bench.traffic_from_ncu(str(log), out_path=str(out), command="ncu ...")
-    assert doc["kernels"]["retrace"] == {"kernel": "scan_kernel<4,1,1,256,8,4>", "launches": 1, "dram_bytes_per_launch": 738400000}
+    assert doc["kernels"]["retrace"] == {"kernel": "scan_kernel<4,1,1,256,8,4,0>", "launches": 1, "dram_bytes_per_launch": 738400000}
     assert doc["kernels"]["gae"]["dram_bytes_per_launch"] == 1024
-    assert bench.load_traffic(str(out))["gae"]["kernel"] == "scan_kernel<0,1,1,128,16,6>"
+    assert bench.load_traffic(str(out))["gae"]["kernel"] == "scan_kernel<0,1,1,128,16,6,0>"
