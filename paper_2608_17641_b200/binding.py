@@ -115,15 +115,21 @@ def _torch():
     return torch
 
 
+_cuda_current_device = None
+
+
 def _current_device() -> int:
-    return _torch().cuda.current_device()
+    global _cuda_current_device
+    if _cuda_current_device is None:
+        _cuda_current_device = _torch().cuda.current_device
+    return _cuda_current_device()
 
 
 def _require_current_device(t, what: str = "tensor"):
     """The library launches on the current device and the current stream of that device: a tensor
     (or workspace) that lives on another GPU would hand the kernel a pointer it must not touch."""
-    index, cur = t.device.index, _current_device()
-    if index is not None and index != cur:
+    index, cur = t.get_device(), _current_device()
+    if index is not None and index >= 0 and index != cur:
         raise ValueError(f"{what} is on cuda:{index} but the current device is cuda:{cur}; "
                          f"call under torch.cuda.device({index})")
 

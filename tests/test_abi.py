@@ -187,6 +187,9 @@ class _FakeTensor:
     def is_contiguous(self):
         return True
 
+    def get_device(self):
+        return self.device.index
+
     def data_ptr(self):
         return 0x7f0000000000 + 4096 * (self.device.index or 0)
 
