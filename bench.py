@@ -268,29 +268,38 @@ class GpuBatch:
         self.ws = B.Workspace(ro.N, ro.T, device=device)
         self.launches = 0
 
-    def call(self, algo: str):
+    def spec(self, algo: str):
+        """(binding wrapper, positional arguments, keyword arguments) of one call."""
         B, i, o, p, ws = self.B, self.inp, self.out, self.ro.params, self.ws
         bw = (i["dones"], i["truncs"], i["trunc_bootstrap"], i["bootstrap"])
         if algo == "gae":
-            B.rlcs_gae(i["rewards"], i["values"], *bw, gamma=p["gamma"], lam=p["lam"], advantages=o[algo][0],
-                       returns=o[algo][1], workspace=ws)
-        elif algo == "vtrace":
-            B.rlcs_vtrace(i["rewards"], i["values"], i["log_rhos"], *bw, gamma=p["gamma"], rho_bar=p["rho_bar"],
-                          c_bar=p["c_bar"], vs=o[algo][0], pg_advantages=o[algo][1], workspace=ws)
-        elif algo == "retrace":
-            B.rlcs_retrace(i["rewards"], i["q_sa"], i["expected_q"], i["log_rhos"], *bw, gamma=p["gamma"],
-                           lam=p["lam"], c_bar=p["c_bar"], q_targets=o[algo], workspace=ws)
-        elif algo == "td_lambda":
-            B.rlcs_td_lambda(i["rewards"], i["values"], *bw, gamma=p["gamma"], lam=p["lam"], returns=o[algo], workspace=ws)
-        elif algo == "discounted_return":
-            B.rlcs_discounted_return(i["rewards"], *bw, gamma=p["gamma"], returns=o[algo], workspace=ws)
-        elif algo == "elig_trace":
-            B.rlcs_elig_trace(i["x"], i["any_done"], gamma=p["gamma"], lam=p["lam"], traces=o[algo], workspace=ws)
-        elif algo == "episodic_prefix_sum":
-            B.rlcs_episodic_prefix_sum(i["x"], i["any_done"], sums=o[algo], workspace=ws)
-        else:
-            raise KeyError(algo)
+            return B.rlcs_gae, (i["rewards"], i["values"], *bw), dict(gamma=p["gamma"], lam=p["lam"], advantages=o[algo][0],
+                                                                       returns=o[algo][1], workspace=ws)
+        if algo == "vtrace":
+            return B.rlcs_vtrace, (i["rewards"], i["values"], i["log_rhos"], *bw), dict(
+                gamma=p["gamma"], rho_bar=p["rho_bar"], c_bar=p["c_bar"], vs=o[algo][0], pg_advantages=o[algo][1], workspace=ws)
+        if algo == "retrace":
+            return B.rlcs_retrace, (i["rewards"], i["q_sa"], i["expected_q"], i["log_rhos"], *bw), dict(
+                gamma=p["gamma"], lam=p["lam"], c_bar=p["c_bar"], q_targets=o[algo], workspace=ws)
+        if algo == "td_lambda":
+            return B.rlcs_td_lambda, (i["rewards"], i["values"], *bw), dict(gamma=p["gamma"], lam=p["lam"], returns=o[algo], workspace=ws)
+        if algo == "discounted_return":
+            return B.rlcs_discounted_return, (i["rewards"], *bw), dict(gamma=p["gamma"], returns=o[algo], workspace=ws)
+        if algo == "elig_trace":
+            return B.rlcs_elig_trace, (i["x"], i["any_done"]), dict(gamma=p["gamma"], lam=p["lam"], traces=o[algo], workspace=ws)
+        if algo == "episodic_prefix_sum":
+            return B.rlcs_episodic_prefix_sum, (i["x"], i["any_done"]), dict(sums=o[algo], workspace=ws)
+        raise KeyError(algo)
+
+    def call(self, algo: str):
+        fn, args, kwargs = self.spec(algo)
+        fn(*args, **kwargs)
         self.launches += 1
+
+    def prepared(self, algo: str):
+        """The same call with its arguments marshalled once (binding.prepare)."""
+        fn, args, kwargs = self.spec(algo)
+        return self.B.prepare(fn, *args, **kwargs)
 
     def step(self, timed=None, events=None):
         """One pass of the seven calls.  `timed` = index of the one call of this step that is
@@ -753,6 +762,21 @@ def sweep_case(torch, B, ro, algo: str, use_truncs: bool, hbm_peak: float, l2_by
         e1.record()
         torch.cuda.synchronize()
         full_call_us.append(1e3 * e0.elapsed_time(e1) / R)
+    # ... and through prepared calls (arguments marshalled once, then only the C call)
+    prepared_us = []
+    if ceilings:
+        steps = [b.prepared(algo) for b in sets]
+        h = torch.cuda.current_stream().cuda_stream
+        for _ in range(trials):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            e0.record()
+            for st in steps:
+                st(h)
+            e1.record()
+            torch.cuda.synchronize()
+            prepared_us.append(1e3 * e0.elapsed_time(e1) / R)
+        del steps
     best = min(per_call_us)
     gbs = algo_bytes / (best * 1e-6) / 1e9
     del sets, graph
@@ -769,7 +793,7 @@ def sweep_case(torch, B, ro, algo: str, use_truncs: bool, hbm_peak: float, l2_by
             "memcpy_ceiling_us": round(memcpy_us, 3), "frac_of_memcpy_ceiling": round(memcpy_us / best, 4),
             "frac_of_copy_ceiling": round(gbs / ceiling_gbs, 4),
             "us_per_call_median": round(statistics.median(per_call_us), 3),
-            "full_call_us": round(min(full_call_us), 3), "env_steps_per_s": ro.N * ro.T / (best * 1e-6),
+            "full_call_us": round(min(full_call_us), 3), "prepared_call_us": round(min(prepared_us), 3), "env_steps_per_s": ro.N * ro.T / (best * 1e-6),
             "algorithmic_bytes": algo_bytes, "gbs": round(gbs, 1), "frac_of_peak": round(gbs / hbm_peak, 4),
             "rotating_sets": R, "l2": "cold (rotating buffer sets > 3x L2)", "timing": "CUDA-graph replay of the rotating launches"}
 

@@ -87,6 +87,76 @@ class RlcsError(RuntimeError):
         super().__init__(lib().rlcs_status_string(status).decode())
 
 
+_recording = threading.local()        # .calls: list while prepare() runs a wrapper, absent otherwise
+
+
+class _Recorder:
+    """Stands in for the library while prepare() runs a wrapper: records (C function, arguments) of
+    every compute call instead of making it; anything else (size queries, ...) goes to the library."""
+
+    def __init__(self, real):
+        self._real = real
+
+    def __getattr__(self, name):
+        fn = getattr(self._real, name)
+        compute = (fn.restype is _int and fn.argtypes and fn.argtypes[-1] is _vp and not name.startswith("rlcs_debug")
+                   and name not in ("rlcs_workspace_init", "rlcs_last_device_status", "rlcs_no_alloc_last_device_status"))
+        if not compute:
+            return fn
+
+        def record(*args):
+            _recording.calls.append((fn, args))
+            return RLCS_OK
+        return record
+
+
+class Prepared:
+    """A call whose arguments were checked and marshalled once (prepare()).  Calling it only makes the
+    C call(s) -- a few microseconds of host time instead of the 12-28 that dtype, shape, device and
+    pointer marshalling cost per call -- on the current stream, or on `stream_handle` (a raw
+    cudaStream_t as int) when given.  The tensors are kept alive by this object; `outputs` is what the
+    wrapper would have returned.  The caller must not free or resize them while it is in use, and must
+    call it with the device current on which it was prepared."""
+
+    def __init__(self, calls, outputs, keep):
+        self._calls, self.outputs, self._keep = calls, outputs, keep
+
+    def __call__(self, stream_handle=None):
+        h = _stream() if stream_handle is None else stream_handle
+        for fn, args in self._calls:
+            st = fn(*args[:-1], h)
+            if st != RLCS_OK:
+                raise RlcsError(st)
+        return self.outputs
+
+
+def prepare(wrapper, *args, **kwargs) -> Prepared:
+    """Run one of this module's rlcs_* wrappers in recording mode: all of its checks happen now,
+    outputs and workspace are allocated (and the workspace initialised) now -- pass them in to control
+    that -- and no kernel is launched.  Not thread-safe: no other thread may use this module meanwhile.
+    The returned object repeats the call at C-call cost, e.g. inside a training loop on fixed buffers:
+
+        step = prepare(rlcs_gae, rewards, values, dones, gamma=0.99, lam=0.95, workspace=ws)
+        ...
+        adv, ret = step()
+    """
+    real = lib()
+    global _lib
+    _recording.calls = []
+    with _lock:
+        _lib = _Recorder(real)
+    try:
+        outputs = wrapper(*args, **kwargs)
+        calls = list(_recording.calls)
+    finally:
+        with _lock:
+            _lib = real
+        del _recording.calls
+    if not calls:
+        raise ValueError("prepare() takes one of the rlcs_* compute wrappers of this module")
+    return Prepared(calls, outputs, (args, kwargs))
+
+
 def lib() -> ctypes.CDLL:
     """The loaded C library (loaded once).  Raises if it has not been built."""
     global _lib

@@ -213,6 +213,27 @@ def test_binding_rejects_tensors_and_workspaces_of_another_device(monkeypatch):
         binding._ptr(_FakeTensor(0), "f32")
 
 
+def test_prepare_records_the_call_instead_of_making_it(monkeypatch):
+    """prepare() runs a wrapper with all its checks but makes no launch: it returns the C function and
+    the marshalled arguments, to be repeated at C-call cost."""
+    import torch
+    from paper_2608_17641_b200 import binding
+    binding.lib()
+    monkeypatch.setattr(binding, "_current_device", lambda: 0)
+    monkeypatch.setattr(binding, "_stream", lambda stream=None: 1234)
+    x, d, z = _FakeTensor(0), _FakeTensor(0, torch.uint8), _FakeTensor(0)
+    step = binding.prepare(binding.rlcs_elig_trace, x, d, gamma=0.9, lam=0.5, traces=z)
+    assert step.outputs is z and len(step._calls) == 1
+    fn, args = step._calls[0]
+    assert fn is binding.lib().rlcs_elig_trace                     # the library is back in place
+    assert args[0] == x.data_ptr() and args[2] == z.data_ptr() and tuple(args[3:5]) == (2, 8) and args[-1] == 1234
+    with pytest.raises(TypeError):                                   # checks still run at prepare time
+        binding.prepare(binding.rlcs_elig_trace, _FakeTensor(0, torch.float64), d, gamma=0.9, lam=0.5, traces=z)
+    assert not isinstance(binding.lib(), binding._Recorder)
+    with pytest.raises(ValueError):
+        binding.prepare(lambda: None)
+
+
 def test_front_end_keeps_one_workspace_per_stream(monkeypatch):
     """Calls on different streams must not share carry records: the cache key holds the stream."""
     from paper_2608_17641_b200 import api

@@ -96,3 +96,36 @@ def test_front_end_argument_errors(env):
         api.compute_eligibility_traces(r, d, beta=r)
     with pytest.raises(TypeError):
         api.compute_gae(r.cpu(), r.cpu(), d.cpu())               # there is no CPU path
+
+
+def test_prepared_calls_repeat_the_direct_call(env, oracle):
+    """binding.prepare(): arguments marshalled once, then only the C call -- same bits as the wrapper."""
+    api, B, W, torch = env
+    ro = W.make_rollout(130, 48, 999, p_done=0.01, p_trunc=0.01)
+    up = lambda a: guarded_upload(a)
+    r, v, d, tr, bv, bt = up(ro.rewards), up(ro.values), up(ro.dones), up(ro.truncs), up(ro.trunc_bootstrap), up(ro.bootstrap)
+    ws = B.Workspace(ro.N, ro.T)
+    want_adv, want_ret = B.rlcs_gae(r, v, d, tr, bv, bt, gamma=0.99, lam=0.95, workspace=ws)
+    step = B.prepare(B.rlcs_gae, r, v, d, tr, bv, bt, gamma=0.99, lam=0.95, workspace=ws)
+    adv, ret = step.outputs
+    adv.fill_(float("nan"))
+    for _ in range(3):
+        out = step()
+        assert out[0] is adv
+    torch.cuda.synchronize()
+    assert torch.equal(adv, want_adv) and torch.equal(ret, want_ret) and ws.device_status() == 0
+    # a wrapper that makes three launches and creates its own workspace
+    norm = B.prepare(B.rlcs_gae_normalized, r, v, d, tr, bv, bt, gamma=0.99, lam=0.95, eps=1e-8, ddof=1)
+    assert len(norm._calls) == 1
+    nadv, _ = norm()
+    torch.cuda.synchronize()
+    want, _ = B.rlcs_gae_normalized(r, v, d, tr, bv, bt, gamma=0.99, lam=0.95, eps=1e-8, ddof=1)
+    assert torch.equal(nadv, want)
+    # on an explicit stream handle
+    s = torch.cuda.Stream()
+    s.wait_stream(torch.cuda.current_stream())
+    adv.fill_(0)
+    torch.cuda.synchronize()
+    step(s.cuda_stream)
+    s.synchronize()
+    assert torch.equal(adv, want_adv)
