@@ -587,6 +587,24 @@ __device__ __forceinline__ void issue_trunc_values(Chunk<ALGO, TRUNC, ITEMS>& c,
                     c.ov[8 * k + j] = (((j < 4 ? n0 : n1) & bit) != 0) ? x[j] : 0.f;
                 }
             }
+        } else if constexpr (SECTORS && kIoBf16 && ITEMS == 16 && ALGO != kTdLambda) {
+            // bfloat16 tensors: a thread's 16 steps are exactly one 32-byte sector
+            unsigned need[4], any = 0;
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                need[k] = nonzero_bytes(c.tw[k]) & ~nonzero_bytes(c.dw[k]);
+                any |= need[k];
+            }
+            unsigned w[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+            asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.u32 q, %9, 0;\n\t"
+                         "@q ld.global.nc.L1::no_allocate.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];\n\t}"
+                         : "+r"(w[0]), "+r"(w[1]), "+r"(w[2]), "+r"(w[3]), "+r"(w[4]), "+r"(w[5]), "+r"(w[6]), "+r"(w[7])
+                         : "l"(p.trunc_boot + i0), "r"(any));
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+                const float x = __uint_as_float((j & 1) ? (w[j / 2] & 0xffff0000u) : (w[j / 2] << 16));
+                c.ov[j] = ((need[j / 4] & (0x80u << (8 * (j % 4)))) != 0) ? x : 0.f;
+            }
         } else {
 #pragma unroll
             for (int j = 0; j < ITEMS; ++j)
