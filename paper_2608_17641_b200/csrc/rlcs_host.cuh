@@ -87,15 +87,13 @@ int choose_variant_unchecked(int algo, bool trunc, int64_t total, int64_t T) {
         return total <= (int64_t(1) << 19) ? 1 : 6;
     }
     if (RLCS_NS::kIoBf16) {
-        // 16 steps per thread (one 32-byte access per tensor); with half the bytes per step the kernels
-        // are bound by issue slots and latency, and more resident blocks pay even with a few spills
-        if (!trunc) return 18;
-        switch (algo) {
-            case RLCS_NS::kGae:
-            case RLCS_NS::kTdLambda:
-            case RLCS_NS::kDisc: return 20;
-            default: return 19;
-        }
+        // 16 steps per thread (one 32-byte access per tensor).  With half the bytes per step the kernels
+        // are bound by issue slots and latency, and resident blocks pay even with a few spills: every
+        // algorithm with truncation handling runs fastest at 8 blocks per SM (measured over all built
+        // shapes at 16384 x 2048: Retrace 0.82 -> 0.90, V-trace 0.75 -> 0.77 against 6 blocks), and the
+        // three lightest kernels at 10 (discounted return 0.70 -> 0.74, forward scans 0.81 -> 0.84).
+        if (algo == RLCS_NS::kDisc || algo == RLCS_NS::kElig || algo == RLCS_NS::kPrefix) return 21;
+        return trunc ? 20 : 18;
     }
     switch (algo) {
         case RLCS_NS::kGae: return trunc ? 19 : 0;

@@ -45,7 +45,7 @@ cudaError_t launch_scan(Kernel kernel, unsigned grid, unsigned block, size_t sme
 // stages == 0: scan_kernel (one tile per block).  stages > 0: scan_kernel_tma (persistent blocks,
 // bulk-copy ring of that many tiles; min_blocks = blocks per SM it is compiled and sized for).
 struct TileVariant { int threads, items, min_blocks, stages; };
-constexpr int kNumVariants = 21;
+constexpr int kNumVariants = 22;
 constexpr TileVariant kVariants[kNumVariants] = {
     {256, 8, 4, 0},    //  0: 2048 steps per tile
     {128, 4, 8, 0},    //  1:  512
@@ -68,6 +68,7 @@ constexpr TileVariant kVariants[kNumVariants] = {
     {128, 16, 5, 0},   // 18: 2048, 16 steps per thread
     {128, 16, 6, 0},   // 19: 2048, 16 steps per thread, at most 80 registers
     {128, 16, 8, 0},   // 20: 2048, 16 steps per thread, at most 64 registers
+    {128, 16, 10, 0},  // 21: 2048, 16 steps per thread, at most 48 registers (bfloat16 build only)
 };
 // Which rows of the table are compiled.  The default build holds the shapes the selection in
 // choose_variant() can return (0, 1, 5, 6, 18, 19, 20) and two persistent bulk-copy ring shapes (8, 11)
@@ -82,7 +83,7 @@ constexpr bool kAllVariants = false;
 #endif
 __host__ __device__ constexpr bool variant_built(int v) {
     if (kIoBf16) return v == 0 || v == 5 || v == 6 || v >= 18;
-    return kAllVariants || v == 0 || v == 1 || v == 5 || v == 6 || v == 8 || v == 11 || v >= 18;
+    return kAllVariants || v == 0 || v == 1 || v == 5 || v == 6 || v == 8 || v == 11 || (v >= 18 && v <= 20);
 }
 __host__ __device__ constexpr bool variant_built_for(int algo, int v) {
     if (!variant_built(v)) return false;

@@ -19,7 +19,7 @@ pytestmark = pytest.mark.gpu
 
 FLOAT_KEYS = ("rewards", "values", "bootstrap", "trunc_bootstrap", "q_sa", "expected_q", "log_rhos", "x")
 BACKWARD = ("gae", "vtrace", "retrace", "td_lambda", "discounted_return")
-BUILT_VARIANTS = (0, 5, 6, 18, 19, 20)
+BUILT_VARIANTS = (0, 5, 6, 18, 19, 20, 21)
 
 
 @pytest.fixture(scope="module")
