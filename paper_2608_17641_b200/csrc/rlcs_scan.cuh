@@ -763,6 +763,12 @@ __device__ __forceinline__ long long take_tile(const ScanParams& p, unsigned& ep
 // waits on it (cluster_exit_wait) after its stores, so that wait overlaps the rest of the tile.
 __device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
 __device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
+// The exit barrier publishes no data -- it only says "I have finished reading your shared memory" (the
+// remote values were consumed by the shuffles before it) -- so its arrive needs no release fence; and
+// of the first barrier's arrivals only the one thread that wrote the aggregate has something to
+// publish, which it does with a fence of its own.  (Measured on 64 x 16384: GAE 6.6 -> 6.0 us,
+// discounted return 4.5 -> 4.3 us against release semantics on every arrive.)
+__device__ __forceinline__ void cluster_arrive_relaxed() { asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory"); }
 __device__ __forceinline__ void cluster_exit_wait() { cluster_wait(); }
 
 template <int NW>
@@ -771,8 +777,11 @@ __device__ __forceinline__ float cluster_carry(Pair tile_agg, ScanSmem<NW>& sm, 
     cg::cluster_group cl = cg::this_cluster();
     const unsigned r = cl.block_rank();
     const int lane = threadIdx.x & 31;
-    if (threadIdx.x == 0) sm.cl_agg = tile_agg;
-    cluster_arrive();
+    if (threadIdx.x == 0) {
+        sm.cl_agg = tile_agg;
+        asm volatile("fence.acq_rel.cluster;" ::: "memory");   // the one writer publishes; nobody else needs a release fence
+    }
+    cluster_arrive_relaxed();
     cluster_wait();                                            // every block's aggregate is in place
     if (threadIdx.x < 32) {
         Pair q = {0.f, 0.f};                                   // lanes >= r: terminators
@@ -789,7 +798,7 @@ __device__ __forceinline__ float cluster_carry(Pair tile_agg, ScanSmem<NW>& sm, 
         }
         if (lane == 0) sm.carry[buf] = cur.a;
     }
-    cluster_arrive();                                          // this thread reads no remote memory any more
+    cluster_arrive_relaxed();                                  // this thread reads no remote memory any more
     __syncthreads();                                           // the carry is visible to the block
     return sm.carry[buf];
 }
