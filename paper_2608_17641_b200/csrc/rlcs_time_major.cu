@@ -168,13 +168,13 @@ template <int ALGO, bool TRUNC>
 __device__ __forceinline__ Coef back_coef(const StepIn& in, const TmParams& p, unsigned last, float bootv, float v_next,
                                           float lr_next) {
     // last: all ones at the window's final step t = T-1, else 0
-    const unsigned term = ones_if(in.dn);
-    const unsigned trunc = TRUNC ? (ones_if(in.tr) & ~term) : 0u;
-    const unsigned cont = ~(term | trunc | last);
-    // successor value: 0 after a termination, the stored continuation value after a truncation, the
-    // bootstrap at the window edge, else the buffer's next entry
-    float succ = blend(last, bootv, v_next);
-    succ = __uint_as_float((__float_as_uint(succ) & ~(term | trunc)) | (TRUNC ? __float_as_uint(in.bv) : 0u));
+    // The step is cut (nothing is carried in) after a termination or a truncation: one test of both
+    // flag bytes.  The successor value is then the truncation's continuation value -- in.bv, which
+    // is 0 unless the step is a truncation that is not also a termination -- else the bootstrap at the
+    // window edge, else the buffer's next entry.
+    const unsigned cut = ones_if(TRUNC ? (in.dn | in.tr) : in.dn);
+    const unsigned cont = ~(cut | last);
+    const float succ = blend(cut, TRUNC ? in.bv : 0.f, blend(last, bootv, v_next));
     Coef c;
     c.pg = 0.f;
     if constexpr (ALGO == kGae) {
@@ -501,28 +501,63 @@ __device__ __forceinline__ void issue_masks(const StageView<ALGO, TRUNC, W, C>& 
     }
 }
 
+// Which of a warp's KR rows of a stage hold a set flag: the rows are KR * 32 C adjacent bytes of the
+// mask ring, every lane takes KR C of them (32 / KR lanes per row) and one ballot shares the answer.
+// Bit 32 / KR * u + x: lane x's share of row u has a nonzero byte.  All 32 lanes must call.
+template <int KR, int C>
+__device__ __forceinline__ unsigned row_flag_bits(const uint8_t* rows, int lane) {
+    constexpr int B = KR * C;
+    static_assert(B == 4 || B == 8 || B == 16 || B == 32, "a lane's share is one or two vector loads");
+    unsigned any;
+    if constexpr (B == 4) {
+        any = *reinterpret_cast<const unsigned*>(rows + 4 * lane);
+    } else if constexpr (B == 8) {
+        const uint2 v = *reinterpret_cast<const uint2*>(rows + 8 * lane);
+        any = v.x | v.y;
+    } else {
+        any = 0;
+#pragma unroll
+        for (int h = 0; h < B / 16; ++h) {
+            const uint4 v = *reinterpret_cast<const uint4*>(rows + B * lane + 16 * h);
+            any |= v.x | v.y | v.z | v.w;
+        }
+    }
+    return __ballot_sync(0xffffffffu, any != 0);
+}
+template <int KR>
+__device__ __forceinline__ bool row_flagged(unsigned bits, int u) {
+    constexpr int L = 32 / KR;
+    return ((bits >> (L * u)) & ((1u << L) - 1u)) != 0;
+}
+
 // truncation continuation values of `nvalid` rows from row0 of a stage whose masks have landed;
-// i = flat index of the first of them for this lane's first column
+// i = flat index of the first of them for this lane's first column.  With flags as rare as they are
+// most rows of 32 C columns hold no truncation at all: those are skipped on a warp-uniform test
+// (no divergence), and only the others read their flags lane by lane.
 template <int ALGO, bool TRUNC, int W, int C>
 __device__ __forceinline__ void stage_bv(float (&bv)[tm_rows(ALGO)][C], const StageView<ALGO, TRUNC, W, C>& sv, const TmParams& p,
-                                         long long i, long long rowstep, int row0, int nvalid, int lane, unsigned write_mask) {
+                                         long long i, int rowbytes, int row0, int nvalid, int lane, unsigned write_mask) {
     constexpr int KR = tm_rows(ALGO);
     if (nvalid <= 0) return;                                 // past the chunk: the values are never used
-    auto rows = [&](auto full) {
-        constexpr bool FULL = decltype(full)::value;
+    const unsigned trbits = row_flag_bits<KR, C>(sv.m(1, row0), lane);
 #pragma unroll
-        for (int u = 0; u < KR; ++u) {
+    for (int u = 0; u < KR; ++u)
+#pragma unroll
+        for (int c = 0; c < C; ++c) bv[u][c] = 0.f;
+    if (trbits == 0) return;
+#pragma unroll
+    for (int u = 0; u < KR; ++u) {
+        if (row_flagged<KR>(trbits, u)) {
             unsigned tr[C], dn[C];
             lds_m<C>(sv.m(1, row0 + u), lane, tr);
             lds_m<C>(sv.m(0, row0 + u), lane, dn);
-            const unsigned rowmask = FULL ? write_mask : (write_mask & (u < nvalid ? ~0u : 0u));
+            const unsigned rowmask = write_mask & (u < nvalid ? ~0u : 0u);
+            // rowbytes * u is one multiply-add onto the 64-bit address (u is a constant here)
+            const float* const src = reinterpret_cast<const float*>(reinterpret_cast<const char*>(p.trunc_boot + i) + (long long)rowbytes * u);
 #pragma unroll
-            for (int c = 0; c < C; ++c) bv[u][c] = ldg_if_mask(p.trunc_boot + i + c, ones_if(tr[c]) & ~ones_if(dn[c]) & rowmask);
-            i += rowstep;
+            for (int c = 0; c < C; ++c) bv[u][c] = ldg_if_mask(src + c, ones_if(tr[c]) & ~ones_if(dn[c]) & rowmask);
         }
-    };
-    if (nvalid >= KR) rows(std::true_type{});
-    else rows(std::false_type{});
+    }
 }
 
 __device__ __forceinline__ int wrap_next(int x, int n) { return x + 1 == n ? 0 : x + 1; }
@@ -539,7 +574,9 @@ __device__ __forceinline__ int wrap_prev(int x, int n) { return x == 0 ? n - 1 :
 //
 // Copies are committed in groups {floats of stage s, masks of stage s+2}: when a stage's floats
 // have landed so have the masks two stages on, and the sparse truncation values they point at are
-// requested two stages before their use (registers bv1, bv2).
+// requested two stages before their use (registers bv1, bv2).  One stage is not enough: with the
+// ring's 16 MB in flight a load takes 2.5 us or more to come back, a stage lasts under 2 (measured:
+// GAE 0.80 -> 0.65 of the copy bandwidth at 16384 x 2048 with a distance of one stage).
 // MODE as in tm_kernel.
 // block_walk: chunk k of the block's 32 C columns from n0.  A: in, the carry into the chunk (MODE 0: 0;
 // MODE 1: 0); out, the recurrence value after the chunk's last step.  P: out, the product of the
@@ -616,11 +653,13 @@ __device__ __forceinline__ void block_walk(const TmParams& p, const long long n0
     long long iw = cp.i_first + cp.rowstep * row0 + C * lane;
     int left = (int)len - row0;                              // steps from this warp's first row to the chunk's end
     const long long stagestep = cp.rowstep * R;
+    const int rowbytes = (int)(cp.rowstep * 4);              // |N| * 4 fits: the host routes larger N to tm_kernel
+    const bool all_write = __all_sync(0xffffffffu, write);
     if constexpr (TRUNC) {
         cp_async_wait(S - 2);                                // stage 0 and the masks of stages 0..2 have landed
         __syncthreads();
-        stage_bv<ALGO, TRUNC>(bvc, SV{nullptr, mring}, p, iw, cp.rowstep, row0, left, lane, write_mask);
-        stage_bv<ALGO, TRUNC>(bv1, SV{nullptr, mring + mstage}, p, iw + stagestep, cp.rowstep, row0, left - R, lane, write_mask);
+        stage_bv<ALGO, TRUNC>(bvc, SV{nullptr, mring}, p, iw, rowbytes, row0, left, lane, write_mask);
+        stage_bv<ALGO, TRUNC>(bv1, SV{nullptr, mring + mstage}, p, iw + stagestep, rowbytes, row0, left - R, lane, write_mask);
     }
     int fs = 0, ms = 0;                                      // ring slots of stage j
     for (unsigned j = 0; j < nst; ++j) {
@@ -631,7 +670,7 @@ __device__ __forceinline__ void block_walk(const TmParams& p, const long long n0
         const int nvalid = left < KR ? (left < 0 ? 0 : left) : KR;
         if constexpr (TRUNC) {
             const int ms2 = ms + 2 >= SM ? ms + 2 - SM : ms + 2;
-            stage_bv<ALGO, TRUNC>(bv2, SV{nullptr, mring + ms2 * mstage}, p, iw + 2 * stagestep, cp.rowstep, row0, left - 2 * R,
+            stage_bv<ALGO, TRUNC>(bv2, SV{nullptr, mring + ms2 * mstage}, p, iw + 2 * stagestep, rowbytes, row0, left - 2 * R,
                                   lane, write_mask);
         }
         // neighbour of this warp's first step: the row before it in the stage, the last row of the
@@ -761,17 +800,21 @@ __device__ __forceinline__ void block_walk(const TmParams& p, const long long n0
                 P[c] *= ab.y;
             }
         }
-        // pass 2: one FMA per step, then the outputs
+        // pass 2: one FMA per step, then the outputs.  The common case -- every row of the warp inside the
+        // chunk, every lane inside N -- has no guard at all; whether there is a second output tensor is
+        // decided once per stage, not per store.
         if (MODE != 1) {
-            auto pass2 = [&](auto full) {
+            auto pass2 = [&](auto full, auto both) {
                 constexpr bool FULL = decltype(full)::value;
+                constexpr bool BOTH = decltype(both)::value;
                 float prev[C];
 #pragma unroll
                 for (int c = 0; c < C; ++c) prev[c] = cin[c];
-                long long i = iw;
+                char* const dst0 = reinterpret_cast<char*>(p.out0 + iw);
+                char* const dst1 = BOTH ? reinterpret_cast<char*>(p.out1 + iw) : nullptr;
 #pragma unroll
                 for (int u = 0; u < KR; ++u) {
-                    if ((FULL || u < nvalid) && write) {
+                    if (FULL || (u < nvalid && write)) {
                         float o0[C], o1[C];
 #pragma unroll
                         for (int c = 0; c < C; ++c) {
@@ -782,16 +825,24 @@ __device__ __forceinline__ void block_walk(const TmParams& p, const long long n0
                             else { o0[c] = val; o1[c] = 0.f; }
                             prev[c] = val;
                         }
-                        stg_f<C>(p.out0 + i, o0);
-                        if constexpr (ALGO == kGae || ALGO == kVtrace) {
-                            if (p.out1 != nullptr) stg_f<C>(p.out1 + i, o1);
-                        }
+                        stg_f<C>(reinterpret_cast<float*>(dst0 + (long long)rowbytes * u), o0);
+                        if constexpr (BOTH) stg_f<C>(reinterpret_cast<float*>(dst1 + (long long)rowbytes * u), o1);
                     }
-                    i += cp.rowstep;
                 }
             };
-            if (nvalid == KR) pass2(std::true_type{});
-            else pass2(std::false_type{});
+            const bool fast = nvalid == KR && all_write;
+            if constexpr (ALGO == kGae || ALGO == kVtrace) {
+                if (p.out1 != nullptr) {
+                    if (fast) pass2(std::true_type{}, std::true_type{});
+                    else pass2(std::false_type{}, std::true_type{});
+                } else {
+                    if (fast) pass2(std::true_type{}, std::false_type{});
+                    else pass2(std::false_type{}, std::false_type{});
+                }
+            } else {
+                if (fast) pass2(std::true_type{}, std::false_type{});
+                else pass2(std::false_type{}, std::false_type{});
+            }
         }
         // everyone is past the barrier, hence done with stage j-1: refill its slots
         {
@@ -1126,7 +1177,8 @@ inline bool unit(float v) { return v >= 0.f && v <= 1.f; }
 
 // the staged kernels copy 16-byte pieces of every per-step input
 bool can_stage(const TmParams& p) {
-    if (p.N % 16 != 0) return false;
+    // (the ring kernels step from row to row with a 32-bit byte offset)
+    if (p.N % 16 != 0 || p.N > (1ll << 28)) return false;
     const void* in[] = {p.f0, p.f1, p.f2, p.f3, p.dones, p.truncs};
     for (const void* q : in)
         if (q != nullptr && !aligned16(q)) return false;
@@ -1197,7 +1249,7 @@ bool vec_trace_block_cuts(int64_t N, int64_t T, int64_t D, bool perdim) {
 // rows and components alone, or from the chunks of a cut time axis
 bool vec_trace_block_shape_ok(int64_t N, int64_t T, int64_t D, bool perdim) {
     if (g_force_path == 1) return false;
-    if (D % 4 != 0 || D < 32 || T < 64 || N > 65535) return false;
+    if (D % 4 != 0 || D < 32 || D > (1ll << 28) || T < 64 || N > 65535) return false;
     return (D + 31) / 32 * N >= 96 || vec_trace_block_cuts(N, T, D, perdim);
 }
 bool vec_trace_block_usable(const float* x, const float* beta, int64_t N, int64_t T, int64_t D) {
