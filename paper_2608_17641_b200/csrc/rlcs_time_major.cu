@@ -877,6 +877,9 @@ __device__ __forceinline__ TmParams batch_slice(const TmParams& p_in, unsigned z
     return p;
 }
 
+// (No register cap: holding these kernels to the 80 registers that six 128-thread blocks per SM would
+// need was measured and loses -- the discounted return spills and halves, V-trace and Retrace lose
+// 0.03-0.10 of the copy bandwidth -- although the ring is planned for up to six blocks.)
 template <int ALGO, bool TRUNC, int MODE, int W, int C>
 __global__ void __launch_bounds__(32 * W) tm_block_kernel(const TmParams p_in) {
     const TmParams p = batch_slice<ALGO>(p_in, blockIdx.z);
