@@ -452,6 +452,11 @@ __device__ __forceinline__ void lds_m(const uint8_t* row, int lane, unsigned (&x
     else x[0] = row[lane];
 }
 template <int C>
+__device__ __forceinline__ void sts_f(float* row, int lane, const float (&x)[C]) {
+    if constexpr (C == 2) *reinterpret_cast<float2*>(row + 2 * lane) = make_float2(x[0], x[1]);
+    else row[lane] = x[0];
+}
+template <int C>
 __device__ __forceinline__ void stg_f(float* p, const float (&x)[C]) {
     if constexpr (C == 2) __stcs(reinterpret_cast<float2*>(p), make_float2(x[0], x[1]));
     else __stcs(p, x[0]);
@@ -577,12 +582,20 @@ __device__ __forceinline__ int wrap_prev(int x, int n) { return x == 0 ? n - 1 :
 // requested two stages before their use (registers bv1, bv2).  One stage is not enough: with the
 // ring's 16 MB in flight a load takes 2.5 us or more to come back, a stage lasts under 2 (measured:
 // GAE 0.80 -> 0.65 of the copy bandwidth at 16384 x 2048 with a distance of one stage).
-// MODE as in tm_kernel.
+// MODE as in tm_kernel, plus MODE 3 for the chained kernel of the vector traces (one flag per
+// timestep, so a cut holds for all columns at once): the walk starts from carry 0; the steps from the
+// first cut on do not depend on the chunk's incoming carry and are written as in MODE 0; the
+// `qdefer` steps before it are not written -- their value from carry 0 replaces the step's f0 entry in
+// the ring (which only its own thread reads) and, with a decay tensor, the product of the betas from
+// the chunk's first step up to and including it replaces the f1 entry -- so that the caller can finish
+// them once the carry is known, without walking the chunk again.  The ring must then hold the whole
+// chunk (stages >= the chunk's stage count, no slot refilled).
 // block_walk: chunk k of the block's 32 C columns from n0.  A: in, the carry into the chunk (MODE 0: 0;
 // MODE 1: 0); out, the recurrence value after the chunk's last step.  P: out, the product of the
 // chunk's betas.  Every thread returns the values of its own columns.
 template <int ALGO, bool TRUNC, int MODE, int W, int C>
-__device__ __forceinline__ void block_walk(const TmParams& p, const long long n0, const unsigned k, float (&A)[C], float (&P)[C]) {
+__device__ __forceinline__ void block_walk(const TmParams& p, const long long n0, const unsigned k, float (&A)[C], float (&P)[C],
+                                           const unsigned qdefer = 0) {
     constexpr bool FWD = tm_forward(ALGO);
     constexpr bool ROWMASK = tm_row_mask(ALGO);
     using SV = StageView<ALGO, TRUNC, W, C>;
@@ -787,15 +800,15 @@ __device__ __forceinline__ void block_walk(const TmParams& p, const long long n0
         }
         __syncthreads();
         // fold the warps' aggregates in scan order onto the block state
-        float cin[C];
+        float cin[C], pin[C];                                // value and beta product at the entry of this warp's rows
 #pragma unroll
-        for (int c = 0; c < C; ++c) cin[c] = A[c];
+        for (int c = 0; c < C; ++c) { cin[c] = A[c]; pin[c] = P[c]; }
 #pragma unroll
         for (int x = 0; x < W; ++x) {
 #pragma unroll
             for (int c = 0; c < C; ++c) {
                 const float2 ab = agg[((par * W + x) * 32 + lane) * C + c];
-                if (x == w) cin[c] = A[c];
+                if (x == w) { cin[c] = A[c]; if (MODE == 3 && tm_vec_beta(ALGO)) pin[c] = P[c]; }
                 A[c] = fmaf(ab.y, A[c], ab.x);
                 P[c] *= ab.y;
             }
@@ -825,8 +838,18 @@ __device__ __forceinline__ void block_walk(const TmParams& p, const long long n0
                             else { o0[c] = val; o1[c] = 0.f; }
                             prev[c] = val;
                         }
-                        stg_f<C>(reinterpret_cast<float*>(dst0 + (long long)rowbytes * u), o0);
-                        if constexpr (BOTH) stg_f<C>(reinterpret_cast<float*>(dst1 + (long long)rowbytes * u), o1);
+                        if (MODE == 3 && j * R + row0 + u < qdefer) {      // (uniform over the warp)
+                            sts_f<C>(cur.f(0, row0 + u), lane, o0);
+                            if constexpr (tm_vec_beta(ALGO)) {
+                                float sens[C];
+#pragma unroll
+                                for (int c = 0; c < C; ++c) sens[c] = pb[u][c] * pin[c];
+                                sts_f<C>(cur.f(1, row0 + u), lane, sens);
+                            }
+                        } else {
+                            stg_f<C>(reinterpret_cast<float*>(dst0 + (long long)rowbytes * u), o0);
+                            if constexpr (BOTH) stg_f<C>(reinterpret_cast<float*>(dst1 + (long long)rowbytes * u), o1);
+                        }
                     }
                 }
             };
@@ -900,13 +923,15 @@ __global__ void __launch_bounds__(32 * W) tm_block_kernel(const TmParams p_in) {
     }
 }
 
-// The time axis cut without a second read from HBM: one launch, every block takes a (column block,
-// chunk) pair from a ticket counter -- chunk index slowest, so that the scan-order predecessors of a
-// chunk hold lower tickets and are running or done when it starts -- walks its chunk for the
-// aggregate (A, P) = (value after the last step from carry 0, product of betas), publishes it, looks
-// back for the carry into its chunk, publishes the value it carries out, and walks the chunk again
-// to write the outputs.  The second walk reads what the first brought into L2 moments before (the
-// chunks of all resident blocks together are a fraction of the L2).
+// The time axis cut without a second read from HBM and without a second walk: one launch, every block
+// takes a (column block, chunk) pair from a ticket counter -- chunk index slowest, so that the
+// scan-order predecessors of a chunk hold lower tickets and are running or done when it starts --
+// walks its chunk once from carry 0, writing the outputs that result and leaving every step's
+// sensitivity to the incoming carry in the ring (block_walk, MODE 3), publishes the aggregate
+// (A, P) = (value after the last step from carry 0, product of betas), looks back for the carry c
+// into its chunk, publishes the value it carries out, and adds sensitivity * c to the outputs of the
+// steps that c reaches: those before the chunk's first cut, a fifth of the chunk at the recipe's
+// flag rate, read back from L2 where the block wrote them moments before.
 //
 // Records are 16 bytes {value, kind, beta product, kind}, kind 0 = not yet (the call zeroes them),
 // 1 = aggregate, 2 = carried-out value; each 8-byte half carries the kind, so a record read while it
@@ -944,6 +969,7 @@ __device__ __forceinline__ float chained_carry(const TmParams& p, long long rec0
 template <int ALGO, bool TRUNC, int W, int C>
 __global__ void __launch_bounds__(32 * W) tm_block_chained_kernel(const TmParams p_in) {
     constexpr bool FWD = tm_forward(ALGO);
+    constexpr bool ONE_WALK = tm_row_mask(ALGO);             // vector traces: one flag per timestep
     __shared__ unsigned s_ticket;
     __shared__ float s_carry[32 * C];
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
@@ -959,10 +985,25 @@ __global__ void __launch_bounds__(32 * W) tm_block_chained_kernel(const TmParams
     const unsigned k = FWD ? ks : p.chunks - 1 - ks;
     const long long n0 = (long long)xb * (32 * C);
     const bool write = n0 + C * lane < p.N;
+    const unsigned t_lo = k * p.chunk, t_hi = min(p.T, t_lo + p.chunk), len = t_hi - t_lo;
+    // Steps the incoming carry reaches: those before the chunk's first cut (the carry into step t is
+    // cut iff dones[t-1]; chunk 0 takes no carry).  Every warp finds the bound for itself.
+    unsigned qdefer = 0;
+    if constexpr (ONE_WALK) {
+        if (ks > 0) {
+            qdefer = len;
+            for (unsigned q0 = 0; q0 < len; q0 += 32) {
+                const unsigned q = q0 + lane;
+                const bool cut = q < len && __ldg(p.dones + t_lo + q - 1) != 0;
+                const unsigned m = __ballot_sync(0xffffffffu, cut);
+                if (m != 0) { qdefer = q0 + (unsigned)__ffs((int)m) - 1; break; }
+            }
+        }
+    }
     float A[C], P[C];
 #pragma unroll
     for (int c = 0; c < C; ++c) A[c] = 0.f;
-    block_walk<ALGO, TRUNC, 1, W, C>(p, n0, k, A, P);
+    block_walk<ALGO, TRUNC, ONE_WALK ? 3 : 1, W, C>(p, n0, k, A, P, qdefer);
     if (w == 0) {
         const long long rec0 = (long long)z * p.chunks * p.npad + n0 + C * lane;
 #pragma unroll
@@ -978,10 +1019,39 @@ __global__ void __launch_bounds__(32 * W) tm_block_chained_kernel(const TmParams
             s_carry[C * lane + c] = carry;
         }
     }
-    __syncthreads();                                         // also: every warp is done with the ring
+    __syncthreads();                                         // the carries are there, and every warp is done with the walk
+    if constexpr (!ONE_WALK) {
 #pragma unroll
-    for (int c = 0; c < C; ++c) A[c] = s_carry[C * lane + c];
-    block_walk<ALGO, TRUNC, 2, W, C>(p, n0, k, A, P);
+        for (int c = 0; c < C; ++c) A[c] = s_carry[C * lane + c];
+        block_walk<ALGO, TRUNC, 2, W, C>(p, n0, k, A, P);
+    } else {
+        // Finish the deferred steps: value from carry 0 (ring, f0 entry) + sensitivity * carry.  Rows go
+        // round-robin over the warps.  With the shared decay the sensitivity of step q is decay^(q+1).
+        if (qdefer == 0 || !write) return;
+        using SV = StageView<ALGO, TRUNC, W, C>;
+        extern __shared__ __align__(16) unsigned char tm_smem[];
+        constexpr int R = SV::KR * W;
+        constexpr int fstage = R * SV::NF * 128 * C;
+        float c0[C];
+#pragma unroll
+        for (int c = 0; c < C; ++c) c0[c] = s_carry[C * lane + c];
+        float pw = p.decay, step = 1.f;                      // decay^(w+1), decay^W
+        if constexpr (!tm_vec_beta(ALGO)) {
+            for (int x = 0; x < w; ++x) pw *= p.decay;
+            for (int x = 0; x < W; ++x) step *= p.decay;
+        }
+        float* dst = p.out0 + (long long)t_lo * p.N + n0 + C * lane;
+        for (unsigned q = w; q < qdefer; q += W) {
+            const SV sv{tm_smem + (q / R) * fstage, nullptr};
+            float v[C], sens[C];
+            lds_f<C>(sv.f(0, q % R), lane, v);
+            if constexpr (tm_vec_beta(ALGO)) lds_f<C>(sv.f(1, q % R), lane, sens);
+#pragma unroll
+            for (int c = 0; c < C; ++c) v[c] = fmaf(tm_vec_beta(ALGO) ? sens[c] : pw, c0[c], v[c]);
+            stg_f<C>(dst + (long long)q * p.N, v);
+            pw *= step;
+        }
+    }
 }
 
 // Chain an environment's chunks in scan order: carry into chunk k = a_j + b_j * (carry into j) for the
@@ -1032,7 +1102,7 @@ void plan_chunks(long long N, long long T, unsigned* chunk, unsigned* chunks) {
 // are scarce (fewer than one or two per SM), else four.  The kernel is bound by issue slots and dependent-ALU latency as much as by
 // HBM, so resident warps come first: the ring is as deep as still lets min(blocks per SM, 6) blocks
 // share an SM, no deeper than keeps about 16 MB in flight over the grid, and at least 3.
-size_t plan_block(TmParams& p, int rows, int row_bytes, bool trunc, bool wide_ok) {
+size_t plan_block(TmParams& p, int rows, int row_bytes, bool trunc, bool wide_ok, bool whole_chunk = false) {
     int C = 1;
     const long long batch = p.batch > 0 ? p.batch : 1;
     if (wide_ok && (p.N + 63) / 64 * p.chunks * batch >= 2 * sm_count()) C = 2;
@@ -1057,6 +1127,9 @@ size_t plan_block(TmParams& p, int rows, int row_bytes, bool trunc, bool wide_ok
     if (S > kMaxStages) S = kMaxStages;
     while (S > 3 && resident * (block_bytes(S) + 1024) > smem) --S;
     if (S < 3) S = 3;
+    // the chained kernel of the vector traces keeps its chunk (about 32 KB) in the ring: the entries of
+    // the steps before the first cut are reused after the walk
+    if (whole_chunk && p.records != nullptr && S < nst) S = nst;
     p.stages = (int)S;
     p.warps_per_block = W;
     p.cols_per_lane = C;
@@ -1073,11 +1146,11 @@ bool allow_smem(K kernel, size_t bytes) {
     return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(smem_per_sm() - 1024)) == cudaSuccess;
 }
 
-// Chunks of the chained kernel: about 32 KB of inputs per block and chunk, so that the chunks of
-// all resident blocks stay in L2 between a block's two walks (measured with the profiler at
-// 64x8192x64, per-component decay: 270 MB read from DRAM for 268 MB of inputs; the kernel is bound
-// by issue slots, 70 % busy, not by HBM); a multiple of 64 steps (every stage size divides it), at
-// least 64.
+// Chunks of the chained kernel: about 32 KB of inputs per block and chunk.  The vector traces keep
+// the chunk in the ring while it is walked once (measured at 64 x 16384 x 64 / 16 x 65536 x 64 with a
+// decay tensor, fraction of the copy bandwidth: 16 KB 0.65 / 0.60, 32 KB 0.67 / 0.69, 64 KB 0.59 /
+// 0.58); the time-major entry points walk it twice, and the chunks of all resident blocks stay in L2
+// in between.  A multiple of 64 steps (every stage size divides it), at least 64.
 constexpr unsigned kChainedMinChunk = 64;
 unsigned chained_chunk_len(int row_bytes) {
     unsigned len = (32768u / (unsigned)row_bytes) / 64u * 64u;
@@ -1291,7 +1364,7 @@ int vec_trace_block(const float* x, const float* beta, const uint8_t* dones, flo
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
     auto go = [&](auto algo_tag) {
         constexpr int ALGO = decltype(algo_tag)::value;
-        const size_t smem = plan_block(p, tm_rows(ALGO), tm_row_bytes(ALGO, false), false, false);
+        const size_t smem = plan_block(p, tm_rows(ALGO), tm_row_bytes(ALGO, false), false, false, true);
         if (p.warps_per_block == 16) return launch_block<ALGO, false, 16, 1>(p, smem, s);
         if (p.warps_per_block == 8) return launch_block<ALGO, false, 8, 1>(p, smem, s);
         return launch_block<ALGO, false, 4, 1>(p, smem, s);
