@@ -692,6 +692,38 @@ def test_vector_trace_plans_agree(oracle, W, B, N, T, D, plan):
     assert_close(f"per-dimension trace, plan {plan}", gotb, oracle.elig_trace_vec_beta(x, beta, d))
 
 
+@pytest.mark.parametrize("p_flag", [0.0, 0.004, 0.02, 0.5])
+@pytest.mark.parametrize("N,T,D", [(3, 2100, 64), (2, 1024, 36), (5, 777, 128)])
+def test_vector_trace_chained_kernel_single_walk(oracle, W, B, N, T, D, p_flag):
+    """The chained kernel of the vector traces walks a chunk once and finishes the steps before the
+    chunk's first cut when the carry arrives: no cut at all (every step of every later chunk waits for
+    its carry), rare cuts, the recipe's rate, every other step cut, and cuts placed on the steps around
+    the chunk boundaries (256 steps with the shared decay, 128 with a decay tensor); the last chunk is
+    ragged.  gamma * lambda = 1 carries a chunk's value undamped through all later chunks."""
+    rng = np.random.default_rng(N * 131 + T * 7 + D + int(p_flag * 1000))
+    x = rng.standard_normal((N, T, D)).astype(np.float32)
+    beta = rng.uniform(0.5, 1.0, (N, T, D)).astype(np.float32)
+    d = (rng.random((N, T)) < p_flag).astype(np.uint8)
+    if p_flag > 0:
+        for t in (126, 127, 128, 255, 256, 257, 511, 512, 768):
+            if t < T:
+                d[t % N, t] = 1
+    xd, bd, dd = guarded_upload(x), guarded_upload(beta), guarded_upload(d)
+    B.rlcs_debug_vec_trace_plan(1, 0)
+    B.rlcs_debug_time_major_path(5)
+    try:
+        got = B.rlcs_elig_trace_vec(xd, dd, gamma=0.99, lam=0.95).cpu().numpy()
+        got1 = B.rlcs_elig_trace_vec(xd, dd, gamma=1.0, lam=1.0).cpu().numpy()
+        gotb = B.rlcs_elig_trace_vec_beta(xd, bd, dd).cpu().numpy()
+        assert np.array_equal(got, B.rlcs_elig_trace_vec(xd, dd, gamma=0.99, lam=0.95).cpu().numpy())
+    finally:
+        B.rlcs_debug_vec_trace_plan(0, 0)
+        B.rlcs_debug_time_major_path(0)
+    assert_close("vector trace, chained", got, oracle.elig_trace_vec(x, d, gamma=0.99, lam=0.95))
+    assert_close("vector trace, chained, undamped", got1, oracle.elig_trace_vec(x, d, gamma=1.0, lam=1.0))
+    assert_close("per-dimension trace, chained", gotb, oracle.elig_trace_vec_beta(x, beta, d))
+
+
 def test_per_dimension_beta_argument_checks(oracle, W, B):
     L = B.lib()
     P = 0x7f0000000000
