@@ -218,9 +218,14 @@ int rlcs_elig_trace(const float* x, const uint8_t* dones, float* traces, int64_t
  * components;  dones: [N, T], the combined flag as for rlcs_elig_trace.
  *   z_t = x_t + ((t > 0 and not dones_{t-1}) ? gamma*lambda * z_{t-1} : 0)        (z_t, x_t in R^D)
  * One pass over x when N*D is large enough to fill the GPU; otherwise the time axis is cut into
- * chunks and x is read twice (chunk ends, ordered carry chain, rescan), which needs `workspace` of
+ * chunks.  Where rows of D floats can be copied in 16-byte pieces (D a multiple of 4, D >= 32, x
+ * 16-byte aligned) one launch chains the chunks: each is walked once from carry 0, and the steps
+ * before its first cut are finished when the carry arrives from the records of the chunks before (a
+ * bounded wait, as for the time-major entry points below), so x is still read once; otherwise three
+ * launches read x twice (chunk ends, ordered carry chain, rescan).  Either way the result does not
+ * depend on timing.  A cut needs `workspace` of
  * rlcs_elig_trace_vec_workspace_bytes(N, T, D) bytes (0 when no cut is needed; no initialisation
- * required).  128-bit accesses when D is a multiple of 4 and x, traces are 16-byte aligned.
+ * required for the results; the status word is as described for the time-major entry points).  128-bit accesses when D is a multiple of 4 and x, traces are 16-byte aligned.
  * Limits: T < 2^31, D <= 2^24, N*T*D < 2^40.
  */
 int rlcs_elig_trace_vec(const float* x, const uint8_t* dones, float* traces, int64_t N, int64_t T, int64_t D,
