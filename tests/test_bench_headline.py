@@ -27,7 +27,7 @@ def _stub_headline():
     return bench.build_headline(value=413123456789.123, world=8, steps=200, warmup=5, ms_per_step=0.56912, workload=workload,
                                 clocks=clocks, e2e=e2e, launches=1400, roofline=roofline, cpu_baseline=cpu,
                                 per_algorithm_frac={a: 0.9876 for a in bench.ALGOS}, small_frac=small,
-                                detail_file="gpurun_out/bench_detail.json")
+                                detail_file="out/bench_detail.json")
 
 
 def test_headline_is_short_and_complete():
