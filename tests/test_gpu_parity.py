@@ -184,6 +184,8 @@ def test_one_block_per_row_agrees_with_the_carry_between_blocks(oracle, W, B, va
 
 def test_one_block_per_row_is_the_default_with_many_rows(oracle, W, B):
     """Enough rows to fill the GPU: the row kernel is what runs (no carry workspace is needed)."""
+    if BASE_VARIANT >= 0:
+        pytest.skip("about the library's own choice of tile shape")
     N, T = 1200, 2064                                     # 2048 + one chunk of 16: no tile shape is filled to 70 % by such rows
     assert B.lib().rlcs_gae_carry_bytes(N, T, 1, 1) > 0   # ... so these rows are carried between blocks
     assert B.lib().rlcs_gae_carry_bytes(1200, 4112, 1, 1) == 0      # 4112 = 5 tiles of 1024 at 80 %: the 1024-step shape is taken
@@ -338,9 +340,10 @@ def test_large_problem_variants_with_carry(oracle, W, B):
     finally:
         B.rlcs_debug_set_row_blocks(-1)
     # the default for this shape: an 8-step tile shape that splits rows of 3000 into whole chunks, one block per row
-    info = B.rlcs_debug_variant_for("gae", True, ro.N, ro.T)
-    assert BASE_VARIANT != -1 or info["steps_per_thread"] == 8, info
-    compare_all(oracle, ro, workspace=None)
+    if BASE_VARIANT == -1:
+        info = B.rlcs_debug_variant_for("gae", True, ro.N, ro.T)
+        assert info["steps_per_thread"] == 8, info
+        compare_all(oracle, ro, workspace=None)
 
 
 @pytest.mark.parametrize("N,T,variant", [(5, 4096, 0), (3, 16384, 0), (64, 2048, 6), (7, 8192, 6), (9, 3072, 6), (2, 16384, 5),
