@@ -176,6 +176,9 @@ int rlcs_retrace(const float* rewards, const float* q_sa, const float* expected_
  * not depend on T.  Rows are read with 256-bit loads when A is 4, 8 or 16 and the three [N,T,A]
  * pointers are 32-byte aligned (for A = 4 and 8 the mu rows are read whole as well: a gather would
  * touch every sector anyway).  Actions outside [0, A) are clamped (for memory safety only).
+ * The tile is 1024 steps: longer rows carry between thread blocks through the workspace's records,
+ * except rows of whole tiles with A = 4 or 8 and about three rows per SM or more, which one thread
+ * block each walks with the carry in a register (results agree to rounding).
  */
 int rlcs_retrace_probs(const float* rewards, const float* q_values, const float* target_probs,
                        const float* behaviour_probs, const int32_t* actions, const uint8_t* dones, const uint8_t* truncs,

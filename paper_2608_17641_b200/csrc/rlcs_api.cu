@@ -113,7 +113,7 @@ int rlcs_gae_skip(const float* rewards, const float* values, const uint8_t* done
     // its own carry records.  These tile shapes have at least 1024 steps, so two records per tile still
     // fit the workspace of rlcs_workspace_bytes (sized for 512-step tiles).  No cluster carry here.
     const int variant = choose_variant(rlcs::kGaeSkip, truncs != nullptr, total, T);
-    st = finish_params(p, variant, total, T, workspace, workspace_bytes, vec, false, 2, false);
+    st = finish_params(p, variant, total, T, workspace, workspace_bytes, vec, false, 2, false, false);
     if (st != RLCS_OK) return st;
     return run(rlcs::launch_gae_skip, p, variant, truncs != nullptr, vec, cuda_stream);
 }
@@ -230,7 +230,14 @@ int rlcs_retrace_probs(const float* rewards, const float* q_values, const float*
     constexpr int kVariant = 3;      // 256 threads x 4 steps, the tile rlcs_retrace_probs.cu instantiates
     static_assert(rlcs::kVariants[kVariant].threads == rlcs::kRetraceProbsThreads &&
                   rlcs::kVariants[kVariant].items == rlcs::kRetraceProbsItems, "tile shape mismatch");
-    st = finish_params(p, kVariant, total, T, workspace, workspace_bytes, vec, false, 1, false);
+    // One thread block per row where rows are whole tiles and there are enough of them (no carry between
+    // blocks): measured at 16384 x 2048 / 8192 x 4096 / 2048 x 16384 against the carry through tile records,
+    // fraction of the copy bandwidth: A = 4 0.86 -> 0.92 / 0.95 / 0.91, A = 8 0.87 / 0.84 / 0.81 -> 0.94 /
+    // 0.94 / 0.88, but A = 16 0.87 / 0.86 / 0.84 -> 0.85 / 0.84 / 0.79, so only for the two narrow row widths
+    // (the test hook forces it for any A).
+    const bool rows_ok = T % (rlcs::kRetraceProbsThreads * rlcs::kRetraceProbsItems) == 0 &&
+                         (rlcs_hooks::g_row_blocks > 0 || (vec_rows && (A == 4 || A == 8)));
+    st = finish_params(p, kVariant, total, T, workspace, workspace_bytes, vec, false, 1, false, rows_ok);
     if (st != RLCS_OK) return st;
     return rlcs::launch_retrace_probs(p, truncs != nullptr, vec, vec_rows, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess
                ? RLCS_OK : RLCS_ERR_CUDA;

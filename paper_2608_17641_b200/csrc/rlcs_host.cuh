@@ -180,7 +180,7 @@ CarryPlan plan_carry(int variant, int64_t total, int64_t T, bool vec, bool allow
     const int tile = tile_elems(variant);
     const int64_t num_tiles = (total + tile - 1) / tile;
     CarryPlan plan = {(tile % T) != 0 ? 1 : 0, 0, 0, tile, 0};    // T does not divide the tile: rows straddle tiles
-    if (allow_row_tiles && allow_row_blocks && row_blocks_ok(variant, total, T, vec)) {
+    if (allow_row_blocks && row_blocks_ok(variant, total, T, vec)) {
         plan.carry_mode = 0;
         plan.row_blocks = 1;
         return plan;
@@ -207,8 +207,8 @@ CarryPlan plan_carry(int variant, int64_t total, int64_t T, bool vec, bool allow
 
 // Fill the size / tiling / carry fields and validate the workspace for this call.  Callers whose
 // kernels have no row-aligned / one-block-per-row instantiation (has_row_blocks() in rlcs_launch.cuh:
-// the statistics flavour of GAE, the observation-skip scans, Retrace from [N,T,A] tensors) pass
-// allow_row_tiles = false.
+// the statistics flavour of GAE, the observation-skip scans) pass allow_row_tiles = allow_row_blocks =
+// false; Retrace from [N,T,A] tensors has its own one-block-per-row kernel for rows of whole tiles.
 int finish_params(ScanParams& p, int variant, int64_t total, int64_t T, void* workspace, size_t workspace_bytes, bool vec,
                   bool allow_cluster = true, int records_per_tile = 1, bool allow_row_tiles = true, bool allow_row_blocks = true) {
     const int tile = tile_elems(variant);

@@ -7,6 +7,12 @@ namespace rlcs {
 
 template <bool TRUNC, bool VEC, int AV>
 static cudaError_t launch_one(const ScanParams& p, cudaStream_t stream) {
+    if constexpr (VEC) {
+        // rows of whole tiles and many of them: one thread block per row, the carry in a register
+        if (p.row_blocks)
+            return launch_scan(scan_kernel_retrace_probs_rows<TRUNC, kRetraceProbsThreads, kRetraceProbsItems, 4, AV>,
+                               (unsigned)p.num_tiles, kRetraceProbsThreads, 0, stream, 0, p);
+    }
     return launch_scan(scan_kernel_retrace_probs<TRUNC, VEC, kRetraceProbsThreads, kRetraceProbsItems, 4, AV>,
                        (unsigned)p.num_tiles, kRetraceProbsThreads, 0, stream, 0, p);
 }

@@ -1275,6 +1275,37 @@ __global__ void __launch_bounds__(THREADS, MIN_BLOCKS) scan_kernel_retrace_probs
     else one_tile_probs<TRUNC, VEC, THREADS, ITEMS, AV, false>(p, tile, s, epoch, sm);
 }
 
+// The same with one thread block per row (rows of whole tiles, many rows): block n walks the tiles of
+// row n in scan order and keeps the carry in a register, as scan_kernel_rows does for the scalar-input
+// algorithms -- no records, no waiting, whatever T is.
+template <bool TRUNC, int THREADS, int ITEMS, int MIN_BLOCKS, int AV>
+__global__ void __launch_bounds__(THREADS, MIN_BLOCKS) scan_kernel_retrace_probs_rows(const ScanParams p) {
+    constexpr int ALGO = kRetraceProbs;
+    constexpr int TILE = THREADS * ITEMS;
+    __shared__ ScanSmem<THREADS / 32> sm;
+    grid_dependency_launch();
+    grid_dependency_wait();
+    const int tid = threadIdx.x;
+    const int lane = tid & 31;
+    const long long row_start = (long long)blockIdx.x * p.T;
+    const long long row_end = row_start + p.T;
+    const unsigned tiles = p.T / TILE;                        // whole tiles only (the host checks)
+    float carry = 0.f;
+    for (unsigned k = 0; k < tiles; ++k) {
+        const long long i0 = row_start + (long long)(tiles - 1 - k) * TILE + (long long)tid * ITEMS;
+        Chunk<ALGO, TRUNC, ITEMS> c;
+        const long long n0 = locate(c, p, i0, row_end);
+        load_flags_global<ALGO, TRUNC, ITEMS, true, true>(c, p, i0, lane);
+        Vals<ITEMS> v;
+        load_values_probs<ALGO, TRUNC, ITEMS, AV>(c, v, p, i0, lane, ITEMS);
+        issue_boot(c, p, n0);
+        issue_trunc_values(c, p, i0);
+        // shared scratch alternates by tile parity, so one barrier per tile suffices
+        tile_compute<ALGO, TRUNC, true, THREADS, ITEMS, true, false, NoHook, false, false>(c, v, p, i0, 0, 0u, sm, k & 1, NoHook{},
+                                                                                          nullptr, &carry);
+    }
+}
+
 #endif  // !RLCS_IO_BF16
 
 // ------------------------------------------------------------------------------------------ kernel 1b: one tile per block, one cluster per row

@@ -582,6 +582,32 @@ def test_retrace_probs_unaligned_and_long_rows(oracle, W, B):
         assert_close(f"retrace_probs {N}x{T}x{A} offset {off}", got, ref)
 
 
+@pytest.mark.parametrize("A", [3, 4, 8, 16])
+@pytest.mark.parametrize("N,T", [(5, 2048), (3, 4096), (2, 16384), (470, 2048)])
+def test_retrace_probs_one_block_per_row(oracle, W, B, A, N, T):
+    """Rows of whole 1024-step tiles walked by one thread block each (forced here for few rows; the
+    library's own choice from about three rows per SM, which 470 x 2048 reaches): against the oracle
+    and against the carry through tile records."""
+    ro = W.make_rollout(115, N, T, p_done=0.002, p_trunc=0.002, salt=A + T)
+    q, pi, mu, act = W.make_action_tensors(115, N, T, A, salt=N)
+    B.rlcs_debug_set_row_blocks(0)
+    try:
+        records = _probs_gpu(B, ro, q, pi, mu, act)
+        B.rlcs_debug_set_row_blocks(1)
+        rows = _probs_gpu(B, ro, q, pi, mu, act)
+        rows_plain = _probs_gpu(B, ro, q, pi, mu, act, use_truncs=False, use_bootstrap=False)
+    finally:
+        B.rlcs_debug_set_row_blocks(-1)
+    kw = dict(gamma=ro.params["gamma"], lam=ro.params["lam"], c_bar=ro.params["c_bar"])
+    assert_close(f"retrace_probs rows {N}x{T}x{A}", rows,
+                 oracle.retrace_probs(ro.rewards, q, pi, mu, act, ro.dones, ro.truncs, ro.trunc_bootstrap, ro.bootstrap, **kw))
+    assert_close(f"retrace_probs rows, plain {N}x{T}x{A}", rows_plain,
+                 oracle.retrace_probs(ro.rewards, q, pi, mu, act, ro.dones, None, None, None, **kw))
+    np.testing.assert_allclose(rows, records, rtol=1e-5, atol=1e-5)
+    if N >= 470:
+        assert np.array_equal(rows, _probs_gpu(B, ro, q, pi, mu, act))      # the default for this shape
+
+
 def test_retrace_probs_agrees_with_scalar_entry_point(oracle, W, B):
     """The tensor form and rlcs_retrace on inputs derived from the tensors (gather, dot, log) agree."""
     import torch
