@@ -23,7 +23,9 @@
 // chunks.  Ring path: one launch; blocks take (column block, chunk) pairs in scan order from a
 // ticket counter, walk their chunk for its aggregate (a, b) of Eq. 2, publish it, look back over
 // the records of the chunks before for the carry into their own, and walk the chunk again -- out of
-// L2 -- to write the outputs.  Register path: three launches (aggregates with carry 0, a small
+// L2 -- to write the outputs (the vector traces, whose flags hold for all columns at once, walk it
+// only once and finish the steps before the chunk's first cut from the ring).  Register path: three
+// launches (aggregates with carry 0, a small
 // kernel that chains an environment's chunks in scan order, second walk from the carry), the inputs
 // read twice.  Deterministic either way.
 #include <cmath>
