@@ -6,44 +6,54 @@ namespace rlcs {
 
 RLCS_DEFINE_LAUNCHER(launch_gae_stats, kGaeStats, true)
 
+// Sum of one double per thread over a block of 1024 threads, in a fixed order (lanes by shuffle
+// distance 16, 8, ..., 1, then the 32 warp sums the same way in warp 0): every thread gets the result.
+__device__ __forceinline__ double block_sum_1024(double x, double* sh /* [33] */) {
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) x += __shfl_down_sync(0xffffffffu, x, d);
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    if (lane == 0) sh[w] = x;
+    __syncthreads();
+    if (w == 0) {
+        double y = sh[lane];
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) y += __shfl_down_sync(0xffffffffu, y, d);
+        if (lane == 0) sh[32] = y;
+    }
+    __syncthreads();
+    const double total = sh[32];
+    __syncthreads();                                         // sh is reused by the next call
+    return total;
+}
+
 // One block: per-tile {sum, sum of squared deviations from the tile mean} -> {mean, 1/(std + eps)}.
-// Two strided passes in double, each followed by a shared-memory tree in a fixed order (the result
-// does not depend on timing): first the mean, then
+// Two strided passes in double, each followed by a block sum in a fixed order (the result does not
+// depend on timing): first the mean, then
 //     sum (A - mean)^2 = sum over tiles of [ q_i + n_i (m_i - mean)^2 ],   m_i = s_i / n_i,
 // which is exact algebra and never subtracts two large numbers.  Tile i of the scan order holds
 // `tile` steps except the one at the array's end (scan-order tile 0 of this backward scan).
 __global__ void __launch_bounds__(1024) norm_finalize_kernel(const float* __restrict__ partial, long long num_tiles,
                                                              long long total, int tile, int ddof, float eps,
                                                              float* __restrict__ out) {
-    __shared__ double sh[1024];
-    __shared__ double mean_sh;
+    __shared__ double sh[33];
+    grid_dependency_launch();
+    grid_dependency_wait();                                  // the per-tile sums come from the kernel before
+    const float2* const pairs = reinterpret_cast<const float2*>(partial);
     double acc = 0.0;
-    for (long long i = threadIdx.x; i < num_tiles; i += 1024) acc += (double)partial[2 * i];
-    sh[threadIdx.x] = acc;
-    __syncthreads();
-    for (int d = 512; d > 0; d >>= 1) {
-        if ((int)threadIdx.x < d) sh[threadIdx.x] += sh[threadIdx.x + d];
-        __syncthreads();
-    }
-    if (threadIdx.x == 0) mean_sh = sh[0] / (double)total;
-    __syncthreads();
-    const double mean = mean_sh;
+    for (long long i = threadIdx.x; i < num_tiles; i += 1024) acc += (double)__ldcg(pairs + i).x;
+    const double mean = block_sum_1024(acc, sh) / (double)total;
     const long long last = total - (num_tiles - 1) * (long long)tile;      // steps in the ragged tile
     acc = 0.0;
     for (long long i = threadIdx.x; i < num_tiles; i += 1024) {
+        const float2 sq = __ldcg(pairs + i);
         const double n = (double)(i == 0 ? last : (long long)tile);
-        const double dm = (double)partial[2 * i] / n - mean;
-        acc += (double)partial[2 * i + 1] + n * dm * dm;
+        const double dm = (double)sq.x / n - mean;
+        acc += (double)sq.y + n * dm * dm;
     }
-    sh[threadIdx.x] = acc;
-    __syncthreads();
-    for (int d = 512; d > 0; d >>= 1) {
-        if ((int)threadIdx.x < d) sh[threadIdx.x] += sh[threadIdx.x + d];
-        __syncthreads();
-    }
+    const double ssd = block_sum_1024(acc, sh);
     if (threadIdx.x == 0) {
         const double denom = (double)total - (double)ddof;
-        const double var = denom > 0.0 ? sh[0] / denom : 0.0;
+        const double var = denom > 0.0 ? ssd / denom : 0.0;
         out[0] = (float)mean;
         out[1] = (float)(1.0 / (sqrt(var) + (double)eps));
     }
@@ -53,8 +63,12 @@ __global__ void __launch_bounds__(1024) norm_finalize_kernel(const float* __rest
 // the pointer allows, element-wise otherwise and for the ragged tail.
 template <bool VEC>
 __global__ void __launch_bounds__(256) norm_rescale_kernel(float* __restrict__ adv, long long total,
-                                                           const float* __restrict__ mean_rstd) {
-    const float mean = __ldg(mean_rstd), rstd = __ldg(mean_rstd + 1);
+                                                           const float* mean_rstd) {
+    grid_dependency_launch();
+    grid_dependency_wait();                                  // mean and 1/(std + eps) come from the kernel before
+    // plain loads: cached in L1 (every thread of the grid reads these two words -- bypassing L1 sends
+    // them all to one L2 slice, measured +30 us), and issued only after the wait above
+    const float mean = mean_rstd[0], rstd = mean_rstd[1];
     const long long i0 = ((long long)blockIdx.x * 256 + threadIdx.x) * 8;
     if (i0 >= total) return;
     if (VEC && i0 + 8 <= total) {
@@ -68,17 +82,32 @@ __global__ void __launch_bounds__(256) norm_rescale_kernel(float* __restrict__ a
     }
 }
 
+// Both follow-up kernels are launched like the scan kernels: their blocks may be placed while the
+// kernel before them drains, and they touch global memory only after grid_dependency_wait().
+template <class Kernel, class... Args>
+static cudaError_t launch_after(Kernel kernel, unsigned grid, unsigned block, cudaStream_t stream, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid, 1, 1);
+    cfg.blockDim = dim3(block, 1, 1);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = rlcs_hooks::g_pdl ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, args...);
+}
+
 cudaError_t launch_norm_finalize(const float* partial, long long num_tiles, long long total, int tile, int ddof, float eps,
                                  float* mean_rstd, cudaStream_t stream) {
-    norm_finalize_kernel<<<1, 1024, 0, stream>>>(partial, num_tiles, total, tile, ddof, eps, mean_rstd);
-    return cudaGetLastError();
+    return launch_after(norm_finalize_kernel, 1u, 1024u, stream, partial, num_tiles, total, tile, ddof, eps, mean_rstd);
 }
 
 cudaError_t launch_norm_rescale(float* adv, long long total, const float* mean_rstd, bool vec, cudaStream_t stream) {
     const long long blocks = (total + 2047) / 2048;
-    if (vec) norm_rescale_kernel<true><<<(unsigned)blocks, 256, 0, stream>>>(adv, total, mean_rstd);
-    else norm_rescale_kernel<false><<<(unsigned)blocks, 256, 0, stream>>>(adv, total, mean_rstd);
-    return cudaGetLastError();
+    const float* mr = mean_rstd;
+    return vec ? launch_after(norm_rescale_kernel<true>, (unsigned)blocks, 256u, stream, adv, total, mr)
+               : launch_after(norm_rescale_kernel<false>, (unsigned)blocks, 256u, stream, adv, total, mr);
 }
 
 }  // namespace rlcs

@@ -497,6 +497,30 @@ def test_gae_normalized(oracle, W, B, N, T, ddof):
     assert np.array_equal(adv2.cpu().numpy(), adv.cpu().numpy())
 
 
+def test_gae_normalized_back_to_back_calls_share_nothing_stale(oracle, W, B):
+    """Three calls queued without a host synchronisation in between, on the same workspace and the same
+    output tensors, with rewards of very different mean and spread: every call must rescale with its own
+    mean and 1/(std + eps) (the follow-up kernels are placed on the SMs while the kernel before them is
+    still running, and all of them read the two words from the same address)."""
+    N, T = 3000, 512
+    ro = W.make_rollout(116, N, T)
+    p = ro.params
+    scales = ((1.0, 0.0), (10.0, 5.0), (0.1, -3.0))
+    ws = B.Workspace(N, T, nbytes=B.lib().rlcs_gae_normalized_workspace_bytes(N, T))
+    dev = Dev(ro)
+    rewards = [guarded_upload((ro.rewards * a + b).astype(np.float32)) for a, b in scales]
+    adv, ret = dev.empty_out(), dev.empty_out()
+    kept = []
+    for r in rewards:
+        B.rlcs_gae_normalized(r, dev.values, dev.dones, dev.truncs, dev.trunc_bootstrap, dev.bootstrap, gamma=p["gamma"],
+                              lam=p["lam"], eps=1e-8, ddof=1, advantages=adv, returns=ret, workspace=ws)
+        kept.append(adv.clone())
+    for (a, b), got in zip(scales, kept):
+        ref_adv, _ = oracle.gae_normalized((ro.rewards * a + b).astype(np.float32), ro.values, ro.dones, ro.truncs,
+                                           ro.trunc_bootstrap, ro.bootstrap, gamma=p["gamma"], lam=p["lam"], eps=1e-8, ddof=1)
+        assert_close(f"normalised advantages, rewards * {a} + {b}", got.cpu().numpy(), ref_adv)
+
+
 def test_gae_normalized_with_a_mean_far_from_zero(oracle, W, B):
     """Rewards ~ N(100, 0.1^2), small values, lambda = 0.1, no flags: every advantage is close to
     100 with a spread of about 0.1, so |mean| is a thousand times the standard deviation -- the case
