@@ -40,6 +40,7 @@
 namespace rlcs_hooks {
 extern long long g_mute_tile;      // scan-order tile / block ticket that does not publish
 extern long long g_spin_cap;       // poll limit (0 = default)
+extern bool g_pdl;                 // launch with programmatic stream serialisation (default on)
 }  // namespace rlcs_hooks
 
 namespace {
@@ -907,6 +908,10 @@ __device__ __forceinline__ TmParams batch_slice(const TmParams& p_in, unsigned z
 // 0.03-0.10 of the copy bandwidth -- although the ring is planned for up to six blocks.)
 template <int ALGO, bool TRUNC, int MODE, int W, int C>
 __global__ void __launch_bounds__(32 * W) tm_block_kernel(const TmParams p_in) {
+    // (no-ops unless launched with programmatic stream serialisation: then the blocks may be placed
+    // while the kernel before this one drains, and nothing in global memory is touched before it is done)
+    rlcs::grid_dependency_launch();
+    rlcs::grid_dependency_wait();
     const TmParams p = batch_slice<ALGO>(p_in, blockIdx.z);
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
     const long long n0 = (long long)blockIdx.x * (32 * C);
@@ -1189,7 +1194,18 @@ int launch_block(const TmParams& p_in, size_t smem, cudaStream_t s) {
     const dim3 grid(colblocks, p.chunks, (unsigned)batch);
     if (p.chunks == 1) {
         if (!allow_smem(tm_block_kernel<ALGO, TRUNC, 0, W, C>, smem)) return RLCS_ERR_CUDA;
-        tm_block_kernel<ALGO, TRUNC, 0, W, C><<<grid, 32 * W, smem, s>>>(p);
+        // the uncut walk is launched like the row-major scan kernels (see launch_scan in rlcs_launch.cuh)
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = grid;
+        cfg.blockDim = dim3(32 * W, 1, 1);
+        cfg.dynamicSmemBytes = smem;
+        cfg.stream = s;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = rlcs_hooks::g_pdl ? 1 : 0;
+        return cudaLaunchKernelEx(&cfg, tm_block_kernel<ALGO, TRUNC, 0, W, C>, p) == cudaSuccess ? RLCS_OK : RLCS_ERR_CUDA;
     } else {
         if (!allow_smem(tm_block_kernel<ALGO, TRUNC, 1, W, C>, smem) || !allow_smem(tm_block_kernel<ALGO, TRUNC, 2, W, C>, smem))
             return RLCS_ERR_CUDA;
