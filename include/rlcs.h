@@ -46,7 +46,8 @@
  *   points, that are ordered on one stream.  Two calls that may run concurrently need two
  *   workspaces.  When rlcs_workspace_bytes(N, T) is 0 the workspace may be NULL.
  * Execution.  Work is enqueued on `cuda_stream` (a cudaStream_t passed as void*; NULL = the
- *   default stream) and the call returns without synchronising.  The row-major scan kernels are
+ *   default stream) and the call returns without synchronising.  The row-major scan kernels, the
+ *   follow-up kernels of rlcs_gae_normalized and the time-major ring kernel (uncut time axis) are
  *   launched with programmatic stream serialisation: their thread blocks may be placed on the GPU
  *   while the preceding kernel of the stream drains, but they wait for that kernel's completion
  *   (and the visibility of its writes) before their first access to global memory -- caller
