@@ -124,8 +124,9 @@ int rlcs_gae(const float* rewards, const float* values, const uint8_t* dones, co
  *   non-finite, as the formula says; pass eps > 0 to get zeros there.
  * Three launches: the GAE kernel (which also leaves, per tile, the sum of A and the sum of squared
  * deviations from the tile's own mean), a one-block reduction in double to mean and 1/(std + eps)
- * (tile statistics are merged as q_i + n_i (m_i - mean)^2, so a mean much larger than the spread
- * does not cancel the variance away), and an in-place rescale of `advantages` -- one read of A
+ * (the centred tile statistics are merged in double as sum(q_i + s_i^2 / n_i) - S^2 / (N*T), which
+ * keeps a relative accuracy of about 2^-52 (mean / std)^2: a mean a thousand times the spread does
+ * not cancel the variance away), and an in-place rescale of `advantages` -- one read of A
  * fewer than GAE, a statistics pass and a rescale.  Deterministic (fixed reduction order).
  * `workspace`: at least rlcs_gae_normalized_workspace_bytes(N, T) bytes (always > 0), 16-byte
  * aligned, initialised once with rlcs_workspace_init; same sharing rules as any workspace.

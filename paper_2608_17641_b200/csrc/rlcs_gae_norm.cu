@@ -6,52 +6,59 @@ namespace rlcs {
 
 RLCS_DEFINE_LAUNCHER(launch_gae_stats, kGaeStats, true)
 
-// Sum of one double per thread over a block of 1024 threads, in a fixed order (lanes by shuffle
-// distance 16, 8, ..., 1, then the 32 warp sums the same way in warp 0): every thread gets the result.
-__device__ __forceinline__ double block_sum_1024(double x, double* sh /* [33] */) {
+// Sums of two doubles per thread over a block of 1024 threads, in a fixed order (lanes by shuffle
+// distance 16, 8, ..., 1, then the 32 warp sums the same way in warp 0): every thread gets both.
+__device__ __forceinline__ void block_sum2_1024(double& x, double& y, double* sh /* [66] */) {
 #pragma unroll
-    for (int d = 16; d > 0; d >>= 1) x += __shfl_down_sync(0xffffffffu, x, d);
+    for (int d = 16; d > 0; d >>= 1) {
+        x += __shfl_down_sync(0xffffffffu, x, d);
+        y += __shfl_down_sync(0xffffffffu, y, d);
+    }
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-    if (lane == 0) sh[w] = x;
+    if (lane == 0) { sh[w] = x; sh[32 + w] = y; }
     __syncthreads();
     if (w == 0) {
-        double y = sh[lane];
+        double u = sh[lane], v = sh[32 + lane];
 #pragma unroll
-        for (int d = 16; d > 0; d >>= 1) y += __shfl_down_sync(0xffffffffu, y, d);
-        if (lane == 0) sh[32] = y;
+        for (int d = 16; d > 0; d >>= 1) {
+            u += __shfl_down_sync(0xffffffffu, u, d);
+            v += __shfl_down_sync(0xffffffffu, v, d);
+        }
+        if (lane == 0) { sh[64] = u; sh[65] = v; }
     }
     __syncthreads();
-    const double total = sh[32];
-    __syncthreads();                                         // sh is reused by the next call
-    return total;
+    x = sh[64];
+    y = sh[65];
 }
 
-// One block: per-tile {sum, sum of squared deviations from the tile mean} -> {mean, 1/(std + eps)}.
-// Two strided passes in double, each followed by a block sum in a fixed order (the result does not
-// depend on timing): first the mean, then
-//     sum (A - mean)^2 = sum over tiles of [ q_i + n_i (m_i - mean)^2 ],   m_i = s_i / n_i,
-// which is exact algebra and never subtracts two large numbers.  Tile i of the scan order holds
-// `tile` steps except the one at the array's end (scan-order tile 0 of this backward scan).
+// One block: per-tile {s_i = sum, q_i = sum of squared deviations from the tile mean} -> {mean,
+// 1/(std + eps)}, in one strided pass in double followed by a block sum in a fixed order (the result
+// does not depend on timing):
+//     S = sum_i s_i,   Q = sum_i (q_i + s_i^2 / n_i),   sum (A - mean)^2 = Q - S^2 / N.
+// The per-tile sums are fp32 and centred on the tile mean, so q_i carries no cancellation; s_i^2 is
+// exact in double and the last subtraction loses 2^-52 (mean / std)^2 of relative accuracy -- 2e-10
+// where the mean is a thousand standard deviations away.  Tile i of the scan order holds `tile` steps
+// except the one at the array's end (scan-order tile 0 of this backward scan).
 __global__ void __launch_bounds__(1024) norm_finalize_kernel(const float* __restrict__ partial, long long num_tiles,
                                                              long long total, int tile, int ddof, float eps,
                                                              float* __restrict__ out) {
-    __shared__ double sh[33];
+    __shared__ double sh[66];
     grid_dependency_launch();
     grid_dependency_wait();                                  // the per-tile sums come from the kernel before
     const float2* const pairs = reinterpret_cast<const float2*>(partial);
-    double acc = 0.0;
-    for (long long i = threadIdx.x; i < num_tiles; i += 1024) acc += (double)__ldcg(pairs + i).x;
-    const double mean = block_sum_1024(acc, sh) / (double)total;
     const long long last = total - (num_tiles - 1) * (long long)tile;      // steps in the ragged tile
-    acc = 0.0;
+    const double inv_tile = 1.0 / (double)tile, inv_last = 1.0 / (double)last;   // (no division per tile: one SM does all of this)
+    double S = 0.0, Q = 0.0;
     for (long long i = threadIdx.x; i < num_tiles; i += 1024) {
         const float2 sq = __ldcg(pairs + i);
-        const double n = (double)(i == 0 ? last : (long long)tile);
-        const double dm = (double)sq.x / n - mean;
-        acc += (double)sq.y + n * dm * dm;
+        const double si = (double)sq.x;
+        S += si;
+        Q += (double)sq.y + si * si * (i == 0 ? inv_last : inv_tile);
     }
-    const double ssd = block_sum_1024(acc, sh);
+    block_sum2_1024(S, Q, sh);
     if (threadIdx.x == 0) {
+        const double mean = S / (double)total;
+        const double ssd = fmax(Q - S * mean, 0.0);
         const double denom = (double)total - (double)ddof;
         const double var = denom > 0.0 ? ssd / denom : 0.0;
         out[0] = (float)mean;
