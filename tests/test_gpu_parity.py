@@ -777,6 +777,36 @@ def test_vector_trace_chained_kernel_single_walk(oracle, W, B, N, T, D, p_flag):
     assert_close("per-dimension trace, chained", gotb, oracle.elig_trace_vec_beta(x, beta, d))
 
 
+def test_vector_trace_chained_wait_runs_out_and_reports_timeout(oracle, W, B):
+    """The single-walk chained kernel with one block that never publishes its chunk and no cut
+    anywhere (every later chunk of that chain needs a carry): the waits run out of polls, the kernel
+    finishes, the status word says TIMEOUT, and the next call on the workspace is right."""
+    import torch
+    N, T, D = 4, 4096, 64
+    rng = np.random.default_rng(4711)
+    x = rng.standard_normal((N, T, D)).astype(np.float32)
+    d = np.zeros((N, T), np.uint8)
+    xd, dd = guarded_upload(x), guarded_upload(d)
+    B.rlcs_debug_vec_trace_plan(1, 0)
+    B.rlcs_debug_time_major_path(5)
+    try:
+        ws = B.Workspace(N, T, nbytes=int(B.lib().rlcs_elig_trace_vec_workspace_bytes(N, T, D)))
+        B.rlcs_debug_set_carry_fault(2, 50)
+        try:
+            B.rlcs_elig_trace_vec(xd, dd, gamma=0.99, lam=0.95, workspace=ws)
+            torch.cuda.synchronize()
+            assert ws.device_status() == B.RLCS_ERR_TIMEOUT
+        finally:
+            B.rlcs_debug_set_carry_fault(-1, 0)
+        assert ws.device_status() == B.RLCS_OK
+        got = B.rlcs_elig_trace_vec(xd, dd, gamma=0.99, lam=0.95, workspace=ws).cpu().numpy()
+        assert ws.device_status() == B.RLCS_OK
+    finally:
+        B.rlcs_debug_vec_trace_plan(0, 0)
+        B.rlcs_debug_time_major_path(0)
+    assert_close("vector trace after the timeout", got, oracle.elig_trace_vec(x, d, gamma=0.99, lam=0.95))
+
+
 def test_per_dimension_beta_argument_checks(oracle, W, B):
     L = B.lib()
     P = 0x7f0000000000
