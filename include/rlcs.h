@@ -364,7 +364,9 @@ int rlcs_episodic_prefix_sum_time_major(const float* x, const uint8_t* dones, fl
  * rlcs_gae of the rows with the masked steps deleted.
  * Outputs: values_filled = W (required), advantages = A, returns = A + W (optional).  One launch:
  * per tile, W by a backward scan and then the masked GAE scan on (rewards, W), each with its own
- * carry between tiles.  Same flags, NULL conventions, alignment rules and workspace as rlcs_gae.
+ * carry between tiles (through the workspace's records; rows of whole 1024-step tiles with about
+ * three rows per SM or more are walked by one thread block each, both carries in registers).
+ * Same flags, NULL conventions, alignment rules and workspace as rlcs_gae.
  */
 int rlcs_gae_skip(const float* rewards, const float* values, const uint8_t* dones, const uint8_t* truncs,
                   const float* trunc_bootstrap, const float* bootstrap, const uint8_t* skip, float* values_filled,

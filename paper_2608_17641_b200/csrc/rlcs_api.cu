@@ -112,8 +112,16 @@ int rlcs_gae_skip(const float* rewards, const float* values, const uint8_t* done
     // One launch runs both scans per tile (value fill, then the masked GAE on its result); each scan has
     // its own carry records.  These tile shapes have at least 1024 steps, so two records per tile still
     // fit the workspace of rlcs_workspace_bytes (sized for 512-step tiles).  No cluster carry here.
-    const int variant = choose_variant(rlcs::kGaeSkip, truncs != nullptr, total, T);
-    st = finish_params(p, variant, total, T, workspace, workspace_bytes, vec, false, 2, false, false);
+    int variant = choose_variant(rlcs::kGaeSkip, truncs != nullptr, total, T);
+    // Rows of whole tiles, about three per SM or more: one thread block per row, both carries in
+    // registers (token-level trajectories are long).  Measured at 4096 x 8192 / 1024 x 32768, fraction of
+    // the copy bandwidth: records through the workspace 0.68 / 0.62; rows with 128 x 16 tiles at 5 / 6 / 8
+    // blocks per SM 0.84 / 0.70, 0.80 / 0.63, 0.58 / 0.55; 256 x 8 0.89 / 0.81; 128 x 8 at 8 blocks 0.90 / 0.85.
+    constexpr int kRowsVariant = 6;
+    if (rlcs_hooks::g_variant < 0 && T > 2048 && T % tile_elems(kRowsVariant) == 0 && row_blocks_ok(kRowsVariant, total, T, vec))
+        variant = kRowsVariant;
+    const bool rows_ok = T % tile_elems(variant) == 0;
+    st = finish_params(p, variant, total, T, workspace, workspace_bytes, vec, false, 2, false, rows_ok);
     if (st != RLCS_OK) return st;
     return run(rlcs::launch_gae_skip, p, variant, truncs != nullptr, vec, cuda_stream);
 }

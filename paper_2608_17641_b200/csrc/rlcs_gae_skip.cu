@@ -7,6 +7,12 @@ namespace rlcs {
 template <bool TRUNC, bool VEC, int V>
 cudaError_t launch_skip_variant(const ScanParams& p, cudaStream_t stream) {
     constexpr TileVariant tv = kVariants[V];
+    if constexpr (VEC) {
+        // rows of whole tiles and many of them: one thread block per row, both carries in registers
+        if (p.row_blocks)
+            return launch_scan(scan_kernel_gae_skip_rows<TRUNC, tv.threads, tv.items, tv.min_blocks>, (unsigned)p.num_tiles,
+                               tv.threads, 0, stream, 0, p);
+    }
     return launch_scan(scan_kernel_gae_skip<TRUNC, VEC, tv.threads, tv.items, tv.min_blocks>, (unsigned)p.num_tiles, tv.threads, 0,
                        stream, 0, p);
 }

@@ -1239,6 +1239,55 @@ __global__ void __launch_bounds__(THREADS, MIN_BLOCKS) scan_kernel_gae_skip(cons
     if (full) one_tile_gae_skip<TRUNC, VEC, THREADS, ITEMS, true>(p, tile, s, epoch, sm);
     else one_tile_gae_skip<TRUNC, VEC, THREADS, ITEMS, false>(p, tile, s, epoch, sm);
 }
+
+// The same with one thread block per row (rows of whole tiles, many rows -- token-level trajectories
+// are long): block n walks the tiles of row n in scan order and keeps both carries, the fill's and
+// the advantage's, in registers; no records, no waiting.  The two scans of a tile use the two halves
+// of the shared scratch, and each scan's block barrier separates a half's reads in one tile from its
+// writes in the next.
+template <bool TRUNC, int THREADS, int ITEMS, int MIN_BLOCKS>
+__global__ void __launch_bounds__(THREADS, MIN_BLOCKS) scan_kernel_gae_skip_rows(const ScanParams p) {
+    constexpr int TILE = THREADS * ITEMS;
+    __shared__ ScanSmem<THREADS / 32> sm;
+    grid_dependency_launch();
+    grid_dependency_wait();
+    const int tid = threadIdx.x;
+    const int lane = tid & 31;
+    const long long row_start = (long long)blockIdx.x * p.T;
+    const long long row_end = row_start + p.T;
+    const unsigned tiles = p.T / TILE;                        // whole tiles only (the host checks)
+    ScanParams pf = p;
+    pf.out0 = p.out2;
+    pf.out1 = nullptr;
+    float carry_w = 0.f, carry_a = 0.f;
+    for (unsigned k = 0; k < tiles; ++k) {
+        const long long i0 = row_start + (long long)(tiles - 1 - k) * TILE + (long long)tid * ITEMS;
+        Chunk<kFillSkip, TRUNC, ITEMS> cf;
+        const long long n0 = locate(cf, p, i0, row_end);
+        load_flags_global<kFillSkip, TRUNC, ITEMS, true, true>(cf, p, i0, lane);
+        Vals<ITEMS> vf, vg;
+        load_f32<ITEMS, true>(p.f1, i0, ITEMS, vf.a);        // values: the fill scan's input
+        load_f32<ITEMS, true>(p.f0, i0, ITEMS, vg.a);        // rewards, for the second scan
+        vf.halo = 0.f; vf.halo_lr = 0.f;
+        issue_boot(cf, p, n0);
+        issue_trunc_values(cf, p, i0);
+        Chunk<kGaeSkip, TRUNC, ITEMS> cg;
+        cg.edge = cf.edge; cg.nvalid = cf.nvalid; cg.halo_d = 0; cg.boot_first = cf.boot_first;
+#pragma unroll
+        for (int q = 0; q < ITEMS / 4; ++q) { cg.dw[q] = cf.dw[q]; cg.tw[q] = cf.tw[q]; cg.kw[q] = cf.kw[q]; }
+#pragma unroll
+        for (int j = 0; j < ITEMS; ++j) cg.ov[j] = cf.ov[j];
+        float w_next = 0.f;
+        tile_compute<kFillSkip, TRUNC, true, THREADS, ITEMS, true, false, NoHook, false, false>(cf, vf, pf, i0, 0, 0u, sm, 0, NoHook{},
+                                                                                               &w_next, &carry_w);
+#pragma unroll
+        for (int j = 0; j < ITEMS; ++j) vg.x1[j] = vf.a[j];  // W of this thread's steps
+        vg.halo = w_next;
+        vg.halo_lr = 0.f;
+        tile_compute<kGaeSkip, TRUNC, true, THREADS, ITEMS, true, false, NoHook, false, false>(cg, vg, p, i0, 0, 0u, sm, 1, NoHook{},
+                                                                                              nullptr, &carry_a);
+    }
+}
 #endif  // !RLCS_IO_BF16
 
 // ------------------------------------------------------------------------------------------ kernel 1c: Retrace from [N,T,A] tensors

@@ -859,6 +859,53 @@ def test_gae_with_observation_skip_masking(oracle, W, B, N, T, p_skip, p_flag):
         assert torch.equal(a0, a1)
 
 
+@pytest.mark.parametrize("p_skip,p_flag", [(0.3, 0.002), (0.9, 0.0), (0.0, 0.02)])
+@pytest.mark.parametrize("N,T", [(5, 4096), (3, 8192), (2, 16384), (470, 4096)])
+def test_gae_skip_one_block_per_row(oracle, W, B, N, T, p_skip, p_flag):
+    """Rows of whole 2048-step tiles walked by one thread block each, both carries (filled value and
+    advantage) in registers -- forced here for few rows; the library's own choice from about three rows
+    per SM, which 470 x 4096 reaches: against the oracle and against the carry through tile records,
+    with and without truncation tensors."""
+    import torch
+    ro, skip = _skip_case(W, N, T, p_skip, p_flag, salt=3)
+    p = ro.params
+    dev = Dev(ro)
+    sk = guarded_upload(skip)
+    ws = B.Workspace(N, T)
+
+    def call(use_tr=True):
+        tr, bv = (dev.truncs, dev.trunc_bootstrap) if use_tr else (None, None)
+        out = B.rlcs_gae_skip(dev.rewards, dev.values, dev.dones, tr, bv, dev.bootstrap, skip=sk, gamma=p["gamma"],
+                              lam=p["lam"], workspace=ws)
+        torch.cuda.synchronize()
+        assert ws.device_status() == 0
+        return [o.cpu().numpy() for o in out]
+
+    B.rlcs_debug_set_row_blocks(0)
+    try:
+        records = call()
+        B.rlcs_debug_set_row_blocks(1)
+        rows = call()
+        rows_plain = call(use_tr=False)
+    finally:
+        B.rlcs_debug_set_row_blocks(-1)
+    ra, rr, rf = oracle.gae_skip(ro.rewards, ro.values, ro.dones, ro.truncs, ro.trunc_bootstrap, ro.bootstrap, skip=skip,
+                                 gamma=p["gamma"], lam=p["lam"])
+    assert np.array_equal(rows[2].astype(np.float64), rf)
+    assert_close("skip adv, rows", rows[0], ra)
+    assert_close("skip ret, rows", rows[1], rr)
+    pa, pr, pf = oracle.gae_skip(ro.rewards, ro.values, ro.dones, None, None, ro.bootstrap, skip=skip, gamma=p["gamma"],
+                                 lam=p["lam"])
+    assert np.array_equal(rows_plain[2].astype(np.float64), pf)
+    assert_close("skip adv, rows, no truncation tensors", rows_plain[0], pa)
+    assert_close("skip ret, rows, no truncation tensors", rows_plain[1], pr)
+    for x, y in zip(rows, records):
+        np.testing.assert_allclose(x, y, rtol=1e-5, atol=1e-5)
+    if N >= 470:
+        for x, y in zip(rows, call()):                                       # the default for this shape
+            assert np.array_equal(x, y)
+
+
 def test_gae_skip_options_alignment_and_large_problem(oracle, W, B):
     import torch
     # no truncation tensors, no bootstrap, no returns; pointers off 16-byte alignment
