@@ -159,14 +159,21 @@ int rlcs_gae_normalized(const float* rewards, const float* values, const uint8_t
     p.stats = mean_rstd + 64;
     p.gamma = gamma; p.decay = gamma * lambda;
     const int variant = choose_variant(rlcs::kGaeStats, truncs != nullptr, total, T);
-    // (the statistics flavour keeps fixed tiles: its per-tile sums are laid out for them, and it has no
-    // one-block-per-row instantiation)
-    st = finish_params(p, variant, total, T, carry_bytes ? workspace : nullptr, carry_bytes, vec, true, 1, false, false);
+    // (the statistics flavour keeps fixed tiles: its per-tile sums are laid out for them; rows of whole
+    // tiles, about three per SM or more, take one thread block per row like plain GAE)
+    // (not when the rows are a little more than the thread blocks the GPU holds at once: the few blocks
+    // of the second wave then finish the call alone, one per SM -- 1024 x 32768: 0.75 against 0.80 with
+    // the carry between blocks)
+    const int64_t slots = (int64_t)rlcs_device::limits().sms * rlcs::kVariants[variant].min_blocks;
+    const bool thin_second_wave = N > slots && N * 5 < slots * 6;
+    const bool rows_ok = T % tile_elems(variant) == 0 && !thin_second_wave;
+    st = finish_params(p, variant, total, T, carry_bytes ? workspace : nullptr, carry_bytes, vec, true, 1, false, rows_ok);
     if (st != RLCS_OK) return st;
     st = run(rlcs::launch_gae_stats, p, variant, truncs != nullptr, vec, cuda_stream);
     if (st != RLCS_OK) return st;
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
-    if (rlcs::launch_norm_finalize(p.stats, p.num_tiles, total, (int)p.tile_steps, ddof, eps, mean_rstd, s) != cudaSuccess) return RLCS_ERR_CUDA;
+    const long long stat_tiles = p.row_blocks ? (total / T) * (T / tile_elems(variant)) : p.num_tiles;   // one pair of sums per tile
+    if (rlcs::launch_norm_finalize(p.stats, stat_tiles, total, (int)p.tile_steps, ddof, eps, mean_rstd, s) != cudaSuccess) return RLCS_ERR_CUDA;
     if (rlcs::launch_norm_rescale(advantages, total, mean_rstd, vec, s) != cudaSuccess) return RLCS_ERR_CUDA;
     return RLCS_OK;
 }

@@ -141,8 +141,11 @@ cudaError_t launch_rows(const ScanParams& p, cudaStream_t stream) {
                        stream, 0, p);
 }
 
-// algorithms that have the one-block-per-row kernel (the seven of the paper and the bare affine scan)
-__host__ __device__ constexpr bool has_row_blocks(int algo) { return algo <= kAffineFwd; }
+// algorithms that have the one-block-per-row kernel (the seven of the paper, the bare affine scan, and
+// GAE with per-tile statistics -- for rows of whole tiles, which the host checks)
+__host__ __device__ constexpr bool has_row_blocks(int algo) { return algo <= kAffineFwd || algo == kGaeStats; }
+// algorithms that have the row-aligned tiling instantiation of the one-tile kernel
+__host__ __device__ constexpr bool has_row_tiles(int algo) { return algo <= kAffineFwd; }
 
 template <int ALGO, bool TRUNC, bool VEC, int V>
 cudaError_t launch_variant(const ScanParams& p, cudaStream_t stream) {
@@ -159,7 +162,7 @@ cudaError_t launch_variant(const ScanParams& p, cudaStream_t stream) {
         return launch_scan(scan_kernel<ALGO, TRUNC, true, tv.threads, tv.items, tv.min_blocks>, (unsigned)p.num_tiles, tv.threads,
                            0, stream, 0, p);
     } else {
-        if constexpr (has_row_blocks(ALGO)) {
+        if constexpr (has_row_tiles(ALGO)) {
             // row-aligned tiling has an instantiation of its own (idle tail threads, tile length at run time)
             if (p.tile_steps != (unsigned)(tv.threads * tv.items))
                 return launch_scan(scan_kernel<ALGO, TRUNC, VEC, tv.threads, tv.items, tv.min_blocks, true>, (unsigned)p.num_tiles,

@@ -1392,7 +1392,7 @@ __global__ void __launch_bounds__(THREADS, MIN_BLOCKS) scan_kernel_cluster(const
 // chunk aligned for 256-bit accesses).  Vector accesses only.
 template <int ALGO, bool TRUNC, int THREADS, int ITEMS, bool IDLE>
 __device__ __forceinline__ void row_tile(const ScanParams& p, long long tile_start, long long row_end, float& carry,
-                                         ScanSmem<THREADS / 32>& sm, int buf) {
+                                         ScanSmem<THREADS / 32>& sm, int buf, long long s) {
     const int tid = threadIdx.x;
     const int lane = tid & 31;
     Chunk<ALGO, TRUNC, ITEMS> c;
@@ -1403,7 +1403,8 @@ __device__ __forceinline__ void row_tile(const ScanParams& p, long long tile_sta
     load_values_global<ALGO, TRUNC, ITEMS, true, true, IDLE>(c, v, p, i0, lane);
     issue_boot(c, p, n0);
     issue_trunc_values<ALGO, TRUNC, ITEMS, true>(c, p, i0);
-    tile_compute<ALGO, TRUNC, true, THREADS, ITEMS, true, false, NoHook, false, IDLE>(c, v, p, i0, 0, 0u, sm, buf, NoHook{}, nullptr,
+    // (s only numbers the tile for the per-tile statistics of kGaeStats)
+    tile_compute<ALGO, TRUNC, true, THREADS, ITEMS, true, false, NoHook, false, IDLE>(c, v, p, i0, s, 0u, sm, buf, NoHook{}, nullptr,
                                                                                      &carry);
 }
 
@@ -1422,8 +1423,9 @@ __global__ void __launch_bounds__(THREADS, MIN_BLOCKS) scan_kernel_rows(const Sc
         const unsigned m = FWD ? k : tiles - 1 - k;           // k-th tile in scan order
         const long long tile_start = row_start + (long long)m * TILE;
         // shared scratch alternates by tile parity, so one barrier per tile suffices (as in the persistent kernel)
-        if (tile_start + TILE <= row_end) row_tile<ALGO, TRUNC, THREADS, ITEMS, false>(p, tile_start, row_end, carry, sm, k & 1);
-        else row_tile<ALGO, TRUNC, THREADS, ITEMS, true>(p, tile_start, row_end, carry, sm, k & 1);
+        const long long s = (long long)blockIdx.x * tiles + k;
+        if (tile_start + TILE <= row_end) row_tile<ALGO, TRUNC, THREADS, ITEMS, false>(p, tile_start, row_end, carry, sm, k & 1, s);
+        else row_tile<ALGO, TRUNC, THREADS, ITEMS, true>(p, tile_start, row_end, carry, sm, k & 1, s);
     }
 }
 

@@ -521,6 +521,34 @@ def test_gae_normalized_back_to_back_calls_share_nothing_stale(oracle, W, B):
         assert_close(f"normalised advantages, rewards * {a} + {b}", got.cpu().numpy(), ref_adv)
 
 
+@pytest.mark.parametrize("N,T", [(5, 4096), (3, 8192), (2, 32768), (470, 4096)])
+def test_gae_normalized_one_block_per_row(oracle, W, B, N, T):
+    """Rows of whole tiles walked by one thread block each (forced for few rows; the library's own
+    choice at 470 x 4096): the per-tile sums are numbered row by row, the reduction sees every one of
+    them once.  Against the oracle and against the carry between blocks."""
+    ro = W.make_rollout(117, N, T, p_done=0.002, p_trunc=0.002, salt=T)
+    dev = Dev(ro)
+    p = ro.params
+    ws = B.Workspace(N, T, nbytes=B.lib().rlcs_gae_normalized_workspace_bytes(N, T))
+    call = lambda: [o.cpu().numpy() for o in B.rlcs_gae_normalized(dev.rewards, dev.values, dev.dones, dev.truncs,
+                                                                   dev.trunc_bootstrap, dev.bootstrap, gamma=p["gamma"],
+                                                                   lam=p["lam"], eps=1e-8, ddof=1, workspace=ws)]
+    B.rlcs_debug_set_row_blocks(0)
+    try:
+        other = call()
+        B.rlcs_debug_set_row_blocks(1)
+        rows = call()
+    finally:
+        B.rlcs_debug_set_row_blocks(-1)
+    ref_adv, ref_ret = oracle.gae_normalized(ro.rewards, ro.values, ro.dones, ro.truncs, ro.trunc_bootstrap, ro.bootstrap,
+                                             gamma=p["gamma"], lam=p["lam"], eps=1e-8, ddof=1)
+    assert_close("normalised advantages, rows", rows[0], ref_adv)
+    assert_close("returns, rows", rows[1], ref_ret)
+    np.testing.assert_allclose(rows[0], other[0], rtol=2e-5, atol=2e-5)
+    if N >= 470:
+        assert np.array_equal(rows[0], call()[0])                            # the default for this shape
+
+
 def test_gae_normalized_with_a_mean_far_from_zero(oracle, W, B):
     """Rewards ~ N(100, 0.1^2), small values, lambda = 0.1, no flags: every advantage is close to
     100 with a spread of about 0.1, so |mean| is a thousand times the standard deviation -- the case
