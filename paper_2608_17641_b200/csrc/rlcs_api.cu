@@ -118,10 +118,10 @@ int rlcs_gae_skip(const float* rewards, const float* values, const uint8_t* done
     // the copy bandwidth: records through the workspace 0.68 / 0.62; rows with 128 x 16 tiles at 5 / 6 / 8
     // blocks per SM 0.84 / 0.70, 0.80 / 0.63, 0.58 / 0.55; 256 x 8 0.89 / 0.81; 128 x 8 at 8 blocks 0.90 / 0.85.
     constexpr int kRowsVariant = 6;
-    if (rlcs_hooks::g_variant < 0 && T > 2048 && T % tile_elems(kRowsVariant) == 0 && row_blocks_ok(kRowsVariant, total, T, vec))
+    if (rlcs_hooks::g_variant < 0 && T > 2048 && T % tile_elems(kRowsVariant) == 0 && row_blocks_ok(kRowsVariant, total, T, vec, true))
         variant = kRowsVariant;
     const bool rows_ok = T % tile_elems(variant) == 0;
-    st = finish_params(p, variant, total, T, workspace, workspace_bytes, vec, false, 2, false, rows_ok);
+    st = finish_params(p, variant, total, T, workspace, workspace_bytes, vec, false, 2, false, rows_ok ? 2 : 0);
     if (st != RLCS_OK) return st;
     return run(rlcs::launch_gae_skip, p, variant, truncs != nullptr, vec, cuda_stream);
 }
@@ -161,13 +161,10 @@ int rlcs_gae_normalized(const float* rewards, const float* values, const uint8_t
     const int variant = choose_variant(rlcs::kGaeStats, truncs != nullptr, total, T);
     // (the statistics flavour keeps fixed tiles: its per-tile sums are laid out for them; rows of whole
     // tiles, about three per SM or more, take one thread block per row like plain GAE)
-    // (not when the rows are a little more than the thread blocks the GPU holds at once: the few blocks
-    // of the second wave then finish the call alone, one per SM -- 1024 x 32768: 0.75 against 0.80 with
-    // the carry between blocks)
-    const int64_t slots = (int64_t)rlcs_device::limits().sms * rlcs::kVariants[variant].min_blocks;
-    const bool thin_second_wave = N > slots && N * 5 < slots * 6;
-    const bool rows_ok = T % tile_elems(variant) == 0 && !thin_second_wave;
-    st = finish_params(p, variant, total, T, carry_bytes ? workspace : nullptr, carry_bytes, vec, true, 1, false, rows_ok);
+    // (1024 x 32768, a thin second wave of blocks: 0.75 with one block per row against 0.80 with the carry
+    // between blocks -- plan_carry's rule keeps such shapes off the row kernel)
+    const bool rows_ok = T % tile_elems(variant) == 0;
+    st = finish_params(p, variant, total, T, carry_bytes ? workspace : nullptr, carry_bytes, vec, true, 1, false, rows_ok ? 1 : 0);
     if (st != RLCS_OK) return st;
     st = run(rlcs::launch_gae_stats, p, variant, truncs != nullptr, vec, cuda_stream);
     if (st != RLCS_OK) return st;
@@ -252,7 +249,7 @@ int rlcs_retrace_probs(const float* rewards, const float* q_values, const float*
     // (the test hook forces it for any A).
     const bool rows_ok = T % (rlcs::kRetraceProbsThreads * rlcs::kRetraceProbsItems) == 0 &&
                          (rlcs_hooks::g_row_blocks > 0 || (vec_rows && (A == 4 || A == 8)));
-    st = finish_params(p, kVariant, total, T, workspace, workspace_bytes, vec, false, 1, false, rows_ok);
+    st = finish_params(p, kVariant, total, T, workspace, workspace_bytes, vec, false, 1, false, rows_ok ? 2 : 0);
     if (st != RLCS_OK) return st;
     return rlcs::launch_retrace_probs(p, truncs != nullptr, vec, vec_rows, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess
                ? RLCS_OK : RLCS_ERR_CUDA;

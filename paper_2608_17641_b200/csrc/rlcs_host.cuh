@@ -120,6 +120,15 @@ bool row_fits(int variant, int64_t T) {
     return T * 10 >= tiles * tile * 7;
 }
 
+// Rows a little more numerous than the thread blocks the GPU holds at once (up to 1.2 times): with one
+// block per row the few blocks of the second wave finish the call alone, one per SM (measured, GAE
+// 900 x 16384: 0.72 of the copy bandwidth against 0.78 with the cluster carry; 1024 x 32768: 0.78 either
+// way; 1200 x 16384: 0.82 against 0.81).
+bool thin_second_wave(int variant, int64_t rows) {
+    const int64_t slots = (int64_t)rlcs_device::limits().sms * RLCS_NS::kVariants[variant].min_blocks;
+    return rows > slots && rows * 5 < slots * 6;
+}
+
 int choose_variant(int algo, bool trunc, int64_t total, int64_t T) {
     if (g_variant >= 0 && RLCS_NS::variant_built_for(algo, g_variant)) return g_variant;
     int v = choose_variant_unchecked(algo, trunc, total, T);
@@ -130,7 +139,7 @@ int choose_variant(int algo, bool trunc, int64_t total, int64_t T) {
         total / T >= 3 * rlcs_device::limits().sms && !row_fits(v, T)) {
         const int alternatives[2] = {0, 6};          // 256 x 8 (2048 steps), 128 x 8 (1024 steps)
         for (int alt : alternatives)
-            if (RLCS_NS::variant_built_for(algo, alt) && row_fits(alt, T)) { v = alt; break; }
+            if (RLCS_NS::variant_built_for(algo, alt) && row_fits(alt, T) && !thin_second_wave(alt, total / T)) { v = alt; break; }
     }
     if (RLCS_NS::variant_built_for(algo, v)) return v;
     // not compiled for this algorithm / element type: the nearest shape that every build has
@@ -165,22 +174,25 @@ int row_aligned_steps(int variant, int64_t T) {
 // chunk whole and aligned), vector access, the row's tiles at least 70 % used, and at least three
 // rows per SM (with fewer rows too many SMs idle: those go to the cluster carry or the look-back;
 // measured cross-over at T = 16384: 384 rows 0.70 against 0.73, 512 rows 0.84 against 0.70).
-bool row_blocks_ok(int variant, int64_t total, int64_t T, bool vec) {
+bool row_blocks_ok(int variant, int64_t total, int64_t T, bool vec, bool any_wave = false) {
     const RLCS_NS::TileVariant tv = RLCS_NS::kVariants[variant];
     const int tile = tv.threads * tv.items;
     if (rlcs_hooks::g_row_blocks == 0 || !vec || tv.stages != 0 || T <= tile || T % tv.items != 0) return false;
     const int64_t tiles = (T + tile - 1) / tile;
     if (T * 10 < tiles * tile * 7) return false;
     if (rlcs_hooks::g_row_blocks > 0) return true;
+    if (!any_wave && thin_second_wave(variant, total / T)) return false;
     return total / T >= 3 * rlcs_device::limits().sms;        // measured cross-over against the cluster carry: about 3 rows per SM
 }
 
+// allow_row_blocks: 0 = never, 1 = where row_blocks_ok() says so, 2 = the same without its rule about a thin
+// second wave (for kernels whose carry between blocks costs more than such a wave does).
 CarryPlan plan_carry(int variant, int64_t total, int64_t T, bool vec, bool allow_cluster, int records_per_tile,
-                     bool allow_row_tiles = true, bool allow_row_blocks = true) {
+                     bool allow_row_tiles = true, int allow_row_blocks = 1) {
     const int tile = tile_elems(variant);
     const int64_t num_tiles = (total + tile - 1) / tile;
     CarryPlan plan = {(tile % T) != 0 ? 1 : 0, 0, 0, tile, 0};    // T does not divide the tile: rows straddle tiles
-    if (allow_row_blocks && row_blocks_ok(variant, total, T, vec)) {
+    if (allow_row_blocks && row_blocks_ok(variant, total, T, vec, allow_row_blocks == 2)) {
         plan.carry_mode = 0;
         plan.row_blocks = 1;
         return plan;
@@ -210,7 +222,7 @@ CarryPlan plan_carry(int variant, int64_t total, int64_t T, bool vec, bool allow
 // the statistics flavour of GAE, the observation-skip scans) pass allow_row_tiles = allow_row_blocks =
 // false; Retrace from [N,T,A] tensors has its own one-block-per-row kernel for rows of whole tiles.
 int finish_params(ScanParams& p, int variant, int64_t total, int64_t T, void* workspace, size_t workspace_bytes, bool vec,
-                  bool allow_cluster = true, int records_per_tile = 1, bool allow_row_tiles = true, bool allow_row_blocks = true) {
+                  bool allow_cluster = true, int records_per_tile = 1, bool allow_row_tiles = true, int allow_row_blocks = 1) {
     const int tile = tile_elems(variant);
     const CarryPlan plan = plan_carry(variant, total, T, vec, allow_cluster, records_per_tile, allow_row_tiles, allow_row_blocks);
     p.total = total;

@@ -70,6 +70,26 @@ def test_row_aligned_tiling_needs_no_carry_workspace(L):
         L.rlcs_debug_allow_row_tiles(1)
 
 
+def test_one_block_per_row_needs_no_carry_workspace_except_for_a_thin_second_wave(L):
+    """Long rows of whole tiles, enough of them: one thread block per row, no carry workspace -- unless the
+    rows are a little more than the blocks the GPU holds at once (148 SMs x 6 blocks here: 888), where the
+    few blocks of the second wave would finish the call alone and the carry between blocks is kept."""
+    T = 32768                                                       # 16 tiles of 2048: too long for a cluster per row
+    assert L.rlcs_gae_carry_bytes(800, T, 1, 1) == 0
+    assert L.rlcs_gae_carry_bytes(888, T, 1, 1) == 0
+    assert L.rlcs_gae_carry_bytes(900, T, 1, 1) > 0
+    assert L.rlcs_gae_carry_bytes(1060, T, 1, 1) > 0
+    assert L.rlcs_gae_carry_bytes(1100, T, 1, 1) == 0
+    assert L.rlcs_gae_carry_bytes(300, T, 1, 1) > 0                 # fewer than three rows per SM
+    try:
+        assert L.rlcs_debug_set_row_blocks(1) == OK                 # forced: any number of rows
+        assert L.rlcs_gae_carry_bytes(900, T, 1, 1) == 0 and L.rlcs_gae_carry_bytes(3, T, 1, 1) == 0
+        assert L.rlcs_debug_set_row_blocks(0) == OK                 # never
+        assert L.rlcs_gae_carry_bytes(800, T, 1, 1) > 0
+    finally:
+        L.rlcs_debug_set_row_blocks(-1)
+
+
 def test_status_strings(L):
     assert L.rlcs_status_string(0) == b"RLCS_OK"
     for s in range(1, 8):

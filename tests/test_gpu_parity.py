@@ -188,7 +188,8 @@ def test_one_block_per_row_is_the_default_with_many_rows(oracle, W, B):
         pytest.skip("about the library's own choice of tile shape")
     N, T = 1200, 2064                                     # 2048 + one chunk of 16: no tile shape is filled to 70 % by such rows
     assert B.lib().rlcs_gae_carry_bytes(N, T, 1, 1) > 0   # ... so these rows are carried between blocks
-    assert B.lib().rlcs_gae_carry_bytes(1200, 4112, 1, 1) == 0      # 4112 = 5 tiles of 1024 at 80 %: the 1024-step shape is taken
+    assert B.lib().rlcs_gae_carry_bytes(1500, 4112, 1, 1) == 0      # 4112 = 5 tiles of 1024 at 80 %: the 1024-step shape is taken
+    assert B.lib().rlcs_gae_carry_bytes(1200, 4112, 1, 1) > 0       # ... but not for a thin second wave (1184 blocks fit at once)
     N, T = 1200, 6000
     ro = W.make_rollout(95, N, T, p_done=0.0005, p_trunc=0.0005)
     assert B.lib().rlcs_gae_carry_bytes(N, T, 1, 1) == 0
