@@ -1069,6 +1069,13 @@ def main():
         del batch
         torch.cuda.empty_cache()
         k30, k20 = max(3, min(args.steps, 30)), max(3, min(args.steps, 20))
+        # the same number of steps as the bench batch in long rows (token-level trajectories): the two
+        # GAE extensions on rows of 8192 steps
+        long_rows = GpuBatch(workloads.config5(N=WORKLOAD["N"] // 4, T=WORKLOAD["T"] * 4, salt=rank), torch.device("cuda", local))
+        ext("gae_skip_long_rows", {"N": long_rows.ro.N, "T": long_rows.ro.T, **time_gae_skip(long_rows, k20, peak)})
+        ext("gae_normalized_long_rows", {"N": long_rows.ro.N, "T": long_rows.ro.T, **time_gae_normalized(long_rows, k20, peak)})
+        del long_rows
+        torch.cuda.empty_cache()
         ext("retrace_probs", time_retrace_probs(torch, binding, k30, peak))
         ext("elig_trace_vec", [time_elig_trace_vec(torch, binding, k30, peak, *shape)
                                for shape in ((4096, 512, 64), (1024, 1024, 64), (64, 16384, 64), (16, 65536, 64))])
